@@ -1,0 +1,376 @@
+/*
+ * TEST INFRASTRUCTURE -- NOT PART OF THE PRODUCT PATH.
+ *
+ * Plain fp64 CPU oracle for alpha-entmax / ASEntmax attention, written from the paper's
+ * definitions.  Only the tests, the smoke check and the CPU-baseline leg of the benchmark may
+ * call it.  It shares no code, header, table or constant with the CUDA library.
+ *
+ * What each function follows:
+ *   oracle_entmax_row          Eq. 1 (alpha-entmax map) and App. A ("alpha-entmax computation"):
+ *                              order-based exact threshold for alpha = 2 (sparsemax) and
+ *                              alpha = 1.5, bisection inside the bracket of Eq. "bounds_entmax"
+ *                              for any other alpha.
+ *   oracle_asentmax_scale      Eq. "asentmax": c = delta + beta * (log n)^gamma.
+ *   oracle_attn_fwd_rows       Sec. 2.1: z_ij = <q_i,k_j>/sqrt(d), causal j <= i, output
+ *                              sum_j p_ij v_j, with the ASEntmax scale applied to the logits.
+ *   oracle_attn_bwd_head       Jacobian of Eq. 1 by implicit differentiation:
+ *                              dp_j/ds_k = u_j (delta_jk - u_k / sum u), u = p^(2-alpha).
+ *
+ * Pins (tests that do not use this file's own arithmetic): the paper's worked sparsemax example,
+ * the two-level closed form of Lemma 2, brute-force enumeration of supports for n <= 8, the
+ * finite-n scalar equation of the representational-collapse construction, the softmax limit,
+ * the Tsallis variational objective, shift/append invariances and central finite differences
+ * for the backward pass.  Parity unpinned: none of the row-level functions; the support sizes on
+ * the large synthetic workloads have no value printed in the paper to compare against.
+ *
+ * Conventions: tau is Eq. 1's threshold, i.e. p_j = max((alpha-1) s_j - tau, 0)^(1/(alpha-1)).
+ * A logit with (alpha-1) s_j <= tau gets exactly 0 and is outside the support.
+ */
+#include <math.h>
+#include <stdint.h>
+#include <stdlib.h>
+#include <string.h>
+#ifdef _OPENMP
+#include <omp.h>
+#endif
+
+#define ORACLE_METHOD_AUTO 0
+#define ORACLE_METHOD_BISECT 1
+#define ORACLE_METHOD_SORT 2
+
+static int cmp_desc(const void* a, const void* b) {
+  double x = *(const double*)a, y = *(const double*)b;
+  return (x < y) - (x > y);
+}
+
+/* y^e for y > 0, with the three exponents that are integers done by multiplication. */
+static double pow_pos(double y, double e) {
+  if (e == 1.0) return y;
+  if (e == 2.0) return y * y;
+  if (e == 4.0) { double t = y * y; return t * t; }
+  return exp(e * log(y));
+}
+
+/* sum_j max(x_j - tau, 0)^e  (x already multiplied by alpha-1) */
+static double mass(const double* x, int n, double tau, double e) {
+  double acc = 0.0;
+  for (int j = 0; j < n; ++j) {
+    double y = x[j] - tau;
+    if (y > 0.0) acc += pow_pos(y, e);
+  }
+  return acc;
+}
+
+/* App. A: bisection on f(tau) = sum_j [x_j - tau]_+^(1/(alpha-1)) - 1 over the bracket
+ * [x_max - 1, x_max - n^(1-alpha)] (the paper's bracket, un-normalised: p_max lies in [1/n, 1]). */
+static double tau_bisect(const double* x, int n, double alpha) {
+  double e = 1.0 / (alpha - 1.0);
+  double xmax = x[0];
+  for (int j = 1; j < n; ++j) if (x[j] > xmax) xmax = x[j];
+  double lo = xmax - 1.0;
+  double hi = xmax - pow((double)n, 1.0 - alpha);
+  for (int it = 0; it < 200 && (hi - lo) > 1e-12; ++it) {
+    double mid = 0.5 * (lo + hi);
+    if (mass(x, n, mid, e) >= 1.0) lo = mid; else hi = mid;
+  }
+  return 0.5 * (lo + hi);
+}
+
+/* alpha = 2 (sparsemax): sort descending, k* = max{k : 1 + k x_(k) > sum_{l<=k} x_(l)},
+ * tau = (sum_{l<=k*} x_(l) - 1) / k*.  x = (alpha-1) z = z. */
+static double tau_sort_sparsemax(const double* x, int n, double* scratch) {
+  memcpy(scratch, x, sizeof(double) * (size_t)n);
+  qsort(scratch, (size_t)n, sizeof(double), cmp_desc);
+  double top = scratch[0];
+  double csum = 0.0, tau = 0.0;
+  for (int k = 1; k <= n; ++k) {
+    double xk = scratch[k - 1] - top; /* shifted so that the largest is 0: keeps sums small */
+    csum += xk;
+    if (1.0 + k * xk > csum) tau = (csum - 1.0) / k; else break;
+  }
+  return tau + top;
+}
+
+/* alpha = 1.5: p_j = (x_j - tau)^2 with x = z/2.  For the k largest, sum (x_(l) - tau)^2 = 1 has
+ * the smaller root tau_k = mean_k - sqrt((1 - ss_k)/k), ss_k = sum (x_(l) - mean_k)^2.  The
+ * support size is the largest k with tau_k <= x_(k). */
+static double tau_sort_15(const double* x, int n, double* scratch) {
+  memcpy(scratch, x, sizeof(double) * (size_t)n);
+  qsort(scratch, (size_t)n, sizeof(double), cmp_desc);
+  double top = scratch[0];
+  double s1 = 0.0, s2 = 0.0, tau = -1.0;
+  for (int k = 1; k <= n; ++k) {
+    double xk = scratch[k - 1] - top;
+    s1 += xk;
+    s2 += xk * xk;
+    double mean = s1 / k;
+    double ss = s2 - k * mean * mean;
+    double rad = (1.0 - ss) / k;
+    if (rad < 0.0) rad = 0.0;
+    double tk = mean - sqrt(rad);
+    if (tk <= xk) tau = tk; else break;
+  }
+  return tau + top;
+}
+
+/* Eq. 1 on one row of logits z (any real values).  Returns the support size.
+ * p may be NULL.  method: ORACLE_METHOD_*. */
+int oracle_entmax_row(const double* z, int n, double alpha, int method, double* p, double* tau_out) {
+  if (n <= 0 || !(alpha > 1.0)) return -1;
+  double* x = (double*)malloc(sizeof(double) * (size_t)n * 2);
+  if (!x) return -2;
+  double* scratch = x + n;
+  double am1 = alpha - 1.0;
+  for (int j = 0; j < n; ++j) x[j] = am1 * z[j];
+  double tau;
+  int use_sort = (method == ORACLE_METHOD_SORT) ||
+                 (method == ORACLE_METHOD_AUTO && (alpha == 2.0 || alpha == 1.5));
+  if (use_sort && alpha == 2.0) tau = tau_sort_sparsemax(x, n, scratch);
+  else if (use_sort && alpha == 1.5) tau = tau_sort_15(x, n, scratch);
+  else tau = tau_bisect(x, n, alpha);
+  double e = 1.0 / am1;
+  int support = 0;
+  for (int j = 0; j < n; ++j) {
+    double y = x[j] - tau;
+    double pj = 0.0;
+    if (y > 0.0) { pj = pow_pos(y, e); ++support; }
+    if (p) p[j] = pj;
+  }
+  if (tau_out) *tau_out = tau;
+  free(x);
+  return support;
+}
+
+/* Eq. "asentmax": c = delta + beta (log n)^gamma, natural log.  A single visible key (n = 1)
+ * has log n = 0, where 0^gamma is undefined for gamma <= 0: the row is one-hot whatever the scale
+ * is, and the reading taken is c = delta. */
+double oracle_asentmax_scale(double beta, double gamma, double delta, long n) {
+  if (n <= 1) return delta;
+  return delta + beta * pow(log((double)n), gamma);
+}
+
+static long visible_keys(long i, long N, int causal) { return causal ? i + 1 : N; }
+
+/* Forward for selected query rows of ONE head.
+ *   q,k,v        [N,d] row-major, float (bf16- or fp32-rounded values, converted exactly)
+ *   use_scale    0: c_i = 1 (fixed temperature); 1: c_i from beta,gamma,delta
+ *   n_mode       0: n_i = number of visible keys of row i; 1: n_i = N
+ *   rows         nrows query indices
+ *   tau_out      [nrows]; o_out [nrows,d]; p_out NULL or [nrows,N] (zeros where masked)
+ *   supp_out     NULL or [nrows] support sizes
+ */
+int oracle_attn_fwd_rows(const float* q, const float* k, const float* v, long N, int d,
+                         double alpha, double sm_scale, int causal, int n_mode, int use_scale,
+                         double beta, double gamma, double delta,
+                         const int64_t* rows, long nrows,
+                         double* tau_out, double* o_out, double* p_out, int64_t* supp_out) {
+  if (N <= 0 || d <= 0 || !(alpha > 1.0)) return -1;
+  int err = 0;
+#pragma omp parallel
+  {
+    double* s = (double*)malloc(sizeof(double) * (size_t)N);
+    double* p = (double*)malloc(sizeof(double) * (size_t)N);
+    if (!s || !p) {
+#pragma omp atomic write
+      err = -2;
+    } else {
+#pragma omp for schedule(dynamic, 4)
+      for (long r = 0; r < nrows; ++r) {
+        long i = rows[r];
+        long nv = visible_keys(i, N, causal);
+        long n_i = n_mode ? N : nv;
+        double c = use_scale ? oracle_asentmax_scale(beta, gamma, delta, n_i) : 1.0;
+        const float* qi = q + (size_t)i * d;
+        for (long j = 0; j < nv; ++j) {
+          const float* kj = k + (size_t)j * d;
+          double dot = 0.0;
+          for (int t = 0; t < d; ++t) dot += (double)qi[t] * (double)kj[t];
+          s[j] = c * (dot * sm_scale);
+        }
+        double tau;
+        int supp = oracle_entmax_row(s, (int)nv, alpha, ORACLE_METHOD_AUTO, p, &tau);
+        tau_out[r] = tau;
+        if (supp_out) supp_out[r] = supp;
+        double* o = o_out + (size_t)r * d;
+        for (int t = 0; t < d; ++t) o[t] = 0.0;
+        for (long j = 0; j < nv; ++j) {
+          if (p[j] > 0.0) {
+            const float* vj = v + (size_t)j * d;
+            for (int t = 0; t < d; ++t) o[t] += p[j] * (double)vj[t];
+          }
+        }
+        if (p_out) {
+          double* pr = p_out + (size_t)r * N;
+          for (long j = 0; j < nv; ++j) pr[j] = p[j];
+          for (long j = nv; j < N; ++j) pr[j] = 0.0;
+        }
+      }
+    }
+    free(s);
+    free(p);
+  }
+  return err;
+}
+
+/* Backward for ONE head, all query rows (dK and dV need every row).
+ *   d_o [N,d] float; outputs dq,dk,dv [N,d] double (overwritten).
+ * dP_ij = <dO_i, v_j>; u_ij = p_ij^(2-alpha) on the support, 0 off it (alpha = 2: u = 1 there);
+ * dS_ij = u_ij (dP_ij - sum_l u_il dP_il / sum_l u_il);
+ * dQ_i = g_i sum_j dS_ij k_j, dK_j = sum_i g_i dS_ij q_i with g_i = c_i * sm_scale;
+ * dV_j = sum_i p_ij dO_i. */
+int oracle_attn_bwd_head(const float* q, const float* k, const float* v, const float* d_o,
+                         long N, int d, double alpha, double sm_scale, int causal, int n_mode,
+                         int use_scale, double beta, double gamma, double delta,
+                         double* dq, double* dk, double* dv) {
+  if (N <= 0 || d <= 0 || !(alpha > 1.0)) return -1;
+  size_t nd = (size_t)N * d;
+  memset(dq, 0, sizeof(double) * nd);
+  memset(dk, 0, sizeof(double) * nd);
+  memset(dv, 0, sizeof(double) * nd);
+  int err = 0;
+#pragma omp parallel
+  {
+    double* s = (double*)malloc(sizeof(double) * (size_t)N);
+    double* p = (double*)malloc(sizeof(double) * (size_t)N);
+    double* dkl = (double*)calloc(nd, sizeof(double));
+    double* dvl = (double*)calloc(nd, sizeof(double));
+    if (!s || !p || !dkl || !dvl) {
+#pragma omp atomic write
+      err = -2;
+    } else {
+#pragma omp for schedule(dynamic, 4)
+      for (long i = 0; i < N; ++i) {
+        long nv = visible_keys(i, N, causal);
+        long n_i = n_mode ? N : nv;
+        double c = use_scale ? oracle_asentmax_scale(beta, gamma, delta, n_i) : 1.0;
+        double g = c * sm_scale;
+        const float* qi = q + (size_t)i * d;
+        const float* doi = d_o + (size_t)i * d;
+        for (long j = 0; j < nv; ++j) {
+          const float* kj = k + (size_t)j * d;
+          double dot = 0.0;
+          for (int t = 0; t < d; ++t) dot += (double)qi[t] * (double)kj[t];
+          s[j] = c * (dot * sm_scale);
+        }
+        double tau;
+        oracle_entmax_row(s, (int)nv, alpha, ORACLE_METHOD_AUTO, p, &tau);
+        /* first sweep: sum u and <u, dP>; dP kept in s[] (scores no longer needed) */
+        double su = 0.0, sud = 0.0;
+        for (long j = 0; j < nv; ++j) {
+          if (p[j] > 0.0) {
+            const float* vj = v + (size_t)j * d;
+            double dp = 0.0;
+            for (int t = 0; t < d; ++t) dp += (double)doi[t] * (double)vj[t];
+            double u = (alpha == 2.0) ? 1.0 : pow(p[j], 2.0 - alpha);
+            s[j] = dp;
+            su += u;
+            sud += u * dp;
+          }
+        }
+        double rho = sud / su;
+        double* dqi = dq + (size_t)i * d;
+        for (long j = 0; j < nv; ++j) {
+          if (p[j] > 0.0) {
+            double u = (alpha == 2.0) ? 1.0 : pow(p[j], 2.0 - alpha);
+            double ds = u * (s[j] - rho);
+            const float* kj = k + (size_t)j * d;
+            double* dkj = dkl + (size_t)j * d;
+            double* dvj = dvl + (size_t)j * d;
+            for (int t = 0; t < d; ++t) {
+              dqi[t] += g * ds * (double)kj[t];
+              dkj[t] += g * ds * (double)qi[t];
+              dvj[t] += p[j] * (double)doi[t];
+            }
+          }
+        }
+      }
+#pragma omp critical
+      {
+        for (size_t t = 0; t < nd; ++t) { dk[t] += dkl[t]; dv[t] += dvl[t]; }
+      }
+    }
+    free(s); free(p); free(dkl); free(dvl);
+  }
+  return err;
+}
+
+/* Row-local part of the backward pass (dQ_i and dS_i) for selected rows of one head.
+ * ds_out NULL or [nrows,N]. */
+int oracle_attn_bwd_rows(const float* q, const float* k, const float* v, const float* d_o,
+                         long N, int d, double alpha, double sm_scale, int causal, int n_mode,
+                         int use_scale, double beta, double gamma, double delta,
+                         const int64_t* rows, long nrows, double* dq_out, double* ds_out) {
+  if (N <= 0 || d <= 0 || !(alpha > 1.0)) return -1;
+  int err = 0;
+#pragma omp parallel
+  {
+    double* s = (double*)malloc(sizeof(double) * (size_t)N);
+    double* p = (double*)malloc(sizeof(double) * (size_t)N);
+    if (!s || !p) {
+#pragma omp atomic write
+      err = -2;
+    } else {
+#pragma omp for schedule(dynamic, 4)
+      for (long r = 0; r < nrows; ++r) {
+        long i = rows[r];
+        long nv = visible_keys(i, N, causal);
+        long n_i = n_mode ? N : nv;
+        double c = use_scale ? oracle_asentmax_scale(beta, gamma, delta, n_i) : 1.0;
+        double g = c * sm_scale;
+        const float* qi = q + (size_t)i * d;
+        const float* doi = d_o + (size_t)i * d;
+        for (long j = 0; j < nv; ++j) {
+          const float* kj = k + (size_t)j * d;
+          double dot = 0.0;
+          for (int t = 0; t < d; ++t) dot += (double)qi[t] * (double)kj[t];
+          s[j] = c * (dot * sm_scale);
+        }
+        double tau;
+        oracle_entmax_row(s, (int)nv, alpha, ORACLE_METHOD_AUTO, p, &tau);
+        double su = 0.0, sud = 0.0;
+        for (long j = 0; j < nv; ++j) {
+          if (p[j] > 0.0) {
+            const float* vj = v + (size_t)j * d;
+            double dp = 0.0;
+            for (int t = 0; t < d; ++t) dp += (double)doi[t] * (double)vj[t];
+            double u = (alpha == 2.0) ? 1.0 : pow(p[j], 2.0 - alpha);
+            s[j] = dp;
+            su += u;
+            sud += u * dp;
+          }
+        }
+        double rho = sud / su;
+        double* dqi = dq_out + (size_t)r * d;
+        for (int t = 0; t < d; ++t) dqi[t] = 0.0;
+        if (ds_out) for (long j = 0; j < N; ++j) ds_out[(size_t)r * N + j] = 0.0;
+        for (long j = 0; j < nv; ++j) {
+          if (p[j] > 0.0) {
+            double u = (alpha == 2.0) ? 1.0 : pow(p[j], 2.0 - alpha);
+            double ds = u * (s[j] - rho);
+            const float* kj = k + (size_t)j * d;
+            for (int t = 0; t < d; ++t) dqi[t] += g * ds * (double)kj[t];
+            if (ds_out) ds_out[(size_t)r * N + j] = ds;
+          }
+        }
+      }
+    }
+    free(s); free(p);
+  }
+  return err;
+}
+
+int oracle_num_threads(void) {
+#ifdef _OPENMP
+  return omp_get_max_threads();
+#else
+  return 1;
+#endif
+}
+
+void oracle_set_num_threads(int n) {
+#ifdef _OPENMP
+  if (n > 0) omp_set_num_threads(n);
+#else
+  (void)n;
+#endif
+}
