@@ -1,0 +1,146 @@
+/*
+ * entmax_attn.h -- C ABI of the fused alpha-entmax / ASEntmax attention library for NVIDIA B200
+ * (sm_100a).  Plain pointers and sizes only; no framework types.
+ *
+ * What the library computes (notation of the paper; row i = query, column j = key):
+ *
+ *   n_i   = number of keys row i attends to: i+1 under the causal mask j <= i (Sec. 2.1, the sum
+ *           over j <= i), N otherwise; with n_mode = 1, N for every row.
+ *   c_i   = delta_h + beta_h * (ln n_i)^gamma_h     ASEntmax scale of head h (Eq. "asentmax");
+ *           c_i = delta_h when n_i = 1; c_i = 1 when beta/gamma/delta are all NULL.
+ *   s_ij  = c_i * <q_i, k_j> * sm_scale             attention logits (Sec. 2.1, z_ij = <q_i,k_j>/sqrt(d))
+ *   tau_i : sum_j [(alpha-1) s_ij - tau_i]_+^(1/(alpha-1)) = 1          (Eq. 1, threshold)
+ *   p_ij  = [(alpha-1) s_ij - tau_i]_+^(1/(alpha-1))                    (Eq. 1); exactly 0 when
+ *           (alpha-1) s_ij <= tau_i (App. A)
+ *   O_i   = sum_j p_ij v_j                                              (Sec. 2.1)
+ *
+ * Backward (Jacobian of Eq. 1 by implicit differentiation):
+ *   dP_ij = <dO_i, v_j>,  u_ij = p_ij^(2-alpha) on the support and 0 off it,
+ *   dS_ij = u_ij * (dP_ij - sum_l u_il dP_il / sum_l u_il),
+ *   dQ_i = c_i sm_scale sum_j dS_ij k_j,  dK_j = sum_i c_i sm_scale dS_ij q_i,  dV_j = sum_i p_ij dO_i.
+ *
+ * General conventions
+ *   - Every tensor pointer is a DEVICE pointer owned by the caller.  The library allocates no device
+ *     memory, never synchronises the device or a stream, and enqueues all work on `cuda_stream`
+ *     (a cudaStream_t passed as void*; NULL = the legacy default stream).
+ *   - Q, K, V, O, dO, dQ, dK, dV share one layout: [batch, heads, seq, head_dim] with head_dim
+ *     innermost and contiguous; the other three strides come from the params struct (in elements).
+ *     tau is [batch, heads, seq] float32, contiguous.  beta, gamma, delta are [heads] float32.
+ *   - All tensor pointers must be 16-byte aligned and all strides multiples of 8 elements.
+ *   - Functions return ENTMAX_ATTN_OK (0) or a negative entmax_attn_status; on a negative return
+ *     nothing has been enqueued.  Device-side conditions are reported through `device_status`.
+ *   - Non-finite values in Q, K, V or dO give unspecified results (never a fault).
+ */
+#ifndef ENTMAX_ATTN_H_
+#define ENTMAX_ATTN_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+#define ENTMAX_ATTN_DTYPE_BF16 0 /* Q,K,V,dO in, O,dQ,dK,dV out: bfloat16; scores on tcgen05 tensor cores */
+#define ENTMAX_ATTN_DTYPE_FP32 1 /* everything float32; scores by fp32 FMA (meets the tighter fp32 tolerance) */
+
+typedef enum {
+  ENTMAX_ATTN_OK = 0,
+  ENTMAX_ATTN_EINVAL_SHAPE = -1,     /* batch/heads/seq < 1, head_dim not 64 or 128, bad strides, too many rows */
+  ENTMAX_ATTN_EINVAL_ALPHA = -2,     /* alpha not in (1, 2] or not finite; sm_scale not finite or negative     */
+  ENTMAX_ATTN_EINVAL_DTYPE = -3,     /* dtype is neither ENTMAX_ATTN_DTYPE_BF16 nor ENTMAX_ATTN_DTYPE_FP32      */
+  ENTMAX_ATTN_EINVAL_ALIGN = -4,     /* a tensor pointer is not 16-byte aligned                                 */
+  ENTMAX_ATTN_EINVAL_WORKSPACE = -5, /* workspace NULL, misaligned (256 B) or smaller than workspace_bytes()    */
+  ENTMAX_ATTN_EINVAL_NULL = -6,      /* a required pointer is NULL, or only some of beta/gamma/delta are given  */
+  ENTMAX_ATTN_ECUDA = -7,            /* a CUDA call failed; see entmax_attn_last_cuda_error()                   */
+  ENTMAX_ATTN_EUNSUPPORTED = -8      /* the device is not sm_100 (bf16 path needs tcgen05/TMA)                  */
+} entmax_attn_status;
+
+typedef struct {
+  int32_t batch, heads, seq, head_dim; /* head_dim in {64, 128}; seq >= 1, any value (tails are predicated)      */
+  int32_t dtype;                       /* ENTMAX_ATTN_DTYPE_*                                                    */
+  int32_t causal;                      /* 0 / 1; causal keeps j <= i, diagonal included                          */
+  int32_t n_mode;                      /* 0: n_i = keys visible to row i; 1: n_i = seq for every row             */
+  float alpha;                         /* 1 < alpha <= 2; 1.25, 1.5 and 2 use multiplication-only powers         */
+  float sm_scale;                      /* 0 means 1/sqrt(head_dim)                                               */
+  int64_t stride_b, stride_h, stride_n; /* elements; all 0 means contiguous [batch, heads, seq, head_dim]        */
+} entmax_attn_params;
+
+/* Words of the optional device status array (int32[ENTMAX_ATTN_STATUS_WORDS], device memory, written
+ * by the kernels of a call; zeroed at the start of that call). */
+#define ENTMAX_ATTN_STATUS_WORDS 4
+#define ENTMAX_ATTN_STATUS_FLAGS 0         /* bit field below; 0 = clean run                                   */
+#define ENTMAX_ATTN_STATUS_DENSE_ROWS 1    /* rows whose support did not fit the sparse list (dense fallback)  */
+#define ENTMAX_ATTN_FLAG_WAIT_EXPIRED 1    /* a bounded on-chip wait ran out; outputs of that call are invalid */
+#define ENTMAX_ATTN_FLAG_BAD_SCALE 2       /* some c_i was not finite                                          */
+
+/* Bytes of scratch the caller must pass to entmax_attn_fwd (is_bwd = 0) or entmax_attn_bwd
+ * (is_bwd = 1) for these params.  Returns 0 if the params are invalid.  No paper counterpart: the
+ * paper does not discuss memory. */
+size_t entmax_attn_workspace_bytes(const entmax_attn_params* params, int is_bwd);
+
+/* Forward pass: Eq. 1 applied to the ASEntmax-scaled logits of every query row (Eq. "asentmax",
+ * Sec. 2.1), output O and the per-row threshold tau.
+ *   q, k, v      in,  device, layout above, dtype per params->dtype
+ *   beta, gamma, delta   in, device float32[heads]; pass all three or none (none: c_i = 1)
+ *   o            out, device, same layout/dtype as q
+ *   tau          out, device float32 [batch, heads, seq]; Eq. 1's tau (a one-hot row has
+ *                tau = (alpha-1) s_max - 1)
+ *   workspace    device scratch, 256-byte aligned, >= entmax_attn_workspace_bytes(params, 0); contents
+ *                on return: see entmax_attn_workspace_layout
+ *   device_status  optional device int32[ENTMAX_ATTN_STATUS_WORDS]
+ * Errors: negative status, nothing enqueued. */
+int entmax_attn_fwd(const entmax_attn_params* params, const void* q, const void* k, const void* v,
+                    const float* beta, const float* gamma, const float* delta, void* o, float* tau,
+                    void* workspace, size_t workspace_bytes, int32_t* device_status, void* cuda_stream);
+
+/* Backward pass: the Jacobian of Eq. 1 (see the top of this file) and the three input gradients.
+ *   tau          in, device float32 [batch, heads, seq]: the thresholds the forward call returned
+ *   d_o          in, gradient w.r.t. O, layout/dtype of q
+ *   dq, dk, dv   out, layout/dtype of q (overwritten, not accumulated into)
+ *   workspace    >= entmax_attn_workspace_bytes(params, 1)
+ * No other state of the forward call is needed. */
+int entmax_attn_bwd(const entmax_attn_params* params, const void* q, const void* k, const void* v,
+                    const float* beta, const float* gamma, const float* delta, const float* tau,
+                    const void* d_o, void* dq, void* dk, void* dv, void* workspace,
+                    size_t workspace_bytes, int32_t* device_status, void* cuda_stream);
+
+/* Where a finished forward call leaves the support of every row inside its workspace (App. A: the
+ * support of row i is {j : (alpha-1) s_ij > tau_i}).  Byte offsets from the workspace base:
+ *   row_count  int32 [batch*heads*seq]: support size of the row, or -2 when the support has more than
+ *              `capacity` entries (the row was computed by the dense path and its list is not kept)
+ *   entries    {float y; int32 j;} [batch*heads*seq][capacity]: the first row_count slots hold the
+ *              support, y = (alpha-1) s_ij as the kernel computed it (fp32), in no particular order
+ *   scale      float32 [heads*seq]: c_i
+ * No paper counterpart (debugging / verification aid). */
+typedef struct {
+  size_t row_count_offset;
+  size_t entries_offset;
+  size_t scale_offset;
+  int32_t capacity;
+  int32_t reserved;
+} entmax_attn_ws_layout;
+int entmax_attn_workspace_layout(const entmax_attn_params* params, entmax_attn_ws_layout* out);
+
+/* The score-tile engine on its own (Sec. 2.1 logits before any scale): writes the raw tensor-core
+ * accumulators <q_i, k_j> (bf16 inputs, fp32 accumulation) of one (batch, head) pair,
+ * bh = b*heads + h, into s_out, a device float32 [seq, seq] row-major matrix, for all i and all j the
+ * mask keeps; other entries are left untouched.  bf16 params only; workspace as for the forward pass.
+ * Meant for verification on small seq. */
+int entmax_attn_scores_debug(const entmax_attn_params* params, const void* q, const void* k,
+                             int32_t bh, float* s_out, void* workspace, size_t workspace_bytes,
+                             int32_t* device_status, void* cuda_stream);
+
+/* Text for a status code (static storage). */
+const char* entmax_attn_strerror(int code);
+
+/* The cudaError_t of the last failing CUDA call made by this library on the calling thread (0 if none). */
+int entmax_attn_last_cuda_error(void);
+
+/* Library version, major*10000 + minor*100 + patch. */
+int entmax_attn_version(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* ENTMAX_ATTN_H_ */

@@ -1,0 +1,203 @@
+"""Thin ctypes binding of ``libentmax_attn.so``: argument marshalling only.
+
+Same entry-point names as ``include/entmax_attn.h``.  PyTorch supplies device memory and streams;
+every step of the computation runs in the library's CUDA kernels.  There is no fallback: if the
+library is missing or a call is rejected, an exception is raised.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+from typing import Optional
+
+import torch
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_HERE, "libentmax_attn.so")
+
+DTYPE_BF16, DTYPE_FP32 = 0, 1
+STATUS_WORDS = 4
+STATUS_FLAGS, STATUS_DENSE_ROWS = 0, 1
+FLAG_WAIT_EXPIRED, FLAG_BAD_SCALE = 1, 2
+
+
+class Params(ctypes.Structure):
+    _fields_ = [("batch", ctypes.c_int32), ("heads", ctypes.c_int32), ("seq", ctypes.c_int32),
+                ("head_dim", ctypes.c_int32), ("dtype", ctypes.c_int32), ("causal", ctypes.c_int32),
+                ("n_mode", ctypes.c_int32), ("alpha", ctypes.c_float), ("sm_scale", ctypes.c_float),
+                ("stride_b", ctypes.c_int64), ("stride_h", ctypes.c_int64), ("stride_n", ctypes.c_int64)]
+
+
+class WsLayout(ctypes.Structure):
+    _fields_ = [("row_count_offset", ctypes.c_size_t), ("entries_offset", ctypes.c_size_t),
+                ("scale_offset", ctypes.c_size_t), ("capacity", ctypes.c_int32), ("reserved", ctypes.c_int32)]
+
+
+class EntmaxAttnError(RuntimeError):
+    pass
+
+
+_lib = None
+
+
+def load():
+    """Loads the CUDA library (raises if it has not been built)."""
+    global _lib
+    if _lib is None:
+        if not os.path.exists(LIB_PATH):
+            raise EntmaxAttnError(
+                "libentmax_attn.so is missing: build it with `python -m paper_2506_16640_b200.build` "
+                "(there is no CPU or PyTorch fallback)")
+        lib = ctypes.CDLL(LIB_PATH)
+        vp, fp, ip = ctypes.c_void_p, ctypes.c_void_p, ctypes.c_void_p
+        pp = ctypes.POINTER(Params)
+        lib.entmax_attn_workspace_bytes.restype = ctypes.c_size_t
+        lib.entmax_attn_workspace_bytes.argtypes = [pp, ctypes.c_int]
+        lib.entmax_attn_workspace_layout.restype = ctypes.c_int
+        lib.entmax_attn_workspace_layout.argtypes = [pp, ctypes.POINTER(WsLayout)]
+        lib.entmax_attn_fwd.restype = ctypes.c_int
+        lib.entmax_attn_fwd.argtypes = [pp, vp, vp, vp, fp, fp, fp, vp, fp, vp, ctypes.c_size_t, ip, vp]
+        lib.entmax_attn_bwd.restype = ctypes.c_int
+        lib.entmax_attn_bwd.argtypes = [pp, vp, vp, vp, fp, fp, fp, fp, vp, vp, vp, vp, vp, ctypes.c_size_t, ip, vp]
+        lib.entmax_attn_scores_debug.restype = ctypes.c_int
+        lib.entmax_attn_scores_debug.argtypes = [pp, vp, vp, ctypes.c_int32, fp, vp, ctypes.c_size_t, ip, vp]
+        lib.entmax_attn_strerror.restype = ctypes.c_char_p
+        lib.entmax_attn_strerror.argtypes = [ctypes.c_int]
+        lib.entmax_attn_last_cuda_error.restype = ctypes.c_int
+        lib.entmax_attn_version.restype = ctypes.c_int
+        _lib = lib
+    return _lib
+
+
+def _check(rc: int, what: str):
+    if rc != 0:
+        lib = load()
+        msg = lib.entmax_attn_strerror(rc).decode()
+        extra = ""
+        if rc == -7:
+            extra = " (cudaError %d)" % lib.entmax_attn_last_cuda_error()
+        raise EntmaxAttnError("%s failed: %s%s" % (what, msg, extra))
+
+
+def _ptr(t: Optional[torch.Tensor]):
+    return None if t is None else ctypes.c_void_p(t.data_ptr())
+
+
+def make_params(q: torch.Tensor, alpha: float, causal: bool, sm_scale: float = 0.0, n_mode: int = 0) -> Params:
+    if q.dim() != 4:
+        raise EntmaxAttnError("expected [batch, heads, seq, head_dim] tensors")
+    if q.dtype == torch.bfloat16:
+        dt = DTYPE_BF16
+    elif q.dtype == torch.float32:
+        dt = DTYPE_FP32
+    else:
+        raise EntmaxAttnError("dtype must be bfloat16 or float32")
+    if q.stride(3) != 1:
+        raise EntmaxAttnError("head_dim must be the innermost, contiguous dimension")
+    B, H, N, D = q.shape
+    return Params(B, H, N, D, dt, int(bool(causal)), int(n_mode), float(alpha), float(sm_scale),
+                  q.stride(0), q.stride(1), q.stride(2))
+
+
+def _same_layout(ref: torch.Tensor, *others):
+    for t in others:
+        if t.shape != ref.shape or t.stride() != ref.stride() or t.dtype != ref.dtype or t.device != ref.device:
+            raise EntmaxAttnError("all [B,H,N,D] tensors of a call must share shape, strides, dtype and device")
+
+
+def entmax_attn_workspace_bytes(params: Params, is_bwd: bool) -> int:
+    return int(load().entmax_attn_workspace_bytes(ctypes.byref(params), int(bool(is_bwd))))
+
+
+def entmax_attn_workspace_layout(params: Params) -> WsLayout:
+    out = WsLayout()
+    _check(load().entmax_attn_workspace_layout(ctypes.byref(params), ctypes.byref(out)), "entmax_attn_workspace_layout")
+    return out
+
+
+def alloc_workspace(params: Params, is_bwd: bool, device) -> torch.Tensor:
+    nbytes = entmax_attn_workspace_bytes(params, is_bwd)
+    if nbytes == 0:
+        raise EntmaxAttnError("invalid parameters (workspace size query returned 0)")
+    return torch.empty(nbytes, dtype=torch.uint8, device=device)   # torch's allocator aligns to >= 512 B
+
+
+def _stream_ptr(stream):
+    s = torch.cuda.current_stream() if stream is None else stream
+    return ctypes.c_void_p(s.cuda_stream)
+
+
+def entmax_attn_fwd(q, k, v, alpha, causal, beta=None, gamma=None, delta=None, *, sm_scale=0.0, n_mode=0,
+                    o=None, tau=None, workspace=None, status=None, stream=None):
+    """Forward pass.  Returns (o, tau).  `workspace` (uint8 CUDA tensor) and `status` (int32[4] CUDA
+    tensor) are allocated when not given; pass your own to inspect them afterwards."""
+    _same_layout(q, k, v)
+    params = make_params(q, alpha, causal, sm_scale, n_mode)
+    if o is None:
+        o = torch.empty_like(q)
+    else:
+        _same_layout(q, o)
+    B, H, N, _ = q.shape
+    if tau is None:
+        tau = torch.empty((B, H, N), dtype=torch.float32, device=q.device)
+    if workspace is None:
+        workspace = alloc_workspace(params, False, q.device)
+    rc = load().entmax_attn_fwd(ctypes.byref(params), _ptr(q), _ptr(k), _ptr(v), _ptr(beta), _ptr(gamma), _ptr(delta),
+                                _ptr(o), _ptr(tau), _ptr(workspace), workspace.numel(), _ptr(status),
+                                _stream_ptr(stream))
+    _check(rc, "entmax_attn_fwd")
+    return o, tau
+
+
+def entmax_attn_bwd(q, k, v, tau, d_o, alpha, causal, beta=None, gamma=None, delta=None, *, sm_scale=0.0, n_mode=0,
+                    dq=None, dk=None, dv=None, workspace=None, status=None, stream=None):
+    """Backward pass.  Returns (dq, dk, dv)."""
+    _same_layout(q, k, v, d_o)
+    params = make_params(q, alpha, causal, sm_scale, n_mode)
+    dq = torch.empty_like(q) if dq is None else dq
+    dk = torch.empty_like(q) if dk is None else dk
+    dv = torch.empty_like(q) if dv is None else dv
+    _same_layout(q, dq, dk, dv)
+    if workspace is None:
+        workspace = alloc_workspace(params, True, q.device)
+    rc = load().entmax_attn_bwd(ctypes.byref(params), _ptr(q), _ptr(k), _ptr(v), _ptr(beta), _ptr(gamma), _ptr(delta),
+                                _ptr(tau), _ptr(d_o), _ptr(dq), _ptr(dk), _ptr(dv), _ptr(workspace),
+                                workspace.numel(), _ptr(status), _stream_ptr(stream))
+    _check(rc, "entmax_attn_bwd")
+    return dq, dk, dv
+
+
+def entmax_attn_scores_debug(q, k, bh, causal, *, workspace=None, status=None, stream=None):
+    """Raw tensor-core accumulators <q_i, k_j> of one (batch, head) pair as a float32 [N, N] tensor
+    (NaN where the mask removes the entry)."""
+    _same_layout(q, k)
+    params = make_params(q, 1.5, causal)
+    N = q.shape[2]
+    out = torch.full((N, N), float("nan"), dtype=torch.float32, device=q.device)
+    if workspace is None:
+        workspace = alloc_workspace(params, False, q.device)
+    rc = load().entmax_attn_scores_debug(ctypes.byref(params), _ptr(q), _ptr(k), int(bh), _ptr(out), _ptr(workspace),
+                                         workspace.numel(), _ptr(status), _stream_ptr(stream))
+    _check(rc, "entmax_attn_scores_debug")
+    return out
+
+
+def read_support(params: Params, workspace: torch.Tensor, rows):
+    """Support lists a forward call left in its workspace, for global row ids `rows`
+    (row id = (b*heads + h)*seq + i).  Returns a list of (indices int64 tensor or None, y float32 tensor or None)."""
+    lay = entmax_attn_workspace_layout(params)
+    total = params.batch * params.heads * params.seq
+    cnt = workspace[lay.row_count_offset: lay.row_count_offset + 4 * total].view(torch.int32)
+    ent = workspace[lay.entries_offset: lay.entries_offset + 8 * total * lay.capacity].view(torch.int32)
+    ent = ent.view(total, lay.capacity, 2)
+    rows_t = torch.as_tensor(rows, dtype=torch.long, device=workspace.device)
+    cnt_h = cnt[rows_t].cpu()
+    ent_h = ent[rows_t].cpu()
+    out = []
+    for r in range(len(rows)):
+        c = int(cnt_h[r])
+        if c < 0:
+            out.append((None, None))
+        else:
+            out.append((ent_h[r, :c, 1].to(torch.int64), ent_h[r, :c, 0].contiguous().view(torch.float32)))
+    return out

@@ -1,0 +1,85 @@
+// Internal declarations shared by the translation units of libentmax_attn.so.
+#pragma once
+
+#include <cuda_runtime.h>
+#include <cuda_bf16.h>
+#include <stddef.h>
+#include <stdint.h>
+
+#include "entmax_attn.h"
+
+namespace entmax {
+
+// Sparse row list: capacity per row and the fill level above which a row is handed to the dense path.
+constexpr int kListCap = 128;
+constexpr int kListKeep = 96;
+
+// One list slot: y = (alpha-1) * s_ij (or the raw accumulator while a sweep is running), j = key index.
+struct __align__(8) Entry {
+  float y;
+  int32_t j;
+};
+
+// Exponent class of 1/(alpha-1): powers by multiplication for 1, 2, 4; powf otherwise.
+enum ExpoClass : int { kExpoGeneral = 0, kExpo1 = 1, kExpo2 = 2, kExpo4 = 4 };
+
+struct Problem {
+  int B, H, N, D;
+  int causal, n_mode;
+  int dtype;
+  float alpha, sm_scale;
+  float expo;        // e = 1/(alpha-1)
+  int expo_class;
+  int64_t sb, sh, sn;  // element strides of the [B,H,N,D] tensors
+  int has_scale;
+};
+
+struct WsLayout {
+  size_t scale, row_cnt, row_thr, entries, fb_count, fb_list, scratch, acc_dk, acc_dv, total;
+  int scratch_ctas;     // CTAs of the dense-row kernels (each owns scratch_floats floats)
+  size_t scratch_floats;
+};
+
+WsLayout make_layout(const Problem& p, bool is_bwd);
+
+// y^e and y^(e-1) for y > 0
+__device__ __forceinline__ void pow_pair(float y, int expo_class, float expo, float& ye, float& ye1) {
+  if (expo_class == kExpo2) { ye1 = y; ye = y * y; }
+  else if (expo_class == kExpo1) { ye1 = 1.0f; ye = y; }
+  else if (expo_class == kExpo4) { float t = y * y; ye1 = t * y; ye = t * t; }
+  else { ye1 = powf(y, expo - 1.0f); ye = ye1 * y; }
+}
+
+// ---- launchers (each enqueues on `stream` and returns the cudaError_t of the launch) -------------
+cudaError_t launch_scale_table(const Problem& p, const float* beta, const float* gamma, const float* delta,
+                               float* scale, int32_t* status, cudaStream_t stream);
+
+// dense-row path (CUDA cores): all rows (row_list == nullptr) or the rows in row_list[0 .. *row_count)
+cudaError_t launch_dense_fwd(const Problem& p, const void* q, const void* k, const void* v, const float* scale,
+                             void* o, float* tau, int32_t* row_cnt, Entry* entries, const int32_t* row_list,
+                             const int32_t* row_count, float* scratch, size_t scratch_floats, int ctas,
+                             cudaStream_t stream);
+cudaError_t launch_dense_bwd(const Problem& p, const void* q, const void* k, const void* v, const void* d_o,
+                             const float* scale, const float* tau, void* dq, float* acc_dk, float* acc_dv,
+                             const int32_t* row_list, const int32_t* row_count, float* scratch,
+                             size_t scratch_floats, int ctas, cudaStream_t stream);
+
+// tcgen05 score sweep (bf16): fills the per-row candidate lists.
+//   mode 0: threshold search (forward); mode 1: threshold given in tau_in (backward)
+cudaError_t launch_sweep(const Problem& p, const void* q, const void* k, const float* scale, const float* tau_in,
+                         int mode, int32_t* row_cnt, float* row_thr, Entry* entries, float* dump, int dump_bh,
+                         int32_t* status, cudaStream_t stream);
+
+// per-row solve + gather kernels working on the lists (bf16 path)
+cudaError_t launch_row_fwd(const Problem& p, const void* v, const float* scale, int32_t* row_cnt,
+                           const float* row_thr, Entry* entries, void* o, float* tau, int32_t* fb_count,
+                           int32_t* fb_list, int32_t* status, cudaStream_t stream);
+cudaError_t launch_row_bwd(const Problem& p, const void* q, const void* k, const void* v, const void* d_o,
+                           const float* scale, const float* tau, int32_t* row_cnt, Entry* entries, void* dq,
+                           float* acc_dk, float* acc_dv, int32_t* fb_count, int32_t* fb_list, int32_t* status,
+                           cudaStream_t stream);
+
+// fp32 accumulators [B,H,N,D] contiguous -> strided output tensor of the problem dtype
+cudaError_t launch_store_grad(const Problem& p, const float* acc, void* out, cudaStream_t stream);
+
+}  // namespace entmax

@@ -1,0 +1,296 @@
+// C ABI of libentmax_attn.so: argument validation, workspace carving and the stream-ordered launch
+// sequences of the forward and backward passes.  See include/entmax_attn.h for the contract.
+#include <cmath>
+#include <cstring>
+
+#include "common.cuh"
+
+namespace entmax {
+
+namespace {
+
+thread_local int g_last_cuda_error = 0;
+
+inline size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
+
+int fail_cuda(cudaError_t err) {
+  g_last_cuda_error = (int)err;
+  return ENTMAX_ATTN_ECUDA;
+}
+
+bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+
+// Validates params and fills the internal problem description.  Returns a status code.
+int make_problem(const entmax_attn_params* params, Problem* out) {
+  if (!params) return ENTMAX_ATTN_EINVAL_NULL;
+  Problem p;
+  p.B = params->batch; p.H = params->heads; p.N = params->seq; p.D = params->head_dim;
+  if (p.B < 1 || p.H < 1 || p.N < 1) return ENTMAX_ATTN_EINVAL_SHAPE;
+  if (p.D != 64 && p.D != 128) return ENTMAX_ATTN_EINVAL_SHAPE;
+  if ((long long)p.B * p.H * p.N > 0x7fffffffLL / 2) return ENTMAX_ATTN_EINVAL_SHAPE;  // row ids are int32
+  if (params->dtype != ENTMAX_ATTN_DTYPE_BF16 && params->dtype != ENTMAX_ATTN_DTYPE_FP32) return ENTMAX_ATTN_EINVAL_DTYPE;
+  p.dtype = params->dtype;
+  p.causal = params->causal ? 1 : 0;
+  p.n_mode = params->n_mode ? 1 : 0;
+  p.alpha = params->alpha;
+  if (!(p.alpha > 1.0f) || !(p.alpha <= 2.0f)) return ENTMAX_ATTN_EINVAL_ALPHA;
+  p.sm_scale = params->sm_scale;
+  if (!std::isfinite(p.sm_scale) || p.sm_scale < 0.f) return ENTMAX_ATTN_EINVAL_ALPHA;
+  if (p.sm_scale == 0.f) p.sm_scale = 1.0f / std::sqrt((float)p.D);
+  p.expo = 1.0f / (p.alpha - 1.0f);
+  p.expo_class = p.alpha == 2.0f ? kExpo1 : p.alpha == 1.5f ? kExpo2 : p.alpha == 1.25f ? kExpo4 : kExpoGeneral;
+  if (params->stride_b == 0 && params->stride_h == 0 && params->stride_n == 0) {
+    p.sn = p.D;
+    p.sh = (int64_t)p.N * p.D;
+    p.sb = (int64_t)p.H * p.N * p.D;
+  } else {
+    p.sb = params->stride_b; p.sh = params->stride_h; p.sn = params->stride_n;
+    if (p.sn < p.D || p.sh < 1 || p.sb < 1) return ENTMAX_ATTN_EINVAL_SHAPE;
+    if (p.sn % 8 || p.sh % 8 || p.sb % 8) return ENTMAX_ATTN_EINVAL_SHAPE;
+  }
+  p.has_scale = 0;
+  *out = p;
+  return ENTMAX_ATTN_OK;
+}
+
+int check_scale_ptrs(const float* beta, const float* gamma, const float* delta, Problem* p) {
+  const int given = (beta != nullptr) + (gamma != nullptr) + (delta != nullptr);
+  if (given != 0 && given != 3) return ENTMAX_ATTN_EINVAL_NULL;
+  p->has_scale = given == 3;
+  return ENTMAX_ATTN_OK;
+}
+
+int check_workspace(const Problem& p, bool is_bwd, void* ws, size_t ws_bytes, WsLayout* lay) {
+  *lay = make_layout(p, is_bwd);
+  if (!ws || (reinterpret_cast<uintptr_t>(ws) & 255u) != 0 || ws_bytes < lay->total) return ENTMAX_ATTN_EINVAL_WORKSPACE;
+  return ENTMAX_ATTN_OK;
+}
+
+int check_device_for_bf16() {
+  int dev = 0, major = 0;
+  cudaError_t err = cudaGetDevice(&dev);
+  if (err != cudaSuccess) return fail_cuda(err);
+  err = cudaDeviceGetAttribute(&major, cudaDevAttrComputeCapabilityMajor, dev);
+  if (err != cudaSuccess) return fail_cuda(err);
+  return major == 10 ? ENTMAX_ATTN_OK : ENTMAX_ATTN_EUNSUPPORTED;
+}
+
+}  // namespace
+
+WsLayout make_layout(const Problem& p, bool is_bwd) {
+  WsLayout l;
+  const size_t rows = (size_t)p.B * p.H * p.N;
+  size_t off = 0;
+  auto take = [&off](size_t bytes) { size_t at = off; off = align_up(off + bytes, 256); return at; };
+  l.scale = take((size_t)p.H * p.N * sizeof(float));
+  l.row_cnt = take(rows * sizeof(int32_t));
+  l.row_thr = take(rows * sizeof(float));
+  l.entries = take(rows * kListCap * sizeof(Entry));
+  l.fb_count = take(256);
+  l.fb_list = take(rows * sizeof(int32_t));
+  // dense-row CTAs: enough to fill the machine, few enough that their score rows stay modest
+  l.scratch_floats = align_up((size_t)p.N, 32) * (is_bwd ? 2 : 1);   // scores (+ dP in backward)
+  size_t ctas = 148 * 4;
+  if (ctas > rows) ctas = rows;
+  l.scratch_ctas = (int)ctas;
+  l.scratch = take(ctas * l.scratch_floats * sizeof(float));
+  l.acc_dk = l.acc_dv = 0;
+  if (is_bwd) {
+    l.acc_dk = take(rows * p.D * sizeof(float));
+    l.acc_dv = take(rows * p.D * sizeof(float));
+  }
+  l.total = off;
+  return l;
+}
+
+}  // namespace entmax
+
+using namespace entmax;
+
+extern "C" {
+
+size_t entmax_attn_workspace_bytes(const entmax_attn_params* params, int is_bwd) {
+  Problem p;
+  if (make_problem(params, &p) != ENTMAX_ATTN_OK) return 0;
+  return make_layout(p, is_bwd != 0).total;
+}
+
+int entmax_attn_workspace_layout(const entmax_attn_params* params, entmax_attn_ws_layout* out) {
+  Problem p;
+  int rc = make_problem(params, &p);
+  if (rc != ENTMAX_ATTN_OK) return rc;
+  if (!out) return ENTMAX_ATTN_EINVAL_NULL;
+  const WsLayout l = make_layout(p, false);
+  out->row_count_offset = l.row_cnt;
+  out->entries_offset = l.entries;
+  out->scale_offset = l.scale;
+  out->capacity = kListCap;
+  out->reserved = 0;
+  return ENTMAX_ATTN_OK;
+}
+
+int entmax_attn_fwd(const entmax_attn_params* params, const void* q, const void* k, const void* v,
+                    const float* beta, const float* gamma, const float* delta, void* o, float* tau,
+                    void* workspace, size_t workspace_bytes, int32_t* device_status, void* cuda_stream) {
+  Problem p;
+  int rc = make_problem(params, &p);
+  if (rc != ENTMAX_ATTN_OK) return rc;
+  if (!q || !k || !v || !o || !tau) return ENTMAX_ATTN_EINVAL_NULL;
+  rc = check_scale_ptrs(beta, gamma, delta, &p);
+  if (rc != ENTMAX_ATTN_OK) return rc;
+  if (!aligned16(q) || !aligned16(k) || !aligned16(v) || !aligned16(o) || !aligned16(tau)) return ENTMAX_ATTN_EINVAL_ALIGN;
+  WsLayout lay;
+  rc = check_workspace(p, false, workspace, workspace_bytes, &lay);
+  if (rc != ENTMAX_ATTN_OK) return rc;
+  if (p.dtype == ENTMAX_ATTN_DTYPE_BF16) {
+    rc = check_device_for_bf16();
+    if (rc != ENTMAX_ATTN_OK) return rc;
+  }
+  cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
+  uint8_t* ws = static_cast<uint8_t*>(workspace);
+  float* scale = reinterpret_cast<float*>(ws + lay.scale);
+  int32_t* row_cnt = reinterpret_cast<int32_t*>(ws + lay.row_cnt);
+  float* row_thr = reinterpret_cast<float*>(ws + lay.row_thr);
+  Entry* entries = reinterpret_cast<Entry*>(ws + lay.entries);
+  int32_t* fb_count = reinterpret_cast<int32_t*>(ws + lay.fb_count);
+  int32_t* fb_list = reinterpret_cast<int32_t*>(ws + lay.fb_list);
+  float* scratch = reinterpret_cast<float*>(ws + lay.scratch);
+  cudaError_t err;
+  if (device_status) {
+    err = cudaMemsetAsync(device_status, 0, sizeof(int32_t) * ENTMAX_ATTN_STATUS_WORDS, stream);
+    if (err != cudaSuccess) return fail_cuda(err);
+  }
+  err = launch_scale_table(p, beta, gamma, delta, scale, device_status, stream);
+  if (err != cudaSuccess) return fail_cuda(err);
+  if (p.dtype == ENTMAX_ATTN_DTYPE_FP32) {
+    err = launch_dense_fwd(p, q, k, v, scale, o, tau, row_cnt, entries, nullptr, nullptr, scratch, lay.scratch_floats,
+                           lay.scratch_ctas, stream);
+    return err == cudaSuccess ? ENTMAX_ATTN_OK : fail_cuda(err);
+  }
+  err = cudaMemsetAsync(fb_count, 0, sizeof(int32_t), stream);
+  if (err != cudaSuccess) return fail_cuda(err);
+  err = launch_sweep(p, q, k, scale, nullptr, 0, row_cnt, row_thr, entries, nullptr, -1, device_status, stream);
+  if (err != cudaSuccess) return fail_cuda(err);
+  err = launch_row_fwd(p, v, scale, row_cnt, row_thr, entries, o, tau, fb_count, fb_list, device_status, stream);
+  if (err != cudaSuccess) return fail_cuda(err);
+  err = launch_dense_fwd(p, q, k, v, scale, o, tau, row_cnt, entries, fb_list, fb_count, scratch, lay.scratch_floats,
+                         lay.scratch_ctas, stream);
+  return err == cudaSuccess ? ENTMAX_ATTN_OK : fail_cuda(err);
+}
+
+int entmax_attn_bwd(const entmax_attn_params* params, const void* q, const void* k, const void* v,
+                    const float* beta, const float* gamma, const float* delta, const float* tau,
+                    const void* d_o, void* dq, void* dk, void* dv, void* workspace,
+                    size_t workspace_bytes, int32_t* device_status, void* cuda_stream) {
+  Problem p;
+  int rc = make_problem(params, &p);
+  if (rc != ENTMAX_ATTN_OK) return rc;
+  if (!q || !k || !v || !tau || !d_o || !dq || !dk || !dv) return ENTMAX_ATTN_EINVAL_NULL;
+  rc = check_scale_ptrs(beta, gamma, delta, &p);
+  if (rc != ENTMAX_ATTN_OK) return rc;
+  if (!aligned16(q) || !aligned16(k) || !aligned16(v) || !aligned16(tau) || !aligned16(d_o) || !aligned16(dq) ||
+      !aligned16(dk) || !aligned16(dv))
+    return ENTMAX_ATTN_EINVAL_ALIGN;
+  WsLayout lay;
+  rc = check_workspace(p, true, workspace, workspace_bytes, &lay);
+  if (rc != ENTMAX_ATTN_OK) return rc;
+  if (p.dtype == ENTMAX_ATTN_DTYPE_BF16) {
+    rc = check_device_for_bf16();
+    if (rc != ENTMAX_ATTN_OK) return rc;
+  }
+  cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
+  uint8_t* ws = static_cast<uint8_t*>(workspace);
+  float* scale = reinterpret_cast<float*>(ws + lay.scale);
+  int32_t* row_cnt = reinterpret_cast<int32_t*>(ws + lay.row_cnt);
+  float* row_thr = reinterpret_cast<float*>(ws + lay.row_thr);
+  Entry* entries = reinterpret_cast<Entry*>(ws + lay.entries);
+  int32_t* fb_count = reinterpret_cast<int32_t*>(ws + lay.fb_count);
+  int32_t* fb_list = reinterpret_cast<int32_t*>(ws + lay.fb_list);
+  float* scratch = reinterpret_cast<float*>(ws + lay.scratch);
+  float* acc_dk = reinterpret_cast<float*>(ws + lay.acc_dk);
+  float* acc_dv = reinterpret_cast<float*>(ws + lay.acc_dv);
+  const size_t acc_bytes = (size_t)p.B * p.H * p.N * p.D * sizeof(float);
+  cudaError_t err;
+  if (device_status) {
+    err = cudaMemsetAsync(device_status, 0, sizeof(int32_t) * ENTMAX_ATTN_STATUS_WORDS, stream);
+    if (err != cudaSuccess) return fail_cuda(err);
+  }
+  err = cudaMemsetAsync(acc_dk, 0, acc_bytes, stream);
+  if (err != cudaSuccess) return fail_cuda(err);
+  err = cudaMemsetAsync(acc_dv, 0, acc_bytes, stream);
+  if (err != cudaSuccess) return fail_cuda(err);
+  err = launch_scale_table(p, beta, gamma, delta, scale, device_status, stream);
+  if (err != cudaSuccess) return fail_cuda(err);
+  if (p.dtype == ENTMAX_ATTN_DTYPE_FP32) {
+    err = launch_dense_bwd(p, q, k, v, d_o, scale, tau, dq, acc_dk, acc_dv, nullptr, nullptr, scratch,
+                           lay.scratch_floats, lay.scratch_ctas, stream);
+    if (err != cudaSuccess) return fail_cuda(err);
+  } else {
+    err = cudaMemsetAsync(fb_count, 0, sizeof(int32_t), stream);
+    if (err != cudaSuccess) return fail_cuda(err);
+    err = launch_sweep(p, q, k, scale, tau, 1, row_cnt, row_thr, entries, nullptr, -1, device_status, stream);
+    if (err != cudaSuccess) return fail_cuda(err);
+    err = launch_row_bwd(p, q, k, v, d_o, scale, tau, row_cnt, entries, dq, acc_dk, acc_dv, fb_count, fb_list,
+                         device_status, stream);
+    if (err != cudaSuccess) return fail_cuda(err);
+    err = launch_dense_bwd(p, q, k, v, d_o, scale, tau, dq, acc_dk, acc_dv, fb_list, fb_count, scratch,
+                           lay.scratch_floats, lay.scratch_ctas, stream);
+    if (err != cudaSuccess) return fail_cuda(err);
+  }
+  err = launch_store_grad(p, acc_dk, dk, stream);
+  if (err != cudaSuccess) return fail_cuda(err);
+  err = launch_store_grad(p, acc_dv, dv, stream);
+  return err == cudaSuccess ? ENTMAX_ATTN_OK : fail_cuda(err);
+}
+
+int entmax_attn_scores_debug(const entmax_attn_params* params, const void* q, const void* k, int32_t bh,
+                             float* s_out, void* workspace, size_t workspace_bytes, int32_t* device_status,
+                             void* cuda_stream) {
+  Problem p;
+  int rc = make_problem(params, &p);
+  if (rc != ENTMAX_ATTN_OK) return rc;
+  if (p.dtype != ENTMAX_ATTN_DTYPE_BF16) return ENTMAX_ATTN_EINVAL_DTYPE;
+  if (!q || !k || !s_out) return ENTMAX_ATTN_EINVAL_NULL;
+  if (bh < 0 || bh >= p.B * p.H) return ENTMAX_ATTN_EINVAL_SHAPE;
+  if (!aligned16(q) || !aligned16(k)) return ENTMAX_ATTN_EINVAL_ALIGN;
+  WsLayout lay;
+  rc = check_workspace(p, false, workspace, workspace_bytes, &lay);
+  if (rc != ENTMAX_ATTN_OK) return rc;
+  rc = check_device_for_bf16();
+  if (rc != ENTMAX_ATTN_OK) return rc;
+  cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
+  uint8_t* ws = static_cast<uint8_t*>(workspace);
+  float* scale = reinterpret_cast<float*>(ws + lay.scale);
+  cudaError_t err;
+  if (device_status) {
+    err = cudaMemsetAsync(device_status, 0, sizeof(int32_t) * ENTMAX_ATTN_STATUS_WORDS, stream);
+    if (err != cudaSuccess) return fail_cuda(err);
+  }
+  err = launch_scale_table(p, nullptr, nullptr, nullptr, scale, device_status, stream);
+  if (err != cudaSuccess) return fail_cuda(err);
+  err = launch_sweep(p, q, k, scale, nullptr, 0, reinterpret_cast<int32_t*>(ws + lay.row_cnt),
+                     reinterpret_cast<float*>(ws + lay.row_thr), reinterpret_cast<Entry*>(ws + lay.entries), s_out, bh,
+                     device_status, stream);
+  return err == cudaSuccess ? ENTMAX_ATTN_OK : fail_cuda(err);
+}
+
+const char* entmax_attn_strerror(int code) {
+  switch (code) {
+    case ENTMAX_ATTN_OK: return "ok";
+    case ENTMAX_ATTN_EINVAL_SHAPE: return "invalid shape or strides (head_dim must be 64 or 128; sizes >= 1; strides multiples of 8)";
+    case ENTMAX_ATTN_EINVAL_ALPHA: return "alpha must lie in (1, 2] and sm_scale must be finite and non-negative";
+    case ENTMAX_ATTN_EINVAL_DTYPE: return "unknown or unsupported dtype";
+    case ENTMAX_ATTN_EINVAL_ALIGN: return "tensor pointers must be 16-byte aligned";
+    case ENTMAX_ATTN_EINVAL_WORKSPACE: return "workspace missing, not 256-byte aligned, or too small";
+    case ENTMAX_ATTN_EINVAL_NULL: return "a required pointer is NULL (beta, gamma, delta: all or none)";
+    case ENTMAX_ATTN_ECUDA: return "a CUDA call failed (see entmax_attn_last_cuda_error)";
+    case ENTMAX_ATTN_EUNSUPPORTED: return "the bf16 path needs an sm_100 device";
+    default: return "unknown status";
+  }
+}
+
+int entmax_attn_last_cuda_error(void) { return g_last_cuda_error; }
+
+int entmax_attn_version(void) { return 100; }
+
+}  // extern "C"

@@ -1,0 +1,136 @@
+"""Helpers of the GPU parity tests: run the CUDA path through the binding, run the CPU oracle on the
+same seeded tensors, compare element by element with the tolerances of the target:
+
+  max |O - O_ref| <= 2e-2
+  |tau - tau_ref| / max(1, |tau_ref|) <= 1e-3 (bf16 inputs) or 1e-4 (fp32 inputs)
+  supports identical except for entries within 1e-3 of the threshold
+  gradients: max |dX - dX_ref| <= 2e-2 * max(1, max |dX_ref|)  (the forward tolerance scaled to the
+  gradient's magnitude; bf16 outputs alone carry 2^-9 relative rounding)
+"""
+from __future__ import annotations
+
+import numpy as np
+import torch
+
+import oracle
+from paper_2506_16640_b200 import binding
+
+O_TOL = 2e-2
+BAND = 1e-3
+
+
+def tau_tol(dtype_name: str) -> float:
+    return 1e-4 if dtype_name == "fp32" else 1e-3
+
+
+def to_device(inp, device="cuda"):
+    d = {name: getattr(inp, name).to(device) for name in ("q", "k", "v")}
+    d["d_o"] = inp.d_o.to(device) if inp.d_o is not None else None
+    for name in ("beta", "gamma", "delta"):
+        t = getattr(inp, name)
+        d[name] = t.to(device) if t is not None else None
+    return d
+
+
+def run_fwd(inp, alpha, dev=None, n_mode=0):
+    """CUDA forward through the C ABI.  Returns dict(o, tau, workspace, status, params) (device tensors)."""
+    dev = dev or to_device(inp)
+    w = inp.workload
+    params = binding.make_params(dev["q"], alpha, w.causal, 0.0, n_mode)
+    ws = binding.alloc_workspace(params, False, dev["q"].device)
+    status = torch.full((binding.STATUS_WORDS,), -1, dtype=torch.int32, device=dev["q"].device)
+    o, tau = binding.entmax_attn_fwd(dev["q"], dev["k"], dev["v"], alpha, w.causal, dev["beta"], dev["gamma"],
+                                     dev["delta"], n_mode=n_mode, workspace=ws, status=status)
+    torch.cuda.synchronize()
+    st = status.cpu()
+    assert int(st[binding.STATUS_FLAGS]) == 0, "device status flags: %d" % int(st[binding.STATUS_FLAGS])
+    return {"o": o, "tau": tau, "workspace": ws, "status": st, "params": params, "dev": dev}
+
+
+def run_bwd(inp, alpha, tau, dev=None, n_mode=0):
+    dev = dev or to_device(inp)
+    w = inp.workload
+    status = torch.full((binding.STATUS_WORDS,), -1, dtype=torch.int32, device=dev["q"].device)
+    dq, dk, dv = binding.entmax_attn_bwd(dev["q"], dev["k"], dev["v"], tau, dev["d_o"], alpha, w.causal, dev["beta"],
+                                         dev["gamma"], dev["delta"], n_mode=n_mode, status=status)
+    torch.cuda.synchronize()
+    st = status.cpu()
+    assert int(st[binding.STATUS_FLAGS]) == 0, "device status flags: %d" % int(st[binding.STATUS_FLAGS])
+    return {"dq": dq, "dk": dk, "dv": dv, "status": st}
+
+
+def check_fwd_rows(inp, alpha, got, bh, rows, n_mode=0, check_support=True):
+    """Compares rows `rows` of head index bh = b*H + h against the oracle.  Returns summary stats."""
+    w = inp.workload
+    b, h = divmod(bh, w.H)
+    q, k, v = (t[b, h].float().numpy() for t in (inp.q, inp.k, inp.v))
+    rows = np.asarray(rows, dtype=np.int64)
+    ref = oracle.attn_fwd_rows(q, k, v, rows, alpha, inp.sm_scale, w.causal, scale=inp.head_scale(h), n_mode=n_mode,
+                               want_p=check_support)
+    rows_t = torch.from_numpy(rows)
+    tau_g = got["tau"][b, h].cpu()[rows_t].double().numpy()
+    o_g = got["o"][b, h].cpu()[rows_t].double().numpy()
+    tau_err = np.abs(tau_g - ref["tau"]) / np.maximum(1.0, np.abs(ref["tau"]))
+    o_err = np.abs(o_g - ref["o"]).max(axis=1)
+    worst_t = int(np.argmax(tau_err))
+    assert tau_err.max() <= tau_tol(w.dtype), "tau: row %d (bh %d) gpu %.7g ref %.7g rel err %.3g" % (
+        rows[worst_t], bh, tau_g[worst_t], ref["tau"][worst_t], tau_err.max())
+    worst_o = int(np.argmax(o_err))
+    assert o_err.max() <= O_TOL, "O: row %d (bh %d) max abs err %.3g" % (rows[worst_o], bh, o_err.max())
+    stats = {"tau_err": float(tau_err.max()), "o_err": float(o_err.max()), "supp_mean": float(ref["supp"].mean()),
+             "supp_max": int(ref["supp"].max()), "band_mismatch": 0, "dense_rows": 0}
+    if check_support:
+        grow = bh * w.N + rows
+        lists = binding.read_support(got["params"], got["workspace"], grow)
+        for r, (idx, _y) in enumerate(lists):
+            i = int(rows[r])
+            if idx is None:
+                stats["dense_rows"] += 1
+                assert ref["supp"][r] > 128, "row %d: list dropped although the support has %d entries" % (i, ref["supp"][r])
+                continue
+            gpu_set = set(int(x) for x in idx)
+            assert len(gpu_set) == len(idx), "row %d: duplicate keys in the support list" % i
+            ref_set = set(int(x) for x in np.flatnonzero(ref["p"][r] > 0))
+            diff = gpu_set ^ ref_set
+            if diff:
+                nv = i + 1 if w.causal else w.N
+                n_i = w.N if n_mode else nv
+                sc = inp.head_scale(h)
+                c = oracle.asentmax_scale(sc[0], sc[1], sc[2], n_i) if sc is not None else 1.0
+                for j in diff:
+                    assert 0 <= j < nv, "row %d: key %d outside the mask" % (i, j)
+                    y = (alpha - 1) * c * float(q[i].astype(np.float64) @ k[j].astype(np.float64)) * inp.sm_scale
+                    assert abs(y - ref["tau"][r]) <= BAND, "row %d key %d: support differs, margin %.3g" % (
+                        i, j, y - ref["tau"][r])
+                stats["band_mismatch"] += len(diff)
+    return stats
+
+
+def grad_close(name, got, ref):
+    ref = np.asarray(ref, dtype=np.float64)
+    got = np.asarray(got, dtype=np.float64)
+    tol = 2e-2 * max(1.0, float(np.abs(ref).max()))
+    err = float(np.abs(got - ref).max())
+    assert err <= tol, "%s: max abs err %.4g > %.4g" % (name, err, tol)
+    return err
+
+
+def check_bwd_head(inp, alpha, got_bwd, bh, n_mode=0):
+    """Full dQ, dK, dV of one head against the oracle."""
+    w = inp.workload
+    b, h = divmod(bh, w.H)
+    q, k, v, d_o = (t[b, h].float().numpy() for t in (inp.q, inp.k, inp.v, inp.d_o))
+    dq, dk, dv = oracle.attn_bwd_head(q, k, v, d_o, alpha, inp.sm_scale, w.causal, scale=inp.head_scale(h), n_mode=n_mode)
+    return {"dq": grad_close("dQ", got_bwd["dq"][b, h].float().cpu().numpy(), dq),
+            "dk": grad_close("dK", got_bwd["dk"][b, h].float().cpu().numpy(), dk),
+            "dv": grad_close("dV", got_bwd["dv"][b, h].float().cpu().numpy(), dv)}
+
+
+def check_bwd_rows(inp, alpha, got_bwd, bh, rows, n_mode=0):
+    w = inp.workload
+    b, h = divmod(bh, w.H)
+    q, k, v, d_o = (t[b, h].float().numpy() for t in (inp.q, inp.k, inp.v, inp.d_o))
+    rows = np.asarray(rows, dtype=np.int64)
+    dq, _ = oracle.attn_bwd_rows(q, k, v, d_o, rows, alpha, inp.sm_scale, w.causal, scale=inp.head_scale(h), n_mode=n_mode)
+    got = got_bwd["dq"][b, h].float().cpu()[torch.from_numpy(rows)].numpy()
+    return grad_close("dQ rows", got, dq)
