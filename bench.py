@@ -1,0 +1,360 @@
+#!/usr/bin/env python
+"""Benchmark of the fused alpha-entmax / ASEntmax attention hot path on B200.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference] [--alpha A]
+
+One step = one forward call + one backward call of the C-ABI library on the long-context workload
+(batch 1, 16 heads, 32768 tokens, head dim 128, causal, bf16, 8 planted keys per planted query,
+per-head ASEntmax scales).  Prints ONE JSON line.  `value` is the useful attention throughput of the
+whole step in TFLOP/s: forward 4*d and backward 10*d FLOPs per visible (query, key) pair, i.e. the
+dense-equivalent work with causal halving, divided by the device time of the step.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+import numpy as np
+import torch
+
+from paper_2506_16640_b200.inputs import WORKLOADS, make_inputs, sample_rows, scaled
+
+METRIC = "entmax_attn_fwd_bwd_useful_tflops_n32k"
+UNIT = "TFLOP/s"
+NOMINAL_BF16_TFLOPS = 2250.0
+FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
+# DRAM bytes (read + write) of one forward score-sweep launch on the benchmark workload, from the ncu
+# capture summarised under profiles/ (None until a capture exists).
+SWEEP_DRAM_TRAFFIC_BYTES = None
+
+
+def visible_pairs(w) -> int:
+    per_head = w.N * (w.N + 1) // 2 if w.causal else w.N * w.N
+    return per_head * w.B * w.H
+
+
+def useful_flops(w):
+    pairs = visible_pairs(w)
+    return 4 * w.d * pairs, 10 * w.d * pairs
+
+
+def load_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        with open(path) as f:
+            return json.load(f), "measured"
+    return dict(FALLBACK_PEAKS), "fallback"
+
+
+class ClockSampler:
+    """Samples SM clocks and throttle reasons with nvidia-smi while the timed region runs."""
+    FIELDS = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
+              "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+              "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index: int):
+        self.index = index
+        self.proc = None
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(
+                ["nvidia-smi", "-i", str(self.index), "--query-gpu=" + self.FIELDS, "--format=csv,noheader,nounits",
+                 "-lms", "100"], stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+        except OSError:
+            self.proc = None
+
+    def stop(self):
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        time.sleep(0.15)
+        self.proc.terminate()
+        try:
+            out, _ = self.proc.communicate(timeout=5)
+        except subprocess.TimeoutExpired:
+            self.proc.kill()
+            out, _ = self.proc.communicate()
+        sm, smax, reasons = [], [], set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for line in out.splitlines():
+            parts = [p.strip() for p in line.split(",")]
+            if len(parts) < 7:
+                continue
+            try:
+                sm.append(float(parts[0]))
+                smax.append(float(parts[1]))
+            except ValueError:
+                continue
+            for name, val in zip(names, parts[3:7]):
+                if val.lower().startswith("active"):
+                    reasons.add(name)
+        return {"sm_mhz": statistics.median(sm) if sm else None, "sm_max_mhz": max(smax) if smax else None,
+                "reasons": sorted(reasons), "samples": len(sm)}
+
+
+def dist_setup(n_gpus: int):
+    """One process per GPU under torchrun; a single process otherwise."""
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    if world > 1:
+        import torch.distributed as dist
+        os.environ.setdefault("MASTER_ADDR", "127.0.0.1")
+        dist.init_process_group(backend="nccl" if torch.cuda.is_available() else "gloo")
+    return rank, world, local
+
+
+def aggregate_over_ranks(step_ms: float, units: float, world: int, device):
+    """Whole-job numbers: the slowest rank's time, the sum of all ranks' work.  The data path has no
+    collective (every rank owns whole (batch, head) problems); these two reductions are bookkeeping."""
+    if world == 1:
+        return step_ms, units
+    import torch.distributed as dist
+    t = torch.tensor([step_ms], dtype=torch.float64, device=device)
+    u = torch.tensor([units], dtype=torch.float64, device=device)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    dist.all_reduce(u, op=dist.ReduceOp.SUM)
+    return float(t.item()), float(u.item())
+
+
+def barrier(world: int):
+    if world > 1:
+        import torch.distributed as dist
+        dist.barrier()
+
+
+def make_bench_inputs(alpha: float):
+    """The long-context workload plus a seeded dO (the workload itself is forward-only)."""
+    w = WORKLOADS[4]
+    inp = make_inputs(w)
+    gen = torch.Generator(device="cpu")
+    gen.manual_seed(20250616 + 404)
+    inp.d_o = torch.randn((w.B, w.H, w.N, w.d), generator=gen, dtype=torch.float32).to(torch.bfloat16)
+    return w, inp
+
+
+def run_ours(args):
+    from paper_2506_16640_b200 import binding
+
+    rank, world, local = dist_setup(args.gpus)
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: there is no CPU fallback for the product path")
+    torch.cuda.set_device(local)
+    dev = torch.device("cuda", local)
+    binding.load()
+    alpha = args.alpha
+    w, inp = make_bench_inputs(alpha)
+    host = {"q": inp.q, "k": inp.k, "v": inp.v, "d_o": inp.d_o, "beta": inp.beta, "gamma": inp.gamma,
+            "delta": inp.delta}
+    host = {n: t.pin_memory() for n, t in host.items()}
+    d = {n: t.to(dev) for n, t in host.items()}
+    params = binding.make_params(d["q"], alpha, w.causal)
+    ws = binding.alloc_workspace(params, True, dev)          # the backward size covers the forward one
+    status = torch.zeros(binding.STATUS_WORDS, dtype=torch.int32, device=dev)
+    o = torch.empty_like(d["q"])
+    tau = torch.empty((w.B, w.H, w.N), dtype=torch.float32, device=dev)
+    dq, dk, dv = (torch.empty_like(d["q"]) for _ in range(3))
+    flush = torch.empty(256 << 20, dtype=torch.uint8, device=dev)
+
+    def fwd():
+        binding.entmax_attn_fwd(d["q"], d["k"], d["v"], alpha, w.causal, d["beta"], d["gamma"], d["delta"], o=o,
+                                tau=tau, workspace=ws, status=status)
+
+    def bwd():
+        binding.entmax_attn_bwd(d["q"], d["k"], d["v"], tau, d["d_o"], alpha, w.causal, d["beta"], d["gamma"],
+                                d["delta"], dq=dq, dk=dk, dv=dv, workspace=ws, status=status)
+
+    for _ in range(max(args.warmup, 3)):
+        fwd()
+        bwd()
+    torch.cuda.synchronize()
+    assert int(status[binding.STATUS_FLAGS].item()) == 0, "device status flags set during warm-up"
+    dense_rows = int(status[binding.STATUS_DENSE_ROWS].item())
+
+    K = args.steps
+    ev = lambda: torch.cuda.Event(enable_timing=True)
+    e_start, e_mid, e_stop = [ev() for _ in range(K)], [ev() for _ in range(K)], [ev() for _ in range(K)]
+    s_start, s_stop = [ev() for _ in range(K)], [ev() for _ in range(K)]
+    for e in s_start + s_stop:
+        e.record()                                          # creates the CUDA handles the hook needs
+    torch.cuda.synchronize()
+    sampler = ClockSampler(local)
+    barrier(world)
+    torch.cuda.synchronize()
+    sampler.start()
+    for i in range(K):
+        flush.zero_()                                       # evict L2 between steps (outside the timed events)
+        binding.entmax_attn_profile_events(0, s_start[i], s_stop[i])
+        e_start[i].record()
+        fwd()
+        e_mid[i].record()
+        bwd()
+        e_stop[i].record()
+    binding.entmax_attn_profile_events(0, None, None)
+    torch.cuda.synchronize()
+    barrier(world)
+    clocks = sampler.stop()
+    fwd_ms = sum(a.elapsed_time(b) for a, b in zip(e_start, e_mid)) / K
+    bwd_ms = sum(a.elapsed_time(b) for a, b in zip(e_mid, e_stop)) / K
+    step_ms = sum(a.elapsed_time(b) for a, b in zip(e_start, e_stop)) / K
+    sweep_ms = sum(a.elapsed_time(b) for a, b in zip(s_start, s_stop)) / K
+    assert int(status[binding.STATUS_FLAGS].item()) == 0, "device status flags set during the timed region"
+
+    # end to end: pinned host buffers in, results back to pinned host buffers, copies inside the timed region
+    names = ("q", "k", "v", "d_o", "beta", "gamma", "delta")
+    outs_dev = {"o": o, "tau": tau, "dq": dq, "dk": dk, "dv": dv}
+    outs_host = {n: torch.empty(t.shape, dtype=t.dtype).pin_memory() for n, t in outs_dev.items()}
+    h2d = sum(host[n].numel() * host[n].element_size() for n in names)
+    d2h = sum(t.numel() * t.element_size() for t in outs_dev.values())
+    E = max(1, min(K, 5))
+    ee_start, ee_stop = [ev() for _ in range(E)], [ev() for _ in range(E)]
+    barrier(world)
+    torch.cuda.synchronize()
+    for i in range(E):
+        ee_start[i].record()
+        for n in names:
+            d[n].copy_(host[n], non_blocking=True)
+        fwd()
+        bwd()
+        for n, t in outs_dev.items():
+            outs_host[n].copy_(t, non_blocking=True)
+        ee_stop[i].record()
+    torch.cuda.synchronize()
+    barrier(world)
+    e2e_ms = sum(a.elapsed_time(b) for a, b in zip(ee_start, ee_stop)) / E
+
+    f_fwd, f_bwd = useful_flops(w)
+    step_ms_all, flops_all = aggregate_over_ranks(step_ms, float(f_fwd + f_bwd), world, dev)
+    e2e_ms_all, _ = aggregate_over_ranks(e2e_ms, 0.0, world, dev)
+    if rank != 0:
+        return
+    peaks, peak_kind = load_peaks()
+    burst = float(peaks.get("bf16_tflops", FALLBACK_PEAKS["bf16_tflops"]))
+    sustained = float(peaks.get("bf16_tflops_sustained", FALLBACK_PEAKS["bf16_tflops_sustained"]))
+    sweep_flops = 2 * w.d * visible_pairs(w)                # algorithmic: one QK^T contraction per visible pair
+    sweep_tflops = sweep_flops / (sweep_ms * 1e-3) / 1e12
+    fwd_tflops = f_fwd / (fwd_ms * 1e-3) / 1e12
+    bwd_tflops = f_bwd / (bwd_ms * 1e-3) / 1e12
+    line = {
+        "metric": METRIC, "value": flops_all / (step_ms_all * 1e-3) / 1e12, "unit": UNIT, "n_gpus": world,
+        "steps": K, "warmup": max(args.warmup, 3), "ms_per_step": step_ms_all, "higher_is_better": True,
+        "scaling": "weak", "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
+        "config": {"workload": w.name, "batch": w.B, "heads": w.H, "seq": w.N, "head_dim": w.d, "causal": w.causal,
+                   "alpha": alpha, "step": "entmax_attn_fwd + entmax_attn_bwd", "l2": "256 MiB memset between steps; "
+                   "inputs (134 MB per tensor) and workspace (>1 GB) larger than L2",
+                   "parallelism": "independent replicas, no collective" if world > 1 else "single GPU",
+                   "useful_flops": "fwd 4*d, bwd 10*d per visible (query,key) pair"},
+        "fwd": {"ms": fwd_ms, "tflops": fwd_tflops, "frac_of_measured_burst": fwd_tflops / burst,
+                "frac_of_measured_sustained": fwd_tflops / sustained, "frac_of_nominal": fwd_tflops / NOMINAL_BF16_TFLOPS},
+        "bwd": {"ms": bwd_ms, "tflops": bwd_tflops, "frac_of_measured_burst": bwd_tflops / burst},
+        "tau_search_extra": {"tensor_flops": 0, "note": "single score sweep: the threshold is solved on the per-row "
+                             "candidate lists, no extra QK^T pass", "dense_fallback_rows": dense_rows},
+        "roofline": {"bound": "tensor", "kernel": "sweep_kernel<128> (forward score sweep)", "achieved": sweep_tflops,
+                     "peak": burst, "unit": "TFLOP/s", "frac": sweep_tflops / burst, "peak_source": peak_kind + " burst",
+                     "frac_of_sustained": sweep_tflops / sustained, "ms_per_launch": sweep_ms,
+                     "algorithmic_flops_per_launch": sweep_flops, "traffic": SWEEP_DRAM_TRAFFIC_BYTES},
+        "e2e": {"value": flops_all / (e2e_ms_all * 1e-3) / 1e12, "unit": UNIT, "ms_per_step": e2e_ms_all,
+                "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h},
+        "gpu_launches": 10 * K,
+        "clocks": clocks,
+    }
+    if world == 1 and not args.no_cpu_baseline:
+        line["cpu_baseline"] = cpu_baseline(inp, w, alpha, budget_s=args.cpu_seconds)
+    print(json.dumps(line), flush=True)
+
+
+def _oracle_pass(inp, w, alpha, rows_per_head: int, seed: int):
+    """Oracle forward rows + row-local backward (dQ) rows on `rows_per_head` sampled rows of every head.
+    Returns (seconds, useful FLOPs of those rows, number of rows)."""
+    import oracle
+    flops = 0
+    nrows = 0
+    t0 = time.perf_counter()
+    for bh in range(w.B * w.H):
+        b, h = divmod(bh, w.H)
+        rows = sample_rows(inp, bh, rows_per_head, seed=seed)
+        q, k, v, g = (t[b, h].float().numpy() for t in (inp.q, inp.k, inp.v, inp.d_o))
+        oracle.attn_fwd_rows(q, k, v, rows, alpha, inp.sm_scale, w.causal, scale=inp.head_scale(h))
+        oracle.attn_bwd_rows(q, k, v, g, rows, alpha, inp.sm_scale, w.causal, scale=inp.head_scale(h))
+        vis = (rows + 1) if w.causal else np.full_like(rows, w.N)
+        flops += int(vis.sum()) * 14 * w.d
+        nrows += len(rows)
+    return time.perf_counter() - t0, flops, nrows
+
+
+def cpu_baseline(inp, w, alpha, budget_s: float = 12.0):
+    """The fp64 oracle, as it stands, on the host cores of this machine, on a bounded row sample of the same
+    workload (a pilot sizes the sample for about `budget_s` seconds)."""
+    import oracle
+    pilot_s, _, pilot_rows = _oracle_pass(inp, w, alpha, 8, seed=1)
+    per_row = max(pilot_s / pilot_rows, 1e-6)
+    rows_per_head = int(max(8, min(w.N, budget_s / per_row / (w.B * w.H))))
+    secs, flops, nrows = _oracle_pass(inp, w, alpha, rows_per_head, seed=2)
+    return {"value": flops / secs / 1e12, "unit": UNIT, "cores": oracle.num_threads(), "kind": "oracle",
+            "sample": "%d sampled query rows (%d per head) of the same workload: oracle forward rows plus the "
+                      "row-local backward (dQ) rows, %.1f s; useful FLOPs of those rows / time" % (nrows, rows_per_head, secs),
+            "rows_per_s": nrows / secs, "extrapolated_full_step_s": (w.B * w.H * w.N) * secs / nrows}
+
+
+def run_reference(args):
+    """The reference arm: the CPU oracle itself, timed on the host cores (rank 0 only)."""
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    import oracle
+    w, inp = make_bench_inputs(args.alpha)
+    pilot_s, _, pilot_rows = _oracle_pass(inp, w, args.alpha, 8, seed=1)
+    per_row = max(pilot_s / pilot_rows, 1e-6)
+    total_budget = 90.0
+    steps = args.steps + max(args.warmup, 1)
+    rows_per_head = int(max(4, min(w.N, total_budget / steps / per_row / (w.B * w.H))))
+    for i in range(max(args.warmup, 1)):
+        _oracle_pass(inp, w, args.alpha, rows_per_head, seed=10 + i)
+    secs = flops = nrows = 0
+    for i in range(args.steps):
+        s, f, n = _oracle_pass(inp, w, args.alpha, rows_per_head, seed=100 + i)
+        secs, flops, nrows = secs + s, flops + f, nrows + n
+    value = flops / secs / 1e12
+    sample = "each step = %d sampled query rows per head (oracle forward + row-local backward)" % rows_per_head
+    line = {"impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": int(os.environ.get("WORLD_SIZE", "1")),
+            "steps": args.steps, "warmup": max(args.warmup, 1), "ms_per_step": secs / args.steps * 1e3,
+            "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+            "config": {"workload": w.name, "batch": w.B, "heads": w.H, "seq": w.N, "head_dim": w.d, "causal": w.causal,
+                       "alpha": args.alpha, "step": sample},
+            "cpu_baseline": {"value": value, "unit": UNIT, "cores": oracle.num_threads(), "kind": "oracle", "sample": sample},
+            "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+            "gpu_launches": 0}
+    print(json.dumps(line), flush=True)
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=10)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--impl", choices=["ours", "reference"], default="ours")
+    ap.add_argument("--alpha", type=float, default=1.5)
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--cpu-seconds", type=float, default=12.0)
+    args = ap.parse_args()
+    if args.impl == "reference":
+        run_reference(args)
+    else:
+        run_ours(args)
+    if int(os.environ.get("WORLD_SIZE", "1")) > 1:
+        import torch.distributed as dist
+        if dist.is_initialized():
+            dist.destroy_process_group()
+
+
+if __name__ == "__main__":
+    main()

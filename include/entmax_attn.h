@@ -131,6 +131,13 @@ int entmax_attn_scores_debug(const entmax_attn_params* params, const void* q, co
                              int32_t bh, float* s_out, void* workspace, size_t workspace_bytes,
                              int32_t* device_status, void* cuda_stream);
 
+/* Timing hook for benchmarks: after this call, every entmax_attn_fwd (which = 0) or entmax_attn_bwd
+ * (which = 1) made by the calling thread records `start_event` immediately before and `stop_event`
+ * immediately after its score-sweep kernel (bf16 problems), on that call's stream.  Both are
+ * cudaEvent_t passed as void*; pass NULL for both to switch the hook off.  The events stay owned by
+ * the caller.  No paper counterpart. */
+int entmax_attn_profile_events(int which, void* start_event, void* stop_event);
+
 /* Text for a status code (static storage). */
 const char* entmax_attn_strerror(int code);
 

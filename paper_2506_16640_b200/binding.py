@@ -61,6 +61,8 @@ def load():
         lib.entmax_attn_bwd.argtypes = [pp, vp, vp, vp, fp, fp, fp, fp, vp, vp, vp, vp, vp, ctypes.c_size_t, ip, vp]
         lib.entmax_attn_scores_debug.restype = ctypes.c_int
         lib.entmax_attn_scores_debug.argtypes = [pp, vp, vp, ctypes.c_int32, fp, vp, ctypes.c_size_t, ip, vp]
+        lib.entmax_attn_profile_events.restype = ctypes.c_int
+        lib.entmax_attn_profile_events.argtypes = [ctypes.c_int, vp, vp]
         lib.entmax_attn_strerror.restype = ctypes.c_char_p
         lib.entmax_attn_strerror.argtypes = [ctypes.c_int]
         lib.entmax_attn_last_cuda_error.restype = ctypes.c_int
@@ -180,6 +182,15 @@ def entmax_attn_scores_debug(q, k, bh, causal, *, workspace=None, status=None, s
                                          workspace.numel(), _ptr(status), _stream_ptr(stream))
     _check(rc, "entmax_attn_scores_debug")
     return out
+
+
+def entmax_attn_profile_events(which: int, start: Optional[torch.cuda.Event], stop: Optional[torch.cuda.Event]):
+    """Record `start`/`stop` around the score-sweep kernel of later forward (which=0) or backward (which=1)
+    calls of this thread; None, None switches the hook off.  The events must have been created with
+    enable_timing=True and recorded once (so that their CUDA handles exist)."""
+    a = None if start is None else ctypes.c_void_p(start.cuda_event)
+    b = None if stop is None else ctypes.c_void_p(stop.cuda_event)
+    _check(load().entmax_attn_profile_events(int(which), a, b), "entmax_attn_profile_events")
 
 
 def read_support(params: Params, workspace: torch.Tensor, rows):

@@ -10,6 +10,8 @@ namespace entmax {
 namespace {
 
 thread_local int g_last_cuda_error = 0;
+thread_local cudaEvent_t g_prof_start[2] = {nullptr, nullptr};
+thread_local cudaEvent_t g_prof_stop[2] = {nullptr, nullptr};
 
 inline size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
 
@@ -169,8 +171,10 @@ int entmax_attn_fwd(const entmax_attn_params* params, const void* q, const void*
   }
   err = cudaMemsetAsync(fb_count, 0, sizeof(int32_t), stream);
   if (err != cudaSuccess) return fail_cuda(err);
+  if (g_prof_start[0]) cudaEventRecord(g_prof_start[0], stream);
   err = launch_sweep(p, q, k, scale, nullptr, 0, row_cnt, row_thr, entries, nullptr, -1, device_status, stream);
   if (err != cudaSuccess) return fail_cuda(err);
+  if (g_prof_stop[0]) cudaEventRecord(g_prof_stop[0], stream);
   err = launch_row_fwd(p, v, scale, row_cnt, row_thr, entries, o, tau, fb_count, fb_list, device_status, stream);
   if (err != cudaSuccess) return fail_cuda(err);
   err = launch_dense_fwd(p, q, k, v, scale, o, tau, row_cnt, entries, fb_list, fb_count, scratch, lay.scratch_floats,
@@ -228,8 +232,10 @@ int entmax_attn_bwd(const entmax_attn_params* params, const void* q, const void*
   } else {
     err = cudaMemsetAsync(fb_count, 0, sizeof(int32_t), stream);
     if (err != cudaSuccess) return fail_cuda(err);
+    if (g_prof_start[1]) cudaEventRecord(g_prof_start[1], stream);
     err = launch_sweep(p, q, k, scale, tau, 1, row_cnt, row_thr, entries, nullptr, -1, device_status, stream);
     if (err != cudaSuccess) return fail_cuda(err);
+    if (g_prof_stop[1]) cudaEventRecord(g_prof_stop[1], stream);
     err = launch_row_bwd(p, q, k, v, d_o, scale, tau, row_cnt, entries, dq, acc_dk, acc_dv, fb_count, fb_list,
                          device_status, stream);
     if (err != cudaSuccess) return fail_cuda(err);
@@ -272,6 +278,14 @@ int entmax_attn_scores_debug(const entmax_attn_params* params, const void* q, co
                      reinterpret_cast<float*>(ws + lay.row_thr), reinterpret_cast<Entry*>(ws + lay.entries), s_out, bh,
                      device_status, stream);
   return err == cudaSuccess ? ENTMAX_ATTN_OK : fail_cuda(err);
+}
+
+int entmax_attn_profile_events(int which, void* start_event, void* stop_event) {
+  if (which != 0 && which != 1) return ENTMAX_ATTN_EINVAL_SHAPE;
+  if ((start_event == nullptr) != (stop_event == nullptr)) return ENTMAX_ATTN_EINVAL_NULL;
+  g_prof_start[which] = static_cast<cudaEvent_t>(start_event);
+  g_prof_stop[which] = static_cast<cudaEvent_t>(stop_event);
+  return ENTMAX_ATTN_OK;
 }
 
 const char* entmax_attn_strerror(int code) {
