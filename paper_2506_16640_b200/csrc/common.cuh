@@ -10,9 +10,15 @@
 
 namespace entmax {
 
-// Sparse row list: capacity per row and the fill level above which a row is handed to the dense path.
-constexpr int kListCap = 128;
-constexpr int kListKeep = 96;
+// Sparse row lists.  The score sweep splits the keys of a row between two threads; each owns one half
+// of the row's kListCap list slots: capacity kHalfCap, the fill level at which the sweep tightens the
+// threshold and filters the half-list (checked after every 8 keys, so the capacity is never exceeded),
+// and the length a filtered half-list may keep -- a row that cannot be brought down to it is handed to
+// the dense path.  The row kernels merge the two halves and leave the support compacted from slot 0.
+constexpr int kHalfCap = 64;
+constexpr int kHalfTrigger = 40;
+constexpr int kHalfKeep = 32;
+constexpr int kListCap = 2 * kHalfCap;
 
 // One list slot: y = (alpha-1) * s_ij (or the raw accumulator while a sweep is running), j = key index.
 struct __align__(8) Entry {
@@ -35,7 +41,7 @@ struct Problem {
 };
 
 struct WsLayout {
-  size_t scale, row_cnt, row_thr, entries, fb_count, fb_list, scratch, acc_dk, acc_dv, total;
+  size_t scale, row_cnt, half_cnt, half_thr, entries, fb_count, sweep_counter, fb_list, scratch, acc_dk, acc_dv, total;
   int scratch_ctas;     // CTAs of the dense-row kernels (each owns scratch_floats floats)
   size_t scratch_floats;
 };
@@ -67,15 +73,15 @@ cudaError_t launch_dense_bwd(const Problem& p, const void* q, const void* k, con
 // tcgen05 score sweep (bf16): fills the per-row candidate lists.
 //   mode 0: threshold search (forward); mode 1: threshold given in tau_in (backward)
 cudaError_t launch_sweep(const Problem& p, const void* q, const void* k, const float* scale, const float* tau_in,
-                         int mode, int32_t* row_cnt, float* row_thr, Entry* entries, float* dump, int dump_bh,
-                         int32_t* status, cudaStream_t stream);
+                         int mode, int32_t* half_cnt, float* half_thr, Entry* entries, int32_t* work_counter,
+                         float* dump, int dump_bh, int32_t* status, cudaStream_t stream);
 
 // per-row solve + gather kernels working on the lists (bf16 path)
 cudaError_t launch_row_fwd(const Problem& p, const void* v, const float* scale, int32_t* row_cnt,
-                           const float* row_thr, Entry* entries, void* o, float* tau, int32_t* fb_count,
+                           const int32_t* half_cnt, const float* half_thr, Entry* entries, void* o, float* tau, int32_t* fb_count,
                            int32_t* fb_list, int32_t* status, cudaStream_t stream);
 cudaError_t launch_row_bwd(const Problem& p, const void* q, const void* k, const void* v, const void* d_o,
-                           const float* scale, const float* tau, int32_t* row_cnt, Entry* entries, void* dq,
+                           const float* scale, const float* tau, const int32_t* half_cnt, Entry* entries, void* dq,
                            float* acc_dk, float* acc_dv, int32_t* fb_count, int32_t* fb_list, int32_t* status,
                            cudaStream_t stream);
 

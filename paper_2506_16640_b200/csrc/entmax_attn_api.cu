@@ -86,9 +86,11 @@ WsLayout make_layout(const Problem& p, bool is_bwd) {
   auto take = [&off](size_t bytes) { size_t at = off; off = align_up(off + bytes, 256); return at; };
   l.scale = take((size_t)p.H * p.N * sizeof(float));
   l.row_cnt = take(rows * sizeof(int32_t));
-  l.row_thr = take(rows * sizeof(float));
+  l.half_cnt = take(rows * 2 * sizeof(int32_t));
+  l.half_thr = take(rows * 2 * sizeof(float));
   l.entries = take(rows * kListCap * sizeof(Entry));
   l.fb_count = take(256);
+  l.sweep_counter = l.fb_count + 64;   // same 256-byte block: [0] dense-row count, [16] sweep work counter
   l.fb_list = take(rows * sizeof(int32_t));
   // dense-row CTAs: enough to fill the machine, few enough that their score rows stay modest
   l.scratch_floats = align_up((size_t)p.N, 32) * (is_bwd ? 2 : 1);   // scores (+ dP in backward)
@@ -152,7 +154,9 @@ int entmax_attn_fwd(const entmax_attn_params* params, const void* q, const void*
   uint8_t* ws = static_cast<uint8_t*>(workspace);
   float* scale = reinterpret_cast<float*>(ws + lay.scale);
   int32_t* row_cnt = reinterpret_cast<int32_t*>(ws + lay.row_cnt);
-  float* row_thr = reinterpret_cast<float*>(ws + lay.row_thr);
+  int32_t* half_cnt = reinterpret_cast<int32_t*>(ws + lay.half_cnt);
+  float* half_thr = reinterpret_cast<float*>(ws + lay.half_thr);
+  int32_t* sweep_counter = reinterpret_cast<int32_t*>(ws + lay.sweep_counter);
   Entry* entries = reinterpret_cast<Entry*>(ws + lay.entries);
   int32_t* fb_count = reinterpret_cast<int32_t*>(ws + lay.fb_count);
   int32_t* fb_list = reinterpret_cast<int32_t*>(ws + lay.fb_list);
@@ -172,10 +176,11 @@ int entmax_attn_fwd(const entmax_attn_params* params, const void* q, const void*
   err = cudaMemsetAsync(fb_count, 0, sizeof(int32_t), stream);
   if (err != cudaSuccess) return fail_cuda(err);
   if (g_prof_start[0]) cudaEventRecord(g_prof_start[0], stream);
-  err = launch_sweep(p, q, k, scale, nullptr, 0, row_cnt, row_thr, entries, nullptr, -1, device_status, stream);
+  err = launch_sweep(p, q, k, scale, nullptr, 0, half_cnt, half_thr, entries, sweep_counter, nullptr, -1, device_status,
+                     stream);
   if (err != cudaSuccess) return fail_cuda(err);
   if (g_prof_stop[0]) cudaEventRecord(g_prof_stop[0], stream);
-  err = launch_row_fwd(p, v, scale, row_cnt, row_thr, entries, o, tau, fb_count, fb_list, device_status, stream);
+  err = launch_row_fwd(p, v, scale, row_cnt, half_cnt, half_thr, entries, o, tau, fb_count, fb_list, device_status, stream);
   if (err != cudaSuccess) return fail_cuda(err);
   err = launch_dense_fwd(p, q, k, v, scale, o, tau, row_cnt, entries, fb_list, fb_count, scratch, lay.scratch_floats,
                          lay.scratch_ctas, stream);
@@ -205,8 +210,9 @@ int entmax_attn_bwd(const entmax_attn_params* params, const void* q, const void*
   cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
   uint8_t* ws = static_cast<uint8_t*>(workspace);
   float* scale = reinterpret_cast<float*>(ws + lay.scale);
-  int32_t* row_cnt = reinterpret_cast<int32_t*>(ws + lay.row_cnt);
-  float* row_thr = reinterpret_cast<float*>(ws + lay.row_thr);
+  int32_t* half_cnt = reinterpret_cast<int32_t*>(ws + lay.half_cnt);
+  float* half_thr = reinterpret_cast<float*>(ws + lay.half_thr);
+  int32_t* sweep_counter = reinterpret_cast<int32_t*>(ws + lay.sweep_counter);
   Entry* entries = reinterpret_cast<Entry*>(ws + lay.entries);
   int32_t* fb_count = reinterpret_cast<int32_t*>(ws + lay.fb_count);
   int32_t* fb_list = reinterpret_cast<int32_t*>(ws + lay.fb_list);
@@ -233,10 +239,11 @@ int entmax_attn_bwd(const entmax_attn_params* params, const void* q, const void*
     err = cudaMemsetAsync(fb_count, 0, sizeof(int32_t), stream);
     if (err != cudaSuccess) return fail_cuda(err);
     if (g_prof_start[1]) cudaEventRecord(g_prof_start[1], stream);
-    err = launch_sweep(p, q, k, scale, tau, 1, row_cnt, row_thr, entries, nullptr, -1, device_status, stream);
+    err = launch_sweep(p, q, k, scale, tau, 1, half_cnt, half_thr, entries, sweep_counter, nullptr, -1, device_status,
+                       stream);
     if (err != cudaSuccess) return fail_cuda(err);
     if (g_prof_stop[1]) cudaEventRecord(g_prof_stop[1], stream);
-    err = launch_row_bwd(p, q, k, v, d_o, scale, tau, row_cnt, entries, dq, acc_dk, acc_dv, fb_count, fb_list,
+    err = launch_row_bwd(p, q, k, v, d_o, scale, tau, half_cnt, entries, dq, acc_dk, acc_dv, fb_count, fb_list,
                          device_status, stream);
     if (err != cudaSuccess) return fail_cuda(err);
     err = launch_dense_bwd(p, q, k, v, d_o, scale, tau, dq, acc_dk, acc_dv, fb_list, fb_count, scratch,
@@ -274,9 +281,9 @@ int entmax_attn_scores_debug(const entmax_attn_params* params, const void* q, co
   }
   err = launch_scale_table(p, nullptr, nullptr, nullptr, scale, device_status, stream);
   if (err != cudaSuccess) return fail_cuda(err);
-  err = launch_sweep(p, q, k, scale, nullptr, 0, reinterpret_cast<int32_t*>(ws + lay.row_cnt),
-                     reinterpret_cast<float*>(ws + lay.row_thr), reinterpret_cast<Entry*>(ws + lay.entries), s_out, bh,
-                     device_status, stream);
+  err = launch_sweep(p, q, k, scale, nullptr, 0, reinterpret_cast<int32_t*>(ws + lay.half_cnt),
+                     reinterpret_cast<float*>(ws + lay.half_thr), reinterpret_cast<Entry*>(ws + lay.entries),
+                     reinterpret_cast<int32_t*>(ws + lay.sweep_counter), s_out, bh, device_status, stream);
   return err == cudaSuccess ? ENTMAX_ATTN_OK : fail_cuda(err);
 }
 

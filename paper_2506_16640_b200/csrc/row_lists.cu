@@ -1,5 +1,5 @@
 // Per-row kernels of the bf16 path that work on the sparse candidate lists left by the tensor-core
-// score sweep: one warp per query row.
+// score sweep (two half-lists per row, see common.cuh): one warp per query row.
 //
 // Forward: exact threshold on the candidates (Eq. 1 with the sum-to-one condition; Newton from the
 // left of the root, see dense_rows.cu), probabilities, and O_i = sum_j p_ij v_j as a gather over the
@@ -68,7 +68,8 @@ template <int D>
 __global__ void __launch_bounds__(kWarpsPerCta * 32) row_fwd_kernel(Problem p, const __nv_bfloat16* __restrict__ v,
                                                                     const float* __restrict__ scale,
                                                                     int32_t* __restrict__ row_cnt,
-                                                                    const float* __restrict__ row_thr,
+                                                                    const int32_t* __restrict__ half_cnt,
+                                                                    const float* __restrict__ half_thr,
                                                                     Entry* __restrict__ entries,
                                                                     __nv_bfloat16* __restrict__ o,
                                                                     float* __restrict__ tau_out, int32_t* fb_count,
@@ -77,9 +78,12 @@ __global__ void __launch_bounds__(kWarpsPerCta * 32) row_fwd_kernel(Problem p, c
   const int lane = threadIdx.x & 31;
   const int total = p.B * p.H * p.N;
   for (int grow = blockIdx.x * kWarpsPerCta + (threadIdx.x >> 5); grow < total; grow += gridDim.x * kWarpsPerCta) {
-    const int cnt = row_cnt[grow];
-    if (cnt <= 0) {
-      if (lane == 0) push_dense_row(grow, fb_count, fb_list, status);
+    const int c0 = half_cnt[2 * (size_t)grow], c1 = half_cnt[2 * (size_t)grow + 1];
+    if (c0 < 0 || c1 < 0 || c0 + c1 == 0) {
+      if (lane == 0) {
+        row_cnt[grow] = -2;
+        push_dense_row(grow, fb_count, fb_list, status);
+      }
       continue;
     }
     const int bh = grow / p.N, i = grow - bh * p.N, b = bh / p.H, h = bh - b * p.H;
@@ -90,10 +94,10 @@ __global__ void __launch_bounds__(kWarpsPerCta * 32) row_fwd_kernel(Problem p, c
     float ymax = -INFINITY;
 #pragma unroll
     for (int s = 0; s < kSlots; ++s) {
-      const int idx = lane + 32 * s;
+      const int idx = lane + 32 * s;                 // slot; half idx / kHalfCap owns it
       y[s] = -INFINITY;
       jj[s] = 0;
-      if (idx < cnt) {
+      if ((idx & (kHalfCap - 1)) < (idx < kHalfCap ? c0 : c1)) {
         const Entry e = list[idx];
         y[s] = a * e.y;
         jj[s] = e.j;
@@ -101,7 +105,9 @@ __global__ void __launch_bounds__(kWarpsPerCta * 32) row_fwd_kernel(Problem p, c
       ymax = fmaxf(ymax, y[s]);
     }
     ymax = warp_max(ymax);
-    float tau = fmaxf(row_thr[grow], ymax - 1.0f);
+    // both half-row bounds and the bracket's lower end are lower bounds on the threshold
+    float tau = fmaxf(fmaxf(half_thr[2 * (size_t)grow], half_thr[2 * (size_t)grow + 1]), ymax - 1.0f);
+    __syncwarp();   // every slot is in registers before the compaction below overwrites the list
     for (int it = 0; it < kMaxNewton; ++it) {
       float s0 = 0.f, s1 = 0.f;
 #pragma unroll
@@ -167,15 +173,15 @@ template <int D>
 __global__ void __launch_bounds__(kWarpsPerCta * 32) row_bwd_kernel(
     Problem p, const __nv_bfloat16* __restrict__ q, const __nv_bfloat16* __restrict__ k,
     const __nv_bfloat16* __restrict__ v, const __nv_bfloat16* __restrict__ d_o, const float* __restrict__ scale,
-    const float* __restrict__ tau_in, const int32_t* __restrict__ row_cnt, const Entry* __restrict__ entries,
+    const float* __restrict__ tau_in, const int32_t* __restrict__ half_cnt, const Entry* __restrict__ entries,
     __nv_bfloat16* __restrict__ dq, float* __restrict__ acc_dk, float* __restrict__ acc_dv, int32_t* fb_count,
     int32_t* fb_list, int32_t* status) {
   constexpr int PER = D / 32;
   const int lane = threadIdx.x & 31;
   const int total = p.B * p.H * p.N;
   for (int grow = blockIdx.x * kWarpsPerCta + (threadIdx.x >> 5); grow < total; grow += gridDim.x * kWarpsPerCta) {
-    const int cnt = row_cnt[grow];
-    if (cnt < 0) {
+    const int c0 = half_cnt[2 * (size_t)grow], c1 = half_cnt[2 * (size_t)grow + 1];
+    if (c0 < 0 || c1 < 0) {
       if (lane == 0) push_dense_row(grow, fb_count, fb_list, status);
       continue;
     }
@@ -196,7 +202,7 @@ __global__ void __launch_bounds__(kWarpsPerCta * 32) row_bwd_kernel(
       yv[s] = -1.0f;
       jj[s] = 0;
       dpv[s] = 0.f;
-      if (idx < cnt) {
+      if ((idx & (kHalfCap - 1)) < (idx < kHalfCap ? c0 : c1)) {
         const Entry e = list[idx];
         yv[s] = fmaf(a, e.y, -tau);
         jj[s] = e.j;
@@ -272,31 +278,31 @@ inline int row_grid(const Problem& p) {
 }  // namespace
 
 cudaError_t launch_row_fwd(const Problem& p, const void* v, const float* scale, int32_t* row_cnt,
-                           const float* row_thr, Entry* entries, void* o, float* tau, int32_t* fb_count,
-                           int32_t* fb_list, int32_t* status, cudaStream_t stream) {
+                           const int32_t* half_cnt, const float* half_thr, Entry* entries, void* o, float* tau,
+                           int32_t* fb_count, int32_t* fb_list, int32_t* status, cudaStream_t stream) {
   const int grid = row_grid(p);
   if (p.D == 64)
-    row_fwd_kernel<64><<<grid, kWarpsPerCta * 32, 0, stream>>>(p, (const __nv_bfloat16*)v, scale, row_cnt, row_thr,
+    row_fwd_kernel<64><<<grid, kWarpsPerCta * 32, 0, stream>>>(p, (const __nv_bfloat16*)v, scale, row_cnt, half_cnt, half_thr,
                                                               entries, (__nv_bfloat16*)o, tau, fb_count, fb_list, status);
   else
-    row_fwd_kernel<128><<<grid, kWarpsPerCta * 32, 0, stream>>>(p, (const __nv_bfloat16*)v, scale, row_cnt, row_thr,
+    row_fwd_kernel<128><<<grid, kWarpsPerCta * 32, 0, stream>>>(p, (const __nv_bfloat16*)v, scale, row_cnt, half_cnt, half_thr,
                                                                entries, (__nv_bfloat16*)o, tau, fb_count, fb_list, status);
   return cudaGetLastError();
 }
 
 cudaError_t launch_row_bwd(const Problem& p, const void* q, const void* k, const void* v, const void* d_o,
-                           const float* scale, const float* tau, int32_t* row_cnt, Entry* entries, void* dq,
+                           const float* scale, const float* tau, const int32_t* half_cnt, Entry* entries, void* dq,
                            float* acc_dk, float* acc_dv, int32_t* fb_count, int32_t* fb_list, int32_t* status,
                            cudaStream_t stream) {
   const int grid = row_grid(p);
   if (p.D == 64)
     row_bwd_kernel<64><<<grid, kWarpsPerCta * 32, 0, stream>>>(
         p, (const __nv_bfloat16*)q, (const __nv_bfloat16*)k, (const __nv_bfloat16*)v, (const __nv_bfloat16*)d_o, scale,
-        tau, row_cnt, entries, (__nv_bfloat16*)dq, acc_dk, acc_dv, fb_count, fb_list, status);
+        tau, half_cnt, entries, (__nv_bfloat16*)dq, acc_dk, acc_dv, fb_count, fb_list, status);
   else
     row_bwd_kernel<128><<<grid, kWarpsPerCta * 32, 0, stream>>>(
         p, (const __nv_bfloat16*)q, (const __nv_bfloat16*)k, (const __nv_bfloat16*)v, (const __nv_bfloat16*)d_o, scale,
-        tau, row_cnt, entries, (__nv_bfloat16*)dq, acc_dk, acc_dv, fb_count, fb_list, status);
+        tau, half_cnt, entries, (__nv_bfloat16*)dq, acc_dk, acc_dv, fb_count, fb_list, status);
   return cudaGetLastError();
 }
 

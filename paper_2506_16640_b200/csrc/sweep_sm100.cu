@@ -1,24 +1,32 @@
 // Score sweep for bf16 problems on sm_100a: S = Q K^T on tcgen05 tensor cores (bf16 in, fp32
 // accumulators in TMEM, Q and K tiles staged by TMA without multicast), one pass over the keys of
-// every query row, leaving a short per-row candidate list that provably contains the support of
+// every query row, leaving short per-row candidate lists that provably contain the support of
 // Eq. 1.
 //
 // Why one pass is enough.  Write y_j = (alpha-1) s_ij and f(tau) = sum_j [y_j - tau]_+^e - 1, e = 1/(alpha-1).
 //  (1) p_max <= 1 gives tau >= y_max - 1 (lower end of the bracket of App. A), and
-//  (2) the threshold of a prefix of the row never exceeds the threshold of the whole row (adding a
-//      logit never lowers tau), while keys at or below the threshold do not change it.
-// So while the keys stream by, each row keeps a lower bound thr on its final tau and the list of keys
-// seen so far with y > thr.  When the list fills up, a few Newton steps on the listed keys, started
-// at thr, raise thr (f is convex and decreasing for e >= 1, so Newton from the left of the root never
-// passes it) and the list is filtered.  A row whose list cannot be kept below kListKeep entries is
-// flagged and later recomputed by the dense-row path.  In backward mode the threshold is the tau of
-// the forward pass and the list is simply the support.
+//  (2) the threshold of a subset of the row's keys never exceeds the threshold of the whole row (adding
+//      a logit never lowers tau), while keys at or below the threshold do not change it.
+// So while the keys stream by, a thread keeps a lower bound thr on the row's final tau and the list of
+// the keys it has seen with y > thr.  When a list grows past kHalfTrigger entries, Newton steps on the
+// listed keys, started at thr, raise thr (f is convex and decreasing for e >= 1, so Newton from the left
+// of the root never passes it) and the list is filtered.  A row whose list cannot be brought down to
+// kHalfKeep entries is flagged and later recomputed by the dense-row path.  In backward mode the
+// threshold is the tau of the forward pass and the lists are simply the support.
 //
-// CTA layout (320 threads, one CTA per SM, persistent over work units):
-//   warp 0        TMA producer: Q tile pair (2 x 128 rows) once per item, K tiles of BN keys through a ring
-//   warp 1        MMA issuer: per K tile two M=128 x N=BN accumulations (one per Q tile) into TMEM
-//   warps 2..5    consumer group 0: TMEM lane = query row of Q tile 0, one thread per row
-//   warps 6..9    consumer group 1: same for Q tile 1
+// CTA layout (576 threads, one CTA per SM, persistent; work items of 2 x 128 query rows are handed out
+// longest-first through an atomic counter):
+//   warp 0        scheduler + TMA producer: the item's two Q tiles, K tiles of 256 keys through a ring
+//   warp 1        MMA issuer: per K tile one M=128 x N=256 accumulation per Q tile into its own 256
+//                 TMEM columns (2 accumulators = all 512 columns).  N = 256 keeps the operand traffic of
+//                 an MMA (A 4 KB + B 8 KB per 128 tensor-core cycles) below the shared-memory bandwidth.
+//   warps 2..17   consumers, eight warps per Q tile: TMEM lane = query row; the 256 columns of a row are
+//                 split between two threads (columns 0-127 and 128-255 of every K tile), each with its
+//                 own running maximum, threshold, list length (registers) and half-list; the two share
+//                 their running maxima through shared memory so that both thresholds stay tight.
+// A consumer first reduces its 128 columns to 16 group maxima (branch-free), and only when some lane of
+// the warp saw a value above its threshold re-reads the groups that hold candidates; then it hands the
+// accumulator back.  While the consumers of one Q tile scan, the tensor core works on the other.
 // Every mbarrier wait is bounded: on expiry the CTA raises ENTMAX_ATTN_FLAG_WAIT_EXPIRED, all roles
 // leave their loops, in-flight copies are given time to land, TMEM is freed and the CTA returns.
 #include <cuda.h>
@@ -30,12 +38,16 @@ namespace entmax {
 namespace {
 
 constexpr int BM = 128;          // query rows per Q tile = TMEM lanes
-constexpr int BN = 256;          // keys per K tile = N of one MMA
+constexpr int BN = 256;          // keys per K tile = N of one MMA = TMEM columns of one accumulator
+constexpr int kHalfCols = BN / 2;   // columns of a K tile one consumer thread scans
 constexpr int kQTiles = 2;       // Q tiles per item
 constexpr int kItemRows = BM * kQTiles;
-constexpr int kThreads = 320;
-constexpr int kTmemCols = 512;
+constexpr int kConsumerWarps = 8 * kQTiles;
+constexpr int kThreads = (2 + kConsumerWarps) * 32;
+constexpr int kTmemCols = kQTiles * BN;
+constexpr int kSchedSlots = 2;
 constexpr uint64_t kWaitLimitNs = 2000000000ull;  // 2 s
+static_assert(kTmemCols == 512 && kHalfCols == 128, "TMEM budget / consumer split");
 
 template <int HD>
 struct Cfg {
@@ -43,7 +55,9 @@ struct Cfg {
   static constexpr int kQBytes = BM * HD * 2;
   static constexpr int kKBytes = BN * HD * 2;
   static constexpr int kStages = HD == 128 ? 2 : 4;
-  static constexpr int kSmemBytes = kQTiles * kQBytes + kStages * kKBytes + 1024 /*align*/ + 256 /*barriers*/;
+  static constexpr int kShareBytes = kQTiles * 2 * BM * 8;   // running maxima shared by the two halves of a row
+  static constexpr int kBarBytes = 512;
+  static constexpr int kSmemBytes = kQTiles * kQBytes + kStages * kKBytes + kShareBytes + 1024 /*align*/ + kBarBytes;
 };
 
 struct SweepArgs {
@@ -56,15 +70,15 @@ struct SweepArgs {
   float sm_scale;
   const float* scale;   // [H, N]
   const float* tau_in;  // [B*H*N] (mode 1)
-  int32_t* row_cnt;
-  float* row_thr;
-  Entry* entries;
+  int32_t* half_cnt;    // [B*H*N][2] list length of each half-row; -1 = hand the row to the dense path
+  float* half_thr;      // [B*H*N][2] lower bound on tau each half-row ended with (Eq. 1's units)
+  Entry* entries;       // [B*H*N][kListCap]; half h of a row owns slots [h*kHalfCap, (h+1)*kHalfCap)
   float* dump;          // optional [N, N] raw accumulators of head dump_bh
   int dump_bh;
   int32_t* status;
+  int32_t* work_counter;  // zeroed before the launch
   int items_per_bh;     // ceil(N / kItemRows)
-  int units_per_bh;
-  int n_units;
+  int n_items;
 };
 
 // ------------------------------------------------------------------------------------------ PTX
@@ -98,8 +112,7 @@ __device__ __forceinline__ uint64_t global_ns() {
   return t;
 }
 // Bounded wait.  Returns false when the CTA is aborting (this or another wait ran out of time).
-__device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, volatile int* abort_flag) {
-  if (mbar_try_wait(bar, parity)) return true;
+__device__ __noinline__ bool mbar_wait_slow(uint64_t* bar, uint32_t parity, volatile int* abort_flag) {
   const uint64_t t0 = global_ns();
   uint32_t spins = 0;
   for (;;) {
@@ -112,6 +125,11 @@ __device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, volati
       }
     }
   }
+}
+__device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, volatile int* abort_flag) {
+  if (mbar_try_wait(bar, parity)) return true;
+  if (mbar_try_wait(bar, parity)) return true;
+  return mbar_wait_slow(bar, parity, abort_flag);
 }
 
 __device__ __forceinline__ void tma_load_4d(void* dst, const CUtensorMap* map, uint64_t* bar, int c0, int c1, int c2,
@@ -135,15 +153,20 @@ __device__ __forceinline__ void tmem_dealloc(uint32_t taddr, uint32_t ncols) {
 __device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
 __device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
 
-// D[tmem] (+)= A[smem] * B[smem]^T, bf16 x bf16 -> fp32, issued by one thread
-__device__ __forceinline__ void umma_bf16(uint32_t d_tmem, uint64_t adesc, uint64_t bdesc, uint32_t idesc,
+// D[tmem] (+)= A[smem] * B[smem]^T, bf16 x bf16 -> fp32, issued by one thread.  The two shared-memory
+// descriptors are passed as their low words (start address and leading-dimension field); the high word
+// is the same for every operand of this kernel.
+__device__ __forceinline__ void umma_bf16(uint32_t d_tmem, uint32_t a_lo, uint32_t b_lo, uint32_t desc_hi, uint32_t idesc,
                                           uint32_t accumulate) {
   asm volatile(
       "{\n"
       " .reg .pred p;\n"
-      " setp.ne.b32 p, %4, 0;\n"
-      " tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n"
-      "}\n" ::"r"(d_tmem), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate)
+      " .reg .b64 da, db;\n"
+      " mov.b64 da, {%1, %3};\n"
+      " mov.b64 db, {%2, %3};\n"
+      " setp.ne.b32 p, %5, 0;\n"
+      " tcgen05.mma.cta_group::1.kind::f16 [%0], da, db, %4, p;\n"
+      "}\n" ::"r"(d_tmem), "r"(a_lo), "r"(b_lo), "r"(desc_hi), "r"(idesc), "r"(accumulate)
       : "memory");
 }
 // mbarrier arrive once every MMA issued so far by this thread has completed
@@ -152,17 +175,22 @@ __device__ __forceinline__ void umma_commit(uint64_t* bar) {
                : "memory");
 }
 
-// 32 lanes x 32 consecutive fp32 columns: thread t of the warp gets lane (base + t)
-__device__ __forceinline__ void tmem_ld32(uint32_t taddr, float (&r)[32]) {
+// 32 lanes x 16 (or 8) consecutive fp32 columns: thread t of the warp gets lane (base + t)
+__device__ __forceinline__ void tmem_ld16(uint32_t taddr, float (&r)[16]) {
   uint32_t* u = reinterpret_cast<uint32_t*>(r);
   asm volatile(
-      "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
-      "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
-      "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];"
+      "tcgen05.ld.sync.aligned.32x32b.x16.b32 "
+      "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15}, [%16];"
       : "=r"(u[0]), "=r"(u[1]), "=r"(u[2]), "=r"(u[3]), "=r"(u[4]), "=r"(u[5]), "=r"(u[6]), "=r"(u[7]), "=r"(u[8]),
-        "=r"(u[9]), "=r"(u[10]), "=r"(u[11]), "=r"(u[12]), "=r"(u[13]), "=r"(u[14]), "=r"(u[15]), "=r"(u[16]),
-        "=r"(u[17]), "=r"(u[18]), "=r"(u[19]), "=r"(u[20]), "=r"(u[21]), "=r"(u[22]), "=r"(u[23]), "=r"(u[24]),
-        "=r"(u[25]), "=r"(u[26]), "=r"(u[27]), "=r"(u[28]), "=r"(u[29]), "=r"(u[30]), "=r"(u[31])
+        "=r"(u[9]), "=r"(u[10]), "=r"(u[11]), "=r"(u[12]), "=r"(u[13]), "=r"(u[14]), "=r"(u[15])
+      : "r"(taddr)
+      : "memory");
+}
+__device__ __forceinline__ void tmem_ld8(uint32_t taddr, float (&r)[8]) {
+  uint32_t* u = reinterpret_cast<uint32_t*>(r);
+  asm volatile(
+      "tcgen05.ld.sync.aligned.32x32b.x8.b32 {%0, %1, %2, %3, %4, %5, %6, %7}, [%8];"
+      : "=r"(u[0]), "=r"(u[1]), "=r"(u[2]), "=r"(u[3]), "=r"(u[4]), "=r"(u[5]), "=r"(u[6]), "=r"(u[7])
       : "r"(taddr)
       : "memory");
 }
@@ -170,15 +198,13 @@ __device__ __forceinline__ void tmem_ld_wait() { asm volatile("tcgen05.wait::ld.
 
 // Shared-memory matrix descriptor, K-major operand, 128-byte swizzle: rows are 128 bytes apart, groups
 // of 8 rows 1024 bytes apart (stride-dimension offset); descriptor version 1 (sm_100).
-__device__ __forceinline__ uint64_t smem_desc_sw128(uint32_t saddr) {
-  uint64_t d = 0;
-  d |= (uint64_t)((saddr & 0x3FFFFu) >> 4);
-  d |= (uint64_t)1 << 16;                 // leading-dimension offset: not used by swizzled K-major layouts
-  d |= (uint64_t)(1024 >> 4) << 32;       // stride-dimension offset
-  d |= (uint64_t)1 << 46;                 // descriptor version
-  d |= (uint64_t)2 << 61;                 // 128-byte swizzle
-  return d;
-}
+//   low word : bits 0-13 start address >> 4, bits 16-29 leading-dimension offset >> 4 (not used by
+//              swizzled K-major layouts; 1)
+//   high word: bits 0-13 stride-dimension offset >> 4, bit 14 descriptor version, bits 29-31 swizzle mode (2 = 128 B)
+// Advancing the operand by `bytes` inside the shared-memory window adds bytes >> 4 to the low word.
+constexpr uint32_t kDescHi = (1024u >> 4) | (1u << 14) | (2u << 29);
+__device__ __forceinline__ uint32_t smem_desc_lo(uint32_t saddr) { return ((saddr & 0x3FFFFu) >> 4) | (1u << 16); }
+
 // Instruction descriptor: fp32 accumulate, A and B bf16, both K-major, M = 128, N = BN
 __host__ __device__ constexpr uint32_t make_idesc() {
   return (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(BN >> 3) << 17) | ((uint32_t)(BM >> 4) << 24);
@@ -189,100 +215,114 @@ __device__ __forceinline__ float max3(float a, float b, float c) {
   asm("max.f32 %0, %1, %2, %3;" : "=f"(r) : "f"(a), "f"(b), "f"(c));
   return r;
 }
+__device__ __forceinline__ float max8(const float* v) {
+  const float x0 = max3(v[0], v[1], v[2]);
+  const float x1 = max3(v[3], v[4], v[5]);
+  return fmaxf(max3(x0, x1, v[6]), v[7]);
+}
+__device__ __forceinline__ float warp_sum(float x) {
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) x += __shfl_xor_sync(0xffffffffu, x, o);
+  return x;
+}
 
 // --------------------------------------------------------------------------------- work schedule
-// Unit u of head-pair bh: causal -> items (long, short) = (n-1-w, w) so that every unit costs the same;
-// non-causal -> one item.  Returns the number of items (1 or 2).
-__device__ __forceinline__ int unit_items(const SweepArgs& a, int unit, int& bh, int (&item)[2]) {
-  bh = unit / a.units_per_bh;
-  const int w = unit - bh * a.units_per_bh;
-  if (!a.causal) { item[0] = w; return 1; }
-  item[0] = a.items_per_bh - 1 - w;
-  item[1] = w;
-  return item[0] == item[1] ? 1 : 2;
+// Items are handed out in the order k = 0, 1, ...: head pair after head pair (so that the CTAs running at
+// the same time stream the same K tiles through L2) and, under the causal mask, the longest rows of a
+// head pair first.
+__device__ __forceinline__ void decode_item(const SweepArgs& a, int k, int& bh, int& item) {
+  bh = k / a.items_per_bh;
+  const int w = k - bh * a.items_per_bh;
+  item = a.causal ? a.items_per_bh - 1 - w : w;
 }
-__device__ __forceinline__ int item_tiles(const SweepArgs& a, int item) {
+// K tiles Q tile x of an item has to see (0 when the Q tile lies past the end of the sequence)
+__device__ __forceinline__ int qtile_tiles(const SweepArgs& a, int item, int x) {
+  const int row0 = item * kItemRows + x * BM;
+  if (row0 >= a.N) return 0;
   if (!a.causal) return (a.N + BN - 1) / BN;
-  int last_row = item * kItemRows + kItemRows - 1;
+  int last_row = row0 + BM - 1;
   if (last_row > a.N - 1) last_row = a.N - 1;
   return last_row / BN + 1;
 }
 
-// ------------------------------------------------------------------------------- per-row state
+// ------------------------------------------------------------- consumer side: one half-row per thread
 struct RowState {
-  float thr_acc;   // candidates are accumulators above this
-  float m_run;     // running maximum accumulator
-  float a, inv_a;  // y = a * acc
-  int cnt;         // list length; -1 = handed to the dense path
-  int lim;         // largest visible key index
-  Entry* list;
+  float thr;       // candidates are accumulators above this (accumulator units)
+  float m_run;     // running maximum accumulator (both halves of the row, as far as known)
+  int cnt;         // half-list length; -1 = handed to the dense path
 };
 
-__device__ __noinline__ void shrink_list(RowState& r, int mode, int expo_class, float expo) {
-  if (mode != 0) {  // threshold given: a full list means the support does not fit
-    r.cnt = -1;
-    r.thr_acc = INFINITY;
-    return;
-  }
-  float tau = r.thr_acc * r.a;
-  for (int it = 0; it < 3; ++it) {
-    float s0 = 0.f, s1 = 0.f;
-    for (int t = 0; t < r.cnt; ++t) {
-      const float y = fmaf(r.a, r.list[t].y, -tau);
-      if (y > 0.f) {
-        float ye, ye1;
-        pow_pair(y, expo_class, expo, ye, ye1);
-        s0 += ye;
-        s1 += ye1;
+// Warp-cooperative list shrink for the lanes whose half-list has grown past kHalfTrigger.  Accumulator
+// units are turned into Eq. 1's units with y = a * acc.  All 32 lanes must call this together.
+__device__ __noinline__ void shrink_lists(RowState& r, Entry* list, float a, float inv_a, unsigned need, int mode,
+                                          int expo_class, float expo) {
+  const int lane = threadIdx.x & 31;
+  constexpr int kSlots = kHalfCap / 32;
+  __syncwarp();   // the owner's list stores are ordered before the other lanes' loads
+  while (need) {
+    const int src = __ffs(need) - 1;
+    need &= need - 1;
+    Entry* l = reinterpret_cast<Entry*>(__shfl_sync(0xffffffffu, reinterpret_cast<unsigned long long>(list), src));
+    const int c = __shfl_sync(0xffffffffu, r.cnt, src);
+    const float th = __shfl_sync(0xffffffffu, r.thr, src);
+    const float aa = __shfl_sync(0xffffffffu, a, src);
+    const float inv_aa = __shfl_sync(0xffffffffu, inv_a, src);
+    float new_thr = INFINITY;
+    int kept = -1;
+    if (mode == 0) {
+      Entry e[kSlots];
+#pragma unroll
+      for (int s = 0; s < kSlots; ++s) {
+        const int idx = lane + 32 * s;
+        e[s].y = -INFINITY;
+        e[s].j = 0;
+        if (idx < c) e[s] = l[idx];
+      }
+      float tau = th * aa;
+      for (int it = 0; it < 8; ++it) {
+        float s0 = 0.f, s1 = 0.f;
+#pragma unroll
+        for (int s = 0; s < kSlots; ++s) {
+          const float y = fmaf(aa, e[s].y, -tau);
+          if (y > 0.f) {
+            float ye, ye1;
+            pow_pair(y, expo_class, expo, ye, ye1);
+            s0 += ye;
+            s1 += ye1;
+          }
+        }
+        s0 = warp_sum(s0);
+        s1 = warp_sum(s1);
+        if (!(s0 > 1.0f) || !(s1 > 0.f)) break;
+        const float step = (s0 - 1.0f) / (expo * s1);
+        tau += step;
+        if (step <= 1e-4f) break;
+      }
+      // a hair below the Newton iterate: rounding must never push the bound past the true threshold
+      new_thr = fmaxf(th, (tau - 4e-6f * fmaxf(1.0f, fabsf(tau))) * inv_aa);
+      __syncwarp();
+      kept = 0;
+#pragma unroll
+      for (int s = 0; s < kSlots; ++s) {
+        const bool keep = e[s].y > new_thr;
+        const unsigned m = __ballot_sync(0xffffffffu, keep);
+        if (keep) l[kept + __popc(m & ((1u << lane) - 1u))] = e[s];
+        kept += __popc(m);
+      }
+      if (kept > kHalfKeep) {
+        kept = -1;
+        new_thr = INFINITY;
       }
     }
-    if (!(s0 > 1.0f) || !(s1 > 0.f)) break;
-    tau += (s0 - 1.0f) / (expo * s1);
-  }
-  const float thr = fmaxf(r.thr_acc, tau * r.inv_a);
-  int kept = 0;
-  for (int t = 0; t < r.cnt; ++t) {
-    const Entry e = r.list[t];
-    if (e.y > thr) r.list[kept++] = e;
-  }
-  r.thr_acc = thr;
-  r.cnt = kept;
-  if (kept > kListKeep) {
-    r.cnt = -1;
-    r.thr_acc = INFINITY;
-  }
-}
-
-__device__ __forceinline__ void push(RowState& r, float acc, int j, int mode, int expo_class, float expo) {
-  r.list[r.cnt].y = acc;
-  r.list[r.cnt].j = j;
-  if (++r.cnt == kListCap) shrink_list(r, mode, expo_class, expo);
-}
-
-// One 32-column chunk of a score tile for this thread's row.
-template <bool kMasked>
-__device__ __forceinline__ void scan_chunk(float (&v)[32], int col0, RowState& r, int mode, int expo_class, float expo) {
-  if (kMasked) {
-#pragma unroll
-    for (int t = 0; t < 32; ++t) v[t] = (col0 + t <= r.lim) ? v[t] : -INFINITY;
-  }
-  float m = max3(v[0], v[1], v[2]);
-#pragma unroll
-  for (int t = 3; t < 31; t += 2) m = max3(m, v[t], v[t + 1]);
-  m = fmaxf(m, v[31]);
-  if (m > r.thr_acc) {
-    if (mode == 0) {
-      r.m_run = fmaxf(r.m_run, m);
-      r.thr_acc = fmaxf(r.thr_acc, r.m_run - r.inv_a);
-    }
-#pragma unroll
-    for (int t = 0; t < 32; ++t) {
-      if (v[t] > r.thr_acc) push(r, v[t], col0 + t, mode, expo_class, expo);
+    if (lane == src) {
+      r.cnt = kept;
+      r.thr = new_thr;
     }
   }
+  __syncwarp();
 }
 
-template <int HD>
+template <int HD, bool kDump>
 __global__ void __launch_bounds__(kThreads, 1) sweep_kernel(const __grid_constant__ CUtensorMap map_q,
                                                             const __grid_constant__ CUtensorMap map_k,
                                                             const SweepArgs a) {
@@ -291,34 +331,47 @@ __global__ void __launch_bounds__(kThreads, 1) sweep_kernel(const __grid_constan
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
   uint8_t* q_smem = smem;                                   // [kQTiles][kHalves][BM rows x 128 B]
   uint8_t* k_smem = smem + kQTiles * C::kQBytes;            // [kStages][kHalves][BN rows x 128 B]
-  uint64_t* bars = reinterpret_cast<uint64_t*>(k_smem + C::kStages * C::kKBytes);
-  uint64_t* q_full = bars;                  // [2]
-  uint64_t* q_empty = bars + 2;             // [2]
-  uint64_t* s_full = bars + 4;              // [2]
-  uint64_t* s_empty = bars + 6;             // [2]
-  uint64_t* k_full = bars + 8;              // [kStages]
-  uint64_t* k_empty = bars + 8 + C::kStages;
-  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 8 + 2 * C::kStages);
+  // running maximum of each half-row, tagged with the work item it belongs to: {item id, float bits}
+  volatile unsigned long long* m_share =
+      reinterpret_cast<volatile unsigned long long*>(k_smem + C::kStages * C::kKBytes);   // [kQTiles][2][BM]
+  uint64_t* bars = reinterpret_cast<uint64_t*>(k_smem + C::kStages * C::kKBytes + C::kShareBytes);
+  uint64_t* q_full = bars;                       // [kQTiles]
+  uint64_t* q_empty = q_full + kQTiles;          // [kQTiles]
+  uint64_t* s_full = q_empty + kQTiles;          // [kQTiles]
+  uint64_t* s_empty = s_full + kQTiles;          // [kQTiles]
+  uint64_t* k_full = s_empty + kQTiles;          // [kStages]
+  uint64_t* k_empty = k_full + C::kStages;       // [kStages]
+  uint64_t* w_full = k_empty + C::kStages;       // [kSchedSlots]
+  uint64_t* w_empty = w_full + kSchedSlots;      // [kSchedSlots]
+  volatile int* w_item = reinterpret_cast<volatile int*>(w_empty + kSchedSlots);   // [kSchedSlots]
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(const_cast<int*>(w_item) + kSchedSlots);
   volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
+  static_assert((4 * kQTiles + 2 * C::kStages + 2 * kSchedSlots) * 8 + kSchedSlots * 4 + 8 <= C::kBarBytes,
+                "barrier area");
 
   const int warp = threadIdx.x >> 5;
   const int lane = threadIdx.x & 31;
 
   if (threadIdx.x == 0) {
-    for (int t = 0; t < 2; ++t) {
+    for (int t = 0; t < kQTiles; ++t) {
       mbar_init(&q_full[t], 1);
       mbar_init(&q_empty[t], 1);
       mbar_init(&s_full[t], 1);
-      mbar_init(&s_empty[t], BM);
+      mbar_init(&s_empty[t], 8);                 // one arrival per consumer warp of the Q tile
     }
     for (int t = 0; t < C::kStages; ++t) {
       mbar_init(&k_full[t], 1);
       mbar_init(&k_empty[t], 1);
     }
+    for (int t = 0; t < kSchedSlots; ++t) {
+      mbar_init(&w_full[t], 1);
+      mbar_init(&w_empty[t], 1 + kConsumerWarps);   // MMA issuer + one arrival per consumer warp
+    }
     *abort_flag = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
   }
+  if (threadIdx.x < kQTiles * 2 * BM) m_share[threadIdx.x] = ~0ull;   // tag -1: belongs to no work item
   if (warp == 1) {
     tmem_alloc(tmem_slot, kTmemCols);
     tmem_relinquish();
@@ -329,34 +382,47 @@ __global__ void __launch_bounds__(kThreads, 1) sweep_kernel(const __grid_constan
   const uint32_t tmem_base = *tmem_slot;
 
   if (warp == 0) {
-    // ------------------------------------------------------------------ TMA producer
+    // ------------------------------------------------------------- scheduler + TMA producer
     if (lane == 0) {
-      int stage = 0;
-      uint32_t kphase = 0, qphase = 0;
+      int stage = 0, slot = 0;
+      uint32_t kphase = 0, qphase = 0 /* bit x: phase of Q tile slot x */, wphase = 0;
       bool alive = true;
-      for (int unit = blockIdx.x; unit < a.n_units && alive; unit += gridDim.x) {
-        int bh, item[2];
-        const int n_items = unit_items(a, unit, bh, item);
+      while (alive) {
+        alive = mbar_wait(&w_empty[slot], wphase ^ 1u, abort_flag);
+        if (!alive) break;
+        int k = atomicAdd(a.work_counter, 1);
+        if (k >= a.n_items) k = -1;
+        w_item[slot] = k;
+        mbar_arrive(&w_full[slot]);
+        if (++slot == kSchedSlots) { slot = 0; wphase ^= 1u; }
+        if (k < 0) break;
+        int bh, item;
+        decode_item(a, k, bh, item);
         const int b = bh / a.H, h = bh - b * a.H;
-        for (int s = 0; s < n_items && alive; ++s) {
-          const int tiles = item_tiles(a, item[s]);
-          for (int t = 0; t < tiles && alive; ++t) {
-            alive = mbar_wait(&k_empty[stage], kphase ^ 1u, abort_flag);
-            if (!alive) break;
-            mbar_expect_tx(&k_full[stage], C::kKBytes);
-            for (int hf = 0; hf < C::kHalves; ++hf)
-              tma_load_4d(k_smem + stage * C::kKBytes + hf * (BN * 128), &map_k, &k_full[stage], hf * 64, t * BN, h, b);
-            if (++stage == C::kStages) { stage = 0; kphase ^= 1u; }
-            if (t == 0) {
-              for (int x = 0; x < kQTiles && alive; ++x) {
-                alive = mbar_wait(&q_empty[x], qphase ^ 1u, abort_flag);
-                if (!alive) break;
-                mbar_expect_tx(&q_full[x], C::kQBytes);
-                for (int hf = 0; hf < C::kHalves; ++hf)
-                  tma_load_4d(q_smem + x * C::kQBytes + hf * (BM * 128), &map_q, &q_full[x], hf * 64,
-                              item[s] * kItemRows + x * BM, h, b);
-              }
-              qphase ^= 1u;
+        int tiles = 0;
+        for (int x = 0; x < kQTiles; ++x) {
+          const int tx = qtile_tiles(a, item, x);
+          tiles = tx > tiles ? tx : tiles;
+        }
+        for (int t = 0; t < tiles && alive; ++t) {
+          alive = mbar_wait(&k_empty[stage], kphase ^ 1u, abort_flag);
+          if (!alive) break;
+          mbar_expect_tx(&k_full[stage], C::kKBytes);
+          for (int hf = 0; hf < C::kHalves; ++hf)
+            tma_load_4d(k_smem + stage * C::kKBytes + hf * (BN * 128), &map_k, &k_full[stage], hf * 64, t * BN, h, b);
+          if (++stage == C::kStages) { stage = 0; kphase ^= 1u; }
+          if (t == 0) {
+            // Q tile slots past the end of the sequence are neither loaded nor used; each slot keeps
+            // its own phase bit so that producer and MMA issuer stay in step
+            for (int x = 0; x < kQTiles && alive; ++x) {
+              if (qtile_tiles(a, item, x) == 0) continue;
+              alive = mbar_wait(&q_empty[x], ((qphase >> x) & 1u) ^ 1u, abort_flag);
+              if (!alive) break;
+              qphase ^= 1u << x;
+              mbar_expect_tx(&q_full[x], C::kQBytes);
+              for (int hf = 0; hf < C::kHalves; ++hf)
+                tma_load_4d(q_smem + x * C::kQBytes + hf * (BM * 128), &map_q, &q_full[x], hf * 64,
+                            item * kItemRows + x * BM, h, b);
             }
           }
         }
@@ -366,113 +432,198 @@ __global__ void __launch_bounds__(kThreads, 1) sweep_kernel(const __grid_constan
     // ------------------------------------------------------------------ MMA issuer
     if (lane == 0) {
       constexpr uint32_t idesc = make_idesc();
-      int stage = 0;
-      uint32_t kphase = 0, qphase = 0, sphase[2] = {0, 0};
+      const uint32_t q_lo = smem_desc_lo(smem_u32(q_smem)), k_lo = smem_desc_lo(smem_u32(k_smem));
+      int stage = 0, slot = 0;
+      uint32_t kphase = 0, qphase = 0, wphase = 0, sphase[kQTiles] = {};
       bool alive = true;
-      for (int unit = blockIdx.x; unit < a.n_units && alive; unit += gridDim.x) {
-        int bh, item[2];
-        const int n_items = unit_items(a, unit, bh, item);
-        for (int s = 0; s < n_items && alive; ++s) {
-          const int tiles = item_tiles(a, item[s]);
-          for (int t = 0; t < tiles && alive; ++t) {
-            alive = mbar_wait(&k_full[stage], kphase, abort_flag);
-            if (!alive) break;
-            const uint32_t kaddr = smem_u32(k_smem + stage * C::kKBytes);
-            for (int x = 0; x < kQTiles && alive; ++x) {
-              if (t == 0) alive = mbar_wait(&q_full[x], qphase, abort_flag);
-              if (alive) alive = mbar_wait(&s_empty[x], sphase[x] ^ 1u, abort_flag);
-              if (!alive) break;
-              sphase[x] ^= 1u;
-              tc_fence_after();
-              const uint32_t qaddr = smem_u32(q_smem + x * C::kQBytes);
+      while (alive) {
+        alive = mbar_wait(&w_full[slot], wphase, abort_flag);
+        if (!alive) break;
+        const int k = w_item[slot];
+        mbar_arrive(&w_empty[slot]);
+        if (++slot == kSchedSlots) { slot = 0; wphase ^= 1u; }
+        if (k < 0) break;
+        int bh, item;
+        decode_item(a, k, bh, item);
+        int tx[kQTiles], tiles = 0;
+        for (int x = 0; x < kQTiles; ++x) {
+          tx[x] = qtile_tiles(a, item, x);
+          tiles = tx[x] > tiles ? tx[x] : tiles;
+        }
+        for (int t = 0; t < tiles && alive; ++t) {
+          alive = mbar_wait(&k_full[stage], kphase, abort_flag);
+          if (!alive) break;
+          const uint32_t b_lo = k_lo + stage * (C::kKBytes >> 4);
 #pragma unroll
-              for (int kk = 0; kk < HD / 16; ++kk) {
-                const uint32_t hf = kk >> 2, within = (kk & 3) * 32;
-                umma_bf16(tmem_base + x * BN, smem_desc_sw128(qaddr + hf * (BM * 128) + within),
-                          smem_desc_sw128(kaddr + hf * (BN * 128) + within), idesc, kk > 0 ? 1u : 0u);
-              }
-              umma_commit(&s_full[x]);
-              if (t == tiles - 1) umma_commit(&q_empty[x]);
+          for (int x = 0; x < kQTiles; ++x) {
+            if (t >= tx[x] || !alive) continue;
+            if (t == 0) {
+              alive = mbar_wait(&q_full[x], (qphase >> x) & 1u, abort_flag);
+              qphase ^= 1u << x;
             }
-            if (!alive) break;
-            umma_commit(&k_empty[stage]);
-            if (++stage == C::kStages) { stage = 0; kphase ^= 1u; }
+            if (alive) alive = mbar_wait(&s_empty[x], sphase[x] ^ 1u, abort_flag);
+            if (!alive) continue;
+            sphase[x] ^= 1u;
+            tc_fence_after();
+            const uint32_t a_lo = q_lo + x * (C::kQBytes >> 4);
+#pragma unroll
+            for (int kk = 0; kk < HD / 16; ++kk) {
+              // k-step kk: 64-column half kk / 4 (its own swizzled block), 32 bytes per step inside the half
+              const uint32_t a_off = (kk >> 2) * ((BM * 128) >> 4) + (kk & 3) * 2;
+              const uint32_t b_off = (kk >> 2) * ((BN * 128) >> 4) + (kk & 3) * 2;
+              umma_bf16(tmem_base + x * BN, a_lo + a_off, b_lo + b_off, kDescHi, idesc, kk > 0 ? 1u : 0u);
+            }
+            umma_commit(&s_full[x]);
+            if (t == tx[x] - 1) umma_commit(&q_empty[x]);
           }
-          qphase ^= 1u;
+          if (!alive) break;
+          umma_commit(&k_empty[stage]);
+          if (++stage == C::kStages) { stage = 0; kphase ^= 1u; }
         }
       }
     }
   } else {
-    // ------------------------------------------------------------------ consumers: one thread per query row
-    const int x = (warp - 2) >> 2;                 // Q tile of this group
+    // -------------------------------------------------- consumers: one thread per half of a query row
+    const int cw = warp - 2;
+    const int x = cw >> 3;                         // Q tile of this warp
+    const int half = (cw >> 2) & 1;                // which 128 columns of every K tile
     const int quad = warp & 3;                     // TMEM lane quadrant this warp may read
     const int row_local = quad * 32 + lane;
-    const uint32_t taddr_row = tmem_base + ((uint32_t)(quad * 32) << 16) + (uint32_t)(x * BN);
-    uint32_t fphase = 0;
+    const uint32_t taddr_row = tmem_base + ((uint32_t)(quad * 32) << 16) + (uint32_t)(x * BN + half * kHalfCols);
+    volatile unsigned long long* my_share = m_share + (x * 2 + half) * BM + row_local;
+    volatile unsigned long long* other_share = m_share + (x * 2 + (half ^ 1)) * BM + row_local;
+    uint32_t fphase = 0, wphase = 0;
+    int slot = 0;
     bool alive = true;
-    for (int unit = blockIdx.x; unit < a.n_units && alive; unit += gridDim.x) {
-      int bh, item[2];
-      const int n_items = unit_items(a, unit, bh, item);
+    while (alive) {
+      alive = __all_sync(0xffffffffu, mbar_wait(&w_full[slot], wphase, abort_flag));
+      if (!alive) break;
+      const int k = w_item[slot];
+      __syncwarp();
+      if (lane == 0) mbar_arrive(&w_empty[slot]);
+      if (++slot == kSchedSlots) { slot = 0; wphase ^= 1u; }
+      if (k < 0) break;
+      int bh, item;
+      decode_item(a, k, bh, item);
+      const int tiles = qtile_tiles(a, item, x);
+      if (tiles == 0) continue;
       const int h = bh % a.H;
-      for (int s = 0; s < n_items && alive; ++s) {
-        const int tiles = item_tiles(a, item[s]);
-        const int tile_row0 = item[s] * kItemRows + x * BM;
-        const int i = tile_row0 + row_local;
-        const bool valid = i < a.N;
-        const size_t grow = (size_t)bh * a.N + (valid ? i : 0);
-        RowState r;
-        r.list = a.entries + grow * kListCap;
-        r.cnt = 0;
-        r.m_run = -INFINITY;
-        r.lim = a.causal ? i : a.N - 1;
-        r.thr_acc = INFINITY;
-        r.a = 1.f;
-        r.inv_a = 1.f;
-        if (valid) {
-          r.a = a.alpha_m1 * (a.scale[(size_t)h * a.N + i] * a.sm_scale);
-          if (r.a > 0.f && r.a < INFINITY) {
-            r.inv_a = 1.0f / r.a;
-            if (a.mode == 0) {
-              r.thr_acc = -INFINITY;
-            } else {
-              const float t_acc = a.tau_in[grow] * r.inv_a;
-              r.thr_acc = t_acc - 1e-6f * fabsf(t_acc);   // a hair below: the row kernel applies the exact test
-            }
+      const int tile_row0 = item * kItemRows + x * BM;
+      const int i = tile_row0 + row_local;
+      const bool valid = i < a.N;
+      const size_t grow = (size_t)bh * a.N + (valid ? i : 0);
+      Entry* list = a.entries + grow * kListCap + half * kHalfCap;
+      const int lim = a.causal ? i : a.N - 1;      // largest visible key index
+      RowState r;
+      r.cnt = 0;
+      r.m_run = -INFINITY;
+      r.thr = INFINITY;
+      float ra = 1.f, inv_a = 1.f;
+      if (valid) {
+        ra = a.alpha_m1 * (a.scale[(size_t)h * a.N + i] * a.sm_scale);
+        if (ra > 0.f && ra < INFINITY) {
+          inv_a = 1.0f / ra;
+          if (a.mode == 0) {
+            r.thr = -INFINITY;
           } else {
-            r.cnt = -1;   // non-positive or non-finite scale: dense path
+            const float t_acc = a.tau_in[grow] * inv_a;
+            r.thr = t_acc - 1e-6f * fabsf(t_acc);   // a hair below: the row kernel applies the exact test
           }
+        } else {
+          r.cnt = -1;   // non-positive or non-finite scale: dense path
         }
-        const bool dump_here = a.dump != nullptr && bh == a.dump_bh && valid;
-        // tiles that reach past the last visible key of this Q tile's first row need the mask
-        const int first_lim = a.causal ? tile_row0 : a.N - 1;
-        for (int t = 0; t < tiles && alive; ++t) {
-          // the warp leaves together: tcgen05.ld needs all 32 lanes
-          alive = __all_sync(0xffffffffu, mbar_wait(&s_full[x], fphase, abort_flag));
-          if (!alive) break;
-          fphase ^= 1u;
-          tc_fence_after();
-          const bool masked = t * BN + BN - 1 > first_lim;
-#pragma unroll 1
-          for (int c = 0; c < BN / 32; ++c) {
-            float v[32];
-            __syncwarp();
-            tmem_ld32(taddr_row + c * 32, v);
+      }
+      const bool searching = a.mode == 0 && r.cnt == 0 && valid;
+      const bool dump_here = kDump && a.dump != nullptr && bh == a.dump_bh && valid;
+      // first / last visible key over the rows of this Q tile: halves past the last one are skipped,
+      // halves that reach past the first one need the mask
+      const int first_lim = a.causal ? tile_row0 : a.N - 1;
+      const int last_lim = a.causal ? (tile_row0 + BM - 1 < a.N - 1 ? tile_row0 + BM - 1 : a.N - 1) : a.N - 1;
+      for (int t = 0; t < tiles && alive; ++t) {
+        // the warp leaves together: tcgen05.ld needs all 32 lanes
+        alive = __all_sync(0xffffffffu, mbar_wait(&s_full[x], fphase, abort_flag));
+        if (!alive) break;
+        fphase ^= 1u;
+        tc_fence_after();
+        const int col_base = t * BN + half * kHalfCols;
+        if (col_base <= last_lim) {
+          const bool masked = col_base + kHalfCols - 1 > first_lim;
+          // ---- pass 1: 128 columns -> 16 group maxima (8 columns each)
+          float g[16];
+          float va[16], vb[16];
+          tmem_ld16(taddr_row, va);
+#pragma unroll
+          for (int c = 0; c < kHalfCols / 16; ++c) {
+            float (&cur)[16] = (c & 1) ? vb : va;
+            float (&nxt)[16] = (c & 1) ? va : vb;
             tmem_ld_wait();
-            const int col0 = t * BN + c * 32;
-            if (dump_here) {
-              for (int u = 0; u < 32; ++u)
-                if (col0 + u <= r.lim) a.dump[(size_t)i * a.N + col0 + u] = v[u];
+            if (c + 1 < kHalfCols / 16) tmem_ld16(taddr_row + (c + 1) * 16, nxt);   // in flight during the maxima
+            if (kDump) {
+              if (dump_here) {
+#pragma unroll
+                for (int u = 0; u < 16; ++u)
+                  if (col_base + c * 16 + u <= lim) a.dump[(size_t)i * a.N + col_base + c * 16 + u] = cur[u];
+              }
             }
-            if (masked) scan_chunk<true>(v, col0, r, a.mode, a.expo_class, a.expo);
-            else scan_chunk<false>(v, col0, r, a.mode, a.expo_class, a.expo);
+            if (masked) {
+#pragma unroll
+              for (int u = 0; u < 16; ++u) cur[u] = (col_base + c * 16 + u <= lim) ? cur[u] : -INFINITY;
+            }
+            g[2 * c] = max8(&cur[0]);
+            g[2 * c + 1] = max8(&cur[8]);
           }
-          tc_fence_before();
-          mbar_arrive(&s_empty[x]);
+          float m_tile = max3(g[0], g[1], g[2]);
+#pragma unroll
+          for (int u = 3; u < 15; u += 2) m_tile = max3(m_tile, g[u], g[u + 1]);
+          m_tile = fmaxf(m_tile, g[15]);
+          if (searching) {
+            // the other half's running maximum (if it already belongs to this item) tightens the bound too
+            const unsigned long long o = *other_share;
+            const float m_other = (int)(o >> 32) == k ? __uint_as_float((unsigned)o) : -INFINITY;
+            r.m_run = max3(r.m_run, m_tile, m_other);
+            if (r.cnt >= 0) r.thr = fmaxf(r.thr, r.m_run - inv_a);
+            *my_share = ((unsigned long long)(unsigned)k << 32) | __float_as_uint(r.m_run);
+          }
+          // ---- pass 2 (only when some lane saw a candidate): re-read the groups that hold one
+          const bool hit = m_tile > r.thr;
+          if (__any_sync(0xffffffffu, hit)) {
+            unsigned mine = 0;
+#pragma unroll
+            for (int u = 0; u < 16; ++u) mine |= (g[u] > r.thr ? 1u : 0u) << u;
+            unsigned todo = __reduce_or_sync(0xffffffffu, mine);
+            while (todo) {
+              const int u = __ffs(todo) - 1;
+              todo &= todo - 1;
+              float v8[8];
+              tmem_ld8(taddr_row + u * 8, v8);
+              tmem_ld_wait();
+              if ((mine >> u) & 1u) {
+                const float thr = r.thr;
+                int cnt = r.cnt;
+#pragma unroll
+                for (int e = 0; e < 8; ++e) {
+                  const int col = col_base + u * 8 + e;
+                  if (v8[e] > thr && col <= lim) {
+                    list[cnt].y = v8[e];
+                    list[cnt].j = col;
+                    ++cnt;
+                  }
+                }
+                r.cnt = cnt;
+              }
+              const unsigned need = __ballot_sync(0xffffffffu, r.cnt > kHalfTrigger);
+              if (need) shrink_lists(r, list, ra, inv_a, need, a.mode, a.expo_class, a.expo);
+            }
+          }
         }
-        if (valid && alive) {
-          a.row_cnt[grow] = r.cnt;
-          a.row_thr[grow] = r.thr_acc * r.a;
-        }
+        // the accumulator has been read: hand it back to the MMA issuer
+        tc_fence_before();
+        __syncwarp();
+        if (lane == 0) mbar_arrive(&s_empty[x]);
+      }
+      if (valid && alive) {
+        a.half_cnt[grow * 2 + half] = r.cnt;
+        a.half_thr[grow * 2 + half] = r.thr * ra;
       }
     }
   }
@@ -527,30 +678,33 @@ cudaError_t make_map(CUtensorMap* map, const void* base, const Problem& p, int b
   return r == CUDA_SUCCESS ? cudaSuccess : cudaErrorInvalidValue;
 }
 
-template <int HD>
+template <int HD, bool kDump>
 cudaError_t launch_impl(const Problem& p, const void* q, const void* k, SweepArgs& args, cudaStream_t stream) {
   CUtensorMap map_q, map_k;
   cudaError_t err = make_map(&map_q, q, p, BM);
   if (err != cudaSuccess) return err;
   err = make_map(&map_k, k, p, BN);
   if (err != cudaSuccess) return err;
-  err = cudaFuncSetAttribute(sweep_kernel<HD>, cudaFuncAttributeMaxDynamicSharedMemorySize, Cfg<HD>::kSmemBytes);
+  err = cudaFuncSetAttribute(sweep_kernel<HD, kDump>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                             Cfg<HD>::kSmemBytes);
   if (err != cudaSuccess) return err;
   int dev = 0, sms = 0;
   err = cudaGetDevice(&dev);
   if (err != cudaSuccess) return err;
   err = cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
   if (err != cudaSuccess) return err;
-  const int grid = args.n_units < sms ? args.n_units : sms;
-  sweep_kernel<HD><<<grid, kThreads, Cfg<HD>::kSmemBytes, stream>>>(map_q, map_k, args);
+  err = cudaMemsetAsync(args.work_counter, 0, sizeof(int32_t), stream);
+  if (err != cudaSuccess) return err;
+  const int grid = args.n_items < sms ? args.n_items : sms;
+  sweep_kernel<HD, kDump><<<grid, kThreads, Cfg<HD>::kSmemBytes, stream>>>(map_q, map_k, args);
   return cudaGetLastError();
 }
 
 }  // namespace
 
 cudaError_t launch_sweep(const Problem& p, const void* q, const void* k, const float* scale, const float* tau_in,
-                         int mode, int32_t* row_cnt, float* row_thr, Entry* entries, float* dump, int dump_bh,
-                         int32_t* status, cudaStream_t stream) {
+                         int mode, int32_t* half_cnt, float* half_thr, Entry* entries, int32_t* work_counter,
+                         float* dump, int dump_bh, int32_t* status, cudaStream_t stream) {
   SweepArgs args;
   args.B = p.B; args.H = p.H; args.N = p.N;
   args.causal = p.causal;
@@ -561,16 +715,17 @@ cudaError_t launch_sweep(const Problem& p, const void* q, const void* k, const f
   args.sm_scale = p.sm_scale;
   args.scale = scale;
   args.tau_in = tau_in;
-  args.row_cnt = row_cnt;
-  args.row_thr = row_thr;
+  args.half_cnt = half_cnt;
+  args.half_thr = half_thr;
   args.entries = entries;
   args.dump = dump;
   args.dump_bh = dump_bh;
   args.status = status;
+  args.work_counter = work_counter;
   args.items_per_bh = (p.N + kItemRows - 1) / kItemRows;
-  args.units_per_bh = p.causal ? (args.items_per_bh + 1) / 2 : args.items_per_bh;
-  args.n_units = args.units_per_bh * p.B * p.H;
-  return p.D == 64 ? launch_impl<64>(p, q, k, args, stream) : launch_impl<128>(p, q, k, args, stream);
+  args.n_items = args.items_per_bh * p.B * p.H;
+  if (dump) return p.D == 64 ? launch_impl<64, true>(p, q, k, args, stream) : launch_impl<128, true>(p, q, k, args, stream);
+  return p.D == 64 ? launch_impl<64, false>(p, q, k, args, stream) : launch_impl<128, false>(p, q, k, args, stream);
 }
 
 }  // namespace entmax
