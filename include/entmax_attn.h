@@ -53,7 +53,8 @@ typedef enum {
   ENTMAX_ATTN_EINVAL_WORKSPACE = -5, /* workspace NULL, misaligned (256 B) or smaller than workspace_bytes()    */
   ENTMAX_ATTN_EINVAL_NULL = -6,      /* a required pointer is NULL, or only some of beta/gamma/delta are given  */
   ENTMAX_ATTN_ECUDA = -7,            /* a CUDA call failed; see entmax_attn_last_cuda_error()                   */
-  ENTMAX_ATTN_EUNSUPPORTED = -8      /* the device is not sm_100 (bf16 path needs tcgen05/TMA)                  */
+  ENTMAX_ATTN_EUNSUPPORTED = -8,     /* the device is not sm_100 (bf16 path needs tcgen05/TMA)                  */
+  ENTMAX_ATTN_ETOOLARGE = -9         /* entmax_attn_fwd_static: the problem does not fit the built-in scratch  */
 } entmax_attn_status;
 
 typedef struct {
@@ -121,6 +122,36 @@ typedef struct {
   int32_t reserved;
 } entmax_attn_ws_layout;
 int entmax_attn_workspace_layout(const entmax_attn_params* params, entmax_attn_ws_layout* out);
+
+/* Forward pass for callers that cannot provide a workspace.  (The paper has no counterpart: it does
+ * not discuss memory management.)
+ *
+ * Who needs it: code that may not, or cannot, allocate device memory at the point of the call -- a
+ * plugin that is handed tensors but no allocator, a start-up or recovery path that runs before the
+ * framework's memory pool exists, a region in which calling the allocator is forbidden.  Such callers
+ * cannot pass the `workspace` that entmax_attn_fwd wants, so this entry point uses a fixed scratch
+ * array that is part of the library image instead.  It calls no cudaMalloc / cudaFree and no
+ * allocating library routine; every GPU on which the library is loaded holds
+ * ENTMAX_ATTN_STATIC_SCRATCH_BYTES of device memory for it until the process exits.
+ *
+ * Same results as entmax_attn_fwd (O and tau; arguments as there, minus the workspace), computed by
+ * the dense-row kernels: every visible key of every row is visited with fp32 arithmetic, for bf16 and
+ * fp32 problems alike, so it is meant for small and medium problems, not for the long-context ones.
+ *
+ * Size limit: round_up(heads*seq, 32) + 64 * round_up(seq, 32) floats must fit the scratch
+ * (e.g. 16 heads up to seq 26214).  Larger problems return ENTMAX_ATTN_ETOOLARGE, nothing enqueued.
+ *
+ * Set-up: the first call on each device looks up the device address of the scratch array
+ * (cudaGetSymbolAddress) with that device current; make that first call outside any stream capture.
+ *
+ * Sharing: all calls on a device use the same array, which keeps whatever the previous call left in it.
+ * Nothing in it has to be cleared between calls (each call overwrites what it later reads), but two
+ * calls that overlap on the GPU -- different streams, or different host threads without ordering --
+ * race on it and produce garbage.  Calls on one stream are safe. */
+#define ENTMAX_ATTN_STATIC_SCRATCH_BYTES (8u << 20)
+int entmax_attn_fwd_static(const entmax_attn_params* params, const void* q, const void* k, const void* v,
+                           const float* beta, const float* gamma, const float* delta, void* o, float* tau,
+                           int32_t* device_status, void* cuda_stream);
 
 /* The score-tile engine on its own (Sec. 2.1 logits before any scale): writes the raw tensor-core
  * accumulators <q_i, k_j> (bf16 inputs, fp32 accumulation) of one (batch, head) pair,

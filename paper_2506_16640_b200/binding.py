@@ -59,6 +59,8 @@ def load():
         lib.entmax_attn_fwd.argtypes = [pp, vp, vp, vp, fp, fp, fp, vp, fp, vp, ctypes.c_size_t, ip, vp]
         lib.entmax_attn_bwd.restype = ctypes.c_int
         lib.entmax_attn_bwd.argtypes = [pp, vp, vp, vp, fp, fp, fp, fp, vp, vp, vp, vp, vp, ctypes.c_size_t, ip, vp]
+        lib.entmax_attn_fwd_static.restype = ctypes.c_int
+        lib.entmax_attn_fwd_static.argtypes = [pp, vp, vp, vp, fp, fp, fp, vp, fp, ip, vp]
         lib.entmax_attn_scores_debug.restype = ctypes.c_int
         lib.entmax_attn_scores_debug.argtypes = [pp, vp, vp, ctypes.c_int32, fp, vp, ctypes.c_size_t, ip, vp]
         lib.entmax_attn_profile_events.restype = ctypes.c_int
@@ -148,6 +150,20 @@ def entmax_attn_fwd(q, k, v, alpha, causal, beta=None, gamma=None, delta=None, *
                                 _ptr(o), _ptr(tau), _ptr(workspace), workspace.numel(), _ptr(status),
                                 _stream_ptr(stream))
     _check(rc, "entmax_attn_fwd")
+    return o, tau
+
+
+def entmax_attn_fwd_static(q, k, v, alpha, causal, beta=None, gamma=None, delta=None, *, sm_scale=0.0, n_mode=0,
+                           o, tau, status=None, stream=None):
+    """Forward pass without a workspace, for callers that cannot allocate device memory: the scratch is
+    a fixed array inside the library.  `o` and `tau` must be passed in (this wrapper allocates nothing
+    either).  Raises EntmaxAttnError when the problem exceeds the built-in scratch.  Calls that overlap
+    on the GPU share that scratch and race; keep them on one stream."""
+    _same_layout(q, k, v, o)
+    params = make_params(q, alpha, causal, sm_scale, n_mode)
+    rc = load().entmax_attn_fwd_static(ctypes.byref(params), _ptr(q), _ptr(k), _ptr(v), _ptr(beta), _ptr(gamma),
+                                       _ptr(delta), _ptr(o), _ptr(tau), _ptr(status), _stream_ptr(stream))
+    _check(rc, "entmax_attn_fwd_static")
     return o, tau
 
 

@@ -306,6 +306,7 @@ const char* entmax_attn_strerror(int code) {
     case ENTMAX_ATTN_EINVAL_NULL: return "a required pointer is NULL (beta, gamma, delta: all or none)";
     case ENTMAX_ATTN_ECUDA: return "a CUDA call failed (see entmax_attn_last_cuda_error)";
     case ENTMAX_ATTN_EUNSUPPORTED: return "the bf16 path needs an sm_100 device";
+    case ENTMAX_ATTN_ETOOLARGE: return "the problem does not fit the library's built-in scratch (see entmax_attn_fwd_static)";
     default: return "unknown status";
   }
 }
