@@ -12,12 +12,13 @@ namespace entmax {
 
 // Sparse row lists.  The score sweep splits the keys of a row between two threads; each owns one half
 // of the row's kListCap list slots: capacity kHalfCap, the fill level at which the sweep tightens the
-// threshold and filters the half-list (checked after every 8 keys, so the capacity is never exceeded),
+// threshold and filters the half-list (checked after every 32 keys, so the capacity is never exceeded),
 // and the length a filtered half-list may keep -- a row that cannot be brought down to it is handed to
 // the dense path.  The row kernels merge the two halves and leave the support compacted from slot 0.
-constexpr int kHalfCap = 64;
-constexpr int kHalfTrigger = 40;
-constexpr int kHalfKeep = 32;
+constexpr int kHalfCap = 128;
+constexpr int kHalfTrigger = 88;
+constexpr int kHalfKeep = 72;
+static_assert(kHalfTrigger + 32 <= kHalfCap && kHalfKeep < kHalfTrigger, "half-list bounds");
 constexpr int kListCap = 2 * kHalfCap;
 
 // One list slot: y = (alpha-1) * s_ij (or the raw accumulator while a sweep is running), j = key index.

@@ -25,8 +25,8 @@
 //                 own running maximum, threshold, list length (registers) and half-list; the two share
 //                 their running maxima through shared memory so that both thresholds stay tight.
 // A consumer first reduces its 128 columns to 16 group maxima (branch-free), and only when some lane of
-// the warp saw a value above its threshold re-reads the groups that hold candidates; then it hands the
-// accumulator back.  While the consumers of one Q tile scan, the tensor core works on the other.
+// the warp saw a value above its threshold re-reads the groups that hold candidates (four groups per
+// round trip to TMEM); it hands the accumulator back as soon as the last values it needs are in registers.  While the consumers of one Q tile scan, the tensor core works on the other.
 // Every mbarrier wait is bounded: on expiry the CTA raises ENTMAX_ATTN_FLAG_WAIT_EXPIRED, all roles
 // leave their loops, in-flight copies are given time to land, TMEM is freed and the CTA returns.
 #include <cuda.h>
@@ -546,6 +546,7 @@ __global__ void __launch_bounds__(kThreads, 1) sweep_kernel(const __grid_constan
         fphase ^= 1u;
         tc_fence_after();
         const int col_base = t * BN + half * kHalfCols;
+        bool released = false;
         if (col_base <= last_lim) {
           const bool masked = col_base + kHalfCols - 1 > first_lim;
           // ---- pass 1: 128 columns -> 16 group maxima (8 columns each)
@@ -592,34 +593,60 @@ __global__ void __launch_bounds__(kThreads, 1) sweep_kernel(const __grid_constan
             for (int u = 0; u < 16; ++u) mine |= (g[u] > r.thr ? 1u : 0u) << u;
             unsigned todo = __reduce_or_sync(0xffffffffu, mine);
             while (todo) {
-              const int u = __ffs(todo) - 1;
-              todo &= todo - 1;
-              float v8[8];
-              tmem_ld8(taddr_row + u * 8, v8);
-              tmem_ld_wait();
-              if ((mine >> u) & 1u) {
-                const float thr = r.thr;
-                int cnt = r.cnt;
+              // up to four groups per round trip to TMEM (todo is the same in every lane)
+              int gu[4];
 #pragma unroll
-                for (int e = 0; e < 8; ++e) {
-                  const int col = col_base + u * 8 + e;
-                  if (v8[e] > thr && col <= lim) {
-                    list[cnt].y = v8[e];
-                    list[cnt].j = col;
-                    ++cnt;
-                  }
-                }
-                r.cnt = cnt;
+              for (int w = 0; w < 4; ++w) {
+                gu[w] = todo ? __ffs(todo) - 1 : -1;
+                todo &= todo - 1;
               }
+              float v8[4][8];
+#pragma unroll
+              for (int w = 0; w < 4; ++w)
+                if (gu[w] >= 0) tmem_ld8(taddr_row + gu[w] * 8, v8[w]);
+              tmem_ld_wait();
+              if (todo == 0) {
+                // the last batch is in registers: hand the accumulator back before the list stores
+                tc_fence_before();
+                __syncwarp();
+                if (lane == 0) mbar_arrive(&s_empty[x]);
+                released = true;
+              }
+              if (masked) {
+#pragma unroll
+                for (int w = 0; w < 4; ++w)
+#pragma unroll
+                  for (int e = 0; e < 8; ++e)
+                    v8[w][e] = (gu[w] >= 0 && col_base + gu[w] * 8 + e <= lim) ? v8[w][e] : -INFINITY;
+              }
+#pragma unroll
+              for (int w = 0; w < 4; ++w) {
+                if (gu[w] >= 0 && ((mine >> gu[w]) & 1u)) {
+                  const float thr = r.thr;
+                  int cnt = r.cnt;
+#pragma unroll
+                  for (int e = 0; e < 8; ++e) {
+                    if (v8[w][e] > thr) {
+                      list[cnt].y = v8[w][e];
+                      list[cnt].j = col_base + gu[w] * 8 + e;
+                      ++cnt;
+                    }
+                  }
+                  r.cnt = cnt;
+                }
+              }
+              // at most 32 entries were appended since the last check: the half-list cannot overflow
               const unsigned need = __ballot_sync(0xffffffffu, r.cnt > kHalfTrigger);
               if (need) shrink_lists(r, list, ra, inv_a, need, a.mode, a.expo_class, a.expo);
             }
           }
         }
-        // the accumulator has been read: hand it back to the MMA issuer
-        tc_fence_before();
-        __syncwarp();
-        if (lane == 0) mbar_arrive(&s_empty[x]);
+        // the accumulator has been read: hand it back to the MMA issuer (unless pass 2 already did)
+        if (!released) {
+          tc_fence_before();
+          __syncwarp();
+          if (lane == 0) mbar_arrive(&s_empty[x]);
+        }
       }
       if (valid && alive) {
         a.half_cnt[grow * 2 + half] = r.cnt;

@@ -45,10 +45,10 @@ def test_workspace_bytes_and_layout(lib):
     fwd = lib.entmax_attn_workspace_bytes(ctypes.byref(p), 0)
     bwd = lib.entmax_attn_workspace_bytes(ctypes.byref(p), 1)
     rows = 1 * 2 * 128
-    assert fwd >= rows * 128 * 8 and bwd >= fwd + 2 * rows * 64 * 4
+    assert fwd >= rows * 256 * 8 and bwd >= fwd + 2 * rows * 64 * 4
     lay = WsLayout()
     assert lib.entmax_attn_workspace_layout(ctypes.byref(p), ctypes.byref(lay)) == 0
-    assert lay.capacity == 128 and lay.entries_offset % 256 == 0 and lay.row_count_offset % 256 == 0
+    assert lay.capacity == 256 and lay.entries_offset % 256 == 0 and lay.row_count_offset % 256 == 0
     big = _params(batch=1, heads=16, seq=32768, head_dim=128, dtype=0)
     assert lib.entmax_attn_workspace_bytes(ctypes.byref(big), 0) < 2 << 30
     for bad in [_params(head_dim=96), _params(seq=0), _params(alpha=1.0), _params(alpha=2.5), _params(dtype=7),
