@@ -84,16 +84,16 @@ struct SweepArgs {
 // ------------------------------------------------------------------------------------------ PTX
 __device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
 
-__device__ __forceinline__ void mbar_init(uint64_t* bar, uint32_t count) {
-  asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(smem_u32(bar)), "r"(count) : "memory");
+__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
+  asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count) : "memory");
 }
-__device__ __forceinline__ void mbar_expect_tx(uint64_t* bar, uint32_t bytes) {
-  asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(smem_u32(bar)), "r"(bytes) : "memory");
+__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
+  asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
 }
-__device__ __forceinline__ void mbar_arrive(uint64_t* bar) {
-  asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(smem_u32(bar)) : "memory");
+__device__ __forceinline__ void mbar_arrive(uint32_t bar) {
+  asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
 }
-__device__ __forceinline__ bool mbar_try_wait(uint64_t* bar, uint32_t parity) {
+__device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
   uint32_t ok;
   asm volatile(
       "{\n"
@@ -102,9 +102,25 @@ __device__ __forceinline__ bool mbar_try_wait(uint64_t* bar, uint32_t parity) {
       " selp.u32 %0, 1, 0, p;\n"
       "}\n"
       : "=r"(ok)
-      : "r"(smem_u32(bar)), "r"(parity)
+      : "r"(bar), "r"(parity)
       : "memory");
   return ok != 0;
+}
+__device__ __forceinline__ uint32_t lds_u32(uint32_t addr) {
+  uint32_t v;
+  asm volatile("ld.volatile.shared::cta.u32 %0, [%1];" : "=r"(v) : "r"(addr) : "memory");
+  return v;
+}
+__device__ __forceinline__ void sts_u32(uint32_t addr, uint32_t v) {
+  asm volatile("st.volatile.shared::cta.u32 [%0], %1;" ::"r"(addr), "r"(v) : "memory");
+}
+__device__ __forceinline__ unsigned long long lds_u64(uint32_t addr) {
+  unsigned long long v;
+  asm volatile("ld.volatile.shared::cta.u64 %0, [%1];" : "=l"(v) : "r"(addr) : "memory");
+  return v;
+}
+__device__ __forceinline__ void sts_u64(uint32_t addr, unsigned long long v) {
+  asm volatile("st.volatile.shared::cta.u64 [%0], %1;" ::"r"(addr), "l"(v) : "memory");
 }
 __device__ __forceinline__ uint64_t global_ns() {
   uint64_t t;
@@ -112,36 +128,37 @@ __device__ __forceinline__ uint64_t global_ns() {
   return t;
 }
 // Bounded wait.  Returns false when the CTA is aborting (this or another wait ran out of time).
-__device__ __noinline__ bool mbar_wait_slow(uint64_t* bar, uint32_t parity, volatile int* abort_flag) {
+// `abort_flag` is the shared-memory address of the CTA's abort word.
+__device__ __noinline__ bool mbar_wait_slow(uint32_t bar, uint32_t parity, uint32_t abort_flag) {
   const uint64_t t0 = global_ns();
   uint32_t spins = 0;
   for (;;) {
     if (mbar_try_wait(bar, parity)) return true;
     if ((++spins & 63u) == 0u) {
-      if (*abort_flag) return false;
+      if (lds_u32(abort_flag)) return false;
       if (global_ns() - t0 > kWaitLimitNs) {
-        *abort_flag = 1;
+        sts_u32(abort_flag, 1u);
         return false;
       }
     }
   }
 }
-__device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, volatile int* abort_flag) {
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, uint32_t abort_flag) {
   if (mbar_try_wait(bar, parity)) return true;
   if (mbar_try_wait(bar, parity)) return true;
   return mbar_wait_slow(bar, parity, abort_flag);
 }
 
-__device__ __forceinline__ void tma_load_4d(void* dst, const CUtensorMap* map, uint64_t* bar, int c0, int c1, int c2,
+__device__ __forceinline__ void tma_load_4d(uint32_t dst, const CUtensorMap* map, uint32_t bar, int c0, int c1, int c2,
                                             int c3) {
   asm volatile(
       "cp.async.bulk.tensor.4d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5, %6}], [%2];"
-      ::"r"(smem_u32(dst)), "l"(reinterpret_cast<uint64_t>(map)), "r"(smem_u32(bar)), "r"(c0), "r"(c1), "r"(c2), "r"(c3)
+      ::"r"(dst), "l"(reinterpret_cast<uint64_t>(map)), "r"(bar), "r"(c0), "r"(c1), "r"(c2), "r"(c3)
       : "memory");
 }
 
-__device__ __forceinline__ void tmem_alloc(uint32_t* dst_smem, uint32_t ncols) {
-  asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(dst_smem)), "r"(ncols)
+__device__ __forceinline__ void tmem_alloc(uint32_t dst_smem, uint32_t ncols) {
+  asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(dst_smem), "r"(ncols)
                : "memory");
 }
 __device__ __forceinline__ void tmem_relinquish() {
@@ -170,8 +187,8 @@ __device__ __forceinline__ void umma_bf16(uint32_t d_tmem, uint32_t a_lo, uint32
       : "memory");
 }
 // mbarrier arrive once every MMA issued so far by this thread has completed
-__device__ __forceinline__ void umma_commit(uint64_t* bar) {
-  asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(smem_u32(bar))
+__device__ __forceinline__ void umma_commit(uint32_t bar) {
+  asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar)
                : "memory");
 }
 
@@ -254,8 +271,10 @@ struct RowState {
 
 // Warp-cooperative list shrink for the lanes whose half-list has grown past kHalfTrigger.  Accumulator
 // units are turned into Eq. 1's units with y = a * acc.  All 32 lanes must call this together.
-__device__ __noinline__ void shrink_lists(RowState& r, Entry* list, float a, float inv_a, unsigned need, int mode,
-                                          int expo_class, float expo) {
+// Takes and returns the row state by value: a state whose address escaped would have to be kept in
+// local memory across every asm statement of the scan loop.
+__device__ __noinline__ RowState shrink_lists(RowState r, Entry* list, float a, float inv_a, unsigned need, int mode,
+                                              int expo_class, float expo) {
   const int lane = threadIdx.x & 31;
   constexpr int kSlots = kHalfCap / 32;
   __syncwarp();   // the owner's list stores are ordered before the other lanes' loads
@@ -320,6 +339,7 @@ __device__ __noinline__ void shrink_lists(RowState& r, Entry* list, float a, flo
     }
   }
   __syncwarp();
+  return r;
 }
 
 template <int HD, bool kDump>
@@ -328,24 +348,24 @@ __global__ void __launch_bounds__(kThreads, 1) sweep_kernel(const __grid_constan
                                                             const SweepArgs a) {
   using C = Cfg<HD>;
   extern __shared__ uint8_t smem_raw[];
-  uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
-  uint8_t* q_smem = smem;                                   // [kQTiles][kHalves][BM rows x 128 B]
-  uint8_t* k_smem = smem + kQTiles * C::kQBytes;            // [kStages][kHalves][BN rows x 128 B]
+  // everything in shared memory is addressed by 32-bit shared-window addresses derived from one base
+  const uint32_t sbase = (smem_u32(smem_raw) + 1023u) & ~1023u;
+  const uint32_t q_smem = sbase;                                   // [kQTiles][kHalves][BM rows x 128 B]
+  const uint32_t k_smem = sbase + kQTiles * C::kQBytes;            // [kStages][kHalves][BN rows x 128 B]
   // running maximum of each half-row, tagged with the work item it belongs to: {item id, float bits}
-  volatile unsigned long long* m_share =
-      reinterpret_cast<volatile unsigned long long*>(k_smem + C::kStages * C::kKBytes);   // [kQTiles][2][BM]
-  uint64_t* bars = reinterpret_cast<uint64_t*>(k_smem + C::kStages * C::kKBytes + C::kShareBytes);
-  uint64_t* q_full = bars;                       // [kQTiles]
-  uint64_t* q_empty = q_full + kQTiles;          // [kQTiles]
-  uint64_t* s_full = q_empty + kQTiles;          // [kQTiles]
-  uint64_t* s_empty = s_full + kQTiles;          // [kQTiles]
-  uint64_t* k_full = s_empty + kQTiles;          // [kStages]
-  uint64_t* k_empty = k_full + C::kStages;       // [kStages]
-  uint64_t* w_full = k_empty + C::kStages;       // [kSchedSlots]
-  uint64_t* w_empty = w_full + kSchedSlots;      // [kSchedSlots]
-  volatile int* w_item = reinterpret_cast<volatile int*>(w_empty + kSchedSlots);   // [kSchedSlots]
-  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(const_cast<int*>(w_item) + kSchedSlots);
-  volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
+  const uint32_t m_share = k_smem + C::kStages * C::kKBytes;       // u64 [kQTiles][2][BM]
+  const uint32_t bars = m_share + C::kShareBytes;                  // mbarriers, 8 bytes each
+  const uint32_t q_full = bars;                            // [kQTiles]
+  const uint32_t q_empty = q_full + 8 * kQTiles;           // [kQTiles]
+  const uint32_t s_full = q_empty + 8 * kQTiles;           // [kQTiles]
+  const uint32_t s_empty = s_full + 8 * kQTiles;           // [kQTiles]
+  const uint32_t k_full = s_empty + 8 * kQTiles;           // [kStages]
+  const uint32_t k_empty = k_full + 8 * C::kStages;        // [kStages]
+  const uint32_t w_full = k_empty + 8 * C::kStages;        // [kSchedSlots]
+  const uint32_t w_empty = w_full + 8 * kSchedSlots;       // [kSchedSlots]
+  const uint32_t w_item = w_empty + 8 * kSchedSlots;       // int32 [kSchedSlots]
+  const uint32_t tmem_slot = w_item + 4 * kSchedSlots;     // uint32
+  const uint32_t abort_flag = tmem_slot + 4;               // uint32
   static_assert((4 * kQTiles + 2 * C::kStages + 2 * kSchedSlots) * 8 + kSchedSlots * 4 + 8 <= C::kBarBytes,
                 "barrier area");
 
@@ -354,24 +374,24 @@ __global__ void __launch_bounds__(kThreads, 1) sweep_kernel(const __grid_constan
 
   if (threadIdx.x == 0) {
     for (int t = 0; t < kQTiles; ++t) {
-      mbar_init(&q_full[t], 1);
-      mbar_init(&q_empty[t], 1);
-      mbar_init(&s_full[t], 1);
-      mbar_init(&s_empty[t], 8);                 // one arrival per consumer warp of the Q tile
+      mbar_init(q_full + 8 * t, 1);
+      mbar_init(q_empty + 8 * t, 1);
+      mbar_init(s_full + 8 * t, 1);
+      mbar_init(s_empty + 8 * t, 8);                 // one arrival per consumer warp of the Q tile
     }
     for (int t = 0; t < C::kStages; ++t) {
-      mbar_init(&k_full[t], 1);
-      mbar_init(&k_empty[t], 1);
+      mbar_init(k_full + 8 * t, 1);
+      mbar_init(k_empty + 8 * t, 1);
     }
     for (int t = 0; t < kSchedSlots; ++t) {
-      mbar_init(&w_full[t], 1);
-      mbar_init(&w_empty[t], 1 + kConsumerWarps);   // MMA issuer + one arrival per consumer warp
+      mbar_init(w_full + 8 * t, 1);
+      mbar_init(w_empty + 8 * t, 1 + kConsumerWarps);   // MMA issuer + one arrival per consumer warp
     }
-    *abort_flag = 0;
+    sts_u32(abort_flag, 0u);
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
   }
-  if (threadIdx.x < kQTiles * 2 * BM) m_share[threadIdx.x] = ~0ull;   // tag -1: belongs to no work item
+  if (threadIdx.x < kQTiles * 2 * BM) sts_u64(m_share + 8 * threadIdx.x, ~0ull);   // tag -1: belongs to no work item
   if (warp == 1) {
     tmem_alloc(tmem_slot, kTmemCols);
     tmem_relinquish();
@@ -379,7 +399,7 @@ __global__ void __launch_bounds__(kThreads, 1) sweep_kernel(const __grid_constan
   tc_fence_before();
   __syncthreads();
   tc_fence_after();
-  const uint32_t tmem_base = *tmem_slot;
+  const uint32_t tmem_base = lds_u32(tmem_slot);
 
   if (warp == 0) {
     // ------------------------------------------------------------- scheduler + TMA producer
@@ -388,12 +408,12 @@ __global__ void __launch_bounds__(kThreads, 1) sweep_kernel(const __grid_constan
       uint32_t kphase = 0, qphase = 0 /* bit x: phase of Q tile slot x */, wphase = 0;
       bool alive = true;
       while (alive) {
-        alive = mbar_wait(&w_empty[slot], wphase ^ 1u, abort_flag);
+        alive = mbar_wait(w_empty + 8 * slot, wphase ^ 1u, abort_flag);
         if (!alive) break;
         int k = atomicAdd(a.work_counter, 1);
         if (k >= a.n_items) k = -1;
-        w_item[slot] = k;
-        mbar_arrive(&w_full[slot]);
+        sts_u32(w_item + 4 * slot, (uint32_t)k);
+        mbar_arrive(w_full + 8 * slot);
         if (++slot == kSchedSlots) { slot = 0; wphase ^= 1u; }
         if (k < 0) break;
         int bh, item;
@@ -405,23 +425,23 @@ __global__ void __launch_bounds__(kThreads, 1) sweep_kernel(const __grid_constan
           tiles = tx > tiles ? tx : tiles;
         }
         for (int t = 0; t < tiles && alive; ++t) {
-          alive = mbar_wait(&k_empty[stage], kphase ^ 1u, abort_flag);
+          alive = mbar_wait(k_empty + 8 * stage, kphase ^ 1u, abort_flag);
           if (!alive) break;
-          mbar_expect_tx(&k_full[stage], C::kKBytes);
+          mbar_expect_tx(k_full + 8 * stage, C::kKBytes);
           for (int hf = 0; hf < C::kHalves; ++hf)
-            tma_load_4d(k_smem + stage * C::kKBytes + hf * (BN * 128), &map_k, &k_full[stage], hf * 64, t * BN, h, b);
+            tma_load_4d(k_smem + stage * C::kKBytes + hf * (BN * 128), &map_k, k_full + 8 * stage, hf * 64, t * BN, h, b);
           if (++stage == C::kStages) { stage = 0; kphase ^= 1u; }
           if (t == 0) {
             // Q tile slots past the end of the sequence are neither loaded nor used; each slot keeps
             // its own phase bit so that producer and MMA issuer stay in step
             for (int x = 0; x < kQTiles && alive; ++x) {
               if (qtile_tiles(a, item, x) == 0) continue;
-              alive = mbar_wait(&q_empty[x], ((qphase >> x) & 1u) ^ 1u, abort_flag);
+              alive = mbar_wait(q_empty + 8 * x, ((qphase >> x) & 1u) ^ 1u, abort_flag);
               if (!alive) break;
               qphase ^= 1u << x;
-              mbar_expect_tx(&q_full[x], C::kQBytes);
+              mbar_expect_tx(q_full + 8 * x, C::kQBytes);
               for (int hf = 0; hf < C::kHalves; ++hf)
-                tma_load_4d(q_smem + x * C::kQBytes + hf * (BM * 128), &map_q, &q_full[x], hf * 64,
+                tma_load_4d(q_smem + x * C::kQBytes + hf * (BM * 128), &map_q, q_full + 8 * x, hf * 64,
                             item * kItemRows + x * BM, h, b);
             }
           }
@@ -432,15 +452,15 @@ __global__ void __launch_bounds__(kThreads, 1) sweep_kernel(const __grid_constan
     // ------------------------------------------------------------------ MMA issuer
     if (lane == 0) {
       constexpr uint32_t idesc = make_idesc();
-      const uint32_t q_lo = smem_desc_lo(smem_u32(q_smem)), k_lo = smem_desc_lo(smem_u32(k_smem));
+      const uint32_t q_lo = smem_desc_lo(q_smem), k_lo = smem_desc_lo(k_smem);
       int stage = 0, slot = 0;
       uint32_t kphase = 0, qphase = 0, wphase = 0, sphase[kQTiles] = {};
       bool alive = true;
       while (alive) {
-        alive = mbar_wait(&w_full[slot], wphase, abort_flag);
+        alive = mbar_wait(w_full + 8 * slot, wphase, abort_flag);
         if (!alive) break;
-        const int k = w_item[slot];
-        mbar_arrive(&w_empty[slot]);
+        const int k = (int)lds_u32(w_item + 4 * slot);
+        mbar_arrive(w_empty + 8 * slot);
         if (++slot == kSchedSlots) { slot = 0; wphase ^= 1u; }
         if (k < 0) break;
         int bh, item;
@@ -451,17 +471,17 @@ __global__ void __launch_bounds__(kThreads, 1) sweep_kernel(const __grid_constan
           tiles = tx[x] > tiles ? tx[x] : tiles;
         }
         for (int t = 0; t < tiles && alive; ++t) {
-          alive = mbar_wait(&k_full[stage], kphase, abort_flag);
+          alive = mbar_wait(k_full + 8 * stage, kphase, abort_flag);
           if (!alive) break;
           const uint32_t b_lo = k_lo + stage * (C::kKBytes >> 4);
 #pragma unroll
           for (int x = 0; x < kQTiles; ++x) {
             if (t >= tx[x] || !alive) continue;
             if (t == 0) {
-              alive = mbar_wait(&q_full[x], (qphase >> x) & 1u, abort_flag);
+              alive = mbar_wait(q_full + 8 * x, (qphase >> x) & 1u, abort_flag);
               qphase ^= 1u << x;
             }
-            if (alive) alive = mbar_wait(&s_empty[x], sphase[x] ^ 1u, abort_flag);
+            if (alive) alive = mbar_wait(s_empty + 8 * x, sphase[x] ^ 1u, abort_flag);
             if (!alive) continue;
             sphase[x] ^= 1u;
             tc_fence_after();
@@ -473,11 +493,11 @@ __global__ void __launch_bounds__(kThreads, 1) sweep_kernel(const __grid_constan
               const uint32_t b_off = (kk >> 2) * ((BN * 128) >> 4) + (kk & 3) * 2;
               umma_bf16(tmem_base + x * BN, a_lo + a_off, b_lo + b_off, kDescHi, idesc, kk > 0 ? 1u : 0u);
             }
-            umma_commit(&s_full[x]);
-            if (t == tx[x] - 1) umma_commit(&q_empty[x]);
+            umma_commit(s_full + 8 * x);
+            if (t == tx[x] - 1) umma_commit(q_empty + 8 * x);
           }
           if (!alive) break;
-          umma_commit(&k_empty[stage]);
+          umma_commit(k_empty + 8 * stage);
           if (++stage == C::kStages) { stage = 0; kphase ^= 1u; }
         }
       }
@@ -490,17 +510,18 @@ __global__ void __launch_bounds__(kThreads, 1) sweep_kernel(const __grid_constan
     const int quad = warp & 3;                     // TMEM lane quadrant this warp may read
     const int row_local = quad * 32 + lane;
     const uint32_t taddr_row = tmem_base + ((uint32_t)(quad * 32) << 16) + (uint32_t)(x * BN + half * kHalfCols);
-    volatile unsigned long long* my_share = m_share + (x * 2 + half) * BM + row_local;
-    volatile unsigned long long* other_share = m_share + (x * 2 + (half ^ 1)) * BM + row_local;
+    const uint32_t my_share = m_share + 8 * ((x * 2 + half) * BM + row_local);
+    const uint32_t other_share = m_share + 8 * ((x * 2 + (half ^ 1)) * BM + row_local);
+    const uint32_t my_full = s_full + 8 * x, my_empty = s_empty + 8 * x;
     uint32_t fphase = 0, wphase = 0;
     int slot = 0;
     bool alive = true;
     while (alive) {
-      alive = __all_sync(0xffffffffu, mbar_wait(&w_full[slot], wphase, abort_flag));
+      alive = __all_sync(0xffffffffu, mbar_wait(w_full + 8 * slot, wphase, abort_flag));
       if (!alive) break;
-      const int k = w_item[slot];
+      const int k = (int)lds_u32(w_item + 4 * slot);
       __syncwarp();
-      if (lane == 0) mbar_arrive(&w_empty[slot]);
+      if (lane == 0) mbar_arrive(w_empty + 8 * slot);
       if (++slot == kSchedSlots) { slot = 0; wphase ^= 1u; }
       if (k < 0) break;
       int bh, item;
@@ -541,7 +562,7 @@ __global__ void __launch_bounds__(kThreads, 1) sweep_kernel(const __grid_constan
       const int last_lim = a.causal ? (tile_row0 + BM - 1 < a.N - 1 ? tile_row0 + BM - 1 : a.N - 1) : a.N - 1;
       for (int t = 0; t < tiles && alive; ++t) {
         // the warp leaves together: tcgen05.ld needs all 32 lanes
-        alive = __all_sync(0xffffffffu, mbar_wait(&s_full[x], fphase, abort_flag));
+        alive = __all_sync(0xffffffffu, mbar_wait(my_full, fphase, abort_flag));
         if (!alive) break;
         fphase ^= 1u;
         tc_fence_after();
@@ -579,11 +600,11 @@ __global__ void __launch_bounds__(kThreads, 1) sweep_kernel(const __grid_constan
           m_tile = fmaxf(m_tile, g[15]);
           if (searching) {
             // the other half's running maximum (if it already belongs to this item) tightens the bound too
-            const unsigned long long o = *other_share;
+            const unsigned long long o = lds_u64(other_share);
             const float m_other = (int)(o >> 32) == k ? __uint_as_float((unsigned)o) : -INFINITY;
             r.m_run = max3(r.m_run, m_tile, m_other);
             if (r.cnt >= 0) r.thr = fmaxf(r.thr, r.m_run - inv_a);
-            *my_share = ((unsigned long long)(unsigned)k << 32) | __float_as_uint(r.m_run);
+            sts_u64(my_share, ((unsigned long long)(unsigned)k << 32) | __float_as_uint(r.m_run));
           }
           // ---- pass 2 (only when some lane saw a candidate): re-read the groups that hold one
           const bool hit = m_tile > r.thr;
@@ -609,7 +630,7 @@ __global__ void __launch_bounds__(kThreads, 1) sweep_kernel(const __grid_constan
                 // the last batch is in registers: hand the accumulator back before the list stores
                 tc_fence_before();
                 __syncwarp();
-                if (lane == 0) mbar_arrive(&s_empty[x]);
+                if (lane == 0) mbar_arrive(my_empty);
                 released = true;
               }
               if (masked) {
@@ -627,8 +648,8 @@ __global__ void __launch_bounds__(kThreads, 1) sweep_kernel(const __grid_constan
 #pragma unroll
                   for (int e = 0; e < 8; ++e) {
                     if (v8[w][e] > thr) {
-                      list[cnt].y = v8[w][e];
-                      list[cnt].j = col_base + gu[w] * 8 + e;
+                      *reinterpret_cast<uint2*>(&list[cnt]) =
+                          make_uint2(__float_as_uint(v8[w][e]), (unsigned)(col_base + gu[w] * 8 + e));
                       ++cnt;
                     }
                   }
@@ -637,7 +658,7 @@ __global__ void __launch_bounds__(kThreads, 1) sweep_kernel(const __grid_constan
               }
               // at most 32 entries were appended since the last check: the half-list cannot overflow
               const unsigned need = __ballot_sync(0xffffffffu, r.cnt > kHalfTrigger);
-              if (need) shrink_lists(r, list, ra, inv_a, need, a.mode, a.expo_class, a.expo);
+              if (need) r = shrink_lists(r, list, ra, inv_a, need, a.mode, a.expo_class, a.expo);
             }
           }
         }
@@ -645,7 +666,7 @@ __global__ void __launch_bounds__(kThreads, 1) sweep_kernel(const __grid_constan
         if (!released) {
           tc_fence_before();
           __syncwarp();
-          if (lane == 0) mbar_arrive(&s_empty[x]);
+          if (lane == 0) mbar_arrive(my_empty);
         }
       }
       if (valid && alive) {
@@ -658,7 +679,7 @@ __global__ void __launch_bounds__(kThreads, 1) sweep_kernel(const __grid_constan
   // ---------------------------------------------------------------------- teardown
   tc_fence_before();
   __syncthreads();
-  if (*abort_flag) {
+  if (lds_u32(abort_flag)) {
     if (threadIdx.x == 0 && a.status) atomicOr(a.status + ENTMAX_ATTN_STATUS_FLAGS, ENTMAX_ATTN_FLAG_WAIT_EXPIRED);
     // give copies and MMAs that may still be in flight time to land before shared memory and TMEM go away
     const uint64_t t0 = global_ns();
