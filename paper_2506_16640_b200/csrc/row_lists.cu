@@ -64,12 +64,139 @@ __device__ __forceinline__ void push_dense_row(int grow, int32_t* fb_count, int3
   if (status) atomicAdd(status + ENTMAX_ATTN_STATUS_DENSE_ROWS, 1);
 }
 
+// Bitonic sort of 32*S (key j, value y) pairs held as S registers per lane (element index = 32*s + lane),
+// ascending by key.  Keys are distinct key indices (padding uses INT_MAX and sorts to the end).
+template <int S>
+__device__ __forceinline__ void sort_by_key(int (&jj)[S], float (&y)[S], int lane) {
+#pragma unroll
+  for (int k = 2; k <= 32 * S; k <<= 1) {
+#pragma unroll
+    for (int st = k >> 1; st > 0; st >>= 1) {
+      if (st >= 32) {
+        // partner sits in another register of the same lane
+#pragma unroll
+        for (int s = 0; s < S; ++s) {
+          const int ps = s ^ (st >> 5);
+          if (ps > s) {
+            const bool up = (((32 * s) & k) == 0);
+            const bool swap = up ? (jj[s] > jj[ps]) : (jj[s] < jj[ps]);
+            const int tj = swap ? jj[ps] : jj[s];
+            const float ty = swap ? y[ps] : y[s];
+            jj[ps] = swap ? jj[s] : jj[ps];
+            y[ps] = swap ? y[s] : y[ps];
+            jj[s] = tj;
+            y[s] = ty;
+          }
+        }
+      } else {
+#pragma unroll
+        for (int s = 0; s < S; ++s) {
+          const int idx = 32 * s + lane;
+          const int oj = __shfl_xor_sync(0xffffffffu, jj[s], st);
+          const float oy = __shfl_xor_sync(0xffffffffu, y[s], st);
+          const bool up = ((idx & k) == 0);
+          const bool lower = ((lane & st) == 0);
+          // the lower index keeps the smaller key when sorting upwards, the larger one otherwise
+          const bool take_other = (lower == up) ? (oj < jj[s]) : (oj > jj[s]);
+          jj[s] = take_other ? oj : jj[s];
+          y[s] = take_other ? oy : y[s];
+        }
+      }
+    }
+  }
+}
+
+// One query row on S*32 candidate slots: exact threshold (Eq. 1 with the sum-to-one condition), the
+// probabilities, O_i as a gather over the support, and the support written back sorted by key index.
+// The candidates are sorted by key index first and Newton starts at the bracket's lower end
+// (App. A: tau >= y_max - 1), so the result does not depend on the order or on the surplus entries
+// the sweep happened to leave in the lists.
+template <int D, int S>
+__device__ __forceinline__ void solve_row(const Problem& p, const __nv_bfloat16* __restrict__ vbase, Entry* list, int c0,
+                                          int c1, float a, __nv_bfloat16* o_row, float* tau_slot, int32_t* cnt_slot,
+                                          int lane) {
+  constexpr int PER = D / 32;
+  float y[S];
+  int jj[S];
+  float ymax = -INFINITY;
+#pragma unroll
+  for (int s = 0; s < S; ++s) {
+    const int e = lane + 32 * s;                   // dense numbering: first half-list, then second
+    y[s] = -INFINITY;
+    jj[s] = 0x7fffffff;
+    if (e < c0 + c1) {
+      const Entry en = list[e < c0 ? e : kHalfCap + e - c0];
+      y[s] = a * en.y;
+      jj[s] = en.j;
+    }
+    ymax = fmaxf(ymax, y[s]);
+  }
+  ymax = warp_max(ymax);
+  __syncwarp();   // every slot is in registers before the compaction below overwrites the list
+  sort_by_key<S>(jj, y, lane);
+  float tau = ymax - 1.0f;
+  for (int it = 0; it < kMaxNewton; ++it) {
+    float s0 = 0.f, s1 = 0.f;
+#pragma unroll
+    for (int s = 0; s < S; ++s) {
+      const float d = y[s] - tau;
+      if (d > 0.f) {
+        float ye, ye1;
+        pow_pair(d, p.expo_class, p.expo, ye, ye1);
+        s0 += ye;
+        s1 += ye1;
+      }
+    }
+    s0 = warp_sum(s0);
+    s1 = warp_sum(s1);
+    if (!(s0 > 1.0f) || !(s1 > 0.f)) break;
+    const float step = (s0 - 1.0f) / (p.expo * s1);
+    const float next = tau + step;
+    if (!(next > tau)) break;
+    tau = next;
+    if (step <= 1e-7f * fmaxf(1.0f, fabsf(tau))) break;
+  }
+  float acc[PER];
+#pragma unroll
+  for (int t = 0; t < PER; ++t) acc[t] = 0.f;
+  int kept = 0;
+#pragma unroll
+  for (int s = 0; s < S; ++s) {
+    const float d = y[s] - tau;
+    float pe = 0.f, pe1;
+    if (d > 0.f) pow_pair(d, p.expo_class, p.expo, pe, pe1);
+    const unsigned m = __ballot_sync(0xffffffffu, d > 0.f);
+    // compact the list to the exact support, y in Eq. 1's units
+    if (d > 0.f) {
+      const int pos = kept + __popc(m & ((1u << lane) - 1u));
+      list[pos].y = y[s];
+      list[pos].j = jj[s];
+    }
+    kept += __popc(m);
+    unsigned rest = m;
+    while (rest) {
+      const int src = __ffs(rest) - 1;
+      rest &= rest - 1;
+      const float pj = __shfl_sync(0xffffffffu, pe, src);
+      const int kj = __shfl_sync(0xffffffffu, jj[s], src);
+      float vs[PER];
+      load_bf16<PER>(vbase + (size_t)kj * p.sn, vs);
+#pragma unroll
+      for (int t = 0; t < PER; ++t) acc[t] = fmaf(pj, vs[t], acc[t]);
+    }
+  }
+  store_bf16<PER>(o_row, acc);
+  if (lane == 0) {
+    *tau_slot = tau;
+    *cnt_slot = kept;
+  }
+}
+
 template <int D>
 __global__ void __launch_bounds__(kWarpsPerCta * 32) row_fwd_kernel(Problem p, const __nv_bfloat16* __restrict__ v,
                                                                     const float* __restrict__ scale,
                                                                     int32_t* __restrict__ row_cnt,
                                                                     const int32_t* __restrict__ half_cnt,
-                                                                    const float* __restrict__ half_thr,
                                                                     Entry* __restrict__ entries,
                                                                     __nv_bfloat16* __restrict__ o,
                                                                     float* __restrict__ tau_out, int32_t* fb_count,
@@ -89,83 +216,13 @@ __global__ void __launch_bounds__(kWarpsPerCta * 32) row_fwd_kernel(Problem p, c
     const int bh = grow / p.N, i = grow - bh * p.N, b = bh / p.H, h = bh - b * p.H;
     const float a = (p.alpha - 1.0f) * (scale[(size_t)h * p.N + i] * p.sm_scale);
     Entry* list = entries + (size_t)grow * kListCap;
-    float y[kSlots];
-    int jj[kSlots];
-    float ymax = -INFINITY;
-#pragma unroll
-    for (int s = 0; s < kSlots; ++s) {
-      const int idx = lane + 32 * s;                 // slot; half idx / kHalfCap owns it
-      y[s] = -INFINITY;
-      jj[s] = 0;
-      if ((idx & (kHalfCap - 1)) < (idx < kHalfCap ? c0 : c1)) {
-        const Entry e = list[idx];
-        y[s] = a * e.y;
-        jj[s] = e.j;
-      }
-      ymax = fmaxf(ymax, y[s]);
-    }
-    ymax = warp_max(ymax);
-    // both half-row bounds and the bracket's lower end are lower bounds on the threshold
-    float tau = fmaxf(fmaxf(half_thr[2 * (size_t)grow], half_thr[2 * (size_t)grow + 1]), ymax - 1.0f);
-    __syncwarp();   // every slot is in registers before the compaction below overwrites the list
-    for (int it = 0; it < kMaxNewton; ++it) {
-      float s0 = 0.f, s1 = 0.f;
-#pragma unroll
-      for (int s = 0; s < kSlots; ++s) {
-        const float d = y[s] - tau;
-        if (d > 0.f) {
-          float ye, ye1;
-          pow_pair(d, p.expo_class, p.expo, ye, ye1);
-          s0 += ye;
-          s1 += ye1;
-        }
-      }
-      s0 = warp_sum(s0);
-      s1 = warp_sum(s1);
-      if (!(s0 > 1.0f) || !(s1 > 0.f)) break;
-      const float step = (s0 - 1.0f) / (p.expo * s1);
-      const float next = tau + step;
-      if (!(next > tau)) break;
-      tau = next;
-      if (step <= 1e-7f * fmaxf(1.0f, fabsf(tau))) break;
-    }
-    float pv[kSlots];
-    float acc[PER];
-#pragma unroll
-    for (int t = 0; t < PER; ++t) acc[t] = 0.f;
     const __nv_bfloat16* vbase = v + (size_t)b * p.sb + (size_t)h * p.sh + lane * PER;
-    int kept = 0;
-#pragma unroll
-    for (int s = 0; s < kSlots; ++s) {
-      const float d = y[s] - tau;
-      float pe = 0.f, pe1;
-      if (d > 0.f) pow_pair(d, p.expo_class, p.expo, pe, pe1);
-      pv[s] = pe;
-      const unsigned m = __ballot_sync(0xffffffffu, d > 0.f);
-      // compact the list to the exact support, y in Eq. 1's units
-      if (d > 0.f) {
-        const int pos = kept + __popc(m & ((1u << lane) - 1u));
-        list[pos].y = y[s];
-        list[pos].j = jj[s];
-      }
-      kept += __popc(m);
-      unsigned rest = m;
-      while (rest) {
-        const int src = __ffs(rest) - 1;
-        rest &= rest - 1;
-        const float pj = __shfl_sync(0xffffffffu, pv[s], src);
-        const int kj = __shfl_sync(0xffffffffu, jj[s], src);
-        float vs[PER];
-        load_bf16<PER>(vbase + (size_t)kj * p.sn, vs);
-#pragma unroll
-        for (int t = 0; t < PER; ++t) acc[t] = fmaf(pj, vs[t], acc[t]);
-      }
-    }
-    store_bf16<PER>(o + (size_t)b * p.sb + (size_t)h * p.sh + (size_t)i * p.sn + lane * PER, acc);
-    if (lane == 0) {
-      tau_out[grow] = tau;
-      row_cnt[grow] = kept;
-    }
+    __nv_bfloat16* o_row = o + (size_t)b * p.sb + (size_t)h * p.sh + (size_t)i * p.sn + lane * PER;
+    const int n = c0 + c1;
+    if (n <= 32) solve_row<D, 1>(p, vbase, list, c0, c1, a, o_row, tau_out + grow, row_cnt + grow, lane);
+    else if (n <= 64) solve_row<D, 2>(p, vbase, list, c0, c1, a, o_row, tau_out + grow, row_cnt + grow, lane);
+    else if (n <= 128) solve_row<D, 4>(p, vbase, list, c0, c1, a, o_row, tau_out + grow, row_cnt + grow, lane);
+    else solve_row<D, kSlots>(p, vbase, list, c0, c1, a, o_row, tau_out + grow, row_cnt + grow, lane);
   }
 }
 
@@ -282,10 +339,10 @@ cudaError_t launch_row_fwd(const Problem& p, const void* v, const float* scale, 
                            int32_t* fb_count, int32_t* fb_list, int32_t* status, cudaStream_t stream) {
   const int grid = row_grid(p);
   if (p.D == 64)
-    row_fwd_kernel<64><<<grid, kWarpsPerCta * 32, 0, stream>>>(p, (const __nv_bfloat16*)v, scale, row_cnt, half_cnt, half_thr,
+    row_fwd_kernel<64><<<grid, kWarpsPerCta * 32, 0, stream>>>(p, (const __nv_bfloat16*)v, scale, row_cnt, half_cnt,
                                                               entries, (__nv_bfloat16*)o, tau, fb_count, fb_list, status);
   else
-    row_fwd_kernel<128><<<grid, kWarpsPerCta * 32, 0, stream>>>(p, (const __nv_bfloat16*)v, scale, row_cnt, half_cnt, half_thr,
+    row_fwd_kernel<128><<<grid, kWarpsPerCta * 32, 0, stream>>>(p, (const __nv_bfloat16*)v, scale, row_cnt, half_cnt,
                                                                entries, (__nv_bfloat16*)o, tau, fb_count, fb_list, status);
   return cudaGetLastError();
 }
