@@ -192,14 +192,17 @@ __device__ __forceinline__ void umma_commit(uint32_t bar) {
                : "memory");
 }
 
-// 32 lanes x 16 (or 8) consecutive fp32 columns: thread t of the warp gets lane (base + t)
-__device__ __forceinline__ void tmem_ld16(uint32_t taddr, float (&r)[16]) {
+// 32 lanes x 32 (or 8) consecutive fp32 columns: thread t of the warp gets lane (base + t)
+__device__ __forceinline__ void tmem_ld32(uint32_t taddr, float (&r)[32]) {
   uint32_t* u = reinterpret_cast<uint32_t*>(r);
   asm volatile(
-      "tcgen05.ld.sync.aligned.32x32b.x16.b32 "
-      "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15}, [%16];"
+      "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
+      "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
+      "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];"
       : "=r"(u[0]), "=r"(u[1]), "=r"(u[2]), "=r"(u[3]), "=r"(u[4]), "=r"(u[5]), "=r"(u[6]), "=r"(u[7]), "=r"(u[8]),
-        "=r"(u[9]), "=r"(u[10]), "=r"(u[11]), "=r"(u[12]), "=r"(u[13]), "=r"(u[14]), "=r"(u[15])
+        "=r"(u[9]), "=r"(u[10]), "=r"(u[11]), "=r"(u[12]), "=r"(u[13]), "=r"(u[14]), "=r"(u[15]), "=r"(u[16]),
+        "=r"(u[17]), "=r"(u[18]), "=r"(u[19]), "=r"(u[20]), "=r"(u[21]), "=r"(u[22]), "=r"(u[23]), "=r"(u[24]),
+        "=r"(u[25]), "=r"(u[26]), "=r"(u[27]), "=r"(u[28]), "=r"(u[29]), "=r"(u[30]), "=r"(u[31])
       : "r"(taddr)
       : "memory");
 }
@@ -570,29 +573,27 @@ __global__ void __launch_bounds__(kThreads, 1) sweep_kernel(const __grid_constan
         bool released = false;
         if (col_base <= last_lim) {
           const bool masked = col_base + kHalfCols - 1 > first_lim;
-          // ---- pass 1: 128 columns -> 16 group maxima (8 columns each)
+          // ---- pass 1: 128 columns -> 16 group maxima (8 columns each); four loads of 32 columns (wider
+          //      loads mean fewer TMEM round trips on the path that holds the accumulator)
           float g[16];
-          float va[16], vb[16];
-          tmem_ld16(taddr_row, va);
+          float va[32];
 #pragma unroll
-          for (int c = 0; c < kHalfCols / 16; ++c) {
-            float (&cur)[16] = (c & 1) ? vb : va;
-            float (&nxt)[16] = (c & 1) ? va : vb;
+          for (int c = 0; c < 4; ++c) {
+            tmem_ld32(taddr_row + c * 32, va);
             tmem_ld_wait();
-            if (c + 1 < kHalfCols / 16) tmem_ld16(taddr_row + (c + 1) * 16, nxt);   // in flight during the maxima
             if (kDump) {
               if (dump_here) {
 #pragma unroll
-                for (int u = 0; u < 16; ++u)
-                  if (col_base + c * 16 + u <= lim) a.dump[(size_t)i * a.N + col_base + c * 16 + u] = cur[u];
+                for (int u = 0; u < 32; ++u)
+                  if (col_base + c * 32 + u <= lim) a.dump[(size_t)i * a.N + col_base + c * 32 + u] = va[u];
               }
             }
             if (masked) {
 #pragma unroll
-              for (int u = 0; u < 16; ++u) cur[u] = (col_base + c * 16 + u <= lim) ? cur[u] : -INFINITY;
+              for (int u = 0; u < 32; ++u) va[u] = (col_base + c * 32 + u <= lim) ? va[u] : -INFINITY;
             }
-            g[2 * c] = max8(&cur[0]);
-            g[2 * c + 1] = max8(&cur[8]);
+#pragma unroll
+            for (int q = 0; q < 4; ++q) g[4 * c + q] = max8(&va[8 * q]);
           }
           float m_tile = max3(g[0], g[1], g[2]);
 #pragma unroll
