@@ -1,5 +1,7 @@
 // Per-row kernels of the bf16 path that work on the sparse candidate lists left by the tensor-core
-// score sweep (two half-lists per row, see common.cuh): one warp per query row.
+// score sweep (two half-lists per row, see common.cuh).  A warp takes four consecutive query rows: when
+// all four have at most eight list entries (the common case on sparse rows) eight lanes work on each
+// row at the same time, otherwise the warp takes the rows one after the other with all 32 lanes.
 //
 // Forward: exact threshold on the candidates (Eq. 1 with the sum-to-one condition; Newton from the
 // left of the root, see dense_rows.cu), probabilities, and O_i = sum_j p_ij v_j as a gather over the
@@ -58,6 +60,55 @@ __device__ __forceinline__ void atomic_add_slice(float* p, const float (&x)[PER]
   else atomicAdd(reinterpret_cast<float4*>(p), make_float4(x[0], x[1], x[2], x[3]));
 }
 
+
+// reductions over aligned groups of eight lanes
+__device__ __forceinline__ float oct_sum(float x) {
+  x += __shfl_xor_sync(0xffffffffu, x, 1);
+  x += __shfl_xor_sync(0xffffffffu, x, 2);
+  x += __shfl_xor_sync(0xffffffffu, x, 4);
+  return x;
+}
+__device__ __forceinline__ float oct_max(float x) {
+  x = fmaxf(x, __shfl_xor_sync(0xffffffffu, x, 1));
+  x = fmaxf(x, __shfl_xor_sync(0xffffffffu, x, 2));
+  x = fmaxf(x, __shfl_xor_sync(0xffffffffu, x, 4));
+  return x;
+}
+// N consecutive bf16 (N = 8 or 16, 16-byte aligned) <-> floats
+template <int N>
+__device__ __forceinline__ void load_bf16_vec(const __nv_bfloat16* p, float (&x)[N]) {
+#pragma unroll
+  for (int c = 0; c < N / 8; ++c) {
+    const uint4 raw = *reinterpret_cast<const uint4*>(p + 8 * c);
+    const uint32_t w[4] = {raw.x, raw.y, raw.z, raw.w};
+#pragma unroll
+    for (int t = 0; t < 4; ++t) {
+      const float2 f = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(&w[t]));
+      x[8 * c + 2 * t] = f.x;
+      x[8 * c + 2 * t + 1] = f.y;
+    }
+  }
+}
+template <int N>
+__device__ __forceinline__ void store_bf16_vec(__nv_bfloat16* p, const float (&x)[N]) {
+#pragma unroll
+  for (int c = 0; c < N / 8; ++c) {
+    uint32_t w[4];
+#pragma unroll
+    for (int t = 0; t < 4; ++t) {
+      const __nv_bfloat162 h = __floats2bfloat162_rn(x[8 * c + 2 * t], x[8 * c + 2 * t + 1]);
+      w[t] = *reinterpret_cast<const uint32_t*>(&h);
+    }
+    *reinterpret_cast<uint4*>(p + 8 * c) = make_uint4(w[0], w[1], w[2], w[3]);
+  }
+}
+template <int N>
+__device__ __forceinline__ void atomic_add_vec(float* p, const float (&x)[N]) {
+#pragma unroll
+  for (int c = 0; c < N / 4; ++c)
+    atomicAdd(reinterpret_cast<float4*>(p + 4 * c), make_float4(x[4 * c], x[4 * c + 1], x[4 * c + 2], x[4 * c + 3]));
+}
+
 __device__ __forceinline__ void push_dense_row(int grow, int32_t* fb_count, int32_t* fb_list, int32_t* status) {
   const int slot = atomicAdd(fb_count, 1);
   fb_list[slot] = grow;
@@ -106,35 +157,18 @@ __device__ __forceinline__ void sort_by_key(int (&jj)[S], float (&y)[S], int lan
   }
 }
 
-// One query row on S*32 candidate slots: exact threshold (Eq. 1 with the sum-to-one condition), the
-// probabilities, O_i as a gather over the support, and the support written back sorted by key index.
-// The candidates are sorted by key index first and Newton starts at the bracket's lower end
-// (App. A: tau >= y_max - 1), so the result does not depend on the order or on the surplus entries
-// the sweep happened to leave in the lists.
-template <int D, int S>
-__device__ __forceinline__ void solve_row(const Problem& p, const __nv_bfloat16* __restrict__ vbase, Entry* list, int c0,
-                                          int c1, float a, __nv_bfloat16* o_row, float* tau_slot, int32_t* cnt_slot,
-                                          int lane) {
-  constexpr int PER = D / 32;
-  float y[S];
-  int jj[S];
-  float ymax = -INFINITY;
-#pragma unroll
-  for (int s = 0; s < S; ++s) {
-    const int e = lane + 32 * s;                   // dense numbering: first half-list, then second
-    y[s] = -INFINITY;
-    jj[s] = 0x7fffffff;
-    if (e < c0 + c1) {
-      const Entry en = list[e < c0 ? e : kHalfCap + e - c0];
-      y[s] = a * en.y;
-      jj[s] = en.j;
-    }
-    ymax = fmaxf(ymax, y[s]);
-  }
-  ymax = warp_max(ymax);
-  __syncwarp();   // every slot is in registers before the compaction below overwrites the list
-  sort_by_key<S>(jj, y, lane);
-  float tau = ymax - 1.0f;
+// The forward row solve runs in two stages so that its result does not depend on what else the sweep
+// happened to leave in the lists (their order and their surplus entries vary from run to run):
+//   stage A  Newton on all candidates, in list order -> tau_A, accurate to fp32 rounding;
+//   stage B  the entries above tau_A minus a small margin are compacted and sorted by key index, and
+//            Newton runs again on this set alone, from the bracket's lower end (App. A: tau >= y_max - 1);
+//            its summation order is fixed by the sorted set, so O and tau come out bit-identical
+//            unless an entry lies within rounding noise of the margin cut.
+constexpr float kKeepMargin = 4e-6f;
+
+// Newton from the left on f(tau) = sum [y - tau]_+^e - 1 (convex, decreasing: monotone, never overshoots)
+template <int S>
+__device__ __forceinline__ float newton_warp(const Problem& p, const float (&y)[S], float tau) {
   for (int it = 0; it < kMaxNewton; ++it) {
     float s0 = 0.f, s1 = 0.f;
 #pragma unroll
@@ -156,6 +190,74 @@ __device__ __forceinline__ void solve_row(const Problem& p, const __nv_bfloat16*
     tau = next;
     if (step <= 1e-7f * fmaxf(1.0f, fabsf(tau))) break;
   }
+  return tau;
+}
+
+// Stage A on S*32 candidate slots.  Leaves the kept entries (y in Eq. 1's units) compacted from slot 0
+// of the row's list and returns how many there are.
+template <int S>
+__device__ __forceinline__ int prefilter_row(const Problem& p, Entry* list, int c0, int c1, float a, int lane) {
+  float y[S];
+  int jj[S];
+  float ymax = -INFINITY;
+#pragma unroll
+  for (int s = 0; s < S; ++s) {
+    const int e = lane + 32 * s;                   // dense numbering: first half-list, then second
+    y[s] = -INFINITY;
+    jj[s] = 0x7fffffff;
+    if (e < c0 + c1) {
+      const Entry en = list[e < c0 ? e : kHalfCap + e - c0];
+      y[s] = a * en.y;
+      jj[s] = en.j;
+    }
+    ymax = fmaxf(ymax, y[s]);
+  }
+  ymax = warp_max(ymax);
+  __syncwarp();   // every slot is in registers before the list is overwritten
+  const float tau_a = newton_warp<S>(p, y, ymax - 1.0f);
+  const float cut = tau_a - kKeepMargin * fmaxf(1.0f, fabsf(tau_a));
+  int kept = 0;
+#pragma unroll
+  for (int s = 0; s < S; ++s) {
+    const bool keep = y[s] > cut;
+    const unsigned m = __ballot_sync(0xffffffffu, keep);
+    if (keep) {
+      const int pos = kept + __popc(m & ((1u << lane) - 1u));
+      list[pos].y = y[s];
+      list[pos].j = jj[s];
+    }
+    kept += __popc(m);
+  }
+  __syncwarp();
+  return kept;
+}
+
+// Stage B on the `kept` compacted entries (kept <= 32*S): sort by key index, threshold, probabilities,
+// O_i as a gather over the support, support written back sorted by key index.
+template <int D, int S>
+__device__ __forceinline__ void finish_row(const Problem& p, const __nv_bfloat16* __restrict__ vbase, Entry* list,
+                                           int kept_in, __nv_bfloat16* o_row, float* tau_slot, int32_t* cnt_slot,
+                                           int lane) {
+  constexpr int PER = D / 32;
+  float y[S];
+  int jj[S];
+  float ymax = -INFINITY;
+#pragma unroll
+  for (int s = 0; s < S; ++s) {
+    const int e = lane + 32 * s;
+    y[s] = -INFINITY;
+    jj[s] = 0x7fffffff;
+    if (e < kept_in) {
+      const Entry en = list[e];
+      y[s] = en.y;
+      jj[s] = en.j;
+    }
+    ymax = fmaxf(ymax, y[s]);
+  }
+  ymax = warp_max(ymax);
+  __syncwarp();
+  sort_by_key<S>(jj, y, lane);
+  const float tau = newton_warp<S>(p, y, ymax - 1.0f);
   float acc[PER];
 #pragma unroll
   for (int t = 0; t < PER; ++t) acc[t] = 0.f;
@@ -166,7 +268,6 @@ __device__ __forceinline__ void solve_row(const Problem& p, const __nv_bfloat16*
     float pe = 0.f, pe1;
     if (d > 0.f) pow_pair(d, p.expo_class, p.expo, pe, pe1);
     const unsigned m = __ballot_sync(0xffffffffu, d > 0.f);
-    // compact the list to the exact support, y in Eq. 1's units
     if (d > 0.f) {
       const int pos = kept + __popc(m & ((1u << lane) - 1u));
       list[pos].y = y[s];
@@ -192,6 +293,131 @@ __device__ __forceinline__ void solve_row(const Problem& p, const __nv_bfloat16*
   }
 }
 
+// One row with the whole warp.
+template <int D>
+__device__ __forceinline__ void solve_row_full(const Problem& p, const __nv_bfloat16* __restrict__ vbase, Entry* list,
+                                               int c0, int c1, float a, __nv_bfloat16* o_row, float* tau_slot,
+                                               int32_t* cnt_slot, int lane) {
+  const int n = c0 + c1;
+  int kept;
+  if (n <= 32) kept = prefilter_row<1>(p, list, c0, c1, a, lane);
+  else if (n <= 64) kept = prefilter_row<2>(p, list, c0, c1, a, lane);
+  else if (n <= 128) kept = prefilter_row<4>(p, list, c0, c1, a, lane);
+  else kept = prefilter_row<kSlots>(p, list, c0, c1, a, lane);
+  if (kept <= 32) finish_row<D, 1>(p, vbase, list, kept, o_row, tau_slot, cnt_slot, lane);
+  else if (kept <= 64) finish_row<D, 2>(p, vbase, list, kept, o_row, tau_slot, cnt_slot, lane);
+  else if (kept <= 128) finish_row<D, 4>(p, vbase, list, kept, o_row, tau_slot, cnt_slot, lane);
+  else finish_row<D, kSlots>(p, vbase, list, kept, o_row, tau_slot, cnt_slot, lane);
+}
+
+// Newton for four rows at once (eight lanes per row); `done` rows keep their tau.
+__device__ __forceinline__ float newton_oct(const Problem& p, float y, float tau, bool done) {
+  for (int it = 0; it < kMaxNewton; ++it) {
+    const float d = y - tau;
+    float ye = 0.f, ye1 = 0.f;
+    if (d > 0.f) pow_pair(d, p.expo_class, p.expo, ye, ye1);
+    const float s0 = oct_sum(ye), s1 = oct_sum(ye1);
+    if (!done) {
+      if (!(s0 > 1.0f) || !(s1 > 0.f)) {
+        done = true;
+      } else {
+        const float step = (s0 - 1.0f) / (p.expo * s1);
+        const float next = tau + step;
+        if (!(next > tau)) {
+          done = true;
+        } else {
+          tau = next;
+          if (step <= 1e-7f * fmaxf(1.0f, fabsf(tau))) done = true;
+        }
+      }
+    }
+    if (__all_sync(0xffffffffu, done)) break;
+  }
+  return tau;
+}
+
+// Four rows at once, eight lanes per row, for rows with 1..8 list entries; same two stages.
+template <int D>
+__device__ __forceinline__ void solve_rows_quad(const Problem& p, const __nv_bfloat16* __restrict__ v,
+                                                const float* __restrict__ scale, Entry* __restrict__ entries,
+                                                __nv_bfloat16* __restrict__ o, float* __restrict__ tau_out,
+                                                int32_t* __restrict__ row_cnt, int grow, bool active, int c0, int c1,
+                                                int lane) {
+  constexpr int PL = D / 8;                        // elements of a V / O row per lane
+  const int sl = lane & 7;
+  const int base = lane & 24;
+  const int n = active ? c0 + c1 : 0;
+  const int bh = grow / p.N, i = grow - bh * p.N, b = bh / p.H, h = bh - b * p.H;
+  const float a = active ? (p.alpha - 1.0f) * (scale[(size_t)h * p.N + i] * p.sm_scale) : 1.0f;
+  Entry* list = entries + (size_t)grow * kListCap;
+  float y = -INFINITY;
+  int j = 0x7fffffff;
+  if (sl < n) {
+    const Entry en = list[sl < c0 ? sl : kHalfCap + sl - c0];
+    y = a * en.y;
+    j = en.j;
+  }
+  __syncwarp();   // every entry is in registers before the compaction below overwrites the lists
+  // stage A
+  const float tau_a = newton_oct(p, y, oct_max(y) - 1.0f, !active);
+  const bool keep = active && y > tau_a - kKeepMargin * fmaxf(1.0f, fabsf(tau_a));
+  // keep only those: they move to the end-stable front when sorted with the others' keys pushed to infinity
+  j = keep ? j : 0x7fffffff;
+  y = keep ? y : -INFINITY;
+  // bitonic sort of the eight (j, y) pairs of each row, ascending by key index
+#pragma unroll
+  for (int k = 2; k <= 8; k <<= 1) {
+#pragma unroll
+    for (int st = k >> 1; st > 0; st >>= 1) {
+      const int oj = __shfl_xor_sync(0xffffffffu, j, st);
+      const float oy = __shfl_xor_sync(0xffffffffu, y, st);
+      const bool up = ((sl & k) == 0);
+      const bool lower = ((sl & st) == 0);
+      const bool take_other = (lower == up) ? (oj < j) : (oj > j);
+      j = take_other ? oj : j;
+      y = take_other ? oy : y;
+    }
+  }
+  // stage B
+  const float tau = newton_oct(p, y, oct_max(y) - 1.0f, !active);
+  const float d = y - tau;
+  const bool in = active && d > 0.f;
+  float pe = 0.f, pe1;
+  if (in) pow_pair(d, p.expo_class, p.expo, pe, pe1);
+  const unsigned m = __ballot_sync(0xffffffffu, in);
+  const unsigned msub = (m >> base) & 0xffu;
+  if (in) {
+    // compact the list to the exact support, y in Eq. 1's units
+    const int pos = __popc(msub & ((1u << sl) - 1u));
+    list[pos].y = y;
+    list[pos].j = j;
+  }
+  float acc[PL];
+#pragma unroll
+  for (int t = 0; t < PL; ++t) acc[t] = 0.f;
+  const __nv_bfloat16* vbase = v + (size_t)b * p.sb + (size_t)h * p.sh + sl * PL;
+#pragma unroll
+  for (int t = 0; t < 8; ++t) {
+    const bool has = (msub >> t) & 1u;
+    if (!__any_sync(0xffffffffu, has)) continue;
+    const float pj = __shfl_sync(0xffffffffu, pe, base + t);
+    const int kj = __shfl_sync(0xffffffffu, j, base + t);
+    if (has) {
+      float vs[PL];
+      load_bf16_vec<PL>(vbase + (size_t)kj * p.sn, vs);
+#pragma unroll
+      for (int u = 0; u < PL; ++u) acc[u] = fmaf(pj, vs[u], acc[u]);
+    }
+  }
+  if (active) {
+    store_bf16_vec<PL>(o + (size_t)b * p.sb + (size_t)h * p.sh + (size_t)i * p.sn + sl * PL, acc);
+    if (sl == 0) {
+      tau_out[grow] = tau;
+      row_cnt[grow] = __popc(msub);
+    }
+  }
+}
+
 template <int D>
 __global__ void __launch_bounds__(kWarpsPerCta * 32) row_fwd_kernel(Problem p, const __nv_bfloat16* __restrict__ v,
                                                                     const float* __restrict__ scale,
@@ -204,25 +430,40 @@ __global__ void __launch_bounds__(kWarpsPerCta * 32) row_fwd_kernel(Problem p, c
   constexpr int PER = D / 32;
   const int lane = threadIdx.x & 31;
   const int total = p.B * p.H * p.N;
-  for (int grow = blockIdx.x * kWarpsPerCta + (threadIdx.x >> 5); grow < total; grow += gridDim.x * kWarpsPerCta) {
-    const int c0 = half_cnt[2 * (size_t)grow], c1 = half_cnt[2 * (size_t)grow + 1];
-    if (c0 < 0 || c1 < 0 || c0 + c1 == 0) {
-      if (lane == 0) {
-        row_cnt[grow] = -2;
-        push_dense_row(grow, fb_count, fb_list, status);
-      }
+  const int groups = (total + 3) / 4;
+  for (int grp = blockIdx.x * kWarpsPerCta + (threadIdx.x >> 5); grp < groups; grp += gridDim.x * kWarpsPerCta) {
+    // lanes 8r .. 8r+7 look at row 4*grp + r
+    const int my_row = 4 * grp + (lane >> 3);
+    const bool my_active = my_row < total;
+    int mc0 = 0, mc1 = 0;
+    if (my_active) {
+      const int2 c = *reinterpret_cast<const int2*>(half_cnt + 2 * (size_t)my_row);
+      mc0 = c.x;
+      mc1 = c.y;
+    }
+    const bool small = !my_active || (mc0 >= 0 && mc1 >= 0 && mc0 + mc1 >= 1 && mc0 + mc1 <= 8);
+    if (__all_sync(0xffffffffu, small)) {
+      solve_rows_quad<D>(p, v, scale, entries, o, tau_out, row_cnt, my_active ? my_row : 0, my_active, mc0, mc1, lane);
       continue;
     }
-    const int bh = grow / p.N, i = grow - bh * p.N, b = bh / p.H, h = bh - b * p.H;
-    const float a = (p.alpha - 1.0f) * (scale[(size_t)h * p.N + i] * p.sm_scale);
-    Entry* list = entries + (size_t)grow * kListCap;
-    const __nv_bfloat16* vbase = v + (size_t)b * p.sb + (size_t)h * p.sh + lane * PER;
-    __nv_bfloat16* o_row = o + (size_t)b * p.sb + (size_t)h * p.sh + (size_t)i * p.sn + lane * PER;
-    const int n = c0 + c1;
-    if (n <= 32) solve_row<D, 1>(p, vbase, list, c0, c1, a, o_row, tau_out + grow, row_cnt + grow, lane);
-    else if (n <= 64) solve_row<D, 2>(p, vbase, list, c0, c1, a, o_row, tau_out + grow, row_cnt + grow, lane);
-    else if (n <= 128) solve_row<D, 4>(p, vbase, list, c0, c1, a, o_row, tau_out + grow, row_cnt + grow, lane);
-    else solve_row<D, kSlots>(p, vbase, list, c0, c1, a, o_row, tau_out + grow, row_cnt + grow, lane);
+    for (int r = 0; r < 4; ++r) {
+      const int grow = 4 * grp + r;
+      if (grow >= total) break;
+      const int c0 = __shfl_sync(0xffffffffu, mc0, 8 * r), c1 = __shfl_sync(0xffffffffu, mc1, 8 * r);
+      if (c0 < 0 || c1 < 0 || c0 + c1 == 0) {
+        if (lane == 0) {
+          row_cnt[grow] = -2;
+          push_dense_row(grow, fb_count, fb_list, status);
+        }
+        continue;
+      }
+      const int bh = grow / p.N, i = grow - bh * p.N, b = bh / p.H, h = bh - b * p.H;
+      const float a = (p.alpha - 1.0f) * (scale[(size_t)h * p.N + i] * p.sm_scale);
+      Entry* list = entries + (size_t)grow * kListCap;
+      const __nv_bfloat16* vbase = v + (size_t)b * p.sb + (size_t)h * p.sh + lane * PER;
+      __nv_bfloat16* o_row = o + (size_t)b * p.sb + (size_t)h * p.sh + (size_t)i * p.sn + lane * PER;
+      solve_row_full<D>(p, vbase, list, c0, c1, a, o_row, tau_out + grow, row_cnt + grow, lane);
+    }
   }
 }
 
@@ -326,7 +567,7 @@ __global__ void __launch_bounds__(kWarpsPerCta * 32) row_bwd_kernel(
 }
 
 inline int row_grid(const Problem& p) {
-  const long total = (long)p.B * p.H * p.N;
+  const long total = ((long)p.B * p.H * p.N + 3) / 4;   // one warp per group of four rows
   const long ctas = (total + kWarpsPerCta - 1) / kWarpsPerCta;
   const long cap = 148L * 8 * 8;
   return (int)(ctas < cap ? ctas : cap);
