@@ -467,6 +467,177 @@ __global__ void __launch_bounds__(kWarpsPerCta * 32) row_fwd_kernel(Problem p, c
   }
 }
 
+// Backward of one row with the whole warp: the entmax Jacobian on the support.
+template <int D>
+__device__ __forceinline__ void bwd_row_full(const Problem& p, const __nv_bfloat16* __restrict__ q,
+                                             const __nv_bfloat16* __restrict__ k, const __nv_bfloat16* __restrict__ v,
+                                             const __nv_bfloat16* __restrict__ d_o, const float* __restrict__ scale,
+                                             const float* __restrict__ tau_in, const Entry* __restrict__ entries,
+                                             __nv_bfloat16* __restrict__ dq, float* __restrict__ acc_dk,
+                                             float* __restrict__ acc_dv, int grow, int c0, int c1, int lane) {
+  constexpr int PER = D / 32;
+  const int bh = grow / p.N, i = grow - bh * p.N, b = bh / p.H, h = bh - b * p.H;
+  const float g = scale[(size_t)h * p.N + i] * p.sm_scale;
+  const float a = (p.alpha - 1.0f) * g;
+  const float tau = tau_in[grow];
+  const size_t hbase = (size_t)b * p.sb + (size_t)h * p.sh + lane * PER;
+  float qs[PER], gs[PER];
+  load_bf16<PER>(q + hbase + (size_t)i * p.sn, qs);
+  load_bf16<PER>(d_o + hbase + (size_t)i * p.sn, gs);
+  const Entry* list = entries + (size_t)grow * kListCap;
+  float yv[kSlots], dpv[kSlots];
+  int jj[kSlots];
+#pragma unroll
+  for (int s = 0; s < kSlots; ++s) {
+    const int e = lane + 32 * s;                     // dense numbering: first half-list, then second
+    yv[s] = -1.0f;
+    jj[s] = 0;
+    dpv[s] = 0.f;
+    if (e < c0 + c1) {
+      const Entry en = list[e < c0 ? e : kHalfCap + e - c0];
+      yv[s] = fmaf(a, en.y, -tau);
+      jj[s] = en.j;
+    }
+  }
+  // dP_ij = <dO_i, v_j> on the support
+#pragma unroll
+  for (int s = 0; s < kSlots; ++s) {
+    unsigned rest = __ballot_sync(0xffffffffu, yv[s] > 0.f);
+    while (rest) {
+      const int src = __ffs(rest) - 1;
+      rest &= rest - 1;
+      const int kj = __shfl_sync(0xffffffffu, jj[s], src);
+      float vs[PER];
+      load_bf16<PER>(v + hbase + (size_t)kj * p.sn, vs);
+      float dp = 0.f;
+#pragma unroll
+      for (int t = 0; t < PER; ++t) dp = fmaf(gs[t], vs[t], dp);
+      dp = warp_sum(dp);
+      if (lane == src) dpv[s] = dp;
+    }
+  }
+  float pe[kSlots], u[kSlots];
+  float su = 0.f, sud = 0.f;
+#pragma unroll
+  for (int s = 0; s < kSlots; ++s) {
+    pe[s] = 0.f;
+    u[s] = 0.f;
+    if (yv[s] > 0.f) pow_pair(yv[s], p.expo_class, p.expo, pe[s], u[s]);
+    su += u[s];
+    sud += u[s] * dpv[s];
+  }
+  su = warp_sum(su);
+  sud = warp_sum(sud);
+  const float rho = su > 0.f ? sud / su : 0.f;
+  float acc[PER];
+#pragma unroll
+  for (int t = 0; t < PER; ++t) acc[t] = 0.f;
+  const size_t arow = (size_t)bh * p.N;
+#pragma unroll
+  for (int s = 0; s < kSlots; ++s) {
+    const float gds_own = g * u[s] * (dpv[s] - rho);
+    unsigned rest = __ballot_sync(0xffffffffu, yv[s] > 0.f);
+    while (rest) {
+      const int src = __ffs(rest) - 1;
+      rest &= rest - 1;
+      const int kj = __shfl_sync(0xffffffffu, jj[s], src);
+      const float gds = __shfl_sync(0xffffffffu, gds_own, src);
+      const float pj = __shfl_sync(0xffffffffu, pe[s], src);
+      float ks[PER], dkv[PER], dvv[PER];
+      load_bf16<PER>(k + hbase + (size_t)kj * p.sn, ks);
+#pragma unroll
+      for (int t = 0; t < PER; ++t) {
+        acc[t] = fmaf(gds, ks[t], acc[t]);
+        dkv[t] = gds * qs[t];
+        dvv[t] = pj * gs[t];
+      }
+      atomic_add_slice<PER>(acc_dk + (arow + kj) * D + lane * PER, dkv);
+      atomic_add_slice<PER>(acc_dv + (arow + kj) * D + lane * PER, dvv);
+    }
+  }
+  store_bf16<PER>(dq + hbase + (size_t)i * p.sn, acc);
+}
+
+// Backward of four rows at once, eight lanes per row, for rows with at most eight list entries.
+template <int D>
+__device__ __forceinline__ void bwd_rows_quad(const Problem& p, const __nv_bfloat16* __restrict__ q,
+                                              const __nv_bfloat16* __restrict__ k, const __nv_bfloat16* __restrict__ v,
+                                              const __nv_bfloat16* __restrict__ d_o, const float* __restrict__ scale,
+                                              const float* __restrict__ tau_in, const Entry* __restrict__ entries,
+                                              __nv_bfloat16* __restrict__ dq, float* __restrict__ acc_dk,
+                                              float* __restrict__ acc_dv, int grow, bool active, int c0, int c1,
+                                              int lane) {
+  constexpr int PL = D / 8;                        // elements of a row per lane
+  const int sl = lane & 7;
+  const int base = lane & 24;
+  const int n = active ? c0 + c1 : 0;
+  const int bh = grow / p.N, i = grow - bh * p.N, b = bh / p.H, h = bh - b * p.H;
+  const float g = active ? scale[(size_t)h * p.N + i] * p.sm_scale : 0.f;
+  const float a = (p.alpha - 1.0f) * g;
+  const float tau = active ? tau_in[grow] : 0.f;
+  const size_t hbase = (size_t)b * p.sb + (size_t)h * p.sh + sl * PL;
+  float qs[PL], gs[PL];
+  load_bf16_vec<PL>(q + hbase + (size_t)i * p.sn, qs);
+  load_bf16_vec<PL>(d_o + hbase + (size_t)i * p.sn, gs);
+  const Entry* list = entries + (size_t)grow * kListCap;
+  float yv = -1.0f;
+  int j = 0;
+  if (sl < n) {
+    const Entry en = list[sl < c0 ? sl : kHalfCap + sl - c0];
+    yv = fmaf(a, en.y, -tau);
+    j = en.j;
+  }
+  const bool in = yv > 0.f;
+  const unsigned msub = (__ballot_sync(0xffffffffu, in) >> base) & 0xffu;
+  // dP_ij = <dO_i, v_j> on the support
+  float dpv = 0.f;
+#pragma unroll
+  for (int t = 0; t < 8; ++t) {
+    const bool has = (msub >> t) & 1u;
+    if (!__any_sync(0xffffffffu, has)) continue;
+    const int kj = __shfl_sync(0xffffffffu, j, base + t);
+    float dp = 0.f;
+    if (has) {
+      float vs[PL];
+      load_bf16_vec<PL>(v + hbase + (size_t)kj * p.sn, vs);
+#pragma unroll
+      for (int u = 0; u < PL; ++u) dp = fmaf(gs[u], vs[u], dp);
+    }
+    dp = oct_sum(dp);
+    if (sl == t) dpv = dp;
+  }
+  float pe = 0.f, u = 0.f;
+  if (in) pow_pair(yv, p.expo_class, p.expo, pe, u);
+  const float su = oct_sum(u), sud = oct_sum(u * dpv);
+  const float rho = su > 0.f ? sud / su : 0.f;
+  const float gds_own = g * u * (dpv - rho);
+  float acc[PL];
+#pragma unroll
+  for (int t = 0; t < PL; ++t) acc[t] = 0.f;
+  const size_t arow = (size_t)bh * p.N;
+#pragma unroll
+  for (int t = 0; t < 8; ++t) {
+    const bool has = (msub >> t) & 1u;
+    if (!__any_sync(0xffffffffu, has)) continue;
+    const int kj = __shfl_sync(0xffffffffu, j, base + t);
+    const float gds = __shfl_sync(0xffffffffu, gds_own, base + t);
+    const float pj = __shfl_sync(0xffffffffu, pe, base + t);
+    if (has) {
+      float ks[PL], dkv[PL], dvv[PL];
+      load_bf16_vec<PL>(k + hbase + (size_t)kj * p.sn, ks);
+#pragma unroll
+      for (int w = 0; w < PL; ++w) {
+        acc[w] = fmaf(gds, ks[w], acc[w]);
+        dkv[w] = gds * qs[w];
+        dvv[w] = pj * gs[w];
+      }
+      atomic_add_vec<PL>(acc_dk + (arow + kj) * D + sl * PL, dkv);
+      atomic_add_vec<PL>(acc_dv + (arow + kj) * D + sl * PL, dvv);
+    }
+  }
+  if (active) store_bf16_vec<PL>(dq + hbase + (size_t)i * p.sn, acc);
+}
+
 template <int D>
 __global__ void __launch_bounds__(kWarpsPerCta * 32) row_bwd_kernel(
     Problem p, const __nv_bfloat16* __restrict__ q, const __nv_bfloat16* __restrict__ k,
@@ -474,95 +645,35 @@ __global__ void __launch_bounds__(kWarpsPerCta * 32) row_bwd_kernel(
     const float* __restrict__ tau_in, const int32_t* __restrict__ half_cnt, const Entry* __restrict__ entries,
     __nv_bfloat16* __restrict__ dq, float* __restrict__ acc_dk, float* __restrict__ acc_dv, int32_t* fb_count,
     int32_t* fb_list, int32_t* status) {
-  constexpr int PER = D / 32;
   const int lane = threadIdx.x & 31;
   const int total = p.B * p.H * p.N;
-  for (int grow = blockIdx.x * kWarpsPerCta + (threadIdx.x >> 5); grow < total; grow += gridDim.x * kWarpsPerCta) {
-    const int c0 = half_cnt[2 * (size_t)grow], c1 = half_cnt[2 * (size_t)grow + 1];
-    if (c0 < 0 || c1 < 0) {
-      if (lane == 0) push_dense_row(grow, fb_count, fb_list, status);
+  const int groups = (total + 3) / 4;
+  for (int grp = blockIdx.x * kWarpsPerCta + (threadIdx.x >> 5); grp < groups; grp += gridDim.x * kWarpsPerCta) {
+    // lanes 8r .. 8r+7 look at row 4*grp + r
+    const int my_row = 4 * grp + (lane >> 3);
+    const bool my_active = my_row < total;
+    int mc0 = 0, mc1 = 0;
+    if (my_active) {
+      const int2 c = *reinterpret_cast<const int2*>(half_cnt + 2 * (size_t)my_row);
+      mc0 = c.x;
+      mc1 = c.y;
+    }
+    const bool small = !my_active || (mc0 >= 0 && mc1 >= 0 && mc0 + mc1 <= 8);
+    if (__all_sync(0xffffffffu, small)) {
+      bwd_rows_quad<D>(p, q, k, v, d_o, scale, tau_in, entries, dq, acc_dk, acc_dv, my_active ? my_row : 0, my_active,
+                       mc0, mc1, lane);
       continue;
     }
-    const int bh = grow / p.N, i = grow - bh * p.N, b = bh / p.H, h = bh - b * p.H;
-    const float g = scale[(size_t)h * p.N + i] * p.sm_scale;
-    const float a = (p.alpha - 1.0f) * g;
-    const float tau = tau_in[grow];
-    const size_t hbase = (size_t)b * p.sb + (size_t)h * p.sh + lane * PER;
-    float qs[PER], gs[PER];
-    load_bf16<PER>(q + hbase + (size_t)i * p.sn, qs);
-    load_bf16<PER>(d_o + hbase + (size_t)i * p.sn, gs);
-    const Entry* list = entries + (size_t)grow * kListCap;
-    float yv[kSlots], dpv[kSlots];
-    int jj[kSlots];
-#pragma unroll
-    for (int s = 0; s < kSlots; ++s) {
-      const int idx = lane + 32 * s;
-      yv[s] = -1.0f;
-      jj[s] = 0;
-      dpv[s] = 0.f;
-      if ((idx & (kHalfCap - 1)) < (idx < kHalfCap ? c0 : c1)) {
-        const Entry e = list[idx];
-        yv[s] = fmaf(a, e.y, -tau);
-        jj[s] = e.j;
+    for (int r = 0; r < 4; ++r) {
+      const int grow = 4 * grp + r;
+      if (grow >= total) break;
+      const int c0 = __shfl_sync(0xffffffffu, mc0, 8 * r), c1 = __shfl_sync(0xffffffffu, mc1, 8 * r);
+      if (c0 < 0 || c1 < 0) {
+        if (lane == 0) push_dense_row(grow, fb_count, fb_list, status);
+        continue;
       }
+      bwd_row_full<D>(p, q, k, v, d_o, scale, tau_in, entries, dq, acc_dk, acc_dv, grow, c0, c1, lane);
     }
-    // dP_ij = <dO_i, v_j> on the support
-#pragma unroll
-    for (int s = 0; s < kSlots; ++s) {
-      unsigned rest = __ballot_sync(0xffffffffu, yv[s] > 0.f);
-      while (rest) {
-        const int src = __ffs(rest) - 1;
-        rest &= rest - 1;
-        const int kj = __shfl_sync(0xffffffffu, jj[s], src);
-        float vs[PER];
-        load_bf16<PER>(v + hbase + (size_t)kj * p.sn, vs);
-        float dp = 0.f;
-#pragma unroll
-        for (int t = 0; t < PER; ++t) dp = fmaf(gs[t], vs[t], dp);
-        dp = warp_sum(dp);
-        if (lane == src) dpv[s] = dp;
-      }
-    }
-    float pe[kSlots], u[kSlots];
-    float su = 0.f, sud = 0.f;
-#pragma unroll
-    for (int s = 0; s < kSlots; ++s) {
-      pe[s] = 0.f;
-      u[s] = 0.f;
-      if (yv[s] > 0.f) pow_pair(yv[s], p.expo_class, p.expo, pe[s], u[s]);
-      su += u[s];
-      sud += u[s] * dpv[s];
-    }
-    su = warp_sum(su);
-    sud = warp_sum(sud);
-    const float rho = su > 0.f ? sud / su : 0.f;
-    float acc[PER];
-#pragma unroll
-    for (int t = 0; t < PER; ++t) acc[t] = 0.f;
-    const size_t arow = (size_t)bh * p.N;
-#pragma unroll
-    for (int s = 0; s < kSlots; ++s) {
-      const float gds_own = g * u[s] * (dpv[s] - rho);
-      unsigned rest = __ballot_sync(0xffffffffu, yv[s] > 0.f);
-      while (rest) {
-        const int src = __ffs(rest) - 1;
-        rest &= rest - 1;
-        const int kj = __shfl_sync(0xffffffffu, jj[s], src);
-        const float gds = __shfl_sync(0xffffffffu, gds_own, src);
-        const float pj = __shfl_sync(0xffffffffu, pe[s], src);
-        float ks[PER], dkv[PER], dvv[PER];
-        load_bf16<PER>(k + hbase + (size_t)kj * p.sn, ks);
-#pragma unroll
-        for (int t = 0; t < PER; ++t) {
-          acc[t] = fmaf(gds, ks[t], acc[t]);
-          dkv[t] = gds * qs[t];
-          dvv[t] = pj * gs[t];
-        }
-        atomic_add_slice<PER>(acc_dk + (arow + kj) * D + lane * PER, dkv);
-        atomic_add_slice<PER>(acc_dv + (arow + kj) * D + lane * PER, dvv);
-      }
-    }
-    store_bf16<PER>(dq + hbase + (size_t)i * p.sn, acc);
   }
 }
 
