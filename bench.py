@@ -69,7 +69,7 @@ class ClockSampler:
         try:
             self.proc = subprocess.Popen(
                 ["nvidia-smi", "-i", str(self.index), "--query-gpu=" + self.FIELDS, "--format=csv,noheader,nounits",
-                 "-lms", "100"], stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+                 "-lms", "50"], stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
         except OSError:
             self.proc = None
 
@@ -215,7 +215,7 @@ def run_ours(args):
     outs_host = {n: torch.empty(t.shape, dtype=t.dtype).pin_memory() for n, t in outs_dev.items()}
     h2d = sum(host[n].numel() * host[n].element_size() for n in names)
     d2h = sum(t.numel() * t.element_size() for t in outs_dev.values())
-    E = max(1, min(K, 5))
+    E = max(1, min(K, 10))
     ee_start, ee_stop = [ev() for _ in range(E)], [ev() for _ in range(E)]
     barrier(world)
     torch.cuda.synchronize()
@@ -272,7 +272,16 @@ def run_ours(args):
     print(json.dumps(line), flush=True)
 
 
-def _oracle_pass(inp, w, alpha, rows_per_head: int, seed: int):
+def _oracle_heads(inp, w):
+    """Per (batch, head) float32 numpy views of the inputs, prepared once outside any timed region."""
+    out = []
+    for bh in range(w.B * w.H):
+        b, h = divmod(bh, w.H)
+        out.append(tuple(t[b, h].float().numpy() for t in (inp.q, inp.k, inp.v, inp.d_o)))
+    return out
+
+
+def _oracle_pass(inp, w, alpha, heads, rows_per_head: int, seed: int):
     """Oracle forward rows + row-local backward (dQ) rows on `rows_per_head` sampled rows of every head.
     Returns (seconds, useful FLOPs of those rows, number of rows)."""
     import oracle
@@ -280,9 +289,9 @@ def _oracle_pass(inp, w, alpha, rows_per_head: int, seed: int):
     nrows = 0
     t0 = time.perf_counter()
     for bh in range(w.B * w.H):
-        b, h = divmod(bh, w.H)
+        h = bh % w.H
         rows = sample_rows(inp, bh, rows_per_head, seed=seed)
-        q, k, v, g = (t[b, h].float().numpy() for t in (inp.q, inp.k, inp.v, inp.d_o))
+        q, k, v, g = heads[bh]
         oracle.attn_fwd_rows(q, k, v, rows, alpha, inp.sm_scale, w.causal, scale=inp.head_scale(h))
         oracle.attn_bwd_rows(q, k, v, g, rows, alpha, inp.sm_scale, w.causal, scale=inp.head_scale(h))
         vis = (rows + 1) if w.causal else np.full_like(rows, w.N)
@@ -291,14 +300,26 @@ def _oracle_pass(inp, w, alpha, rows_per_head: int, seed: int):
     return time.perf_counter() - t0, flops, nrows
 
 
-def cpu_baseline(inp, w, alpha, budget_s: float = 12.0):
+def _sized_rows_per_head(inp, w, alpha, heads, budget_s: float):
+    """Rows per head that make one oracle pass last about `budget_s` seconds (two pilots, the second
+    large enough that fixed per-call costs no longer dominate the estimate)."""
+    rows = 16
+    for _ in range(2):
+        secs, _, n = _oracle_pass(inp, w, alpha, heads, rows, seed=1)
+        per_row = max(secs / n, 1e-7)
+        rows = int(max(8, min(w.N, budget_s / per_row / (w.B * w.H))))
+        if secs > 0.2 * budget_s:
+            break
+    return rows
+
+
+def cpu_baseline(inp, w, alpha, budget_s: float = 15.0):
     """The fp64 oracle, as it stands, on the host cores of this machine, on a bounded row sample of the same
-    workload (a pilot sizes the sample for about `budget_s` seconds)."""
+    workload (pilots size the sample for about `budget_s` seconds)."""
     import oracle
-    pilot_s, _, pilot_rows = _oracle_pass(inp, w, alpha, 8, seed=1)
-    per_row = max(pilot_s / pilot_rows, 1e-6)
-    rows_per_head = int(max(8, min(w.N, budget_s / per_row / (w.B * w.H))))
-    secs, flops, nrows = _oracle_pass(inp, w, alpha, rows_per_head, seed=2)
+    heads = _oracle_heads(inp, w)
+    rows_per_head = _sized_rows_per_head(inp, w, alpha, heads, budget_s)
+    secs, flops, nrows = _oracle_pass(inp, w, alpha, heads, rows_per_head, seed=2)
     return {"value": flops / secs / 1e12, "unit": UNIT, "cores": oracle.num_threads(), "kind": "oracle",
             "sample": "%d sampled query rows (%d per head) of the same workload: oracle forward rows plus the "
                       "row-local backward (dQ) rows, %.1f s; useful FLOPs of those rows / time" % (nrows, rows_per_head, secs),
@@ -312,16 +333,15 @@ def run_reference(args):
         return
     import oracle
     w, inp = make_bench_inputs(args.alpha)
-    pilot_s, _, pilot_rows = _oracle_pass(inp, w, args.alpha, 8, seed=1)
-    per_row = max(pilot_s / pilot_rows, 1e-6)
+    heads = _oracle_heads(inp, w)
     total_budget = 90.0
     steps = args.steps + max(args.warmup, 1)
-    rows_per_head = int(max(4, min(w.N, total_budget / steps / per_row / (w.B * w.H))))
+    rows_per_head = _sized_rows_per_head(inp, w, args.alpha, heads, total_budget / steps)
     for i in range(max(args.warmup, 1)):
-        _oracle_pass(inp, w, args.alpha, rows_per_head, seed=10 + i)
+        _oracle_pass(inp, w, args.alpha, heads, rows_per_head, seed=10 + i)
     secs = flops = nrows = 0
     for i in range(args.steps):
-        s, f, n = _oracle_pass(inp, w, args.alpha, rows_per_head, seed=100 + i)
+        s, f, n = _oracle_pass(inp, w, args.alpha, heads, rows_per_head, seed=100 + i)
         secs, flops, nrows = secs + s, flops + f, nrows + n
     value = flops / secs / 1e12
     sample = "each step = %d sampled query rows per head (oracle forward + row-local backward)" % rows_per_head
@@ -339,12 +359,12 @@ def run_reference(args):
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=10)
+    ap.add_argument("--steps", type=int, default=40)
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", choices=["ours", "reference"], default="ours")
     ap.add_argument("--alpha", type=float, default=1.5)
     ap.add_argument("--no-cpu-baseline", action="store_true")
-    ap.add_argument("--cpu-seconds", type=float, default=12.0)
+    ap.add_argument("--cpu-seconds", type=float, default=15.0)
     args = ap.parse_args()
     if args.impl == "reference":
         run_reference(args)
