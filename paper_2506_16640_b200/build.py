@@ -31,7 +31,7 @@ def needs_build() -> bool:
     if not os.path.exists(LIB):
         return True
     t = os.path.getmtime(LIB)
-    deps = _sources() + [os.path.join(CSRC, "common.cuh"), os.path.join(INCLUDE, "entmax_attn.h")]
+    deps = _sources() + [os.path.join(CSRC, "common.cuh"), os.path.join(CSRC, "sm100_ptx.cuh"), os.path.join(INCLUDE, "entmax_attn.h")]
     return any(os.path.getmtime(d) > t for d in deps)
 
 
