@@ -30,7 +30,7 @@ class Params(ctypes.Structure):
 
 class WsLayout(ctypes.Structure):
     _fields_ = [("row_count_offset", ctypes.c_size_t), ("entries_offset", ctypes.c_size_t),
-                ("scale_offset", ctypes.c_size_t), ("capacity", ctypes.c_int32), ("reserved", ctypes.c_int32)]
+                ("scale_offset", ctypes.c_size_t), ("capacity", ctypes.c_int32), ("keep_limit", ctypes.c_int32)]
 
 
 class EntmaxAttnError(RuntimeError):

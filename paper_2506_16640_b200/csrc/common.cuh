@@ -42,7 +42,7 @@ struct Problem {
 };
 
 struct WsLayout {
-  size_t scale, row_cnt, half_cnt, half_thr, entries, fb_count, sweep_counter, fb_list, scratch, acc_dk, acc_dv, total;
+  size_t scale, row_cnt, half_cnt, half_thr, entries, fb_count, sweep_counter, tile_count, fb_list, tile_flag, tile_list, scratch, acc_dk, acc_dv, total;
   int scratch_ctas;     // CTAs of the dense-row kernels (each owns scratch_floats floats)
   size_t scratch_floats;
 };
@@ -77,10 +77,18 @@ cudaError_t launch_sweep(const Problem& p, const void* q, const void* k, const f
                          int mode, int32_t* half_cnt, float* half_thr, Entry* entries, int32_t* work_counter,
                          float* dump, int dump_bh, int32_t* status, cudaStream_t stream);
 
-// per-row solve + gather kernels working on the lists (bf16 path)
+// Dense-tile forward on the tensor cores (bf16): recomputes the Q tiles (128 rows) listed in tile_list
+// and writes O and tau of their rows marked row_cnt == -2.
+cudaError_t launch_tile_fwd(const Problem& p, const void* q, const void* k, const void* v, const float* scale,
+                            const int32_t* tile_list, const int32_t* tile_count, const int32_t* row_cnt, void* o,
+                            float* tau, int32_t* status, cudaStream_t stream);
+
+// per-row solve + gather kernels working on the lists (bf16 path); the forward one also lists the
+// 128-row Q tiles that hold rows for the dense-tile path (tile_flag must be zero on entry)
 cudaError_t launch_row_fwd(const Problem& p, const void* v, const float* scale, int32_t* row_cnt,
                            const int32_t* half_cnt, const float* half_thr, Entry* entries, void* o, float* tau, int32_t* fb_count,
-                           int32_t* fb_list, int32_t* status, cudaStream_t stream);
+                           int32_t* fb_list, int32_t* tile_flag, int32_t* tile_list, int32_t* tile_count, int32_t* status,
+                           cudaStream_t stream);
 cudaError_t launch_row_bwd(const Problem& p, const void* q, const void* k, const void* v, const void* d_o,
                            const float* scale, const float* tau, const int32_t* half_cnt, Entry* entries, void* dq,
                            float* acc_dk, float* acc_dv, int32_t* fb_count, int32_t* fb_list, int32_t* status,

@@ -90,8 +90,12 @@ WsLayout make_layout(const Problem& p, bool is_bwd) {
   l.half_thr = take(rows * 2 * sizeof(float));
   l.entries = take(rows * kListCap * sizeof(Entry));
   l.fb_count = take(256);
-  l.sweep_counter = l.fb_count + 64;   // same 256-byte block: [0] dense-row count, [16] sweep work counter
+  l.sweep_counter = l.fb_count + 64;   // same 256-byte block: [0] dense-row count, [16] sweep work counter,
+  l.tile_count = l.fb_count + 128;     // [32] number of listed dense tiles
   l.fb_list = take(rows * sizeof(int32_t));
+  const size_t q_tiles = (size_t)p.B * p.H * ((p.N + 127) / 128);
+  l.tile_flag = take(q_tiles * sizeof(int32_t));
+  l.tile_list = take(q_tiles * sizeof(int32_t));
   // dense-row CTAs: enough to fill the machine, few enough that their score rows stay modest
   l.scratch_floats = align_up((size_t)p.N, 32) * (is_bwd ? 2 : 1);   // scores (+ dP in backward)
   size_t ctas = 148 * 4;
@@ -129,7 +133,7 @@ int entmax_attn_workspace_layout(const entmax_attn_params* params, entmax_attn_w
   out->entries_offset = l.entries;
   out->scale_offset = l.scale;
   out->capacity = kListCap;
-  out->reserved = 0;
+  out->keep_limit = kHalfKeep;
   return ENTMAX_ATTN_OK;
 }
 
@@ -173,17 +177,23 @@ int entmax_attn_fwd(const entmax_attn_params* params, const void* q, const void*
                            lay.scratch_ctas, stream);
     return err == cudaSuccess ? ENTMAX_ATTN_OK : fail_cuda(err);
   }
-  err = cudaMemsetAsync(fb_count, 0, sizeof(int32_t), stream);
+  int32_t* tile_flag = reinterpret_cast<int32_t*>(ws + lay.tile_flag);
+  int32_t* tile_list = reinterpret_cast<int32_t*>(ws + lay.tile_list);
+  int32_t* tile_count = reinterpret_cast<int32_t*>(ws + lay.tile_count);
+  err = cudaMemsetAsync(fb_count, 0, 256, stream);   // the whole counter block
+  if (err != cudaSuccess) return fail_cuda(err);
+  err = cudaMemsetAsync(tile_flag, 0, (size_t)p.B * p.H * ((p.N + 127) / 128) * sizeof(int32_t), stream);
   if (err != cudaSuccess) return fail_cuda(err);
   if (g_prof_start[0]) cudaEventRecord(g_prof_start[0], stream);
   err = launch_sweep(p, q, k, scale, nullptr, 0, half_cnt, half_thr, entries, sweep_counter, nullptr, -1, device_status,
                      stream);
   if (err != cudaSuccess) return fail_cuda(err);
   if (g_prof_stop[0]) cudaEventRecord(g_prof_stop[0], stream);
-  err = launch_row_fwd(p, v, scale, row_cnt, half_cnt, half_thr, entries, o, tau, fb_count, fb_list, device_status, stream);
+  err = launch_row_fwd(p, v, scale, row_cnt, half_cnt, half_thr, entries, o, tau, fb_count, fb_list, tile_flag, tile_list,
+                       tile_count, device_status, stream);
   if (err != cudaSuccess) return fail_cuda(err);
-  err = launch_dense_fwd(p, q, k, v, scale, o, tau, row_cnt, entries, fb_list, fb_count, scratch, lay.scratch_floats,
-                         lay.scratch_ctas, stream);
+  // rows whose support does not fit the lists: dense tiles on the tensor cores
+  err = launch_tile_fwd(p, q, k, v, scale, tile_list, tile_count, row_cnt, o, tau, device_status, stream);
   return err == cudaSuccess ? ENTMAX_ATTN_OK : fail_cuda(err);
 }
 

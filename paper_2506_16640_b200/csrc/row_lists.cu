@@ -418,6 +418,17 @@ __device__ __forceinline__ void solve_rows_quad(const Problem& p, const __nv_bfl
   }
 }
 
+// Forward: a row for the dense-tile path.  Its 128-row Q tile is listed once (tile_flag arbitrates).
+__device__ __forceinline__ void push_dense_tile(const Problem& p, int grow, int32_t* fb_count, int32_t* fb_list,
+                                                int32_t* tile_flag, int32_t* tile_list, int32_t* tile_count,
+                                                int32_t* status) {
+  push_dense_row(grow, fb_count, fb_list, status);
+  const int tiles_per_head = (p.N + 127) / 128;
+  const int bh = grow / p.N, i = grow - bh * p.N;
+  const int id = bh * tiles_per_head + i / 128;
+  if (atomicExch(tile_flag + id, 1) == 0) tile_list[atomicAdd(tile_count, 1)] = id;
+}
+
 template <int D>
 __global__ void __launch_bounds__(kWarpsPerCta * 32) row_fwd_kernel(Problem p, const __nv_bfloat16* __restrict__ v,
                                                                     const float* __restrict__ scale,
@@ -426,7 +437,9 @@ __global__ void __launch_bounds__(kWarpsPerCta * 32) row_fwd_kernel(Problem p, c
                                                                     Entry* __restrict__ entries,
                                                                     __nv_bfloat16* __restrict__ o,
                                                                     float* __restrict__ tau_out, int32_t* fb_count,
-                                                                    int32_t* fb_list, int32_t* status) {
+                                                                    int32_t* fb_list, int32_t* tile_flag,
+                                                                    int32_t* tile_list, int32_t* tile_count,
+                                                                    int32_t* status) {
   constexpr int PER = D / 32;
   const int lane = threadIdx.x & 31;
   const int total = p.B * p.H * p.N;
@@ -453,7 +466,7 @@ __global__ void __launch_bounds__(kWarpsPerCta * 32) row_fwd_kernel(Problem p, c
       if (c0 < 0 || c1 < 0 || c0 + c1 == 0) {
         if (lane == 0) {
           row_cnt[grow] = -2;
-          push_dense_row(grow, fb_count, fb_list, status);
+          push_dense_tile(p, grow, fb_count, fb_list, tile_flag, tile_list, tile_count, status);
         }
         continue;
       }
@@ -688,14 +701,17 @@ inline int row_grid(const Problem& p) {
 
 cudaError_t launch_row_fwd(const Problem& p, const void* v, const float* scale, int32_t* row_cnt,
                            const int32_t* half_cnt, const float* half_thr, Entry* entries, void* o, float* tau,
-                           int32_t* fb_count, int32_t* fb_list, int32_t* status, cudaStream_t stream) {
+                           int32_t* fb_count, int32_t* fb_list, int32_t* tile_flag, int32_t* tile_list,
+                           int32_t* tile_count, int32_t* status, cudaStream_t stream) {
   const int grid = row_grid(p);
   if (p.D == 64)
     row_fwd_kernel<64><<<grid, kWarpsPerCta * 32, 0, stream>>>(p, (const __nv_bfloat16*)v, scale, row_cnt, half_cnt,
-                                                              entries, (__nv_bfloat16*)o, tau, fb_count, fb_list, status);
+                                                              entries, (__nv_bfloat16*)o, tau, fb_count, fb_list, tile_flag, tile_list,
+        tile_count, status);
   else
     row_fwd_kernel<128><<<grid, kWarpsPerCta * 32, 0, stream>>>(p, (const __nv_bfloat16*)v, scale, row_cnt, half_cnt,
-                                                               entries, (__nv_bfloat16*)o, tau, fb_count, fb_list, status);
+                                                               entries, (__nv_bfloat16*)o, tau, fb_count, fb_list, tile_flag, tile_list,
+        tile_count, status);
   return cudaGetLastError();
 }
 

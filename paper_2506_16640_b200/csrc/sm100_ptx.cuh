@@ -61,7 +61,7 @@ __device__ __forceinline__ uint64_t global_ns() {
 }
 // Bounded wait.  Returns false when the CTA is aborting (this or another wait ran out of time).
 // `abort_flag` is the shared-memory address of the CTA's abort word.
-__device__ __noinline__ bool mbar_wait_slow(uint32_t bar, uint32_t parity, uint32_t abort_flag) {
+static __device__ __noinline__ bool mbar_wait_slow(uint32_t bar, uint32_t parity, uint32_t abort_flag) {
   const uint64_t t0 = global_ns();
   uint32_t spins = 0;
   for (;;) {

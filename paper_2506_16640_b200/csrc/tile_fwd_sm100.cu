@@ -1,0 +1,543 @@
+// Dense-tile forward for bf16 problems on sm_100a: the rows whose support does not fit the sparse
+// lists of the score sweep are recomputed tile by tile on the tensor cores, the way the method reads
+// when nothing is known about the sparsity:
+//   threshold   tau_i by Newton from the left on f(tau) = sum_j [y_ij - tau]_+^e - 1 (Eq. 1 with the
+//               sum-to-one condition), every iteration one sweep S = Q K^T over the visible K tiles
+//               (tcgen05, fp32 accumulators in TMEM), started at the lower end of the bracket of
+//               App. A, tau >= y_max - 1, which a first sweep finds;
+//   output      one more sweep: P = [y - tau]_+^e, rounded to bf16 and written to shared memory as the
+//               A operand of a second tcgen05 contraction O += P V (V tile as the N-major B operand),
+//               O accumulated in TMEM over all K tiles.
+// A work item is one Q tile of 128 rows that holds at least one such row (a list written by the row
+// kernel); only the rows flagged there are written back.
+//
+// CTA: warp 0 TMA producer, warp 1 MMA issuer, warps 2..5 consumers (TMEM lane = query row, one thread
+// per row, all 128 columns of a K tile).  The number of Newton sweeps is decided by the consumers; they
+// publish "all rows converged" through shared memory and a control mbarrier that every role waits on
+// between sweeps.  Every wait is bounded (see sm100_ptx.cuh); on expiry the CTA flags the call's status
+// word and leaves.
+#include <cuda.h>
+
+#include "common.cuh"
+#include "sm100_ptx.cuh"
+
+namespace entmax {
+
+namespace {
+
+using namespace sm100;
+
+constexpr int TM = 128;            // query rows per item = TMEM lanes
+constexpr int TN = 128;            // keys per K/V tile
+constexpr int kThreadsT = 6 * 32;
+constexpr int kStagesT = 2;
+constexpr int kMaxSweeps = 48;     // 1 max sweep + at most 46 Newton sweeps + the output sweep
+constexpr int kPBytes = TM * TN * 2;
+
+template <int HD>
+struct TCfg {
+  static constexpr int kHalves = HD / 64;
+  static constexpr int kQBytes = TM * HD * 2;
+  static constexpr int kKBytes = TN * HD * 2;      // also the size of a V tile
+  static constexpr int kBarBytes = 256;
+  static constexpr int kSmemBytes = kQBytes + kStagesT * 2 * kKBytes + kPBytes + 1024 + kBarBytes;
+  static constexpr int kTmemO = 2 * TN;            // first TMEM column of the O accumulator
+};
+
+struct TileArgsK {
+  int B, H, N;
+  int causal;
+  int expo_class;
+  float expo;
+  float alpha_m1;
+  float sm_scale;
+  const float* scale;        // [H, N]
+  const int32_t* tile_list;  // ids of the Q tiles to process: bh * tiles_per_head + tile
+  const int32_t* tile_count;
+  const int32_t* row_cnt;    // -2 marks the rows to write
+  void* o;                   // bf16 [B,H,N,D]
+  float* tau;
+  int64_t sb, sh, sn;
+  int32_t* status;
+  int tiles_per_head;
+};
+
+// tcgen05.mma with separate descriptor high words for A and B
+__device__ __forceinline__ void umma_bf16_ab(uint32_t d_tmem, uint32_t a_lo, uint32_t a_hi, uint32_t b_lo, uint32_t b_hi,
+                                             uint32_t idesc, uint32_t accumulate) {
+  asm volatile(
+      "{\n"
+      " .reg .pred p;\n"
+      " .reg .b64 da, db;\n"
+      " mov.b64 da, {%1, %2};\n"
+      " mov.b64 db, {%3, %4};\n"
+      " setp.ne.b32 p, %6, 0;\n"
+      " tcgen05.mma.cta_group::1.kind::f16 [%0], da, db, %5, p;\n"
+      "}\n" ::"r"(d_tmem), "r"(a_lo), "r"(a_hi), "r"(b_lo), "r"(b_hi), "r"(idesc), "r"(accumulate)
+      : "memory");
+}
+
+// S = Q K^T: A, B bf16 K-major, fp32 accumulate, M = 128, N = TN
+__host__ __device__ constexpr uint32_t idesc_qk() {
+  return (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(TN >> 3) << 17) | ((uint32_t)(TM >> 4) << 24);
+}
+// O += P V: A = P K-major, B = V with N (head dim) contiguous ("MN-major", bit 16), M = 128, N = HD
+template <int HD>
+__host__ __device__ constexpr uint32_t idesc_pv() {
+  return (1u << 4) | (1u << 7) | (1u << 10) | (1u << 16) | ((uint32_t)(HD >> 3) << 17) | ((uint32_t)(TM >> 4) << 24);
+}
+// Descriptor words of the V tile as an N-major operand with 128-byte swizzle: a swizzle atom is 64
+// head-dim elements (one 128-byte row) by 8 keys; atoms repeat every 1024 bytes along the keys
+// (stride-dimension offset) and, for head_dim 128, every TN*128 bytes along the head dimension
+// (leading-dimension offset: the second 64-column block of the tile).
+__device__ __forceinline__ uint32_t v_desc_lo(uint32_t saddr) {
+  return ((saddr & 0x3FFFFu) >> 4) | ((uint32_t)((TN * 128) >> 4) << 16);
+}
+
+__device__ __forceinline__ float pow_e(float y, int expo_class, float expo) {
+  if (expo_class == kExpo2) return y * y;
+  if (expo_class == kExpo1) return y;
+  if (expo_class == kExpo4) { const float t = y * y; return t * t; }
+  return powf(y, expo);
+}
+
+template <int HD>
+__global__ void __launch_bounds__(kThreadsT, 1) tile_fwd_kernel(const __grid_constant__ CUtensorMap map_q,
+                                                               const __grid_constant__ CUtensorMap map_k,
+                                                               const __grid_constant__ CUtensorMap map_v,
+                                                               const TileArgsK a) {
+  using C = TCfg<HD>;
+  extern __shared__ uint8_t smem_raw[];
+  const uint32_t sbase = (smem_u32(smem_raw) + 1023u) & ~1023u;
+  const uint32_t q_smem = sbase;
+  const uint32_t k_smem = q_smem + C::kQBytes;                       // [kStagesT] K tiles
+  const uint32_t v_smem = k_smem + kStagesT * C::kKBytes;            // [kStagesT] V tiles
+  const uint32_t p_smem = v_smem + kStagesT * C::kKBytes;            // P tile, A-operand layout
+  const uint32_t bars = p_smem + kPBytes;
+  const uint32_t q_full = bars, q_empty = bars + 8;
+  const uint32_t kv_full = bars + 16;                                 // [kStagesT]
+  const uint32_t kv_empty = kv_full + 8 * kStagesT;                   // [kStagesT]
+  const uint32_t s_full = kv_empty + 8 * kStagesT;                    // [2]
+  const uint32_t s_empty = s_full + 16;                               // [2]
+  const uint32_t p_full = s_empty + 16, p_empty = p_full + 8;
+  const uint32_t o_full = p_empty + 8, o_empty = o_full + 8;
+  const uint32_t ctl = o_empty + 8;                                   // consumers' verdict on a sweep is in
+  const uint32_t done_word = ctl + 8;                                 // uint32 [3]
+  const uint32_t tmem_slot = done_word + 12;
+  const uint32_t abort_flag = tmem_slot + 4;
+  static_assert(8 * (2 + 2 * kStagesT + 4 + 4 + 1) + 12 + 8 <= C::kBarBytes, "barrier area");
+
+  const int warp = threadIdx.x >> 5;
+  const int lane = threadIdx.x & 31;
+  const int n_tiles = *a.tile_count;
+
+  if (threadIdx.x == 0) {
+    mbar_init(q_full, 1);
+    mbar_init(q_empty, 1);
+    for (int t = 0; t < kStagesT; ++t) {
+      mbar_init(kv_full + 8 * t, 1);
+      mbar_init(kv_empty + 8 * t, 1);
+    }
+    for (int t = 0; t < 2; ++t) {
+      mbar_init(s_full + 8 * t, 1);
+      mbar_init(s_empty + 8 * t, 4);
+    }
+    mbar_init(p_full, 4);
+    mbar_init(p_empty, 1);
+    mbar_init(o_full, 1);
+    mbar_init(o_empty, 4);
+    mbar_init(ctl, 4);
+    for (int t = 0; t < 3; ++t) sts_u32(done_word + 4 * t, 1u);
+    sts_u32(abort_flag, 0u);
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+  }
+  if (warp == 1) {
+    tmem_alloc(tmem_slot, 512);
+    tmem_relinquish();
+  }
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem_base = lds_u32(tmem_slot);
+
+  // Sweep s of an item: 0 finds the row maxima, then Newton sweeps until the consumers report that every
+  // row has converged (or the cap is reached), then the output sweep.  All roles evaluate this the same way.
+  auto sweep_is_output = [&](int s) -> bool {
+    return s == kMaxSweeps - 1 || (s >= 2 && lds_u32(done_word + 4 * ((s - 1) % 3)) != 0u);
+  };
+  auto item_tiles = [&](int tile) -> int {
+    const int row0 = tile * TM;
+    if (!a.causal) return (a.N + TN - 1) / TN;
+    int last_row = row0 + TM - 1;
+    if (last_row > a.N - 1) last_row = a.N - 1;
+    return last_row / TN + 1;
+  };
+
+  if (warp == 0) {
+    // ------------------------------------------------------------------ TMA producer
+    if (lane == 0) {
+      int stage = 0;
+      uint32_t kvphase = 0, qphase = 0, cphase = 0;
+      bool alive = true;
+      for (int it = blockIdx.x; it < n_tiles && alive; it += gridDim.x) {
+        const int id = a.tile_list[it];
+        const int bh = id / a.tiles_per_head, tile = id - bh * a.tiles_per_head;
+        const int b = bh / a.H, h = bh - b * a.H;
+        const int tiles = item_tiles(tile);
+        alive = mbar_wait(q_empty, qphase ^ 1u, abort_flag);
+        if (!alive) break;
+        mbar_expect_tx(q_full, C::kQBytes);
+        for (int hf = 0; hf < C::kHalves; ++hf)
+          tma_load_4d(q_smem + hf * (TM * 128), &map_q, q_full, hf * 64, tile * TM, h, b);
+        qphase ^= 1u;
+        for (int s = 0; s < kMaxSweeps && alive; ++s) {
+          if (s > 0) {
+            alive = mbar_wait(ctl, cphase, abort_flag);
+            cphase ^= 1u;
+            if (!alive) break;
+          }
+          const bool output = sweep_is_output(s);
+          for (int t = 0; t < tiles && alive; ++t) {
+            alive = mbar_wait(kv_empty + 8 * stage, kvphase ^ 1u, abort_flag);
+            if (!alive) break;
+            mbar_expect_tx(kv_full + 8 * stage, output ? 2 * C::kKBytes : C::kKBytes);
+            for (int hf = 0; hf < C::kHalves; ++hf)
+              tma_load_4d(k_smem + stage * C::kKBytes + hf * (TN * 128), &map_k, kv_full + 8 * stage, hf * 64, t * TN, h, b);
+            if (output) {
+              for (int hf = 0; hf < C::kHalves; ++hf)
+                tma_load_4d(v_smem + stage * C::kKBytes + hf * (TN * 128), &map_v, kv_full + 8 * stage, hf * 64, t * TN, h,
+                            b);
+            }
+            if (++stage == kStagesT) { stage = 0; kvphase ^= 1u; }
+          }
+          if (output) break;
+        }
+      }
+    }
+  } else if (warp == 1) {
+    // ------------------------------------------------------------------ MMA issuer
+    if (lane == 0) {
+      constexpr uint32_t id_qk = idesc_qk();
+      constexpr uint32_t id_pv = idesc_pv<HD>();
+      const uint32_t q_lo = smem_desc_lo(q_smem), k_lo = smem_desc_lo(k_smem), p_lo = smem_desc_lo(p_smem);
+      const uint32_t v_lo = v_desc_lo(v_smem);
+      int stage = 0;
+      uint32_t kvphase = 0, qphase = 0, cphase = 0, sphase[2] = {0, 0}, pphase = 0, ophase = 0;
+      int sbuf = 0;
+      bool alive = true;
+      for (int it = blockIdx.x; it < n_tiles && alive; it += gridDim.x) {
+        const int id = a.tile_list[it];
+        const int tile = id % a.tiles_per_head;
+        const int tiles = item_tiles(tile);
+        alive = mbar_wait(q_full, qphase, abort_flag);
+        qphase ^= 1u;
+        if (!alive) break;
+        for (int s = 0; s < kMaxSweeps && alive; ++s) {
+          if (s > 0) {
+            alive = mbar_wait(ctl, cphase, abort_flag);
+            cphase ^= 1u;
+            if (!alive) break;
+          }
+          const bool output = sweep_is_output(s);
+          if (output) {
+            // the previous item's O must have been read before this item's first PV overwrites it
+            alive = mbar_wait(o_empty, ophase ^ 1u, abort_flag);
+            ophase ^= 1u;
+            if (!alive) break;
+          }
+          for (int t = 0; t < tiles && alive; ++t) {
+            alive = mbar_wait(kv_full + 8 * stage, kvphase, abort_flag);
+            if (alive) alive = mbar_wait(s_empty + 8 * sbuf, sphase[sbuf] ^ 1u, abort_flag);
+            if (!alive) break;
+            sphase[sbuf] ^= 1u;
+            tc_fence_after();
+            const uint32_t b_lo = k_lo + stage * (C::kKBytes >> 4);
+#pragma unroll
+            for (int kk = 0; kk < HD / 16; ++kk) {
+              const uint32_t a_off = (kk >> 2) * ((TM * 128) >> 4) + (kk & 3) * 2;
+              const uint32_t b_off = (kk >> 2) * ((TN * 128) >> 4) + (kk & 3) * 2;
+              umma_bf16(tmem_base + sbuf * TN, q_lo + a_off, b_lo + b_off, kDescHi, id_qk, kk > 0 ? 1u : 0u);
+            }
+            umma_commit(s_full + 8 * sbuf);
+            sbuf ^= 1;
+            if (!output) {
+              umma_commit(kv_empty + 8 * stage);
+            } else {
+              // O += P V for this tile once the consumers have written P
+              alive = mbar_wait(p_full, pphase, abort_flag);
+              pphase ^= 1u;
+              if (!alive) break;
+              tc_fence_after();
+              const uint32_t vb_lo = v_lo + stage * (C::kKBytes >> 4);
+#pragma unroll
+              for (int kk = 0; kk < TN / 16; ++kk) {
+                const uint32_t a_off = (kk >> 2) * ((TM * 128) >> 4) + (kk & 3) * 2;   // 64 keys per 128-byte row
+                const uint32_t b_off = kk * ((16 * 128) >> 4);                           // 16 keys = 16 rows of 128 B
+                umma_bf16_ab(tmem_base + C::kTmemO, p_lo + a_off, kDescHi, vb_lo + b_off, kDescHi, id_pv,
+                             (t > 0 || kk > 0) ? 1u : 0u);
+              }
+              umma_commit(p_empty);
+              umma_commit(kv_empty + 8 * stage);
+              if (t == tiles - 1) umma_commit(o_full);
+            }
+            if (++stage == kStagesT) { stage = 0; kvphase ^= 1u; }
+          }
+          if (output) break;
+        }
+        umma_commit(q_empty);
+      }
+    }
+  } else {
+    // ------------------------------------------------------------------ consumers: one thread per query row
+    const int quad = warp & 3;
+    const int row_local = quad * 32 + lane;
+    const uint32_t taddr_row = tmem_base + ((uint32_t)(quad * 32) << 16);
+    uint32_t sphase[2] = {0, 0}, pphase = 0, ophase = 0, cphase = 0;
+    int sbuf = 0;
+    bool alive = true;
+    for (int it = blockIdx.x; it < n_tiles && alive; it += gridDim.x) {
+      const int id = a.tile_list[it];
+      const int bh = id / a.tiles_per_head, tile = id - bh * a.tiles_per_head;
+      const int b = bh / a.H, h = bh - b * a.H;
+      const int tiles = item_tiles(tile);
+      const int i = tile * TM + row_local;
+      const bool valid = i < a.N;
+      const size_t grow = (size_t)bh * a.N + (valid ? i : 0);
+      const int lim = a.causal ? i : a.N - 1;
+      const float ra = valid ? a.alpha_m1 * (a.scale[(size_t)h * a.N + i] * a.sm_scale) : 0.f;
+      float tau = 0.f, ymax = -INFINITY;
+      bool done = !valid;
+      for (int s = 0; s < kMaxSweeps && alive; ++s) {
+        if (s > 0) {
+          alive = __all_sync(0xffffffffu, mbar_wait(ctl, cphase, abort_flag));
+          cphase ^= 1u;
+          if (!alive) break;
+        }
+        const bool output = sweep_is_output(s);
+        // the verdict slot two sweeps ahead is free again: nobody reads it before the next vote
+        if (warp == 2 && lane == 0) sts_u32(done_word + 4 * ((s + 1) % 3), 1u);
+        float s0 = 0.f, s1 = 0.f;
+        for (int t = 0; t < tiles && alive; ++t) {
+          alive = __all_sync(0xffffffffu, mbar_wait(s_full + 8 * sbuf, sphase[sbuf], abort_flag));
+          if (!alive) break;
+          sphase[sbuf] ^= 1u;
+          tc_fence_after();
+          if (output) {
+            // P of the previous tile must have been consumed before its buffer is rewritten
+            alive = __all_sync(0xffffffffu, mbar_wait(p_empty, pphase ^ 1u, abort_flag));
+            pphase ^= 1u;
+            if (!alive) break;
+          }
+#pragma unroll
+          for (int c = 0; c < TN / 32; ++c) {
+            float va[32];
+            tmem_ld32(taddr_row + sbuf * TN + c * 32, va);
+            tmem_ld_wait();
+            const int col0 = t * TN + c * 32;
+            if (s == 0) {
+#pragma unroll
+              for (int u = 0; u < 32; ++u)
+                if (col0 + u <= lim) ymax = fmaxf(ymax, ra * va[u]);
+            } else if (!output) {
+#pragma unroll
+              for (int u = 0; u < 32; ++u) {
+                const float y = fmaf(ra, va[u], -tau);
+                if (y > 0.f && col0 + u <= lim) {
+                  float ye, ye1;
+                  pow_pair(y, a.expo_class, a.expo, ye, ye1);
+                  s0 += ye;
+                  s1 += ye1;
+                }
+              }
+            } else {
+              // P -> bf16 -> shared memory, K-major with 128-byte swizzle: row r, 16-byte unit u of the
+              // 64-key block sits at r*128 + ((u ^ (r & 7)) * 16)
+              const uint32_t blk = p_smem + (uint32_t)(c >> 1) * (TM * 128) + (uint32_t)row_local * 128u;
+#pragma unroll
+              for (int u4 = 0; u4 < 4; ++u4) {
+                uint32_t w[4];
+#pragma unroll
+                for (int e2 = 0; e2 < 4; ++e2) {
+                  float pv[2];
+#pragma unroll
+                  for (int z = 0; z < 2; ++z) {
+                    const int u = u4 * 8 + e2 * 2 + z;
+                    const float y = fmaf(ra, va[u], -tau);
+                    pv[z] = (y > 0.f && col0 + u <= lim && valid) ? pow_e(y, a.expo_class, a.expo) : 0.f;
+                  }
+                  const __nv_bfloat162 hh = __floats2bfloat162_rn(pv[0], pv[1]);
+                  w[e2] = *reinterpret_cast<const uint32_t*>(&hh);
+                }
+                const uint32_t unit = (uint32_t)((c & 1) * 4 + u4);
+                const uint32_t addr = blk + ((unit ^ (uint32_t)(row_local & 7)) << 4);
+                asm volatile("st.shared::cta.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(addr), "r"(w[0]), "r"(w[1]), "r"(w[2]),
+                             "r"(w[3])
+                             : "memory");
+              }
+            }
+          }
+          // the accumulator has been read
+          tc_fence_before();
+          __syncwarp();
+          if (lane == 0) mbar_arrive(s_empty + 8 * sbuf);
+          sbuf ^= 1;
+          if (output) {
+            // make the P stores visible to the tensor core (async proxy), then hand the tile over
+            asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+            __syncwarp();
+            if (lane == 0) mbar_arrive(p_full);
+          }
+        }
+        if (!alive) break;
+        if (output) {
+          alive = __all_sync(0xffffffffu, mbar_wait(o_full, ophase, abort_flag));
+          ophase ^= 1u;
+          if (!alive) break;
+          tc_fence_after();
+          const bool write = valid && a.row_cnt[grow] == -2;
+          __nv_bfloat16* orow =
+              reinterpret_cast<__nv_bfloat16*>(a.o) + (size_t)b * a.sb + (size_t)h * a.sh + (size_t)i * a.sn;
+#pragma unroll
+          for (int c = 0; c < HD / 32; ++c) {
+            float va[32];
+            tmem_ld32(taddr_row + C::kTmemO + c * 32, va);
+            tmem_ld_wait();
+            if (write) {
+#pragma unroll
+              for (int u8 = 0; u8 < 4; ++u8) {
+                uint32_t w[4];
+#pragma unroll
+                for (int e2 = 0; e2 < 4; ++e2) {
+                  const __nv_bfloat162 hh = __floats2bfloat162_rn(va[u8 * 8 + e2 * 2], va[u8 * 8 + e2 * 2 + 1]);
+                  w[e2] = *reinterpret_cast<const uint32_t*>(&hh);
+                }
+                *reinterpret_cast<uint4*>(orow + c * 32 + u8 * 8) = make_uint4(w[0], w[1], w[2], w[3]);
+              }
+            }
+          }
+          if (write) a.tau[grow] = tau;
+          tc_fence_before();
+          __syncwarp();
+          if (lane == 0) mbar_arrive(o_empty);
+          break;
+        }
+        // ---- between sweeps: Newton update and the verdict "every row of the tile has converged"
+        if (s == 0) {
+          tau = ymax - 1.0f;
+        } else if (!done) {
+          if (!(s0 > 1.0f) || !(s1 > 0.f)) {
+            done = true;
+          } else {
+            const float step = (s0 - 1.0f) / (a.expo * s1);
+            const float next = tau + step;
+            if (!(next > tau)) done = true;
+            tau = next > tau ? next : tau;
+            if (step <= 2e-6f * fmaxf(1.0f, fabsf(tau))) done = true;
+          }
+        }
+        const bool warp_done = __all_sync(0xffffffffu, done);
+        if (lane == 0) {
+          if (!warp_done || s == 0) atomicAnd(reinterpret_cast<unsigned*>(__cvta_shared_to_generic(done_word + 4 * (s % 3))), 0u);
+          mbar_arrive(ctl);
+        }
+      }
+    }
+  }
+
+  // ---------------------------------------------------------------------- teardown
+  tc_fence_before();
+  __syncthreads();
+  if (lds_u32(abort_flag)) {
+    if (threadIdx.x == 0 && a.status) atomicOr(a.status + ENTMAX_ATTN_STATUS_FLAGS, ENTMAX_ATTN_FLAG_WAIT_EXPIRED);
+    const uint64_t t0 = global_ns();
+    while (global_ns() - t0 < 200000ull) { }
+    __syncthreads();
+  }
+  if (warp == 1) {
+    tc_fence_after();
+    tmem_dealloc(tmem_base, 512);
+  }
+}
+
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+cudaError_t encode_fn(EncodeTiledFn* fn) {
+  static EncodeTiledFn cached = nullptr;
+  if (!cached) {
+    void* p = nullptr;
+    cudaDriverEntryPointQueryResult qres;
+    cudaError_t err = cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &qres);
+    if (err != cudaSuccess) return err;
+    if (qres != cudaDriverEntryPointSuccess || !p) return cudaErrorNotSupported;
+    cached = reinterpret_cast<EncodeTiledFn>(p);
+  }
+  *fn = cached;
+  return cudaSuccess;
+}
+
+// [B,H,N,D] bf16 tensor as a 4-D map (D, N, H, B); box = 64 columns (one 128-byte swizzle row) x 128 rows
+cudaError_t tile_map(CUtensorMap* map, const void* base, const Problem& p) {
+  EncodeTiledFn fn;
+  cudaError_t err = encode_fn(&fn);
+  if (err != cudaSuccess) return err;
+  cuuint64_t dims[4] = {(cuuint64_t)p.D, (cuuint64_t)p.N, (cuuint64_t)p.H, (cuuint64_t)p.B};
+  cuuint64_t strides[3] = {(cuuint64_t)p.sn * 2, (cuuint64_t)p.sh * 2, (cuuint64_t)p.sb * 2};
+  cuuint32_t box[4] = {64, 128, 1, 1};
+  cuuint32_t estr[4] = {1, 1, 1, 1};
+  CUresult r = fn(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, const_cast<void*>(base), dims, strides, box, estr,
+                  CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                  CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  return r == CUDA_SUCCESS ? cudaSuccess : cudaErrorInvalidValue;
+}
+
+template <int HD>
+cudaError_t launch_tile_impl(const Problem& p, const void* q, const void* k, const void* v, const TileArgsK& args,
+                             cudaStream_t stream) {
+  CUtensorMap map_q, map_k, map_v;
+  cudaError_t err = tile_map(&map_q, q, p);
+  if (err != cudaSuccess) return err;
+  err = tile_map(&map_k, k, p);
+  if (err != cudaSuccess) return err;
+  err = tile_map(&map_v, v, p);
+  if (err != cudaSuccess) return err;
+  err = cudaFuncSetAttribute(tile_fwd_kernel<HD>, cudaFuncAttributeMaxDynamicSharedMemorySize, TCfg<HD>::kSmemBytes);
+  if (err != cudaSuccess) return err;
+  int dev = 0, sms = 0;
+  err = cudaGetDevice(&dev);
+  if (err != cudaSuccess) return err;
+  err = cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+  if (err != cudaSuccess) return err;
+  const long all_tiles = (long)p.B * p.H * args.tiles_per_head;
+  const int grid = (int)(all_tiles < sms ? all_tiles : sms);
+  tile_fwd_kernel<HD><<<grid, kThreadsT, TCfg<HD>::kSmemBytes, stream>>>(map_q, map_k, map_v, args);
+  return cudaGetLastError();
+}
+
+}  // namespace
+
+cudaError_t launch_tile_fwd(const Problem& p, const void* q, const void* k, const void* v, const float* scale,
+                            const int32_t* tile_list, const int32_t* tile_count, const int32_t* row_cnt, void* o,
+                            float* tau, int32_t* status, cudaStream_t stream) {
+  TileArgsK args;
+  args.B = p.B; args.H = p.H; args.N = p.N;
+  args.causal = p.causal;
+  args.expo_class = p.expo_class;
+  args.expo = p.expo;
+  args.alpha_m1 = p.alpha - 1.0f;
+  args.sm_scale = p.sm_scale;
+  args.scale = scale;
+  args.tile_list = tile_list;
+  args.tile_count = tile_count;
+  args.row_cnt = row_cnt;
+  args.o = o;
+  args.tau = tau;
+  args.sb = p.sb; args.sh = p.sh; args.sn = p.sn;
+  args.status = status;
+  args.tiles_per_head = (p.N + TM - 1) / TM;
+  return p.D == 64 ? launch_tile_impl<64>(p, q, k, v, args, stream) : launch_tile_impl<128>(p, q, k, v, args, stream);
+}
+
+}  // namespace entmax
