@@ -109,7 +109,8 @@ int entmax_attn_bwd(const entmax_attn_params* params, const void* q, const void*
 /* Where a finished forward call leaves the support of every row inside its workspace (App. A: the
  * support of row i is {j : (alpha-1) s_ij > tau_i}).  Byte offsets from the workspace base:
  *   row_count  int32 [batch*heads*seq]: support size of the row, or -2 when the row was computed by the
- *              dense path and its list is not kept (only rows with more than `keep_limit` support entries)
+ *              dense path and its list is not kept (a row goes there when one of its two candidate
+ *              half-lists could not be kept at `keep_limit` entries at some point of the sweep)
  *   entries    {float y; int32 j;} [batch*heads*seq][capacity]: the first row_count slots hold the
  *              support, y = (alpha-1) s_ij as the kernel computed it (fp32), in no particular order
  *   scale      float32 [heads*seq]: c_i
@@ -119,7 +120,7 @@ typedef struct {
   size_t entries_offset;
   size_t scale_offset;
   int32_t capacity;
-  int32_t keep_limit; /* a row whose support exceeds this may be computed by the dense path (row_count -2)   */
+  int32_t keep_limit; /* see row_count                                                                        */
 } entmax_attn_ws_layout;
 int entmax_attn_workspace_layout(const entmax_attn_params* params, entmax_attn_ws_layout* out);
 

