@@ -56,6 +56,8 @@ def _load():
             lib.oracle_attn_bwd_head.argtypes = [fp, fp, fp, fp] + common + [dp, dp, dp]
             lib.oracle_attn_bwd_rows.restype = ctypes.c_int
             lib.oracle_attn_bwd_rows.argtypes = [fp, fp, fp, fp] + common + [ip, ctypes.c_long, dp, dp]
+            lib.oracle_attn_bwd_scale_head.restype = ctypes.c_int
+            lib.oracle_attn_bwd_scale_head.argtypes = [fp, fp, fp, fp] + common + [dp, dp]
             lib.oracle_num_threads.restype = ctypes.c_int
             lib.oracle_set_num_threads.argtypes = [ctypes.c_int]
             _lib = lib
@@ -164,3 +166,19 @@ def attn_bwd_rows(q, k, v, d_o, rows, alpha, sm_scale, causal, scale=None, n_mod
     if rc != 0:
         raise RuntimeError("oracle_attn_bwd_rows failed: %d" % rc)
     return dq, ds
+
+
+def attn_bwd_scale_head(q, k, v, d_o, alpha, sm_scale, causal, scale=None, n_mode=0):
+    """Gradients with respect to the ASEntmax scale of one head.
+    Returns (dc float64 [N], (dbeta, dgamma, ddelta))."""
+    q, k, v, d_o = _f32(q), _f32(k), _f32(v), _f32(d_o)
+    N, d = q.shape
+    dc = np.empty(N, dtype=np.float64)
+    grads = np.zeros(3, dtype=np.float64)
+    us, b, g, dl = _scale_args(scale)
+    rc = _load().oracle_attn_bwd_scale_head(_fptr(q), _fptr(k), _fptr(v), _fptr(d_o), N, d, float(alpha),
+                                            float(sm_scale), int(bool(causal)), int(n_mode), us, b, g, dl,
+                                            _dptr(dc), _dptr(grads))
+    if rc != 0:
+        raise RuntimeError("oracle_attn_bwd_scale_head failed: %d" % rc)
+    return dc, (float(grads[0]), float(grads[1]), float(grads[2]))

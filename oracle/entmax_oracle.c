@@ -15,6 +15,8 @@
  *                              sum_j p_ij v_j, with the ASEntmax scale applied to the logits.
  *   oracle_attn_bwd_head       Jacobian of Eq. 1 by implicit differentiation:
  *                              dp_j/ds_k = u_j (delta_jk - u_k / sum u), u = p^(2-alpha).
+ *   oracle_attn_bwd_scale_head chain rule through Eq. "asentmax": gradients of the per-row scale c_i and of
+ *                              the head's beta, gamma, delta.
  *
  * Pins (tests that do not use this file's own arithmetic): the paper's worked sparsemax example,
  * the two-level closed form of Lemma 2, brute-force enumeration of supports for n <= 8, the
@@ -357,6 +359,87 @@ int oracle_attn_bwd_rows(const float* q, const float* k, const float* v, const f
     free(s); free(p);
   }
   return err;
+}
+
+/* Gradients with respect to the ASEntmax scale, ONE head, all query rows.
+ * The logits are s_ij = c_i z_ij with z_ij = <q_i,k_j> * sm_scale (Sec. 2.1) and
+ * c_i = delta + beta (log n_i)^gamma (Eq. "asentmax"), so by the chain rule
+ *   dL/dc_i     = sum_j dS_ij z_ij                       (dc_out [N])
+ *   dL/ddelta   = sum_i dL/dc_i
+ *   dL/dbeta    = sum_{i: n_i > 1} dL/dc_i (log n_i)^gamma
+ *   dL/dgamma   = sum_{i: n_i > 1} dL/dc_i beta (log n_i)^gamma log(log n_i)
+ * (rows with n_i = 1 have c_i = delta).  dS as in oracle_attn_bwd_head.  grads_out = {dbeta, dgamma, ddelta}. */
+int oracle_attn_bwd_scale_head(const float* q, const float* k, const float* v, const float* d_o,
+                               long N, int d, double alpha, double sm_scale, int causal, int n_mode,
+                               int use_scale, double beta, double gamma, double delta,
+                               double* dc_out, double* grads_out) {
+  if (N <= 0 || d <= 0 || !(alpha > 1.0)) return -1;
+  int err = 0;
+#pragma omp parallel
+  {
+    double* z = (double*)malloc(sizeof(double) * (size_t)N);
+    double* s = (double*)malloc(sizeof(double) * (size_t)N);
+    double* p = (double*)malloc(sizeof(double) * (size_t)N);
+    if (!z || !s || !p) {
+#pragma omp atomic write
+      err = -2;
+    } else {
+#pragma omp for schedule(dynamic, 4)
+      for (long i = 0; i < N; ++i) {
+        long nv = visible_keys(i, N, causal);
+        long n_i = n_mode ? N : nv;
+        double c = use_scale ? oracle_asentmax_scale(beta, gamma, delta, n_i) : 1.0;
+        const float* qi = q + (size_t)i * d;
+        const float* doi = d_o + (size_t)i * d;
+        for (long j = 0; j < nv; ++j) {
+          const float* kj = k + (size_t)j * d;
+          double dot = 0.0;
+          for (int t = 0; t < d; ++t) dot += (double)qi[t] * (double)kj[t];
+          z[j] = dot * sm_scale;
+          s[j] = c * z[j];
+        }
+        double tau;
+        oracle_entmax_row(s, (int)nv, alpha, ORACLE_METHOD_AUTO, p, &tau);
+        double su = 0.0, sud = 0.0;
+        for (long j = 0; j < nv; ++j) {
+          if (p[j] > 0.0) {
+            const float* vj = v + (size_t)j * d;
+            double dp = 0.0;
+            for (int t = 0; t < d; ++t) dp += (double)doi[t] * (double)vj[t];
+            double u = (alpha == 2.0) ? 1.0 : pow(p[j], 2.0 - alpha);
+            s[j] = dp;
+            su += u;
+            sud += u * dp;
+          }
+        }
+        double rho = sud / su;
+        double dc = 0.0;
+        for (long j = 0; j < nv; ++j) {
+          if (p[j] > 0.0) {
+            double u = (alpha == 2.0) ? 1.0 : pow(p[j], 2.0 - alpha);
+            dc += u * (s[j] - rho) * z[j];
+          }
+        }
+        dc_out[i] = dc;
+      }
+    }
+    free(z); free(s); free(p);
+  }
+  if (err) return err;
+  double gb = 0.0, gg = 0.0, gd = 0.0;
+  for (long i = 0; i < N; ++i) {
+    long nv = visible_keys(i, N, causal);
+    long n_i = n_mode ? N : nv;
+    gd += dc_out[i];
+    if (n_i > 1) {
+      double L = log((double)n_i);
+      double Lg = pow(L, gamma);
+      gb += dc_out[i] * Lg;
+      gg += dc_out[i] * beta * Lg * log(L);
+    }
+  }
+  grads_out[0] = gb; grads_out[1] = gg; grads_out[2] = gd;
+  return 0;
 }
 
 int oracle_num_threads(void) {

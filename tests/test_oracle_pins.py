@@ -376,5 +376,32 @@ def test_backward_sparsemax_form_and_single_key_rows():
     assert np.all(ds[0] == 0.0)          # row 0 sees one key: one-hot, zero Jacobian
 
 
+@pytest.mark.parametrize("alpha", [1.25, 1.5, 2.0])
+@pytest.mark.parametrize("causal", [True, False])
+def test_scale_parameter_gradients_match_finite_differences(alpha, causal):
+    # L(beta, gamma, delta) = sum_i <O_i, dO_i>; central differences of the fp64 forward in each parameter
+    rng = np.random.default_rng(77)
+    N, d = 24, 8
+    q, k, v, g = (rng.normal(size=(N, d)).astype(np.float32) for _ in range(4))
+    sm = 1.0 / np.sqrt(d)
+    params = np.array([0.9, 0.7, 1.1])          # beta, gamma, delta
+    rows = np.arange(N)
+
+    def loss(par):
+        out = oracle.attn_fwd_rows(q, k, v, rows, alpha, sm, causal, scale=tuple(par))
+        return float((out["o"] * g.astype(np.float64)).sum())
+
+    dc, grads = oracle.attn_bwd_scale_head(q, k, v, g, alpha, sm, causal, scale=tuple(params))
+    for idx in range(3):
+        h = 1e-6
+        up, dn = params.copy(), params.copy()
+        up[idx] += h
+        dn[idx] -= h
+        fd = (loss(up) - loss(dn)) / (2 * h)
+        assert abs(fd - grads[idx]) <= 1e-5 * max(1.0, abs(fd)), (idx, fd, grads[idx])
+    # delta's gradient is the plain sum of the per-row scale gradients
+    assert abs(dc.sum() - grads[2]) <= 1e-12 * max(1.0, abs(grads[2]))
+
+
 def test_threads_reported():
     assert oracle.num_threads() >= 1
