@@ -106,6 +106,22 @@ int entmax_attn_bwd(const entmax_attn_params* params, const void* q, const void*
                     const void* d_o, void* dq, void* dk, void* dv, void* workspace,
                     size_t workspace_bytes, int32_t* device_status, void* cuda_stream);
 
+/* Backward pass that also returns the gradients of the ASEntmax scale (Eq. "asentmax": the temperature
+ * c_i = delta_h + beta_h (log n_i)^gamma_h is learnable).  By the chain rule through s_ij = c_i z_ij,
+ * z_ij = <q_i,k_j> sm_scale:
+ *   d_scale_rows[b,h,i] = dL/dc_i = sum_j dS_ij z_ij            out, device float32 [batch,heads,seq] or NULL
+ *   ddelta[h] = sum_{b,i} dL/dc_i,  dbeta[h] = sum_{b,i: n_i>1} dL/dc_i (log n_i)^gamma_h,
+ *   dgamma[h] = sum_{b,i: n_i>1} dL/dc_i beta_h (log n_i)^gamma_h log(log n_i)
+ *                                                               out, device float32 [heads]; all three or none;
+ *                                                               they need beta, gamma, delta to be given
+ * d_scale_rows is what a caller with per-query scales (its own c_i table) differentiates further.
+ * Everything else as entmax_attn_bwd, which is this call with the four extra outputs NULL. */
+int entmax_attn_bwd_scale(const entmax_attn_params* params, const void* q, const void* k, const void* v,
+                          const float* beta, const float* gamma, const float* delta, const float* tau,
+                          const void* d_o, void* dq, void* dk, void* dv, float* d_scale_rows, float* dbeta,
+                          float* dgamma, float* ddelta, void* workspace, size_t workspace_bytes,
+                          int32_t* device_status, void* cuda_stream);
+
 /* Where a finished forward call leaves the support of every row inside its workspace (App. A: the
  * support of row i is {j : (alpha-1) s_ij > tau_i}).  Byte offsets from the workspace base:
  *   row_count  int32 [batch*heads*seq]: support size of the row, or -2 when the row was computed by the

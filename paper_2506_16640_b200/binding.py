@@ -59,6 +59,9 @@ def load():
         lib.entmax_attn_fwd.argtypes = [pp, vp, vp, vp, fp, fp, fp, vp, fp, vp, ctypes.c_size_t, ip, vp]
         lib.entmax_attn_bwd.restype = ctypes.c_int
         lib.entmax_attn_bwd.argtypes = [pp, vp, vp, vp, fp, fp, fp, fp, vp, vp, vp, vp, vp, ctypes.c_size_t, ip, vp]
+        lib.entmax_attn_bwd_scale.restype = ctypes.c_int
+        lib.entmax_attn_bwd_scale.argtypes = [pp, vp, vp, vp, fp, fp, fp, fp, vp, vp, vp, vp, fp, fp, fp, fp, vp,
+                                              ctypes.c_size_t, ip, vp]
         lib.entmax_attn_fwd_static.restype = ctypes.c_int
         lib.entmax_attn_fwd_static.argtypes = [pp, vp, vp, vp, fp, fp, fp, vp, fp, ip, vp]
         lib.entmax_attn_scores_debug.restype = ctypes.c_int
@@ -183,6 +186,34 @@ def entmax_attn_bwd(q, k, v, tau, d_o, alpha, causal, beta=None, gamma=None, del
                                 workspace.numel(), _ptr(status), _stream_ptr(stream))
     _check(rc, "entmax_attn_bwd")
     return dq, dk, dv
+
+
+def entmax_attn_bwd_scale(q, k, v, tau, d_o, alpha, causal, beta, gamma, delta, *, sm_scale=0.0, n_mode=0,
+                          dq=None, dk=None, dv=None, d_scale_rows=None, want_param_grads=True, workspace=None,
+                          status=None, stream=None):
+    """Backward pass with the gradients of the ASEntmax scale.
+    Returns (dq, dk, dv, d_scale_rows, (dbeta, dgamma, ddelta) or None)."""
+    _same_layout(q, k, v, d_o)
+    params = make_params(q, alpha, causal, sm_scale, n_mode)
+    dq = torch.empty_like(q) if dq is None else dq
+    dk = torch.empty_like(q) if dk is None else dk
+    dv = torch.empty_like(q) if dv is None else dv
+    _same_layout(q, dq, dk, dv)
+    B, H, N, _ = q.shape
+    if d_scale_rows is None:
+        d_scale_rows = torch.empty((B, H, N), dtype=torch.float32, device=q.device)
+    grads = None
+    if want_param_grads:
+        grads = tuple(torch.empty((H,), dtype=torch.float32, device=q.device) for _ in range(3))
+    if workspace is None:
+        workspace = alloc_workspace(params, True, q.device)
+    g = grads if grads is not None else (None, None, None)
+    rc = load().entmax_attn_bwd_scale(ctypes.byref(params), _ptr(q), _ptr(k), _ptr(v), _ptr(beta), _ptr(gamma),
+                                      _ptr(delta), _ptr(tau), _ptr(d_o), _ptr(dq), _ptr(dk), _ptr(dv),
+                                      _ptr(d_scale_rows), _ptr(g[0]), _ptr(g[1]), _ptr(g[2]), _ptr(workspace),
+                                      workspace.numel(), _ptr(status), _stream_ptr(stream))
+    _check(rc, "entmax_attn_bwd_scale")
+    return dq, dk, dv, d_scale_rows, grads
 
 
 def entmax_attn_scores_debug(q, k, bh, causal, *, workspace=None, status=None, stream=None):

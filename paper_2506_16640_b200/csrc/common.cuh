@@ -42,7 +42,7 @@ struct Problem {
 };
 
 struct WsLayout {
-  size_t scale, row_cnt, half_cnt, half_thr, entries, fb_count, sweep_counter, tile_count, fb_list, tile_flag, tile_list, scratch, acc_dk, acc_dv, total;
+  size_t scale, row_cnt, half_cnt, half_thr, entries, fb_count, sweep_counter, tile_count, fb_list, tile_flag, tile_list, scratch, acc_dk, acc_dv, dc_rows, total;
   int scratch_ctas;     // CTAs of the dense-row kernels (each owns scratch_floats floats)
   size_t scratch_floats;
 };
@@ -68,8 +68,11 @@ cudaError_t launch_dense_fwd(const Problem& p, const void* q, const void* k, con
                              cudaStream_t stream);
 cudaError_t launch_dense_bwd(const Problem& p, const void* q, const void* k, const void* v, const void* d_o,
                              const float* scale, const float* tau, void* dq, float* acc_dk, float* acc_dv,
-                             const int32_t* row_list, const int32_t* row_count, float* scratch,
+                             float* dc_rows, const int32_t* row_list, const int32_t* row_count, float* scratch,
                              size_t scratch_floats, int ctas, cudaStream_t stream);
+// dbeta, dgamma, ddelta [H] from the per-row scale gradients dc_rows [B,H,N]
+cudaError_t launch_scale_grad(const Problem& p, const float* beta, const float* gamma, const float* dc_rows,
+                              float* dbeta, float* dgamma, float* ddelta, cudaStream_t stream);
 
 // tcgen05 score sweep (bf16): fills the per-row candidate lists.
 //   mode 0: threshold search (forward); mode 1: threshold given in tau_in (backward)
@@ -91,8 +94,8 @@ cudaError_t launch_row_fwd(const Problem& p, const void* v, const float* scale, 
                            cudaStream_t stream);
 cudaError_t launch_row_bwd(const Problem& p, const void* q, const void* k, const void* v, const void* d_o,
                            const float* scale, const float* tau, const int32_t* half_cnt, Entry* entries, void* dq,
-                           float* acc_dk, float* acc_dv, int32_t* fb_count, int32_t* fb_list, int32_t* status,
-                           cudaStream_t stream);
+                           float* acc_dk, float* acc_dv, float* dc_rows, int32_t* fb_count, int32_t* fb_list,
+                           int32_t* status, cudaStream_t stream);
 
 // fp32 accumulators [B,H,N,D] contiguous -> strided output tensor of the problem dtype
 cudaError_t launch_store_grad(const Problem& p, const float* acc, void* out, cudaStream_t stream);

@@ -231,7 +231,8 @@ __global__ void __launch_bounds__(kThreads) dense_bwd_kernel(Problem p, const T*
                                                              const T* __restrict__ v, const T* __restrict__ d_o,
                                                              const float* __restrict__ scale, const float* __restrict__ tau_in,
                                                              T* __restrict__ dq, float* __restrict__ acc_dk,
-                                                             float* __restrict__ acc_dv, const int32_t* __restrict__ row_list,
+                                                             float* __restrict__ acc_dv, float* __restrict__ dc_rows,
+                                                             const int32_t* __restrict__ row_list,
                                                              const int32_t* __restrict__ row_count,
                                                              float* __restrict__ scratch, size_t scratch_floats) {
   constexpr int PER = D / 32;
@@ -266,6 +267,7 @@ __global__ void __launch_bounds__(kThreads) dense_bwd_kernel(Problem p, const T*
     }
     const float2 s = block_sum2(su, sud, red);
     const float rho = s.x > 0.f ? s.y / s.x : 0.f;
+    float dcp = 0.f;                                  // sum_j dS_ij y_ij (lane 0 of every warp)
     float acc[PER];
 #pragma unroll
     for (int t = 0; t < PER; ++t) acc[t] = 0.f;
@@ -276,6 +278,7 @@ __global__ void __launch_bounds__(kThreads) dense_bwd_kernel(Problem p, const T*
         float pe, u;
         pow_pair(y, p.expo_class, p.expo, pe, u);
         const float gds = r.g * u * (dpbuf[j] - rho);
+        if (l == 0) dcp = fmaf(u * (dpbuf[j] - rho), ybuf[j], dcp);
         float ks[PER], dkv[PER], dvv[PER];
         load_slice<PER>(k + r.base + (size_t)j * p.sn + l * PER, ks);
 #pragma unroll
@@ -302,7 +305,56 @@ __global__ void __launch_bounds__(kThreads) dense_bwd_kernel(Problem p, const T*
       }
       store_slice<PER>(dq + r.base + (size_t)r.i * p.sn + threadIdx.x * PER, out);
     }
+    if (dc_rows) {
+      // dL/dc_i = sum_j dS_ij z_ij, z_ij = y_ij / ((alpha-1) c_i)  (y = (alpha-1) c z)
+      const float2 t = block_sum2(dcp, 0.f, red);
+      const float denom = (p.alpha - 1.0f) * r.c;
+      if (threadIdx.x == 0) dc_rows[r.grow] = denom != 0.f ? t.x / denom : 0.f;
+    }
     __syncthreads();
+  }
+}
+
+// dbeta_h, dgamma_h, ddelta_h from the per-row scale gradients: c_i = delta + beta L^gamma with L = ln n_i
+// (rows with n_i = 1 have c_i = delta), so d/ddelta = 1, d/dbeta = L^gamma, d/dgamma = beta L^gamma ln L.
+// One CTA per head, fp64 accumulation in a fixed order (reproducible).
+__global__ void __launch_bounds__(256) scale_grad_kernel(Problem p, const float* __restrict__ beta,
+                                                        const float* __restrict__ gamma,
+                                                        const float* __restrict__ dc_rows, float* __restrict__ dbeta,
+                                                        float* __restrict__ dgamma, float* __restrict__ ddelta) {
+  __shared__ double red[3][256];
+  const int h = blockIdx.x;
+  const double b = beta[h], g = gamma[h];
+  double sb = 0.0, sg = 0.0, sd = 0.0;
+  for (long t = threadIdx.x; t < (long)p.B * p.N; t += blockDim.x) {
+    const long bb = t / p.N;
+    const int i = (int)(t - bb * p.N);
+    const double dc = dc_rows[((size_t)bb * p.H + h) * p.N + i];
+    const long n = (p.n_mode || !p.causal) ? p.N : i + 1;
+    sd += dc;
+    if (n > 1) {
+      const double L = log((double)n);
+      const double Lg = pow(L, g);
+      sb += dc * Lg;
+      sg += dc * b * Lg * log(L);
+    }
+  }
+  red[0][threadIdx.x] = sb;
+  red[1][threadIdx.x] = sg;
+  red[2][threadIdx.x] = sd;
+  __syncthreads();
+  for (int o = 128; o > 0; o >>= 1) {
+    if (threadIdx.x < o) {
+      red[0][threadIdx.x] += red[0][threadIdx.x + o];
+      red[1][threadIdx.x] += red[1][threadIdx.x + o];
+      red[2][threadIdx.x] += red[2][threadIdx.x + o];
+    }
+    __syncthreads();
+  }
+  if (threadIdx.x == 0) {
+    dbeta[h] = (float)red[0][0];
+    dgamma[h] = (float)red[1][0];
+    ddelta[h] = (float)red[2][0];
   }
 }
 
@@ -369,11 +421,12 @@ cudaError_t launch_dense_fwd(const Problem& p, const void* q, const void* k, con
 
 cudaError_t launch_dense_bwd(const Problem& p, const void* q, const void* k, const void* v, const void* d_o,
                              const float* scale, const float* tau, void* dq, float* acc_dk, float* acc_dv,
-                             const int32_t* row_list, const int32_t* row_count, float* scratch,
+                             float* dc_rows, const int32_t* row_list, const int32_t* row_count, float* scratch,
                              size_t scratch_floats, int ctas, cudaStream_t stream) {
 #define ENTMAX_LAUNCH(T, D)                                                                                      \
   dense_bwd_kernel<T, D><<<ctas, kThreads, 0, stream>>>(p, (const T*)q, (const T*)k, (const T*)v, (const T*)d_o, \
-                                                        scale, tau, (T*)dq, acc_dk, acc_dv, row_list, row_count, \
+                                                        scale, tau, (T*)dq, acc_dk, acc_dv, dc_rows, row_list,    \
+                                                        row_count,                                                 \
                                                         scratch, scratch_floats)
   if (p.dtype == ENTMAX_ATTN_DTYPE_FP32) {
     if (p.D == 64) ENTMAX_LAUNCH(float, 64); else ENTMAX_LAUNCH(float, 128);
@@ -381,6 +434,12 @@ cudaError_t launch_dense_bwd(const Problem& p, const void* q, const void* k, con
     if (p.D == 64) ENTMAX_LAUNCH(__nv_bfloat16, 64); else ENTMAX_LAUNCH(__nv_bfloat16, 128);
   }
 #undef ENTMAX_LAUNCH
+  return cudaGetLastError();
+}
+
+cudaError_t launch_scale_grad(const Problem& p, const float* beta, const float* gamma, const float* dc_rows,
+                              float* dbeta, float* dgamma, float* ddelta, cudaStream_t stream) {
+  scale_grad_kernel<<<p.H, 256, 0, stream>>>(p, beta, gamma, dc_rows, dbeta, dgamma, ddelta);
   return cudaGetLastError();
 }
 

@@ -102,10 +102,11 @@ WsLayout make_layout(const Problem& p, bool is_bwd) {
   if (ctas > rows) ctas = rows;
   l.scratch_ctas = (int)ctas;
   l.scratch = take(ctas * l.scratch_floats * sizeof(float));
-  l.acc_dk = l.acc_dv = 0;
+  l.acc_dk = l.acc_dv = l.dc_rows = 0;
   if (is_bwd) {
     l.acc_dk = take(rows * p.D * sizeof(float));
     l.acc_dv = take(rows * p.D * sizeof(float));
+    l.dc_rows = take(rows * sizeof(float));
   }
   l.total = off;
   return l;
@@ -197,16 +198,19 @@ int entmax_attn_fwd(const entmax_attn_params* params, const void* q, const void*
   return err == cudaSuccess ? ENTMAX_ATTN_OK : fail_cuda(err);
 }
 
-int entmax_attn_bwd(const entmax_attn_params* params, const void* q, const void* k, const void* v,
-                    const float* beta, const float* gamma, const float* delta, const float* tau,
-                    const void* d_o, void* dq, void* dk, void* dv, void* workspace,
-                    size_t workspace_bytes, int32_t* device_status, void* cuda_stream) {
+int entmax_attn_bwd_scale(const entmax_attn_params* params, const void* q, const void* k, const void* v,
+                          const float* beta, const float* gamma, const float* delta, const float* tau,
+                          const void* d_o, void* dq, void* dk, void* dv, float* d_scale_rows, float* dbeta,
+                          float* dgamma, float* ddelta, void* workspace, size_t workspace_bytes,
+                          int32_t* device_status, void* cuda_stream) {
   Problem p;
   int rc = make_problem(params, &p);
   if (rc != ENTMAX_ATTN_OK) return rc;
   if (!q || !k || !v || !tau || !d_o || !dq || !dk || !dv) return ENTMAX_ATTN_EINVAL_NULL;
   rc = check_scale_ptrs(beta, gamma, delta, &p);
   if (rc != ENTMAX_ATTN_OK) return rc;
+  const int n_param_grads = (dbeta != nullptr) + (dgamma != nullptr) + (ddelta != nullptr);
+  if (n_param_grads != 0 && (n_param_grads != 3 || !p.has_scale)) return ENTMAX_ATTN_EINVAL_NULL;
   if (!aligned16(q) || !aligned16(k) || !aligned16(v) || !aligned16(tau) || !aligned16(d_o) || !aligned16(dq) ||
       !aligned16(dk) || !aligned16(dv))
     return ENTMAX_ATTN_EINVAL_ALIGN;
@@ -230,6 +234,9 @@ int entmax_attn_bwd(const entmax_attn_params* params, const void* q, const void*
   float* acc_dk = reinterpret_cast<float*>(ws + lay.acc_dk);
   float* acc_dv = reinterpret_cast<float*>(ws + lay.acc_dv);
   const size_t acc_bytes = (size_t)p.B * p.H * p.N * p.D * sizeof(float);
+  // per-row scale gradients: into the caller's array, else (when only the parameter gradients are wanted)
+  // into the workspace, else not computed
+  float* dc_rows = d_scale_rows ? d_scale_rows : (n_param_grads ? reinterpret_cast<float*>(ws + lay.dc_rows) : nullptr);
   cudaError_t err;
   if (device_status) {
     err = cudaMemsetAsync(device_status, 0, sizeof(int32_t) * ENTMAX_ATTN_STATUS_WORDS, stream);
@@ -242,7 +249,7 @@ int entmax_attn_bwd(const entmax_attn_params* params, const void* q, const void*
   err = launch_scale_table(p, beta, gamma, delta, scale, device_status, stream);
   if (err != cudaSuccess) return fail_cuda(err);
   if (p.dtype == ENTMAX_ATTN_DTYPE_FP32) {
-    err = launch_dense_bwd(p, q, k, v, d_o, scale, tau, dq, acc_dk, acc_dv, nullptr, nullptr, scratch,
+    err = launch_dense_bwd(p, q, k, v, d_o, scale, tau, dq, acc_dk, acc_dv, dc_rows, nullptr, nullptr, scratch,
                            lay.scratch_floats, lay.scratch_ctas, stream);
     if (err != cudaSuccess) return fail_cuda(err);
   } else {
@@ -253,17 +260,30 @@ int entmax_attn_bwd(const entmax_attn_params* params, const void* q, const void*
                        stream);
     if (err != cudaSuccess) return fail_cuda(err);
     if (g_prof_stop[1]) cudaEventRecord(g_prof_stop[1], stream);
-    err = launch_row_bwd(p, q, k, v, d_o, scale, tau, half_cnt, entries, dq, acc_dk, acc_dv, fb_count, fb_list,
+    err = launch_row_bwd(p, q, k, v, d_o, scale, tau, half_cnt, entries, dq, acc_dk, acc_dv, dc_rows, fb_count, fb_list,
                          device_status, stream);
     if (err != cudaSuccess) return fail_cuda(err);
-    err = launch_dense_bwd(p, q, k, v, d_o, scale, tau, dq, acc_dk, acc_dv, fb_list, fb_count, scratch,
+    err = launch_dense_bwd(p, q, k, v, d_o, scale, tau, dq, acc_dk, acc_dv, dc_rows, fb_list, fb_count, scratch,
                            lay.scratch_floats, lay.scratch_ctas, stream);
     if (err != cudaSuccess) return fail_cuda(err);
   }
   err = launch_store_grad(p, acc_dk, dk, stream);
   if (err != cudaSuccess) return fail_cuda(err);
   err = launch_store_grad(p, acc_dv, dv, stream);
-  return err == cudaSuccess ? ENTMAX_ATTN_OK : fail_cuda(err);
+  if (err != cudaSuccess) return fail_cuda(err);
+  if (n_param_grads) {
+    err = launch_scale_grad(p, beta, gamma, dc_rows, dbeta, dgamma, ddelta, stream);
+    if (err != cudaSuccess) return fail_cuda(err);
+  }
+  return ENTMAX_ATTN_OK;
+}
+
+int entmax_attn_bwd(const entmax_attn_params* params, const void* q, const void* k, const void* v,
+                    const float* beta, const float* gamma, const float* delta, const float* tau,
+                    const void* d_o, void* dq, void* dk, void* dv, void* workspace,
+                    size_t workspace_bytes, int32_t* device_status, void* cuda_stream) {
+  return entmax_attn_bwd_scale(params, q, k, v, beta, gamma, delta, tau, d_o, dq, dk, dv, nullptr, nullptr, nullptr,
+                               nullptr, workspace, workspace_bytes, device_status, cuda_stream);
 }
 
 int entmax_attn_scores_debug(const entmax_attn_params* params, const void* q, const void* k, int32_t bh,

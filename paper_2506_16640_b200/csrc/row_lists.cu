@@ -490,7 +490,8 @@ __device__ __forceinline__ void bwd_row_full(const Problem& p, const __nv_bfloat
                                              const __nv_bfloat16* __restrict__ d_o, const float* __restrict__ scale,
                                              const float* __restrict__ tau_in, const Entry* __restrict__ entries,
                                              __nv_bfloat16* __restrict__ dq, float* __restrict__ acc_dk,
-                                             float* __restrict__ acc_dv, int grow, int c0, int c1, int lane) {
+                                             float* __restrict__ acc_dv, float* __restrict__ dc_rows, int grow, int c0,
+                                             int c1, int lane) {
   constexpr int PER = D / 32;
   const int bh = grow / p.N, i = grow - bh * p.N, b = bh / p.H, h = bh - b * p.H;
   const float g = scale[(size_t)h * p.N + i] * p.sm_scale;
@@ -501,7 +502,7 @@ __device__ __forceinline__ void bwd_row_full(const Problem& p, const __nv_bfloat
   load_bf16<PER>(q + hbase + (size_t)i * p.sn, qs);
   load_bf16<PER>(d_o + hbase + (size_t)i * p.sn, gs);
   const Entry* list = entries + (size_t)grow * kListCap;
-  float yv[kSlots], dpv[kSlots];
+  float yv[kSlots], dpv[kSlots], zz[kSlots];
   int jj[kSlots];
 #pragma unroll
   for (int s = 0; s < kSlots; ++s) {
@@ -509,10 +510,12 @@ __device__ __forceinline__ void bwd_row_full(const Problem& p, const __nv_bfloat
     yv[s] = -1.0f;
     jj[s] = 0;
     dpv[s] = 0.f;
+    zz[s] = 0.f;
     if (e < c0 + c1) {
       const Entry en = list[e < c0 ? e : kHalfCap + e - c0];
       yv[s] = fmaf(a, en.y, -tau);
       jj[s] = en.j;
+      zz[s] = en.y;                                  // raw <q_i, k_j>
     }
   }
   // dP_ij = <dO_i, v_j> on the support
@@ -545,6 +548,14 @@ __device__ __forceinline__ void bwd_row_full(const Problem& p, const __nv_bfloat
   su = warp_sum(su);
   sud = warp_sum(sud);
   const float rho = su > 0.f ? sud / su : 0.f;
+  if (dc_rows) {
+    // dL/dc_i = sum_j dS_ij z_ij with z_ij = <q_i,k_j> sm_scale (chain rule through s = c z)
+    float dc = 0.f;
+#pragma unroll
+    for (int s = 0; s < kSlots; ++s) dc = fmaf(u[s] * (dpv[s] - rho), zz[s], dc);
+    dc = warp_sum(dc);
+    if (lane == 0) dc_rows[grow] = dc * p.sm_scale;
+  }
   float acc[PER];
 #pragma unroll
   for (int t = 0; t < PER; ++t) acc[t] = 0.f;
@@ -581,8 +592,8 @@ __device__ __forceinline__ void bwd_rows_quad(const Problem& p, const __nv_bfloa
                                               const __nv_bfloat16* __restrict__ d_o, const float* __restrict__ scale,
                                               const float* __restrict__ tau_in, const Entry* __restrict__ entries,
                                               __nv_bfloat16* __restrict__ dq, float* __restrict__ acc_dk,
-                                              float* __restrict__ acc_dv, int grow, bool active, int c0, int c1,
-                                              int lane) {
+                                              float* __restrict__ acc_dv, float* __restrict__ dc_rows, int grow,
+                                              bool active, int c0, int c1, int lane) {
   constexpr int PL = D / 8;                        // elements of a row per lane
   const int sl = lane & 7;
   const int base = lane & 24;
@@ -596,12 +607,13 @@ __device__ __forceinline__ void bwd_rows_quad(const Problem& p, const __nv_bfloa
   load_bf16_vec<PL>(q + hbase + (size_t)i * p.sn, qs);
   load_bf16_vec<PL>(d_o + hbase + (size_t)i * p.sn, gs);
   const Entry* list = entries + (size_t)grow * kListCap;
-  float yv = -1.0f;
+  float yv = -1.0f, zz = 0.f;
   int j = 0;
   if (sl < n) {
     const Entry en = list[sl < c0 ? sl : kHalfCap + sl - c0];
     yv = fmaf(a, en.y, -tau);
     j = en.j;
+    zz = en.y;                                     // raw <q_i, k_j>
   }
   const bool in = yv > 0.f;
   const unsigned msub = (__ballot_sync(0xffffffffu, in) >> base) & 0xffu;
@@ -627,6 +639,11 @@ __device__ __forceinline__ void bwd_rows_quad(const Problem& p, const __nv_bfloa
   const float su = oct_sum(u), sud = oct_sum(u * dpv);
   const float rho = su > 0.f ? sud / su : 0.f;
   const float gds_own = g * u * (dpv - rho);
+  if (dc_rows) {
+    // dL/dc_i = sum_j dS_ij z_ij with z_ij = <q_i,k_j> sm_scale (chain rule through s = c z)
+    const float dc = oct_sum(u * (dpv - rho) * zz);
+    if (active && sl == 0) dc_rows[grow] = dc * p.sm_scale;
+  }
   float acc[PL];
 #pragma unroll
   for (int t = 0; t < PL; ++t) acc[t] = 0.f;
@@ -659,8 +676,8 @@ __global__ void __launch_bounds__(kWarpsPerCta * 32) row_bwd_kernel(
     Problem p, const __nv_bfloat16* __restrict__ q, const __nv_bfloat16* __restrict__ k,
     const __nv_bfloat16* __restrict__ v, const __nv_bfloat16* __restrict__ d_o, const float* __restrict__ scale,
     const float* __restrict__ tau_in, const int32_t* __restrict__ half_cnt, const Entry* __restrict__ entries,
-    __nv_bfloat16* __restrict__ dq, float* __restrict__ acc_dk, float* __restrict__ acc_dv, int32_t* fb_count,
-    int32_t* fb_list, int32_t* status) {
+    __nv_bfloat16* __restrict__ dq, float* __restrict__ acc_dk, float* __restrict__ acc_dv,
+    float* __restrict__ dc_rows, int32_t* fb_count, int32_t* fb_list, int32_t* status) {
   const int lane = threadIdx.x & 31;
   const int total = p.B * p.H * p.N;
   const int groups = (total + 3) / 4;
@@ -676,8 +693,8 @@ __global__ void __launch_bounds__(kWarpsPerCta * 32) row_bwd_kernel(
     }
     const bool small = !my_active || (mc0 >= 0 && mc1 >= 0 && mc0 + mc1 <= 8);
     if (__all_sync(0xffffffffu, small)) {
-      bwd_rows_quad<D>(p, q, k, v, d_o, scale, tau_in, entries, dq, acc_dk, acc_dv, my_active ? my_row : 0, my_active,
-                       mc0, mc1, lane);
+      bwd_rows_quad<D>(p, q, k, v, d_o, scale, tau_in, entries, dq, acc_dk, acc_dv, dc_rows, my_active ? my_row : 0,
+                       my_active, mc0, mc1, lane);
       continue;
     }
     for (int r = 0; r < 4; ++r) {
@@ -688,7 +705,7 @@ __global__ void __launch_bounds__(kWarpsPerCta * 32) row_bwd_kernel(
         if (lane == 0) push_dense_row(grow, fb_count, fb_list, status);
         continue;
       }
-      bwd_row_full<D>(p, q, k, v, d_o, scale, tau_in, entries, dq, acc_dk, acc_dv, grow, c0, c1, lane);
+      bwd_row_full<D>(p, q, k, v, d_o, scale, tau_in, entries, dq, acc_dk, acc_dv, dc_rows, grow, c0, c1, lane);
     }
   }
 }
@@ -720,17 +737,17 @@ cudaError_t launch_row_fwd(const Problem& p, const void* v, const float* scale, 
 
 cudaError_t launch_row_bwd(const Problem& p, const void* q, const void* k, const void* v, const void* d_o,
                            const float* scale, const float* tau, const int32_t* half_cnt, Entry* entries, void* dq,
-                           float* acc_dk, float* acc_dv, int32_t* fb_count, int32_t* fb_list, int32_t* status,
-                           cudaStream_t stream) {
+                           float* acc_dk, float* acc_dv, float* dc_rows, int32_t* fb_count, int32_t* fb_list,
+                           int32_t* status, cudaStream_t stream) {
   const int grid = row_grid(p);
   if (p.D == 64)
     row_bwd_kernel<64><<<grid, kWarpsPerCta * 32, 0, stream>>>(
         p, (const __nv_bfloat16*)q, (const __nv_bfloat16*)k, (const __nv_bfloat16*)v, (const __nv_bfloat16*)d_o, scale,
-        tau, half_cnt, entries, (__nv_bfloat16*)dq, acc_dk, acc_dv, fb_count, fb_list, status);
+        tau, half_cnt, entries, (__nv_bfloat16*)dq, acc_dk, acc_dv, dc_rows, fb_count, fb_list, status);
   else
     row_bwd_kernel<128><<<grid, kWarpsPerCta * 32, 0, stream>>>(
         p, (const __nv_bfloat16*)q, (const __nv_bfloat16*)k, (const __nv_bfloat16*)v, (const __nv_bfloat16*)d_o, scale,
-        tau, half_cnt, entries, (__nv_bfloat16*)dq, acc_dk, acc_dv, fb_count, fb_list, status);
+        tau, half_cnt, entries, (__nv_bfloat16*)dq, acc_dk, acc_dv, dc_rows, fb_count, fb_list, status);
   return cudaGetLastError();
 }
 

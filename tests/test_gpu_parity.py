@@ -9,6 +9,7 @@ import torch
 from paper_2506_16640_b200 import binding, inputs
 from paper_2506_16640_b200.inputs import WORKLOADS, Workload, make_inputs, sample_rows, scaled
 
+import oracle as oracle_mod
 import parity
 
 pytestmark = pytest.mark.gpu
@@ -144,6 +145,34 @@ def test_backward_small_full_heads(N, d, dtype, causal, alpha):
     bwd = parity.run_bwd(inp, alpha, got["tau"], got["dev"])
     for bh in range(inp.workload.H):
         parity.check_bwd_head(inp, alpha, bwd, bh)
+
+
+# ------------------------------------------------------------------ gradients of the ASEntmax scale
+@pytest.mark.parametrize("alpha", [1.25, 1.5, 2.0])
+@pytest.mark.parametrize("N,d,dtype,causal,sigma,plant", [(300, 64, "bf16", True, 1.0, 2), (700, 128, "bf16", False, 1.0, 0),
+                                                          (260, 64, "bf16", True, 0.05, 0), (97, 64, "fp32", True, 1.0, 0)])
+def test_scale_gradients(N, d, dtype, causal, sigma, plant, alpha):
+    # sigma 0.05 makes every row dense (the dense backward path computes the same gradients)
+    inp = make_inputs(_small("dscale", N, d, causal, dtype=dtype, plant=plant, backward=True, sigma=sigma, seed=N + 1))
+    w = inp.workload
+    got = parity.run_fwd(inp, alpha)
+    dev = got["dev"]
+    dq, dk, dv, dc, grads = binding.entmax_attn_bwd_scale(dev["q"], dev["k"], dev["v"], got["tau"], dev["d_o"], alpha,
+                                                          causal, dev["beta"], dev["gamma"], dev["delta"])
+    torch.cuda.synchronize()
+    ref_g = np.zeros((w.H, 3))
+    for h in range(w.H):
+        q, k, v, g = (t[0, h].float().numpy() for t in (inp.q, inp.k, inp.v, inp.d_o))
+        dc_ref, gr = oracle_mod.attn_bwd_scale_head(q, k, v, g, alpha, inp.sm_scale, causal, scale=inp.head_scale(h))
+        ref_g[h] = gr
+        parity.grad_close("dc rows", dc[0, h].cpu().numpy(), dc_ref)
+    for idx, name in enumerate(("dbeta", "dgamma", "ddelta")):
+        got_g = grads[idx].cpu().double().numpy()
+        tol = 2e-2 * max(1.0, np.abs(ref_g[:, idx]).max())
+        assert np.abs(got_g - ref_g[:, idx]).max() <= tol, (name, got_g, ref_g[:, idx])
+    # the plain backward entry point is the same call without the extra outputs
+    plain = parity.run_bwd(inp, alpha, got["tau"], dev)
+    assert torch.equal(plain["dq"], dq)
 
 
 # ------------------------------------------------------------------ the benchmark workloads
