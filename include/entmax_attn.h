@@ -122,6 +122,23 @@ int entmax_attn_bwd_scale(const entmax_attn_params* params, const void* q, const
                           float* dgamma, float* ddelta, void* workspace, size_t workspace_bytes,
                           int32_t* device_status, void* cuda_stream);
 
+/* Forward / backward with a per-query scale table instead of per-head beta, gamma, delta: the paper's
+ * full ASEntmax makes beta and gamma functions of the query (Sec. 4.1: beta = softplus(X w_beta),
+ * gamma = s tanh(X w_gamma)), so c_i differs per batch element.  The caller evaluates Eq. "asentmax"
+ * upstream and passes
+ *   c_rows        in, device float32 [batch, heads, seq]: c_i of every query row (any finite value)
+ * and gets back, from the backward call,
+ *   d_scale_rows  out, device float32 [batch, heads, seq] or NULL: dL/dc_i, to be chained into its own
+ *                 projection weights.
+ * params->n_mode is ignored; everything else as entmax_attn_fwd / entmax_attn_bwd. */
+int entmax_attn_fwd_rowscale(const entmax_attn_params* params, const void* q, const void* k, const void* v,
+                             const float* c_rows, void* o, float* tau, void* workspace, size_t workspace_bytes,
+                             int32_t* device_status, void* cuda_stream);
+int entmax_attn_bwd_rowscale(const entmax_attn_params* params, const void* q, const void* k, const void* v,
+                             const float* c_rows, const float* tau, const void* d_o, void* dq, void* dk, void* dv,
+                             float* d_scale_rows, void* workspace, size_t workspace_bytes, int32_t* device_status,
+                             void* cuda_stream);
+
 /* Where a finished forward call leaves the support of every row inside its workspace (App. A: the
  * support of row i is {j : (alpha-1) s_ij > tau_i}).  Byte offsets from the workspace base:
  *   row_count  int32 [batch*heads*seq]: support size of the row, or -2 when the row was computed by the

@@ -62,6 +62,10 @@ def load():
         lib.entmax_attn_bwd_scale.restype = ctypes.c_int
         lib.entmax_attn_bwd_scale.argtypes = [pp, vp, vp, vp, fp, fp, fp, fp, vp, vp, vp, vp, fp, fp, fp, fp, vp,
                                               ctypes.c_size_t, ip, vp]
+        lib.entmax_attn_fwd_rowscale.restype = ctypes.c_int
+        lib.entmax_attn_fwd_rowscale.argtypes = [pp, vp, vp, vp, fp, vp, fp, vp, ctypes.c_size_t, ip, vp]
+        lib.entmax_attn_bwd_rowscale.restype = ctypes.c_int
+        lib.entmax_attn_bwd_rowscale.argtypes = [pp, vp, vp, vp, fp, fp, vp, vp, vp, vp, fp, vp, ctypes.c_size_t, ip, vp]
         lib.entmax_attn_fwd_static.restype = ctypes.c_int
         lib.entmax_attn_fwd_static.argtypes = [pp, vp, vp, vp, fp, fp, fp, vp, fp, ip, vp]
         lib.entmax_attn_scores_debug.restype = ctypes.c_int
@@ -214,6 +218,45 @@ def entmax_attn_bwd_scale(q, k, v, tau, d_o, alpha, causal, beta, gamma, delta, 
                                       workspace.numel(), _ptr(status), _stream_ptr(stream))
     _check(rc, "entmax_attn_bwd_scale")
     return dq, dk, dv, d_scale_rows, grads
+
+
+def entmax_attn_fwd_rowscale(q, k, v, c_rows, alpha, causal, *, sm_scale=0.0, o=None, tau=None, workspace=None,
+                             status=None, stream=None):
+    """Forward pass with a per-query scale table c_rows (float32 [B,H,N]).  Returns (o, tau)."""
+    _same_layout(q, k, v)
+    params = make_params(q, alpha, causal, sm_scale, 0)
+    B, H, N, _ = q.shape
+    if c_rows.shape != (B, H, N) or c_rows.dtype != torch.float32 or not c_rows.is_contiguous():
+        raise EntmaxAttnError("c_rows must be a contiguous float32 [batch, heads, seq] tensor")
+    o = torch.empty_like(q) if o is None else o
+    if tau is None:
+        tau = torch.empty((B, H, N), dtype=torch.float32, device=q.device)
+    if workspace is None:
+        workspace = alloc_workspace(params, False, q.device)
+    rc = load().entmax_attn_fwd_rowscale(ctypes.byref(params), _ptr(q), _ptr(k), _ptr(v), _ptr(c_rows), _ptr(o),
+                                         _ptr(tau), _ptr(workspace), workspace.numel(), _ptr(status), _stream_ptr(stream))
+    _check(rc, "entmax_attn_fwd_rowscale")
+    return o, tau
+
+
+def entmax_attn_bwd_rowscale(q, k, v, c_rows, tau, d_o, alpha, causal, *, sm_scale=0.0, dq=None, dk=None, dv=None,
+                             d_scale_rows=None, workspace=None, status=None, stream=None):
+    """Backward pass with a per-query scale table.  Returns (dq, dk, dv, d_scale_rows)."""
+    _same_layout(q, k, v, d_o)
+    params = make_params(q, alpha, causal, sm_scale, 0)
+    B, H, N, _ = q.shape
+    dq = torch.empty_like(q) if dq is None else dq
+    dk = torch.empty_like(q) if dk is None else dk
+    dv = torch.empty_like(q) if dv is None else dv
+    if d_scale_rows is None:
+        d_scale_rows = torch.empty((B, H, N), dtype=torch.float32, device=q.device)
+    if workspace is None:
+        workspace = alloc_workspace(params, True, q.device)
+    rc = load().entmax_attn_bwd_rowscale(ctypes.byref(params), _ptr(q), _ptr(k), _ptr(v), _ptr(c_rows), _ptr(tau),
+                                         _ptr(d_o), _ptr(dq), _ptr(dk), _ptr(dv), _ptr(d_scale_rows), _ptr(workspace),
+                                         workspace.numel(), _ptr(status), _stream_ptr(stream))
+    _check(rc, "entmax_attn_bwd_rowscale")
+    return dq, dk, dv, d_scale_rows
 
 
 def entmax_attn_scores_debug(q, k, bh, causal, *, workspace=None, status=None, stream=None):

@@ -110,7 +110,7 @@ __device__ __forceinline__ RowCtx make_row(const Problem& p, const float* scale,
   r.b = r.bh / p.H;
   r.h = r.bh - r.b * p.H;
   r.nv = p.causal ? r.i + 1 : p.N;
-  r.c = scale[(size_t)r.h * p.N + r.i];
+  r.c = scale[(size_t)r.b * p.scale_sb + (size_t)r.h * p.N + r.i];
   r.g = r.c * p.sm_scale;
   r.a = (p.alpha - 1.0f) * r.g;
   r.base = (size_t)r.b * p.sb + (size_t)r.h * p.sh;

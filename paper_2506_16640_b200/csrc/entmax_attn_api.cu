@@ -51,6 +51,7 @@ int make_problem(const entmax_attn_params* params, Problem* out) {
     if (p.sn % 8 || p.sh % 8 || p.sb % 8) return ENTMAX_ATTN_EINVAL_SHAPE;
   }
   p.has_scale = 0;
+  p.scale_sb = 0;
   *out = p;
   return ENTMAX_ATTN_OK;
 }
@@ -138,15 +139,22 @@ int entmax_attn_workspace_layout(const entmax_attn_params* params, entmax_attn_w
   return ENTMAX_ATTN_OK;
 }
 
-int entmax_attn_fwd(const entmax_attn_params* params, const void* q, const void* k, const void* v,
-                    const float* beta, const float* gamma, const float* delta, void* o, float* tau,
-                    void* workspace, size_t workspace_bytes, int32_t* device_status, void* cuda_stream) {
+}  // extern "C"
+
+namespace {
+
+// Forward pass; c_rows, when given, is a per-query scale table [B,H,N] that replaces the one the library
+// computes from beta, gamma, delta.
+int fwd_impl(const entmax_attn_params* params, const void* q, const void* k, const void* v, const float* beta,
+             const float* gamma, const float* delta, const float* c_rows, void* o, float* tau, void* workspace,
+             size_t workspace_bytes, int32_t* device_status, void* cuda_stream) {
   Problem p;
   int rc = make_problem(params, &p);
   if (rc != ENTMAX_ATTN_OK) return rc;
   if (!q || !k || !v || !o || !tau) return ENTMAX_ATTN_EINVAL_NULL;
   rc = check_scale_ptrs(beta, gamma, delta, &p);
   if (rc != ENTMAX_ATTN_OK) return rc;
+  if (c_rows && (reinterpret_cast<uintptr_t>(c_rows) & 3u)) return ENTMAX_ATTN_EINVAL_ALIGN;
   if (!aligned16(q) || !aligned16(k) || !aligned16(v) || !aligned16(o) || !aligned16(tau)) return ENTMAX_ATTN_EINVAL_ALIGN;
   WsLayout lay;
   rc = check_workspace(p, false, workspace, workspace_bytes, &lay);
@@ -157,7 +165,7 @@ int entmax_attn_fwd(const entmax_attn_params* params, const void* q, const void*
   }
   cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
   uint8_t* ws = static_cast<uint8_t*>(workspace);
-  float* scale = reinterpret_cast<float*>(ws + lay.scale);
+  const float* scale = reinterpret_cast<float*>(ws + lay.scale);
   int32_t* row_cnt = reinterpret_cast<int32_t*>(ws + lay.row_cnt);
   int32_t* half_cnt = reinterpret_cast<int32_t*>(ws + lay.half_cnt);
   float* half_thr = reinterpret_cast<float*>(ws + lay.half_thr);
@@ -171,8 +179,13 @@ int entmax_attn_fwd(const entmax_attn_params* params, const void* q, const void*
     err = cudaMemsetAsync(device_status, 0, sizeof(int32_t) * ENTMAX_ATTN_STATUS_WORDS, stream);
     if (err != cudaSuccess) return fail_cuda(err);
   }
-  err = launch_scale_table(p, beta, gamma, delta, scale, device_status, stream);
-  if (err != cudaSuccess) return fail_cuda(err);
+  if (c_rows) {
+    scale = c_rows;
+    p.scale_sb = (int64_t)p.H * p.N;
+  } else {
+    err = launch_scale_table(p, beta, gamma, delta, reinterpret_cast<float*>(ws + lay.scale), device_status, stream);
+    if (err != cudaSuccess) return fail_cuda(err);
+  }
   if (p.dtype == ENTMAX_ATTN_DTYPE_FP32) {
     err = launch_dense_fwd(p, q, k, v, scale, o, tau, row_cnt, entries, nullptr, nullptr, scratch, lay.scratch_floats,
                            lay.scratch_ctas, stream);
@@ -198,11 +211,33 @@ int entmax_attn_fwd(const entmax_attn_params* params, const void* q, const void*
   return err == cudaSuccess ? ENTMAX_ATTN_OK : fail_cuda(err);
 }
 
-int entmax_attn_bwd_scale(const entmax_attn_params* params, const void* q, const void* k, const void* v,
-                          const float* beta, const float* gamma, const float* delta, const float* tau,
-                          const void* d_o, void* dq, void* dk, void* dv, float* d_scale_rows, float* dbeta,
-                          float* dgamma, float* ddelta, void* workspace, size_t workspace_bytes,
-                          int32_t* device_status, void* cuda_stream) {
+}  // namespace
+
+extern "C" {
+
+int entmax_attn_fwd(const entmax_attn_params* params, const void* q, const void* k, const void* v,
+                    const float* beta, const float* gamma, const float* delta, void* o, float* tau,
+                    void* workspace, size_t workspace_bytes, int32_t* device_status, void* cuda_stream) {
+  return fwd_impl(params, q, k, v, beta, gamma, delta, nullptr, o, tau, workspace, workspace_bytes, device_status,
+                  cuda_stream);
+}
+
+int entmax_attn_fwd_rowscale(const entmax_attn_params* params, const void* q, const void* k, const void* v,
+                             const float* c_rows, void* o, float* tau, void* workspace, size_t workspace_bytes,
+                             int32_t* device_status, void* cuda_stream) {
+  if (!c_rows) return ENTMAX_ATTN_EINVAL_NULL;
+  return fwd_impl(params, q, k, v, nullptr, nullptr, nullptr, c_rows, o, tau, workspace, workspace_bytes, device_status,
+                  cuda_stream);
+}
+
+}  // extern "C"
+
+namespace {
+
+int bwd_impl(const entmax_attn_params* params, const void* q, const void* k, const void* v, const float* beta,
+             const float* gamma, const float* delta, const float* c_rows, const float* tau, const void* d_o, void* dq,
+             void* dk, void* dv, float* d_scale_rows, float* dbeta, float* dgamma, float* ddelta, void* workspace,
+             size_t workspace_bytes, int32_t* device_status, void* cuda_stream) {
   Problem p;
   int rc = make_problem(params, &p);
   if (rc != ENTMAX_ATTN_OK) return rc;
@@ -210,7 +245,8 @@ int entmax_attn_bwd_scale(const entmax_attn_params* params, const void* q, const
   rc = check_scale_ptrs(beta, gamma, delta, &p);
   if (rc != ENTMAX_ATTN_OK) return rc;
   const int n_param_grads = (dbeta != nullptr) + (dgamma != nullptr) + (ddelta != nullptr);
-  if (n_param_grads != 0 && (n_param_grads != 3 || !p.has_scale)) return ENTMAX_ATTN_EINVAL_NULL;
+  if (n_param_grads != 0 && (n_param_grads != 3 || !p.has_scale || c_rows)) return ENTMAX_ATTN_EINVAL_NULL;
+  if (c_rows && (reinterpret_cast<uintptr_t>(c_rows) & 3u)) return ENTMAX_ATTN_EINVAL_ALIGN;
   if (!aligned16(q) || !aligned16(k) || !aligned16(v) || !aligned16(tau) || !aligned16(d_o) || !aligned16(dq) ||
       !aligned16(dk) || !aligned16(dv))
     return ENTMAX_ATTN_EINVAL_ALIGN;
@@ -223,7 +259,7 @@ int entmax_attn_bwd_scale(const entmax_attn_params* params, const void* q, const
   }
   cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
   uint8_t* ws = static_cast<uint8_t*>(workspace);
-  float* scale = reinterpret_cast<float*>(ws + lay.scale);
+  const float* scale = reinterpret_cast<float*>(ws + lay.scale);
   int32_t* half_cnt = reinterpret_cast<int32_t*>(ws + lay.half_cnt);
   float* half_thr = reinterpret_cast<float*>(ws + lay.half_thr);
   int32_t* sweep_counter = reinterpret_cast<int32_t*>(ws + lay.sweep_counter);
@@ -246,8 +282,13 @@ int entmax_attn_bwd_scale(const entmax_attn_params* params, const void* q, const
   if (err != cudaSuccess) return fail_cuda(err);
   err = cudaMemsetAsync(acc_dv, 0, acc_bytes, stream);
   if (err != cudaSuccess) return fail_cuda(err);
-  err = launch_scale_table(p, beta, gamma, delta, scale, device_status, stream);
-  if (err != cudaSuccess) return fail_cuda(err);
+  if (c_rows) {
+    scale = c_rows;
+    p.scale_sb = (int64_t)p.H * p.N;
+  } else {
+    err = launch_scale_table(p, beta, gamma, delta, reinterpret_cast<float*>(ws + lay.scale), device_status, stream);
+    if (err != cudaSuccess) return fail_cuda(err);
+  }
   if (p.dtype == ENTMAX_ATTN_DTYPE_FP32) {
     err = launch_dense_bwd(p, q, k, v, d_o, scale, tau, dq, acc_dk, acc_dv, dc_rows, nullptr, nullptr, scratch,
                            lay.scratch_floats, lay.scratch_ctas, stream);
@@ -276,6 +317,28 @@ int entmax_attn_bwd_scale(const entmax_attn_params* params, const void* q, const
     if (err != cudaSuccess) return fail_cuda(err);
   }
   return ENTMAX_ATTN_OK;
+}
+
+}  // namespace
+
+extern "C" {
+
+int entmax_attn_bwd_scale(const entmax_attn_params* params, const void* q, const void* k, const void* v,
+                          const float* beta, const float* gamma, const float* delta, const float* tau,
+                          const void* d_o, void* dq, void* dk, void* dv, float* d_scale_rows, float* dbeta,
+                          float* dgamma, float* ddelta, void* workspace, size_t workspace_bytes,
+                          int32_t* device_status, void* cuda_stream) {
+  return bwd_impl(params, q, k, v, beta, gamma, delta, nullptr, tau, d_o, dq, dk, dv, d_scale_rows, dbeta, dgamma,
+                  ddelta, workspace, workspace_bytes, device_status, cuda_stream);
+}
+
+int entmax_attn_bwd_rowscale(const entmax_attn_params* params, const void* q, const void* k, const void* v,
+                             const float* c_rows, const float* tau, const void* d_o, void* dq, void* dk, void* dv,
+                             float* d_scale_rows, void* workspace, size_t workspace_bytes, int32_t* device_status,
+                             void* cuda_stream) {
+  if (!c_rows) return ENTMAX_ATTN_EINVAL_NULL;
+  return bwd_impl(params, q, k, v, nullptr, nullptr, nullptr, c_rows, tau, d_o, dq, dk, dv, d_scale_rows, nullptr,
+                  nullptr, nullptr, workspace, workspace_bytes, device_status, cuda_stream);
 }
 
 int entmax_attn_bwd(const entmax_attn_params* params, const void* q, const void* k, const void* v,

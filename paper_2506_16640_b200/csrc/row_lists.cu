@@ -351,7 +351,7 @@ __device__ __forceinline__ void solve_rows_quad(const Problem& p, const __nv_bfl
   const int base = lane & 24;
   const int n = active ? c0 + c1 : 0;
   const int bh = grow / p.N, i = grow - bh * p.N, b = bh / p.H, h = bh - b * p.H;
-  const float a = active ? (p.alpha - 1.0f) * (scale[(size_t)h * p.N + i] * p.sm_scale) : 1.0f;
+  const float a = active ? (p.alpha - 1.0f) * (scale[(size_t)b * p.scale_sb + (size_t)h * p.N + i] * p.sm_scale) : 1.0f;
   Entry* list = entries + (size_t)grow * kListCap;
   float y = -INFINITY;
   int j = 0x7fffffff;
@@ -474,7 +474,7 @@ __global__ void __launch_bounds__(kWarpsPerCta * 32) row_fwd_kernel(Problem p, c
         continue;
       }
       const int bh = grow / p.N, i = grow - bh * p.N, b = bh / p.H, h = bh - b * p.H;
-      const float a = (p.alpha - 1.0f) * (scale[(size_t)h * p.N + i] * p.sm_scale);
+      const float a = (p.alpha - 1.0f) * (scale[(size_t)b * p.scale_sb + (size_t)h * p.N + i] * p.sm_scale);
       Entry* list = entries + (size_t)grow * kListCap;
       const __nv_bfloat16* vbase = v + (size_t)b * p.sb + (size_t)h * p.sh + lane * PER;
       __nv_bfloat16* o_row = o + (size_t)b * p.sb + (size_t)h * p.sh + (size_t)i * p.sn + lane * PER;
@@ -494,7 +494,7 @@ __device__ __forceinline__ void bwd_row_full(const Problem& p, const __nv_bfloat
                                              int c1, int lane) {
   constexpr int PER = D / 32;
   const int bh = grow / p.N, i = grow - bh * p.N, b = bh / p.H, h = bh - b * p.H;
-  const float g = scale[(size_t)h * p.N + i] * p.sm_scale;
+  const float g = scale[(size_t)b * p.scale_sb + (size_t)h * p.N + i] * p.sm_scale;
   const float a = (p.alpha - 1.0f) * g;
   const float tau = tau_in[grow];
   const size_t hbase = (size_t)b * p.sb + (size_t)h * p.sh + lane * PER;
@@ -599,7 +599,7 @@ __device__ __forceinline__ void bwd_rows_quad(const Problem& p, const __nv_bfloa
   const int base = lane & 24;
   const int n = active ? c0 + c1 : 0;
   const int bh = grow / p.N, i = grow - bh * p.N, b = bh / p.H, h = bh - b * p.H;
-  const float g = active ? scale[(size_t)h * p.N + i] * p.sm_scale : 0.f;
+  const float g = active ? scale[(size_t)b * p.scale_sb + (size_t)h * p.N + i] * p.sm_scale : 0.f;
   const float a = (p.alpha - 1.0f) * g;
   const float tau = active ? tau_in[grow] : 0.f;
   const size_t hbase = (size_t)b * p.sb + (size_t)h * p.sh + sl * PL;

@@ -68,7 +68,8 @@ struct SweepArgs {
   float expo;
   float alpha_m1;       // alpha - 1
   float sm_scale;
-  const float* scale;   // [H, N]
+  const float* scale;   // [H, N] (scale_sb = 0) or [B, H, N] (scale_sb = H*N)
+  long long scale_sb;
   const float* tau_in;  // [B*H*N] (mode 1)
   int32_t* half_cnt;    // [B*H*N][2] list length of each half-row; -1 = hand the row to the dense path
   float* half_thr;      // [B*H*N][2] lower bound on tau each half-row ended with (Eq. 1's units)
@@ -387,7 +388,7 @@ __global__ void __launch_bounds__(kThreads, 1) sweep_kernel(const __grid_constan
       r.thr = INFINITY;
       float ra = 1.f, inv_a = 1.f;
       if (valid) {
-        ra = a.alpha_m1 * (a.scale[(size_t)h * a.N + i] * a.sm_scale);
+        ra = a.alpha_m1 * (a.scale[(size_t)(bh / a.H) * a.scale_sb + (size_t)h * a.N + i] * a.sm_scale);
         if (ra > 0.f && ra < INFINITY) {
           inv_a = 1.0f / ra;
           if (a.mode == 0) {
@@ -606,6 +607,7 @@ cudaError_t launch_sweep(const Problem& p, const void* q, const void* k, const f
   args.alpha_m1 = p.alpha - 1.0f;
   args.sm_scale = p.sm_scale;
   args.scale = scale;
+  args.scale_sb = p.scale_sb;
   args.tau_in = tau_in;
   args.half_cnt = half_cnt;
   args.half_thr = half_thr;

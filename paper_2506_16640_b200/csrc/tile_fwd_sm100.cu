@@ -51,7 +51,8 @@ struct TileArgsK {
   float expo;
   float alpha_m1;
   float sm_scale;
-  const float* scale;        // [H, N]
+  const float* scale;        // [H, N] (scale_sb = 0) or [B, H, N] (scale_sb = H*N)
+  long long scale_sb;
   const int32_t* tile_list;  // ids of the Q tiles to process: bh * tiles_per_head + tile
   const int32_t* tile_count;
   const int32_t* row_cnt;    // -2 marks the rows to write
@@ -305,7 +306,7 @@ __global__ void __launch_bounds__(kThreadsT, 1) tile_fwd_kernel(const __grid_con
       const bool valid = i < a.N;
       const size_t grow = (size_t)bh * a.N + (valid ? i : 0);
       const int lim = a.causal ? i : a.N - 1;
-      const float ra = valid ? a.alpha_m1 * (a.scale[(size_t)h * a.N + i] * a.sm_scale) : 0.f;
+      const float ra = valid ? a.alpha_m1 * (a.scale[(size_t)b * a.scale_sb + (size_t)h * a.N + i] * a.sm_scale) : 0.f;
       float tau = 0.f, ymax = -INFINITY;
       bool done = !valid;
       for (int s = 0; s < kMaxSweeps && alive; ++s) {
@@ -529,6 +530,7 @@ cudaError_t launch_tile_fwd(const Problem& p, const void* q, const void* k, cons
   args.alpha_m1 = p.alpha - 1.0f;
   args.sm_scale = p.sm_scale;
   args.scale = scale;
+  args.scale_sb = p.scale_sb;
   args.tile_list = tile_list;
   args.tile_count = tile_count;
   args.row_cnt = row_cnt;

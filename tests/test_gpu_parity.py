@@ -175,6 +175,58 @@ def test_scale_gradients(N, d, dtype, causal, sigma, plant, alpha):
     assert torch.equal(plain["dq"], dq)
 
 
+# ------------------------------------------------------------------ per-query scale tables
+def test_rowscale_equals_per_head_call_when_given_the_same_table():
+    inp = make_inputs(_small("rowscale_same", 700, 128, True, plant=3, backward=True, B=2, seed=41))
+    w = inp.workload
+    got = parity.run_fwd(inp, 1.5)
+    dev = got["dev"]
+    lay = binding.entmax_attn_workspace_layout(got["params"])
+    table = got["workspace"][lay.scale_offset: lay.scale_offset + 4 * w.H * w.N].view(torch.float32).view(w.H, w.N)
+    c_rows = table.unsqueeze(0).expand(w.B, w.H, w.N).contiguous()
+    o, tau = binding.entmax_attn_fwd_rowscale(dev["q"], dev["k"], dev["v"], c_rows, 1.5, True)
+    torch.cuda.synchronize()
+    assert torch.equal(o, got["o"]) and torch.equal(tau, got["tau"])
+    ref = binding.entmax_attn_bwd_scale(dev["q"], dev["k"], dev["v"], tau, dev["d_o"], 1.5, True, dev["beta"],
+                                        dev["gamma"], dev["delta"], want_param_grads=False)
+    dq, dk, dv, dc = binding.entmax_attn_bwd_rowscale(dev["q"], dev["k"], dev["v"], c_rows, tau, dev["d_o"], 1.5, True)
+    torch.cuda.synchronize()
+    assert torch.equal(dq, ref[0]) and torch.equal(dc, ref[3])
+    # dK, dV are sums of fp32 atomics: equal up to the order of the additions
+    for a_, b_ in ((dk, ref[1]), (dv, ref[2])):
+        assert (a_.float() - b_.float()).abs().max().item() <= 2e-2 * max(1.0, b_.float().abs().max().item())
+
+
+@pytest.mark.parametrize("alpha", [1.5, 2.0])
+@pytest.mark.parametrize("dtype", ["bf16", "fp32"])
+def test_rowscale_with_a_batch_dependent_table_matches_the_oracle(dtype, alpha):
+    # c differs per batch element and per row; the oracle sees row i with beta = 0, delta = c_i
+    N, d = 96, 64
+    inp = make_inputs(_small("rowscale_rows", N, d, True, dtype=dtype, backward=True, B=2, use_scale=False, seed=43))
+    w = inp.workload
+    gen = torch.Generator().manual_seed(4343)
+    c_host = torch.rand((w.B, w.H, N), generator=gen) * 6.0 + 0.5
+    dev = parity.to_device(inp)
+    c_rows = c_host.cuda()
+    o, tau = binding.entmax_attn_fwd_rowscale(dev["q"], dev["k"], dev["v"], c_rows, alpha, True)
+    dq, dk, dv, dc = binding.entmax_attn_bwd_rowscale(dev["q"], dev["k"], dev["v"], c_rows, tau, dev["d_o"], alpha, True)
+    torch.cuda.synchronize()
+    tol_tau = parity.tau_tol(dtype)
+    for b in range(w.B):
+        for h in range(w.H):
+            q, k, v, g = (t[b, h].float().numpy() for t in (inp.q, inp.k, inp.v, inp.d_o))
+            for i in range(0, N, 5):
+                sc = (0.0, 1.0, float(c_host[b, h, i]))
+                rows = np.array([i])
+                f = oracle_mod.attn_fwd_rows(q, k, v, rows, alpha, inp.sm_scale, True, scale=sc)
+                assert abs(float(tau[b, h, i]) - f["tau"][0]) <= tol_tau * max(1.0, abs(f["tau"][0]))
+                assert np.abs(o[b, h, i].float().cpu().numpy() - f["o"][0]).max() <= parity.O_TOL
+                dq_ref, _ = oracle_mod.attn_bwd_rows(q, k, v, g, rows, alpha, inp.sm_scale, True, scale=sc)
+                parity.grad_close("dQ row", dq[b, h, i].float().cpu().numpy(), dq_ref[0])
+                dc_ref, _ = oracle_mod.attn_bwd_scale_head(q, k, v, g, alpha, inp.sm_scale, True, scale=sc)
+                parity.grad_close("dc row", np.array([float(dc[b, h, i])]), np.array([dc_ref[i]]))
+
+
 # ------------------------------------------------------------------ the benchmark workloads
 def test_cfg2_all_rows():
     inp = make_inputs(WORKLOADS[2])
