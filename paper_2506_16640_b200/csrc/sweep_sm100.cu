@@ -109,6 +109,31 @@ __device__ __forceinline__ int qtile_tiles(const SweepArgs& a, int item, int x) 
   return last_row / BN + 1;
 }
 
+// Sampled tiles.  In forward mode an item first scores its query rows against every kSampleStride-th
+// key (a second view of K: the key index split into (index / stride, index % stride), phase 0 taken),
+// maxima only: the running maxima and thresholds the real stream then starts from are already close to
+// their final values, which roughly halves the candidates it pushes (a one-pass stream pushes every new
+// running maximum, about ln n of them per row; after a 1/32 sample about ln 32 are left).
+constexpr int kSampleStride = 32;
+constexpr int kSampleMinKeys = 4096;   // below this the stream is too short for the sample to pay
+__device__ __forceinline__ int sample_tiles(const SweepArgs& a, int item) {
+  if (a.mode != 0) return 0;
+  int last_row = item * kItemRows + kItemRows - 1;
+  if (last_row > a.N - 1) last_row = a.N - 1;
+  const int n_vis = a.causal ? last_row + 1 : a.N;
+  if (n_vis < kSampleMinKeys) return 0;
+  int groups = (n_vis + kSampleStride - 1) / kSampleStride;
+  if (groups > a.N / kSampleStride) groups = a.N / kSampleStride;
+  return (groups + BN - 1) / BN;
+}
+__device__ __forceinline__ void tma_load_5d(uint32_t dst, const CUtensorMap* map, uint32_t bar, int c0, int c1, int c2,
+                                            int c3, int c4) {
+  asm volatile(
+      "cp.async.bulk.tensor.5d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5, %6, %7}], [%2];"
+      ::"r"(dst), "l"(reinterpret_cast<uint64_t>(map)), "r"(bar), "r"(c0), "r"(c1), "r"(c2), "r"(c3), "r"(c4)
+      : "memory");
+}
+
 // ------------------------------------------------------------- consumer side: one half-row per thread
 struct RowState {
   float thr;       // candidates are accumulators above this (accumulator units)
@@ -192,6 +217,7 @@ __device__ __noinline__ RowState shrink_lists(RowState r, Entry* list, float a, 
 template <int HD, bool kDump>
 __global__ void __launch_bounds__(kThreads, 1) sweep_kernel(const __grid_constant__ CUtensorMap map_q,
                                                             const __grid_constant__ CUtensorMap map_k,
+                                                            const __grid_constant__ CUtensorMap map_ks,
                                                             const SweepArgs a) {
   using C = Cfg<HD>;
   extern __shared__ uint8_t smem_raw[];
@@ -271,12 +297,16 @@ __global__ void __launch_bounds__(kThreads, 1) sweep_kernel(const __grid_constan
           const int tx = qtile_tiles(a, item, x);
           tiles = tx > tiles ? tx : tiles;
         }
-        for (int t = 0; t < tiles && alive; ++t) {
+        const int ts = sample_tiles(a, item);
+        for (int t = 0; t < ts + tiles && alive; ++t) {
           alive = mbar_wait(k_empty + 8 * stage, kphase ^ 1u, abort_flag);
           if (!alive) break;
           mbar_expect_tx(k_full + 8 * stage, C::kKBytes);
-          for (int hf = 0; hf < C::kHalves; ++hf)
-            tma_load_4d(k_smem + stage * C::kKBytes + hf * (BN * 128), &map_k, k_full + 8 * stage, hf * 64, t * BN, h, b);
+          for (int hf = 0; hf < C::kHalves; ++hf) {
+            const uint32_t dst = k_smem + stage * C::kKBytes + hf * (BN * 128);
+            if (t < ts) tma_load_5d(dst, &map_ks, k_full + 8 * stage, hf * 64, 0, t * BN, h, b);
+            else tma_load_4d(dst, &map_k, k_full + 8 * stage, hf * 64, (t - ts) * BN, h, b);
+          }
           if (++stage == C::kStages) { stage = 0; kphase ^= 1u; }
           if (t == 0) {
             // Q tile slots past the end of the sequence are neither loaded nor used; each slot keeps
@@ -317,13 +347,15 @@ __global__ void __launch_bounds__(kThreads, 1) sweep_kernel(const __grid_constan
           tx[x] = qtile_tiles(a, item, x);
           tiles = tx[x] > tiles ? tx[x] : tiles;
         }
-        for (int t = 0; t < tiles && alive; ++t) {
+        const int ts = sample_tiles(a, item);
+        for (int t = 0; t < ts + tiles && alive; ++t) {
           alive = mbar_wait(k_full + 8 * stage, kphase, abort_flag);
           if (!alive) break;
           const uint32_t b_lo = k_lo + stage * (C::kKBytes >> 4);
 #pragma unroll
           for (int x = 0; x < kQTiles; ++x) {
-            if (t >= tx[x] || !alive) continue;
+            // every valid Q tile takes all sampled tiles, then its own share of the real ones
+            if (tx[x] == 0 || t >= ts + tx[x] || !alive) continue;
             if (t == 0) {
               alive = mbar_wait(q_full + 8 * x, (qphase >> x) & 1u, abort_flag);
               qphase ^= 1u << x;
@@ -341,7 +373,7 @@ __global__ void __launch_bounds__(kThreads, 1) sweep_kernel(const __grid_constan
               umma_bf16(tmem_base + x * BN, a_lo + a_off, b_lo + b_off, kDescHi, idesc, kk > 0 ? 1u : 0u);
             }
             umma_commit(s_full + 8 * x);
-            if (t == tx[x] - 1) umma_commit(q_empty + 8 * x);
+            if (t == ts + tx[x] - 1) umma_commit(q_empty + 8 * x);
           }
           if (!alive) break;
           umma_commit(k_empty + 8 * stage);
@@ -407,6 +439,41 @@ __global__ void __launch_bounds__(kThreads, 1) sweep_kernel(const __grid_constan
       // halves that reach past the first one need the mask
       const int first_lim = a.causal ? tile_row0 : a.N - 1;
       const int last_lim = a.causal ? (tile_row0 + BM - 1 < a.N - 1 ? tile_row0 + BM - 1 : a.N - 1) : a.N - 1;
+      // ---- sampled tiles first (forward mode, long rows): maxima only, nothing is pushed -- every sampled
+      //      key comes by again in the real stream.  Column c of sampled tile t is key kSampleStride * (t*BN + c).
+      const int ts = sample_tiles(a, item);
+      if (ts > 0) {
+        // largest sampled group index that is a key this row may look at
+        int glim = lim / kSampleStride;
+        if (glim > a.N / kSampleStride - 1) glim = a.N / kSampleStride - 1;
+        for (int t = 0; t < ts && alive; ++t) {
+          alive = __all_sync(0xffffffffu, mbar_wait(my_full, fphase, abort_flag));
+          if (!alive) break;
+          fphase ^= 1u;
+          tc_fence_after();
+          const int g_base = t * BN + half * kHalfCols;
+          float m_s = -INFINITY;
+          float va[32];
+#pragma unroll
+          for (int c = 0; c < 4; ++c) {
+            tmem_ld32(taddr_row + c * 32, va);
+            tmem_ld_wait();
+#pragma unroll
+            for (int u = 0; u < 32; ++u) va[u] = (g_base + c * 32 + u <= glim) ? va[u] : -INFINITY;
+            m_s = max3(m_s, fmaxf(max8(&va[0]), max8(&va[8])), fmaxf(max8(&va[16]), max8(&va[24])));
+          }
+          tc_fence_before();
+          __syncwarp();
+          if (lane == 0) mbar_arrive(my_empty);
+          if (searching) {
+            const unsigned long long o = lds_u64(other_share);
+            const float m_other = (int)(o >> 32) == k ? __uint_as_float((unsigned)o) : -INFINITY;
+            r.m_run = max3(r.m_run, m_s, m_other);
+            r.thr = fmaxf(r.thr, r.m_run - inv_a);
+            sts_u64(my_share, ((unsigned long long)(unsigned)k << 32) | __float_as_uint(r.m_run));
+          }
+        }
+      }
       for (int t = 0; t < tiles && alive; ++t) {
         // the warp leaves together: tcgen05.ld needs all 32 lanes
         alive = __all_sync(0xffffffffu, mbar_wait(my_full, fphase, abort_flag));
@@ -571,13 +638,38 @@ cudaError_t make_map(CUtensorMap* map, const void* base, const Problem& p, int b
   return r == CUDA_SUCCESS ? cudaSuccess : cudaErrorInvalidValue;
 }
 
+// K as a 5-D map (D, key % stride, key / stride, H, B): a box of BN rows along "key / stride" at phase 0
+// is every kSampleStride-th key.  Keys past stride * (N / stride) are not part of the view.
+cudaError_t make_sample_map(CUtensorMap* map, const void* base, const Problem& p) {
+  EncodeTiledFn fn;
+  cudaError_t err = get_encode_fn(&fn);
+  if (err != cudaSuccess) return err;
+  const cuuint64_t groups = (cuuint64_t)(p.N / kSampleStride);
+  cuuint64_t dims[5] = {(cuuint64_t)p.D, (cuuint64_t)kSampleStride, groups > 0 ? groups : 1, (cuuint64_t)p.H,
+                        (cuuint64_t)p.B};
+  cuuint64_t strides[4] = {(cuuint64_t)p.sn * 2, (cuuint64_t)p.sn * 2 * kSampleStride, (cuuint64_t)p.sh * 2,
+                           (cuuint64_t)p.sb * 2};
+  cuuint32_t box[5] = {64, 1, (cuuint32_t)BN, 1, 1};
+  cuuint32_t estr[5] = {1, 1, 1, 1, 1};
+  CUresult r = fn(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 5, const_cast<void*>(base), dims, strides, box, estr,
+                  CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                  CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  return r == CUDA_SUCCESS ? cudaSuccess : cudaErrorInvalidValue;
+}
+
 template <int HD, bool kDump>
 cudaError_t launch_impl(const Problem& p, const void* q, const void* k, SweepArgs& args, cudaStream_t stream) {
-  CUtensorMap map_q, map_k;
+  CUtensorMap map_q, map_k, map_ks;
   cudaError_t err = make_map(&map_q, q, p, BM);
   if (err != cudaSuccess) return err;
   err = make_map(&map_k, k, p, BN);
   if (err != cudaSuccess) return err;
+  if (p.N >= kSampleMinKeys) {
+    err = make_sample_map(&map_ks, k, p);
+    if (err != cudaSuccess) return err;
+  } else {
+    map_ks = map_k;   // never used: sample_tiles() is 0 for short sequences
+  }
   err = cudaFuncSetAttribute(sweep_kernel<HD, kDump>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                              Cfg<HD>::kSmemBytes);
   if (err != cudaSuccess) return err;
@@ -589,7 +681,7 @@ cudaError_t launch_impl(const Problem& p, const void* q, const void* k, SweepArg
   err = cudaMemsetAsync(args.work_counter, 0, sizeof(int32_t), stream);
   if (err != cudaSuccess) return err;
   const int grid = args.n_items < sms ? args.n_items : sms;
-  sweep_kernel<HD, kDump><<<grid, kThreads, Cfg<HD>::kSmemBytes, stream>>>(map_q, map_k, args);
+  sweep_kernel<HD, kDump><<<grid, kThreads, Cfg<HD>::kSmemBytes, stream>>>(map_q, map_k, map_ks, args);
   return cudaGetLastError();
 }
 
