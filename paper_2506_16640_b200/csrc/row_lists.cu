@@ -671,8 +671,9 @@ __device__ __forceinline__ void bwd_rows_quad(const Problem& p, const __nv_bfloa
   if (active) store_bf16_vec<PL>(dq + hbase + (size_t)i * p.sn, acc);
 }
 
+// (register cap: three CTAs per SM -- this kernel waits on gathers and atomics, occupancy is what hides them)
 template <int D>
-__global__ void __launch_bounds__(kWarpsPerCta * 32) row_bwd_kernel(
+__global__ void __launch_bounds__(kWarpsPerCta * 32, 4) row_bwd_kernel(
     Problem p, const __nv_bfloat16* __restrict__ q, const __nv_bfloat16* __restrict__ k,
     const __nv_bfloat16* __restrict__ v, const __nv_bfloat16* __restrict__ d_o, const float* __restrict__ scale,
     const float* __restrict__ tau_in, const int32_t* __restrict__ half_cnt, const Entry* __restrict__ entries,
