@@ -49,7 +49,7 @@ def _load():
             lib.oracle_asentmax_scale.restype = ctypes.c_double
             lib.oracle_asentmax_scale.argtypes = [ctypes.c_double] * 3 + [ctypes.c_long]
             common = [ctypes.c_long, ctypes.c_int, ctypes.c_double, ctypes.c_double, ctypes.c_int,
-                      ctypes.c_int, ctypes.c_int, ctypes.c_double, ctypes.c_double, ctypes.c_double]
+                      ctypes.c_int, ctypes.c_int, ctypes.c_double, ctypes.c_double, ctypes.c_double, ctypes.c_double]
             lib.oracle_attn_fwd_rows.restype = ctypes.c_int
             lib.oracle_attn_fwd_rows.argtypes = [fp, fp, fp] + common + [ip, ctypes.c_long, dp, dp, dp, ip]
             lib.oracle_attn_bwd_head.restype = ctypes.c_int
@@ -111,11 +111,12 @@ def _scale_args(scale):
     return 1, float(b), float(g), float(dl)
 
 
-def attn_fwd_rows(q, k, v, rows, alpha, sm_scale, causal, scale=None, n_mode=0, want_p=False):
+def attn_fwd_rows(q, k, v, rows, alpha, sm_scale, causal, scale=None, n_mode=0, want_p=False, alibi=0.0):
     """Forward of one head for the query rows in ``rows``.
 
     q, k, v: [N, d] arrays (values already rounded to the precision under test).
     scale: None (fixed temperature) or (beta, gamma, delta) of this head.
+    alibi: ALiBi slope m of this head (0 = no positional term).
     Returns dict(tau [R], o [R, d], supp [R], p [R, N] or None).
     """
     q, k, v = _f32(q), _f32(k), _f32(v)
@@ -128,14 +129,14 @@ def attn_fwd_rows(q, k, v, rows, alpha, sm_scale, causal, scale=None, n_mode=0, 
     p = np.empty((R, N), dtype=np.float64) if want_p else None
     us, b, g, dl = _scale_args(scale)
     rc = _load().oracle_attn_fwd_rows(_fptr(q), _fptr(k), _fptr(v), N, d, float(alpha), float(sm_scale),
-                                      int(bool(causal)), int(n_mode), us, b, g, dl, _iptr(rows), R,
+                                      int(bool(causal)), int(n_mode), us, b, g, dl, float(alibi), _iptr(rows), R,
                                       _dptr(tau), _dptr(o), _dptr(p) if want_p else None, _iptr(supp))
     if rc != 0:
         raise RuntimeError("oracle_attn_fwd_rows failed: %d" % rc)
     return {"tau": tau, "o": o, "supp": supp, "p": p}
 
 
-def attn_bwd_head(q, k, v, d_o, alpha, sm_scale, causal, scale=None, n_mode=0):
+def attn_bwd_head(q, k, v, d_o, alpha, sm_scale, causal, scale=None, n_mode=0, alibi=0.0):
     """Backward of one head, every row. Returns (dq, dk, dv) as float64 [N, d]."""
     q, k, v, d_o = _f32(q), _f32(k), _f32(v), _f32(d_o)
     N, d = q.shape
@@ -144,14 +145,14 @@ def attn_bwd_head(q, k, v, d_o, alpha, sm_scale, causal, scale=None, n_mode=0):
     dv = np.empty((N, d), dtype=np.float64)
     us, b, g, dl = _scale_args(scale)
     rc = _load().oracle_attn_bwd_head(_fptr(q), _fptr(k), _fptr(v), _fptr(d_o), N, d, float(alpha),
-                                      float(sm_scale), int(bool(causal)), int(n_mode), us, b, g, dl,
+                                      float(sm_scale), int(bool(causal)), int(n_mode), us, b, g, dl, float(alibi),
                                       _dptr(dq), _dptr(dk), _dptr(dv))
     if rc != 0:
         raise RuntimeError("oracle_attn_bwd_head failed: %d" % rc)
     return dq, dk, dv
 
 
-def attn_bwd_rows(q, k, v, d_o, rows, alpha, sm_scale, causal, scale=None, n_mode=0, want_ds=False):
+def attn_bwd_rows(q, k, v, d_o, rows, alpha, sm_scale, causal, scale=None, n_mode=0, want_ds=False, alibi=0.0):
     """Row-local backward (dQ rows, optionally dS rows) of one head for ``rows``."""
     q, k, v, d_o = _f32(q), _f32(k), _f32(v), _f32(d_o)
     N, d = q.shape
@@ -161,14 +162,14 @@ def attn_bwd_rows(q, k, v, d_o, rows, alpha, sm_scale, causal, scale=None, n_mod
     ds = np.empty((R, N), dtype=np.float64) if want_ds else None
     us, b, g, dl = _scale_args(scale)
     rc = _load().oracle_attn_bwd_rows(_fptr(q), _fptr(k), _fptr(v), _fptr(d_o), N, d, float(alpha),
-                                      float(sm_scale), int(bool(causal)), int(n_mode), us, b, g, dl,
+                                      float(sm_scale), int(bool(causal)), int(n_mode), us, b, g, dl, float(alibi),
                                       _iptr(rows), R, _dptr(dq), _dptr(ds) if want_ds else None)
     if rc != 0:
         raise RuntimeError("oracle_attn_bwd_rows failed: %d" % rc)
     return dq, ds
 
 
-def attn_bwd_scale_head(q, k, v, d_o, alpha, sm_scale, causal, scale=None, n_mode=0):
+def attn_bwd_scale_head(q, k, v, d_o, alpha, sm_scale, causal, scale=None, n_mode=0, alibi=0.0):
     """Gradients with respect to the ASEntmax scale of one head.
     Returns (dc float64 [N], (dbeta, dgamma, ddelta))."""
     q, k, v, d_o = _f32(q), _f32(k), _f32(v), _f32(d_o)
@@ -177,7 +178,7 @@ def attn_bwd_scale_head(q, k, v, d_o, alpha, sm_scale, causal, scale=None, n_mod
     grads = np.zeros(3, dtype=np.float64)
     us, b, g, dl = _scale_args(scale)
     rc = _load().oracle_attn_bwd_scale_head(_fptr(q), _fptr(k), _fptr(v), _fptr(d_o), N, d, float(alpha),
-                                            float(sm_scale), int(bool(causal)), int(n_mode), us, b, g, dl,
+                                            float(sm_scale), int(bool(causal)), int(n_mode), us, b, g, dl, float(alibi),
                                             _dptr(dc), _dptr(grads))
     if rc != 0:
         raise RuntimeError("oracle_attn_bwd_scale_head failed: %d" % rc)

@@ -11,8 +11,9 @@
  *                              alpha = 1.5, bisection inside the bracket of Eq. "bounds_entmax"
  *                              for any other alpha.
  *   oracle_asentmax_scale      Eq. "asentmax": c = delta + beta * (log n)^gamma.
- *   oracle_attn_fwd_rows       Sec. 2.1: z_ij = <q_i,k_j>/sqrt(d), causal j <= i, output
- *                              sum_j p_ij v_j, with the ASEntmax scale applied to the logits.
+ *   oracle_attn_fwd_rows       Sec. 2.1: z_ij = <q_i,k_j>/sqrt(d) (+ the ALiBi term m (j - i) of App. B when a
+ *                              slope is given), causal j <= i, output sum_j p_ij v_j, with the ASEntmax scale
+ *                              applied to the whole logit.
  *   oracle_attn_bwd_head       Jacobian of Eq. 1 by implicit differentiation:
  *                              dp_j/ds_k = u_j (delta_jk - u_k / sum u), u = p^(2-alpha).
  *   oracle_attn_bwd_scale_head chain rule through Eq. "asentmax": gradients of the per-row scale c_i and of
@@ -153,6 +154,14 @@ double oracle_asentmax_scale(double beta, double gamma, double delta, long n) {
 
 static long visible_keys(long i, long N, int causal) { return causal ? i + 1 : N; }
 
+/* ALiBi positional term of the logits (App. B "Positional encodings"): z_ij = <q_i,k_j>/sqrt(d) + m (j - i)
+ * for j <= i, a penalty linear in the distance; for keys after the query (non-causal use) the same penalty
+ * by distance, -m |j - i|.  m = 0 is NoPE. */
+static double alibi_bias(double slope, long i, long j) {
+  long dist = j <= i ? i - j : j - i;
+  return -slope * (double)dist;
+}
+
 /* Forward for selected query rows of ONE head.
  *   q,k,v        [N,d] row-major, float (bf16- or fp32-rounded values, converted exactly)
  *   use_scale    0: c_i = 1 (fixed temperature); 1: c_i from beta,gamma,delta
@@ -163,7 +172,7 @@ static long visible_keys(long i, long N, int causal) { return causal ? i + 1 : N
  */
 int oracle_attn_fwd_rows(const float* q, const float* k, const float* v, long N, int d,
                          double alpha, double sm_scale, int causal, int n_mode, int use_scale,
-                         double beta, double gamma, double delta,
+                         double beta, double gamma, double delta, double alibi_slope,
                          const int64_t* rows, long nrows,
                          double* tau_out, double* o_out, double* p_out, int64_t* supp_out) {
   if (N <= 0 || d <= 0 || !(alpha > 1.0)) return -1;
@@ -187,7 +196,7 @@ int oracle_attn_fwd_rows(const float* q, const float* k, const float* v, long N,
           const float* kj = k + (size_t)j * d;
           double dot = 0.0;
           for (int t = 0; t < d; ++t) dot += (double)qi[t] * (double)kj[t];
-          s[j] = c * (dot * sm_scale);
+          s[j] = c * (dot * sm_scale + alibi_bias(alibi_slope, i, j));
         }
         double tau;
         int supp = oracle_entmax_row(s, (int)nv, alpha, ORACLE_METHOD_AUTO, p, &tau);
@@ -222,7 +231,7 @@ int oracle_attn_fwd_rows(const float* q, const float* k, const float* v, long N,
  * dV_j = sum_i p_ij dO_i. */
 int oracle_attn_bwd_head(const float* q, const float* k, const float* v, const float* d_o,
                          long N, int d, double alpha, double sm_scale, int causal, int n_mode,
-                         int use_scale, double beta, double gamma, double delta,
+                         int use_scale, double beta, double gamma, double delta, double alibi_slope,
                          double* dq, double* dk, double* dv) {
   if (N <= 0 || d <= 0 || !(alpha > 1.0)) return -1;
   size_t nd = (size_t)N * d;
@@ -252,7 +261,7 @@ int oracle_attn_bwd_head(const float* q, const float* k, const float* v, const f
           const float* kj = k + (size_t)j * d;
           double dot = 0.0;
           for (int t = 0; t < d; ++t) dot += (double)qi[t] * (double)kj[t];
-          s[j] = c * (dot * sm_scale);
+          s[j] = c * (dot * sm_scale + alibi_bias(alibi_slope, i, j));
         }
         double tau;
         oracle_entmax_row(s, (int)nv, alpha, ORACLE_METHOD_AUTO, p, &tau);
@@ -300,7 +309,7 @@ int oracle_attn_bwd_head(const float* q, const float* k, const float* v, const f
  * ds_out NULL or [nrows,N]. */
 int oracle_attn_bwd_rows(const float* q, const float* k, const float* v, const float* d_o,
                          long N, int d, double alpha, double sm_scale, int causal, int n_mode,
-                         int use_scale, double beta, double gamma, double delta,
+                         int use_scale, double beta, double gamma, double delta, double alibi_slope,
                          const int64_t* rows, long nrows, double* dq_out, double* ds_out) {
   if (N <= 0 || d <= 0 || !(alpha > 1.0)) return -1;
   int err = 0;
@@ -325,7 +334,7 @@ int oracle_attn_bwd_rows(const float* q, const float* k, const float* v, const f
           const float* kj = k + (size_t)j * d;
           double dot = 0.0;
           for (int t = 0; t < d; ++t) dot += (double)qi[t] * (double)kj[t];
-          s[j] = c * (dot * sm_scale);
+          s[j] = c * (dot * sm_scale + alibi_bias(alibi_slope, i, j));
         }
         double tau;
         oracle_entmax_row(s, (int)nv, alpha, ORACLE_METHOD_AUTO, p, &tau);
@@ -371,7 +380,7 @@ int oracle_attn_bwd_rows(const float* q, const float* k, const float* v, const f
  * (rows with n_i = 1 have c_i = delta).  dS as in oracle_attn_bwd_head.  grads_out = {dbeta, dgamma, ddelta}. */
 int oracle_attn_bwd_scale_head(const float* q, const float* k, const float* v, const float* d_o,
                                long N, int d, double alpha, double sm_scale, int causal, int n_mode,
-                               int use_scale, double beta, double gamma, double delta,
+                               int use_scale, double beta, double gamma, double delta, double alibi_slope,
                                double* dc_out, double* grads_out) {
   if (N <= 0 || d <= 0 || !(alpha > 1.0)) return -1;
   int err = 0;
@@ -395,7 +404,7 @@ int oracle_attn_bwd_scale_head(const float* q, const float* k, const float* v, c
           const float* kj = k + (size_t)j * d;
           double dot = 0.0;
           for (int t = 0; t < d; ++t) dot += (double)qi[t] * (double)kj[t];
-          z[j] = dot * sm_scale;
+          z[j] = dot * sm_scale + alibi_bias(alibi_slope, i, j);
           s[j] = c * z[j];
         }
         double tau;

@@ -403,5 +403,82 @@ def test_scale_parameter_gradients_match_finite_differences(alpha, causal):
     assert abs(dc.sum() - grads[2]) <= 1e-12 * max(1.0, abs(grads[2]))
 
 
+# ------------------------------------------------------------------ ALiBi term (App. B, positional encodings)
+@pytest.mark.parametrize("alpha", [1.25, 1.5, 2.0])
+def test_alibi_equals_plain_attention_on_augmented_vectors(alpha):
+    # m (j - i) = m j - m i: the first part is one more feature (q' = [q, 1], k'_j = [k_j, m j / sm_scale]),
+    # the second a per-row shift, which leaves p unchanged and moves tau by (alpha-1) c_i (-m i)
+    rng = np.random.default_rng(5)
+    N, d, m, sm = 40, 4, 0.25, 0.5
+    q, k, v = (rng.normal(size=(N, d)).astype(np.float32) for _ in range(3))
+    scale = (0.7, 0.9, 1.2)
+    rows = np.arange(N)
+    with_bias = oracle.attn_fwd_rows(q, k, v, rows, alpha, sm, True, scale=scale, want_p=True, alibi=m)
+    q2 = np.concatenate([q, np.ones((N, 1), np.float32)], axis=1)
+    k2 = np.concatenate([k, (m * np.arange(N) / sm).astype(np.float32)[:, None]], axis=1)
+    v2 = np.concatenate([v, np.zeros((N, 1), np.float32)], axis=1)
+    plain = oracle.attn_fwd_rows(q2, k2, v2, rows, alpha, sm, True, scale=scale, want_p=True)
+    np.testing.assert_allclose(with_bias["p"], plain["p"], atol=1e-12)
+    np.testing.assert_allclose(with_bias["o"], plain["o"][:, :d], atol=1e-12)
+    c = np.array([oracle.asentmax_scale(*scale, i + 1) for i in range(N)])
+    np.testing.assert_allclose(with_bias["tau"], plain["tau"] - (alpha - 1) * c * m * np.arange(N), atol=1e-10)
+
+
+@pytest.mark.parametrize("alpha", [1.5, 2.0])
+def test_alibi_hard_cutoff_distance(alpha):
+    # the paper's ALiBi proposition: a key farther than d_max = floor((z_max - z_min + 1/(alpha-1)) / m + 1)
+    # from the query gets exactly zero weight (z: content logits of the row)
+    rng = np.random.default_rng(9)
+    N, d, m, sm = 300, 8, 0.05, 1.0 / np.sqrt(8)
+    q, k, v = (rng.normal(size=(N, d)).astype(np.float32) for _ in range(3))
+    out = oracle.attn_fwd_rows(q, k, v, np.arange(N), alpha, sm, True, want_p=True, alibi=m)
+    z = (q.astype(np.float64) @ k.astype(np.float64).T) * sm
+    checked = 0
+    for i in range(N):
+        zi = z[i, : i + 1]
+        d_max = int(np.floor((zi.max() - zi.min() + 1.0 / (alpha - 1)) / m + 1))
+        far = np.arange(i + 1) < i - d_max
+        checked += int(far.sum())
+        assert np.all(out["p"][i, : i + 1][far] == 0.0)
+    assert checked > 1000       # the bound actually bites on this input
+
+
+def test_alibi_backward_matches_finite_differences():
+    rng = np.random.default_rng(31)
+    N, d, m, sm, alpha = 9, 4, 0.3, 0.5, 1.5
+    q, k, v = _attn_case(rng, N, d)
+    d_o = rng.normal(size=(N, d)).astype(np.float32)
+    scale = (0.8, 0.5, 0.6)
+    rows = np.arange(N)
+
+    def loss(q_, k_, v_, sc=scale):
+        o = oracle.attn_fwd_rows(q_, k_, v_, rows, alpha, sm, True, scale=sc, alibi=m)["o"]
+        return float(np.sum(o * d_o.astype(np.float64)))
+
+    h = 2.0 ** -9
+    for which in range(3):
+        for _ in range(8):
+            i, t = int(rng.integers(N)), int(rng.integers(d))
+            args = [q.copy(), k.copy(), v.copy()]
+            base = np.float32(np.round(args[which][i, t] * 512) / 512)
+            args[which][i, t] = base
+            g0 = oracle.attn_bwd_head(*args, d_o, alpha, sm, True, scale=scale, alibi=m)[which][i, t]
+            up = [a.copy() for a in args]
+            dn = [a.copy() for a in args]
+            up[which][i, t] = base + np.float32(h)
+            dn[which][i, t] = base - np.float32(h)
+            fd = (loss(*up) - loss(*dn)) / (2 * h)
+            assert abs(fd - g0) < 5e-4 * max(1.0, abs(g0)), (which, i, t, fd, g0)
+    # scale parameters: the ASEntmax scale multiplies the whole logit, bias included
+    _, grads = oracle.attn_bwd_scale_head(q, k, v, d_o, alpha, sm, True, scale=scale, alibi=m)
+    for idx in range(3):
+        e = 1e-6
+        up, dn = list(scale), list(scale)
+        up[idx] += e
+        dn[idx] -= e
+        fd = (loss(q, k, v, tuple(up)) - loss(q, k, v, tuple(dn))) / (2 * e)
+        assert abs(fd - grads[idx]) <= 1e-5 * max(1.0, abs(fd)), (idx, fd, grads[idx])
+
+
 def test_threads_reported():
     assert oracle.num_threads() >= 1
