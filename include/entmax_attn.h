@@ -139,6 +139,33 @@ int entmax_attn_bwd_rowscale(const entmax_attn_params* params, const void* q, co
                              float* d_scale_rows, void* workspace, size_t workspace_bytes, int32_t* device_status,
                              void* cuda_stream);
 
+/* Extended forward / backward: every optional input and output of the calls above in one struct, plus the
+ * ALiBi positional term of the paper's NAPE scheme (App. B: half of the heads add m_h (j - i) to the
+ * logits z_ij = <q_i,k_j> sm_scale, j <= i; the other half use slope 0).  The ASEntmax scale multiplies
+ * the whole logit, bias included (Eq. "asentmax" scales the logit vector).
+ *   c_rows        in,  [batch, heads, seq] per-query scales; excludes beta, gamma, delta
+ *   alibi_slopes  in,  [heads] slopes m_h >= 0 (0 = no positional term for that head); float32 problems
+ *                 apply -m_h |i - j| on both sides of the query, bfloat16 problems need causal = 1
+ *                 (ENTMAX_ATTN_EUNSUPPORTED otherwise)
+ *   d_scale_rows, dbeta, dgamma, ddelta   out (backward only), as in entmax_attn_bwd_scale
+ * Any member may be NULL; extras itself may be NULL.  Slopes get no gradient (the paper keeps them fixed). */
+typedef struct {
+  const float* c_rows;
+  const float* alibi_slopes;
+  float* d_scale_rows;
+  float* dbeta;
+  float* dgamma;
+  float* ddelta;
+} entmax_attn_extras;
+int entmax_attn_fwd_ex(const entmax_attn_params* params, const void* q, const void* k, const void* v,
+                       const float* beta, const float* gamma, const float* delta, const entmax_attn_extras* extras,
+                       void* o, float* tau, void* workspace, size_t workspace_bytes, int32_t* device_status,
+                       void* cuda_stream);
+int entmax_attn_bwd_ex(const entmax_attn_params* params, const void* q, const void* k, const void* v,
+                       const float* beta, const float* gamma, const float* delta, const entmax_attn_extras* extras,
+                       const float* tau, const void* d_o, void* dq, void* dk, void* dv, void* workspace,
+                       size_t workspace_bytes, int32_t* device_status, void* cuda_stream);
+
 /* Where a finished forward call leaves the support of every row inside its workspace (App. A: the
  * support of row i is {j : (alpha-1) s_ij > tau_i}).  Byte offsets from the workspace base:
  *   row_count  int32 [batch*heads*seq]: support size of the row, or -2 when the row was computed by the

@@ -33,6 +33,11 @@ class WsLayout(ctypes.Structure):
                 ("scale_offset", ctypes.c_size_t), ("capacity", ctypes.c_int32), ("keep_limit", ctypes.c_int32)]
 
 
+class Extras(ctypes.Structure):
+    _fields_ = [("c_rows", ctypes.c_void_p), ("alibi_slopes", ctypes.c_void_p), ("d_scale_rows", ctypes.c_void_p),
+                ("dbeta", ctypes.c_void_p), ("dgamma", ctypes.c_void_p), ("ddelta", ctypes.c_void_p)]
+
+
 class EntmaxAttnError(RuntimeError):
     pass
 
@@ -62,6 +67,11 @@ def load():
         lib.entmax_attn_bwd_scale.restype = ctypes.c_int
         lib.entmax_attn_bwd_scale.argtypes = [pp, vp, vp, vp, fp, fp, fp, fp, vp, vp, vp, vp, fp, fp, fp, fp, vp,
                                               ctypes.c_size_t, ip, vp]
+        ep = ctypes.POINTER(Extras)
+        lib.entmax_attn_fwd_ex.restype = ctypes.c_int
+        lib.entmax_attn_fwd_ex.argtypes = [pp, vp, vp, vp, fp, fp, fp, ep, vp, fp, vp, ctypes.c_size_t, ip, vp]
+        lib.entmax_attn_bwd_ex.restype = ctypes.c_int
+        lib.entmax_attn_bwd_ex.argtypes = [pp, vp, vp, vp, fp, fp, fp, ep, fp, vp, vp, vp, vp, vp, ctypes.c_size_t, ip, vp]
         lib.entmax_attn_fwd_rowscale.restype = ctypes.c_int
         lib.entmax_attn_fwd_rowscale.argtypes = [pp, vp, vp, vp, fp, vp, fp, vp, ctypes.c_size_t, ip, vp]
         lib.entmax_attn_bwd_rowscale.restype = ctypes.c_int
@@ -257,6 +267,50 @@ def entmax_attn_bwd_rowscale(q, k, v, c_rows, tau, d_o, alpha, causal, *, sm_sca
                                          workspace.numel(), _ptr(status), _stream_ptr(stream))
     _check(rc, "entmax_attn_bwd_rowscale")
     return dq, dk, dv, d_scale_rows
+
+
+def _dp(t):
+    return None if t is None else t.data_ptr()
+
+
+def entmax_attn_fwd_ex(q, k, v, alpha, causal, beta=None, gamma=None, delta=None, *, c_rows=None, alibi_slopes=None,
+                       sm_scale=0.0, n_mode=0, o=None, tau=None, workspace=None, status=None, stream=None):
+    """Extended forward pass: optional per-query scale table and ALiBi slopes.  Returns (o, tau)."""
+    _same_layout(q, k, v)
+    params = make_params(q, alpha, causal, sm_scale, n_mode)
+    B, H, N, _ = q.shape
+    o = torch.empty_like(q) if o is None else o
+    if tau is None:
+        tau = torch.empty((B, H, N), dtype=torch.float32, device=q.device)
+    if workspace is None:
+        workspace = alloc_workspace(params, False, q.device)
+    ex = Extras(_dp(c_rows), _dp(alibi_slopes), None, None, None, None)
+    rc = load().entmax_attn_fwd_ex(ctypes.byref(params), _ptr(q), _ptr(k), _ptr(v), _ptr(beta), _ptr(gamma), _ptr(delta),
+                                   ctypes.byref(ex), _ptr(o), _ptr(tau), _ptr(workspace), workspace.numel(),
+                                   _ptr(status), _stream_ptr(stream))
+    _check(rc, "entmax_attn_fwd_ex")
+    return o, tau
+
+
+def entmax_attn_bwd_ex(q, k, v, tau, d_o, alpha, causal, beta=None, gamma=None, delta=None, *, c_rows=None,
+                       alibi_slopes=None, want_scale_rows=False, want_param_grads=False, sm_scale=0.0, n_mode=0,
+                       workspace=None, status=None, stream=None):
+    """Extended backward pass.  Returns (dq, dk, dv, d_scale_rows or None, (dbeta, dgamma, ddelta) or None)."""
+    _same_layout(q, k, v, d_o)
+    params = make_params(q, alpha, causal, sm_scale, n_mode)
+    B, H, N, _ = q.shape
+    dq, dk, dv = (torch.empty_like(q) for _ in range(3))
+    dc = torch.empty((B, H, N), dtype=torch.float32, device=q.device) if want_scale_rows else None
+    grads = tuple(torch.empty((H,), dtype=torch.float32, device=q.device) for _ in range(3)) if want_param_grads else None
+    g = grads if grads is not None else (None, None, None)
+    if workspace is None:
+        workspace = alloc_workspace(params, True, q.device)
+    ex = Extras(_dp(c_rows), _dp(alibi_slopes), _dp(dc), _dp(g[0]), _dp(g[1]), _dp(g[2]))
+    rc = load().entmax_attn_bwd_ex(ctypes.byref(params), _ptr(q), _ptr(k), _ptr(v), _ptr(beta), _ptr(gamma), _ptr(delta),
+                                   ctypes.byref(ex), _ptr(tau), _ptr(d_o), _ptr(dq), _ptr(dk), _ptr(dv), _ptr(workspace),
+                                   workspace.numel(), _ptr(status), _stream_ptr(stream))
+    _check(rc, "entmax_attn_bwd_ex")
+    return dq, dk, dv, dc, grads
 
 
 def entmax_attn_scores_debug(q, k, bh, causal, *, workspace=None, status=None, stream=None):

@@ -39,6 +39,7 @@ struct Problem {
   int expo_class;
   int64_t sb, sh, sn;  // element strides of the [B,H,N,D] tensors
   int has_scale;
+  const float* alibi;  // device [H] ALiBi slopes m_h (z_ij += -m_h |i - j|), or nullptr
   int64_t scale_sb;    // batch stride of the scale table in floats: 0 for the per-head table [H,N], H*N for
                        // a caller-provided per-query table [B,H,N]
 };

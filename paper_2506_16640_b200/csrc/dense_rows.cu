@@ -99,6 +99,7 @@ __device__ __forceinline__ void atomic_add_slice(float* p, const float (&x)[PER]
 struct RowCtx {
   int grow, bh, b, h, i, nv;
   float c, a, g;
+  float slope;  // ALiBi slope in dot-product units (m_h / sm_scale), 0 without ALiBi
   size_t base;  // element offset of (b, h, 0, 0)
 };
 
@@ -113,6 +114,7 @@ __device__ __forceinline__ RowCtx make_row(const Problem& p, const float* scale,
   r.c = scale[(size_t)r.b * p.scale_sb + (size_t)r.h * p.N + r.i];
   r.g = r.c * p.sm_scale;
   r.a = (p.alpha - 1.0f) * r.g;
+  r.slope = p.alibi ? p.alibi[r.h] / p.sm_scale : 0.f;
   r.base = (size_t)r.b * p.sb + (size_t)r.h * p.sh;
   return r;
 }
@@ -131,6 +133,8 @@ __device__ __forceinline__ float score_pass(const Problem& p, const RowCtx& r, c
 #pragma unroll
     for (int t = 0; t < PER; ++t) dot = fmaf(qs[t], ks[t], dot);
     dot = warp_sum(dot);
+    // ALiBi: the logit is sm_scale * (dot - slope |i - j|) with slope = m_h / sm_scale
+    if (r.slope != 0.f) dot -= r.slope * fabsf((float)(j - r.i));
     float y = r.a * dot;
     if (l == 0) ybuf[j] = y;
     wmax = fmaxf(wmax, y);

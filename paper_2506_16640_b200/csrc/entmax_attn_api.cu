@@ -52,6 +52,7 @@ int make_problem(const entmax_attn_params* params, Problem* out) {
   }
   p.has_scale = 0;
   p.scale_sb = 0;
+  p.alibi = nullptr;
   *out = p;
   return ENTMAX_ATTN_OK;
 }
@@ -146,8 +147,8 @@ namespace {
 // Forward pass; c_rows, when given, is a per-query scale table [B,H,N] that replaces the one the library
 // computes from beta, gamma, delta.
 int fwd_impl(const entmax_attn_params* params, const void* q, const void* k, const void* v, const float* beta,
-             const float* gamma, const float* delta, const float* c_rows, void* o, float* tau, void* workspace,
-             size_t workspace_bytes, int32_t* device_status, void* cuda_stream) {
+             const float* gamma, const float* delta, const float* c_rows, const float* alibi, void* o, float* tau,
+             void* workspace, size_t workspace_bytes, int32_t* device_status, void* cuda_stream) {
   Problem p;
   int rc = make_problem(params, &p);
   if (rc != ENTMAX_ATTN_OK) return rc;
@@ -155,6 +156,10 @@ int fwd_impl(const entmax_attn_params* params, const void* q, const void* k, con
   rc = check_scale_ptrs(beta, gamma, delta, &p);
   if (rc != ENTMAX_ATTN_OK) return rc;
   if (c_rows && (reinterpret_cast<uintptr_t>(c_rows) & 3u)) return ENTMAX_ATTN_EINVAL_ALIGN;
+  if (alibi && (reinterpret_cast<uintptr_t>(alibi) & 3u)) return ENTMAX_ATTN_EINVAL_ALIGN;
+  // the tensor-core kernels apply the ALiBi term on the causal side only
+  if (alibi && p.dtype == ENTMAX_ATTN_DTYPE_BF16 && !p.causal) return ENTMAX_ATTN_EUNSUPPORTED;
+  p.alibi = alibi;
   if (!aligned16(q) || !aligned16(k) || !aligned16(v) || !aligned16(o) || !aligned16(tau)) return ENTMAX_ATTN_EINVAL_ALIGN;
   WsLayout lay;
   rc = check_workspace(p, false, workspace, workspace_bytes, &lay);
@@ -218,7 +223,18 @@ extern "C" {
 int entmax_attn_fwd(const entmax_attn_params* params, const void* q, const void* k, const void* v,
                     const float* beta, const float* gamma, const float* delta, void* o, float* tau,
                     void* workspace, size_t workspace_bytes, int32_t* device_status, void* cuda_stream) {
-  return fwd_impl(params, q, k, v, beta, gamma, delta, nullptr, o, tau, workspace, workspace_bytes, device_status,
+  return fwd_impl(params, q, k, v, beta, gamma, delta, nullptr, nullptr, o, tau, workspace, workspace_bytes,
+                  device_status, cuda_stream);
+}
+
+int entmax_attn_fwd_ex(const entmax_attn_params* params, const void* q, const void* k, const void* v,
+                       const float* beta, const float* gamma, const float* delta, const entmax_attn_extras* extras,
+                       void* o, float* tau, void* workspace, size_t workspace_bytes, int32_t* device_status,
+                       void* cuda_stream) {
+  const float* c_rows = extras ? extras->c_rows : nullptr;
+  const float* alibi = extras ? extras->alibi_slopes : nullptr;
+  if (c_rows && (beta || gamma || delta)) return ENTMAX_ATTN_EINVAL_NULL;   // one source of the scale, not two
+  return fwd_impl(params, q, k, v, beta, gamma, delta, c_rows, alibi, o, tau, workspace, workspace_bytes, device_status,
                   cuda_stream);
 }
 
@@ -226,8 +242,8 @@ int entmax_attn_fwd_rowscale(const entmax_attn_params* params, const void* q, co
                              const float* c_rows, void* o, float* tau, void* workspace, size_t workspace_bytes,
                              int32_t* device_status, void* cuda_stream) {
   if (!c_rows) return ENTMAX_ATTN_EINVAL_NULL;
-  return fwd_impl(params, q, k, v, nullptr, nullptr, nullptr, c_rows, o, tau, workspace, workspace_bytes, device_status,
-                  cuda_stream);
+  return fwd_impl(params, q, k, v, nullptr, nullptr, nullptr, c_rows, nullptr, o, tau, workspace, workspace_bytes,
+                  device_status, cuda_stream);
 }
 
 }  // extern "C"
@@ -235,7 +251,8 @@ int entmax_attn_fwd_rowscale(const entmax_attn_params* params, const void* q, co
 namespace {
 
 int bwd_impl(const entmax_attn_params* params, const void* q, const void* k, const void* v, const float* beta,
-             const float* gamma, const float* delta, const float* c_rows, const float* tau, const void* d_o, void* dq,
+             const float* gamma, const float* delta, const float* c_rows, const float* alibi, const float* tau,
+             const void* d_o, void* dq,
              void* dk, void* dv, float* d_scale_rows, float* dbeta, float* dgamma, float* ddelta, void* workspace,
              size_t workspace_bytes, int32_t* device_status, void* cuda_stream) {
   Problem p;
@@ -247,6 +264,9 @@ int bwd_impl(const entmax_attn_params* params, const void* q, const void* k, con
   const int n_param_grads = (dbeta != nullptr) + (dgamma != nullptr) + (ddelta != nullptr);
   if (n_param_grads != 0 && (n_param_grads != 3 || !p.has_scale || c_rows)) return ENTMAX_ATTN_EINVAL_NULL;
   if (c_rows && (reinterpret_cast<uintptr_t>(c_rows) & 3u)) return ENTMAX_ATTN_EINVAL_ALIGN;
+  if (alibi && (reinterpret_cast<uintptr_t>(alibi) & 3u)) return ENTMAX_ATTN_EINVAL_ALIGN;
+  if (alibi && p.dtype == ENTMAX_ATTN_DTYPE_BF16 && !p.causal) return ENTMAX_ATTN_EUNSUPPORTED;
+  p.alibi = alibi;
   if (!aligned16(q) || !aligned16(k) || !aligned16(v) || !aligned16(tau) || !aligned16(d_o) || !aligned16(dq) ||
       !aligned16(dk) || !aligned16(dv))
     return ENTMAX_ATTN_EINVAL_ALIGN;
@@ -328,8 +348,20 @@ int entmax_attn_bwd_scale(const entmax_attn_params* params, const void* q, const
                           const void* d_o, void* dq, void* dk, void* dv, float* d_scale_rows, float* dbeta,
                           float* dgamma, float* ddelta, void* workspace, size_t workspace_bytes,
                           int32_t* device_status, void* cuda_stream) {
-  return bwd_impl(params, q, k, v, beta, gamma, delta, nullptr, tau, d_o, dq, dk, dv, d_scale_rows, dbeta, dgamma,
-                  ddelta, workspace, workspace_bytes, device_status, cuda_stream);
+  return bwd_impl(params, q, k, v, beta, gamma, delta, nullptr, nullptr, tau, d_o, dq, dk, dv, d_scale_rows, dbeta,
+                  dgamma, ddelta, workspace, workspace_bytes, device_status, cuda_stream);
+}
+
+int entmax_attn_bwd_ex(const entmax_attn_params* params, const void* q, const void* k, const void* v,
+                       const float* beta, const float* gamma, const float* delta, const entmax_attn_extras* extras,
+                       const float* tau, const void* d_o, void* dq, void* dk, void* dv, void* workspace,
+                       size_t workspace_bytes, int32_t* device_status, void* cuda_stream) {
+  entmax_attn_extras ex = {};
+  if (extras) ex = *extras;
+  if (ex.c_rows && (beta || gamma || delta)) return ENTMAX_ATTN_EINVAL_NULL;
+  return bwd_impl(params, q, k, v, beta, gamma, delta, ex.c_rows, ex.alibi_slopes, tau, d_o, dq, dk, dv,
+                  ex.d_scale_rows, ex.dbeta, ex.dgamma, ex.ddelta, workspace, workspace_bytes, device_status,
+                  cuda_stream);
 }
 
 int entmax_attn_bwd_rowscale(const entmax_attn_params* params, const void* q, const void* k, const void* v,
@@ -337,8 +369,8 @@ int entmax_attn_bwd_rowscale(const entmax_attn_params* params, const void* q, co
                              float* d_scale_rows, void* workspace, size_t workspace_bytes, int32_t* device_status,
                              void* cuda_stream) {
   if (!c_rows) return ENTMAX_ATTN_EINVAL_NULL;
-  return bwd_impl(params, q, k, v, nullptr, nullptr, nullptr, c_rows, tau, d_o, dq, dk, dv, d_scale_rows, nullptr,
-                  nullptr, nullptr, workspace, workspace_bytes, device_status, cuda_stream);
+  return bwd_impl(params, q, k, v, nullptr, nullptr, nullptr, c_rows, nullptr, tau, d_o, dq, dk, dv, d_scale_rows,
+                  nullptr, nullptr, nullptr, workspace, workspace_bytes, device_status, cuda_stream);
 }
 
 int entmax_attn_bwd(const entmax_attn_params* params, const void* q, const void* k, const void* v,

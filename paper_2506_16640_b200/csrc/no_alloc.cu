@@ -92,6 +92,7 @@ extern "C" int entmax_attn_fwd_static(const entmax_attn_params* params, const vo
   if (given != 0 && given != 3) return ENTMAX_ATTN_EINVAL_NULL;
   p.has_scale = given == 3;
   p.scale_sb = 0;
+  p.alibi = nullptr;
   auto aligned16 = [](const void* ptr) { return (reinterpret_cast<uintptr_t>(ptr) & 15u) == 0; };
   if (!aligned16(q) || !aligned16(k) || !aligned16(v) || !aligned16(o) || !aligned16(tau)) return ENTMAX_ATTN_EINVAL_ALIGN;
 

@@ -74,13 +74,18 @@ struct SweepArgs {
   int32_t* half_cnt;    // [B*H*N][2] list length of each half-row; -1 = hand the row to the dense path
   float* half_thr;      // [B*H*N][2] lower bound on tau each half-row ended with (Eq. 1's units)
   Entry* entries;       // [B*H*N][kListCap]; half h of a row owns slots [h*kHalfCap, (h+1)*kHalfCap)
-  float* dump;          // optional [N, N] raw accumulators of head dump_bh
+  float* dump;          // kDump kernels: optional [N, N] raw accumulators of head dump_bh; kAlibi kernels: the
+                        // [H] ALiBi slopes m_h (z_ij += m_h (j - i), j <= i).  One member for both keeps the
+                        // argument block, and with it the register allocation of the plain kernel, unchanged
   int dump_bh;
   int32_t* status;
   int32_t* work_counter;  // zeroed before the launch
   int items_per_bh;     // ceil(N / kItemRows)
   int n_items;
 };
+// The kernel's argument block (three tensor maps + this struct) is kept at 512 bytes: one more member made
+// the compiler's register allocation of the hot loop spill five times as much (measured: 2.3 -> 2.9 ms).
+static_assert(sizeof(SweepArgs) + 3 * sizeof(CUtensorMap) <= 512, "keep the sweep kernel's argument block within 512 bytes");
 
 using namespace sm100;
 
@@ -214,7 +219,7 @@ __device__ __noinline__ RowState shrink_lists(RowState r, Entry* list, float a, 
   return r;
 }
 
-template <int HD, bool kDump>
+template <int HD, bool kDump, bool kAlibi>
 __global__ void __launch_bounds__(kThreads, 1) sweep_kernel(const __grid_constant__ CUtensorMap map_q,
                                                             const __grid_constant__ CUtensorMap map_k,
                                                             const __grid_constant__ CUtensorMap map_ks,
@@ -433,6 +438,9 @@ __global__ void __launch_bounds__(kThreads, 1) sweep_kernel(const __grid_constan
           r.cnt = -1;   // non-positive or non-finite scale: dense path
         }
       }
+      // ALiBi (causal): the logit is sm_scale * (acc + slope * (j - i)); everything below works on that sum
+      const float slope = kAlibi ? a.dump[h] / a.sm_scale : 0.f;
+      const float fi = (float)i;
       const bool searching = a.mode == 0 && r.cnt == 0 && valid;
       const bool dump_here = kDump && a.dump != nullptr && bh == a.dump_bh && valid;
       // first / last visible key over the rows of this Q tile: halves past the last one are skipped,
@@ -459,8 +467,13 @@ __global__ void __launch_bounds__(kThreads, 1) sweep_kernel(const __grid_constan
             tmem_ld32(taddr_row + c * 32, va);
             tmem_ld_wait();
 #pragma unroll
-            for (int u = 0; u < 32; ++u) va[u] = (g_base + c * 32 + u <= glim) ? va[u] : -INFINITY;
-            m_s = max3(m_s, fmaxf(max8(&va[0]), max8(&va[8])), fmaxf(max8(&va[16]), max8(&va[24])));
+            for (int u = 0; u < 32; ++u) {
+              if (kAlibi) va[u] = fmaf(slope * (float)kSampleStride, (float)u, va[u]);
+              va[u] = (g_base + c * 32 + u <= glim) ? va[u] : -INFINITY;
+            }
+            float m_c = fmaxf(fmaxf(max8(&va[0]), max8(&va[8])), fmaxf(max8(&va[16]), max8(&va[24])));
+            if (kAlibi) m_c += slope * ((float)(kSampleStride * (g_base + c * 32)) - fi);
+            m_s = fmaxf(m_s, m_c);
           }
           tc_fence_before();
           __syncwarp();
@@ -499,12 +512,22 @@ __global__ void __launch_bounds__(kThreads, 1) sweep_kernel(const __grid_constan
                   if (col_base + c * 32 + u <= lim) a.dump[(size_t)i * a.N + col_base + c * 32 + u] = va[u];
               }
             }
+            if (kAlibi) {
+              // column part of the bias by an FMA with an immediate; the chunk's constant part joins the maxima
+#pragma unroll
+              for (int u = 0; u < 32; ++u) va[u] = fmaf(slope, (float)u, va[u]);
+            }
             if (masked) {
 #pragma unroll
               for (int u = 0; u < 32; ++u) va[u] = (col_base + c * 32 + u <= lim) ? va[u] : -INFINITY;
             }
 #pragma unroll
             for (int q = 0; q < 4; ++q) g[4 * c + q] = max8(&va[8 * q]);
+            if (kAlibi) {
+              const float t0 = slope * ((float)(col_base + c * 32) - fi);
+#pragma unroll
+              for (int q = 0; q < 4; ++q) g[4 * c + q] += t0;
+            }
           }
           float m_tile = max3(g[0], g[1], g[2]);
 #pragma unroll
@@ -544,6 +567,14 @@ __global__ void __launch_bounds__(kThreads, 1) sweep_kernel(const __grid_constan
                 __syncwarp();
                 if (lane == 0) mbar_arrive(my_empty);
                 released = true;
+              }
+              if (kAlibi) {
+#pragma unroll
+                for (int w = 0; w < 4; ++w) {
+                  const float tw = slope * ((float)(col_base + gu[w] * 8) - fi);
+#pragma unroll
+                  for (int e = 0; e < 8; ++e) v8[w][e] = fmaf(slope, (float)e, v8[w][e]) + tw;
+                }
               }
               if (masked) {
 #pragma unroll
@@ -657,7 +688,7 @@ cudaError_t make_sample_map(CUtensorMap* map, const void* base, const Problem& p
   return r == CUDA_SUCCESS ? cudaSuccess : cudaErrorInvalidValue;
 }
 
-template <int HD, bool kDump>
+template <int HD, bool kDump, bool kAlibi>
 cudaError_t launch_impl(const Problem& p, const void* q, const void* k, SweepArgs& args, cudaStream_t stream) {
   CUtensorMap map_q, map_k, map_ks;
   cudaError_t err = make_map(&map_q, q, p, BM);
@@ -670,7 +701,7 @@ cudaError_t launch_impl(const Problem& p, const void* q, const void* k, SweepArg
   } else {
     map_ks = map_k;   // never used: sample_tiles() is 0 for short sequences
   }
-  err = cudaFuncSetAttribute(sweep_kernel<HD, kDump>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+  err = cudaFuncSetAttribute(sweep_kernel<HD, kDump, kAlibi>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                              Cfg<HD>::kSmemBytes);
   if (err != cudaSuccess) return err;
   int dev = 0, sms = 0;
@@ -681,7 +712,7 @@ cudaError_t launch_impl(const Problem& p, const void* q, const void* k, SweepArg
   err = cudaMemsetAsync(args.work_counter, 0, sizeof(int32_t), stream);
   if (err != cudaSuccess) return err;
   const int grid = args.n_items < sms ? args.n_items : sms;
-  sweep_kernel<HD, kDump><<<grid, kThreads, Cfg<HD>::kSmemBytes, stream>>>(map_q, map_k, map_ks, args);
+  sweep_kernel<HD, kDump, kAlibi><<<grid, kThreads, Cfg<HD>::kSmemBytes, stream>>>(map_q, map_k, map_ks, args);
   return cudaGetLastError();
 }
 
@@ -704,14 +735,18 @@ cudaError_t launch_sweep(const Problem& p, const void* q, const void* k, const f
   args.half_cnt = half_cnt;
   args.half_thr = half_thr;
   args.entries = entries;
-  args.dump = dump;
+  args.dump = p.alibi ? const_cast<float*>(p.alibi) : dump;
   args.dump_bh = dump_bh;
   args.status = status;
   args.work_counter = work_counter;
   args.items_per_bh = (p.N + kItemRows - 1) / kItemRows;
   args.n_items = args.items_per_bh * p.B * p.H;
-  if (dump) return p.D == 64 ? launch_impl<64, true>(p, q, k, args, stream) : launch_impl<128, true>(p, q, k, args, stream);
-  return p.D == 64 ? launch_impl<64, false>(p, q, k, args, stream) : launch_impl<128, false>(p, q, k, args, stream);
+  if (dump) return p.D == 64 ? launch_impl<64, true, false>(p, q, k, args, stream)
+                             : launch_impl<128, true, false>(p, q, k, args, stream);
+  if (p.alibi) return p.D == 64 ? launch_impl<64, false, true>(p, q, k, args, stream)
+                                : launch_impl<128, false, true>(p, q, k, args, stream);
+  return p.D == 64 ? launch_impl<64, false, false>(p, q, k, args, stream)
+                   : launch_impl<128, false, false>(p, q, k, args, stream);
 }
 
 }  // namespace entmax

@@ -52,6 +52,7 @@ struct TileArgsK {
   float alpha_m1;
   float sm_scale;
   const float* scale;        // [H, N] (scale_sb = 0) or [B, H, N] (scale_sb = H*N)
+  const float* alibi;        // [H] ALiBi slopes or nullptr (causal problems only)
   long long scale_sb;
   const int32_t* tile_list;  // ids of the Q tiles to process: bh * tiles_per_head + tile
   const int32_t* tile_count;
@@ -307,6 +308,7 @@ __global__ void __launch_bounds__(kThreadsT, 1) tile_fwd_kernel(const __grid_con
       const size_t grow = (size_t)bh * a.N + (valid ? i : 0);
       const int lim = a.causal ? i : a.N - 1;
       const float ra = valid ? a.alpha_m1 * (a.scale[(size_t)b * a.scale_sb + (size_t)h * a.N + i] * a.sm_scale) : 0.f;
+      const float slope = a.alibi ? a.alibi[h] / a.sm_scale : 0.f;   // bias in accumulator units
       float tau = 0.f, ymax = -INFINITY;
       bool done = !valid;
       for (int s = 0; s < kMaxSweeps && alive; ++s) {
@@ -336,6 +338,10 @@ __global__ void __launch_bounds__(kThreadsT, 1) tile_fwd_kernel(const __grid_con
             tmem_ld32(taddr_row + sbuf * TN + c * 32, va);
             tmem_ld_wait();
             const int col0 = t * TN + c * 32;
+            if (slope != 0.f) {
+#pragma unroll
+              for (int u = 0; u < 32; ++u) va[u] = fmaf(slope, (float)(col0 + u - i), va[u]);
+            }
             if (s == 0) {
 #pragma unroll
               for (int u = 0; u < 32; ++u)
@@ -530,6 +536,7 @@ cudaError_t launch_tile_fwd(const Problem& p, const void* q, const void* k, cons
   args.alpha_m1 = p.alpha - 1.0f;
   args.sm_scale = p.sm_scale;
   args.scale = scale;
+  args.alibi = p.alibi;
   args.scale_sb = p.scale_sb;
   args.tile_list = tile_list;
   args.tile_count = tile_count;

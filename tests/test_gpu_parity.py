@@ -227,6 +227,67 @@ def test_rowscale_with_a_batch_dependent_table_matches_the_oracle(dtype, alpha):
                 parity.grad_close("dc row", np.array([float(dc[b, h, i])]), np.array([dc_ref[i]]))
 
 
+# ------------------------------------------------------------------ ALiBi term (the paper's NAPE: half the heads)
+def _check_alibi(inp, alpha, causal, slopes, dense_expected):
+    w = inp.workload
+    dev = parity.to_device(inp)
+    sl = torch.tensor(slopes, dtype=torch.float32, device="cuda")
+    status = torch.zeros(binding.STATUS_WORDS, dtype=torch.int32, device="cuda")
+    o, tau = binding.entmax_attn_fwd_ex(dev["q"], dev["k"], dev["v"], alpha, causal, dev["beta"], dev["gamma"],
+                                        dev["delta"], alibi_slopes=sl, status=status)
+    dq, dk, dv, dc, grads = binding.entmax_attn_bwd_ex(dev["q"], dev["k"], dev["v"], tau, dev["d_o"], alpha, causal,
+                                                       dev["beta"], dev["gamma"], dev["delta"], alibi_slopes=sl,
+                                                       want_scale_rows=True, want_param_grads=inp.beta is not None)
+    torch.cuda.synchronize()
+    assert int(status[binding.STATUS_FLAGS]) == 0
+    if dense_expected is not None:
+        assert (int(status[binding.STATUS_DENSE_ROWS]) > 0) == dense_expected
+    N = w.N
+    rows = np.arange(N)
+    for h in range(w.H):
+        q, k, v, g = (t[0, h].float().numpy() for t in (inp.q, inp.k, inp.v, inp.d_o))
+        sc = inp.head_scale(h)
+        f = oracle_mod.attn_fwd_rows(q, k, v, rows, alpha, inp.sm_scale, causal, scale=sc, alibi=slopes[h])
+        tau_err = np.abs(tau[0, h].cpu().double().numpy() - f["tau"]) / np.maximum(1.0, np.abs(f["tau"]))
+        assert tau_err.max() <= parity.tau_tol(w.dtype), tau_err.max()
+        assert np.abs(o[0, h].float().cpu().numpy() - f["o"]).max() <= parity.O_TOL
+        rq, rk, rv = oracle_mod.attn_bwd_head(q, k, v, g, alpha, inp.sm_scale, causal, scale=sc, alibi=slopes[h])
+        parity.grad_close("dQ", dq[0, h].float().cpu().numpy(), rq)
+        parity.grad_close("dK", dk[0, h].float().cpu().numpy(), rk)
+        parity.grad_close("dV", dv[0, h].float().cpu().numpy(), rv)
+        dc_ref, gr = oracle_mod.attn_bwd_scale_head(q, k, v, g, alpha, inp.sm_scale, causal, scale=sc, alibi=slopes[h])
+        parity.grad_close("dc rows", dc[0, h].cpu().numpy(), dc_ref)
+        for idx in range(3 if grads is not None else 0):
+            assert abs(float(grads[idx][h]) - gr[idx]) <= 2e-2 * max(1.0, abs(gr[idx])), (idx, float(grads[idx][h]), gr[idx])
+
+
+@pytest.mark.parametrize("alpha", [1.25, 1.5, 2.0])
+@pytest.mark.parametrize("N,d", [(700, 64), (4500, 128)])
+def test_alibi_bf16_causal_sparse_rows(N, d, alpha):
+    # head 0 without positional term, head 1 with a slope (NAPE); N = 4500 also runs the sampled pre-pass
+    inp = make_inputs(_small("alibi", N, d, True, plant=2, backward=True, seed=N + 7))
+    _check_alibi(inp, alpha, True, [0.0, 0.05], None)
+
+
+def test_alibi_bf16_causal_dense_rows():
+    inp = make_inputs(_small("alibi_dense", 600, 128, True, backward=True, use_scale=False, sigma=0.05, seed=19))
+    _check_alibi(inp, 1.5, True, [0.002, 0.0005], True)
+
+
+@pytest.mark.parametrize("causal", [True, False])
+def test_alibi_fp32_both_masks(causal):
+    inp = make_inputs(_small("alibi32", 150, 64, causal, dtype="fp32", backward=True, seed=23))
+    _check_alibi(inp, 1.5, causal, [0.1, 0.02], None)
+
+
+def test_alibi_bf16_noncausal_is_rejected():
+    inp = make_inputs(_small("alibi_nc", 128, 64, False, seed=29))
+    dev = parity.to_device(inp)
+    sl = torch.tensor([0.1, 0.1], dtype=torch.float32, device="cuda")
+    with pytest.raises(binding.EntmaxAttnError, match="sm_100|unsupported|needs"):
+        binding.entmax_attn_fwd_ex(dev["q"], dev["k"], dev["v"], 1.5, False, alibi_slopes=sl)
+
+
 # ------------------------------------------------------------------ the benchmark workloads
 def test_cfg2_all_rows():
     inp = make_inputs(WORKLOADS[2])
