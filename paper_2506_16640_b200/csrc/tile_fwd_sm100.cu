@@ -342,19 +342,67 @@ __global__ void __launch_bounds__(kThreadsT, 1) tile_fwd_kernel(const __grid_con
 #pragma unroll
               for (int u = 0; u < 32; ++u) va[u] = fmaf(slope, (float)(col0 + u - i), va[u]);
             }
+            // columns past the row's last visible key only occur in the tiles at the causal diagonal / the tail
+            if (col0 + 31 > lim) {
+#pragma unroll
+              for (int u = 0; u < 32; ++u) va[u] = (col0 + u <= lim) ? va[u] : -INFINITY;
+            }
             if (s == 0) {
+              // y_max: with ra > 0 the largest accumulator, otherwise (negative scale) the smallest
+              float m = va[0];
+              if (ra >= 0.f) {
 #pragma unroll
-              for (int u = 0; u < 32; ++u)
-                if (col0 + u <= lim) ymax = fmaxf(ymax, ra * va[u]);
+                for (int u = 1; u < 32; ++u) m = fmaxf(m, va[u]);
+                if (m > -INFINITY) ymax = fmaxf(ymax, ra * m);
+              } else {
+#pragma unroll
+                for (int u = 0; u < 32; ++u)
+                  if (col0 + u <= lim) ymax = fmaxf(ymax, ra * va[u]);
+              }
             } else if (!output) {
+              // masked columns hold -inf: y = ra * acc - tau is -inf (ra > 0) and clamps to 0; a negative
+              // scale is rare enough for the general loop
+              // four independent partial sums each: one thread owns the row, so the additions would
+              // otherwise form two serial chains of 128 dependent operations per tile
+              float p0[4] = {0.f, 0.f, 0.f, 0.f}, p1[4] = {0.f, 0.f, 0.f, 0.f};
+              if (a.expo_class == kExpo2 && ra > 0.f) {
 #pragma unroll
-              for (int u = 0; u < 32; ++u) {
-                const float y = fmaf(ra, va[u], -tau);
-                if (y > 0.f && col0 + u <= lim) {
-                  float ye, ye1;
-                  pow_pair(y, a.expo_class, a.expo, ye, ye1);
-                  s0 += ye;
-                  s1 += ye1;
+                for (int u = 0; u < 32; ++u) {
+                  const float y = fmaxf(fmaf(ra, va[u], -tau), 0.f);
+                  p0[u & 3] = fmaf(y, y, p0[u & 3]);
+                  p1[u & 3] += y;
+                }
+                s0 += (p0[0] + p0[1]) + (p0[2] + p0[3]);
+                s1 += (p1[0] + p1[1]) + (p1[2] + p1[3]);
+              } else if (a.expo_class == kExpo1 && ra > 0.f) {
+#pragma unroll
+                for (int u = 0; u < 32; ++u) {
+                  const float y = fmaf(ra, va[u], -tau);
+                  p0[u & 3] += fmaxf(y, 0.f);
+                  p1[u & 3] += y > 0.f ? 1.0f : 0.f;
+                }
+                s0 += (p0[0] + p0[1]) + (p0[2] + p0[3]);
+                s1 += (p1[0] + p1[1]) + (p1[2] + p1[3]);
+              } else if (a.expo_class == kExpo4 && ra > 0.f) {
+#pragma unroll
+                for (int u = 0; u < 32; ++u) {
+                  const float y = fmaxf(fmaf(ra, va[u], -tau), 0.f);
+                  const float y2 = y * y;
+                  p0[u & 3] = fmaf(y2, y2, p0[u & 3]);
+                  p1[u & 3] = fmaf(y2, y, p1[u & 3]);
+                }
+                s0 += (p0[0] + p0[1]) + (p0[2] + p0[3]);
+                s1 += (p1[0] + p1[1]) + (p1[2] + p1[3]);
+              } else {
+#pragma unroll
+                for (int u = 0; u < 32; ++u) {
+                  const float y = fmaf(ra, va[u], -tau);
+                  if (y > 0.f && col0 + u <= lim) {
+                    float ye, ye1;
+                    pow_pair(y, a.expo_class, a.expo, ye, ye1);
+                    s0 += ye;
+                    s1 += ye1;
+                  }
                 }
               }
             } else {
