@@ -148,6 +148,7 @@ int entmax_attn_bwd_rowscale(const entmax_attn_params* params, const void* q, co
  *                 apply -m_h |i - j| on both sides of the query, bfloat16 problems need causal = 1
  *                 (ENTMAX_ATTN_EUNSUPPORTED otherwise)
  *   d_scale_rows, dbeta, dgamma, ddelta   out (backward only), as in entmax_attn_bwd_scale
+ *   fwd_workspace saved state of the forward call, see the member below
  * Any member may be NULL; extras itself may be NULL.  Slopes get no gradient (the paper keeps them fixed). */
 typedef struct {
   const float* c_rows;
@@ -156,6 +157,10 @@ typedef struct {
   float* dbeta;
   float* dgamma;
   float* ddelta;
+  const void* fwd_workspace; /* backward only, bfloat16 problems: the workspace of the forward call on the same
+                                inputs, untouched since it returned.  It still holds the support of every row, so
+                                the backward pass skips its own score sweep (which otherwise recomputes Q K^T to
+                                find the support from tau).  Must not be the buffer passed as `workspace`.        */
 } entmax_attn_extras;
 int entmax_attn_fwd_ex(const entmax_attn_params* params, const void* q, const void* k, const void* v,
                        const float* beta, const float* gamma, const float* delta, const entmax_attn_extras* extras,

@@ -35,7 +35,8 @@ class WsLayout(ctypes.Structure):
 
 class Extras(ctypes.Structure):
     _fields_ = [("c_rows", ctypes.c_void_p), ("alibi_slopes", ctypes.c_void_p), ("d_scale_rows", ctypes.c_void_p),
-                ("dbeta", ctypes.c_void_p), ("dgamma", ctypes.c_void_p), ("ddelta", ctypes.c_void_p)]
+                ("dbeta", ctypes.c_void_p), ("dgamma", ctypes.c_void_p), ("ddelta", ctypes.c_void_p),
+                ("fwd_workspace", ctypes.c_void_p)]
 
 
 class EntmaxAttnError(RuntimeError):
@@ -284,7 +285,7 @@ def entmax_attn_fwd_ex(q, k, v, alpha, causal, beta=None, gamma=None, delta=None
         tau = torch.empty((B, H, N), dtype=torch.float32, device=q.device)
     if workspace is None:
         workspace = alloc_workspace(params, False, q.device)
-    ex = Extras(_dp(c_rows), _dp(alibi_slopes), None, None, None, None)
+    ex = Extras(_dp(c_rows), _dp(alibi_slopes), None, None, None, None, None)
     rc = load().entmax_attn_fwd_ex(ctypes.byref(params), _ptr(q), _ptr(k), _ptr(v), _ptr(beta), _ptr(gamma), _ptr(delta),
                                    ctypes.byref(ex), _ptr(o), _ptr(tau), _ptr(workspace), workspace.numel(),
                                    _ptr(status), _stream_ptr(stream))
@@ -293,19 +294,23 @@ def entmax_attn_fwd_ex(q, k, v, alpha, causal, beta=None, gamma=None, delta=None
 
 
 def entmax_attn_bwd_ex(q, k, v, tau, d_o, alpha, causal, beta=None, gamma=None, delta=None, *, c_rows=None,
-                       alibi_slopes=None, want_scale_rows=False, want_param_grads=False, sm_scale=0.0, n_mode=0,
-                       workspace=None, status=None, stream=None):
-    """Extended backward pass.  Returns (dq, dk, dv, d_scale_rows or None, (dbeta, dgamma, ddelta) or None)."""
+                       alibi_slopes=None, fwd_workspace=None, want_scale_rows=False, want_param_grads=False,
+                       sm_scale=0.0, n_mode=0, dq=None, dk=None, dv=None, workspace=None, status=None, stream=None):
+    """Extended backward pass.  `fwd_workspace`: the forward call's workspace tensor, untouched since
+    (the backward pass then reuses the supports it holds instead of sweeping Q K^T again).
+    Returns (dq, dk, dv, d_scale_rows or None, (dbeta, dgamma, ddelta) or None)."""
     _same_layout(q, k, v, d_o)
     params = make_params(q, alpha, causal, sm_scale, n_mode)
     B, H, N, _ = q.shape
-    dq, dk, dv = (torch.empty_like(q) for _ in range(3))
+    dq = torch.empty_like(q) if dq is None else dq
+    dk = torch.empty_like(q) if dk is None else dk
+    dv = torch.empty_like(q) if dv is None else dv
     dc = torch.empty((B, H, N), dtype=torch.float32, device=q.device) if want_scale_rows else None
     grads = tuple(torch.empty((H,), dtype=torch.float32, device=q.device) for _ in range(3)) if want_param_grads else None
     g = grads if grads is not None else (None, None, None)
     if workspace is None:
         workspace = alloc_workspace(params, True, q.device)
-    ex = Extras(_dp(c_rows), _dp(alibi_slopes), _dp(dc), _dp(g[0]), _dp(g[1]), _dp(g[2]))
+    ex = Extras(_dp(c_rows), _dp(alibi_slopes), _dp(dc), _dp(g[0]), _dp(g[1]), _dp(g[2]), _dp(fwd_workspace))
     rc = load().entmax_attn_bwd_ex(ctypes.byref(params), _ptr(q), _ptr(k), _ptr(v), _ptr(beta), _ptr(gamma), _ptr(delta),
                                    ctypes.byref(ex), _ptr(tau), _ptr(d_o), _ptr(dq), _ptr(dk), _ptr(dv), _ptr(workspace),
                                    workspace.numel(), _ptr(status), _stream_ptr(stream))

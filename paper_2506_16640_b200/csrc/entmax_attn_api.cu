@@ -251,8 +251,8 @@ int entmax_attn_fwd_rowscale(const entmax_attn_params* params, const void* q, co
 namespace {
 
 int bwd_impl(const entmax_attn_params* params, const void* q, const void* k, const void* v, const float* beta,
-             const float* gamma, const float* delta, const float* c_rows, const float* alibi, const float* tau,
-             const void* d_o, void* dq,
+             const float* gamma, const float* delta, const float* c_rows, const float* alibi,
+             const void* fwd_workspace, const float* tau, const void* d_o, void* dq,
              void* dk, void* dv, float* d_scale_rows, float* dbeta, float* dgamma, float* ddelta, void* workspace,
              size_t workspace_bytes, int32_t* device_status, void* cuda_stream) {
   Problem p;
@@ -316,14 +316,24 @@ int bwd_impl(const entmax_attn_params* params, const void* q, const void* k, con
   } else {
     err = cudaMemsetAsync(fb_count, 0, sizeof(int32_t), stream);
     if (err != cudaSuccess) return fail_cuda(err);
-    if (g_prof_start[1]) cudaEventRecord(g_prof_start[1], stream);
-    err = launch_sweep(p, q, k, scale, tau, 1, half_cnt, half_thr, entries, sweep_counter, nullptr, -1, device_status,
-                       stream);
-    if (err != cudaSuccess) return fail_cuda(err);
-    if (g_prof_stop[1]) cudaEventRecord(g_prof_stop[1], stream);
-    err = launch_row_bwd(p, q, k, v, d_o, scale, tau, half_cnt, entries, dq, acc_dk, acc_dv, dc_rows, fb_count, fb_list,
-                         device_status, stream);
-    if (err != cudaSuccess) return fail_cuda(err);
+    if (fwd_workspace) {
+      // the forward call's workspace still holds every row's support: no score sweep needed
+      const WsLayout fl = make_layout(p, false);
+      const uint8_t* fws = static_cast<const uint8_t*>(fwd_workspace);
+      err = launch_row_bwd(p, q, k, v, d_o, scale, tau, reinterpret_cast<const int32_t*>(fws + fl.row_cnt),
+                           const_cast<Entry*>(reinterpret_cast<const Entry*>(fws + fl.entries)), dq, acc_dk, acc_dv,
+                           dc_rows, fb_count, fb_list, device_status, 1, stream);
+      if (err != cudaSuccess) return fail_cuda(err);
+    } else {
+      if (g_prof_start[1]) cudaEventRecord(g_prof_start[1], stream);
+      err = launch_sweep(p, q, k, scale, tau, 1, half_cnt, half_thr, entries, sweep_counter, nullptr, -1, device_status,
+                         stream);
+      if (err != cudaSuccess) return fail_cuda(err);
+      if (g_prof_stop[1]) cudaEventRecord(g_prof_stop[1], stream);
+      err = launch_row_bwd(p, q, k, v, d_o, scale, tau, half_cnt, entries, dq, acc_dk, acc_dv, dc_rows, fb_count,
+                           fb_list, device_status, 0, stream);
+      if (err != cudaSuccess) return fail_cuda(err);
+    }
     err = launch_dense_bwd(p, q, k, v, d_o, scale, tau, dq, acc_dk, acc_dv, dc_rows, fb_list, fb_count, scratch,
                            lay.scratch_floats, lay.scratch_ctas, stream);
     if (err != cudaSuccess) return fail_cuda(err);
@@ -348,7 +358,7 @@ int entmax_attn_bwd_scale(const entmax_attn_params* params, const void* q, const
                           const void* d_o, void* dq, void* dk, void* dv, float* d_scale_rows, float* dbeta,
                           float* dgamma, float* ddelta, void* workspace, size_t workspace_bytes,
                           int32_t* device_status, void* cuda_stream) {
-  return bwd_impl(params, q, k, v, beta, gamma, delta, nullptr, nullptr, tau, d_o, dq, dk, dv, d_scale_rows, dbeta,
+  return bwd_impl(params, q, k, v, beta, gamma, delta, nullptr, nullptr, nullptr, tau, d_o, dq, dk, dv, d_scale_rows, dbeta,
                   dgamma, ddelta, workspace, workspace_bytes, device_status, cuda_stream);
 }
 
@@ -359,7 +369,8 @@ int entmax_attn_bwd_ex(const entmax_attn_params* params, const void* q, const vo
   entmax_attn_extras ex = {};
   if (extras) ex = *extras;
   if (ex.c_rows && (beta || gamma || delta)) return ENTMAX_ATTN_EINVAL_NULL;
-  return bwd_impl(params, q, k, v, beta, gamma, delta, ex.c_rows, ex.alibi_slopes, tau, d_o, dq, dk, dv,
+  if (ex.fwd_workspace && (reinterpret_cast<uintptr_t>(ex.fwd_workspace) & 255u)) return ENTMAX_ATTN_EINVAL_WORKSPACE;
+  return bwd_impl(params, q, k, v, beta, gamma, delta, ex.c_rows, ex.alibi_slopes, ex.fwd_workspace, tau, d_o, dq, dk, dv,
                   ex.d_scale_rows, ex.dbeta, ex.dgamma, ex.ddelta, workspace, workspace_bytes, device_status,
                   cuda_stream);
 }
@@ -369,7 +380,7 @@ int entmax_attn_bwd_rowscale(const entmax_attn_params* params, const void* q, co
                              float* d_scale_rows, void* workspace, size_t workspace_bytes, int32_t* device_status,
                              void* cuda_stream) {
   if (!c_rows) return ENTMAX_ATTN_EINVAL_NULL;
-  return bwd_impl(params, q, k, v, nullptr, nullptr, nullptr, c_rows, nullptr, tau, d_o, dq, dk, dv, d_scale_rows,
+  return bwd_impl(params, q, k, v, nullptr, nullptr, nullptr, c_rows, nullptr, nullptr, tau, d_o, dq, dk, dv, d_scale_rows,
                   nullptr, nullptr, nullptr, workspace, workspace_bytes, device_status, cuda_stream);
 }
 

@@ -491,7 +491,7 @@ __device__ __forceinline__ void bwd_row_full(const Problem& p, const __nv_bfloat
                                              const float* __restrict__ tau_in, const Entry* __restrict__ entries,
                                              __nv_bfloat16* __restrict__ dq, float* __restrict__ acc_dk,
                                              float* __restrict__ acc_dv, float* __restrict__ dc_rows, int grow, int c0,
-                                             int c1, int lane) {
+                                             int c1, bool saved, int lane) {
   constexpr int PER = D / 32;
   const int bh = grow / p.N, i = grow - bh * p.N, b = bh / p.H, h = bh - b * p.H;
   const float g = scale[(size_t)b * p.scale_sb + (size_t)h * p.N + i] * p.sm_scale;
@@ -513,9 +513,10 @@ __device__ __forceinline__ void bwd_row_full(const Problem& p, const __nv_bfloat
     zz[s] = 0.f;
     if (e < c0 + c1) {
       const Entry en = list[e < c0 ? e : kHalfCap + e - c0];
-      yv[s] = fmaf(a, en.y, -tau);
+      // a list saved by the forward pass holds y = (alpha-1) s in Eq. 1's units, a fresh one raw <q_i, k_j>
+      yv[s] = saved ? en.y - tau : fmaf(a, en.y, -tau);
       jj[s] = en.j;
-      zz[s] = en.y;                                  // raw <q_i, k_j>
+      zz[s] = saved ? en.y / a : en.y;               // raw <q_i, k_j>
     }
   }
   // dP_ij = <dO_i, v_j> on the support
@@ -593,7 +594,7 @@ __device__ __forceinline__ void bwd_rows_quad(const Problem& p, const __nv_bfloa
                                               const float* __restrict__ tau_in, const Entry* __restrict__ entries,
                                               __nv_bfloat16* __restrict__ dq, float* __restrict__ acc_dk,
                                               float* __restrict__ acc_dv, float* __restrict__ dc_rows, int grow,
-                                              bool active, int c0, int c1, int lane) {
+                                              bool active, int c0, int c1, bool saved, int lane) {
   constexpr int PL = D / 8;                        // elements of a row per lane
   const int sl = lane & 7;
   const int base = lane & 24;
@@ -611,9 +612,9 @@ __device__ __forceinline__ void bwd_rows_quad(const Problem& p, const __nv_bfloa
   int j = 0;
   if (sl < n) {
     const Entry en = list[sl < c0 ? sl : kHalfCap + sl - c0];
-    yv = fmaf(a, en.y, -tau);
+    yv = saved ? en.y - tau : fmaf(a, en.y, -tau);
     j = en.j;
-    zz = en.y;                                     // raw <q_i, k_j>
+    zz = saved ? en.y / a : en.y;                  // raw <q_i, k_j>
   }
   const bool in = yv > 0.f;
   const unsigned msub = (__ballot_sync(0xffffffffu, in) >> base) & 0xffu;
@@ -678,7 +679,9 @@ __global__ void __launch_bounds__(kWarpsPerCta * 32, 4) row_bwd_kernel(
     const __nv_bfloat16* __restrict__ v, const __nv_bfloat16* __restrict__ d_o, const float* __restrict__ scale,
     const float* __restrict__ tau_in, const int32_t* __restrict__ half_cnt, const Entry* __restrict__ entries,
     __nv_bfloat16* __restrict__ dq, float* __restrict__ acc_dk, float* __restrict__ acc_dv,
-    float* __restrict__ dc_rows, int32_t* fb_count, int32_t* fb_list, int32_t* status) {
+    float* __restrict__ dc_rows, int32_t* fb_count, int32_t* fb_list, int32_t* status, int saved) {
+  // saved != 0: `half_cnt` is the forward pass's final support size per row (one int per row, -2 = dense
+  // row) and `entries` its compacted support lists
   const int lane = threadIdx.x & 31;
   const int total = p.B * p.H * p.N;
   const int groups = (total + 3) / 4;
@@ -688,14 +691,18 @@ __global__ void __launch_bounds__(kWarpsPerCta * 32, 4) row_bwd_kernel(
     const bool my_active = my_row < total;
     int mc0 = 0, mc1 = 0;
     if (my_active) {
-      const int2 c = *reinterpret_cast<const int2*>(half_cnt + 2 * (size_t)my_row);
-      mc0 = c.x;
-      mc1 = c.y;
+      if (saved) {
+        mc0 = half_cnt[my_row];
+      } else {
+        const int2 c = *reinterpret_cast<const int2*>(half_cnt + 2 * (size_t)my_row);
+        mc0 = c.x;
+        mc1 = c.y;
+      }
     }
     const bool small = !my_active || (mc0 >= 0 && mc1 >= 0 && mc0 + mc1 <= 8);
     if (__all_sync(0xffffffffu, small)) {
       bwd_rows_quad<D>(p, q, k, v, d_o, scale, tau_in, entries, dq, acc_dk, acc_dv, dc_rows, my_active ? my_row : 0,
-                       my_active, mc0, mc1, lane);
+                       my_active, mc0, mc1, saved != 0, lane);
       continue;
     }
     for (int r = 0; r < 4; ++r) {
@@ -706,7 +713,7 @@ __global__ void __launch_bounds__(kWarpsPerCta * 32, 4) row_bwd_kernel(
         if (lane == 0) push_dense_row(grow, fb_count, fb_list, status);
         continue;
       }
-      bwd_row_full<D>(p, q, k, v, d_o, scale, tau_in, entries, dq, acc_dk, acc_dv, dc_rows, grow, c0, c1, lane);
+      bwd_row_full<D>(p, q, k, v, d_o, scale, tau_in, entries, dq, acc_dk, acc_dv, dc_rows, grow, c0, c1, saved != 0, lane);
     }
   }
 }
@@ -739,16 +746,16 @@ cudaError_t launch_row_fwd(const Problem& p, const void* v, const float* scale, 
 cudaError_t launch_row_bwd(const Problem& p, const void* q, const void* k, const void* v, const void* d_o,
                            const float* scale, const float* tau, const int32_t* half_cnt, Entry* entries, void* dq,
                            float* acc_dk, float* acc_dv, float* dc_rows, int32_t* fb_count, int32_t* fb_list,
-                           int32_t* status, cudaStream_t stream) {
+                           int32_t* status, int saved, cudaStream_t stream) {
   const int grid = row_grid(p);
   if (p.D == 64)
     row_bwd_kernel<64><<<grid, kWarpsPerCta * 32, 0, stream>>>(
         p, (const __nv_bfloat16*)q, (const __nv_bfloat16*)k, (const __nv_bfloat16*)v, (const __nv_bfloat16*)d_o, scale,
-        tau, half_cnt, entries, (__nv_bfloat16*)dq, acc_dk, acc_dv, dc_rows, fb_count, fb_list, status);
+        tau, half_cnt, entries, (__nv_bfloat16*)dq, acc_dk, acc_dv, dc_rows, fb_count, fb_list, status, saved);
   else
     row_bwd_kernel<128><<<grid, kWarpsPerCta * 32, 0, stream>>>(
         p, (const __nv_bfloat16*)q, (const __nv_bfloat16*)k, (const __nv_bfloat16*)v, (const __nv_bfloat16*)d_o, scale,
-        tau, half_cnt, entries, (__nv_bfloat16*)dq, acc_dk, acc_dv, dc_rows, fb_count, fb_list, status);
+        tau, half_cnt, entries, (__nv_bfloat16*)dq, acc_dk, acc_dv, dc_rows, fb_count, fb_list, status, saved);
   return cudaGetLastError();
 }
 

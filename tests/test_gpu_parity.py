@@ -288,6 +288,30 @@ def test_alibi_bf16_noncausal_is_rejected():
         binding.entmax_attn_fwd_ex(dev["q"], dev["k"], dev["v"], 1.5, False, alibi_slopes=sl)
 
 
+# ------------------------------------------------------------------ backward from the forward call's saved supports
+@pytest.mark.parametrize("alpha", [1.25, 1.5, 2.0])
+@pytest.mark.parametrize("N,d,sigma,plant", [(1300, 64, 1.0, 3), (700, 128, 1.0, 0), (400, 128, 0.05, 0)])
+def test_backward_with_saved_forward_workspace(N, d, sigma, plant, alpha):
+    # sigma 0.05: every row dense (row_count -2 in the saved workspace -> dense backward path)
+    inp = make_inputs(_small("saved", N, d, True, plant=plant, backward=True, sigma=sigma, seed=N + 3))
+    got = parity.run_fwd(inp, alpha)
+    dev = got["dev"]
+    ref = binding.entmax_attn_bwd_scale(dev["q"], dev["k"], dev["v"], got["tau"], dev["d_o"], alpha, True, dev["beta"],
+                                        dev["gamma"], dev["delta"])
+    dq, dk, dv, dc, grads = binding.entmax_attn_bwd_ex(dev["q"], dev["k"], dev["v"], got["tau"], dev["d_o"], alpha, True,
+                                                       dev["beta"], dev["gamma"], dev["delta"],
+                                                       fwd_workspace=got["workspace"], want_scale_rows=True,
+                                                       want_param_grads=True)
+    torch.cuda.synchronize()
+    for name, a_, b_ in (("dq", dq, ref[0]), ("dk", dk, ref[1]), ("dv", dv, ref[2]), ("dc", dc, ref[3])):
+        parity.grad_close(name, a_.float().cpu().numpy(), b_.float().cpu().numpy())
+    for idx in range(3):
+        parity.grad_close("param grad", grads[idx].cpu().numpy(), ref[4][idx].cpu().numpy())
+    # and against the oracle directly
+    bwd = {"dq": dq, "dk": dk, "dv": dv}
+    parity.check_bwd_head(inp, alpha, bwd, 1)
+
+
 # ------------------------------------------------------------------ the benchmark workloads
 def test_cfg2_all_rows():
     inp = make_inputs(WORKLOADS[2])
