@@ -60,6 +60,18 @@ __device__ __forceinline__ void pow_pair(float y, int expo_class, float expo, fl
   else { ye1 = powf(y, expo - 1.0f); ye = ye1 * y; }
 }
 
+// One threshold step from the left of the root, given S = sum [y - tau]_+^e (> 1) and S1 = sum [y - tau]_+^(e-1).
+// It is Newton on F(tau) = S^(1/e) - 1 rather than on S - 1: the e-norm of an affine function of tau is convex and
+// decreasing just like S (so steps from the left never pass the root, Eq. 1's threshold), but nearly linear in tau
+// -- exactly linear while the support does not change and the values are equal -- where S is a polynomial of
+// degree e.  -F / F' = (S - S^(1-1/e)) / S1.  For e = 1 (sparsemax) it is the plain Newton step (S - 1) / S1.
+__device__ __forceinline__ float threshold_step(float s0, float s1, int expo_class, float expo) {
+  const float root = expo_class == kExpo1 ? s0
+                     : expo_class == kExpo2 ? sqrtf(s0)
+                     : expo_class == kExpo4 ? sqrtf(sqrtf(s0)) : powf(s0, 1.0f / expo);
+  return (s0 - s0 / root) / s1;
+}
+
 // ---- launchers (each enqueues on `stream` and returns the cudaError_t of the launch) -------------
 cudaError_t launch_scale_table(const Problem& p, const float* beta, const float* gamma, const float* delta,
                                float* scale, int32_t* status, cudaStream_t stream);

@@ -157,7 +157,7 @@ __device__ __forceinline__ float newton_tau(const Problem& p, const float* ybuf,
     }
     float2 s = block_sum2(s0, s1, red);
     if (!(s.x > 1.0f) || !(s.y > 0.f)) break;
-    float step = (s.x - 1.0f) / (p.expo * s.y);
+    float step = threshold_step(s.x, s.y, p.expo_class, p.expo);
     float next = tau + step;
     if (!(next > tau)) break;
     tau = next;

@@ -187,7 +187,7 @@ __device__ __forceinline__ float newton_warp(const Problem& p, const float (&y)[
     s0 = warp_sum(s0);
     s1 = warp_sum(s1);
     if (!(s0 > 1.0f) || !(s1 > 0.f)) break;
-    const float step = (s0 - 1.0f) / (p.expo * s1);
+    const float step = threshold_step(s0, s1, p.expo_class, p.expo);
     const float next = tau + step;
     if (!(next > tau)) break;
     tau = next;
@@ -324,7 +324,7 @@ __device__ __forceinline__ float newton_oct(const Problem& p, float y, float tau
       if (!(s0 > 1.0f) || !(s1 > 0.f)) {
         done = true;
       } else {
-        const float step = (s0 - 1.0f) / (p.expo * s1);
+        const float step = threshold_step(s0, s1, p.expo_class, p.expo);
         const float next = tau + step;
         if (!(next > tau)) {
           done = true;

@@ -190,7 +190,7 @@ __device__ __noinline__ RowState shrink_lists(RowState r, Entry* list, float a, 
         s0 = warp_sum(s0);
         s1 = warp_sum(s1);
         if (!(s0 > 1.0f) || !(s1 > 0.f)) break;
-        const float step = (s0 - 1.0f) / (expo * s1);
+        const float step = threshold_step(s0, s1, expo_class, expo);
         tau += step;
         if (step <= 1e-4f) break;
       }

@@ -489,15 +489,7 @@ __global__ void __launch_bounds__(kThreadsT, 1) tile_fwd_kernel(const __grid_con
           if (!(s0 > 1.0f) || !(s1 > 0.f)) {
             done = true;
           } else {
-            // Newton on F(tau) = (sum [y - tau]_+^e)^(1/e) - 1 instead of f = sum - 1: the e-norm of an affine
-            // function of tau is convex and decreasing like f, so steps from the left still never pass the
-            // root, but it is nearly linear in tau (exactly linear while the support does not change and
-            // the values are equal), where f is a polynomial of degree e: a row with thousands of keys in
-            // its support needs a handful of sweeps instead of 20-30.  -F / F' = (S - S^(1-1/e)) / S1, S = s0
-            const float root = a.expo_class == kExpo1 ? s0
-                               : a.expo_class == kExpo2 ? sqrtf(s0)
-                               : a.expo_class == kExpo4 ? sqrtf(sqrtf(s0)) : powf(s0, 1.0f / a.expo);
-            const float step = (s0 - s0 / root) / s1;
+            const float step = threshold_step(s0, s1, a.expo_class, a.expo);   // e-norm step, see common.cuh
             const float next = tau + step;
             if (!(next > tau)) done = true;
             tau = next > tau ? next : tau;
