@@ -123,7 +123,7 @@ __global__ void __launch_bounds__(kThreadsT, 1) tile_fwd_kernel(const __grid_con
   const uint32_t s_empty = s_full + 16;                               // [2]
   const uint32_t p_full = s_empty + 16, p_empty = p_full + 8;
   const uint32_t o_full = p_empty + 8, o_empty = o_full + 8;
-  const uint32_t ctl = o_empty + 8;                                   // consumers' verdict on a sweep is in
+  const uint32_t ctl = o_empty + 8;                                   // the consumers' vote on a sweep is in
   const uint32_t done_word = ctl + 8;                                 // uint32 [3]
   const uint32_t tmem_slot = done_word + 12;
   const uint32_t abort_flag = tmem_slot + 4;
@@ -318,7 +318,7 @@ __global__ void __launch_bounds__(kThreadsT, 1) tile_fwd_kernel(const __grid_con
           if (!alive) break;
         }
         const bool output = sweep_is_output(s);
-        // the verdict slot two sweeps ahead is free again: nobody reads it before the next vote
+        // the vote slot two sweeps ahead is free again: nobody reads it before the next vote
         if (warp == 2 && lane == 0) sts_u32(done_word + 4 * ((s + 1) % 3), 1u);
         float s0 = 0.f, s1 = 0.f;
         for (int t = 0; t < tiles && alive; ++t) {
@@ -482,7 +482,7 @@ __global__ void __launch_bounds__(kThreadsT, 1) tile_fwd_kernel(const __grid_con
           if (lane == 0) mbar_arrive(o_empty);
           break;
         }
-        // ---- between sweeps: Newton update and the verdict "every row of the tile has converged"
+        // ---- between sweeps: Newton update and the vote "every row of the tile has converged"
         if (s == 0) {
           tau = ymax - 1.0f;
         } else if (!done) {
