@@ -17,7 +17,7 @@ LIB_PATH = os.path.join(_HERE, "libentmax_attn.so")
 
 DTYPE_BF16, DTYPE_FP32 = 0, 1
 STATUS_WORDS = 4
-STATUS_FLAGS, STATUS_DENSE_ROWS = 0, 1
+STATUS_FLAGS, STATUS_DENSE_ROWS, STATUS_TILE_SWEEPS, STATUS_TILES = 0, 1, 2, 3
 FLAG_WAIT_EXPIRED, FLAG_BAD_SCALE = 1, 2
 
 

@@ -45,7 +45,7 @@ struct Problem {
 };
 
 struct WsLayout {
-  size_t scale, row_cnt, half_cnt, half_thr, entries, fb_count, sweep_counter, tile_count, fb_list, tile_flag, tile_list, scratch, acc_dk, acc_dv, dc_rows, total;
+  size_t scale, row_cnt, half_cnt, half_thr, entries, fb_count, sweep_counter, tile_count, fb_list, tile_flag, tile_list, tile_mask, scratch, acc_dk, acc_dv, dc_rows, total;
   int scratch_ctas;     // CTAs of the dense-row kernels (each owns scratch_floats floats)
   size_t scratch_floats;
 };
@@ -100,6 +100,14 @@ cudaError_t launch_sweep(const Problem& p, const void* q, const void* k, const f
 cudaError_t launch_tile_fwd(const Problem& p, const void* q, const void* k, const void* v, const float* scale,
                             const int32_t* tile_list, const int32_t* tile_count, const int32_t* row_cnt, void* o,
                             float* tau, int32_t* status, cudaStream_t stream);
+
+// Dense-tile backward on the tensor cores (bf16): the rows in row_list[0 .. *row_count) are marked in
+// tile_mask, their 128-row Q tiles listed, and dQ (and dc_rows) of those rows written; their dK and dV
+// contributions are added to the fp32 accumulators.  tile_mask, tile_flag and *tile_count must be zero on entry.
+cudaError_t launch_tile_bwd(const Problem& p, const void* q, const void* k, const void* v, const void* d_o,
+                            const float* scale, const float* tau, const int32_t* row_list, const int32_t* row_count,
+                            uint32_t* tile_mask, int32_t* tile_flag, int32_t* tile_list, int32_t* tile_count, void* dq,
+                            float* acc_dk, float* acc_dv, float* dc_rows, int32_t* status, cudaStream_t stream);
 
 // per-row solve + gather kernels working on the lists (bf16 path); the forward one also lists the
 // 128-row Q tiles that hold rows for the dense-tile path (tile_flag must be zero on entry)

@@ -98,6 +98,7 @@ WsLayout make_layout(const Problem& p, bool is_bwd) {
   const size_t q_tiles = (size_t)p.B * p.H * ((p.N + 127) / 128);
   l.tile_flag = take(q_tiles * sizeof(int32_t));
   l.tile_list = take(q_tiles * sizeof(int32_t));
+  l.tile_mask = take(q_tiles * 4 * sizeof(uint32_t));   // 128 row bits per Q tile (dense-tile backward)
   // dense-row CTAs: enough to fill the machine, few enough that their score rows stay modest
   l.scratch_floats = align_up((size_t)p.N, 32) * (is_bwd ? 2 : 1);   // scores (+ dP in backward)
   size_t ctas = 148 * 4;
@@ -314,7 +315,15 @@ int bwd_impl(const entmax_attn_params* params, const void* q, const void* k, con
                            lay.scratch_floats, lay.scratch_ctas, stream);
     if (err != cudaSuccess) return fail_cuda(err);
   } else {
-    err = cudaMemsetAsync(fb_count, 0, sizeof(int32_t), stream);
+    int32_t* tile_flag = reinterpret_cast<int32_t*>(ws + lay.tile_flag);
+    int32_t* tile_list = reinterpret_cast<int32_t*>(ws + lay.tile_list);
+    int32_t* tile_count = reinterpret_cast<int32_t*>(ws + lay.tile_count);
+    uint32_t* tile_mask = reinterpret_cast<uint32_t*>(ws + lay.tile_mask);
+    const size_t q_tiles = (size_t)p.B * p.H * ((p.N + 127) / 128);
+    err = cudaMemsetAsync(fb_count, 0, 256, stream);   // the whole counter block
+    if (err != cudaSuccess) return fail_cuda(err);
+    // tile flags, tile list and tile masks are adjacent in the workspace: one memset clears all three
+    err = cudaMemsetAsync(tile_flag, 0, lay.tile_mask + q_tiles * 4 * sizeof(uint32_t) - lay.tile_flag, stream);
     if (err != cudaSuccess) return fail_cuda(err);
     if (fwd_workspace) {
       // the forward call's workspace still holds every row's support: no score sweep needed
@@ -334,8 +343,9 @@ int bwd_impl(const entmax_attn_params* params, const void* q, const void* k, con
                            fb_list, device_status, 0, stream);
       if (err != cudaSuccess) return fail_cuda(err);
     }
-    err = launch_dense_bwd(p, q, k, v, d_o, scale, tau, dq, acc_dk, acc_dv, dc_rows, fb_list, fb_count, scratch,
-                           lay.scratch_floats, lay.scratch_ctas, stream);
+    // rows whose support does not fit the lists: dense tiles on the tensor cores
+    err = launch_tile_bwd(p, q, k, v, d_o, scale, tau, fb_list, fb_count, tile_mask, tile_flag, tile_list, tile_count, dq,
+                          acc_dk, acc_dv, dc_rows, device_status, stream);
     if (err != cudaSuccess) return fail_cuda(err);
   }
   err = launch_store_grad(p, acc_dk, dk, stream);

@@ -1,0 +1,534 @@
+// Dense-tile backward for bf16 problems on sm_100a: the rows whose support does not fit the sparse
+// lists are differentiated tile by tile on the tensor cores.  With y_ij = (alpha-1) c_i z_ij - tau_i,
+// p_ij = [y_ij]_+^e (Eq. 1) and u_ij = [y_ij]_+^(e-1) = p_ij^(2-alpha), the entmax Jacobian gives
+//   dP_ij = dO_i . v_j,   rho_i = sum_j u_ij dP_ij / sum_j u_ij,   dS_ij = u_ij (dP_ij - rho_i),
+//   dQ_i = g_i sum_j dS_ij k_j,   dK_j = sum_i g_i dS_ij q_i,   dV_j = sum_i p_ij dO_i,
+//   dL/dc_i = sum_j dS_ij z_ij                      (g_i = c_i * sm_scale, c_i the ASEntmax scale)
+// A work item is one Q tile of 128 rows that holds at least one such row.  Two passes over its visible
+// K/V tiles, five tcgen05 contractions:
+//   pass A   S = Q K^T and dP = dO V^T into TMEM; the row threads accumulate sum u and sum u dP;
+//   pass B   S and dP again; the row threads write P and g dS (bf16) to shared memory; then
+//            dQ += (g dS) K     (A = g dS K-major, B = K tile with the head dim contiguous)   kept in TMEM,
+//            dK_t = (g dS)^T Q  (A = the same shared tile read M-major, B = Q tile, head dim contiguous)
+//            dV_t = P^T dO      (likewise), both through one TMEM buffer, added to the fp32 dK / dV
+//            accumulators in global memory (vector reductions) by the thread that owns the key.
+// Rows of the tile that are not marked contribute zeros (their P and dS rows are written as zero) and
+// their dQ is not stored: the list kernels have already handled them.
+//
+// CTA: warp 0 TMA producer, warp 1 MMA issuer, warps 2..5 one thread per TMEM lane.  Every wait is
+// bounded (see sm100_ptx.cuh); on expiry the CTA flags the call's status word and leaves.
+#include <cuda.h>
+
+#include "common.cuh"
+#include "sm100_ptx.cuh"
+
+namespace entmax {
+
+namespace {
+
+using namespace sm100;
+
+constexpr int TM = 128;            // query rows per item = TMEM lanes
+constexpr int TN = 128;            // keys per K/V tile
+constexpr int kThreadsB = 6 * 32;
+constexpr int kTileBytes = TM * TN * 2;   // P or dS tile, bf16
+
+template <int HD>
+struct BCfg {
+  static constexpr int kHalves = HD / 64;
+  static constexpr int kQBytes = TM * HD * 2;       // Q tile; also dO, K, V tiles
+  static constexpr int kBarBytes = 256;
+  static constexpr int kSmemBytes = 4 * kQBytes + 2 * kTileBytes + 1024 + kBarBytes;
+  static constexpr int kTmemS = 0, kTmemDP = TN, kTmemDQ = 2 * TN, kTmemT = 2 * TN + 128;
+};
+
+struct TileBwdArgs {
+  int B, H, N;
+  int causal;
+  int expo_class;
+  float expo;
+  float alpha_m1;
+  float sm_scale;
+  const float* scale;        // [H, N] (scale_sb = 0) or [B, H, N] (scale_sb = H*N)
+  const float* alibi;        // [H] ALiBi slopes or nullptr (causal problems only)
+  long long scale_sb;
+  const int32_t* tile_list;  // ids of the Q tiles to process: bh * tiles_per_head + tile
+  const int32_t* tile_count;
+  const uint32_t* tile_mask; // [tiles, 4]: bit r of a tile's 128-bit mask marks row r for this kernel
+  const float* tau;
+  void* dq;                  // bf16 [B,H,N,D]
+  float* acc_dk;             // fp32 [B,H,N,D] contiguous
+  float* acc_dv;
+  float* dc_rows;            // [B,H,N] or nullptr
+  int64_t sb, sh, sn;
+  int32_t* status;
+  int tiles_per_head;
+};
+
+// A, B bf16 K-major, fp32 accumulate, M = 128, N = TN (S = Q K^T and dP = dO V^T)
+__host__ __device__ constexpr uint32_t idesc_kk() {
+  return (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(TN >> 3) << 17) | ((uint32_t)(TM >> 4) << 24);
+}
+// A K-major, B with N contiguous (bit 16), N = HD (dQ += dS K)
+template <int HD>
+__host__ __device__ constexpr uint32_t idesc_kn() {
+  return (1u << 4) | (1u << 7) | (1u << 10) | (1u << 16) | ((uint32_t)(HD >> 3) << 17) | ((uint32_t)(TM >> 4) << 24);
+}
+// A with M contiguous (bit 15), B with N contiguous (bit 16), N = HD (dK = dS^T Q, dV = P^T dO)
+template <int HD>
+__host__ __device__ constexpr uint32_t idesc_mn() {
+  return (1u << 4) | (1u << 7) | (1u << 10) | (1u << 15) | (1u << 16) | ((uint32_t)(HD >> 3) << 17) |
+         ((uint32_t)(TM >> 4) << 24);
+}
+// Low descriptor word of a [128 x 64-element-blocks] tile read with its 128-byte rows as the M (or N)
+// direction, 128-byte swizzle: a swizzle atom is one 128-byte row of 64 elements by 8 rows; atoms repeat
+// every 1024 bytes along the rows (stride-dimension offset, in the high word) and every 128*128 bytes from
+// one 64-element block to the next (leading-dimension offset).  Sixteen rows (one MMA K step) are 2048 bytes.
+__device__ __forceinline__ uint32_t mn_desc_lo(uint32_t saddr) {
+  return ((saddr & 0x3FFFFu) >> 4) | ((uint32_t)((128 * 128) >> 4) << 16);
+}
+
+__device__ __forceinline__ uint32_t pack_bf16(float a, float b) {
+  const __nv_bfloat162 hh = __floats2bfloat162_rn(a, b);
+  return *reinterpret_cast<const uint32_t*>(&hh);
+}
+
+// fire-and-forget vector add to global memory (no value returned)
+__device__ __forceinline__ void red_add_v4(float* dst, float x, float y, float z, float w) {
+  asm volatile("red.global.add.v4.f32 [%0], {%1, %2, %3, %4};" ::"l"(dst), "f"(x), "f"(y), "f"(z), "f"(w) : "memory");
+}
+
+// Marks the rows of row_list[0 .. *row_count) in the per-tile masks and lists every tile once.
+__global__ void mark_tiles_kernel(int N, int tiles_per_head, const int32_t* __restrict__ row_list,
+                                  const int32_t* __restrict__ row_count, uint32_t* __restrict__ tile_mask,
+                                  int32_t* __restrict__ tile_flag, int32_t* __restrict__ tile_list,
+                                  int32_t* __restrict__ tile_count) {
+  const int total = *row_count;
+  for (int t = blockIdx.x * blockDim.x + threadIdx.x; t < total; t += gridDim.x * blockDim.x) {
+    const int grow = row_list[t];
+    const int bh = grow / N, i = grow - bh * N;
+    const int id = bh * tiles_per_head + i / TM;
+    const int r = i % TM;
+    atomicOr(tile_mask + 4 * (size_t)id + (r >> 5), 1u << (r & 31));
+    if (atomicExch(tile_flag + id, 1) == 0) tile_list[atomicAdd(tile_count, 1)] = id;
+  }
+}
+
+template <int HD>
+__global__ void __launch_bounds__(kThreadsB, 1) tile_bwd_kernel(const __grid_constant__ CUtensorMap map_q,
+                                                               const __grid_constant__ CUtensorMap map_k,
+                                                               const __grid_constant__ CUtensorMap map_v,
+                                                               const __grid_constant__ CUtensorMap map_do,
+                                                               const TileBwdArgs a) {
+  using C = BCfg<HD>;
+  extern __shared__ uint8_t smem_raw[];
+  const uint32_t sbase = (smem_u32(smem_raw) + 1023u) & ~1023u;
+  const uint32_t q_smem = sbase;
+  const uint32_t do_smem = q_smem + C::kQBytes;
+  const uint32_t k_smem = do_smem + C::kQBytes;
+  const uint32_t v_smem = k_smem + C::kQBytes;
+  const uint32_t p_smem = v_smem + C::kQBytes;           // P tile, [128 rows][128 keys] bf16, swizzled
+  const uint32_t ds_smem = p_smem + kTileBytes;           // g dS tile, same layout
+  const uint32_t bars = ds_smem + kTileBytes;
+  const uint32_t qdo_full = bars, qdo_empty = bars + 8;
+  const uint32_t kv_full = bars + 16, kv_empty = bars + 24;
+  const uint32_t sd_full = bars + 32, sd_empty = bars + 40;
+  const uint32_t pds_full = bars + 48, pds_empty = bars + 56;
+  const uint32_t t_full = bars + 64, t_empty = bars + 72;
+  const uint32_t dq_full = bars + 80, dq_empty = bars + 88;
+  const uint32_t tmem_slot = bars + 96;
+  const uint32_t abort_flag = bars + 100;
+
+  const int warp = threadIdx.x >> 5;
+  const int lane = threadIdx.x & 31;
+  const int n_tiles = *a.tile_count;
+
+  if (threadIdx.x == 0) {
+    mbar_init(qdo_full, 1);
+    mbar_init(qdo_empty, 1);
+    mbar_init(kv_full, 1);
+    mbar_init(kv_empty, 1);
+    mbar_init(sd_full, 1);
+    mbar_init(sd_empty, 4);
+    mbar_init(pds_full, 4);
+    mbar_init(pds_empty, 1);
+    mbar_init(t_full, 1);
+    mbar_init(t_empty, 4);
+    mbar_init(dq_full, 1);
+    mbar_init(dq_empty, 4);
+    sts_u32(abort_flag, 0u);
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+  }
+  if (warp == 1) {
+    tmem_alloc(tmem_slot, 512);
+    tmem_relinquish();
+  }
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem_base = lds_u32(tmem_slot);
+
+  auto item_tiles = [&](int tile) -> int {
+    const int row0 = tile * TM;
+    if (!a.causal) return (a.N + TN - 1) / TN;
+    int last_row = row0 + TM - 1;
+    if (last_row > a.N - 1) last_row = a.N - 1;
+    return last_row / TN + 1;
+  };
+
+  if (warp == 0) {
+    // ------------------------------------------------------------------ TMA producer
+    if (lane == 0) {
+      uint32_t kvphase = 0, qphase = 0;
+      bool alive = true;
+      for (int it = blockIdx.x; it < n_tiles && alive; it += gridDim.x) {
+        const int id = a.tile_list[it];
+        const int bh = id / a.tiles_per_head, tile = id - bh * a.tiles_per_head;
+        const int b = bh / a.H, h = bh - b * a.H;
+        const int tiles = item_tiles(tile);
+        alive = mbar_wait(qdo_empty, qphase ^ 1u, abort_flag);
+        if (!alive) break;
+        qphase ^= 1u;
+        mbar_expect_tx(qdo_full, 2 * C::kQBytes);
+        for (int hf = 0; hf < C::kHalves; ++hf) {
+          tma_load_4d(q_smem + hf * (TM * 128), &map_q, qdo_full, hf * 64, tile * TM, h, b);
+          tma_load_4d(do_smem + hf * (TM * 128), &map_do, qdo_full, hf * 64, tile * TM, h, b);
+        }
+        for (int t = 0; t < 2 * tiles && alive; ++t) {
+          const int kt = t < tiles ? t : t - tiles;
+          alive = mbar_wait(kv_empty, kvphase ^ 1u, abort_flag);
+          if (!alive) break;
+          kvphase ^= 1u;
+          mbar_expect_tx(kv_full, 2 * C::kQBytes);
+          for (int hf = 0; hf < C::kHalves; ++hf) {
+            tma_load_4d(k_smem + hf * (TN * 128), &map_k, kv_full, hf * 64, kt * TN, h, b);
+            tma_load_4d(v_smem + hf * (TN * 128), &map_v, kv_full, hf * 64, kt * TN, h, b);
+          }
+        }
+      }
+    }
+  } else if (warp == 1) {
+    // ------------------------------------------------------------------ MMA issuer
+    if (lane == 0) {
+      constexpr uint32_t id_kk = idesc_kk();
+      constexpr uint32_t id_kn = idesc_kn<HD>();
+      constexpr uint32_t id_mn = idesc_mn<HD>();
+      const uint32_t q_lo = smem_desc_lo(q_smem), do_lo = smem_desc_lo(do_smem);
+      const uint32_t k_lo = smem_desc_lo(k_smem), v_lo = smem_desc_lo(v_smem);
+      const uint32_t ds_lo = smem_desc_lo(ds_smem);
+      const uint32_t k_n_lo = mn_desc_lo(k_smem), q_n_lo = mn_desc_lo(q_smem), do_n_lo = mn_desc_lo(do_smem);
+      const uint32_t ds_m_lo = mn_desc_lo(ds_smem), p_m_lo = mn_desc_lo(p_smem);
+      uint32_t kvphase = 0, qphase = 0, sdphase = 0, pdsphase = 0, tphase = 0, dqphase = 0;
+      bool alive = true;
+      for (int it = blockIdx.x; it < n_tiles && alive; it += gridDim.x) {
+        const int id = a.tile_list[it];
+        const int tile = id % a.tiles_per_head;
+        const int tiles = item_tiles(tile);
+        alive = mbar_wait(qdo_full, qphase, abort_flag);
+        qphase ^= 1u;
+        if (!alive) break;
+        for (int t = 0; t < 2 * tiles && alive; ++t) {
+          const bool pass_b = t >= tiles;
+          if (t == tiles) {
+            // the previous item's dQ must have been read before this item's first dQ MMA overwrites it
+            alive = mbar_wait(dq_empty, dqphase ^ 1u, abort_flag);
+            dqphase ^= 1u;
+            if (!alive) break;
+          }
+          alive = mbar_wait(kv_full, kvphase, abort_flag);
+          kvphase ^= 1u;
+          if (alive) alive = mbar_wait(sd_empty, sdphase ^ 1u, abort_flag);
+          if (!alive) break;
+          sdphase ^= 1u;
+          tc_fence_after();
+#pragma unroll
+          for (int kk = 0; kk < HD / 16; ++kk) {
+            const uint32_t off = (kk >> 2) * ((TM * 128) >> 4) + (kk & 3) * 2;
+            umma_bf16(tmem_base + C::kTmemS, q_lo + off, k_lo + off, kDescHi, id_kk, kk > 0 ? 1u : 0u);
+          }
+#pragma unroll
+          for (int kk = 0; kk < HD / 16; ++kk) {
+            const uint32_t off = (kk >> 2) * ((TM * 128) >> 4) + (kk & 3) * 2;
+            umma_bf16(tmem_base + C::kTmemDP, do_lo + off, v_lo + off, kDescHi, id_kk, kk > 0 ? 1u : 0u);
+          }
+          umma_commit(sd_full);
+          if (!pass_b) {
+            umma_commit(kv_empty);
+            continue;
+          }
+          // P and g dS of this tile are in shared memory
+          alive = mbar_wait(pds_full, pdsphase, abort_flag);
+          pdsphase ^= 1u;
+          if (!alive) break;
+          tc_fence_after();
+#pragma unroll
+          for (int kk = 0; kk < TN / 16; ++kk) {
+            const uint32_t a_off = (kk >> 2) * ((TM * 128) >> 4) + (kk & 3) * 2;   // 64 keys per 128-byte row
+            const uint32_t b_off = kk * ((16 * 128) >> 4);                           // 16 keys = 16 rows of 128 B
+            umma_bf16_ab(tmem_base + C::kTmemDQ, ds_lo + a_off, kDescHi, k_n_lo + b_off, kDescHi, id_kn,
+                         (t > tiles || kk > 0) ? 1u : 0u);
+          }
+          alive = mbar_wait(t_empty, tphase ^ 1u, abort_flag);
+          tphase ^= 1u;
+          if (!alive) break;
+          tc_fence_after();
+#pragma unroll
+          for (int kk = 0; kk < TM / 16; ++kk) {
+            const uint32_t off = kk * ((16 * 128) >> 4);                             // 16 query rows
+            umma_bf16_ab(tmem_base + C::kTmemT, ds_m_lo + off, kDescHi, q_n_lo + off, kDescHi, id_mn, kk > 0 ? 1u : 0u);
+          }
+          umma_commit(t_full);
+          alive = mbar_wait(t_empty, tphase ^ 1u, abort_flag);
+          tphase ^= 1u;
+          if (!alive) break;
+          tc_fence_after();
+#pragma unroll
+          for (int kk = 0; kk < TM / 16; ++kk) {
+            const uint32_t off = kk * ((16 * 128) >> 4);
+            umma_bf16_ab(tmem_base + C::kTmemT, p_m_lo + off, kDescHi, do_n_lo + off, kDescHi, id_mn, kk > 0 ? 1u : 0u);
+          }
+          umma_commit(t_full);
+          umma_commit(pds_empty);
+          umma_commit(kv_empty);
+          if (t == 2 * tiles - 1) umma_commit(dq_full);
+        }
+        umma_commit(qdo_empty);
+      }
+    }
+  } else {
+    // ------------------------------------------------------------------ one thread per TMEM lane
+    const int quad = warp & 3;
+    const int row_local = quad * 32 + lane;
+    const uint32_t taddr_row = tmem_base + ((uint32_t)(quad * 32) << 16);
+    uint32_t sdphase = 0, pdsphase = 0, tphase = 0, dqphase = 0;
+    bool alive = true;
+    for (int it = blockIdx.x; it < n_tiles && alive; it += gridDim.x) {
+      const int id = a.tile_list[it];
+      const int bh = id / a.tiles_per_head, tile = id - bh * a.tiles_per_head;
+      const int b = bh / a.H, h = bh - b * a.H;
+      const int tiles = item_tiles(tile);
+      const int i = tile * TM + row_local;
+      const bool valid = i < a.N;
+      const bool marked = valid && ((a.tile_mask[4 * (size_t)id + (row_local >> 5)] >> (row_local & 31)) & 1u);
+      const size_t grow = (size_t)bh * a.N + (valid ? i : 0);
+      const int lim = a.causal ? i : a.N - 1;
+      const float c_i = valid ? a.scale[(size_t)b * a.scale_sb + (size_t)h * a.N + i] : 0.f;
+      const float ra = a.alpha_m1 * (c_i * a.sm_scale);
+      const float g = c_i * a.sm_scale;
+      const float slope = a.alibi ? a.alibi[h] / a.sm_scale : 0.f;   // bias in accumulator units
+      const float tau = marked ? a.tau[grow] : 0.f;
+      float su = 0.f, sud = 0.f, rho = 0.f, dcp = 0.f;
+      for (int t = 0; t < 2 * tiles && alive; ++t) {
+        const bool pass_b = t >= tiles;
+        const int kt = pass_b ? t - tiles : t;
+        if (t == tiles) rho = su > 0.f ? sud / su : 0.f;
+        alive = __all_sync(0xffffffffu, mbar_wait(sd_full, sdphase, abort_flag));
+        if (!alive) break;
+        sdphase ^= 1u;
+        tc_fence_after();
+        if (pass_b) {
+          // P and dS of the previous tile must have been consumed before their buffers are rewritten
+          alive = __all_sync(0xffffffffu, mbar_wait(pds_empty, pdsphase ^ 1u, abort_flag));
+          pdsphase ^= 1u;
+          if (!alive) break;
+        }
+#pragma unroll
+        for (int c = 0; c < TN / 32; ++c) {
+          float sa[32], dp[32];
+          tmem_ld32(taddr_row + C::kTmemS + c * 32, sa);
+          tmem_ld32(taddr_row + C::kTmemDP + c * 32, dp);
+          tmem_ld_wait();
+          const int col0 = kt * TN + c * 32;
+          if (slope != 0.f) {
+#pragma unroll
+            for (int u = 0; u < 32; ++u) sa[u] = fmaf(slope, (float)(col0 + u - i), sa[u]);
+          }
+          const bool edge = col0 + 31 > lim;
+          if (!pass_b) {
+#pragma unroll
+            for (int u = 0; u < 32; ++u) {
+              const float y = fmaf(ra, sa[u], -tau);
+              if (y > 0.f && (!edge || col0 + u <= lim)) {
+                float ye, ye1;
+                pow_pair(y, a.expo_class, a.expo, ye, ye1);
+                su += ye1;
+                sud = fmaf(ye1, dp[u], sud);
+              }
+            }
+          } else {
+            // P and g dS -> bf16 -> shared memory, K-major with 128-byte swizzle: row r, 16-byte unit u of
+            // the 64-key block sits at r*128 + ((u ^ (r & 7)) * 16)
+            const uint32_t blk = (uint32_t)(c >> 1) * (TM * 128) + (uint32_t)row_local * 128u;
+#pragma unroll
+            for (int u4 = 0; u4 < 4; ++u4) {
+              float pv[8], dv[8];
+#pragma unroll
+              for (int z = 0; z < 8; ++z) {
+                const int u = u4 * 8 + z;
+                const float y = fmaf(ra, sa[u], -tau);
+                pv[z] = 0.f;
+                dv[z] = 0.f;
+                if (marked && y > 0.f && (!edge || col0 + u <= lim)) {
+                  float ye, ye1;
+                  pow_pair(y, a.expo_class, a.expo, ye, ye1);
+                  const float ds = ye1 * (dp[u] - rho);
+                  pv[z] = ye;
+                  dv[z] = g * ds;
+                  dcp = fmaf(ds, sa[u], dcp);
+                }
+              }
+              const uint32_t unit = (uint32_t)((c & 1) * 4 + u4);
+              const uint32_t off = blk + ((unit ^ (uint32_t)(row_local & 7)) << 4);
+              asm volatile("st.shared::cta.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(p_smem + off),
+                           "r"(pack_bf16(pv[0], pv[1])), "r"(pack_bf16(pv[2], pv[3])), "r"(pack_bf16(pv[4], pv[5])),
+                           "r"(pack_bf16(pv[6], pv[7]))
+                           : "memory");
+              asm volatile("st.shared::cta.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(ds_smem + off),
+                           "r"(pack_bf16(dv[0], dv[1])), "r"(pack_bf16(dv[2], dv[3])), "r"(pack_bf16(dv[4], dv[5])),
+                           "r"(pack_bf16(dv[6], dv[7]))
+                           : "memory");
+            }
+          }
+        }
+        // S and dP have been read
+        tc_fence_before();
+        __syncwarp();
+        if (lane == 0) mbar_arrive(sd_empty);
+        if (!pass_b) continue;
+        // make the P / dS stores visible to the tensor core (async proxy), then hand the tiles over
+        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+        __syncwarp();
+        if (lane == 0) mbar_arrive(pds_full);
+        // dK then dV of this K tile: TMEM lane = key
+        const int key = kt * TN + row_local;
+#pragma unroll 1
+        for (int which = 0; which < 2 && alive; ++which) {
+          alive = __all_sync(0xffffffffu, mbar_wait(t_full, tphase, abort_flag));
+          if (!alive) break;
+          tphase ^= 1u;
+          tc_fence_after();
+          float* dst = (which == 0 ? a.acc_dk : a.acc_dv) + ((size_t)bh * a.N + (key < a.N ? key : 0)) * HD;
+#pragma unroll
+          for (int c = 0; c < HD / 32; ++c) {
+            float va[32];
+            tmem_ld32(taddr_row + C::kTmemT + c * 32, va);
+            tmem_ld_wait();
+            if (key < a.N) {
+#pragma unroll
+              for (int m = 0; m < 8; ++m)
+                red_add_v4(dst + c * 32 + 4 * m, va[4 * m], va[4 * m + 1], va[4 * m + 2], va[4 * m + 3]);
+            }
+          }
+          tc_fence_before();
+          __syncwarp();
+          if (lane == 0) mbar_arrive(t_empty);
+        }
+      }
+      if (!alive) break;
+      // ---- dQ of the item
+      alive = __all_sync(0xffffffffu, mbar_wait(dq_full, dqphase, abort_flag));
+      dqphase ^= 1u;
+      if (!alive) break;
+      tc_fence_after();
+      __nv_bfloat16* dqrow =
+          reinterpret_cast<__nv_bfloat16*>(a.dq) + (size_t)b * a.sb + (size_t)h * a.sh + (size_t)i * a.sn;
+#pragma unroll
+      for (int c = 0; c < HD / 32; ++c) {
+        float va[32];
+        tmem_ld32(taddr_row + C::kTmemDQ + c * 32, va);
+        tmem_ld_wait();
+        if (marked) {
+#pragma unroll
+          for (int u8 = 0; u8 < 4; ++u8)
+            *reinterpret_cast<uint4*>(dqrow + c * 32 + u8 * 8) =
+                make_uint4(pack_bf16(va[u8 * 8], va[u8 * 8 + 1]), pack_bf16(va[u8 * 8 + 2], va[u8 * 8 + 3]),
+                           pack_bf16(va[u8 * 8 + 4], va[u8 * 8 + 5]), pack_bf16(va[u8 * 8 + 6], va[u8 * 8 + 7]));
+        }
+      }
+      // dL/dc_i = sum_j dS_ij z_ij with z_ij = sm_scale * (accumulator + bias in accumulator units)
+      if (marked && a.dc_rows) a.dc_rows[grow] = dcp * a.sm_scale;
+      if (a.status && threadIdx.x == 64) atomicAdd(a.status + ENTMAX_ATTN_STATUS_TILES, 1);
+      tc_fence_before();
+      __syncwarp();
+      if (lane == 0) mbar_arrive(dq_empty);
+    }
+  }
+
+  // ---------------------------------------------------------------------- teardown
+  tc_fence_before();
+  __syncthreads();
+  if (lds_u32(abort_flag)) {
+    if (threadIdx.x == 0 && a.status) atomicOr(a.status + ENTMAX_ATTN_STATUS_FLAGS, ENTMAX_ATTN_FLAG_WAIT_EXPIRED);
+    const uint64_t t0 = global_ns();
+    while (global_ns() - t0 < 200000ull) { }
+    __syncthreads();
+  }
+  if (warp == 1) {
+    tc_fence_after();
+    tmem_dealloc(tmem_base, 512);
+  }
+}
+
+template <int HD>
+cudaError_t launch_tile_bwd_impl(const Problem& p, const void* q, const void* k, const void* v, const void* d_o,
+                                 const TileBwdArgs& args, cudaStream_t stream) {
+  CUtensorMap map_q, map_k, map_v, map_do;
+  cudaError_t err = make_tile_map(&map_q, q, p.D, p.N, p.H, p.B, p.sn, p.sh, p.sb);
+  if (err != cudaSuccess) return err;
+  err = make_tile_map(&map_k, k, p.D, p.N, p.H, p.B, p.sn, p.sh, p.sb);
+  if (err != cudaSuccess) return err;
+  err = make_tile_map(&map_v, v, p.D, p.N, p.H, p.B, p.sn, p.sh, p.sb);
+  if (err != cudaSuccess) return err;
+  err = make_tile_map(&map_do, d_o, p.D, p.N, p.H, p.B, p.sn, p.sh, p.sb);
+  if (err != cudaSuccess) return err;
+  err = cudaFuncSetAttribute(tile_bwd_kernel<HD>, cudaFuncAttributeMaxDynamicSharedMemorySize, BCfg<HD>::kSmemBytes);
+  if (err != cudaSuccess) return err;
+  int dev = 0, sms = 0;
+  err = cudaGetDevice(&dev);
+  if (err != cudaSuccess) return err;
+  err = cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+  if (err != cudaSuccess) return err;
+  const long all_tiles = (long)p.B * p.H * args.tiles_per_head;
+  const int grid = (int)(all_tiles < sms ? all_tiles : sms);
+  tile_bwd_kernel<HD><<<grid, kThreadsB, BCfg<HD>::kSmemBytes, stream>>>(map_q, map_k, map_v, map_do, args);
+  return cudaGetLastError();
+}
+
+}  // namespace
+
+cudaError_t launch_tile_bwd(const Problem& p, const void* q, const void* k, const void* v, const void* d_o,
+                            const float* scale, const float* tau, const int32_t* row_list, const int32_t* row_count,
+                            uint32_t* tile_mask, int32_t* tile_flag, int32_t* tile_list, int32_t* tile_count, void* dq,
+                            float* acc_dk, float* acc_dv, float* dc_rows, int32_t* status, cudaStream_t stream) {
+  const int tiles_per_head = (p.N + TM - 1) / TM;
+  mark_tiles_kernel<<<148, 256, 0, stream>>>(p.N, tiles_per_head, row_list, row_count, tile_mask, tile_flag, tile_list,
+                                             tile_count);
+  cudaError_t err = cudaGetLastError();
+  if (err != cudaSuccess) return err;
+  TileBwdArgs args;
+  args.B = p.B; args.H = p.H; args.N = p.N;
+  args.causal = p.causal;
+  args.expo_class = p.expo_class;
+  args.expo = p.expo;
+  args.alpha_m1 = p.alpha - 1.0f;
+  args.sm_scale = p.sm_scale;
+  args.scale = scale;
+  args.alibi = p.alibi;
+  args.scale_sb = p.scale_sb;
+  args.tile_list = tile_list;
+  args.tile_count = tile_count;
+  args.tile_mask = tile_mask;
+  args.tau = tau;
+  args.dq = dq;
+  args.acc_dk = acc_dk;
+  args.acc_dv = acc_dv;
+  args.dc_rows = dc_rows;
+  args.sb = p.sb; args.sh = p.sh; args.sn = p.sn;
+  args.status = status;
+  args.tiles_per_head = tiles_per_head;
+  return p.D == 64 ? launch_tile_bwd_impl<64>(p, q, k, v, d_o, args, stream)
+                   : launch_tile_bwd_impl<128>(p, q, k, v, d_o, args, stream);
+}
+
+}  // namespace entmax

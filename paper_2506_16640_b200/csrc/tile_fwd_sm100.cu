@@ -64,21 +64,6 @@ struct TileArgsK {
   int tiles_per_head;
 };
 
-// tcgen05.mma with separate descriptor high words for A and B
-__device__ __forceinline__ void umma_bf16_ab(uint32_t d_tmem, uint32_t a_lo, uint32_t a_hi, uint32_t b_lo, uint32_t b_hi,
-                                             uint32_t idesc, uint32_t accumulate) {
-  asm volatile(
-      "{\n"
-      " .reg .pred p;\n"
-      " .reg .b64 da, db;\n"
-      " mov.b64 da, {%1, %2};\n"
-      " mov.b64 db, {%3, %4};\n"
-      " setp.ne.b32 p, %6, 0;\n"
-      " tcgen05.mma.cta_group::1.kind::f16 [%0], da, db, %5, p;\n"
-      "}\n" ::"r"(d_tmem), "r"(a_lo), "r"(a_hi), "r"(b_lo), "r"(b_hi), "r"(idesc), "r"(accumulate)
-      : "memory");
-}
-
 // S = Q K^T: A, B bf16 K-major, fp32 accumulate, M = 128, N = TN
 __host__ __device__ constexpr uint32_t idesc_qk() {
   return (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(TN >> 3) << 17) | ((uint32_t)(TM >> 4) << 24);
@@ -520,6 +505,33 @@ __global__ void __launch_bounds__(kThreadsT, 1) tile_fwd_kernel(const __grid_con
   }
 }
 
+template <int HD>
+cudaError_t launch_tile_impl(const Problem& p, const void* q, const void* k, const void* v, const TileArgsK& args,
+                             cudaStream_t stream) {
+  CUtensorMap map_q, map_k, map_v;
+  cudaError_t err = make_tile_map(&map_q, q, p.D, p.N, p.H, p.B, p.sn, p.sh, p.sb);
+  if (err != cudaSuccess) return err;
+  err = make_tile_map(&map_k, k, p.D, p.N, p.H, p.B, p.sn, p.sh, p.sb);
+  if (err != cudaSuccess) return err;
+  err = make_tile_map(&map_v, v, p.D, p.N, p.H, p.B, p.sn, p.sh, p.sb);
+  if (err != cudaSuccess) return err;
+  err = cudaFuncSetAttribute(tile_fwd_kernel<HD>, cudaFuncAttributeMaxDynamicSharedMemorySize, TCfg<HD>::kSmemBytes);
+  if (err != cudaSuccess) return err;
+  int dev = 0, sms = 0;
+  err = cudaGetDevice(&dev);
+  if (err != cudaSuccess) return err;
+  err = cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+  if (err != cudaSuccess) return err;
+  const long all_tiles = (long)p.B * p.H * args.tiles_per_head;
+  const int grid = (int)(all_tiles < sms ? all_tiles : sms);
+  tile_fwd_kernel<HD><<<grid, kThreadsT, TCfg<HD>::kSmemBytes, stream>>>(map_q, map_k, map_v, args);
+  return cudaGetLastError();
+}
+
+}  // namespace
+
+namespace {
+
 typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
                                   const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
                                   CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
@@ -538,13 +550,18 @@ cudaError_t encode_fn(EncodeTiledFn* fn) {
   return cudaSuccess;
 }
 
+}  // namespace
+
+namespace sm100 {
+
 // [B,H,N,D] bf16 tensor as a 4-D map (D, N, H, B); box = 64 columns (one 128-byte swizzle row) x 128 rows
-cudaError_t tile_map(CUtensorMap* map, const void* base, const Problem& p) {
+cudaError_t make_tile_map(CUtensorMap* map, const void* base, int D, int N, int H, int B, int64_t sn, int64_t sh,
+                          int64_t sb) {
   EncodeTiledFn fn;
   cudaError_t err = encode_fn(&fn);
   if (err != cudaSuccess) return err;
-  cuuint64_t dims[4] = {(cuuint64_t)p.D, (cuuint64_t)p.N, (cuuint64_t)p.H, (cuuint64_t)p.B};
-  cuuint64_t strides[3] = {(cuuint64_t)p.sn * 2, (cuuint64_t)p.sh * 2, (cuuint64_t)p.sb * 2};
+  cuuint64_t dims[4] = {(cuuint64_t)D, (cuuint64_t)N, (cuuint64_t)H, (cuuint64_t)B};
+  cuuint64_t strides[3] = {(cuuint64_t)sn * 2, (cuuint64_t)sh * 2, (cuuint64_t)sb * 2};
   cuuint32_t box[4] = {64, 128, 1, 1};
   cuuint32_t estr[4] = {1, 1, 1, 1};
   CUresult r = fn(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, const_cast<void*>(base), dims, strides, box, estr,
@@ -553,30 +570,7 @@ cudaError_t tile_map(CUtensorMap* map, const void* base, const Problem& p) {
   return r == CUDA_SUCCESS ? cudaSuccess : cudaErrorInvalidValue;
 }
 
-template <int HD>
-cudaError_t launch_tile_impl(const Problem& p, const void* q, const void* k, const void* v, const TileArgsK& args,
-                             cudaStream_t stream) {
-  CUtensorMap map_q, map_k, map_v;
-  cudaError_t err = tile_map(&map_q, q, p);
-  if (err != cudaSuccess) return err;
-  err = tile_map(&map_k, k, p);
-  if (err != cudaSuccess) return err;
-  err = tile_map(&map_v, v, p);
-  if (err != cudaSuccess) return err;
-  err = cudaFuncSetAttribute(tile_fwd_kernel<HD>, cudaFuncAttributeMaxDynamicSharedMemorySize, TCfg<HD>::kSmemBytes);
-  if (err != cudaSuccess) return err;
-  int dev = 0, sms = 0;
-  err = cudaGetDevice(&dev);
-  if (err != cudaSuccess) return err;
-  err = cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
-  if (err != cudaSuccess) return err;
-  const long all_tiles = (long)p.B * p.H * args.tiles_per_head;
-  const int grid = (int)(all_tiles < sms ? all_tiles : sms);
-  tile_fwd_kernel<HD><<<grid, kThreadsT, TCfg<HD>::kSmemBytes, stream>>>(map_q, map_k, map_v, args);
-  return cudaGetLastError();
-}
-
-}  // namespace
+}  // namespace sm100
 
 cudaError_t launch_tile_fwd(const Problem& p, const void* q, const void* k, const void* v, const float* scale,
                             const int32_t* tile_list, const int32_t* tile_count, const int32_t* row_cnt, void* o,

@@ -106,6 +106,32 @@ def test_mixed_sparse_and_dense_rows_in_one_tile():
     assert 0 < dense < 2 * 1000
 
 
+@pytest.mark.parametrize("alpha", [1.25, 1.5, 2.0, 1.7])
+@pytest.mark.parametrize("N,d,causal", [(900, 128, True), (700, 64, False), (515, 128, False), (130, 64, True)])
+def test_dense_tiles_backward_on_tensor_cores(N, d, causal, alpha):
+    # every row dense: the backward runs as two passes of tensor-core tiles per Q tile (sum u, sum u dP; then
+    # P and dS tiles feeding dQ, dK, dV); several K tiles, a ragged tail, both head dims
+    inp = make_inputs(_small("dense_tiles_bwd", N, d, causal, use_scale=True, sigma=0.01 if alpha == 2.0 else 0.04,
+                             backward=True, seed=N + 7))
+    got = parity.run_fwd(inp, alpha)
+    bwd = parity.run_bwd(inp, alpha, got["tau"], got["dev"])
+    dense, tiles = int(bwd["status"][binding.STATUS_DENSE_ROWS]), int(bwd["status"][binding.STATUS_TILES])
+    assert dense > N // 8 and 1 <= tiles <= inp.workload.H * ((N + 127) // 128)
+    for bh in range(inp.workload.H):
+        parity.check_bwd_head(inp, alpha, bwd, bh)
+
+
+def test_mixed_sparse_and_dense_rows_backward():
+    # one-hot rows (list path) and dense rows (tile path) share Q tiles and key rows of dK, dV
+    inp = make_inputs(_small("mixed_bwd", 1000, 128, True, plant=3, use_scale=False, sigma=0.05, backward=True, seed=22))
+    got = parity.run_fwd(inp, 1.5)
+    bwd = parity.run_bwd(inp, 1.5, got["tau"], got["dev"])
+    dense = int(bwd["status"][binding.STATUS_DENSE_ROWS])
+    assert 0 < dense < 2 * 1000
+    for bh in range(inp.workload.H):
+        parity.check_bwd_head(inp, 1.5, bwd, bh)
+
+
 def test_n_mode_total_length_and_strided_layout():
     inp = make_inputs(_small("nmode", 300, 64, True, seed=11))
     got = parity.run_fwd(inp, 1.5, n_mode=1)
