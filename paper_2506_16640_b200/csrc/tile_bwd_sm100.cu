@@ -114,7 +114,20 @@ __global__ void mark_tiles_kernel(int N, int tiles_per_head, const int32_t* __re
   }
 }
 
-template <int HD>
+// y^e and y^(e-1) of a clamped y >= 0 (0 where the entry is outside the support: ok == false), with the
+// exponent class fixed at compile time so that the per-element code stays a few instructions
+template <int EC>
+__device__ __forceinline__ void pow_pair_c(float y, bool ok, float expo, float& ye, float& ye1) {
+  if constexpr (EC == kExpo2) { ye1 = y; ye = y * y; }
+  else if constexpr (EC == kExpo1) { ye1 = ok ? 1.0f : 0.f; ye = y; }
+  else if constexpr (EC == kExpo4) { const float t = y * y; ye1 = t * y; ye = t * t; }
+  else {
+    ye = 0.f; ye1 = 0.f;
+    if (ok) { ye1 = powf(y, expo - 1.0f); ye = ye1 * y; }
+  }
+}
+
+template <int HD, int EC>
 __global__ void __launch_bounds__(kThreadsB, 1) tile_bwd_kernel(const __grid_constant__ CUtensorMap map_q,
                                                                const __grid_constant__ CUtensorMap map_k,
                                                                const __grid_constant__ CUtensorMap map_v,
@@ -318,7 +331,8 @@ __global__ void __launch_bounds__(kThreadsB, 1) tile_bwd_kernel(const __grid_con
       const float g = c_i * a.sm_scale;
       const float slope = a.alibi ? a.alibi[h] / a.sm_scale : 0.f;   // bias in accumulator units
       const float tau = marked ? a.tau[grow] : 0.f;
-      float su = 0.f, sud = 0.f, rho = 0.f, dcp = 0.f;
+      float su = 0.f, sud = 0.f, rho = 0.f;
+      float dcs[2] = {0.f, 0.f};   // sum_j dS_ij * (accumulator + bias), two partial sums
       for (int t = 0; t < 2 * tiles && alive; ++t) {
         const bool pass_b = t >= tiles;
         const int kt = pass_b ? t - tiles : t;
@@ -333,7 +347,7 @@ __global__ void __launch_bounds__(kThreadsB, 1) tile_bwd_kernel(const __grid_con
           pdsphase ^= 1u;
           if (!alive) break;
         }
-#pragma unroll
+#pragma unroll 1
         for (int c = 0; c < TN / 32; ++c) {
           float sa[32], dp[32];
           tmem_ld32(taddr_row + C::kTmemS + c * 32, sa);
@@ -346,16 +360,20 @@ __global__ void __launch_bounds__(kThreadsB, 1) tile_bwd_kernel(const __grid_con
           }
           const bool edge = col0 + 31 > lim;
           if (!pass_b) {
+            // four independent partial sums each: one thread owns the row, so the additions would otherwise
+            // form two serial chains of 128 dependent operations per tile
+            float p0[4] = {0.f, 0.f, 0.f, 0.f}, p1[4] = {0.f, 0.f, 0.f, 0.f};
 #pragma unroll
             for (int u = 0; u < 32; ++u) {
-              const float y = fmaf(ra, sa[u], -tau);
-              if (y > 0.f && (!edge || col0 + u <= lim)) {
-                float ye, ye1;
-                pow_pair(y, a.expo_class, a.expo, ye, ye1);
-                su += ye1;
-                sud = fmaf(ye1, dp[u], sud);
-              }
+              const float yr = fmaf(ra, sa[u], -tau);
+              const bool ok = yr > 0.f && (!edge || col0 + u <= lim);
+              float ye, ye1;
+              pow_pair_c<EC>(ok ? yr : 0.f, ok, a.expo, ye, ye1);
+              p0[u & 3] += ye1;
+              p1[u & 3] = fmaf(ye1, dp[u], p1[u & 3]);
             }
+            su += (p0[0] + p0[1]) + (p0[2] + p0[3]);
+            sud += (p1[0] + p1[1]) + (p1[2] + p1[3]);
           } else {
             // P and g dS -> bf16 -> shared memory, K-major with 128-byte swizzle: row r, 16-byte unit u of
             // the 64-key block sits at r*128 + ((u ^ (r & 7)) * 16)
@@ -366,17 +384,14 @@ __global__ void __launch_bounds__(kThreadsB, 1) tile_bwd_kernel(const __grid_con
 #pragma unroll
               for (int z = 0; z < 8; ++z) {
                 const int u = u4 * 8 + z;
-                const float y = fmaf(ra, sa[u], -tau);
-                pv[z] = 0.f;
-                dv[z] = 0.f;
-                if (marked && y > 0.f && (!edge || col0 + u <= lim)) {
-                  float ye, ye1;
-                  pow_pair(y, a.expo_class, a.expo, ye, ye1);
-                  const float ds = ye1 * (dp[u] - rho);
-                  pv[z] = ye;
-                  dv[z] = g * ds;
-                  dcp = fmaf(ds, sa[u], dcp);
-                }
+                const float yr = fmaf(ra, sa[u], -tau);
+                const bool ok = marked && yr > 0.f && (!edge || col0 + u <= lim);
+                float ye, ye1;
+                pow_pair_c<EC>(ok ? yr : 0.f, ok, a.expo, ye, ye1);
+                const float ds = ye1 * (dp[u] - rho);
+                pv[z] = ye;
+                dv[z] = g * ds;
+                dcs[z & 1] = fmaf(ds, sa[u], dcs[z & 1]);
               }
               const uint32_t unit = (uint32_t)((c & 1) * 4 + u4);
               const uint32_t off = blk + ((unit ^ (uint32_t)(row_local & 7)) << 4);
@@ -447,7 +462,7 @@ __global__ void __launch_bounds__(kThreadsB, 1) tile_bwd_kernel(const __grid_con
         }
       }
       // dL/dc_i = sum_j dS_ij z_ij with z_ij = sm_scale * (accumulator + bias in accumulator units)
-      if (marked && a.dc_rows) a.dc_rows[grow] = dcp * a.sm_scale;
+      if (marked && a.dc_rows) a.dc_rows[grow] = (dcs[0] + dcs[1]) * a.sm_scale;
       if (a.status && threadIdx.x == 64) atomicAdd(a.status + ENTMAX_ATTN_STATUS_TILES, 1);
       tc_fence_before();
       __syncwarp();
@@ -470,7 +485,7 @@ __global__ void __launch_bounds__(kThreadsB, 1) tile_bwd_kernel(const __grid_con
   }
 }
 
-template <int HD>
+template <int HD, int EC>
 cudaError_t launch_tile_bwd_impl(const Problem& p, const void* q, const void* k, const void* v, const void* d_o,
                                  const TileBwdArgs& args, cudaStream_t stream) {
   CUtensorMap map_q, map_k, map_v, map_do;
@@ -482,7 +497,7 @@ cudaError_t launch_tile_bwd_impl(const Problem& p, const void* q, const void* k,
   if (err != cudaSuccess) return err;
   err = make_tile_map(&map_do, d_o, p.D, p.N, p.H, p.B, p.sn, p.sh, p.sb);
   if (err != cudaSuccess) return err;
-  err = cudaFuncSetAttribute(tile_bwd_kernel<HD>, cudaFuncAttributeMaxDynamicSharedMemorySize, BCfg<HD>::kSmemBytes);
+  err = cudaFuncSetAttribute(tile_bwd_kernel<HD, EC>, cudaFuncAttributeMaxDynamicSharedMemorySize, BCfg<HD>::kSmemBytes);
   if (err != cudaSuccess) return err;
   int dev = 0, sms = 0;
   err = cudaGetDevice(&dev);
@@ -491,7 +506,7 @@ cudaError_t launch_tile_bwd_impl(const Problem& p, const void* q, const void* k,
   if (err != cudaSuccess) return err;
   const long all_tiles = (long)p.B * p.H * args.tiles_per_head;
   const int grid = (int)(all_tiles < sms ? all_tiles : sms);
-  tile_bwd_kernel<HD><<<grid, kThreadsB, BCfg<HD>::kSmemBytes, stream>>>(map_q, map_k, map_v, map_do, args);
+  tile_bwd_kernel<HD, EC><<<grid, kThreadsB, BCfg<HD>::kSmemBytes, stream>>>(map_q, map_k, map_v, map_do, args);
   return cudaGetLastError();
 }
 
@@ -527,8 +542,16 @@ cudaError_t launch_tile_bwd(const Problem& p, const void* q, const void* k, cons
   args.sb = p.sb; args.sh = p.sh; args.sn = p.sn;
   args.status = status;
   args.tiles_per_head = tiles_per_head;
-  return p.D == 64 ? launch_tile_bwd_impl<64>(p, q, k, v, d_o, args, stream)
-                   : launch_tile_bwd_impl<128>(p, q, k, v, d_o, args, stream);
+#define ENTMAX_TILE_BWD(EC)                                                                 \
+  (p.D == 64 ? launch_tile_bwd_impl<64, EC>(p, q, k, v, d_o, args, stream)                   \
+             : launch_tile_bwd_impl<128, EC>(p, q, k, v, d_o, args, stream))
+  switch (p.expo_class) {
+    case kExpo2: return ENTMAX_TILE_BWD(kExpo2);
+    case kExpo1: return ENTMAX_TILE_BWD(kExpo1);
+    case kExpo4: return ENTMAX_TILE_BWD(kExpo4);
+    default: return ENTMAX_TILE_BWD(kExpoGeneral);
+  }
+#undef ENTMAX_TILE_BWD
 }
 
 }  // namespace entmax
