@@ -52,6 +52,19 @@ struct WsLayout {
 
 WsLayout make_layout(const Problem& p, bool is_bwd);
 
+// y^e and y^(e-1) of a clamped y >= 0 (0 where the entry is outside the support: ok == false), with the
+// exponent class fixed at compile time so that the per-element code stays a few instructions
+template <int EC>
+__device__ __forceinline__ void pow_pair_c(float y, bool ok, float expo, float& ye, float& ye1) {
+  if constexpr (EC == kExpo2) { ye1 = y; ye = y * y; }
+  else if constexpr (EC == kExpo1) { ye1 = ok ? 1.0f : 0.f; ye = y; }
+  else if constexpr (EC == kExpo4) { const float t = y * y; ye1 = t * y; ye = t * t; }
+  else {
+    ye = 0.f; ye1 = 0.f;
+    if (ok) { ye1 = powf(y, expo - 1.0f); ye = ye1 * y; }
+  }
+}
+
 // y^e and y^(e-1) for y > 0
 __device__ __forceinline__ void pow_pair(float y, int expo_class, float expo, float& ye, float& ye1) {
   if (expo_class == kExpo2) { ye1 = y; ye = y * y; }

@@ -114,19 +114,6 @@ __global__ void mark_tiles_kernel(int N, int tiles_per_head, const int32_t* __re
   }
 }
 
-// y^e and y^(e-1) of a clamped y >= 0 (0 where the entry is outside the support: ok == false), with the
-// exponent class fixed at compile time so that the per-element code stays a few instructions
-template <int EC>
-__device__ __forceinline__ void pow_pair_c(float y, bool ok, float expo, float& ye, float& ye1) {
-  if constexpr (EC == kExpo2) { ye1 = y; ye = y * y; }
-  else if constexpr (EC == kExpo1) { ye1 = ok ? 1.0f : 0.f; ye = y; }
-  else if constexpr (EC == kExpo4) { const float t = y * y; ye1 = t * y; ye = t * t; }
-  else {
-    ye = 0.f; ye1 = 0.f;
-    if (ok) { ye1 = powf(y, expo - 1.0f); ye = ye1 * y; }
-  }
-}
-
 template <int HD, int EC>
 __global__ void __launch_bounds__(kThreadsB, 1) tile_bwd_kernel(const __grid_constant__ CUtensorMap map_q,
                                                                const __grid_constant__ CUtensorMap map_k,

@@ -81,14 +81,7 @@ __device__ __forceinline__ uint32_t v_desc_lo(uint32_t saddr) {
   return ((saddr & 0x3FFFFu) >> 4) | ((uint32_t)((TN * 128) >> 4) << 16);
 }
 
-__device__ __forceinline__ float pow_e(float y, int expo_class, float expo) {
-  if (expo_class == kExpo2) return y * y;
-  if (expo_class == kExpo1) return y;
-  if (expo_class == kExpo4) { const float t = y * y; return t * t; }
-  return powf(y, expo);
-}
-
-template <int HD>
+template <int HD, int EC>
 __global__ void __launch_bounds__(kThreadsT, 1) tile_fwd_kernel(const __grid_constant__ CUtensorMap map_q,
                                                                const __grid_constant__ CUtensorMap map_k,
                                                                const __grid_constant__ CUtensorMap map_v,
@@ -317,7 +310,7 @@ __global__ void __launch_bounds__(kThreadsT, 1) tile_fwd_kernel(const __grid_con
             pphase ^= 1u;
             if (!alive) break;
           }
-#pragma unroll
+#pragma unroll 1
           for (int c = 0; c < TN / 32; ++c) {
             float va[32];
             tmem_ld32(taddr_row + sbuf * TN + c * 32, va);
@@ -328,68 +321,31 @@ __global__ void __launch_bounds__(kThreadsT, 1) tile_fwd_kernel(const __grid_con
               for (int u = 0; u < 32; ++u) va[u] = fmaf(slope, (float)(col0 + u - i), va[u]);
             }
             // columns past the row's last visible key only occur in the tiles at the causal diagonal / the tail
-            if (col0 + 31 > lim) {
-#pragma unroll
-              for (int u = 0; u < 32; ++u) va[u] = (col0 + u <= lim) ? va[u] : -INFINITY;
-            }
+            const bool edge = col0 + 31 > lim;
             if (s == 0) {
-              // y_max: with ra > 0 the largest accumulator, otherwise (negative scale) the smallest
-              float m = va[0];
-              if (ra >= 0.f) {
+              // y_max over the visible keys
+              float m[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
 #pragma unroll
-                for (int u = 1; u < 32; ++u) m = fmaxf(m, va[u]);
-                if (m > -INFINITY) ymax = fmaxf(ymax, ra * m);
-              } else {
-#pragma unroll
-                for (int u = 0; u < 32; ++u)
-                  if (col0 + u <= lim) ymax = fmaxf(ymax, ra * va[u]);
+              for (int u = 0; u < 32; ++u) {
+                const float yv = ra * va[u];
+                m[u & 3] = fmaxf(m[u & 3], (!edge || col0 + u <= lim) ? yv : -INFINITY);
               }
+              ymax = fmaxf(ymax, fmaxf(fmaxf(m[0], m[1]), fmaxf(m[2], m[3])));
             } else if (!output) {
-              // masked columns hold -inf: y = ra * acc - tau is -inf (ra > 0) and clamps to 0; a negative
-              // scale is rare enough for the general loop
               // four independent partial sums each: one thread owns the row, so the additions would
               // otherwise form two serial chains of 128 dependent operations per tile
               float p0[4] = {0.f, 0.f, 0.f, 0.f}, p1[4] = {0.f, 0.f, 0.f, 0.f};
-              if (a.expo_class == kExpo2 && ra > 0.f) {
 #pragma unroll
-                for (int u = 0; u < 32; ++u) {
-                  const float y = fmaxf(fmaf(ra, va[u], -tau), 0.f);
-                  p0[u & 3] = fmaf(y, y, p0[u & 3]);
-                  p1[u & 3] += y;
-                }
-                s0 += (p0[0] + p0[1]) + (p0[2] + p0[3]);
-                s1 += (p1[0] + p1[1]) + (p1[2] + p1[3]);
-              } else if (a.expo_class == kExpo1 && ra > 0.f) {
-#pragma unroll
-                for (int u = 0; u < 32; ++u) {
-                  const float y = fmaf(ra, va[u], -tau);
-                  p0[u & 3] += fmaxf(y, 0.f);
-                  p1[u & 3] += y > 0.f ? 1.0f : 0.f;
-                }
-                s0 += (p0[0] + p0[1]) + (p0[2] + p0[3]);
-                s1 += (p1[0] + p1[1]) + (p1[2] + p1[3]);
-              } else if (a.expo_class == kExpo4 && ra > 0.f) {
-#pragma unroll
-                for (int u = 0; u < 32; ++u) {
-                  const float y = fmaxf(fmaf(ra, va[u], -tau), 0.f);
-                  const float y2 = y * y;
-                  p0[u & 3] = fmaf(y2, y2, p0[u & 3]);
-                  p1[u & 3] = fmaf(y2, y, p1[u & 3]);
-                }
-                s0 += (p0[0] + p0[1]) + (p0[2] + p0[3]);
-                s1 += (p1[0] + p1[1]) + (p1[2] + p1[3]);
-              } else {
-#pragma unroll
-                for (int u = 0; u < 32; ++u) {
-                  const float y = fmaf(ra, va[u], -tau);
-                  if (y > 0.f && col0 + u <= lim) {
-                    float ye, ye1;
-                    pow_pair(y, a.expo_class, a.expo, ye, ye1);
-                    s0 += ye;
-                    s1 += ye1;
-                  }
-                }
+              for (int u = 0; u < 32; ++u) {
+                const float yr = fmaf(ra, va[u], -tau);
+                const bool ok = yr > 0.f && (!edge || col0 + u <= lim);
+                float ye, ye1;
+                pow_pair_c<EC>(ok ? yr : 0.f, ok, a.expo, ye, ye1);
+                p0[u & 3] += ye;
+                p1[u & 3] += ye1;
               }
+              s0 += (p0[0] + p0[1]) + (p0[2] + p0[3]);
+              s1 += (p1[0] + p1[1]) + (p1[2] + p1[3]);
             } else {
               // P -> bf16 -> shared memory, K-major with 128-byte swizzle: row r, 16-byte unit u of the
               // 64-key block sits at r*128 + ((u ^ (r & 7)) * 16)
@@ -403,8 +359,10 @@ __global__ void __launch_bounds__(kThreadsT, 1) tile_fwd_kernel(const __grid_con
 #pragma unroll
                   for (int z = 0; z < 2; ++z) {
                     const int u = u4 * 8 + e2 * 2 + z;
-                    const float y = fmaf(ra, va[u], -tau);
-                    pv[z] = (y > 0.f && col0 + u <= lim && valid) ? pow_e(y, a.expo_class, a.expo) : 0.f;
+                    const float yr = fmaf(ra, va[u], -tau);
+                    const bool ok = valid && yr > 0.f && (!edge || col0 + u <= lim);
+                    float ye1;
+                    pow_pair_c<EC>(ok ? yr : 0.f, ok, a.expo, pv[z], ye1);
                   }
                   const __nv_bfloat162 hh = __floats2bfloat162_rn(pv[0], pv[1]);
                   w[e2] = *reinterpret_cast<const uint32_t*>(&hh);
@@ -505,7 +463,7 @@ __global__ void __launch_bounds__(kThreadsT, 1) tile_fwd_kernel(const __grid_con
   }
 }
 
-template <int HD>
+template <int HD, int EC>
 cudaError_t launch_tile_impl(const Problem& p, const void* q, const void* k, const void* v, const TileArgsK& args,
                              cudaStream_t stream) {
   CUtensorMap map_q, map_k, map_v;
@@ -515,7 +473,7 @@ cudaError_t launch_tile_impl(const Problem& p, const void* q, const void* k, con
   if (err != cudaSuccess) return err;
   err = make_tile_map(&map_v, v, p.D, p.N, p.H, p.B, p.sn, p.sh, p.sb);
   if (err != cudaSuccess) return err;
-  err = cudaFuncSetAttribute(tile_fwd_kernel<HD>, cudaFuncAttributeMaxDynamicSharedMemorySize, TCfg<HD>::kSmemBytes);
+  err = cudaFuncSetAttribute(tile_fwd_kernel<HD, EC>, cudaFuncAttributeMaxDynamicSharedMemorySize, TCfg<HD>::kSmemBytes);
   if (err != cudaSuccess) return err;
   int dev = 0, sms = 0;
   err = cudaGetDevice(&dev);
@@ -524,7 +482,7 @@ cudaError_t launch_tile_impl(const Problem& p, const void* q, const void* k, con
   if (err != cudaSuccess) return err;
   const long all_tiles = (long)p.B * p.H * args.tiles_per_head;
   const int grid = (int)(all_tiles < sms ? all_tiles : sms);
-  tile_fwd_kernel<HD><<<grid, kThreadsT, TCfg<HD>::kSmemBytes, stream>>>(map_q, map_k, map_v, args);
+  tile_fwd_kernel<HD, EC><<<grid, kThreadsT, TCfg<HD>::kSmemBytes, stream>>>(map_q, map_k, map_v, args);
   return cudaGetLastError();
 }
 
@@ -593,7 +551,16 @@ cudaError_t launch_tile_fwd(const Problem& p, const void* q, const void* k, cons
   args.sb = p.sb; args.sh = p.sh; args.sn = p.sn;
   args.status = status;
   args.tiles_per_head = (p.N + TM - 1) / TM;
-  return p.D == 64 ? launch_tile_impl<64>(p, q, k, v, args, stream) : launch_tile_impl<128>(p, q, k, v, args, stream);
+#define ENTMAX_TILE_FWD(EC)                                                  \
+  (p.D == 64 ? launch_tile_impl<64, EC>(p, q, k, v, args, stream)             \
+             : launch_tile_impl<128, EC>(p, q, k, v, args, stream))
+  switch (p.expo_class) {
+    case kExpo2: return ENTMAX_TILE_FWD(kExpo2);
+    case kExpo1: return ENTMAX_TILE_FWD(kExpo1);
+    case kExpo4: return ENTMAX_TILE_FWD(kExpo4);
+    default: return ENTMAX_TILE_FWD(kExpoGeneral);
+  }
+#undef ENTMAX_TILE_FWD
 }
 
 }  // namespace entmax
