@@ -73,7 +73,7 @@ typedef struct {
 #define ENTMAX_ATTN_STATUS_FLAGS 0         /* bit field below; 0 = clean run                                   */
 #define ENTMAX_ATTN_STATUS_DENSE_ROWS 1    /* rows whose support did not fit the sparse list (dense fallback)  */
 #define ENTMAX_ATTN_STATUS_TILE_SWEEPS 2   /* forward: sweeps over K spent by the dense-tile path, summed over tiles */
-#define ENTMAX_ATTN_STATUS_TILES 3         /* forward: 128-row Q tiles the dense-tile path processed               */
+#define ENTMAX_ATTN_STATUS_TILES 3         /* 128-row Q tiles the dense-tile path of this call processed           */
 #define ENTMAX_ATTN_FLAG_WAIT_EXPIRED 1    /* a bounded on-chip wait ran out; outputs of that call are invalid */
 #define ENTMAX_ATTN_FLAG_BAD_SCALE 2       /* some c_i was not finite                                          */
 
