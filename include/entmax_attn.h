@@ -76,6 +76,7 @@ typedef struct {
 #define ENTMAX_ATTN_STATUS_TILES 3         /* 128-row Q tiles the dense-tile path of this call processed           */
 #define ENTMAX_ATTN_FLAG_WAIT_EXPIRED 1    /* a bounded on-chip wait ran out; outputs of that call are invalid */
 #define ENTMAX_ATTN_FLAG_BAD_SCALE 2       /* some c_i was not finite                                          */
+#define ENTMAX_ATTN_FLAG_BAD_LENGTH 4      /* entmax_attn_decode_fwd: some kv_len[b] outside [q_len, kv_capacity] */
 
 /* Bytes of scratch the caller must pass to entmax_attn_fwd (is_bwd = 0) or entmax_attn_bwd
  * (is_bwd = 1) for these params.  Returns 0 if the params are invalid.  No paper counterpart: the
@@ -190,6 +191,43 @@ typedef struct {
   int32_t keep_limit; /* see row_count                                                                        */
 } entmax_attn_ws_layout;
 int entmax_attn_workspace_layout(const entmax_attn_params* params, entmax_attn_ws_layout* out);
+
+/* Decode-shape forward (inference with a key/value cache): q_len new query rows per sequence against
+ * that sequence's cached keys and values, sequences of different lengths in one batch.  The paper
+ * evaluates its models at contexts far beyond the training length (Sec. 4, App. G: up to 65K tokens);
+ * generating there means exactly this shape.  Query t of sequence b sits at position
+ * pos = kv_len[b] - q_len + t, sees the keys j <= pos (causal among the new rows), and is row pos of the
+ * full causal problem: Eq. 1 on s_j = c (sm_scale <q,k_j> - m_h (pos - j)), c from Eq. "asentmax" with
+ * n = pos + 1 (c = delta_h for n = 1), the ALiBi term only if slopes are given.
+ *   q            in,  device bf16 [batch, heads, q_len, head_dim] contiguous; 1 <= q_len <= ENTMAX_ATTN_DECODE_MAX_Q
+ *   k, v         in,  device bf16 [batch, heads, kv_capacity, head_dim] with element strides
+ *                kv_stride_b/h/n (all 0 = contiguous; multiples of 8; head_dim innermost), the same for both
+ *   kv_len       in,  device int32 [batch], q_len <= kv_len[b] <= kv_capacity (the new rows' keys included);
+ *                NULL = every sequence has kv_capacity keys.  A value outside the range sets
+ *                ENTMAX_ATTN_FLAG_BAD_LENGTH in device_status and is clamped into it.
+ *   beta, gamma, delta   in, device float32 [heads]; all three or none
+ *   alibi_slopes in,  device float32 [heads] or NULL
+ *   o            out, device bf16 [batch, heads, q_len, head_dim] contiguous
+ *   tau          out, device float32 [batch, heads, q_len]
+ *   support_size out, device int32 [batch, heads, q_len] or NULL: number of keys with p > 0
+ *   workspace    device scratch, 256-byte aligned, >= entmax_attn_decode_workspace_bytes(params)
+ *                (one fp32 score per query row and cached key, chunk maxima)
+ * K is read once (the HBM traffic that bounds this shape), V only on the support.  Results are
+ * bitwise reproducible.  device_status word ENTMAX_ATTN_STATUS_DENSE_ROWS counts query rows whose
+ * candidate set did not fit on chip (they are solved on the score row in the workspace instead).
+ * Errors as for entmax_attn_fwd; bf16 only. */
+#define ENTMAX_ATTN_DECODE_MAX_Q 8
+typedef struct {
+  int32_t batch, heads, q_len, kv_capacity, head_dim; /* head_dim in {64, 128}                              */
+  float alpha;                                         /* 1 < alpha <= 2                                     */
+  float sm_scale;                                      /* 0 means 1/sqrt(head_dim)                           */
+  int64_t kv_stride_b, kv_stride_h, kv_stride_n;       /* elements; all 0 = contiguous                       */
+} entmax_attn_decode_params;
+size_t entmax_attn_decode_workspace_bytes(const entmax_attn_decode_params* params);
+int entmax_attn_decode_fwd(const entmax_attn_decode_params* params, const void* q, const void* k, const void* v,
+                           const int32_t* kv_len, const float* beta, const float* gamma, const float* delta,
+                           const float* alibi_slopes, void* o, float* tau, int32_t* support_size, void* workspace,
+                           size_t workspace_bytes, int32_t* device_status, void* cuda_stream);
 
 /* Forward pass for callers that cannot provide a workspace.  (The paper has no counterpart: it does
  * not discuss memory management.)

@@ -18,7 +18,7 @@ LIB_PATH = os.path.join(_HERE, "libentmax_attn.so")
 DTYPE_BF16, DTYPE_FP32 = 0, 1
 STATUS_WORDS = 4
 STATUS_FLAGS, STATUS_DENSE_ROWS, STATUS_TILE_SWEEPS, STATUS_TILES = 0, 1, 2, 3
-FLAG_WAIT_EXPIRED, FLAG_BAD_SCALE = 1, 2
+FLAG_WAIT_EXPIRED, FLAG_BAD_SCALE, FLAG_BAD_LENGTH = 1, 2, 4
 
 
 class Params(ctypes.Structure):
@@ -26,6 +26,13 @@ class Params(ctypes.Structure):
                 ("head_dim", ctypes.c_int32), ("dtype", ctypes.c_int32), ("causal", ctypes.c_int32),
                 ("n_mode", ctypes.c_int32), ("alpha", ctypes.c_float), ("sm_scale", ctypes.c_float),
                 ("stride_b", ctypes.c_int64), ("stride_h", ctypes.c_int64), ("stride_n", ctypes.c_int64)]
+
+
+class DecodeParams(ctypes.Structure):
+    _fields_ = [("batch", ctypes.c_int32), ("heads", ctypes.c_int32), ("q_len", ctypes.c_int32),
+                ("kv_capacity", ctypes.c_int32), ("head_dim", ctypes.c_int32), ("alpha", ctypes.c_float),
+                ("sm_scale", ctypes.c_float), ("kv_stride_b", ctypes.c_int64), ("kv_stride_h", ctypes.c_int64),
+                ("kv_stride_n", ctypes.c_int64)]
 
 
 class WsLayout(ctypes.Structure):
@@ -79,6 +86,11 @@ def load():
         lib.entmax_attn_bwd_rowscale.argtypes = [pp, vp, vp, vp, fp, fp, vp, vp, vp, vp, fp, vp, ctypes.c_size_t, ip, vp]
         lib.entmax_attn_fwd_static.restype = ctypes.c_int
         lib.entmax_attn_fwd_static.argtypes = [pp, vp, vp, vp, fp, fp, fp, vp, fp, ip, vp]
+        dp = ctypes.POINTER(DecodeParams)
+        lib.entmax_attn_decode_workspace_bytes.restype = ctypes.c_size_t
+        lib.entmax_attn_decode_workspace_bytes.argtypes = [dp]
+        lib.entmax_attn_decode_fwd.restype = ctypes.c_int
+        lib.entmax_attn_decode_fwd.argtypes = [dp, vp, vp, vp, ip, fp, fp, fp, fp, vp, fp, ip, vp, ctypes.c_size_t, ip, vp]
         lib.entmax_attn_scores_debug.restype = ctypes.c_int
         lib.entmax_attn_scores_debug.argtypes = [pp, vp, vp, ctypes.c_int32, fp, vp, ctypes.c_size_t, ip, vp]
         lib.entmax_attn_profile_events.restype = ctypes.c_int
@@ -183,6 +195,37 @@ def entmax_attn_fwd_static(q, k, v, alpha, causal, beta=None, gamma=None, delta=
                                        _ptr(delta), _ptr(o), _ptr(tau), _ptr(status), _stream_ptr(stream))
     _check(rc, "entmax_attn_fwd_static")
     return o, tau
+
+
+def entmax_attn_decode_fwd(q, k, v, alpha, kv_len=None, beta=None, gamma=None, delta=None, *, alibi_slopes=None,
+                           sm_scale=0.0, o=None, tau=None, support_size=None, workspace=None, status=None,
+                           stream=None):
+    """Decode-shape forward: q [B,H,q_len,d] (contiguous) against the cache k, v [B,H,kv_capacity,d] (any
+    strides with d innermost, e.g. a view of a [B,kv_capacity,H,d] cache), kv_len int32 [B] or None.
+    Returns (o, tau, support_size)."""
+    if q.dtype != torch.bfloat16 or k.dtype != torch.bfloat16 or v.dtype != torch.bfloat16:
+        raise EntmaxAttnError("entmax_attn_decode_fwd: bf16 tensors only")
+    if not q.is_contiguous() or k.stride() != v.stride() or k.shape != v.shape or k.stride(3) != 1:
+        raise EntmaxAttnError("entmax_attn_decode_fwd: q contiguous; k and v the same shape and strides, d innermost")
+    B, H, QL, D = q.shape
+    if k.shape[0] != B or k.shape[1] != H or k.shape[3] != D:
+        raise EntmaxAttnError("entmax_attn_decode_fwd: q and k/v disagree on batch, heads or head_dim")
+    params = DecodeParams(B, H, QL, k.shape[2], D, float(alpha), float(sm_scale), k.stride(0), k.stride(1), k.stride(2))
+    o = torch.empty_like(q) if o is None else o
+    tau = torch.empty((B, H, QL), dtype=torch.float32, device=q.device) if tau is None else tau
+    if support_size is None:
+        support_size = torch.empty((B, H, QL), dtype=torch.int32, device=q.device)
+    if workspace is None:
+        nbytes = load().entmax_attn_decode_workspace_bytes(ctypes.byref(params))
+        if nbytes == 0:
+            raise EntmaxAttnError("entmax_attn_decode_workspace_bytes: invalid parameters")
+        workspace = torch.empty(nbytes, dtype=torch.uint8, device=q.device)
+    rc = load().entmax_attn_decode_fwd(ctypes.byref(params), _ptr(q), _ptr(k), _ptr(v), _ptr(kv_len), _ptr(beta),
+                                       _ptr(gamma), _ptr(delta), _ptr(alibi_slopes), _ptr(o), _ptr(tau),
+                                       _ptr(support_size), _ptr(workspace), workspace.numel(), _ptr(status),
+                                       _stream_ptr(stream))
+    _check(rc, "entmax_attn_decode_fwd")
+    return o, tau, support_size
 
 
 def entmax_attn_bwd(q, k, v, tau, d_o, alpha, causal, beta=None, gamma=None, delta=None, *, sm_scale=0.0, n_mode=0,

@@ -1,0 +1,501 @@
+// Decode-shape forward: a few new query rows per sequence against a long key/value cache, sequences of
+// different lengths in one batch.  Query t of sequence b sits at position pos = kv_len[b] - q_len + t,
+// sees the keys j <= pos, and gets Eq. 1 on its ASEntmax-scaled logits like any row of the full problem
+// (n_i = pos + 1).  With one to eight query rows there is no tile for the tensor cores to fill: the
+// path is bound by reading K once from HBM, so it runs on plain loads and FMAs:
+//   decode_scale_kernel    a_t = (alpha-1) c_t sm_scale per (sequence, head, query), c_t in fp64;
+//   decode_scores_kernel   streams K (16 bytes per lane, a key row per 8 or 16 lanes), fp32 dot products with
+//                          the query rows held in registers, y = a_t (q.k + bias) to a score row in the
+//                          workspace, and the maximum of every 512-key chunk;
+//   decode_solve_kernel    one CTA per query row: y_max, the candidates above the lower end of the bracket
+//                          of App. A (tau >= y_max - 1), Newton from the left on them (e-norm step), then
+//                          p = [y - tau]_+^e and O = sum_j p_j v_j as a gather of the support's V rows.
+// V is read only on the support.  Rows with more candidates than the CTA's list holds run the same
+// Newton iteration and output loop over the whole score row instead.
+// All sums are taken in a fixed order: repeated calls give identical bits.
+#include "common.cuh"
+
+namespace entmax {
+
+namespace {
+
+constexpr int kChunk = 512;        // keys per CTA of the score kernel
+constexpr int kScoreThreads = 256;
+constexpr int kSolveThreads = 256;
+constexpr int kPerThread = 8;      // candidate slots per thread of the solve kernel
+constexpr int kMaxNewtonD = 64;
+
+struct DecodeArgs {
+  int B, H, QL, NC, D;             // NC = kv_capacity
+  int expo_class;
+  float expo, alpha_m1, sm_scale;
+  int64_t ksb, ksh, ksn;           // element strides of K and V
+  const int32_t* kv_len;           // [B] or nullptr
+  const float* alibi;              // [H] or nullptr
+  int n_chunks;
+  size_t score_stride;             // floats per score row
+};
+
+__device__ __forceinline__ int seq_len(const DecodeArgs& a, int b, int32_t* status) {
+  int len = a.kv_len ? a.kv_len[b] : a.NC;
+  if (len < a.QL || len > a.NC) {
+    if (status) atomicOr(status + ENTMAX_ATTN_STATUS_FLAGS, ENTMAX_ATTN_FLAG_BAD_LENGTH);
+    len = len < a.QL ? a.QL : a.NC;
+  }
+  return len;
+}
+
+// a_t = (alpha-1) * c_t * sm_scale with c_t = delta + beta (ln n)^gamma in fp64 (c_t = delta for n = 1; 1 without scale)
+__global__ void decode_scale_kernel(DecodeArgs a, const float* __restrict__ beta, const float* __restrict__ gamma,
+                                    const float* __restrict__ delta, float* __restrict__ a_table,
+                                    int32_t* __restrict__ status) {
+  const int idx = blockIdx.x * blockDim.x + threadIdx.x;
+  if (idx >= a.B * a.H * a.QL) return;
+  const int t = idx % a.QL, bh = idx / a.QL, h = bh % a.H, b = bh / a.H;
+  float c = 1.0f;
+  if (beta) {
+    const long n = (long)seq_len(a, b, status) - a.QL + t + 1;
+    double cd = (double)delta[h];
+    if (n > 1) cd += (double)beta[h] * pow(log((double)n), (double)gamma[h]);
+    c = (float)cd;
+    if (!isfinite(c) && status) atomicOr(status + ENTMAX_ATTN_STATUS_FLAGS, ENTMAX_ATTN_FLAG_BAD_SCALE);
+  }
+  a_table[idx] = a.alpha_m1 * (c * a.sm_scale);
+}
+
+// PER consecutive bf16 values (PER = 2 or 4) as floats
+template <int PER>
+__device__ __forceinline__ void load_bf16_row(const __nv_bfloat16* p, float (&f)[PER]) {
+  if constexpr (PER == 4) {
+    const uint2 raw = *reinterpret_cast<const uint2*>(p);
+    f[0] = __uint_as_float(raw.x << 16); f[1] = __uint_as_float(raw.x & 0xffff0000u);
+    f[2] = __uint_as_float(raw.y << 16); f[3] = __uint_as_float(raw.y & 0xffff0000u);
+  } else {
+    const uint32_t raw = *reinterpret_cast<const uint32_t*>(p);
+    f[0] = __uint_as_float(raw << 16); f[1] = __uint_as_float(raw & 0xffff0000u);
+  }
+}
+
+__device__ __forceinline__ void unpack8(const uint4& raw, float (&f)[8]) {
+  const uint32_t w[4] = {raw.x, raw.y, raw.z, raw.w};
+#pragma unroll
+  for (int i = 0; i < 4; ++i) {
+    f[2 * i] = __uint_as_float(w[i] << 16);
+    f[2 * i + 1] = __uint_as_float(w[i] & 0xffff0000u);
+  }
+}
+
+// Sums vals[t] over the LPK lanes that share a key.  While more than one value is left, every step halves
+// them: a lane keeps one half and receives its partner's partial sums of that half (QL - 1 shuffles in all
+// instead of QL log2 LPK).  Returns in vals[0] the total of query `owned`; lanes that differ only in the
+// lane bits used after the values ran out hold copies.
+template <int QL, int LPK>
+__device__ __forceinline__ int reduce_queries(float (&vals)[QL], int lane) {
+  int owned = 0;
+  int count = QL;
+#pragma unroll
+  for (int off = LPK / 2; off > 0; off >>= 1) {
+    const bool upper = (lane & off) != 0;
+    if (count > 1) {
+      const int half = count / 2;
+#pragma unroll
+      for (int i = 0; i < QL / 2; ++i) {
+        if (i < half) {
+          const float keep = upper ? vals[half + i] : vals[i];
+          const float give = upper ? vals[i] : vals[half + i];
+          vals[i] = keep + __shfl_xor_sync(0xffffffffu, give, off);
+        }
+      }
+      if (upper) owned += half;
+      count = half;
+    } else {
+      vals[0] += __shfl_xor_sync(0xffffffffu, vals[0], off);
+    }
+  }
+  return owned;
+}
+
+template <int D, int QL>
+__global__ void __launch_bounds__(kScoreThreads) decode_scores_kernel(DecodeArgs a, const __nv_bfloat16* __restrict__ q,
+                                                                     const __nv_bfloat16* __restrict__ k,
+                                                                     const float* __restrict__ a_table,
+                                                                     float* __restrict__ scores,
+                                                                     float* __restrict__ chunk_max,
+                                                                     int32_t* __restrict__ status) {
+  constexpr int LPK = D / 8;            // lanes per key row (16 bytes each)
+  constexpr int KPW = 32 / LPK;         // keys per warp load
+  constexpr int kWarps = kScoreThreads / 32;
+  constexpr int kKeysPerWarp = kChunk / kWarps;
+  constexpr int kUnroll = 4;
+  // number of lane bits left after the halving steps of reduce_queries: lanes equal in the others hold copies
+  __shared__ float smax[kWarps][QL];
+  const int chunk = blockIdx.x, h = blockIdx.y, b = blockIdx.z;
+  const int len = seq_len(a, b, status);
+  const int key0 = chunk * kChunk;
+  if (key0 >= len) return;
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int sub = lane % LPK, kslot = lane / LPK;
+  const int bh = b * a.H + h;
+  // this lane's 8 elements of every query row
+  float qf[QL][8];
+#pragma unroll
+  for (int t = 0; t < QL; ++t) {
+    if (t < a.QL) {
+      const uint4 raw = *reinterpret_cast<const uint4*>(q + ((size_t)bh * a.QL + t) * D + sub * 8);
+      unpack8(raw, qf[t]);
+    } else {
+#pragma unroll
+      for (int e = 0; e < 8; ++e) qf[t][e] = 0.f;
+    }
+  }
+  const __nv_bfloat16* kbase = k + (size_t)b * a.ksb + (size_t)h * a.ksh + sub * 8;
+  const float slope = a.alibi ? a.alibi[h] / a.sm_scale : 0.f;   // bias in dot-product units
+  const int pos0 = len - a.QL;                                   // position of query 0
+  float vmax = -INFINITY;                                        // maximum of the values this lane writes
+  int owned = 0;
+  for (int it = 0; it < kKeysPerWarp / KPW; it += kUnroll) {
+    uint4 raw[kUnroll];
+    int jj[kUnroll];
+#pragma unroll
+    for (int u = 0; u < kUnroll; ++u) {
+      jj[u] = key0 + warp * kKeysPerWarp + (it + u) * KPW + kslot;
+      raw[u] = make_uint4(0u, 0u, 0u, 0u);
+      if (jj[u] < len) raw[u] = *reinterpret_cast<const uint4*>(kbase + (size_t)jj[u] * a.ksn);
+    }
+#pragma unroll
+    for (int u = 0; u < kUnroll; ++u) {
+      float kf[8];
+      unpack8(raw[u], kf);
+      float vals[QL];
+#pragma unroll
+      for (int t = 0; t < QL; ++t) {
+        float acc = 0.f;
+#pragma unroll
+        for (int e = 0; e < 8; ++e) acc = fmaf(qf[t][e], kf[e], acc);
+        vals[t] = acc;
+      }
+      owned = reduce_queries<QL, LPK>(vals, lane);
+      // one writer per (key, query): the lane whose bits below the halving steps are zero
+      constexpr int kHalvings = QL >= 8 ? 3 : QL >= 4 ? 2 : QL >= 2 ? 1 : 0;
+      constexpr int kCopyMask = (LPK >> kHalvings) - 1;          // lane bits used by the plain all-reduce steps
+      const int j = jj[u];
+      if ((sub & kCopyMask) == 0 && owned < a.QL && j < len) {
+        const int pos = pos0 + owned;
+        float y = -INFINITY;
+        if (j <= pos) y = a_table[bh * a.QL + owned] * fmaf(slope, (float)(j - pos), vals[0]);
+        scores[((size_t)bh * a.QL + owned) * a.score_stride + j] = y;
+        vmax = fmaxf(vmax, y);
+      }
+    }
+  }
+  // chunk maximum per query: lanes owning the same query within the warp, then the warps
+#pragma unroll
+  for (int t = 0; t < QL; ++t) {
+    float m = owned == t ? vmax : -INFINITY;
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) m = fmaxf(m, __shfl_xor_sync(0xffffffffu, m, o));
+    if (lane == 0) smax[warp][t] = m;
+  }
+  __syncthreads();
+  if (threadIdx.x < a.QL) {
+    float m = smax[0][threadIdx.x];
+#pragma unroll
+    for (int w = 1; w < kWarps; ++w) m = fmaxf(m, smax[w][threadIdx.x]);
+    chunk_max[((size_t)bh * a.QL + threadIdx.x) * a.n_chunks + chunk] = m;
+  }
+}
+
+// Sum over the CTA in a fixed order; every thread returns the same value.  `slot` alternates between
+// calls so that one barrier per call is enough.
+__device__ __forceinline__ float block_sum(float x, float (*red)[kSolveThreads / 32], int slot) {
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) x += __shfl_xor_sync(0xffffffffu, x, o);
+  if ((threadIdx.x & 31) == 0) red[slot][threadIdx.x >> 5] = x;
+  __syncthreads();
+  float s = 0.f;
+#pragma unroll
+  for (int w = 0; w < kSolveThreads / 32; ++w) s += red[slot][w];
+  return s;
+}
+
+template <int D>
+__global__ void __launch_bounds__(kSolveThreads) decode_solve_kernel(DecodeArgs a, const __nv_bfloat16* __restrict__ v,
+                                                                    const float* __restrict__ scores,
+                                                                    const float* __restrict__ chunk_max,
+                                                                    __nv_bfloat16* __restrict__ o,
+                                                                    float* __restrict__ tau_out,
+                                                                    int32_t* __restrict__ support_out,
+                                                                    int32_t* __restrict__ status) {
+  constexpr int kWarps = kSolveThreads / 32;
+  constexpr int PER = D / 32;
+  __shared__ float cand_y[kSolveThreads * kPerThread];
+  __shared__ int cand_j[kSolveThreads * kPerThread];
+  __shared__ float supp_p[kSolveThreads * kPerThread];
+  __shared__ int supp_j[kSolveThreads * kPerThread];
+  __shared__ float red[4][kWarps];
+  __shared__ int scan[kWarps];
+  __shared__ float opart[kWarps][D];
+  __shared__ int s_overflow;
+  const int row = blockIdx.x;                       // (b * H + h) * QL + t
+  const int t = row % a.QL, bh = row / a.QL, h = bh % a.H, b = bh / a.H;
+  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+  const int len = seq_len(a, b, nullptr);
+  const int nv = len - a.QL + t + 1;                // visible keys
+  const float* y_row = scores + (size_t)row * a.score_stride;
+  if (tid == 0) s_overflow = 0;
+  // ---- y_max from the chunk maxima
+  float m = -INFINITY;
+  const int chunks = (nv + kChunk - 1) / kChunk;
+  for (int c = tid; c < chunks; c += kSolveThreads) m = fmaxf(m, chunk_max[(size_t)row * a.n_chunks + c]);
+#pragma unroll
+  for (int off = 16; off > 0; off >>= 1) m = fmaxf(m, __shfl_xor_sync(0xffffffffu, m, off));
+  if (lane == 0) red[3][warp] = m;
+  __syncthreads();
+  float ymax = red[3][0];
+#pragma unroll
+  for (int w = 1; w < kWarps; ++w) ymax = fmaxf(ymax, red[3][w]);
+  // ---- candidates: y > y_max - 1 (App. A: tau >= y_max - 1), kept per thread in key order
+  const float floor_y = ymax - 1.0f;
+  int cnt = 0;
+  for (int j = tid; j < nv; j += kSolveThreads) {
+    const float y = y_row[j];
+    if (y > floor_y) {
+      if (cnt < kPerThread) {
+        cand_y[tid * kPerThread + cnt] = y;
+        cand_j[tid * kPerThread + cnt] = j;
+      }
+      ++cnt;
+    }
+  }
+  if (cnt > kPerThread) s_overflow = 1;
+  __syncthreads();
+  const bool dense = s_overflow != 0;
+  if (dense && tid == 0 && status) atomicAdd(status + ENTMAX_ATTN_STATUS_DENSE_ROWS, 1);
+  // ---- Newton from the left on f(tau) = sum [y - tau]_+^e - 1, e-norm step
+  float tau = floor_y;
+  for (int it = 0; it < kMaxNewtonD; ++it) {
+    float s0 = 0.f, s1 = 0.f;
+    if (!dense) {
+      for (int c = 0; c < cnt; ++c) {
+        const float d = cand_y[tid * kPerThread + c] - tau;
+        if (d > 0.f) {
+          float ye, ye1;
+          pow_pair(d, a.expo_class, a.expo, ye, ye1);
+          s0 += ye;
+          s1 += ye1;
+        }
+      }
+    } else {
+      for (int j = tid; j < nv; j += kSolveThreads) {
+        const float d = y_row[j] - tau;
+        if (d > 0.f) {
+          float ye, ye1;
+          pow_pair(d, a.expo_class, a.expo, ye, ye1);
+          s0 += ye;
+          s1 += ye1;
+        }
+      }
+    }
+    s0 = block_sum(s0, red, it & 1);
+    s1 = block_sum(s1, red, 2 + (it & 1));
+    if (!(s0 > 1.0f) || !(s1 > 0.f)) break;
+    const float step = threshold_step(s0, s1, a.expo_class, a.expo);
+    const float next = tau + step;
+    if (!(next > tau)) break;
+    tau = next;
+    if (step <= 1e-7f * fmaxf(1.0f, fabsf(tau))) break;
+  }
+  __syncthreads();
+  // ---- O = sum_j p_j v_j
+  const __nv_bfloat16* vbase = v + (size_t)b * a.ksb + (size_t)h * a.ksh + lane * PER;
+  float acc[PER];
+#pragma unroll
+  for (int e = 0; e < PER; ++e) acc[e] = 0.f;
+  int support = 0;
+  if (!dense) {
+    // compact the support in (thread, slot) order
+    int mine = 0;
+    for (int c = 0; c < cnt; ++c) mine += cand_y[tid * kPerThread + c] > tau ? 1 : 0;
+    int incl = mine;
+#pragma unroll
+    for (int off = 1; off < 32; off <<= 1) {
+      const int up = __shfl_up_sync(0xffffffffu, incl, off);
+      if (lane >= off) incl += up;
+    }
+    if (lane == 31) scan[warp] = incl;
+    __syncthreads();
+    int base = 0;
+    for (int w = 0; w < kWarps; ++w) {
+      if (w < warp) base += scan[w];
+      support += scan[w];
+    }
+    int at = base + incl - mine;
+    for (int c = 0; c < cnt; ++c) {
+      const float d = cand_y[tid * kPerThread + c] - tau;
+      if (d > 0.f) {
+        float ye, ye1;
+        pow_pair(d, a.expo_class, a.expo, ye, ye1);
+        supp_p[at] = ye;
+        supp_j[at] = cand_j[tid * kPerThread + c];
+        ++at;
+      }
+    }
+    __syncthreads();
+    for (int s = warp; s < support; s += kWarps) {
+      const float p = supp_p[s];
+      float vf[PER];
+      load_bf16_row<PER>(vbase + (size_t)supp_j[s] * a.ksn, vf);
+#pragma unroll
+      for (int e = 0; e < PER; ++e) acc[e] = fmaf(p, vf[e], acc[e]);
+    }
+  } else {
+    int local = 0;
+    for (int j = warp; j < nv; j += kWarps) {
+      const float d = y_row[j] - tau;
+      if (d > 0.f) {
+        float ye, ye1;
+        pow_pair(d, a.expo_class, a.expo, ye, ye1);
+        float vf[PER];
+        load_bf16_row<PER>(vbase + (size_t)j * a.ksn, vf);
+#pragma unroll
+        for (int e = 0; e < PER; ++e) acc[e] = fmaf(ye, vf[e], acc[e]);
+        ++local;
+      }
+    }
+    if (lane == 0) scan[warp] = local;
+    __syncthreads();
+    for (int w = 0; w < kWarps; ++w) support += scan[w];
+  }
+#pragma unroll
+  for (int e = 0; e < PER; ++e) opart[warp][lane * PER + e] = acc[e];
+  __syncthreads();
+  if (tid < D) {
+    float s = 0.f;
+#pragma unroll
+    for (int w = 0; w < kWarps; ++w) s += opart[w][tid];
+    o[(size_t)row * D + tid] = __float2bfloat16(s);
+  }
+  if (tid == 0) {
+    tau_out[row] = tau;
+    if (support_out) support_out[row] = support;
+  }
+}
+
+struct DecodeLayout {
+  size_t a_table, chunk_max, scores, total;
+  size_t score_stride;
+  int n_chunks;
+};
+
+DecodeLayout decode_layout(int B, int H, int QL, int NC) {
+  DecodeLayout l;
+  const size_t rows = (size_t)B * H * QL;
+  l.n_chunks = (NC + kChunk - 1) / kChunk;
+  l.score_stride = ((size_t)NC + 31) / 32 * 32;
+  size_t off = 0;
+  auto take = [&off](size_t bytes) { size_t at = off; off = (off + bytes + 255) / 256 * 256; return at; };
+  l.a_table = take(rows * sizeof(float));
+  l.chunk_max = take(rows * l.n_chunks * sizeof(float));
+  l.scores = take(rows * l.score_stride * sizeof(float));
+  l.total = off;
+  return l;
+}
+
+int check_decode_params(const entmax_attn_decode_params* p, DecodeArgs* a) {
+  if (!p) return ENTMAX_ATTN_EINVAL_NULL;
+  if (p->batch < 1 || p->heads < 1 || p->q_len < 1 || p->q_len > ENTMAX_ATTN_DECODE_MAX_Q) return ENTMAX_ATTN_EINVAL_SHAPE;
+  if (p->kv_capacity < p->q_len) return ENTMAX_ATTN_EINVAL_SHAPE;
+  if (p->head_dim != 64 && p->head_dim != 128) return ENTMAX_ATTN_EINVAL_SHAPE;
+  if ((long long)p->batch * p->heads * p->q_len > 0x7fffffffLL / 4) return ENTMAX_ATTN_EINVAL_SHAPE;
+  if (!(p->alpha > 1.0f) || !(p->alpha <= 2.0f)) return ENTMAX_ATTN_EINVAL_ALPHA;
+  if (!(p->sm_scale >= 0.f) || !(p->sm_scale < INFINITY)) return ENTMAX_ATTN_EINVAL_ALPHA;
+  a->B = p->batch; a->H = p->heads; a->QL = p->q_len; a->NC = p->kv_capacity; a->D = p->head_dim;
+  a->alpha_m1 = p->alpha - 1.0f;
+  a->sm_scale = p->sm_scale == 0.f ? 1.0f / sqrtf((float)p->head_dim) : p->sm_scale;
+  a->expo = 1.0f / (p->alpha - 1.0f);
+  a->expo_class = p->alpha == 2.0f ? kExpo1 : p->alpha == 1.5f ? kExpo2 : p->alpha == 1.25f ? kExpo4 : kExpoGeneral;
+  if (p->kv_stride_b == 0 && p->kv_stride_h == 0 && p->kv_stride_n == 0) {
+    a->ksn = p->head_dim;
+    a->ksh = (int64_t)p->kv_capacity * p->head_dim;
+    a->ksb = (int64_t)p->heads * p->kv_capacity * p->head_dim;
+  } else {
+    a->ksb = p->kv_stride_b; a->ksh = p->kv_stride_h; a->ksn = p->kv_stride_n;
+    if (a->ksn < p->head_dim || a->ksh < 1 || a->ksb < 1) return ENTMAX_ATTN_EINVAL_SHAPE;
+    if (a->ksn % 8 || a->ksh % 8 || a->ksb % 8) return ENTMAX_ATTN_EINVAL_SHAPE;
+  }
+  return ENTMAX_ATTN_OK;
+}
+
+template <int D>
+cudaError_t launch_scores(const DecodeArgs& a, dim3 grid, const __nv_bfloat16* q, const __nv_bfloat16* k,
+                          const float* a_table, float* scores, float* chunk_max, int32_t* status, cudaStream_t stream) {
+  if (a.QL == 1) decode_scores_kernel<D, 1><<<grid, kScoreThreads, 0, stream>>>(a, q, k, a_table, scores, chunk_max, status);
+  else if (a.QL == 2) decode_scores_kernel<D, 2><<<grid, kScoreThreads, 0, stream>>>(a, q, k, a_table, scores, chunk_max, status);
+  else if (a.QL <= 4) decode_scores_kernel<D, 4><<<grid, kScoreThreads, 0, stream>>>(a, q, k, a_table, scores, chunk_max, status);
+  else decode_scores_kernel<D, 8><<<grid, kScoreThreads, 0, stream>>>(a, q, k, a_table, scores, chunk_max, status);
+  return cudaGetLastError();
+}
+
+}  // namespace
+
+}  // namespace entmax
+
+using namespace entmax;
+
+extern "C" size_t entmax_attn_decode_workspace_bytes(const entmax_attn_decode_params* params) {
+  DecodeArgs a;
+  if (check_decode_params(params, &a) != ENTMAX_ATTN_OK) return 0;
+  return decode_layout(a.B, a.H, a.QL, a.NC).total;
+}
+
+extern "C" int entmax_attn_decode_fwd(const entmax_attn_decode_params* params, const void* q, const void* k,
+                                      const void* v, const int32_t* kv_len, const float* beta, const float* gamma,
+                                      const float* delta, const float* alibi_slopes, void* o, float* tau,
+                                      int32_t* support_size, void* workspace, size_t workspace_bytes,
+                                      int32_t* device_status, void* cuda_stream) {
+  DecodeArgs a;
+  int rc = check_decode_params(params, &a);
+  if (rc != ENTMAX_ATTN_OK) return rc;
+  if (!q || !k || !v || !o || !tau) return ENTMAX_ATTN_EINVAL_NULL;
+  const int given = (beta != nullptr) + (gamma != nullptr) + (delta != nullptr);
+  if (given != 0 && given != 3) return ENTMAX_ATTN_EINVAL_NULL;
+  auto aligned = [](const void* p, uintptr_t m) { return (reinterpret_cast<uintptr_t>(p) & (m - 1)) == 0; };
+  if (!aligned(q, 16) || !aligned(k, 16) || !aligned(v, 16) || !aligned(o, 16) || !aligned(tau, 4)) return ENTMAX_ATTN_EINVAL_ALIGN;
+  if ((kv_len && !aligned(kv_len, 4)) || (alibi_slopes && !aligned(alibi_slopes, 4)) ||
+      (support_size && !aligned(support_size, 4)))
+    return ENTMAX_ATTN_EINVAL_ALIGN;
+  const DecodeLayout lay = decode_layout(a.B, a.H, a.QL, a.NC);
+  if (!workspace || !aligned(workspace, 256) || workspace_bytes < lay.total) return ENTMAX_ATTN_EINVAL_WORKSPACE;
+  a.kv_len = kv_len;
+  a.alibi = alibi_slopes;
+  a.n_chunks = lay.n_chunks;
+  a.score_stride = lay.score_stride;
+  cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
+  uint8_t* ws = static_cast<uint8_t*>(workspace);
+  float* a_table = reinterpret_cast<float*>(ws + lay.a_table);
+  float* chunk_max = reinterpret_cast<float*>(ws + lay.chunk_max);
+  float* scores = reinterpret_cast<float*>(ws + lay.scores);
+  cudaError_t err;
+  if (device_status) {
+    err = cudaMemsetAsync(device_status, 0, sizeof(int32_t) * ENTMAX_ATTN_STATUS_WORDS, stream);
+    if (err != cudaSuccess) return ENTMAX_ATTN_ECUDA;
+  }
+  const int rows = a.B * a.H * a.QL;
+  decode_scale_kernel<<<(rows + 127) / 128, 128, 0, stream>>>(a, beta, gamma, delta, a_table, device_status);
+  err = cudaGetLastError();
+  if (err != cudaSuccess) return ENTMAX_ATTN_ECUDA;
+  const dim3 grid(lay.n_chunks, a.H, a.B);
+  const __nv_bfloat16* qb = static_cast<const __nv_bfloat16*>(q);
+  const __nv_bfloat16* kb = static_cast<const __nv_bfloat16*>(k);
+  err = a.D == 64 ? launch_scores<64>(a, grid, qb, kb, a_table, scores, chunk_max, device_status, stream)
+                  : launch_scores<128>(a, grid, qb, kb, a_table, scores, chunk_max, device_status, stream);
+  if (err != cudaSuccess) return ENTMAX_ATTN_ECUDA;
+  const __nv_bfloat16* vb = static_cast<const __nv_bfloat16*>(v);
+  __nv_bfloat16* ob = static_cast<__nv_bfloat16*>(o);
+  if (a.D == 64)
+    decode_solve_kernel<64><<<rows, kSolveThreads, 0, stream>>>(a, vb, scores, chunk_max, ob, tau, support_size, device_status);
+  else
+    decode_solve_kernel<128><<<rows, kSolveThreads, 0, stream>>>(a, vb, scores, chunk_max, ob, tau, support_size, device_status);
+  err = cudaGetLastError();
+  return err == cudaSuccess ? ENTMAX_ATTN_OK : ENTMAX_ATTN_ECUDA;
+}

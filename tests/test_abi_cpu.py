@@ -85,6 +85,31 @@ def test_rejections_happen_before_any_device_work(lib):
     assert lib.entmax_attn_version() >= 100
 
 
+def test_decode_entry_point_rejections(lib):
+    from paper_2506_16640_b200.binding import DecodeParams
+
+    def dparams(**kw):
+        base = dict(batch=2, heads=4, q_len=2, kv_capacity=1000, head_dim=128, alpha=1.5, sm_scale=0.0, kv_stride_b=0,
+                    kv_stride_h=0, kv_stride_n=0)
+        base.update(kw)
+        return DecodeParams(**base)
+
+    p = dparams()
+    need = lib.entmax_attn_decode_workspace_bytes(ctypes.byref(p))
+    assert need >= 2 * 4 * 2 * 1000 * 4
+    for bad in [dparams(q_len=0), dparams(q_len=9), dparams(kv_capacity=1), dparams(head_dim=96), dparams(alpha=1.0),
+                dparams(alpha=2.5), dparams(kv_stride_b=8, kv_stride_h=8, kv_stride_n=64)]:
+        assert lib.entmax_attn_decode_workspace_bytes(ctypes.byref(bad)) == 0
+    fake, odd, nul = ctypes.c_void_p(4096), ctypes.c_void_p(4100), ctypes.c_void_p(0)
+    call = lambda q, ws, nbytes, beta=None: lib.entmax_attn_decode_fwd(
+        ctypes.byref(p), q, fake, fake, None, beta, None, None, None, fake, fake, None, ws, nbytes, None, None)
+    assert call(nul, fake, 1 << 30) == -6
+    assert call(odd, fake, 1 << 30) == -4
+    assert call(fake, fake, 1 << 30, beta=fake) == -6          # beta without gamma/delta
+    assert call(fake, fake, 16) == -5
+    assert call(fake, nul, 1 << 30) == -5
+
+
 def test_binding_fails_loudly_without_library(monkeypatch, tmp_path):
     from paper_2506_16640_b200 import binding
     monkeypatch.setattr(binding, "_lib", None)
