@@ -13,7 +13,7 @@ _ROOT = os.path.dirname(_HERE)
 CSRC = os.path.join(_HERE, "csrc")
 INCLUDE = os.path.join(_ROOT, "include")
 LIB = os.path.join(_HERE, "libentmax_attn.so")
-SOURCES = ["entmax_attn_api.cu", "dense_rows.cu", "row_lists.cu", "sweep_sm100.cu", "tile_fwd_sm100.cu", "tile_bwd_sm100.cu", "decode.cu", "no_alloc.cu"]
+SOURCES = ["entmax_attn_api.cu", "dense_rows.cu", "row_lists.cu", "sweep_sm100.cu", "tile_fwd_sm100.cu", "tile_bwd_sm100.cu", "decode.cu", "decode_scores_sm100.cu", "no_alloc.cu"]
 
 
 def _nvcc() -> str:
@@ -31,7 +31,7 @@ def needs_build() -> bool:
     if not os.path.exists(LIB):
         return True
     t = os.path.getmtime(LIB)
-    deps = _sources() + [os.path.join(CSRC, "common.cuh"), os.path.join(CSRC, "sm100_ptx.cuh"), os.path.join(INCLUDE, "entmax_attn.h")]
+    deps = _sources() + [os.path.join(CSRC, "common.cuh"), os.path.join(CSRC, "sm100_ptx.cuh"), os.path.join(CSRC, "decode.cuh"), os.path.join(INCLUDE, "entmax_attn.h")]
     return any(os.path.getmtime(d) > t for d in deps)
 
 

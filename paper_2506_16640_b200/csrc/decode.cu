@@ -1,49 +1,26 @@
 // Decode-shape forward: a few new query rows per sequence against a long key/value cache, sequences of
 // different lengths in one batch.  Query t of sequence b sits at position pos = kv_len[b] - q_len + t,
 // sees the keys j <= pos, and gets Eq. 1 on its ASEntmax-scaled logits like any row of the full problem
-// (n_i = pos + 1).  With one to eight query rows there is no tile for the tensor cores to fill: the
-// path is bound by reading K once from HBM, so it runs on plain loads and FMAs:
-//   decode_scale_kernel    a_t = (alpha-1) c_t sm_scale per (sequence, head, query), c_t in fp64;
-//   decode_scores_kernel   streams K (16 bytes per lane, a key row per 8 or 16 lanes), fp32 dot products with
-//                          the query rows held in registers, y = a_t (q.k + bias) to a score row in the
-//                          workspace, and the maximum of every 512-key chunk;
-//   decode_solve_kernel    one CTA per query row: y_max, the candidates above the lower end of the bracket
-//                          of App. A (tau >= y_max - 1), Newton from the left on them (e-norm step), then
-//                          p = [y - tau]_+^e and O = sum_j p_j v_j as a gather of the support's V rows.
+// (n_i = pos + 1).  The path is bound by reading K once from HBM:
+//   decode_scale_kernel       a_t = (alpha-1) c_t sm_scale per (sequence, head, query), c_t in fp64;
+//   decode_scores_tc_kernel   (decode_scores_sm100.cu) streams K through TMA and tcgen05, writes
+//                             y = a_t (q.k + bias) to a score row in the workspace and the maximum of every chunk;
+//   decode_solve_kernel       one CTA per query row: y_max, the candidates above the lower end of the bracket
+//                             of App. A (tau >= y_max - 1), Newton from the left on them (e-norm step), then
+//                             p = [y - tau]_+^e and O = sum_j p_j v_j as a gather of the support's V rows.
 // V is read only on the support.  Rows with more candidates than the CTA's list holds run the same
 // Newton iteration and output loop over the whole score row instead.
 // All sums are taken in a fixed order: repeated calls give identical bits.
 #include "common.cuh"
+#include "decode.cuh"
 
 namespace entmax {
 
 namespace {
 
-constexpr int kChunk = 512;        // keys per CTA of the score kernel
-constexpr int kScoreThreads = 256;
 constexpr int kSolveThreads = 256;
 constexpr int kPerThread = 8;      // candidate slots per thread of the solve kernel
 constexpr int kMaxNewtonD = 64;
-
-struct DecodeArgs {
-  int B, H, QL, NC, D;             // NC = kv_capacity
-  int expo_class;
-  float expo, alpha_m1, sm_scale;
-  int64_t ksb, ksh, ksn;           // element strides of K and V
-  const int32_t* kv_len;           // [B] or nullptr
-  const float* alibi;              // [H] or nullptr
-  int n_chunks;
-  size_t score_stride;             // floats per score row
-};
-
-__device__ __forceinline__ int seq_len(const DecodeArgs& a, int b, int32_t* status) {
-  int len = a.kv_len ? a.kv_len[b] : a.NC;
-  if (len < a.QL || len > a.NC) {
-    if (status) atomicOr(status + ENTMAX_ATTN_STATUS_FLAGS, ENTMAX_ATTN_FLAG_BAD_LENGTH);
-    len = len < a.QL ? a.QL : a.NC;
-  }
-  return len;
-}
 
 // a_t = (alpha-1) * c_t * sm_scale with c_t = delta + beta (ln n)^gamma in fp64 (c_t = delta for n = 1; 1 without scale)
 __global__ void decode_scale_kernel(DecodeArgs a, const float* __restrict__ beta, const float* __restrict__ gamma,
@@ -73,135 +50,6 @@ __device__ __forceinline__ void load_bf16_row(const __nv_bfloat16* p, float (&f)
   } else {
     const uint32_t raw = *reinterpret_cast<const uint32_t*>(p);
     f[0] = __uint_as_float(raw << 16); f[1] = __uint_as_float(raw & 0xffff0000u);
-  }
-}
-
-__device__ __forceinline__ void unpack8(const uint4& raw, float (&f)[8]) {
-  const uint32_t w[4] = {raw.x, raw.y, raw.z, raw.w};
-#pragma unroll
-  for (int i = 0; i < 4; ++i) {
-    f[2 * i] = __uint_as_float(w[i] << 16);
-    f[2 * i + 1] = __uint_as_float(w[i] & 0xffff0000u);
-  }
-}
-
-// Sums vals[t] over the LPK lanes that share a key.  While more than one value is left, every step halves
-// them: a lane keeps one half and receives its partner's partial sums of that half (QL - 1 shuffles in all
-// instead of QL log2 LPK).  Returns in vals[0] the total of query `owned`; lanes that differ only in the
-// lane bits used after the values ran out hold copies.
-template <int QL, int LPK>
-__device__ __forceinline__ int reduce_queries(float (&vals)[QL], int lane) {
-  int owned = 0;
-  int count = QL;
-#pragma unroll
-  for (int off = LPK / 2; off > 0; off >>= 1) {
-    const bool upper = (lane & off) != 0;
-    if (count > 1) {
-      const int half = count / 2;
-#pragma unroll
-      for (int i = 0; i < QL / 2; ++i) {
-        if (i < half) {
-          const float keep = upper ? vals[half + i] : vals[i];
-          const float give = upper ? vals[i] : vals[half + i];
-          vals[i] = keep + __shfl_xor_sync(0xffffffffu, give, off);
-        }
-      }
-      if (upper) owned += half;
-      count = half;
-    } else {
-      vals[0] += __shfl_xor_sync(0xffffffffu, vals[0], off);
-    }
-  }
-  return owned;
-}
-
-template <int D, int QL>
-__global__ void __launch_bounds__(kScoreThreads) decode_scores_kernel(DecodeArgs a, const __nv_bfloat16* __restrict__ q,
-                                                                     const __nv_bfloat16* __restrict__ k,
-                                                                     const float* __restrict__ a_table,
-                                                                     float* __restrict__ scores,
-                                                                     float* __restrict__ chunk_max,
-                                                                     int32_t* __restrict__ status) {
-  constexpr int LPK = D / 8;            // lanes per key row (16 bytes each)
-  constexpr int KPW = 32 / LPK;         // keys per warp load
-  constexpr int kWarps = kScoreThreads / 32;
-  constexpr int kKeysPerWarp = kChunk / kWarps;
-  constexpr int kUnroll = 4;
-  // number of lane bits left after the halving steps of reduce_queries: lanes equal in the others hold copies
-  __shared__ float smax[kWarps][QL];
-  const int chunk = blockIdx.x, h = blockIdx.y, b = blockIdx.z;
-  const int len = seq_len(a, b, status);
-  const int key0 = chunk * kChunk;
-  if (key0 >= len) return;
-  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  const int sub = lane % LPK, kslot = lane / LPK;
-  const int bh = b * a.H + h;
-  // this lane's 8 elements of every query row
-  float qf[QL][8];
-#pragma unroll
-  for (int t = 0; t < QL; ++t) {
-    if (t < a.QL) {
-      const uint4 raw = *reinterpret_cast<const uint4*>(q + ((size_t)bh * a.QL + t) * D + sub * 8);
-      unpack8(raw, qf[t]);
-    } else {
-#pragma unroll
-      for (int e = 0; e < 8; ++e) qf[t][e] = 0.f;
-    }
-  }
-  const __nv_bfloat16* kbase = k + (size_t)b * a.ksb + (size_t)h * a.ksh + sub * 8;
-  const float slope = a.alibi ? a.alibi[h] / a.sm_scale : 0.f;   // bias in dot-product units
-  const int pos0 = len - a.QL;                                   // position of query 0
-  float vmax = -INFINITY;                                        // maximum of the values this lane writes
-  int owned = 0;
-  for (int it = 0; it < kKeysPerWarp / KPW; it += kUnroll) {
-    uint4 raw[kUnroll];
-    int jj[kUnroll];
-#pragma unroll
-    for (int u = 0; u < kUnroll; ++u) {
-      jj[u] = key0 + warp * kKeysPerWarp + (it + u) * KPW + kslot;
-      raw[u] = make_uint4(0u, 0u, 0u, 0u);
-      if (jj[u] < len) raw[u] = *reinterpret_cast<const uint4*>(kbase + (size_t)jj[u] * a.ksn);
-    }
-#pragma unroll
-    for (int u = 0; u < kUnroll; ++u) {
-      float kf[8];
-      unpack8(raw[u], kf);
-      float vals[QL];
-#pragma unroll
-      for (int t = 0; t < QL; ++t) {
-        float acc = 0.f;
-#pragma unroll
-        for (int e = 0; e < 8; ++e) acc = fmaf(qf[t][e], kf[e], acc);
-        vals[t] = acc;
-      }
-      owned = reduce_queries<QL, LPK>(vals, lane);
-      // one writer per (key, query): the lane whose bits below the halving steps are zero
-      constexpr int kHalvings = QL >= 8 ? 3 : QL >= 4 ? 2 : QL >= 2 ? 1 : 0;
-      constexpr int kCopyMask = (LPK >> kHalvings) - 1;          // lane bits used by the plain all-reduce steps
-      const int j = jj[u];
-      if ((sub & kCopyMask) == 0 && owned < a.QL && j < len) {
-        const int pos = pos0 + owned;
-        float y = -INFINITY;
-        if (j <= pos) y = a_table[bh * a.QL + owned] * fmaf(slope, (float)(j - pos), vals[0]);
-        scores[((size_t)bh * a.QL + owned) * a.score_stride + j] = y;
-        vmax = fmaxf(vmax, y);
-      }
-    }
-  }
-  // chunk maximum per query: lanes owning the same query within the warp, then the warps
-#pragma unroll
-  for (int t = 0; t < QL; ++t) {
-    float m = owned == t ? vmax : -INFINITY;
-#pragma unroll
-    for (int o = 16; o > 0; o >>= 1) m = fmaxf(m, __shfl_xor_sync(0xffffffffu, m, o));
-    if (lane == 0) smax[warp][t] = m;
-  }
-  __syncthreads();
-  if (threadIdx.x < a.QL) {
-    float m = smax[0][threadIdx.x];
-#pragma unroll
-    for (int w = 1; w < kWarps; ++w) m = fmaxf(m, smax[w][threadIdx.x]);
-    chunk_max[((size_t)bh * a.QL + threadIdx.x) * a.n_chunks + chunk] = m;
   }
 }
 
@@ -245,7 +93,7 @@ __global__ void __launch_bounds__(kSolveThreads) decode_solve_kernel(DecodeArgs 
   if (tid == 0) s_overflow = 0;
   // ---- y_max from the chunk maxima
   float m = -INFINITY;
-  const int chunks = (nv + kChunk - 1) / kChunk;
+  const int chunks = (nv + a.chunk_keys - 1) / a.chunk_keys;
   for (int c = tid; c < chunks; c += kSolveThreads) m = fmaxf(m, chunk_max[(size_t)row * a.n_chunks + c]);
 #pragma unroll
   for (int off = 16; off > 0; off >>= 1) m = fmaxf(m, __shfl_xor_sync(0xffffffffu, m, off));
@@ -257,14 +105,33 @@ __global__ void __launch_bounds__(kSolveThreads) decode_solve_kernel(DecodeArgs 
   // ---- candidates: y > y_max - 1 (App. A: tau >= y_max - 1), kept per thread in key order
   const float floor_y = ymax - 1.0f;
   int cnt = 0;
-  for (int j = tid; j < nv; j += kSolveThreads) {
-    const float y = y_row[j];
-    if (y > floor_y) {
-      if (cnt < kPerThread) {
-        cand_y[tid * kPerThread + cnt] = y;
-        cand_j[tid * kPerThread + cnt] = j;
+  {
+    // four 16-byte loads in flight per thread; a thread meets its keys in increasing order
+    const float4* y_row4 = reinterpret_cast<const float4*>(y_row);
+    const int groups = (nv + 3) / 4;
+    const float4 none = make_float4(-INFINITY, -INFINITY, -INFINITY, -INFINITY);
+    for (int g0 = tid; g0 < groups; g0 += 4 * kSolveThreads) {
+      float4 yv[4];
+#pragma unroll
+      for (int u = 0; u < 4; ++u) {
+        const int g = g0 + u * kSolveThreads;
+        yv[u] = g < groups ? y_row4[g] : none;
       }
-      ++cnt;
+#pragma unroll
+      for (int u = 0; u < 4; ++u) {
+        const float ye[4] = {yv[u].x, yv[u].y, yv[u].z, yv[u].w};
+#pragma unroll
+        for (int e = 0; e < 4; ++e) {
+          const int j = 4 * (g0 + u * kSolveThreads) + e;
+          if (j < nv && ye[e] > floor_y) {
+            if (cnt < kPerThread) {
+              cand_y[tid * kPerThread + cnt] = ye[e];
+              cand_j[tid * kPerThread + cnt] = j;
+            }
+            ++cnt;
+          }
+        }
+      }
     }
   }
   if (cnt > kPerThread) s_overflow = 1;
@@ -384,13 +251,16 @@ __global__ void __launch_bounds__(kSolveThreads) decode_solve_kernel(DecodeArgs 
 struct DecodeLayout {
   size_t a_table, chunk_max, scores, total;
   size_t score_stride;
-  int n_chunks;
+  int chunk_keys, n_chunks;
 };
 
+// A CTA of the score kernel takes up to 1024 keys, fewer when the problem would otherwise leave SMs idle.
 DecodeLayout decode_layout(int B, int H, int QL, int NC) {
   DecodeLayout l;
   const size_t rows = (size_t)B * H * QL;
-  l.n_chunks = (NC + kChunk - 1) / kChunk;
+  l.chunk_keys = 1024;
+  while (l.chunk_keys > 128 && (long long)B * H * ((NC + l.chunk_keys - 1) / l.chunk_keys) < 4 * 148) l.chunk_keys /= 2;
+  l.n_chunks = (NC + l.chunk_keys - 1) / l.chunk_keys;
   l.score_stride = ((size_t)NC + 31) / 32 * 32;
   size_t off = 0;
   auto take = [&off](size_t bytes) { size_t at = off; off = (off + bytes + 255) / 256 * 256; return at; };
@@ -426,16 +296,6 @@ int check_decode_params(const entmax_attn_decode_params* p, DecodeArgs* a) {
   return ENTMAX_ATTN_OK;
 }
 
-template <int D>
-cudaError_t launch_scores(const DecodeArgs& a, dim3 grid, const __nv_bfloat16* q, const __nv_bfloat16* k,
-                          const float* a_table, float* scores, float* chunk_max, int32_t* status, cudaStream_t stream) {
-  if (a.QL == 1) decode_scores_kernel<D, 1><<<grid, kScoreThreads, 0, stream>>>(a, q, k, a_table, scores, chunk_max, status);
-  else if (a.QL == 2) decode_scores_kernel<D, 2><<<grid, kScoreThreads, 0, stream>>>(a, q, k, a_table, scores, chunk_max, status);
-  else if (a.QL <= 4) decode_scores_kernel<D, 4><<<grid, kScoreThreads, 0, stream>>>(a, q, k, a_table, scores, chunk_max, status);
-  else decode_scores_kernel<D, 8><<<grid, kScoreThreads, 0, stream>>>(a, q, k, a_table, scores, chunk_max, status);
-  return cudaGetLastError();
-}
-
 }  // namespace
 
 }  // namespace entmax
@@ -468,8 +328,13 @@ extern "C" int entmax_attn_decode_fwd(const entmax_attn_decode_params* params, c
   if (!workspace || !aligned(workspace, 256) || workspace_bytes < lay.total) return ENTMAX_ATTN_EINVAL_WORKSPACE;
   a.kv_len = kv_len;
   a.alibi = alibi_slopes;
+  a.chunk_keys = lay.chunk_keys;
   a.n_chunks = lay.n_chunks;
   a.score_stride = lay.score_stride;
+  int dev = 0, major = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess || cudaDeviceGetAttribute(&major, cudaDevAttrComputeCapabilityMajor, dev) != cudaSuccess)
+    return ENTMAX_ATTN_ECUDA;
+  if (major != 10) return ENTMAX_ATTN_EUNSUPPORTED;          // the score kernel needs tcgen05 / TMA
   cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
   uint8_t* ws = static_cast<uint8_t*>(workspace);
   float* a_table = reinterpret_cast<float*>(ws + lay.a_table);
@@ -484,11 +349,7 @@ extern "C" int entmax_attn_decode_fwd(const entmax_attn_decode_params* params, c
   decode_scale_kernel<<<(rows + 127) / 128, 128, 0, stream>>>(a, beta, gamma, delta, a_table, device_status);
   err = cudaGetLastError();
   if (err != cudaSuccess) return ENTMAX_ATTN_ECUDA;
-  const dim3 grid(lay.n_chunks, a.H, a.B);
-  const __nv_bfloat16* qb = static_cast<const __nv_bfloat16*>(q);
-  const __nv_bfloat16* kb = static_cast<const __nv_bfloat16*>(k);
-  err = a.D == 64 ? launch_scores<64>(a, grid, qb, kb, a_table, scores, chunk_max, device_status, stream)
-                  : launch_scores<128>(a, grid, qb, kb, a_table, scores, chunk_max, device_status, stream);
+  err = launch_decode_scores_tc(a, q, k, a_table, scores, chunk_max, device_status, stream);
   if (err != cudaSuccess) return ENTMAX_ATTN_ECUDA;
   const __nv_bfloat16* vb = static_cast<const __nv_bfloat16*>(v);
   __nv_bfloat16* ob = static_cast<__nv_bfloat16*>(o);

@@ -188,10 +188,10 @@ __device__ __forceinline__ float warp_sum(float x) {
 }
 
 // Host: a bf16 [B,H,N,D] tensor with element strides (sb, sh, sn) as a 4-D tensor map (D, N, H, B), box
-// 64 columns (one 128-byte swizzle row) by 128 rows, 128-byte swizzle, out-of-range rows read as zero.
+// 64 columns (one 128-byte swizzle row) by box_rows rows, 128-byte swizzle, out-of-range rows read as zero.
 // Defined in tile_fwd_sm100.cu.
 cudaError_t make_tile_map(CUtensorMap* map, const void* base, int D, int N, int H, int B, int64_t sn, int64_t sh,
-                          int64_t sb);
+                          int64_t sb, int box_rows = 128);
 
 
 }  // namespace sm100

@@ -512,15 +512,15 @@ cudaError_t encode_fn(EncodeTiledFn* fn) {
 
 namespace sm100 {
 
-// [B,H,N,D] bf16 tensor as a 4-D map (D, N, H, B); box = 64 columns (one 128-byte swizzle row) x 128 rows
+// [B,H,N,D] bf16 tensor as a 4-D map (D, N, H, B); box = 64 columns (one 128-byte swizzle row) x box_rows rows
 cudaError_t make_tile_map(CUtensorMap* map, const void* base, int D, int N, int H, int B, int64_t sn, int64_t sh,
-                          int64_t sb) {
+                          int64_t sb, int box_rows) {
   EncodeTiledFn fn;
   cudaError_t err = encode_fn(&fn);
   if (err != cudaSuccess) return err;
   cuuint64_t dims[4] = {(cuuint64_t)D, (cuuint64_t)N, (cuuint64_t)H, (cuuint64_t)B};
   cuuint64_t strides[3] = {(cuuint64_t)sn * 2, (cuuint64_t)sh * 2, (cuuint64_t)sb * 2};
-  cuuint32_t box[4] = {64, 128, 1, 1};
+  cuuint32_t box[4] = {64, (cuuint32_t)box_rows, 1, 1};
   cuuint32_t estr[4] = {1, 1, 1, 1};
   CUresult r = fn(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, const_cast<void*>(base), dims, strides, box, estr,
                   CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
