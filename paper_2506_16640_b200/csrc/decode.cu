@@ -2,9 +2,9 @@
 // different lengths in one batch.  Query t of sequence b sits at position pos = kv_len[b] - q_len + t,
 // sees the keys j <= pos, and gets Eq. 1 on its ASEntmax-scaled logits like any row of the full problem
 // (n_i = pos + 1).  The path is bound by reading K once from HBM:
-//   decode_scale_kernel       a_t = (alpha-1) c_t sm_scale per (sequence, head, query), c_t in fp64;
 //   decode_scores_tc_kernel   (decode_scores_sm100.cu) streams K through TMA and tcgen05, writes
-//                             y = a_t (q.k + bias) to a score row in the workspace and the maximum of every chunk;
+//                             y = a_t (q.k + bias), a_t = (alpha-1) c_t sm_scale, to a score row in the
+//                             workspace and the maximum of every chunk of keys;
 //   decode_solve_kernel       one CTA per query row: y_max, the candidates above the lower end of the bracket
 //                             of App. A (tau >= y_max - 1), Newton from the left on them (e-norm step), then
 //                             p = [y - tau]_+^e and O = sum_j p_j v_j as a gather of the support's V rows.
@@ -18,27 +18,8 @@ namespace entmax {
 
 namespace {
 
-constexpr int kSolveThreads = 256;
-constexpr int kPerThread = 8;      // candidate slots per thread of the solve kernel
+constexpr int kListSlots = 2048;   // candidate slots of a solve CTA, split evenly among its threads
 constexpr int kMaxNewtonD = 64;
-
-// a_t = (alpha-1) * c_t * sm_scale with c_t = delta + beta (ln n)^gamma in fp64 (c_t = delta for n = 1; 1 without scale)
-__global__ void decode_scale_kernel(DecodeArgs a, const float* __restrict__ beta, const float* __restrict__ gamma,
-                                    const float* __restrict__ delta, float* __restrict__ a_table,
-                                    int32_t* __restrict__ status) {
-  const int idx = blockIdx.x * blockDim.x + threadIdx.x;
-  if (idx >= a.B * a.H * a.QL) return;
-  const int t = idx % a.QL, bh = idx / a.QL, h = bh % a.H, b = bh / a.H;
-  float c = 1.0f;
-  if (beta) {
-    const long n = (long)seq_len(a, b, status) - a.QL + t + 1;
-    double cd = (double)delta[h];
-    if (n > 1) cd += (double)beta[h] * pow(log((double)n), (double)gamma[h]);
-    c = (float)cd;
-    if (!isfinite(c) && status) atomicOr(status + ENTMAX_ATTN_STATUS_FLAGS, ENTMAX_ATTN_FLAG_BAD_SCALE);
-  }
-  a_table[idx] = a.alpha_m1 * (c * a.sm_scale);
-}
 
 // PER consecutive bf16 values (PER = 2 or 4) as floats
 template <int PER>
@@ -55,18 +36,35 @@ __device__ __forceinline__ void load_bf16_row(const __nv_bfloat16* p, float (&f)
 
 // Sum over the CTA in a fixed order; every thread returns the same value.  `slot` alternates between
 // calls so that one barrier per call is enough.
-__device__ __forceinline__ float block_sum(float x, float (*red)[kSolveThreads / 32], int slot) {
+template <int kSolveThreads>
+__device__ __forceinline__ float2 block_sum2(float x, float y, float2 (*red)[kSolveThreads / 32], int slot) {
 #pragma unroll
-  for (int o = 16; o > 0; o >>= 1) x += __shfl_xor_sync(0xffffffffu, x, o);
-  if ((threadIdx.x & 31) == 0) red[slot][threadIdx.x >> 5] = x;
+  for (int o = 16; o > 0; o >>= 1) {
+    x += __shfl_xor_sync(0xffffffffu, x, o);
+    y += __shfl_xor_sync(0xffffffffu, y, o);
+  }
+  if ((threadIdx.x & 31) == 0) red[slot][threadIdx.x >> 5] = make_float2(x, y);
   __syncthreads();
-  float s = 0.f;
+  float2 s = make_float2(0.f, 0.f);
 #pragma unroll
-  for (int w = 0; w < kSolveThreads / 32; ++w) s += red[slot][w];
+  for (int w = 0; w < kSolveThreads / 32; ++w) {
+    s.x += red[slot][w].x;
+    s.y += red[slot][w].y;
+  }
   return s;
 }
 
-template <int D>
+// One Newton step from the left with the e-norm step; returns false when the iteration has converged.
+__device__ __forceinline__ bool newton_update(float s0, float s1, const DecodeArgs& a, float& tau) {
+  if (!(s0 > 1.0f) || !(s1 > 0.f)) return false;
+  const float step = threshold_step(s0, s1, a.expo_class, a.expo);
+  const float next = tau + step;
+  if (!(next > tau)) return false;
+  tau = next;
+  return step > 1e-7f * fmaxf(1.0f, fabsf(tau));
+}
+
+template <int D, int kSolveThreads>
 __global__ void __launch_bounds__(kSolveThreads) decode_solve_kernel(DecodeArgs a, const __nv_bfloat16* __restrict__ v,
                                                                     const float* __restrict__ scores,
                                                                     const float* __restrict__ chunk_max,
@@ -75,15 +73,20 @@ __global__ void __launch_bounds__(kSolveThreads) decode_solve_kernel(DecodeArgs 
                                                                     int32_t* __restrict__ support_out,
                                                                     int32_t* __restrict__ status) {
   constexpr int kWarps = kSolveThreads / 32;
+  constexpr int kPerThread = kListSlots / kSolveThreads;
+  constexpr int kCap = kListSlots;
   constexpr int PER = D / 32;
-  __shared__ float cand_y[kSolveThreads * kPerThread];
-  __shared__ int cand_j[kSolveThreads * kPerThread];
-  __shared__ float supp_p[kSolveThreads * kPerThread];
-  __shared__ int supp_j[kSolveThreads * kPerThread];
-  __shared__ float red[4][kWarps];
+  __shared__ float cand_y[kCap];      // per-thread slots, then the compact list's p values
+  __shared__ int cand_j[kCap];
+  __shared__ float list_y[kCap];      // candidates compacted in (thread, slot) order
+  __shared__ int list_j[kCap];
+  __shared__ float2 red[2][kWarps];
+  __shared__ float wmax[kWarps];
   __shared__ int scan[kWarps];
   __shared__ float opart[kWarps][D];
   __shared__ int s_overflow;
+  __shared__ float s_tau;
+  __shared__ int s_support;
   const int row = blockIdx.x;                       // (b * H + h) * QL + t
   const int t = row % a.QL, bh = row / a.QL, h = bh % a.H, b = bh / a.H;
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
@@ -97,28 +100,28 @@ __global__ void __launch_bounds__(kSolveThreads) decode_solve_kernel(DecodeArgs 
   for (int c = tid; c < chunks; c += kSolveThreads) m = fmaxf(m, chunk_max[(size_t)row * a.n_chunks + c]);
 #pragma unroll
   for (int off = 16; off > 0; off >>= 1) m = fmaxf(m, __shfl_xor_sync(0xffffffffu, m, off));
-  if (lane == 0) red[3][warp] = m;
+  if (lane == 0) wmax[warp] = m;
   __syncthreads();
-  float ymax = red[3][0];
+  float ymax = wmax[0];
 #pragma unroll
-  for (int w = 1; w < kWarps; ++w) ymax = fmaxf(ymax, red[3][w]);
+  for (int w = 1; w < kWarps; ++w) ymax = fmaxf(ymax, wmax[w]);
   // ---- candidates: y > y_max - 1 (App. A: tau >= y_max - 1), kept per thread in key order
   const float floor_y = ymax - 1.0f;
   int cnt = 0;
   {
-    // four 16-byte loads in flight per thread; a thread meets its keys in increasing order
+    // eight 16-byte loads in flight per thread; a thread meets its keys in increasing order
     const float4* y_row4 = reinterpret_cast<const float4*>(y_row);
     const int groups = (nv + 3) / 4;
     const float4 none = make_float4(-INFINITY, -INFINITY, -INFINITY, -INFINITY);
-    for (int g0 = tid; g0 < groups; g0 += 4 * kSolveThreads) {
-      float4 yv[4];
+    for (int g0 = tid; g0 < groups; g0 += 8 * kSolveThreads) {
+      float4 yv[8];
 #pragma unroll
-      for (int u = 0; u < 4; ++u) {
+      for (int u = 0; u < 8; ++u) {
         const int g = g0 + u * kSolveThreads;
         yv[u] = g < groups ? y_row4[g] : none;
       }
 #pragma unroll
-      for (int u = 0; u < 4; ++u) {
+      for (int u = 0; u < 8; ++u) {
         const float ye[4] = {yv[u].x, yv[u].y, yv[u].z, yv[u].w};
 #pragma unroll
         for (int e = 0; e < 4; ++e) {
@@ -135,24 +138,79 @@ __global__ void __launch_bounds__(kSolveThreads) decode_solve_kernel(DecodeArgs 
     }
   }
   if (cnt > kPerThread) s_overflow = 1;
+  // ---- compact the candidates in (thread, slot) order
+  int incl = cnt < kPerThread ? cnt : kPerThread;
+  const int mine = incl;
+#pragma unroll
+  for (int off = 1; off < 32; off <<= 1) {
+    const int up = __shfl_up_sync(0xffffffffu, incl, off);
+    if (lane >= off) incl += up;
+  }
+  if (lane == 31) scan[warp] = incl;
   __syncthreads();
   const bool dense = s_overflow != 0;
+  int base = 0, n_cand = 0;
+  for (int w = 0; w < kWarps; ++w) {
+    if (w < warp) base += scan[w];
+    n_cand += scan[w];
+  }
+  if (!dense) {
+    const int at = base + incl - mine;
+    for (int c = 0; c < mine; ++c) {
+      list_y[at + c] = cand_y[tid * kPerThread + c];
+      list_j[at + c] = cand_j[tid * kPerThread + c];
+    }
+  }
+  __syncthreads();
   if (dense && tid == 0 && status) atomicAdd(status + ENTMAX_ATTN_STATUS_DENSE_ROWS, 1);
   // ---- Newton from the left on f(tau) = sum [y - tau]_+^e - 1, e-norm step
   float tau = floor_y;
-  for (int it = 0; it < kMaxNewtonD; ++it) {
-    float s0 = 0.f, s1 = 0.f;
-    if (!dense) {
-      for (int c = 0; c < cnt; ++c) {
-        const float d = cand_y[tid * kPerThread + c] - tau;
-        if (d > 0.f) {
-          float ye, ye1;
-          pow_pair(d, a.expo_class, a.expo, ye, ye1);
-          s0 += ye;
-          s1 += ye1;
+  int support = 0;
+  if (!dense) {
+    // the first warp alone: shuffles only, no CTA barriers inside the iteration
+    if (warp == 0) {
+      for (int it = 0; it < kMaxNewtonD; ++it) {
+        float s0 = 0.f, s1 = 0.f;
+        for (int c = lane; c < n_cand; c += 32) {
+          const float d = list_y[c] - tau;
+          if (d > 0.f) {
+            float ye, ye1;
+            pow_pair(d, a.expo_class, a.expo, ye, ye1);
+            s0 += ye;
+            s1 += ye1;
+          }
         }
+#pragma unroll
+        for (int off = 16; off > 0; off >>= 1) {
+          s0 += __shfl_xor_sync(0xffffffffu, s0, off);
+          s1 += __shfl_xor_sync(0xffffffffu, s1, off);
+        }
+        if (!newton_update(s0, s1, a, tau)) break;
       }
-    } else {
+      // p of every candidate (0 outside the support), in list order
+      int local = 0;
+      for (int c = lane; c < n_cand; c += 32) {
+        const float d = list_y[c] - tau;
+        float ye = 0.f, ye1;
+        if (d > 0.f) {
+          pow_pair(d, a.expo_class, a.expo, ye, ye1);
+          ++local;
+        }
+        cand_y[c] = ye;
+      }
+#pragma unroll
+      for (int off = 16; off > 0; off >>= 1) local += __shfl_xor_sync(0xffffffffu, local, off);
+      if (lane == 0) {
+        s_tau = tau;
+        s_support = local;
+      }
+    }
+    __syncthreads();
+    tau = s_tau;
+    support = s_support;
+  } else {
+    for (int it = 0; it < kMaxNewtonD; ++it) {
+      float s0 = 0.f, s1 = 0.f;
       for (int j = tid; j < nv; j += kSolveThreads) {
         const float d = y_row[j] - tau;
         if (d > 0.f) {
@@ -162,58 +220,25 @@ __global__ void __launch_bounds__(kSolveThreads) decode_solve_kernel(DecodeArgs 
           s1 += ye1;
         }
       }
+      const float2 s = block_sum2<kSolveThreads>(s0, s1, red, it & 1);
+      if (!newton_update(s.x, s.y, a, tau)) break;
     }
-    s0 = block_sum(s0, red, it & 1);
-    s1 = block_sum(s1, red, 2 + (it & 1));
-    if (!(s0 > 1.0f) || !(s1 > 0.f)) break;
-    const float step = threshold_step(s0, s1, a.expo_class, a.expo);
-    const float next = tau + step;
-    if (!(next > tau)) break;
-    tau = next;
-    if (step <= 1e-7f * fmaxf(1.0f, fabsf(tau))) break;
+    __syncthreads();
   }
-  __syncthreads();
   // ---- O = sum_j p_j v_j
   const __nv_bfloat16* vbase = v + (size_t)b * a.ksb + (size_t)h * a.ksh + lane * PER;
   float acc[PER];
 #pragma unroll
   for (int e = 0; e < PER; ++e) acc[e] = 0.f;
-  int support = 0;
   if (!dense) {
-    // compact the support in (thread, slot) order
-    int mine = 0;
-    for (int c = 0; c < cnt; ++c) mine += cand_y[tid * kPerThread + c] > tau ? 1 : 0;
-    int incl = mine;
+    for (int c = warp; c < n_cand; c += kWarps) {
+      const float p = cand_y[c];
+      if (p > 0.f) {
+        float vf[PER];
+        load_bf16_row<PER>(vbase + (size_t)list_j[c] * a.ksn, vf);
 #pragma unroll
-    for (int off = 1; off < 32; off <<= 1) {
-      const int up = __shfl_up_sync(0xffffffffu, incl, off);
-      if (lane >= off) incl += up;
-    }
-    if (lane == 31) scan[warp] = incl;
-    __syncthreads();
-    int base = 0;
-    for (int w = 0; w < kWarps; ++w) {
-      if (w < warp) base += scan[w];
-      support += scan[w];
-    }
-    int at = base + incl - mine;
-    for (int c = 0; c < cnt; ++c) {
-      const float d = cand_y[tid * kPerThread + c] - tau;
-      if (d > 0.f) {
-        float ye, ye1;
-        pow_pair(d, a.expo_class, a.expo, ye, ye1);
-        supp_p[at] = ye;
-        supp_j[at] = cand_j[tid * kPerThread + c];
-        ++at;
+        for (int e = 0; e < PER; ++e) acc[e] = fmaf(p, vf[e], acc[e]);
       }
-    }
-    __syncthreads();
-    for (int s = warp; s < support; s += kWarps) {
-      const float p = supp_p[s];
-      float vf[PER];
-      load_bf16_row<PER>(vbase + (size_t)supp_j[s] * a.ksn, vf);
-#pragma unroll
-      for (int e = 0; e < PER; ++e) acc[e] = fmaf(p, vf[e], acc[e]);
     }
   } else {
     int local = 0;
@@ -249,7 +274,7 @@ __global__ void __launch_bounds__(kSolveThreads) decode_solve_kernel(DecodeArgs 
 }
 
 struct DecodeLayout {
-  size_t a_table, chunk_max, scores, total;
+  size_t chunk_max, scores, total;
   size_t score_stride;
   int chunk_keys, n_chunks;
 };
@@ -264,7 +289,6 @@ DecodeLayout decode_layout(int B, int H, int QL, int NC) {
   l.score_stride = ((size_t)NC + 31) / 32 * 32;
   size_t off = 0;
   auto take = [&off](size_t bytes) { size_t at = off; off = (off + bytes + 255) / 256 * 256; return at; };
-  l.a_table = take(rows * sizeof(float));
   l.chunk_max = take(rows * l.n_chunks * sizeof(float));
   l.scores = take(rows * l.score_stride * sizeof(float));
   l.total = off;
@@ -328,6 +352,7 @@ extern "C" int entmax_attn_decode_fwd(const entmax_attn_decode_params* params, c
   if (!workspace || !aligned(workspace, 256) || workspace_bytes < lay.total) return ENTMAX_ATTN_EINVAL_WORKSPACE;
   a.kv_len = kv_len;
   a.alibi = alibi_slopes;
+  a.beta = beta; a.gamma = gamma; a.delta = delta;
   a.chunk_keys = lay.chunk_keys;
   a.n_chunks = lay.n_chunks;
   a.score_stride = lay.score_stride;
@@ -337,7 +362,6 @@ extern "C" int entmax_attn_decode_fwd(const entmax_attn_decode_params* params, c
   if (major != 10) return ENTMAX_ATTN_EUNSUPPORTED;          // the score kernel needs tcgen05 / TMA
   cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
   uint8_t* ws = static_cast<uint8_t*>(workspace);
-  float* a_table = reinterpret_cast<float*>(ws + lay.a_table);
   float* chunk_max = reinterpret_cast<float*>(ws + lay.chunk_max);
   float* scores = reinterpret_cast<float*>(ws + lay.scores);
   cudaError_t err;
@@ -346,17 +370,19 @@ extern "C" int entmax_attn_decode_fwd(const entmax_attn_decode_params* params, c
     if (err != cudaSuccess) return ENTMAX_ATTN_ECUDA;
   }
   const int rows = a.B * a.H * a.QL;
-  decode_scale_kernel<<<(rows + 127) / 128, 128, 0, stream>>>(a, beta, gamma, delta, a_table, device_status);
-  err = cudaGetLastError();
-  if (err != cudaSuccess) return ENTMAX_ATTN_ECUDA;
-  err = launch_decode_scores_tc(a, q, k, a_table, scores, chunk_max, device_status, stream);
+  err = launch_decode_scores_tc(a, q, k, scores, chunk_max, device_status, stream);
   if (err != cudaSuccess) return ENTMAX_ATTN_ECUDA;
   const __nv_bfloat16* vb = static_cast<const __nv_bfloat16*>(v);
   __nv_bfloat16* ob = static_cast<__nv_bfloat16*>(o);
-  if (a.D == 64)
-    decode_solve_kernel<64><<<rows, kSolveThreads, 0, stream>>>(a, vb, scores, chunk_max, ob, tau, support_size, device_status);
-  else
-    decode_solve_kernel<128><<<rows, kSolveThreads, 0, stream>>>(a, vb, scores, chunk_max, ob, tau, support_size, device_status);
+  // long rows: more threads per row (more loads in flight); many short rows: smaller CTAs
+#define ENTMAX_SOLVE(D, T) \
+  decode_solve_kernel<D, T><<<rows, T, 0, stream>>>(a, vb, scores, chunk_max, ob, tau, support_size, device_status)
+  if (a.NC >= 16384) {
+    if (a.D == 64) ENTMAX_SOLVE(64, 512); else ENTMAX_SOLVE(128, 512);
+  } else {
+    if (a.D == 64) ENTMAX_SOLVE(64, 256); else ENTMAX_SOLVE(128, 256);
+  }
+#undef ENTMAX_SOLVE
   err = cudaGetLastError();
   return err == cudaSuccess ? ENTMAX_ATTN_OK : ENTMAX_ATTN_ECUDA;
 }

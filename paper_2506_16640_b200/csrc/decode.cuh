@@ -12,6 +12,7 @@ struct DecodeArgs {
   int64_t ksb, ksh, ksn;           // element strides of K and V
   const int32_t* kv_len;           // [B] or nullptr
   const float* alibi;              // [H] or nullptr
+  const float *beta, *gamma, *delta;   // [H] each, or all nullptr (c = 1)
   int chunk_keys;                  // keys per chunk maximum (a multiple of 128)
   int n_chunks;
   size_t score_stride;             // floats per score row
@@ -28,7 +29,7 @@ __device__ __forceinline__ int seq_len(const DecodeArgs& a, int b, int32_t* stat
 
 // Score stream on the tensor cores: K tiles of 128 keys as the M side of tcgen05 MMAs against the (zero-padded)
 // query rows, one thread per key afterwards.  Writes the score rows and the chunk maxima.
-cudaError_t launch_decode_scores_tc(const DecodeArgs& a, const void* q, const void* k, const float* a_table,
-                                    float* scores, float* chunk_max, int32_t* status, cudaStream_t stream);
+cudaError_t launch_decode_scores_tc(const DecodeArgs& a, const void* q, const void* k, float* scores, float* chunk_max,
+                                    int32_t* status, cudaStream_t stream);
 
 }  // namespace entmax

@@ -43,7 +43,6 @@ template <int HD>
 __global__ void __launch_bounds__(kThreadsD, 2) decode_scores_tc_kernel(const __grid_constant__ CUtensorMap map_q,
                                                                        const __grid_constant__ CUtensorMap map_k,
                                                                        const DecodeArgs a,
-                                                                       const float* __restrict__ a_table,
                                                                        float* __restrict__ scores,
                                                                        float* __restrict__ chunk_max,
                                                                        int32_t* __restrict__ status) {
@@ -147,10 +146,23 @@ __global__ void __launch_bounds__(kThreadsD, 2) decode_scores_tc_kernel(const __
     const int bh = b * a.H + h;
     const int pos0 = len - a.QL;                                   // position of query 0
     const float slope = a.alibi ? a.alibi[h] / a.sm_scale : 0.f;   // bias in dot-product units
+    // a_t = (alpha-1) c_t sm_scale with c_t = delta + beta (ln n_t)^gamma, n_t = pos_t + 1 (c_t = delta for
+    // n_t = 1; 1 without scale parameters): lane t evaluates it in fp32 and the warp shares the values
+    float a_lane = 0.f;
+    if (lane < a.QL) {
+      float c = 1.0f;
+      if (a.beta) {
+        const int n = pos0 + lane + 1;
+        c = a.delta[h];
+        if (n > 1) c += a.beta[h] * powf(logf((float)n), a.gamma[h]);
+        if (!isfinite(c) && status) atomicOr(status + ENTMAX_ATTN_STATUS_FLAGS, ENTMAX_ATTN_FLAG_BAD_SCALE);
+      }
+      a_lane = a.alpha_m1 * (c * a.sm_scale);
+    }
     float at[ENTMAX_ATTN_DECODE_MAX_Q], vmax[ENTMAX_ATTN_DECODE_MAX_Q];
 #pragma unroll
     for (int t = 0; t < ENTMAX_ATTN_DECODE_MAX_Q; ++t) {
-      at[t] = t < a.QL ? a_table[bh * a.QL + t] : 0.f;
+      at[t] = __shfl_sync(0xffffffffu, a_lane, t);
       vmax[t] = -INFINITY;
     }
     uint32_t sphase[2] = {0, 0};
@@ -212,8 +224,8 @@ __global__ void __launch_bounds__(kThreadsD, 2) decode_scores_tc_kernel(const __
 }
 
 template <int HD>
-cudaError_t launch_impl(const DecodeArgs& a, const void* q, const void* k, const float* a_table, float* scores,
-                        float* chunk_max, int32_t* status, cudaStream_t stream) {
+cudaError_t launch_impl(const DecodeArgs& a, const void* q, const void* k, float* scores, float* chunk_max,
+                        int32_t* status, cudaStream_t stream) {
   CUtensorMap map_q, map_k;
   cudaError_t err = make_tile_map(&map_q, q, a.D, a.QL, a.H, a.B, a.D, (int64_t)a.QL * a.D, (int64_t)a.H * a.QL * a.D, kQPad);
   if (err != cudaSuccess) return err;
@@ -222,17 +234,17 @@ cudaError_t launch_impl(const DecodeArgs& a, const void* q, const void* k, const
   err = cudaFuncSetAttribute(decode_scores_tc_kernel<HD>, cudaFuncAttributeMaxDynamicSharedMemorySize, DCfg<HD>::kSmemBytes);
   if (err != cudaSuccess) return err;
   const dim3 grid(a.n_chunks, a.H, a.B);
-  decode_scores_tc_kernel<HD><<<grid, kThreadsD, DCfg<HD>::kSmemBytes, stream>>>(map_q, map_k, a, a_table, scores,
-                                                                                chunk_max, status);
+  decode_scores_tc_kernel<HD><<<grid, kThreadsD, DCfg<HD>::kSmemBytes, stream>>>(map_q, map_k, a, scores, chunk_max,
+                                                                                status);
   return cudaGetLastError();
 }
 
 }  // namespace
 
-cudaError_t launch_decode_scores_tc(const DecodeArgs& a, const void* q, const void* k, const float* a_table,
-                                    float* scores, float* chunk_max, int32_t* status, cudaStream_t stream) {
-  return a.D == 64 ? launch_impl<64>(a, q, k, a_table, scores, chunk_max, status, stream)
-                   : launch_impl<128>(a, q, k, a_table, scores, chunk_max, status, stream);
+cudaError_t launch_decode_scores_tc(const DecodeArgs& a, const void* q, const void* k, float* scores, float* chunk_max,
+                                    int32_t* status, cudaStream_t stream) {
+  return a.D == 64 ? launch_impl<64>(a, q, k, scores, chunk_max, status, stream)
+                   : launch_impl<128>(a, q, k, scores, chunk_max, status, stream);
 }
 
 }  // namespace entmax

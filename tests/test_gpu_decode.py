@@ -118,7 +118,7 @@ def test_decode_dense_rows_are_solved_on_the_score_row(alpha):
     lens = _lengths(1, 5000, 4, 0, False)
     got = _run(inp, lens, 4, alpha)
     assert int(got["status"][binding.STATUS_DENSE_ROWS]) == 2 * 4
-    assert int(got["supp"].min()) > 256 * 8
+    assert int(got["supp"].min()) > 2048
     _check(inp, lens, 4, alpha, got)
 
 
