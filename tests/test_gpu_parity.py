@@ -422,6 +422,22 @@ def test_cfg5_noncausal_retrieval():
     _gradient_invariants(inp, bwd)
 
 
+def test_long_sequences_with_byte_offsets_beyond_32_bits():
+    # 18 heads x 131072 rows: 2.36 M rows, so the candidate lists span 4.8 GB and the row index times the list pitch
+    # no longer fits 32 bits; the longest sequence any test runs.  Sampled rows of three heads, forward and dQ.
+    inp = make_inputs(Workload("long_rows", 1, 18, 131072, 64, "bf16", True, (1.5,), backward=True, seed_offset=77))
+    w = inp.workload
+    got = parity.run_fwd(inp, 1.5)
+    bwd = parity.run_bwd(inp, 1.5, got["tau"], got["dev"])
+    for bh in (0, 9, 17):
+        rows = sample_rows(inp, bh, 48)
+        parity.check_fwd_rows(inp, 1.5, got, bh, rows)
+        parity.check_bwd_rows(inp, 1.5, bwd, bh, rows)
+    _gradient_invariants(inp, bwd)
+    del got, bwd
+    torch.cuda.empty_cache()
+
+
 def test_cfg5_shape_reduced_full_backward():
     # same recipe at N = 4096 so that dK and dV of a whole head can be checked against the oracle
     inp = make_inputs(scaled(WORKLOADS[5], N=4096, H=2, name="cfg5_reduced"))
