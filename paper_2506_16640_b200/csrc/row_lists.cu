@@ -1,11 +1,11 @@
 // Per-row kernels of the bf16 path that work on the sparse candidate lists left by the tensor-core
-// score sweep (two half-lists per row, see common.cuh).  A warp takes four consecutive query rows: when
-// all four have at most eight list entries (the common case on sparse rows) eight lanes work on each
-// row at the same time, otherwise the warp takes the rows one after the other with all 32 lanes.
+// score sweep (two half-lists per row, see common.cuh).
 //
-// Forward: exact threshold on the candidates (Eq. 1 with the sum-to-one condition; Newton from the
-// left of the root, see dense_rows.cu), probabilities, and O_i = sum_j p_ij v_j as a gather over the
-// support only -- every zero of P is skipped, not just all-zero tiles.
+// Forward: exact threshold on the candidates (Eq. 1 with the sum-to-one condition), probabilities, and
+// O_i = sum_j p_ij v_j as a gather over the support only -- every zero of P is skipped, not just
+// all-zero tiles.  A warp takes 16 consecutive rows and serves them by list length (8, 16 or 32 lanes per
+// row).  alpha = 1.5 and alpha = 2 use the closed form on the sorted candidates (solve_rows_closed); other
+// exponents iterate (Newton from the left of the root, see dense_rows.cu) in two stages.
 // Backward: the entmax Jacobian dS = u (dP - <u,dP>/sum u), u = p^(2-alpha), on the support, dQ by
 // gathering K rows, dK / dV by vector atomics into fp32 accumulators.
 #include "common.cuh"
@@ -75,6 +75,19 @@ __device__ __forceinline__ float oct_max(float x) {
   x = fmaxf(x, __shfl_xor_sync(0xffffffffu, x, 1));
   x = fmaxf(x, __shfl_xor_sync(0xffffffffu, x, 2));
   x = fmaxf(x, __shfl_xor_sync(0xffffffffu, x, 4));
+  return x;
+}
+// reductions over aligned groups of W lanes (W = 8 or 16); the sum takes ascending strides like warp_sum
+template <int W>
+__device__ __forceinline__ float sub_sum(float x) {
+#pragma unroll
+  for (int o = 1; o < W; o <<= 1) x += __shfl_xor_sync(0xffffffffu, x, o);
+  return x;
+}
+template <int W>
+__device__ __forceinline__ float sub_max(float x) {
+#pragma unroll
+  for (int o = 1; o < W; o <<= 1) x = fmaxf(x, __shfl_xor_sync(0xffffffffu, x, o));
   return x;
 }
 // N consecutive bf16 (N = 8 or 16, 16-byte aligned) <-> floats
@@ -313,13 +326,14 @@ __device__ __forceinline__ void solve_row_full(const Problem& p, const __nv_bflo
   else finish_row<D, kSlots>(p, vbase, list, kept, o_row, tau_slot, cnt_slot, lane);
 }
 
-// Newton for four rows at once (eight lanes per row); `done` rows keep their tau.
-__device__ __forceinline__ float newton_oct(const Problem& p, float y, float tau, bool done) {
+// Newton for 32 / W rows at once (W lanes per row); `done` rows keep their tau.
+template <int W>
+__device__ __forceinline__ float newton_sub(const Problem& p, float y, float tau, bool done) {
   for (int it = 0; it < kMaxNewton; ++it) {
     const float d = y - tau;
     float ye = 0.f, ye1 = 0.f;
     if (d > 0.f) pow_pair(d, p.expo_class, p.expo, ye, ye1);
-    const float s0 = oct_sum(ye), s1 = oct_sum(ye1);
+    const float s0 = sub_sum<W>(ye), s1 = sub_sum<W>(ye1);
     if (!done) {
       if (!(s0 > 1.0f) || !(s1 > 0.f)) {
         done = true;
@@ -339,16 +353,16 @@ __device__ __forceinline__ float newton_oct(const Problem& p, float y, float tau
   return tau;
 }
 
-// Four rows at once, eight lanes per row, for rows with 1..8 list entries; same two stages.
-template <int D>
-__device__ __forceinline__ void solve_rows_quad(const Problem& p, const __nv_bfloat16* __restrict__ v,
+// 32 / W rows at once, W lanes per row (W = 8 or 16), for rows with 1..W list entries; same two stages.
+template <int D, int W>
+__device__ __forceinline__ void solve_rows_sub(const Problem& p, const __nv_bfloat16* __restrict__ v,
                                                 const float* __restrict__ scale, Entry* __restrict__ entries,
                                                 __nv_bfloat16* __restrict__ o, float* __restrict__ tau_out,
                                                 int32_t* __restrict__ row_cnt, int grow, bool active, int c0, int c1,
                                                 int lane) {
-  constexpr int PL = D / 8;                        // elements of a V / O row per lane
-  const int sl = lane & 7;
-  const int base = lane & 24;
+  constexpr int PL = D / W;                        // elements of a V / O row per lane
+  const int sl = lane & (W - 1);
+  const int base = lane & (32 - W);
   const int n = active ? c0 + c1 : 0;
   const int bh = grow / p.N, i = grow - bh * p.N, b = bh / p.H, h = bh - b * p.H;
   const float a = active ? (p.alpha - 1.0f) * (scale[(size_t)b * p.scale_sb + (size_t)h * p.N + i] * p.sm_scale) : 1.0f;
@@ -362,14 +376,14 @@ __device__ __forceinline__ void solve_rows_quad(const Problem& p, const __nv_bfl
   }
   __syncwarp();   // every entry is in registers before the compaction below overwrites the lists
   // stage A
-  const float tau_a = newton_oct(p, y, oct_max(y) - 1.0f, !active);
+  const float tau_a = newton_sub<W>(p, y, sub_max<W>(y) - 1.0f, !active);
   const bool keep = active && y > tau_a - kKeepMargin * fmaxf(1.0f, fabsf(tau_a));
   // keep only those: they move to the end-stable front when sorted with the others' keys pushed to infinity
   j = keep ? j : 0x7fffffff;
   y = keep ? y : -INFINITY;
-  // bitonic sort of the eight (j, y) pairs of each row, ascending by key index
+  // bitonic sort of the W (j, y) pairs of each row, ascending by key index
 #pragma unroll
-  for (int k = 2; k <= 8; k <<= 1) {
+  for (int k = 2; k <= W; k <<= 1) {
 #pragma unroll
     for (int st = k >> 1; st > 0; st >>= 1) {
       const int oj = __shfl_xor_sync(0xffffffffu, j, st);
@@ -382,13 +396,13 @@ __device__ __forceinline__ void solve_rows_quad(const Problem& p, const __nv_bfl
     }
   }
   // stage B
-  const float tau = newton_oct(p, y, oct_max(y) - 1.0f, !active);
+  const float tau = newton_sub<W>(p, y, sub_max<W>(y) - 1.0f, !active);
   const float d = y - tau;
   const bool in = active && d > 0.f;
   float pe = 0.f, pe1;
   if (in) pow_pair(d, p.expo_class, p.expo, pe, pe1);
   const unsigned m = __ballot_sync(0xffffffffu, in);
-  const unsigned msub = (m >> base) & 0xffu;
+  const unsigned msub = (m >> base) & ((1u << W) - 1u);
   if (in) {
     // compact the list to the exact support, y in Eq. 1's units
     const int pos = __popc(msub & ((1u << sl) - 1u));
@@ -400,23 +414,137 @@ __device__ __forceinline__ void solve_rows_quad(const Problem& p, const __nv_bfl
   for (int t = 0; t < PL; ++t) acc[t] = 0.f;
   const __nv_bfloat16* vbase = v + (size_t)b * p.sb + (size_t)h * p.sh + sl * PL;
 #pragma unroll
-  for (int t = 0; t < 8; ++t) {
+  for (int t = 0; t < W; ++t) {
     const bool has = (msub >> t) & 1u;
     if (!__any_sync(0xffffffffu, has)) continue;
     const float pj = __shfl_sync(0xffffffffu, pe, base + t);
     const int kj = __shfl_sync(0xffffffffu, j, base + t);
     if (has) {
       float vs[PL];
-      load_bf16_vec<PL>(vbase + (size_t)kj * p.sn, vs);
+      if constexpr (PL >= 8) load_bf16_vec<PL>(vbase + (size_t)kj * p.sn, vs);
+      else load_bf16<PL>(vbase + (size_t)kj * p.sn, vs);
 #pragma unroll
       for (int u = 0; u < PL; ++u) acc[u] = fmaf(pj, vs[u], acc[u]);
     }
   }
   if (active) {
-    store_bf16_vec<PL>(o + (size_t)b * p.sb + (size_t)h * p.sh + (size_t)i * p.sn + sl * PL, acc);
+    __nv_bfloat16* o_row = o + (size_t)b * p.sb + (size_t)h * p.sh + (size_t)i * p.sn + sl * PL;
+    if constexpr (PL >= 8) store_bf16_vec<PL>(o_row, acc);
+    else store_bf16<PL>(o_row, acc);
     if (sl == 0) {
       tau_out[grow] = tau;
       row_cnt[grow] = __popc(msub);
+    }
+  }
+}
+
+// Closed-form row solve for e = 2 (alpha = 1.5) and e = 1 (alpha = 2), 32 / W rows at once with W lanes per row
+// (W = 8, 16 or 32) and at most W list entries per row.  With the entries sorted by decreasing y and
+// u_j = y_max - y_j, the threshold that makes the top k sum to one is, in units below the maximum,
+//   e = 2:  t_k = (U1 + sqrt(U1^2 - k (U2 - 1))) / k      (the root of sum_{j<=k} (t - u_j)^2 = 1 with t >= u_k)
+//   e = 1:  t_k = (1 + U1) / k                             (sum_{j<=k} (t - u_j) = 1)
+// with U1, U2 the prefix sums of u and u^2; the support size k* is the number of k with u_k < t_k (they form a
+// prefix) and tau = y_max - t_{k*} -- Eq. 1's threshold without iterating.  Only the top k* entries enter the
+// result, so candidates outside the support, which differ from run to run, do not change a bit of it.
+// `prescaled`: the list already holds y in Eq. 1's units from slot 0 (c1 = 0).
+template <int D, int W, int EC>
+__device__ __forceinline__ void solve_rows_closed(const Problem& p, const __nv_bfloat16* __restrict__ v,
+                                                  const float* __restrict__ scale, Entry* __restrict__ entries,
+                                                  __nv_bfloat16* __restrict__ o, float* __restrict__ tau_out,
+                                                  int32_t* __restrict__ row_cnt, int grow, bool active, int c0, int c1,
+                                                  bool prescaled, int lane) {
+  static_assert(EC == kExpo2 || EC == kExpo1, "closed forms exist for e = 2 and e = 1");
+  constexpr int PL = D / W;                        // elements of a V / O row per lane
+  constexpr unsigned kWMask = W == 32 ? 0xffffffffu : ((1u << (W & 31)) - 1u);
+  const int sl = lane & (W - 1);
+  const int base = lane & (32 - W);
+  const int n = active ? c0 + c1 : 0;
+  const int bh = grow / p.N, i = grow - bh * p.N, b = bh / p.H, h = bh - b * p.H;
+  const float a = (active && !prescaled)
+                      ? (p.alpha - 1.0f) * (scale[(size_t)b * p.scale_sb + (size_t)h * p.N + i] * p.sm_scale) : 1.0f;
+  Entry* list = entries + (size_t)grow * kListCap;
+  float y = -INFINITY;
+  int j = 0x7fffffff;
+  if (sl < n) {
+    const Entry en = list[sl < c0 ? sl : kHalfCap + sl - c0];
+    y = a * en.y;
+    j = en.j;
+  }
+  __syncwarp();   // every entry is in registers before the compaction below overwrites the lists
+  const float ymax = sub_max<W>(y);
+  // bitonic sort of the W (y, j) pairs of each row: decreasing y, equal values by increasing key index
+#pragma unroll
+  for (int k = 2; k <= W; k <<= 1) {
+#pragma unroll
+    for (int st = k >> 1; st > 0; st >>= 1) {
+      const int oj = __shfl_xor_sync(0xffffffffu, j, st);
+      const float oy = __shfl_xor_sync(0xffffffffu, y, st);
+      const bool up = ((sl & k) == 0);
+      const bool lower = ((sl & st) == 0);
+      const bool other_first = oy > y || (oy == y && oj < j);
+      const bool mine_first = y > oy || (y == oy && j < oj);
+      const bool take_other = (lower == up) ? other_first : mine_first;
+      j = take_other ? oj : j;
+      y = take_other ? oy : y;
+    }
+  }
+  const bool have = sl < n;
+  const float u = have ? ymax - y : 0.f;
+  float u1 = u, u2 = u * u;
+#pragma unroll
+  for (int off = 1; off < W; off <<= 1) {
+    const float t1 = __shfl_up_sync(0xffffffffu, u1, off, W);
+    const float t2 = __shfl_up_sync(0xffffffffu, u2, off, W);
+    if (sl >= off) {
+      u1 += t1;
+      u2 += t2;
+    }
+  }
+  const float kf = (float)(sl + 1);
+  float tk;
+  if constexpr (EC == kExpo2) {
+    const float disc = fmaf(u1, u1, -kf * (u2 - 1.0f));
+    tk = disc >= 0.f ? (u1 + sqrtf(disc)) / kf : -INFINITY;
+  } else {
+    tk = (1.0f + u1) / kf;
+  }
+  const unsigned okm = (__ballot_sync(0xffffffffu, have && u < tk) >> base) & kWMask;
+  const int kstar = okm == kWMask ? W : __ffs(~okm) - 1;          // leading ones; >= 1 for a row with entries
+  const float tprime = __shfl_sync(0xffffffffu, tk, base + (kstar > 0 ? kstar - 1 : 0));
+  const float tau = ymax - tprime;
+  const bool in = active && sl < kstar;
+  const float d = tprime - u;
+  const float pe = in ? (EC == kExpo2 ? d * d : d) : 0.f;
+  if (in) {
+    // the list becomes the exact support (by decreasing y), y in Eq. 1's units
+    list[sl].y = y;
+    list[sl].j = j;
+  }
+  float acc[PL];
+#pragma unroll
+  for (int t = 0; t < PL; ++t) acc[t] = 0.f;
+  const __nv_bfloat16* vbase = v + (size_t)b * p.sb + (size_t)h * p.sh + sl * PL;
+#pragma unroll
+  for (int t = 0; t < W; ++t) {
+    const bool has = active && t < kstar;
+    if (!__any_sync(0xffffffffu, has)) break;                      // supports are prefixes: nothing further either
+    const float pj = __shfl_sync(0xffffffffu, pe, base + t);
+    const int kj = __shfl_sync(0xffffffffu, j, base + t);
+    if (has) {
+      float vs[PL];
+      if constexpr (PL >= 8) load_bf16_vec<PL>(vbase + (size_t)kj * p.sn, vs);
+      else load_bf16<PL>(vbase + (size_t)kj * p.sn, vs);
+#pragma unroll
+      for (int u_ = 0; u_ < PL; ++u_) acc[u_] = fmaf(pj, vs[u_], acc[u_]);
+    }
+  }
+  if (active) {
+    __nv_bfloat16* o_row = o + (size_t)b * p.sb + (size_t)h * p.sh + (size_t)i * p.sn + sl * PL;
+    if constexpr (PL >= 8) store_bf16_vec<PL>(o_row, acc);
+    else store_bf16<PL>(o_row, acc);
+    if (sl == 0) {
+      tau_out[grow] = tau;
+      row_cnt[grow] = kstar;
     }
   }
 }
@@ -432,7 +560,8 @@ __device__ __forceinline__ void push_dense_tile(const Problem& p, int grow, int3
   if (atomicExch(tile_flag + id, 1) == 0) tile_list[atomicAdd(tile_count, 1)] = id;
 }
 
-template <int D>
+// EC: kExpo2 / kExpo1 select the closed-form solvers, kExpoGeneral the Newton ones (any exponent)
+template <int D, int EC>
 __global__ void __launch_bounds__(kWarpsPerCta * 32) row_fwd_kernel(Problem p, const __nv_bfloat16* __restrict__ v,
                                                                     const float* __restrict__ scale,
                                                                     int32_t* __restrict__ row_cnt,
@@ -446,26 +575,66 @@ __global__ void __launch_bounds__(kWarpsPerCta * 32) row_fwd_kernel(Problem p, c
   constexpr int PER = D / 32;
   const int lane = threadIdx.x & 31;
   const int total = p.B * p.H * p.N;
-  const int groups = (total + 3) / 4;
-  for (int grp = blockIdx.x * kWarpsPerCta + (threadIdx.x >> 5); grp < groups; grp += gridDim.x * kWarpsPerCta) {
-    // lanes 8r .. 8r+7 look at row 4*grp + r
-    const int my_row = 4 * grp + (lane >> 3);
-    const bool my_active = my_row < total;
+  const int blocks = (total + 15) / 16;
+  for (int blk = blockIdx.x * kWarpsPerCta + (threadIdx.x >> 5); blk < blocks; blk += gridDim.x * kWarpsPerCta) {
+    // A warp takes 16 consecutive rows; lane l (and l + 16) looks at row 16*blk + l.  Rows are then served by
+    // list length: four at a time with eight lanes each (1..8 entries), two at a time with sixteen lanes
+    // each (9..16 entries), the rest one by one with the whole warp.
+    constexpr bool kClosed = EC == kExpo2 || EC == kExpo1;
+    const int my_row = 16 * blk + (lane & 15);
     int mc0 = 0, mc1 = 0;
-    if (my_active) {
+    int cls = 3;                                     // 0: <= 8 entries, 1: <= 16, 2: whole warp / dense, 3: no row
+    if (my_row < total) {
       const int2 c = *reinterpret_cast<const int2*>(half_cnt + 2 * (size_t)my_row);
       mc0 = c.x;
       mc1 = c.y;
+      const int n = mc0 + mc1;
+      cls = (mc0 < 0 || mc1 < 0 || n < 1 || n > 16) ? 2 : n <= 8 ? 0 : 1;
     }
-    const bool small = !my_active || (mc0 >= 0 && mc1 >= 0 && mc0 + mc1 >= 1 && mc0 + mc1 <= 8);
-    if (__all_sync(0xffffffffu, small)) {
-      solve_rows_quad<D>(p, v, scale, entries, o, tau_out, row_cnt, my_active ? my_row : 0, my_active, mc0, mc1, lane);
-      continue;
+    unsigned m8 = __ballot_sync(0xffffffffu, lane < 16 && cls == 0);
+    unsigned m16 = __ballot_sync(0xffffffffu, lane < 16 && cls == 1);
+    unsigned mfull = __ballot_sync(0xffffffffu, lane < 16 && cls == 2);
+    if constexpr (kClosed) {
+      while (m8) {
+        const unsigned src = __fns(m8, 0, (lane >> 3) + 1);        // the row of this group of eight lanes
+        const bool active = src < 32u;
+        const int c0 = __shfl_sync(0xffffffffu, mc0, active ? src : 0), c1 = __shfl_sync(0xffffffffu, mc1, active ? src : 0);
+        solve_rows_closed<D, 8, EC>(p, v, scale, entries, o, tau_out, row_cnt, active ? 16 * blk + (int)src : 0, active, c0,
+                                    c1, false, lane);
+#pragma unroll
+        for (int t = 0; t < 4; ++t) m8 &= m8 - 1;
+      }
+      while (m16) {
+        const unsigned src = __fns(m16, 0, (lane >> 4) + 1);
+        const bool active = src < 32u;
+        const int c0 = __shfl_sync(0xffffffffu, mc0, active ? src : 0), c1 = __shfl_sync(0xffffffffu, mc1, active ? src : 0);
+        solve_rows_closed<D, 16, EC>(p, v, scale, entries, o, tau_out, row_cnt, active ? 16 * blk + (int)src : 0, active,
+                                     c0, c1, false, lane);
+        m16 &= m16 - 1;
+        m16 &= m16 - 1;
+      }
+    } else {
+      // Newton solvers: rows that iterate together wait for the slowest, so only groups of four consecutive
+      // rows that all have at most eight entries share a warp; every other row takes the whole warp.
+      const unsigned none = __ballot_sync(0xffffffffu, lane < 16 && cls == 3);
+#pragma unroll
+      for (int g = 0; g < 4; ++g) {
+        const unsigned gm = 0xFu << (4 * g);
+        if ((m8 & gm) != 0u && ((m8 | none) & gm) == gm) {
+          const int src = 4 * g + (lane >> 3);
+          const bool active = (m8 >> src) & 1u;
+          const int c0 = __shfl_sync(0xffffffffu, mc0, src), c1 = __shfl_sync(0xffffffffu, mc1, src);
+          solve_rows_sub<D, 8>(p, v, scale, entries, o, tau_out, row_cnt, active ? 16 * blk + src : 0, active, c0, c1, lane);
+        } else {
+          mfull |= (m8 | m16) & gm;
+        }
+      }
     }
-    for (int r = 0; r < 4; ++r) {
-      const int grow = 4 * grp + r;
-      if (grow >= total) break;
-      const int c0 = __shfl_sync(0xffffffffu, mc0, 8 * r), c1 = __shfl_sync(0xffffffffu, mc1, 8 * r);
+    while (mfull) {
+      const int src = __ffs(mfull) - 1;
+      mfull &= mfull - 1;
+      const int grow = 16 * blk + src;
+      const int c0 = __shfl_sync(0xffffffffu, mc0, src), c1 = __shfl_sync(0xffffffffu, mc1, src);
       if (c0 < 0 || c1 < 0 || c0 + c1 == 0) {
         if (lane == 0) {
           row_cnt[grow] = -2;
@@ -476,9 +645,32 @@ __global__ void __launch_bounds__(kWarpsPerCta * 32) row_fwd_kernel(Problem p, c
       const int bh = grow / p.N, i = grow - bh * p.N, b = bh / p.H, h = bh - b * p.H;
       const float a = (p.alpha - 1.0f) * (scale[(size_t)b * p.scale_sb + (size_t)h * p.N + i] * p.sm_scale);
       Entry* list = entries + (size_t)grow * kListCap;
-      const __nv_bfloat16* vbase = v + (size_t)b * p.sb + (size_t)h * p.sh + lane * PER;
-      __nv_bfloat16* o_row = o + (size_t)b * p.sb + (size_t)h * p.sh + (size_t)i * p.sn + lane * PER;
-      solve_row_full<D>(p, vbase, list, c0, c1, a, o_row, tau_out + grow, row_cnt + grow, lane);
+      if constexpr (kClosed) {
+        // up to 32 entries: closed form with the whole warp; more: Newton prefilter first, and the closed form
+        // if what it keeps fits the warp
+        const int n = c0 + c1;
+        if (n <= 32) {
+          solve_rows_closed<D, 32, EC>(p, v, scale, entries, o, tau_out, row_cnt, grow, true, c0, c1, false, lane);
+          continue;
+        }
+        int kept;
+        if (n <= 64) kept = prefilter_row<2>(p, list, c0, c1, a, lane);
+        else if (n <= 128) kept = prefilter_row<4>(p, list, c0, c1, a, lane);
+        else kept = prefilter_row<kSlots>(p, list, c0, c1, a, lane);
+        if (kept <= 32) {
+          solve_rows_closed<D, 32, EC>(p, v, scale, entries, o, tau_out, row_cnt, grow, true, kept, 0, true, lane);
+          continue;
+        }
+        const __nv_bfloat16* vbase = v + (size_t)b * p.sb + (size_t)h * p.sh + lane * PER;
+        __nv_bfloat16* o_row = o + (size_t)b * p.sb + (size_t)h * p.sh + (size_t)i * p.sn + lane * PER;
+        if (kept <= 64) finish_row<D, 2>(p, vbase, list, kept, o_row, tau_out + grow, row_cnt + grow, lane);
+        else if (kept <= 128) finish_row<D, 4>(p, vbase, list, kept, o_row, tau_out + grow, row_cnt + grow, lane);
+        else finish_row<D, kSlots>(p, vbase, list, kept, o_row, tau_out + grow, row_cnt + grow, lane);
+      } else {
+        const __nv_bfloat16* vbase = v + (size_t)b * p.sb + (size_t)h * p.sh + lane * PER;
+        __nv_bfloat16* o_row = o + (size_t)b * p.sb + (size_t)h * p.sh + (size_t)i * p.sn + lane * PER;
+        solve_row_full<D>(p, vbase, list, c0, c1, a, o_row, tau_out + grow, row_cnt + grow, lane);
+      }
     }
   }
 }
@@ -732,14 +924,20 @@ cudaError_t launch_row_fwd(const Problem& p, const void* v, const float* scale, 
                            int32_t* fb_count, int32_t* fb_list, int32_t* tile_flag, int32_t* tile_list,
                            int32_t* tile_count, int32_t* status, cudaStream_t stream) {
   const int grid = row_grid(p);
-  if (p.D == 64)
-    row_fwd_kernel<64><<<grid, kWarpsPerCta * 32, 0, stream>>>(p, (const __nv_bfloat16*)v, scale, row_cnt, half_cnt,
-                                                              entries, (__nv_bfloat16*)o, tau, fb_count, fb_list, tile_flag, tile_list,
-        tile_count, status);
-  else
-    row_fwd_kernel<128><<<grid, kWarpsPerCta * 32, 0, stream>>>(p, (const __nv_bfloat16*)v, scale, row_cnt, half_cnt,
-                                                               entries, (__nv_bfloat16*)o, tau, fb_count, fb_list, tile_flag, tile_list,
-        tile_count, status);
+#define ENTMAX_ROW_FWD(D, EC)                                                                                         \
+  row_fwd_kernel<D, EC><<<grid, kWarpsPerCta * 32, 0, stream>>>(p, (const __nv_bfloat16*)v, scale, row_cnt, half_cnt, \
+                                                                entries, (__nv_bfloat16*)o, tau, fb_count, fb_list,   \
+                                                                tile_flag, tile_list, tile_count, status)
+  if (p.D == 64) {
+    if (p.expo_class == kExpo2) ENTMAX_ROW_FWD(64, kExpo2);
+    else if (p.expo_class == kExpo1) ENTMAX_ROW_FWD(64, kExpo1);
+    else ENTMAX_ROW_FWD(64, kExpoGeneral);
+  } else {
+    if (p.expo_class == kExpo2) ENTMAX_ROW_FWD(128, kExpo2);
+    else if (p.expo_class == kExpo1) ENTMAX_ROW_FWD(128, kExpo1);
+    else ENTMAX_ROW_FWD(128, kExpoGeneral);
+  }
+#undef ENTMAX_ROW_FWD
   return cudaGetLastError();
 }
 
