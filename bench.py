@@ -236,17 +236,41 @@ def run_ours(args):
     d2h = sum(t.numel() * t.element_size() for t in outs_dev.values())
     E = max(1, min(K, 10))
     ee_start, ee_stop = [ev() for _ in range(E)], [ev() for _ in range(E)]
+    # three streams: copies in, compute, copies out; dO travels while the forward pass runs and O, tau leave while
+    # the backward pass runs (PCIe is full duplex).  A step starts when the previous one has fully finished.
+    s_in, s_cmp, s_out = torch.cuda.Stream(dev), torch.cuda.Stream(dev), torch.cuda.Stream(dev)
+    e_in1, e_in2, e_f, e_b, e_done = ev(), ev(), ev(), ev(), ev()
+    fwd_names = ("q", "k", "v", "beta", "gamma", "delta")
     barrier(world)
     torch.cuda.synchronize()
     for i in range(E):
-        ee_start[i].record()
-        for n in names:
-            d[n].copy_(host[n], non_blocking=True)
-        fwd()
-        bwd()
-        for n, t in outs_dev.items():
-            outs_host[n].copy_(t, non_blocking=True)
-        ee_stop[i].record()
+        ee_start[i].record(s_in)
+        s_cmp.wait_event(ee_start[i])
+        with torch.cuda.stream(s_in):
+            for n in fwd_names:
+                d[n].copy_(host[n], non_blocking=True)
+            e_in1.record(s_in)
+            d["d_o"].copy_(host["d_o"], non_blocking=True)
+            e_in2.record(s_in)
+        with torch.cuda.stream(s_cmp):
+            s_cmp.wait_event(e_in1)
+            binding.entmax_attn_fwd(d["q"], d["k"], d["v"], alpha, w.causal, d["beta"], d["gamma"], d["delta"], o=o,
+                                    tau=tau, workspace=ws, status=status, stream=s_cmp)
+            e_f.record(s_cmp)
+            s_cmp.wait_event(e_in2)
+            binding.entmax_attn_bwd(d["q"], d["k"], d["v"], tau, d["d_o"], alpha, w.causal, d["beta"], d["gamma"],
+                                    d["delta"], dq=dq, dk=dk, dv=dv, workspace=ws, status=status, stream=s_cmp)
+            e_b.record(s_cmp)
+        with torch.cuda.stream(s_out):
+            s_out.wait_event(e_f)
+            outs_host["o"].copy_(o, non_blocking=True)
+            outs_host["tau"].copy_(tau, non_blocking=True)
+            s_out.wait_event(e_b)
+            for n in ("dq", "dk", "dv"):
+                outs_host[n].copy_(outs_dev[n], non_blocking=True)
+            ee_stop[i].record(s_out)
+        # the next step's input copies must not overwrite tensors this step still reads
+        s_in.wait_event(ee_stop[i])
     torch.cuda.synchronize()
     barrier(world)
     e2e_ms = sum(a.elapsed_time(b) for a, b in zip(ee_start, ee_stop)) / E

@@ -71,12 +71,6 @@ __device__ __forceinline__ float oct_sum(float x) {
   x += __shfl_xor_sync(0xffffffffu, x, 4);
   return x;
 }
-__device__ __forceinline__ float oct_max(float x) {
-  x = fmaxf(x, __shfl_xor_sync(0xffffffffu, x, 1));
-  x = fmaxf(x, __shfl_xor_sync(0xffffffffu, x, 2));
-  x = fmaxf(x, __shfl_xor_sync(0xffffffffu, x, 4));
-  return x;
-}
 // reductions over aligned groups of W lanes (W = 8 or 16); the sum takes ascending strides like warp_sum
 template <int W>
 __device__ __forceinline__ float sub_sum(float x) {
