@@ -85,6 +85,15 @@ __device__ __forceinline__ float threshold_step(float s0, float s1, int expo_cla
   return (s0 - s0 / root) / s1;
 }
 
+// Fire-and-forget vector adds to global memory (sm_90+): reductions that return nothing, so no thread waits
+// for the old value to come back.
+__device__ __forceinline__ void red_add_v4(float* dst, float x, float y, float z, float w) {
+  asm volatile("red.global.add.v4.f32 [%0], {%1, %2, %3, %4};" ::"l"(dst), "f"(x), "f"(y), "f"(z), "f"(w) : "memory");
+}
+__device__ __forceinline__ void red_add_v2(float* dst, float x, float y) {
+  asm volatile("red.global.add.v2.f32 [%0], {%1, %2};" ::"l"(dst), "f"(x), "f"(y) : "memory");
+}
+
 // ---- launchers (each enqueues on `stream` and returns the cudaError_t of the launch) -------------
 cudaError_t launch_scale_table(const Problem& p, const float* beta, const float* gamma, const float* delta,
                                float* scale, int32_t* status, cudaStream_t stream);

@@ -92,8 +92,8 @@ __device__ __forceinline__ void store_slice(__nv_bfloat16* p, const float (&x)[P
 }
 template <int PER>
 __device__ __forceinline__ void atomic_add_slice(float* p, const float (&x)[PER]) {
-  if constexpr (PER == 2) atomicAdd(reinterpret_cast<float2*>(p), make_float2(x[0], x[1]));
-  else atomicAdd(reinterpret_cast<float4*>(p), make_float4(x[0], x[1], x[2], x[3]));
+  if constexpr (PER == 2) red_add_v2(p, x[0], x[1]);
+  else red_add_v4(p, x[0], x[1], x[2], x[3]);
 }
 
 struct RowCtx {

@@ -59,8 +59,8 @@ __device__ __forceinline__ void store_bf16(__nv_bfloat16* p, const float (&x)[PE
 }
 template <int PER>
 __device__ __forceinline__ void atomic_add_slice(float* p, const float (&x)[PER]) {
-  if constexpr (PER == 2) atomicAdd(reinterpret_cast<float2*>(p), make_float2(x[0], x[1]));
-  else atomicAdd(reinterpret_cast<float4*>(p), make_float4(x[0], x[1], x[2], x[3]));
+  if constexpr (PER == 2) red_add_v2(p, x[0], x[1]);
+  else red_add_v4(p, x[0], x[1], x[2], x[3]);
 }
 
 
@@ -116,7 +116,7 @@ template <int N>
 __device__ __forceinline__ void atomic_add_vec(float* p, const float (&x)[N]) {
 #pragma unroll
   for (int c = 0; c < N / 4; ++c)
-    atomicAdd(reinterpret_cast<float4*>(p + 4 * c), make_float4(x[4 * c], x[4 * c + 1], x[4 * c + 2], x[4 * c + 3]));
+    red_add_v4(p + 4 * c, x[4 * c], x[4 * c + 1], x[4 * c + 2], x[4 * c + 3]);
 }
 
 __device__ __forceinline__ void push_dense_row(int grow, int32_t* fb_count, int32_t* fb_list, int32_t* status) {

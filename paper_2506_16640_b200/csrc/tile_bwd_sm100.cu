@@ -93,11 +93,6 @@ __device__ __forceinline__ uint32_t pack_bf16(float a, float b) {
   return *reinterpret_cast<const uint32_t*>(&hh);
 }
 
-// fire-and-forget vector add to global memory (no value returned)
-__device__ __forceinline__ void red_add_v4(float* dst, float x, float y, float z, float w) {
-  asm volatile("red.global.add.v4.f32 [%0], {%1, %2, %3, %4};" ::"l"(dst), "f"(x), "f"(y), "f"(z), "f"(w) : "memory");
-}
-
 // Marks the rows of row_list[0 .. *row_count) in the per-tile masks and lists every tile once.
 __global__ void mark_tiles_kernel(int N, int tiles_per_head, const int32_t* __restrict__ row_list,
                                   const int32_t* __restrict__ row_count, uint32_t* __restrict__ tile_mask,
