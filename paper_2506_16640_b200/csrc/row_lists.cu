@@ -18,9 +18,9 @@ constexpr int kWarpsPerCta = 8;
 constexpr int kSlots = kListCap / 32;
 constexpr int kMaxNewton = 400;
 
-// Butterfly sum with ascending strides: for values held by lanes 0..7 only (zeros elsewhere) the first
-// three steps are exactly oct_sum's tree and the rest add zeros, so the full-warp and the
-// eight-lanes-per-row paths give the same bits for the same sorted support.
+// Butterfly sum with ascending strides: for values held by lanes 0..W-1 only (zeros elsewhere) the first
+// log2(W) steps are exactly sub_sum<W>'s tree and the rest add zeros, so the full-warp and the
+// W-lanes-per-row paths give the same bits for the same sorted support.
 __device__ __forceinline__ float warp_sum(float x) {
 #pragma unroll
   for (int o = 1; o < 32; o <<= 1) x += __shfl_xor_sync(0xffffffffu, x, o);
@@ -64,13 +64,6 @@ __device__ __forceinline__ void atomic_add_slice(float* p, const float (&x)[PER]
 }
 
 
-// reductions over aligned groups of eight lanes
-__device__ __forceinline__ float oct_sum(float x) {
-  x += __shfl_xor_sync(0xffffffffu, x, 1);
-  x += __shfl_xor_sync(0xffffffffu, x, 2);
-  x += __shfl_xor_sync(0xffffffffu, x, 4);
-  return x;
-}
 // reductions over aligned groups of W lanes (W = 8 or 16); the sum takes ascending strides like warp_sum
 template <int W>
 __device__ __forceinline__ float sub_sum(float x) {
@@ -772,18 +765,36 @@ __device__ __forceinline__ void bwd_row_full(const Problem& p, const __nv_bfloat
   store_bf16<PER>(dq + hbase + (size_t)i * p.sn, acc);
 }
 
-// Backward of four rows at once, eight lanes per row, for rows with at most eight list entries.
-template <int D>
-__device__ __forceinline__ void bwd_rows_quad(const Problem& p, const __nv_bfloat16* __restrict__ q,
-                                              const __nv_bfloat16* __restrict__ k, const __nv_bfloat16* __restrict__ v,
-                                              const __nv_bfloat16* __restrict__ d_o, const float* __restrict__ scale,
-                                              const float* __restrict__ tau_in, const Entry* __restrict__ entries,
-                                              __nv_bfloat16* __restrict__ dq, float* __restrict__ acc_dk,
-                                              float* __restrict__ acc_dv, float* __restrict__ dc_rows, int grow,
-                                              bool active, int c0, int c1, bool saved, int lane) {
-  constexpr int PL = D / 8;                        // elements of a row per lane
-  const int sl = lane & 7;
-  const int base = lane & 24;
+// PL consecutive elements of a row: loads, stores and accumulator adds for any slice width used here
+template <int PL>
+__device__ __forceinline__ void load_slice_bf16(const __nv_bfloat16* p, float (&x)[PL]) {
+  if constexpr (PL >= 8) load_bf16_vec<PL>(p, x);
+  else load_bf16<PL>(p, x);
+}
+template <int PL>
+__device__ __forceinline__ void store_slice_bf16(__nv_bfloat16* p, const float (&x)[PL]) {
+  if constexpr (PL >= 8) store_bf16_vec<PL>(p, x);
+  else store_bf16<PL>(p, x);
+}
+template <int PL>
+__device__ __forceinline__ void add_slice(float* p, const float (&x)[PL]) {
+  if constexpr (PL >= 8) atomic_add_vec<PL>(p, x);
+  else atomic_add_slice<PL>(p, x);
+}
+
+// Backward of 32 / W rows at once, W lanes per row (W = 8, 16 or 32), for rows with at most W list entries.
+template <int D, int W>
+__device__ __forceinline__ void bwd_rows_sub(const Problem& p, const __nv_bfloat16* __restrict__ q,
+                                             const __nv_bfloat16* __restrict__ k, const __nv_bfloat16* __restrict__ v,
+                                             const __nv_bfloat16* __restrict__ d_o, const float* __restrict__ scale,
+                                             const float* __restrict__ tau_in, const Entry* __restrict__ entries,
+                                             __nv_bfloat16* __restrict__ dq, float* __restrict__ acc_dk,
+                                             float* __restrict__ acc_dv, float* __restrict__ dc_rows, int grow,
+                                             bool active, int c0, int c1, bool saved, int lane) {
+  constexpr int PL = D / W;                        // elements of a row per lane
+  constexpr unsigned kWMask = W == 32 ? 0xffffffffu : ((1u << (W & 31)) - 1u);
+  const int sl = lane & (W - 1);
+  const int base = lane & (32 - W);
   const int n = active ? c0 + c1 : 0;
   const int bh = grow / p.N, i = grow - bh * p.N, b = bh / p.H, h = bh - b * p.H;
   const float g = active ? scale[(size_t)b * p.scale_sb + (size_t)h * p.N + i] * p.sm_scale : 0.f;
@@ -791,74 +802,75 @@ __device__ __forceinline__ void bwd_rows_quad(const Problem& p, const __nv_bfloa
   const float tau = active ? tau_in[grow] : 0.f;
   const size_t hbase = (size_t)b * p.sb + (size_t)h * p.sh + sl * PL;
   float qs[PL], gs[PL];
-  load_bf16_vec<PL>(q + hbase + (size_t)i * p.sn, qs);
-  load_bf16_vec<PL>(d_o + hbase + (size_t)i * p.sn, gs);
+  load_slice_bf16<PL>(q + hbase + (size_t)i * p.sn, qs);
+  load_slice_bf16<PL>(d_o + hbase + (size_t)i * p.sn, gs);
   const Entry* list = entries + (size_t)grow * kListCap;
   float yv = -1.0f, zz = 0.f;
   int j = 0;
   if (sl < n) {
     const Entry en = list[sl < c0 ? sl : kHalfCap + sl - c0];
+    // a list saved by the forward pass holds y = (alpha-1) s in Eq. 1's units, a fresh one raw <q_i, k_j>
     yv = saved ? en.y - tau : fmaf(a, en.y, -tau);
     j = en.j;
     zz = saved ? en.y / a : en.y;                  // raw <q_i, k_j>
   }
   const bool in = yv > 0.f;
-  const unsigned msub = (__ballot_sync(0xffffffffu, in) >> base) & 0xffu;
+  const unsigned msub = (__ballot_sync(0xffffffffu, in) >> base) & kWMask;
   // dP_ij = <dO_i, v_j> on the support
   float dpv = 0.f;
-#pragma unroll
-  for (int t = 0; t < 8; ++t) {
+#pragma unroll 4
+  for (int t = 0; t < W; ++t) {
+    if (!__any_sync(0xffffffffu, (msub >> t) != 0u)) break;        // no row has entries from slot t on
     const bool has = (msub >> t) & 1u;
-    if (!__any_sync(0xffffffffu, has)) continue;
     const int kj = __shfl_sync(0xffffffffu, j, base + t);
     float dp = 0.f;
     if (has) {
       float vs[PL];
-      load_bf16_vec<PL>(v + hbase + (size_t)kj * p.sn, vs);
+      load_slice_bf16<PL>(v + hbase + (size_t)kj * p.sn, vs);
 #pragma unroll
       for (int u = 0; u < PL; ++u) dp = fmaf(gs[u], vs[u], dp);
     }
-    dp = oct_sum(dp);
+    dp = sub_sum<W>(dp);
     if (sl == t) dpv = dp;
   }
   float pe = 0.f, u = 0.f;
   if (in) pow_pair(yv, p.expo_class, p.expo, pe, u);
-  const float su = oct_sum(u), sud = oct_sum(u * dpv);
+  const float su = sub_sum<W>(u), sud = sub_sum<W>(u * dpv);
   const float rho = su > 0.f ? sud / su : 0.f;
   const float gds_own = g * u * (dpv - rho);
   if (dc_rows) {
     // dL/dc_i = sum_j dS_ij z_ij with z_ij = <q_i,k_j> sm_scale (chain rule through s = c z)
-    const float dc = oct_sum(u * (dpv - rho) * zz);
+    const float dc = sub_sum<W>(u * (dpv - rho) * zz);
     if (active && sl == 0) dc_rows[grow] = dc * p.sm_scale;
   }
   float acc[PL];
 #pragma unroll
   for (int t = 0; t < PL; ++t) acc[t] = 0.f;
   const size_t arow = (size_t)bh * p.N;
-#pragma unroll
-  for (int t = 0; t < 8; ++t) {
+#pragma unroll 4
+  for (int t = 0; t < W; ++t) {
+    if (!__any_sync(0xffffffffu, (msub >> t) != 0u)) break;
     const bool has = (msub >> t) & 1u;
-    if (!__any_sync(0xffffffffu, has)) continue;
     const int kj = __shfl_sync(0xffffffffu, j, base + t);
     const float gds = __shfl_sync(0xffffffffu, gds_own, base + t);
     const float pj = __shfl_sync(0xffffffffu, pe, base + t);
     if (has) {
       float ks[PL], dkv[PL], dvv[PL];
-      load_bf16_vec<PL>(k + hbase + (size_t)kj * p.sn, ks);
+      load_slice_bf16<PL>(k + hbase + (size_t)kj * p.sn, ks);
 #pragma unroll
       for (int w = 0; w < PL; ++w) {
         acc[w] = fmaf(gds, ks[w], acc[w]);
         dkv[w] = gds * qs[w];
         dvv[w] = pj * gs[w];
       }
-      atomic_add_vec<PL>(acc_dk + (arow + kj) * D + sl * PL, dkv);
-      atomic_add_vec<PL>(acc_dv + (arow + kj) * D + sl * PL, dvv);
+      add_slice<PL>(acc_dk + (arow + kj) * D + sl * PL, dkv);
+      add_slice<PL>(acc_dv + (arow + kj) * D + sl * PL, dvv);
     }
   }
-  if (active) store_bf16_vec<PL>(dq + hbase + (size_t)i * p.sn, acc);
+  if (active) store_slice_bf16<PL>(dq + hbase + (size_t)i * p.sn, acc);
 }
 
-// (register cap: three CTAs per SM -- this kernel waits on gathers and atomics, occupancy is what hides them)
+// (register cap: four CTAs per SM -- this kernel waits on gathers and reductions, occupancy is what hides them)
 template <int D>
 __global__ void __launch_bounds__(kWarpsPerCta * 32, 4) row_bwd_kernel(
     Problem p, const __nv_bfloat16* __restrict__ q, const __nv_bfloat16* __restrict__ k,
@@ -870,13 +882,14 @@ __global__ void __launch_bounds__(kWarpsPerCta * 32, 4) row_bwd_kernel(
   // row) and `entries` its compacted support lists
   const int lane = threadIdx.x & 31;
   const int total = p.B * p.H * p.N;
-  const int groups = (total + 3) / 4;
-  for (int grp = blockIdx.x * kWarpsPerCta + (threadIdx.x >> 5); grp < groups; grp += gridDim.x * kWarpsPerCta) {
-    // lanes 8r .. 8r+7 look at row 4*grp + r
-    const int my_row = 4 * grp + (lane >> 3);
-    const bool my_active = my_row < total;
+  const int blocks = (total + 15) / 16;
+  for (int blk = blockIdx.x * kWarpsPerCta + (threadIdx.x >> 5); blk < blocks; blk += gridDim.x * kWarpsPerCta) {
+    // A warp takes 16 consecutive rows; lane l (and l + 16) looks at row 16*blk + l.  Rows are served by list
+    // length: four at a time (<= 8 entries), two at a time (<= 16), one at a time (<= 32, or the long form).
+    const int my_row = 16 * blk + (lane & 15);
     int mc0 = 0, mc1 = 0;
-    if (my_active) {
+    int cls = 4;                                     // 0: <= 8 entries, 1: <= 16, 2: <= 32, 3: more / dense, 4: no row
+    if (my_row < total) {
       if (saved) {
         mc0 = half_cnt[my_row];
       } else {
@@ -884,17 +897,43 @@ __global__ void __launch_bounds__(kWarpsPerCta * 32, 4) row_bwd_kernel(
         mc0 = c.x;
         mc1 = c.y;
       }
+      const int n = mc0 + mc1;
+      cls = (mc0 < 0 || mc1 < 0 || n > 32) ? 3 : n <= 8 ? 0 : n <= 16 ? 1 : 2;
     }
-    const bool small = !my_active || (mc0 >= 0 && mc1 >= 0 && mc0 + mc1 <= 8);
-    if (__all_sync(0xffffffffu, small)) {
-      bwd_rows_quad<D>(p, q, k, v, d_o, scale, tau_in, entries, dq, acc_dk, acc_dv, dc_rows, my_active ? my_row : 0,
-                       my_active, mc0, mc1, saved != 0, lane);
-      continue;
+    unsigned m8 = __ballot_sync(0xffffffffu, lane < 16 && cls == 0);
+    unsigned m16 = __ballot_sync(0xffffffffu, lane < 16 && cls == 1);
+    unsigned m32 = __ballot_sync(0xffffffffu, lane < 16 && cls == 2);
+    unsigned mlong = __ballot_sync(0xffffffffu, lane < 16 && cls == 3);
+    while (m8) {
+      const unsigned src = __fns(m8, 0, (lane >> 3) + 1);          // the row of this group of eight lanes
+      const bool active = src < 32u;
+      const int c0 = __shfl_sync(0xffffffffu, mc0, active ? src : 0), c1 = __shfl_sync(0xffffffffu, mc1, active ? src : 0);
+      bwd_rows_sub<D, 8>(p, q, k, v, d_o, scale, tau_in, entries, dq, acc_dk, acc_dv, dc_rows,
+                         active ? 16 * blk + (int)src : 0, active, c0, c1, saved != 0, lane);
+#pragma unroll
+      for (int t = 0; t < 4; ++t) m8 &= m8 - 1;
     }
-    for (int r = 0; r < 4; ++r) {
-      const int grow = 4 * grp + r;
-      if (grow >= total) break;
-      const int c0 = __shfl_sync(0xffffffffu, mc0, 8 * r), c1 = __shfl_sync(0xffffffffu, mc1, 8 * r);
+    while (m16) {
+      const unsigned src = __fns(m16, 0, (lane >> 4) + 1);
+      const bool active = src < 32u;
+      const int c0 = __shfl_sync(0xffffffffu, mc0, active ? src : 0), c1 = __shfl_sync(0xffffffffu, mc1, active ? src : 0);
+      bwd_rows_sub<D, 16>(p, q, k, v, d_o, scale, tau_in, entries, dq, acc_dk, acc_dv, dc_rows,
+                          active ? 16 * blk + (int)src : 0, active, c0, c1, saved != 0, lane);
+      m16 &= m16 - 1;
+      m16 &= m16 - 1;
+    }
+    while (m32) {
+      const int src = __ffs(m32) - 1;
+      m32 &= m32 - 1;
+      const int c0 = __shfl_sync(0xffffffffu, mc0, src), c1 = __shfl_sync(0xffffffffu, mc1, src);
+      bwd_rows_sub<D, 32>(p, q, k, v, d_o, scale, tau_in, entries, dq, acc_dk, acc_dv, dc_rows, 16 * blk + src, true, c0, c1,
+                          saved != 0, lane);
+    }
+    while (mlong) {
+      const int src = __ffs(mlong) - 1;
+      mlong &= mlong - 1;
+      const int grow = 16 * blk + src;
+      const int c0 = __shfl_sync(0xffffffffu, mc0, src), c1 = __shfl_sync(0xffffffffu, mc1, src);
       if (c0 < 0 || c1 < 0) {
         if (lane == 0) push_dense_row(grow, fb_count, fb_list, status);
         continue;
