@@ -296,6 +296,21 @@ __device__ __forceinline__ void finish_row(const Problem& p, const __nv_bfloat16
   }
 }
 
+// Out-of-line forms for the rare rows with more than 32 candidates (kept out of the hot loop's code)
+__device__ __noinline__ int prefilter_long(const Problem& p, Entry* list, int c0, int c1, float a, int lane) {
+  const int n = c0 + c1;
+  if (n <= 64) return prefilter_row<2>(p, list, c0, c1, a, lane);
+  if (n <= 128) return prefilter_row<4>(p, list, c0, c1, a, lane);
+  return prefilter_row<kSlots>(p, list, c0, c1, a, lane);
+}
+template <int D>
+__device__ __noinline__ void finish_long(const Problem& p, const __nv_bfloat16* __restrict__ vbase, Entry* list, int kept,
+                                         __nv_bfloat16* o_row, float* tau_slot, int32_t* cnt_slot, int lane) {
+  if (kept <= 64) finish_row<D, 2>(p, vbase, list, kept, o_row, tau_slot, cnt_slot, lane);
+  else if (kept <= 128) finish_row<D, 4>(p, vbase, list, kept, o_row, tau_slot, cnt_slot, lane);
+  else finish_row<D, kSlots>(p, vbase, list, kept, o_row, tau_slot, cnt_slot, lane);
+}
+
 // One row with the whole warp.
 template <int D>
 __device__ __forceinline__ void solve_row_full(const Problem& p, const __nv_bfloat16* __restrict__ vbase, Entry* list,
@@ -511,7 +526,8 @@ __device__ __forceinline__ void solve_rows_closed(const Problem& p, const __nv_b
 #pragma unroll
   for (int t = 0; t < PL; ++t) acc[t] = 0.f;
   const __nv_bfloat16* vbase = v + (size_t)b * p.sb + (size_t)h * p.sh + sl * PL;
-#pragma unroll
+  // (not unrolled: a handful of iterations run, and the three widths of this function share the instruction cache)
+#pragma unroll 1
   for (int t = 0; t < W; ++t) {
     const bool has = active && t < kstar;
     if (!__any_sync(0xffffffffu, has)) break;                      // supports are prefixes: nothing further either
@@ -640,19 +656,14 @@ __global__ void __launch_bounds__(kWarpsPerCta * 32) row_fwd_kernel(Problem p, c
           solve_rows_closed<D, 32, EC>(p, v, scale, entries, o, tau_out, row_cnt, grow, true, c0, c1, false, lane);
           continue;
         }
-        int kept;
-        if (n <= 64) kept = prefilter_row<2>(p, list, c0, c1, a, lane);
-        else if (n <= 128) kept = prefilter_row<4>(p, list, c0, c1, a, lane);
-        else kept = prefilter_row<kSlots>(p, list, c0, c1, a, lane);
+        const int kept = prefilter_long(p, list, c0, c1, a, lane);
         if (kept <= 32) {
           solve_rows_closed<D, 32, EC>(p, v, scale, entries, o, tau_out, row_cnt, grow, true, kept, 0, true, lane);
           continue;
         }
         const __nv_bfloat16* vbase = v + (size_t)b * p.sb + (size_t)h * p.sh + lane * PER;
         __nv_bfloat16* o_row = o + (size_t)b * p.sb + (size_t)h * p.sh + (size_t)i * p.sn + lane * PER;
-        if (kept <= 64) finish_row<D, 2>(p, vbase, list, kept, o_row, tau_out + grow, row_cnt + grow, lane);
-        else if (kept <= 128) finish_row<D, 4>(p, vbase, list, kept, o_row, tau_out + grow, row_cnt + grow, lane);
-        else finish_row<D, kSlots>(p, vbase, list, kept, o_row, tau_out + grow, row_cnt + grow, lane);
+        finish_long<D>(p, vbase, list, kept, o_row, tau_out + grow, row_cnt + grow, lane);
       } else {
         const __nv_bfloat16* vbase = v + (size_t)b * p.sb + (size_t)h * p.sh + lane * PER;
         __nv_bfloat16* o_row = o + (size_t)b * p.sb + (size_t)h * p.sh + (size_t)i * p.sn + lane * PER;
@@ -664,7 +675,7 @@ __global__ void __launch_bounds__(kWarpsPerCta * 32) row_fwd_kernel(Problem p, c
 
 // Backward of one row with the whole warp: the entmax Jacobian on the support.
 template <int D>
-__device__ __forceinline__ void bwd_row_full(const Problem& p, const __nv_bfloat16* __restrict__ q,
+__device__ __noinline__ void bwd_row_full(const Problem& p, const __nv_bfloat16* __restrict__ q,
                                              const __nv_bfloat16* __restrict__ k, const __nv_bfloat16* __restrict__ v,
                                              const __nv_bfloat16* __restrict__ d_o, const float* __restrict__ scale,
                                              const float* __restrict__ tau_in, const Entry* __restrict__ entries,

@@ -119,7 +119,7 @@ __device__ __forceinline__ int qtile_tiles(const SweepArgs& a, int item, int x) 
 // maxima only: the running maxima and thresholds the real stream then starts from are already close to
 // their final values, which roughly halves the candidates it pushes (a one-pass stream pushes every new
 // running maximum, about ln n of them per row; after a 1/16 sample about ln 16 are left; measured best among 8, 16, 32, 64).
-constexpr int kSampleStride = 16;
+constexpr int kSampleStride = 8;
 constexpr int kSampleMinKeys = 4096;   // below this the stream is too short for the sample to pay
 __device__ __forceinline__ int sample_tiles(const SweepArgs& a, int item) {
   if (a.mode != 0) return 0;
