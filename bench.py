@@ -35,7 +35,7 @@ NOMINAL_BF16_TFLOPS = 2250.0
 FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
 # DRAM bytes (read + write) of one forward score-sweep launch on the benchmark workload, from the ncu
 # capture summarised under profiles/ (None until a capture exists).
-SWEEP_DRAM_TRAFFIC_BYTES = 363791104   # dram__bytes_read 295798016 + dram__bytes_write 67993088
+SWEEP_DRAM_TRAFFIC_BYTES = 355845632   # dram__bytes_read 295181056 + dram__bytes_write 60664576
 
 
 def visible_pairs(w) -> int:
