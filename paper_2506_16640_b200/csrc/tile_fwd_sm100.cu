@@ -11,10 +11,11 @@
 // A work item is one Q tile of 128 rows that holds at least one such row (a list written by the row
 // kernel); only the rows flagged there are written back.
 //
-// CTA: warp 0 TMA producer, warp 1 MMA issuer, warps 2..5 consumers (TMEM lane = query row, one thread
-// per row, all 128 columns of a K tile).  The number of Newton sweeps is decided by the consumers; they
-// publish "all rows converged" through shared memory and a control mbarrier that every role waits on
-// between sweeps.  Every wait is bounded (see sm100_ptx.cuh); on expiry the CTA flags the call's status
+// CTA: warp 0 TMA producer, warp 1 MMA issuer, warps 2..9 consumers: TMEM lane = query row, two threads per
+// row (warps w and w + 4 read the same lane quadrant), each scanning 64 of a K tile's 128 columns; at the end of a
+// sweep the two swap their partial sums through shared memory.  The number of Newton sweeps is decided by the
+// consumers; they publish "all rows converged" through shared memory and a control mbarrier that every role
+// waits on between sweeps.  Every wait is bounded (see sm100_ptx.cuh); on expiry the CTA flags the call's status
 // word and leaves.
 #include <cuda.h>
 
@@ -29,7 +30,7 @@ using namespace sm100;
 
 constexpr int TM = 128;            // query rows per item = TMEM lanes
 constexpr int TN = 128;            // keys per K/V tile
-constexpr int kThreadsT = 6 * 32;
+constexpr int kThreadsT = 10 * 32;    // TMA warp, MMA warp, eight consumer warps
 constexpr int kStagesT = 2;
 constexpr int kMaxSweeps = 48;     // 1 max sweep + at most 46 Newton sweeps + the output sweep
 constexpr int kPBytes = TM * TN * 2;
@@ -40,7 +41,8 @@ struct TCfg {
   static constexpr int kQBytes = TM * HD * 2;
   static constexpr int kKBytes = TN * HD * 2;      // also the size of a V tile
   static constexpr int kBarBytes = 256;
-  static constexpr int kSmemBytes = kQBytes + kStagesT * 2 * kKBytes + kPBytes + 1024 + kBarBytes;
+  static constexpr int kXchgBytes = 2 * TM * 8;    // one float2 per (half, row): partial sums between the two threads of a row
+  static constexpr int kSmemBytes = kQBytes + kStagesT * 2 * kKBytes + kPBytes + 1024 + kBarBytes + kXchgBytes;
   static constexpr int kTmemO = 2 * TN;            // first TMEM column of the O accumulator
 };
 
@@ -103,9 +105,11 @@ __global__ void __launch_bounds__(kThreadsT, 1) tile_fwd_kernel(const __grid_con
   const uint32_t o_full = p_empty + 8, o_empty = o_full + 8;
   const uint32_t ctl = o_empty + 8;                                   // the consumers' vote on a sweep is in
   const uint32_t done_word = ctl + 8;                                 // uint32 [3]
-  const uint32_t tmem_slot = done_word + 12;
+  const uint32_t x_bar = done_word + 16;                              // partial sums of a sweep are in shared memory
+  const uint32_t tmem_slot = x_bar + 8;
   const uint32_t abort_flag = tmem_slot + 4;
-  static_assert(8 * (2 + 2 * kStagesT + 4 + 4 + 1) + 12 + 8 <= C::kBarBytes, "barrier area");
+  const uint32_t xchg = bars + C::kBarBytes;                          // float2 [2][TM]
+  static_assert(8 * (2 + 2 * kStagesT + 4 + 4 + 1) + 16 + 8 + 8 <= C::kBarBytes, "barrier area");
 
   const int warp = threadIdx.x >> 5;
   const int lane = threadIdx.x & 31;
@@ -120,13 +124,14 @@ __global__ void __launch_bounds__(kThreadsT, 1) tile_fwd_kernel(const __grid_con
     }
     for (int t = 0; t < 2; ++t) {
       mbar_init(s_full + 8 * t, 1);
-      mbar_init(s_empty + 8 * t, 4);
+      mbar_init(s_empty + 8 * t, 8);
     }
-    mbar_init(p_full, 4);
+    mbar_init(p_full, 8);
     mbar_init(p_empty, 1);
     mbar_init(o_full, 1);
-    mbar_init(o_empty, 4);
-    mbar_init(ctl, 4);
+    mbar_init(o_empty, 8);
+    mbar_init(ctl, 8);
+    mbar_init(x_bar, 8);
     for (int t = 0; t < 3; ++t) sts_u32(done_word + 4 * t, 1u);
     sts_u32(abort_flag, 0u);
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -269,11 +274,13 @@ __global__ void __launch_bounds__(kThreadsT, 1) tile_fwd_kernel(const __grid_con
       }
     }
   } else {
-    // ------------------------------------------------------------------ consumers: one thread per query row
+    // ------------------------------------------------------------------ consumers: two threads per query row
+    // (warps w and w + 4 share a TMEM lane quadrant; `half` picks the 64 of a tile's 128 columns a thread scans)
     const int quad = warp & 3;
+    const int half = (warp - 2) >> 2;
     const int row_local = quad * 32 + lane;
     const uint32_t taddr_row = tmem_base + ((uint32_t)(quad * 32) << 16);
-    uint32_t sphase[2] = {0, 0}, pphase = 0, ophase = 0, cphase = 0;
+    uint32_t sphase[2] = {0, 0}, pphase = 0, ophase = 0, cphase = 0, xphase = 0;
     int sbuf = 0;
     bool alive = true;
     for (int it = blockIdx.x; it < n_tiles && alive; it += gridDim.x) {
@@ -311,7 +318,7 @@ __global__ void __launch_bounds__(kThreadsT, 1) tile_fwd_kernel(const __grid_con
             if (!alive) break;
           }
 #pragma unroll 1
-          for (int c = 0; c < TN / 32; ++c) {
+          for (int c = 2 * half; c < 2 * half + 2; ++c) {
             float va[32];
             tmem_ld32(taddr_row + sbuf * TN + c * 32, va);
             tmem_ld_wait();
@@ -397,7 +404,7 @@ __global__ void __launch_bounds__(kThreadsT, 1) tile_fwd_kernel(const __grid_con
           __nv_bfloat16* orow =
               reinterpret_cast<__nv_bfloat16*>(a.o) + (size_t)b * a.sb + (size_t)h * a.sh + (size_t)i * a.sn;
 #pragma unroll
-          for (int c = 0; c < HD / 32; ++c) {
+          for (int c = half * (HD / 64); c < (half + 1) * (HD / 64); ++c) {
             float va[32];
             tmem_ld32(taddr_row + C::kTmemO + c * 32, va);
             tmem_ld_wait();
@@ -414,7 +421,7 @@ __global__ void __launch_bounds__(kThreadsT, 1) tile_fwd_kernel(const __grid_con
               }
             }
           }
-          if (write) a.tau[grow] = tau;
+          if (write && half == 0) a.tau[grow] = tau;
           if (a.status && threadIdx.x == 64) {
             // diagnostics: sweeps spent (y_max sweep + Newton sweeps + output sweep) and tiles processed
             atomicAdd(a.status + ENTMAX_ATTN_STATUS_TILE_SWEEPS, s + 1);
@@ -425,7 +432,27 @@ __global__ void __launch_bounds__(kThreadsT, 1) tile_fwd_kernel(const __grid_con
           if (lane == 0) mbar_arrive(o_empty);
           break;
         }
-        // ---- between sweeps: Newton update and the vote "every row of the tile has converged"
+        // ---- between sweeps: the two threads of a row swap their partial results through shared memory (both
+        //      then hold the same totals, added in the same order), Newton update, and the vote "every row of
+        //      the tile has converged"
+        {
+          const uint32_t mine = xchg + (uint32_t)(half * TM + row_local) * 8u;
+          const uint32_t theirs = xchg + (uint32_t)((half ^ 1) * TM + row_local) * 8u;
+          sts_u32(mine, __float_as_uint(s == 0 ? ymax : s0));
+          sts_u32(mine + 4, __float_as_uint(s1));
+          __syncwarp();
+          if (lane == 0) mbar_arrive(x_bar);
+          alive = __all_sync(0xffffffffu, mbar_wait(x_bar, xphase, abort_flag));
+          xphase ^= 1u;
+          if (!alive) break;
+          const float o0 = __uint_as_float(lds_u32(theirs)), o1 = __uint_as_float(lds_u32(theirs + 4));
+          if (s == 0) {
+            ymax = fmaxf(ymax, o0);
+          } else {
+            s0 = half == 0 ? s0 + o0 : o0 + s0;
+            s1 = half == 0 ? s1 + o1 : o1 + s1;
+          }
+        }
         if (s == 0) {
           tau = ymax - 1.0f;
         } else if (!done) {
