@@ -1,4 +1,4 @@
-"""The forward / backward / decode entry points only enqueue work on the caller's stream (no allocation, no
+"""The workspace-taking forward / backward entry points and the decode entry point only enqueue work on the caller's stream (no allocation, no
 synchronisation), so a caller can record them into a CUDA graph and replay it on new data in the same buffers."""
 import pytest
 import torch
