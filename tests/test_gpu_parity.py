@@ -132,6 +132,24 @@ def test_mixed_sparse_and_dense_rows_backward():
         parity.check_bwd_head(inp, 1.5, bwd, bh)
 
 
+@pytest.mark.parametrize("alpha", [1.25, 1.5, 2.0])
+@pytest.mark.parametrize("dtype", ["bf16", "fp32"])
+def test_all_logits_equal_gives_uniform_rows(alpha, dtype):
+    # q = 0: every visible key ties, p_i is uniform over the i + 1 visible keys, tau_i = -(i + 1)^-(alpha-1) (Eq. 1 with
+    # sum p = 1), O_i the running mean of V; rows grow from one key to a dense 600
+    inp = make_inputs(_small("ties", 600, 64, True, dtype=dtype, use_scale=True, seed=31))
+    inp.q.zero_()
+    got = parity.run_fwd(inp, alpha)
+    n = torch.arange(1, 601, dtype=torch.float64)
+    tau_ref = -n.pow(-(alpha - 1.0))
+    for bh in range(inp.workload.H):
+        tau = got["tau"][0, bh].double().cpu()
+        assert (tau - tau_ref).abs().max().item() <= parity.tau_tol(dtype)
+        o_ref = inp.v[0, bh].double().cumsum(dim=0) / n[:, None]
+        assert (got["o"][0, bh].double().cpu() - o_ref).abs().max().item() <= parity.O_TOL
+        parity.check_fwd_rows(inp, alpha, got, bh, np.arange(0, 600, 7), check_support=False)
+
+
 def test_n_mode_total_length_and_strided_layout():
     inp = make_inputs(_small("nmode", 300, 64, True, seed=11))
     got = parity.run_fwd(inp, 1.5, n_mode=1)
