@@ -169,6 +169,33 @@ def test_n_mode_total_length_and_strided_layout():
     parity.check_fwd_rows(inp, 1.5, got2, 1, np.arange(300))
 
 
+@pytest.mark.parametrize("d", [64, 128])
+def test_dense_tiles_with_strided_layout_and_batches(d):
+    # every row dense, two batch elements, tensors stored [B, N, H, D] and passed as [B, H, N, D] views: the tile
+    # kernels' tensor maps, row addressing and the fp32 dK / dV accumulators all see the strides
+    inp = make_inputs(_small("dense_strided", 700, d, True, B=2, H=3, use_scale=True, sigma=0.04, backward=True, seed=61))
+    w = inp.workload
+    dev = parity.to_device(inp)
+    for name in ("q", "k", "v", "d_o"):
+        dev[name] = dev[name].permute(0, 2, 1, 3).contiguous().permute(0, 2, 1, 3)
+    status = torch.zeros(binding.STATUS_WORDS, dtype=torch.int32, device="cuda")
+    o, tau = binding.entmax_attn_fwd(dev["q"], dev["k"], dev["v"], 1.5, True, dev["beta"], dev["gamma"], dev["delta"],
+                                     status=status)
+    dq, dk, dv = (torch.empty_like(dev["q"]) for _ in range(3))
+    st2 = torch.zeros(binding.STATUS_WORDS, dtype=torch.int32, device="cuda")
+    binding.entmax_attn_bwd(dev["q"], dev["k"], dev["v"], tau, dev["d_o"], 1.5, True, dev["beta"], dev["gamma"],
+                            dev["delta"], dq=dq, dk=dk, dv=dv, status=st2)
+    torch.cuda.synchronize()
+    assert int(status[binding.STATUS_FLAGS]) == 0 and int(st2[binding.STATUS_FLAGS]) == 0
+    assert int(status[binding.STATUS_DENSE_ROWS]) > w.B * w.H * 500 and int(st2[binding.STATUS_DENSE_ROWS]) > w.B * w.H * 500
+    assert not dq.is_contiguous()
+    got = {"o": o, "tau": tau}
+    bwd = {"dq": dq, "dk": dk, "dv": dv}
+    for bh in (0, 4, 5):
+        parity.check_fwd_rows(inp, 1.5, got, bh, np.arange(0, 700, 5), check_support=False)
+        parity.check_bwd_head(inp, 1.5, bwd, bh)
+
+
 def test_two_calls_are_bitwise_identical():
     # the lists the sweep leaves vary from run to run (order, surplus candidates); O and tau must not
     for N, d, plant in [(513, 128, 4), (3000, 64, 0)]:
