@@ -31,7 +31,6 @@ using namespace sm100;
 constexpr int TM = 128;            // query rows per item = TMEM lanes
 constexpr int TN = 128;            // keys per K/V tile
 constexpr int kThreadsT = 10 * 32;    // TMA warp, MMA warp, eight consumer warps
-constexpr int kStagesT = 2;
 constexpr int kMaxSweeps = 48;     // 1 max sweep + at most 46 Newton sweeps + the output sweep
 constexpr int kPBytes = TM * TN * 2;
 
@@ -42,7 +41,8 @@ struct TCfg {
   static constexpr int kKBytes = TN * HD * 2;      // also the size of a V tile
   static constexpr int kBarBytes = 256;
   static constexpr int kXchgBytes = 2 * TM * 8;    // one float2 per (half, row): partial sums between the two threads of a row
-  static constexpr int kSmemBytes = kQBytes + kStagesT * 2 * kKBytes + kPBytes + 1024 + kBarBytes + kXchgBytes;
+  static constexpr int kStages = HD == 64 ? 4 : 2;   // K/V ring depth: what fits beside Q and P
+  static constexpr int kSmemBytes = kQBytes + kStages * 2 * kKBytes + kPBytes + 1024 + kBarBytes + kXchgBytes;
   static constexpr int kTmemO = 2 * TN;            // first TMEM column of the O accumulator
 };
 
@@ -92,14 +92,14 @@ __global__ void __launch_bounds__(kThreadsT, 1) tile_fwd_kernel(const __grid_con
   extern __shared__ uint8_t smem_raw[];
   const uint32_t sbase = (smem_u32(smem_raw) + 1023u) & ~1023u;
   const uint32_t q_smem = sbase;
-  const uint32_t k_smem = q_smem + C::kQBytes;                       // [kStagesT] K tiles
-  const uint32_t v_smem = k_smem + kStagesT * C::kKBytes;            // [kStagesT] V tiles
-  const uint32_t p_smem = v_smem + kStagesT * C::kKBytes;            // P tile, A-operand layout
+  const uint32_t k_smem = q_smem + C::kQBytes;                       // [C::kStages] K tiles
+  const uint32_t v_smem = k_smem + C::kStages * C::kKBytes;            // [C::kStages] V tiles
+  const uint32_t p_smem = v_smem + C::kStages * C::kKBytes;            // P tile, A-operand layout
   const uint32_t bars = p_smem + kPBytes;
   const uint32_t q_full = bars, q_empty = bars + 8;
-  const uint32_t kv_full = bars + 16;                                 // [kStagesT]
-  const uint32_t kv_empty = kv_full + 8 * kStagesT;                   // [kStagesT]
-  const uint32_t s_full = kv_empty + 8 * kStagesT;                    // [2]
+  const uint32_t kv_full = bars + 16;                                 // [C::kStages]
+  const uint32_t kv_empty = kv_full + 8 * C::kStages;                   // [C::kStages]
+  const uint32_t s_full = kv_empty + 8 * C::kStages;                    // [2]
   const uint32_t s_empty = s_full + 16;                               // [2]
   const uint32_t p_full = s_empty + 16, p_empty = p_full + 8;
   const uint32_t o_full = p_empty + 8, o_empty = o_full + 8;
@@ -109,7 +109,7 @@ __global__ void __launch_bounds__(kThreadsT, 1) tile_fwd_kernel(const __grid_con
   const uint32_t tmem_slot = x_bar + 8;
   const uint32_t abort_flag = tmem_slot + 4;
   const uint32_t xchg = bars + C::kBarBytes;                          // float2 [2][TM]
-  static_assert(8 * (2 + 2 * kStagesT + 4 + 4 + 1) + 16 + 8 + 8 <= C::kBarBytes, "barrier area");
+  static_assert(8 * (2 + 2 * C::kStages + 4 + 4 + 1) + 16 + 8 + 8 <= C::kBarBytes, "barrier area");
 
   const int warp = threadIdx.x >> 5;
   const int lane = threadIdx.x & 31;
@@ -118,7 +118,7 @@ __global__ void __launch_bounds__(kThreadsT, 1) tile_fwd_kernel(const __grid_con
   if (threadIdx.x == 0) {
     mbar_init(q_full, 1);
     mbar_init(q_empty, 1);
-    for (int t = 0; t < kStagesT; ++t) {
+    for (int t = 0; t < C::kStages; ++t) {
       mbar_init(kv_full + 8 * t, 1);
       mbar_init(kv_empty + 8 * t, 1);
     }
@@ -194,7 +194,7 @@ __global__ void __launch_bounds__(kThreadsT, 1) tile_fwd_kernel(const __grid_con
                 tma_load_4d(v_smem + stage * C::kKBytes + hf * (TN * 128), &map_v, kv_full + 8 * stage, hf * 64, t * TN, h,
                             b);
             }
-            if (++stage == kStagesT) { stage = 0; kvphase ^= 1u; }
+            if (++stage == C::kStages) { stage = 0; kvphase ^= 1u; }
           }
           if (output) break;
         }
@@ -266,7 +266,7 @@ __global__ void __launch_bounds__(kThreadsT, 1) tile_fwd_kernel(const __grid_con
               umma_commit(kv_empty + 8 * stage);
               if (t == tiles - 1) umma_commit(o_full);
             }
-            if (++stage == kStagesT) { stage = 0; kvphase ^= 1u; }
+            if (++stage == C::kStages) { stage = 0; kvphase ^= 1u; }
           }
           if (output) break;
         }
