@@ -30,6 +30,10 @@
  *   - Functions return ENTMAX_ATTN_OK (0) or a negative entmax_attn_status; on a negative return
  *     nothing has been enqueued.  Device-side conditions are reported through `device_status`.
  *   - Non-finite values in Q, K, V or dO give unspecified results (never a fault).
+ *   - Sequences of different lengths in one batch: pad them on the right.  Under the causal mask a valid
+ *     row never sees a padded key, so no extra mask is needed; give the padded rows dO = 0 and their
+ *     content cannot reach dK, dV either (their own O, tau, dQ rows are to be ignored).  Non-causal
+ *     problems have no padding mask.
  */
 #ifndef ENTMAX_ATTN_H_
 #define ENTMAX_ATTN_H_

@@ -196,6 +196,31 @@ def test_dense_tiles_with_strided_layout_and_batches(d):
         parity.check_bwd_head(inp, 1.5, bwd, bh)
 
 
+def test_right_padded_sequences_need_no_mask_under_the_causal_mask():
+    # a batch of sequences of different lengths, right-padded to N: a valid row i < L sees only keys j <= i < L, so
+    # whatever sits in the padding cannot reach it; with dO = 0 on the padding rows it cannot reach dK, dV either
+    inp = make_inputs(_small("padded", 1000, 64, True, plant=2, backward=True, seed=71))
+    L = 700
+    dev = parity.to_device(inp)
+    dev["d_o"][:, :, L:] = 0
+    o1, tau1 = binding.entmax_attn_fwd(dev["q"], dev["k"], dev["v"], 1.5, True, dev["beta"], dev["gamma"], dev["delta"])
+    g1 = binding.entmax_attn_bwd(dev["q"], dev["k"], dev["v"], tau1, dev["d_o"], 1.5, True, dev["beta"], dev["gamma"],
+                                 dev["delta"])
+    gen = torch.Generator(device="cuda").manual_seed(3)
+    for name in ("q", "k", "v"):
+        junk = torch.randn(dev[name][:, :, L:].shape, generator=gen, device="cuda") * 50.0
+        dev[name][:, :, L:] = junk.to(dev[name].dtype)
+    o2, tau2 = binding.entmax_attn_fwd(dev["q"], dev["k"], dev["v"], 1.5, True, dev["beta"], dev["gamma"], dev["delta"])
+    g2 = binding.entmax_attn_bwd(dev["q"], dev["k"], dev["v"], tau2, dev["d_o"], 1.5, True, dev["beta"], dev["gamma"],
+                                 dev["delta"])
+    torch.cuda.synchronize()
+    assert torch.equal(o1[:, :, :L], o2[:, :, :L]) and torch.equal(tau1[:, :, :L], tau2[:, :, :L])
+    assert torch.equal(g1[0][:, :, :L], g2[0][:, :, :L])                       # dQ of the valid rows
+    for a_, b_ in zip(g1[1:], g2[1:]):                                         # dK, dV of the valid keys
+        ref = a_[:, :, :L].float()
+        assert (ref - b_[:, :, :L].float()).abs().max().item() <= 1e-2 * max(1.0, ref.abs().max().item())
+
+
 def test_two_calls_are_bitwise_identical():
     # the lists the sweep leaves vary from run to run (order, surplus candidates); O and tau must not
     for N, d, plant in [(513, 128, 4), (3000, 64, 0)]:
