@@ -459,6 +459,6 @@ const char* entmax_attn_strerror(int code) {
 
 int entmax_attn_last_cuda_error(void) { return g_last_cuda_error; }
 
-int entmax_attn_version(void) { return 100; }
+int entmax_attn_version(void) { return 200; }   // 0.2.0: decode entry point, dense-tile backward
 
 }  // extern "C"
