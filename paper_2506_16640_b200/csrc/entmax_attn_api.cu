@@ -15,6 +15,38 @@ thread_local cudaEvent_t g_prof_stop[2] = {nullptr, nullptr};
 
 inline size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
 
+// A second stream per (host thread, device) on which the backward call clears its fp32 accumulators while the
+// score sweep, which does not touch them, runs on the caller's stream: forked from and joined back to the
+// caller's stream with events, so the caller sees ordinary stream order (and a stream capture stays one graph).
+struct SideStream {
+  cudaStream_t stream = nullptr;
+  cudaEvent_t fork = nullptr, join = nullptr;
+};
+thread_local SideStream g_side[64];
+
+cudaError_t side_stream(SideStream** out) {
+  int dev = 0;
+  cudaError_t err = cudaGetDevice(&dev);
+  if (err != cudaSuccess) return err;
+  if (dev < 0 || dev >= 64) return cudaErrorInvalidDevice;
+  SideStream& s = g_side[dev];
+  if (!s.stream) {
+    cudaStream_t st = nullptr;
+    cudaEvent_t e0 = nullptr, e1 = nullptr;
+    err = cudaStreamCreateWithFlags(&st, cudaStreamNonBlocking);
+    if (err == cudaSuccess) err = cudaEventCreateWithFlags(&e0, cudaEventDisableTiming);
+    if (err == cudaSuccess) err = cudaEventCreateWithFlags(&e1, cudaEventDisableTiming);
+    if (err != cudaSuccess) {
+      if (e0) cudaEventDestroy(e0);
+      if (st) cudaStreamDestroy(st);
+      return err;
+    }
+    s.stream = st; s.fork = e0; s.join = e1;
+  }
+  *out = &s;
+  return cudaSuccess;
+}
+
 int fail_cuda(cudaError_t err) {
   g_last_cuda_error = (int)err;
   return ENTMAX_ATTN_ECUDA;
@@ -299,10 +331,24 @@ int bwd_impl(const entmax_attn_params* params, const void* q, const void* k, con
     err = cudaMemsetAsync(device_status, 0, sizeof(int32_t) * ENTMAX_ATTN_STATUS_WORDS, stream);
     if (err != cudaSuccess) return fail_cuda(err);
   }
-  err = cudaMemsetAsync(acc_dk, 0, acc_bytes, stream);
-  if (err != cudaSuccess) return fail_cuda(err);
-  err = cudaMemsetAsync(acc_dv, 0, acc_bytes, stream);
-  if (err != cudaSuccess) return fail_cuda(err);
+  // with a score sweep ahead (bf16, no saved supports) the accumulators are cleared beside it, otherwise in line
+  const bool clear_aside = p.dtype == ENTMAX_ATTN_DTYPE_BF16 && !fwd_workspace;
+  SideStream* side = nullptr;
+  if (clear_aside) {
+    err = side_stream(&side);
+    if (err != cudaSuccess) return fail_cuda(err);
+    err = cudaEventRecord(side->fork, stream);
+    if (err == cudaSuccess) err = cudaStreamWaitEvent(side->stream, side->fork, 0);
+    if (err == cudaSuccess) err = cudaMemsetAsync(acc_dk, 0, acc_bytes, side->stream);
+    if (err == cudaSuccess) err = cudaMemsetAsync(acc_dv, 0, acc_bytes, side->stream);
+    if (err == cudaSuccess) err = cudaEventRecord(side->join, side->stream);
+    if (err != cudaSuccess) return fail_cuda(err);
+  } else {
+    err = cudaMemsetAsync(acc_dk, 0, acc_bytes, stream);
+    if (err != cudaSuccess) return fail_cuda(err);
+    err = cudaMemsetAsync(acc_dv, 0, acc_bytes, stream);
+    if (err != cudaSuccess) return fail_cuda(err);
+  }
   if (c_rows) {
     scale = c_rows;
     p.scale_sb = (int64_t)p.H * p.N;
@@ -339,6 +385,8 @@ int bwd_impl(const entmax_attn_params* params, const void* q, const void* k, con
                          stream);
       if (err != cudaSuccess) return fail_cuda(err);
       if (g_prof_stop[1]) cudaEventRecord(g_prof_stop[1], stream);
+      err = cudaStreamWaitEvent(stream, side->join, 0);     // the accumulators are clear from here on
+      if (err != cudaSuccess) return fail_cuda(err);
       err = launch_row_bwd(p, q, k, v, d_o, scale, tau, half_cnt, entries, dq, acc_dk, acc_dv, dc_rows, fb_count,
                            fb_list, device_status, 0, stream);
       if (err != cudaSuccess) return fail_cuda(err);
