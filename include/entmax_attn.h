@@ -21,8 +21,10 @@
  *
  * General conventions
  *   - Every tensor pointer is a DEVICE pointer owned by the caller.  The library allocates no device
- *     memory, never synchronises the device or a stream, and enqueues all work on `cuda_stream`
- *     (a cudaStream_t passed as void*; NULL = the legacy default stream).
+ *     memory, never synchronises the device or a stream, and enqueues all work in the order of
+ *     `cuda_stream` (a cudaStream_t passed as void*; NULL = the legacy default stream).  The backward
+ *     calls clear their accumulators on a stream of the library's own that is forked from and joined
+ *     back to `cuda_stream` with events inside the call: the caller sees plain stream order.
  *   - Q, K, V, O, dO, dQ, dK, dV share one layout: [batch, heads, seq, head_dim] with head_dim
  *     innermost and contiguous; the other three strides come from the params struct (in elements).
  *     tau is [batch, heads, seq] float32, contiguous.  beta, gamma, delta are [heads] float32.
