@@ -223,7 +223,24 @@ def run_ours(args):
         b_stop[j].record()
     torch.cuda.synchronize()
     bwd_saved_ms = sum(a.elapsed_time(b) for a, b in zip(b_start, b_stop)) / K
-    del ws_fwd
+    # the same with the compact copy of the supports (260 bytes per row instead of the whole forward workspace):
+    # the copy itself and the backward pass fed with it are timed together
+    saved = binding.entmax_attn_save_supports(d["q"], alpha, w.causal, ws_fwd)
+    c_start, c_stop = [ev() for _ in range(K)], [ev() for _ in range(K)]
+    for i in range(K + 2):
+        binding.entmax_attn_fwd(d["q"], d["k"], d["v"], alpha, w.causal, d["beta"], d["gamma"], d["delta"], o=o, tau=tau,
+                                workspace=ws_fwd, status=status)
+        j = max(i - 2, 0)
+        c_start[j].record()
+        binding.entmax_attn_save_supports(d["q"], alpha, w.causal, ws_fwd, saved=saved)
+        binding.entmax_attn_bwd_ex(d["q"], d["k"], d["v"], tau, d["d_o"], alpha, w.causal, d["beta"], d["gamma"],
+                                   d["delta"], saved_supports=saved, dq=dq, dk=dk, dv=dv, workspace=ws, status=status)
+        c_stop[j].record()
+    torch.cuda.synchronize()
+    bwd_compact_ms = sum(a.elapsed_time(b) for a, b in zip(c_start, c_stop)) / K
+    compact_recomputed = int(status[binding.STATUS_DENSE_ROWS].item())
+    saved_bytes = saved.numel()
+    del ws_fwd, saved
 
     # secondary: the decode shape on the same tensors: the last q_len rows of Q as the new queries, K and V as the cache
     decode = time_decode(d, w, alpha, flush) if world == 1 else None
@@ -328,6 +345,10 @@ def run_ours(args):
         "bwd_with_saved_forward_workspace": {"ms": bwd_saved_ms, "tflops": f_bwd / (bwd_saved_ms * 1e-3) / 1e12,
                                              "note": "not part of `value`: entmax_attn_bwd_ex given the forward call's "
                                                      "workspace reuses its support lists instead of sweeping QK^T again"},
+        "bwd_with_compact_saved_supports": {"ms": bwd_compact_ms, "tflops": f_bwd / (bwd_compact_ms * 1e-3) / 1e12,
+                                            "saved_bytes": saved_bytes, "rows_recomputed": compact_recomputed,
+                                            "note": "not part of `value`: entmax_attn_save_supports after the forward call "
+                                                    "+ entmax_attn_bwd_ex fed with the compact copy"},
         "tau_search_extra": {"tensor_flops": 0, "note": "single score sweep: the threshold is solved on the per-row "
                              "candidate lists, no extra QK^T pass", "dense_fallback_rows": dense_rows},
         # the sweep is timed inside the back-to-back step loop (power cap active, see `clocks`): the sustained

@@ -170,7 +170,22 @@ typedef struct {
                                 inputs, untouched since it returned.  It still holds the support of every row, so
                                 the backward pass skips its own score sweep (which otherwise recomputes Q K^T to
                                 find the support from tau).  Must not be the buffer passed as `workspace`.        */
+  const void* saved_supports; /* backward only, bfloat16 problems: the compact copy entmax_attn_save_supports made
+                                of the forward call's supports (takes precedence over fwd_workspace).              */
 } entmax_attn_extras;
+/* Compact saved state for the backward pass.  Keeping the whole forward workspace alive until the backward
+ * pass costs about 2 KB per query row; the supports themselves are a few entries per row.  This call copies,
+ * for every row, its support size and up to ENTMAX_ATTN_SAVED_SLOTS support entries out of a finished forward
+ * call's workspace into `saved` (entmax_attn_saved_bytes(params) bytes, 256-byte aligned: 4 + 8 *
+ * ENTMAX_ATTN_SAVED_SLOTS bytes per row).  Passed as extras.saved_supports, it lets the backward pass skip its
+ * score sweep like fwd_workspace does; rows whose support has more entries than the slots, and rows the
+ * dense-tile path computed, are recomputed on the tensor cores instead.  bfloat16 problems only.  (The paper
+ * has no counterpart: it does not discuss what the backward pass keeps.) */
+#define ENTMAX_ATTN_SAVED_SLOTS 32
+size_t entmax_attn_saved_bytes(const entmax_attn_params* params);
+int entmax_attn_save_supports(const entmax_attn_params* params, const void* fwd_workspace, void* saved,
+                              size_t saved_bytes, void* cuda_stream);
+
 int entmax_attn_fwd_ex(const entmax_attn_params* params, const void* q, const void* k, const void* v,
                        const float* beta, const float* gamma, const float* delta, const entmax_attn_extras* extras,
                        void* o, float* tau, void* workspace, size_t workspace_bytes, int32_t* device_status,

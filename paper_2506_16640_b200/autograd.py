@@ -7,8 +7,8 @@ the temperature c_i = delta_h + beta_h (log n_i)^gamma_h is learnable), or with 
 scale table ``c_rows`` [B,H,N] when the caller evaluates the paper's content-dependent beta, gamma itself
 (Sec. 4.1) and wants dL/dc_i back.  Every number comes from entmax_attn_fwd_ex / entmax_attn_bwd_ex.
 
-``keep_supports=True`` keeps the forward call's workspace alive until the backward pass, which then
-reuses the supports it holds instead of sweeping Q K^T again (about 2 KB of workspace per query row).
+``keep_supports=True`` keeps a compact copy of every row's support (260 bytes per query row, made by
+entmax_attn_save_supports) until the backward pass, which then skips its score sweep: no second Q K^T.
 """
 from __future__ import annotations
 
@@ -23,13 +23,15 @@ class _EntmaxAttention(torch.autograd.Function):
     @staticmethod
     def forward(ctx, q, k, v, beta, gamma, delta, c_rows, alibi_slopes, alpha, causal, sm_scale, keep_supports):
         params = binding.make_params(q, alpha, causal, sm_scale, 0)
-        ws = binding.alloc_workspace(params, False, q.device) if keep_supports else None
+        ws = binding.alloc_workspace(params, False, q.device) if keep_supports and q.dtype == torch.bfloat16 else None
+        keep_supports = ws is not None
         det = lambda t: None if t is None else t.detach()
         o, tau = binding.entmax_attn_fwd_ex(q.detach(), k.detach(), v.detach(), alpha, causal, det(beta), det(gamma),
                                             det(delta), c_rows=det(c_rows), alibi_slopes=det(alibi_slopes),
                                             sm_scale=sm_scale, workspace=ws)
+        saved = binding.entmax_attn_save_supports(q, alpha, causal, ws, sm_scale=sm_scale) if keep_supports else None
         ctx.save_for_backward(q, k, v, beta, gamma, delta, c_rows, alibi_slopes, tau)
-        ctx.alpha, ctx.causal, ctx.sm_scale, ctx.fwd_workspace = alpha, causal, sm_scale, ws
+        ctx.alpha, ctx.causal, ctx.sm_scale, ctx.saved_supports = alpha, causal, sm_scale, saved
         ctx.mark_non_differentiable(tau)
         return o, tau
 
@@ -41,9 +43,9 @@ class _EntmaxAttention(torch.autograd.Function):
         want_rows = c_rows is not None and ctx.needs_input_grad[6]
         dq, dk, dv, dc, grads = binding.entmax_attn_bwd_ex(
             q.detach(), k.detach(), v.detach(), tau, d_o.contiguous(), ctx.alpha, ctx.causal, det(beta), det(gamma),
-            det(delta), c_rows=det(c_rows), alibi_slopes=det(alibi_slopes), fwd_workspace=ctx.fwd_workspace,
+            det(delta), c_rows=det(c_rows), alibi_slopes=det(alibi_slopes), saved_supports=ctx.saved_supports,
             want_scale_rows=want_rows, want_param_grads=want_params, sm_scale=ctx.sm_scale)
-        ctx.fwd_workspace = None
+        ctx.saved_supports = None
         db, dg, dd = grads if grads is not None else (None, None, None)
         return dq, dk, dv, db, dg, dd, (dc if want_rows else None), None, None, None, None, None
 

@@ -43,7 +43,7 @@ class WsLayout(ctypes.Structure):
 class Extras(ctypes.Structure):
     _fields_ = [("c_rows", ctypes.c_void_p), ("alibi_slopes", ctypes.c_void_p), ("d_scale_rows", ctypes.c_void_p),
                 ("dbeta", ctypes.c_void_p), ("dgamma", ctypes.c_void_p), ("ddelta", ctypes.c_void_p),
-                ("fwd_workspace", ctypes.c_void_p)]
+                ("fwd_workspace", ctypes.c_void_p), ("saved_supports", ctypes.c_void_p)]
 
 
 class EntmaxAttnError(RuntimeError):
@@ -91,6 +91,10 @@ def load():
         lib.entmax_attn_decode_workspace_bytes.argtypes = [dp]
         lib.entmax_attn_decode_fwd.restype = ctypes.c_int
         lib.entmax_attn_decode_fwd.argtypes = [dp, vp, vp, vp, ip, fp, fp, fp, fp, vp, fp, ip, vp, ctypes.c_size_t, ip, vp]
+        lib.entmax_attn_saved_bytes.restype = ctypes.c_size_t
+        lib.entmax_attn_saved_bytes.argtypes = [pp]
+        lib.entmax_attn_save_supports.restype = ctypes.c_int
+        lib.entmax_attn_save_supports.argtypes = [pp, vp, vp, ctypes.c_size_t, vp]
         lib.entmax_attn_scores_debug.restype = ctypes.c_int
         lib.entmax_attn_scores_debug.argtypes = [pp, vp, vp, ctypes.c_int32, fp, vp, ctypes.c_size_t, ip, vp]
         lib.entmax_attn_profile_events.restype = ctypes.c_int
@@ -336,8 +340,23 @@ def entmax_attn_fwd_ex(q, k, v, alpha, causal, beta=None, gamma=None, delta=None
     return o, tau
 
 
+def entmax_attn_save_supports(q, alpha, causal, fwd_workspace, *, sm_scale=0.0, n_mode=0, saved=None, stream=None):
+    """Compact copy of a finished forward call's supports (uint8 CUDA tensor) for entmax_attn_bwd_ex(saved_supports=...)."""
+    params = make_params(q, alpha, causal, sm_scale, n_mode)
+    nbytes = load().entmax_attn_saved_bytes(ctypes.byref(params))
+    if nbytes == 0:
+        raise EntmaxAttnError("entmax_attn_saved_bytes: invalid parameters (bf16 problems only)")
+    if saved is None:
+        saved = torch.empty(nbytes, dtype=torch.uint8, device=q.device)
+    rc = load().entmax_attn_save_supports(ctypes.byref(params), _ptr(fwd_workspace), _ptr(saved), saved.numel(),
+                                          _stream_ptr(stream))
+    _check(rc, "entmax_attn_save_supports")
+    return saved
+
+
 def entmax_attn_bwd_ex(q, k, v, tau, d_o, alpha, causal, beta=None, gamma=None, delta=None, *, c_rows=None,
-                       alibi_slopes=None, fwd_workspace=None, want_scale_rows=False, want_param_grads=False,
+                       alibi_slopes=None, fwd_workspace=None, saved_supports=None, want_scale_rows=False,
+                       want_param_grads=False,
                        sm_scale=0.0, n_mode=0, dq=None, dk=None, dv=None, workspace=None, status=None, stream=None):
     """Extended backward pass.  `fwd_workspace`: the forward call's workspace tensor, untouched since
     (the backward pass then reuses the supports it holds instead of sweeping Q K^T again).
@@ -353,7 +372,8 @@ def entmax_attn_bwd_ex(q, k, v, tau, d_o, alpha, causal, beta=None, gamma=None, 
     g = grads if grads is not None else (None, None, None)
     if workspace is None:
         workspace = alloc_workspace(params, True, q.device)
-    ex = Extras(_dp(c_rows), _dp(alibi_slopes), _dp(dc), _dp(g[0]), _dp(g[1]), _dp(g[2]), _dp(fwd_workspace))
+    ex = Extras(_dp(c_rows), _dp(alibi_slopes), _dp(dc), _dp(g[0]), _dp(g[1]), _dp(g[2]), _dp(fwd_workspace),
+                _dp(saved_supports))
     rc = load().entmax_attn_bwd_ex(ctypes.byref(params), _ptr(q), _ptr(k), _ptr(v), _ptr(beta), _ptr(gamma), _ptr(delta),
                                    ctypes.byref(ex), _ptr(tau), _ptr(d_o), _ptr(dq), _ptr(dk), _ptr(dv), _ptr(workspace),
                                    workspace.numel(), _ptr(status), _stream_ptr(stream))

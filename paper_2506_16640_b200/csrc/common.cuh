@@ -140,7 +140,10 @@ cudaError_t launch_row_fwd(const Problem& p, const void* v, const float* scale, 
 cudaError_t launch_row_bwd(const Problem& p, const void* q, const void* k, const void* v, const void* d_o,
                            const float* scale, const float* tau, const int32_t* half_cnt, Entry* entries, void* dq,
                            float* acc_dk, float* acc_dv, float* dc_rows, int32_t* fb_count, int32_t* fb_list,
-                           int32_t* status, int saved, cudaStream_t stream);
+                           int32_t* status, int saved, int pitch, cudaStream_t stream);
+// compact copy of the forward call's supports (see entmax_attn_save_supports)
+cudaError_t launch_save_supports(const Problem& p, int slots, const int32_t* row_cnt, const Entry* entries,
+                                 int32_t* out_cnt, Entry* out_entries, cudaStream_t stream);
 
 // fp32 accumulators [B,H,N,D] contiguous -> strided output tensor of the problem dtype
 cudaError_t launch_store_grad(const Problem& p, const float* acc, void* out, cudaStream_t stream);

@@ -47,6 +47,18 @@ cudaError_t side_stream(SideStream** out) {
   return cudaSuccess;
 }
 
+struct SavedLayout {
+  size_t counts, entries, total;
+};
+SavedLayout saved_layout(const Problem& p) {
+  const size_t rows = (size_t)p.B * p.H * p.N;
+  SavedLayout l;
+  l.counts = 0;
+  l.entries = align_up(rows * sizeof(int32_t), 256);
+  l.total = l.entries + align_up(rows * ENTMAX_ATTN_SAVED_SLOTS * sizeof(Entry), 256);
+  return l;
+}
+
 int fail_cuda(cudaError_t err) {
   g_last_cuda_error = (int)err;
   return ENTMAX_ATTN_ECUDA;
@@ -285,7 +297,7 @@ namespace {
 
 int bwd_impl(const entmax_attn_params* params, const void* q, const void* k, const void* v, const float* beta,
              const float* gamma, const float* delta, const float* c_rows, const float* alibi,
-             const void* fwd_workspace, const float* tau, const void* d_o, void* dq,
+             const void* fwd_workspace, const void* saved_supports, const float* tau, const void* d_o, void* dq,
              void* dk, void* dv, float* d_scale_rows, float* dbeta, float* dgamma, float* ddelta, void* workspace,
              size_t workspace_bytes, int32_t* device_status, void* cuda_stream) {
   Problem p;
@@ -332,7 +344,7 @@ int bwd_impl(const entmax_attn_params* params, const void* q, const void* k, con
     if (err != cudaSuccess) return fail_cuda(err);
   }
   // with a score sweep ahead (bf16, no saved supports) the accumulators are cleared beside it, otherwise in line
-  const bool clear_aside = p.dtype == ENTMAX_ATTN_DTYPE_BF16 && !fwd_workspace;
+  const bool clear_aside = p.dtype == ENTMAX_ATTN_DTYPE_BF16 && !fwd_workspace && !saved_supports;
   SideStream* side = nullptr;
   if (clear_aside) {
     err = side_stream(&side);
@@ -371,13 +383,21 @@ int bwd_impl(const entmax_attn_params* params, const void* q, const void* k, con
     // tile flags, tile list and tile masks are adjacent in the workspace: one memset clears all three
     err = cudaMemsetAsync(tile_flag, 0, lay.tile_mask + q_tiles * 4 * sizeof(uint32_t) - lay.tile_flag, stream);
     if (err != cudaSuccess) return fail_cuda(err);
-    if (fwd_workspace) {
+    if (saved_supports) {
+      // the compact copy of the forward call's supports: no score sweep; rows it does not hold count as dense
+      const SavedLayout sl = saved_layout(p);
+      const uint8_t* sv = static_cast<const uint8_t*>(saved_supports);
+      err = launch_row_bwd(p, q, k, v, d_o, scale, tau, reinterpret_cast<const int32_t*>(sv + sl.counts),
+                           const_cast<Entry*>(reinterpret_cast<const Entry*>(sv + sl.entries)), dq, acc_dk, acc_dv,
+                           dc_rows, fb_count, fb_list, device_status, 1, ENTMAX_ATTN_SAVED_SLOTS, stream);
+      if (err != cudaSuccess) return fail_cuda(err);
+    } else if (fwd_workspace) {
       // the forward call's workspace still holds every row's support: no score sweep needed
       const WsLayout fl = make_layout(p, false);
       const uint8_t* fws = static_cast<const uint8_t*>(fwd_workspace);
       err = launch_row_bwd(p, q, k, v, d_o, scale, tau, reinterpret_cast<const int32_t*>(fws + fl.row_cnt),
                            const_cast<Entry*>(reinterpret_cast<const Entry*>(fws + fl.entries)), dq, acc_dk, acc_dv,
-                           dc_rows, fb_count, fb_list, device_status, 1, stream);
+                           dc_rows, fb_count, fb_list, device_status, 1, kListCap, stream);
       if (err != cudaSuccess) return fail_cuda(err);
     } else {
       if (g_prof_start[1]) cudaEventRecord(g_prof_start[1], stream);
@@ -388,7 +408,7 @@ int bwd_impl(const entmax_attn_params* params, const void* q, const void* k, con
       err = cudaStreamWaitEvent(stream, side->join, 0);     // the accumulators are clear from here on
       if (err != cudaSuccess) return fail_cuda(err);
       err = launch_row_bwd(p, q, k, v, d_o, scale, tau, half_cnt, entries, dq, acc_dk, acc_dv, dc_rows, fb_count,
-                           fb_list, device_status, 0, stream);
+                           fb_list, device_status, 0, kListCap, stream);
       if (err != cudaSuccess) return fail_cuda(err);
     }
     // rows whose support does not fit the lists: dense tiles on the tensor cores
@@ -416,7 +436,7 @@ int entmax_attn_bwd_scale(const entmax_attn_params* params, const void* q, const
                           const void* d_o, void* dq, void* dk, void* dv, float* d_scale_rows, float* dbeta,
                           float* dgamma, float* ddelta, void* workspace, size_t workspace_bytes,
                           int32_t* device_status, void* cuda_stream) {
-  return bwd_impl(params, q, k, v, beta, gamma, delta, nullptr, nullptr, nullptr, tau, d_o, dq, dk, dv, d_scale_rows, dbeta,
+  return bwd_impl(params, q, k, v, beta, gamma, delta, nullptr, nullptr, nullptr, nullptr, tau, d_o, dq, dk, dv, d_scale_rows, dbeta,
                   dgamma, ddelta, workspace, workspace_bytes, device_status, cuda_stream);
 }
 
@@ -428,7 +448,9 @@ int entmax_attn_bwd_ex(const entmax_attn_params* params, const void* q, const vo
   if (extras) ex = *extras;
   if (ex.c_rows && (beta || gamma || delta)) return ENTMAX_ATTN_EINVAL_NULL;
   if (ex.fwd_workspace && (reinterpret_cast<uintptr_t>(ex.fwd_workspace) & 255u)) return ENTMAX_ATTN_EINVAL_WORKSPACE;
-  return bwd_impl(params, q, k, v, beta, gamma, delta, ex.c_rows, ex.alibi_slopes, ex.fwd_workspace, tau, d_o, dq, dk, dv,
+  if (ex.saved_supports && (reinterpret_cast<uintptr_t>(ex.saved_supports) & 255u)) return ENTMAX_ATTN_EINVAL_WORKSPACE;
+  return bwd_impl(params, q, k, v, beta, gamma, delta, ex.c_rows, ex.alibi_slopes, ex.fwd_workspace, ex.saved_supports, tau,
+                  d_o, dq, dk, dv,
                   ex.d_scale_rows, ex.dbeta, ex.dgamma, ex.ddelta, workspace, workspace_bytes, device_status,
                   cuda_stream);
 }
@@ -438,7 +460,7 @@ int entmax_attn_bwd_rowscale(const entmax_attn_params* params, const void* q, co
                              float* d_scale_rows, void* workspace, size_t workspace_bytes, int32_t* device_status,
                              void* cuda_stream) {
   if (!c_rows) return ENTMAX_ATTN_EINVAL_NULL;
-  return bwd_impl(params, q, k, v, nullptr, nullptr, nullptr, c_rows, nullptr, nullptr, tau, d_o, dq, dk, dv, d_scale_rows,
+  return bwd_impl(params, q, k, v, nullptr, nullptr, nullptr, c_rows, nullptr, nullptr, nullptr, tau, d_o, dq, dk, dv, d_scale_rows,
                   nullptr, nullptr, nullptr, workspace, workspace_bytes, device_status, cuda_stream);
 }
 
@@ -478,6 +500,33 @@ int entmax_attn_scores_debug(const entmax_attn_params* params, const void* q, co
   err = launch_sweep(p, q, k, scale, nullptr, 0, reinterpret_cast<int32_t*>(ws + lay.half_cnt),
                      reinterpret_cast<float*>(ws + lay.half_thr), reinterpret_cast<Entry*>(ws + lay.entries),
                      reinterpret_cast<int32_t*>(ws + lay.sweep_counter), s_out, bh, device_status, stream);
+  return err == cudaSuccess ? ENTMAX_ATTN_OK : fail_cuda(err);
+}
+
+size_t entmax_attn_saved_bytes(const entmax_attn_params* params) {
+  Problem p;
+  if (make_problem(params, &p) != ENTMAX_ATTN_OK || p.dtype != ENTMAX_ATTN_DTYPE_BF16) return 0;
+  return saved_layout(p).total;
+}
+
+int entmax_attn_save_supports(const entmax_attn_params* params, const void* fwd_workspace, void* saved, size_t saved_bytes,
+                              void* cuda_stream) {
+  Problem p;
+  int rc = make_problem(params, &p);
+  if (rc != ENTMAX_ATTN_OK) return rc;
+  if (p.dtype != ENTMAX_ATTN_DTYPE_BF16) return ENTMAX_ATTN_EINVAL_DTYPE;
+  if (!fwd_workspace || !saved) return ENTMAX_ATTN_EINVAL_NULL;
+  const SavedLayout sl = saved_layout(p);
+  if ((reinterpret_cast<uintptr_t>(fwd_workspace) & 255u) || (reinterpret_cast<uintptr_t>(saved) & 255u) ||
+      saved_bytes < sl.total)
+    return ENTMAX_ATTN_EINVAL_WORKSPACE;
+  const WsLayout fl = make_layout(p, false);
+  const uint8_t* fws = static_cast<const uint8_t*>(fwd_workspace);
+  uint8_t* sv = static_cast<uint8_t*>(saved);
+  cudaError_t err = launch_save_supports(p, ENTMAX_ATTN_SAVED_SLOTS, reinterpret_cast<const int32_t*>(fws + fl.row_cnt),
+                                         reinterpret_cast<const Entry*>(fws + fl.entries),
+                                         reinterpret_cast<int32_t*>(sv + sl.counts), reinterpret_cast<Entry*>(sv + sl.entries),
+                                         static_cast<cudaStream_t>(cuda_stream));
   return err == cudaSuccess ? ENTMAX_ATTN_OK : fail_cuda(err);
 }
 

@@ -681,7 +681,7 @@ __device__ __noinline__ void bwd_row_full(const Problem& p, const __nv_bfloat16*
                                              const float* __restrict__ tau_in, const Entry* __restrict__ entries,
                                              __nv_bfloat16* __restrict__ dq, float* __restrict__ acc_dk,
                                              float* __restrict__ acc_dv, float* __restrict__ dc_rows, int grow, int c0,
-                                             int c1, bool saved, int lane) {
+                                             int c1, bool saved, int pitch, int lane) {
   constexpr int PER = D / 32;
   const int bh = grow / p.N, i = grow - bh * p.N, b = bh / p.H, h = bh - b * p.H;
   const float g = scale[(size_t)b * p.scale_sb + (size_t)h * p.N + i] * p.sm_scale;
@@ -691,7 +691,7 @@ __device__ __noinline__ void bwd_row_full(const Problem& p, const __nv_bfloat16*
   float qs[PER], gs[PER];
   load_bf16<PER>(q + hbase + (size_t)i * p.sn, qs);
   load_bf16<PER>(d_o + hbase + (size_t)i * p.sn, gs);
-  const Entry* list = entries + (size_t)grow * kListCap;
+  const Entry* list = entries + (size_t)grow * pitch;
   float yv[kSlots], dpv[kSlots], zz[kSlots];
   int jj[kSlots];
 #pragma unroll
@@ -801,7 +801,7 @@ __device__ __forceinline__ void bwd_rows_sub(const Problem& p, const __nv_bfloat
                                              const float* __restrict__ tau_in, const Entry* __restrict__ entries,
                                              __nv_bfloat16* __restrict__ dq, float* __restrict__ acc_dk,
                                              float* __restrict__ acc_dv, float* __restrict__ dc_rows, int grow,
-                                             bool active, int c0, int c1, bool saved, int lane) {
+                                             bool active, int c0, int c1, bool saved, int pitch, int lane) {
   constexpr int PL = D / W;                        // elements of a row per lane
   constexpr unsigned kWMask = W == 32 ? 0xffffffffu : ((1u << (W & 31)) - 1u);
   const int sl = lane & (W - 1);
@@ -815,7 +815,7 @@ __device__ __forceinline__ void bwd_rows_sub(const Problem& p, const __nv_bfloat
   float qs[PL], gs[PL];
   load_slice_bf16<PL>(q + hbase + (size_t)i * p.sn, qs);
   load_slice_bf16<PL>(d_o + hbase + (size_t)i * p.sn, gs);
-  const Entry* list = entries + (size_t)grow * kListCap;
+  const Entry* list = entries + (size_t)grow * pitch;
   float yv = -1.0f, zz = 0.f;
   int j = 0;
   if (sl < n) {
@@ -888,9 +888,9 @@ __global__ void __launch_bounds__(kWarpsPerCta * 32, 4) row_bwd_kernel(
     const __nv_bfloat16* __restrict__ v, const __nv_bfloat16* __restrict__ d_o, const float* __restrict__ scale,
     const float* __restrict__ tau_in, const int32_t* __restrict__ half_cnt, const Entry* __restrict__ entries,
     __nv_bfloat16* __restrict__ dq, float* __restrict__ acc_dk, float* __restrict__ acc_dv,
-    float* __restrict__ dc_rows, int32_t* fb_count, int32_t* fb_list, int32_t* status, int saved) {
+    float* __restrict__ dc_rows, int32_t* fb_count, int32_t* fb_list, int32_t* status, int saved, int pitch) {
   // saved != 0: `half_cnt` is the forward pass's final support size per row (one int per row, -2 = dense
-  // row) and `entries` its compacted support lists
+  // row) and `entries` its compacted support lists; `pitch` = list slots per row in `entries`
   const int lane = threadIdx.x & 31;
   const int total = p.B * p.H * p.N;
   const int blocks = (total + 15) / 16;
@@ -920,7 +920,7 @@ __global__ void __launch_bounds__(kWarpsPerCta * 32, 4) row_bwd_kernel(
       const bool active = src < 32u;
       const int c0 = __shfl_sync(0xffffffffu, mc0, active ? src : 0), c1 = __shfl_sync(0xffffffffu, mc1, active ? src : 0);
       bwd_rows_sub<D, 8>(p, q, k, v, d_o, scale, tau_in, entries, dq, acc_dk, acc_dv, dc_rows,
-                         active ? 16 * blk + (int)src : 0, active, c0, c1, saved != 0, lane);
+                         active ? 16 * blk + (int)src : 0, active, c0, c1, saved != 0, pitch, lane);
 #pragma unroll
       for (int t = 0; t < 4; ++t) m8 &= m8 - 1;
     }
@@ -929,7 +929,7 @@ __global__ void __launch_bounds__(kWarpsPerCta * 32, 4) row_bwd_kernel(
       const bool active = src < 32u;
       const int c0 = __shfl_sync(0xffffffffu, mc0, active ? src : 0), c1 = __shfl_sync(0xffffffffu, mc1, active ? src : 0);
       bwd_rows_sub<D, 16>(p, q, k, v, d_o, scale, tau_in, entries, dq, acc_dk, acc_dv, dc_rows,
-                          active ? 16 * blk + (int)src : 0, active, c0, c1, saved != 0, lane);
+                          active ? 16 * blk + (int)src : 0, active, c0, c1, saved != 0, pitch, lane);
       m16 &= m16 - 1;
       m16 &= m16 - 1;
     }
@@ -938,7 +938,7 @@ __global__ void __launch_bounds__(kWarpsPerCta * 32, 4) row_bwd_kernel(
       m32 &= m32 - 1;
       const int c0 = __shfl_sync(0xffffffffu, mc0, src), c1 = __shfl_sync(0xffffffffu, mc1, src);
       bwd_rows_sub<D, 32>(p, q, k, v, d_o, scale, tau_in, entries, dq, acc_dk, acc_dv, dc_rows, 16 * blk + src, true, c0, c1,
-                          saved != 0, lane);
+                          saved != 0, pitch, lane);
     }
     while (mlong) {
       const int src = __ffs(mlong) - 1;
@@ -949,8 +949,23 @@ __global__ void __launch_bounds__(kWarpsPerCta * 32, 4) row_bwd_kernel(
         if (lane == 0) push_dense_row(grow, fb_count, fb_list, status);
         continue;
       }
-      bwd_row_full<D>(p, q, k, v, d_o, scale, tau_in, entries, dq, acc_dk, acc_dv, dc_rows, grow, c0, c1, saved != 0, lane);
+      bwd_row_full<D>(p, q, k, v, d_o, scale, tau_in, entries, dq, acc_dk, acc_dv, dc_rows, grow, c0, c1, saved != 0, pitch, lane);
     }
+  }
+}
+
+// Copies every row's final support (at most `slots` entries) from the forward call's lists into a compact
+// table; rows without a list, or with a longer one, get the count -2 and are recomputed by the backward pass.
+__global__ void save_supports_kernel(int rows, int slots, const int32_t* __restrict__ row_cnt,
+                                     const Entry* __restrict__ entries, int32_t* __restrict__ out_cnt,
+                                     Entry* __restrict__ out_entries) {
+  const long total = (long)rows * slots;
+  for (long t = (long)blockIdx.x * blockDim.x + threadIdx.x; t < total; t += (long)gridDim.x * blockDim.x) {
+    const int row = (int)(t / slots), slot = (int)(t - (long)row * slots);
+    const int cnt = row_cnt[row];
+    const bool fits = cnt >= 0 && cnt <= slots;
+    if (slot == 0) out_cnt[row] = fits ? cnt : -2;
+    if (fits && slot < cnt) out_entries[(size_t)row * slots + slot] = entries[(size_t)row * kListCap + slot];
   }
 }
 
@@ -985,19 +1000,28 @@ cudaError_t launch_row_fwd(const Problem& p, const void* v, const float* scale, 
   return cudaGetLastError();
 }
 
+cudaError_t launch_save_supports(const Problem& p, int slots, const int32_t* row_cnt, const Entry* entries,
+                                 int32_t* out_cnt, Entry* out_entries, cudaStream_t stream) {
+  const int rows = p.B * p.H * p.N;
+  const long total = (long)rows * slots;
+  const int blocks = (int)((total + 255) / 256 < 148L * 16 ? (total + 255) / 256 : 148L * 16);
+  save_supports_kernel<<<blocks, 256, 0, stream>>>(rows, slots, row_cnt, entries, out_cnt, out_entries);
+  return cudaGetLastError();
+}
+
 cudaError_t launch_row_bwd(const Problem& p, const void* q, const void* k, const void* v, const void* d_o,
                            const float* scale, const float* tau, const int32_t* half_cnt, Entry* entries, void* dq,
                            float* acc_dk, float* acc_dv, float* dc_rows, int32_t* fb_count, int32_t* fb_list,
-                           int32_t* status, int saved, cudaStream_t stream) {
+                           int32_t* status, int saved, int pitch, cudaStream_t stream) {
   const int grid = row_grid(p);
   if (p.D == 64)
     row_bwd_kernel<64><<<grid, kWarpsPerCta * 32, 0, stream>>>(
         p, (const __nv_bfloat16*)q, (const __nv_bfloat16*)k, (const __nv_bfloat16*)v, (const __nv_bfloat16*)d_o, scale,
-        tau, half_cnt, entries, (__nv_bfloat16*)dq, acc_dk, acc_dv, dc_rows, fb_count, fb_list, status, saved);
+        tau, half_cnt, entries, (__nv_bfloat16*)dq, acc_dk, acc_dv, dc_rows, fb_count, fb_list, status, saved, pitch);
   else
     row_bwd_kernel<128><<<grid, kWarpsPerCta * 32, 0, stream>>>(
         p, (const __nv_bfloat16*)q, (const __nv_bfloat16*)k, (const __nv_bfloat16*)v, (const __nv_bfloat16*)d_o, scale,
-        tau, half_cnt, entries, (__nv_bfloat16*)dq, acc_dk, acc_dv, dc_rows, fb_count, fb_list, status, saved);
+        tau, half_cnt, entries, (__nv_bfloat16*)dq, acc_dk, acc_dv, dc_rows, fb_count, fb_list, status, saved, pitch);
   return cudaGetLastError();
 }
 

@@ -271,6 +271,37 @@ def test_scale_gradients(N, d, dtype, causal, sigma, plant, alpha):
     assert torch.equal(plain["dq"], dq)
 
 
+def test_backward_from_compact_saved_supports():
+    # sparse rows (compact lists hold them), rows with more than 32 support entries and dense rows (both recomputed
+    # on the tensor cores): the compact saved state gives the gradients of the plain backward call
+    for sigma, plant, N in [(1.0, 3, 900), (0.35, 0, 900), (0.05, 0, 600)]:
+        inp = make_inputs(_small("compact", N, 128, True, plant=plant, backward=True, sigma=sigma, seed=81))
+        got = parity.run_fwd(inp, 1.5)
+        dev = got["dev"]
+        saved = binding.entmax_attn_save_supports(dev["q"], 1.5, True, got["workspace"])
+        status = torch.zeros(binding.STATUS_WORDS, dtype=torch.int32, device="cuda")
+        dq, dk, dv, _, _ = binding.entmax_attn_bwd_ex(dev["q"], dev["k"], dev["v"], got["tau"], dev["d_o"], 1.5, True,
+                                                      dev["beta"], dev["gamma"], dev["delta"], saved_supports=saved,
+                                                      status=status)
+        torch.cuda.synchronize()
+        assert int(status[binding.STATUS_FLAGS]) == 0
+        rows = inp.workload.H * N
+        recomputed = int(status[binding.STATUS_DENSE_ROWS])
+        if sigma == 1.0:
+            assert recomputed == 0
+        elif sigma == 0.35:
+            assert recomputed < rows              # most supports fit the slots
+        else:
+            assert recomputed > rows // 2
+        bwd = {"dq": dq, "dk": dk, "dv": dv}
+        for bh in range(inp.workload.H):
+            parity.check_bwd_head(inp, 1.5, bwd, bh)
+        if sigma == 1.0:
+            full = binding.entmax_attn_bwd_ex(dev["q"], dev["k"], dev["v"], got["tau"], dev["d_o"], 1.5, True, dev["beta"],
+                                              dev["gamma"], dev["delta"], fwd_workspace=got["workspace"])
+            assert torch.equal(full[0], dq)        # the same lists in the same order
+
+
 # ------------------------------------------------------------------ per-query scale tables
 def test_rowscale_equals_per_head_call_when_given_the_same_table():
     inp = make_inputs(_small("rowscale_same", 700, 128, True, plant=3, backward=True, B=2, seed=41))
