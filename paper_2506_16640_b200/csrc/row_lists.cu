@@ -793,6 +793,46 @@ __device__ __forceinline__ void add_slice(float* p, const float (&x)[PL]) {
   else atomic_add_slice<PL>(p, x);
 }
 
+// A lane's share of a row of D elements, W lanes per row: PL = D / W elements.  They are taken as chunks of four
+// that interleave across the lanes (chunk c of lane sl = elements [4 W c + 4 sl, +4)), so that what the W lanes
+// move in one instruction is contiguous: 16-byte reductions of neighbouring lanes fall into the same 32-byte
+// sector instead of half-filling one each, loads and stores stay coalesced.  (PL < 4: one contiguous piece.)
+template <int PL, int W>
+__device__ __forceinline__ void load_share(const __nv_bfloat16* row, int sl, float (&x)[PL]) {
+  if constexpr (PL < 4) {
+    load_bf16<PL>(row + sl * PL, x);
+  } else {
+#pragma unroll
+    for (int c = 0; c < PL / 4; ++c) {
+      float t[4];
+      load_bf16<4>(row + 4 * W * c + 4 * sl, t);
+#pragma unroll
+      for (int e = 0; e < 4; ++e) x[4 * c + e] = t[e];
+    }
+  }
+}
+template <int PL, int W>
+__device__ __forceinline__ void store_share(__nv_bfloat16* row, int sl, const float (&x)[PL]) {
+  if constexpr (PL < 4) {
+    store_bf16<PL>(row + sl * PL, x);
+  } else {
+#pragma unroll
+    for (int c = 0; c < PL / 4; ++c) {
+      const float t[4] = {x[4 * c], x[4 * c + 1], x[4 * c + 2], x[4 * c + 3]};
+      store_bf16<4>(row + 4 * W * c + 4 * sl, t);
+    }
+  }
+}
+template <int PL, int W>
+__device__ __forceinline__ void add_share(float* row, int sl, const float (&x)[PL]) {
+  if constexpr (PL < 4) {
+    atomic_add_slice<PL>(row + sl * PL, x);
+  } else {
+#pragma unroll
+    for (int c = 0; c < PL / 4; ++c) red_add_v4(row + 4 * W * c + 4 * sl, x[4 * c], x[4 * c + 1], x[4 * c + 2], x[4 * c + 3]);
+  }
+}
+
 // Backward of 32 / W rows at once, W lanes per row (W = 8, 16 or 32), for rows with at most W list entries.
 template <int D, int W>
 __device__ __forceinline__ void bwd_rows_sub(const Problem& p, const __nv_bfloat16* __restrict__ q,
@@ -811,10 +851,10 @@ __device__ __forceinline__ void bwd_rows_sub(const Problem& p, const __nv_bfloat
   const float g = active ? scale[(size_t)b * p.scale_sb + (size_t)h * p.N + i] * p.sm_scale : 0.f;
   const float a = (p.alpha - 1.0f) * g;
   const float tau = active ? tau_in[grow] : 0.f;
-  const size_t hbase = (size_t)b * p.sb + (size_t)h * p.sh + sl * PL;
+  const size_t hbase = (size_t)b * p.sb + (size_t)h * p.sh;
   float qs[PL], gs[PL];
-  load_slice_bf16<PL>(q + hbase + (size_t)i * p.sn, qs);
-  load_slice_bf16<PL>(d_o + hbase + (size_t)i * p.sn, gs);
+  load_share<PL, W>(q + hbase + (size_t)i * p.sn, sl, qs);
+  load_share<PL, W>(d_o + hbase + (size_t)i * p.sn, sl, gs);
   const Entry* list = entries + (size_t)grow * pitch;
   float yv = -1.0f, zz = 0.f;
   int j = 0;
@@ -837,7 +877,7 @@ __device__ __forceinline__ void bwd_rows_sub(const Problem& p, const __nv_bfloat
     float dp = 0.f;
     if (has) {
       float vs[PL];
-      load_slice_bf16<PL>(v + hbase + (size_t)kj * p.sn, vs);
+      load_share<PL, W>(v + hbase + (size_t)kj * p.sn, sl, vs);
 #pragma unroll
       for (int u = 0; u < PL; ++u) dp = fmaf(gs[u], vs[u], dp);
     }
@@ -867,18 +907,18 @@ __device__ __forceinline__ void bwd_rows_sub(const Problem& p, const __nv_bfloat
     const float pj = __shfl_sync(0xffffffffu, pe, base + t);
     if (has) {
       float ks[PL], dkv[PL], dvv[PL];
-      load_slice_bf16<PL>(k + hbase + (size_t)kj * p.sn, ks);
+      load_share<PL, W>(k + hbase + (size_t)kj * p.sn, sl, ks);
 #pragma unroll
       for (int w = 0; w < PL; ++w) {
         acc[w] = fmaf(gds, ks[w], acc[w]);
         dkv[w] = gds * qs[w];
         dvv[w] = pj * gs[w];
       }
-      add_slice<PL>(acc_dk + (arow + kj) * D + sl * PL, dkv);
-      add_slice<PL>(acc_dv + (arow + kj) * D + sl * PL, dvv);
+      add_share<PL, W>(acc_dk + (arow + kj) * D, sl, dkv);
+      add_share<PL, W>(acc_dv + (arow + kj) * D, sl, dvv);
     }
   }
-  if (active) store_slice_bf16<PL>(dq + hbase + (size_t)i * p.sn, acc);
+  if (active) store_share<PL, W>(dq + hbase + (size_t)i * p.sn, sl, acc);
 }
 
 // (register cap: four CTAs per SM -- this kernel waits on gathers and reductions, occupancy is what hides them)
