@@ -64,19 +64,23 @@ static double mass(const double* x, int n, double tau, double e) {
   return acc;
 }
 
-/* App. A: bisection on f(tau) = sum_j [x_j - tau]_+^(1/(alpha-1)) - 1 over the bracket
- * [x_max - 1, x_max - n^(1-alpha)] (the paper's bracket, un-normalised: p_max lies in [1/n, 1]). */
+/* App. A: bisection on f(tau) = sum_j [x_j - tau]_+^(1/(alpha-1)) - 1.  The paper states the bracket for
+ * logits normalised by their maximum; the caller passes x already shifted so that max x = 0, which turns
+ * it into [-1, -n^(1-alpha)] (p_max lies in [1/n, 1]).  Halving stops at an interval of 1e-12; for
+ * alpha > 2 it goes on until the interval no longer shrinks in double precision, because there
+ * p = y^(1/(alpha-1)) is not Lipschitz at y = 0 and sum p = 1 needs tau at the spacing of doubles near 1
+ * (this is also why the search runs on the shifted logits: the spacing near |x_max| would be coarser). */
 static double tau_bisect(const double* x, int n, double alpha) {
   double e = 1.0 / (alpha - 1.0);
-  double xmax = x[0];
-  for (int j = 1; j < n; ++j) if (x[j] > xmax) xmax = x[j];
-  double lo = xmax - 1.0;
-  double hi = xmax - pow((double)n, 1.0 - alpha);
-  for (int it = 0; it < 200 && (hi - lo) > 1e-12; ++it) {
+  double lo = -1.0;
+  double hi = -pow((double)n, 1.0 - alpha);
+  double tol = alpha > 2.0 ? 0.0 : 1e-12;
+  for (int it = 0; it < 200 && (hi - lo) > tol; ++it) {
     double mid = 0.5 * (lo + hi);
+    if (!(mid > lo && mid < hi)) break;
     if (mass(x, n, mid, e) >= 1.0) lo = mid; else hi = mid;
   }
-  return 0.5 * (lo + hi);
+  return alpha > 2.0 ? lo : 0.5 * (lo + hi);
 }
 
 /* alpha = 2 (sparsemax): sort descending, k* = max{k : 1 + k x_(k) > sum_{l<=k} x_(l)},
@@ -124,7 +128,11 @@ int oracle_entmax_row(const double* z, int n, double alpha, int method, double* 
   if (!x) return -2;
   double* scratch = x + n;
   double am1 = alpha - 1.0;
-  for (int j = 0; j < n; ++j) x[j] = am1 * z[j];
+  /* x = (alpha-1) z, shifted so that its maximum is 0 (App. A normalises the logits the same way): the
+   * threshold of the shifted row lies in [-1, 0), and tau = that threshold + the maximum. */
+  double xmax = am1 * z[0];
+  for (int j = 1; j < n; ++j) if (am1 * z[j] > xmax) xmax = am1 * z[j];
+  for (int j = 0; j < n; ++j) x[j] = am1 * z[j] - xmax;
   double tau;
   int use_sort = (method == ORACLE_METHOD_SORT) ||
                  (method == ORACLE_METHOD_AUTO && (alpha == 2.0 || alpha == 1.5));
@@ -139,7 +147,7 @@ int oracle_entmax_row(const double* z, int n, double alpha, int method, double* 
     if (y > 0.0) { pj = pow_pos(y, e); ++support; }
     if (p) p[j] = pj;
   }
-  if (tau_out) *tau_out = tau;
+  if (tau_out) *tau_out = tau + xmax;
   free(x);
   return support;
 }

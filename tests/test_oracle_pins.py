@@ -11,7 +11,7 @@ from scipy.optimize import brentq, minimize
 
 import oracle
 
-ALPHAS = [1.25, 1.5, 2.0, 1.1, 1.75, 3.0]
+ALPHAS = [1.25, 1.5, 2.0, 1.1, 1.75, 3.0, 4.0, 16.0]
 
 
 def _rows(rng, n, kind):
@@ -39,17 +39,30 @@ def test_row_sums_to_one_bracket_and_exact_zeros(alpha, kind):
     for n in [1, 2, 3, 7, 64, 1000]:
         z = _rows(rng, n, kind)
         p, tau, supp = oracle.entmax_row(z, alpha)
-        # tau is bisected to 1e-12; for alpha > 2 the mass is steep in tau near zero probabilities
-        assert abs(p.sum() - 1.0) < (1e-9 if alpha <= 2 else 1e-5)
+        # tau is bisected to 1e-12; for alpha > 2, p = y^(1/(alpha-1)) is not Lipschitz at y = 0 and tau (of the
+        # row shifted to max 0, so in [-1, 0)) cannot be told apart below the spacing of doubles there, 2^-53:
+        # an entry at the edge of the support moves by up to that spacing to the power 1/(alpha-1)
+        # (1e-8 at alpha = 3, 5e-6 at alpha = 4, 0.09 at alpha = 16 -- the map itself is that ill-conditioned)
+        assert abs(p.sum() - 1.0) < (1e-9 if alpha <= 2 else 4 * (2.0 ** -53) ** (1.0 / (alpha - 1)))
         x = (alpha - 1) * z
         # bracket of App. A, un-normalised: p_max in [1/n, 1]
         assert x.max() - 1.0 - 1e-12 <= tau <= x.max() - n ** (1.0 - alpha) + 1e-9
-        below = x <= tau
-        assert np.all(p[below] == 0.0)
-        assert np.all(p[~below] > 0.0)
-        assert supp == int((~below).sum())
-        # Eq. 1 itself, evaluated here with numpy's power
-        np.testing.assert_allclose(p, np.maximum(x - tau, 0.0) ** (1.0 / (alpha - 1)), rtol=1e-9, atol=1e-15)
+        supp_ref = int((p > 0).sum())
+        assert supp == supp_ref
+        if alpha <= 2:
+            below = x <= tau
+            assert np.all(p[below] == 0.0)
+            assert np.all(p[~below] > 0.0)
+            # Eq. 1 itself, evaluated here with numpy's power
+            np.testing.assert_allclose(p, np.maximum(x - tau, 0.0) ** (1.0 / (alpha - 1)), rtol=1e-9, atol=1e-15)
+        else:
+            # the returned tau carries the rounding of "+ max": compare on the shifted row, where the oracle works
+            xs = x - x.max()
+            ts = tau - x.max()
+            y = np.maximum(xs - ts, 0.0)
+            far = np.abs(xs - ts) > 1e-9 * max(1.0, abs(x.max()))
+            assert np.all(p[far & (xs < ts)] == 0.0) and np.all(p[far & (xs > ts)] > 0.0)
+            np.testing.assert_allclose(p[far], y[far] ** (1.0 / (alpha - 1)), rtol=1e-5, atol=1e-15)
 
 
 @pytest.mark.parametrize("alpha", [1.5, 2.0])
@@ -135,8 +148,9 @@ def test_two_level_closed_form(alpha, k):
             assert abs(tau - ((alpha - 1) * M - k ** (-(alpha - 1)))) < 1e-9
             np.testing.assert_allclose(p[idx], 1.0 / k, rtol=1e-8)
             assert np.all(np.delete(p, idx) == 0.0)
-        if n > k:
-            # just inside the gap the low level is attended too
+        if n > k and k ** (-(alpha - 1)) > 1e-12:
+            # just inside the gap the low level is attended too (skipped where the gap itself is below the
+            # spacing of the doubles that hold the logits: k = 8 at alpha = 16 has a gap of 2e-15)
             z = np.full(n, M - gap_min * 0.9)
             z[:k] = M
             _, _, supp = oracle.entmax_row(z, alpha)
@@ -167,7 +181,7 @@ def _brute_force(z, alpha):
     return found
 
 
-@pytest.mark.parametrize("alpha", [1.25, 1.5, 2.0, 1.7])
+@pytest.mark.parametrize("alpha", [1.25, 1.5, 2.0, 1.7, 3.0, 4.0])
 def test_brute_force_support_enumeration(alpha):
     rng = np.random.default_rng(int(alpha * 100))
     for trial in range(12):
@@ -322,7 +336,7 @@ def test_attention_matches_dense_numpy_formula():
 
 
 # ---------------------------------------------------------------- backward
-@pytest.mark.parametrize("alpha", [1.25, 1.5, 2.0, 1.7])
+@pytest.mark.parametrize("alpha", [1.25, 1.5, 2.0, 1.7, 3.0, 4.0])
 @pytest.mark.parametrize("causal", [True, False])
 def test_backward_matches_finite_differences(alpha, causal):
     rng = np.random.default_rng(int(alpha * 1000) + causal)
@@ -478,6 +492,85 @@ def test_alibi_backward_matches_finite_differences():
         dn[idx] -= e
         fd = (loss(q, k, v, tuple(up)) - loss(q, k, v, tuple(dn))) / (2 * e)
         assert abs(fd - grads[idx]) <= 1e-5 * max(1.0, abs(fd)), (idx, fd, grads[idx])
+
+
+def test_alibi_noncausal_hand_built_rows():
+    # q = 0: the content logits vanish and row i's logits are -m |j - i| alone, keys on both sides of the query.
+    # Sparsemax (alpha = 2) of three such logits, m = 1/4, worked by hand from Eq. 1 with sum p = 1:
+    #   row 1: z = [-1/4, 0, -1/4]: all three in the support, tau = (-1/2 - 1)/3 = -1/2, p = [1/4, 1/2, 1/4]
+    #   row 0: z = [0, -1/4, -1/2]: tau = (-3/4 - 1)/3 = -7/12, p = [7/12, 1/3, 1/12]
+    #   row 2: the mirror image of row 0
+    N, d, m = 3, 2, 0.25
+    q = np.zeros((N, d), np.float32)
+    k = np.ones((N, d), np.float32)
+    v = np.eye(N, d, dtype=np.float32)
+    out = oracle.attn_fwd_rows(q, k, v, np.arange(N), 2.0, 1.0, False, want_p=True, alibi=m)
+    np.testing.assert_allclose(out["p"][1], [0.25, 0.5, 0.25], atol=1e-15)
+    np.testing.assert_allclose(out["p"][0], [7 / 12, 1 / 3, 1 / 12], atol=1e-15)
+    np.testing.assert_allclose(out["p"][2], [1 / 12, 1 / 3, 7 / 12], atol=1e-15)
+    np.testing.assert_allclose(out["tau"], [-7 / 12, -0.5, -7 / 12], atol=1e-15)
+    # a steeper slope pushes the far key out of the support: m = 1 on row 0 gives z = [0, -1, -2],
+    # tau = -1 exactly at the second key (a tie: p = 0 there), p = [1, 0, 0]
+    out = oracle.attn_fwd_rows(q, k, v, np.arange(N), 2.0, 1.0, False, want_p=True, alibi=1.0)
+    np.testing.assert_allclose(out["p"][0], [1.0, 0.0, 0.0], atol=1e-15)
+    np.testing.assert_allclose(out["p"][1], [0.0, 1.0, 0.0], atol=1e-15)
+
+
+@pytest.mark.parametrize("alpha", [1.5, 2.0, 1.25])
+def test_alibi_noncausal_mirror_and_two_sided_decomposition(alpha):
+    # (1) the penalty depends on the distance only: reversing the sequence (queries, keys and values alike)
+    #     reverses the result.  A bias with the wrong sign on one side of the query breaks this.
+    # (2) for one query row i the non-causal logits are those of two causal problems glued together: keys
+    #     j <= i carry m (j - i) as they stand; keys j >= i, read backwards, are the causal keys of the reversed
+    #     sequence for query N - 1 - i.  Entmax of the concatenation, computed by the row function, must agree.
+    rng = np.random.default_rng(77)
+    N, d, m, sm = 23, 4, 0.3, 0.5
+    q, k, v = (rng.normal(size=(N, d)).astype(np.float32) for _ in range(3))
+    scale = (0.6, 0.8, 1.1)
+    rows = np.arange(N)
+    fwd = oracle.attn_fwd_rows(q, k, v, rows, alpha, sm, False, scale=scale, want_p=True, alibi=m)
+    rev = oracle.attn_fwd_rows(q[::-1].copy(), k[::-1].copy(), v[::-1].copy(), rows, alpha, sm, False, scale=scale,
+                               want_p=True, alibi=m)
+    np.testing.assert_allclose(fwd["p"], rev["p"][::-1, ::-1], atol=1e-13)
+    np.testing.assert_allclose(fwd["o"], rev["o"][::-1], atol=1e-13)
+    np.testing.assert_allclose(fwd["tau"], rev["tau"][::-1], atol=1e-13)
+    c = oracle.asentmax_scale(*scale, N)
+    z = (q.astype(np.float64) @ k.astype(np.float64).T) * sm
+    for i in (0, 5, 11, 22):
+        bias = np.array([m * (j - i) if j <= i else -m * (j - i) for j in range(N)])
+        p, tau, _ = oracle.entmax_row(c * (z[i] + bias), alpha)
+        np.testing.assert_allclose(fwd["p"][i], p, atol=1e-13)
+        assert abs(fwd["tau"][i] - tau) < 1e-12
+    # the bias is not symmetric content: a row far from the middle puts more mass on its own side
+    assert not np.allclose(fwd["p"], fwd["p"][:, ::-1])
+
+
+def test_alibi_noncausal_backward_matches_finite_differences():
+    rng = np.random.default_rng(33)
+    N, d, m, sm, alpha = 8, 4, 0.3, 0.5, 1.5
+    q, k, v = _attn_case(rng, N, d)
+    d_o = rng.normal(size=(N, d)).astype(np.float32)
+    scale = (0.8, 0.5, 0.6)
+    rows = np.arange(N)
+
+    def loss(q_, k_, v_):
+        o = oracle.attn_fwd_rows(q_, k_, v_, rows, alpha, sm, False, scale=scale, alibi=m)["o"]
+        return float(np.sum(o * d_o.astype(np.float64)))
+
+    h = 2.0 ** -9
+    for which in range(3):
+        for _ in range(8):
+            i, t = int(rng.integers(N)), int(rng.integers(d))
+            args = [q.copy(), k.copy(), v.copy()]
+            base = np.float32(np.round(args[which][i, t] * 512) / 512)
+            args[which][i, t] = base
+            g0 = oracle.attn_bwd_head(*args, d_o, alpha, sm, False, scale=scale, alibi=m)[which][i, t]
+            up = [a.copy() for a in args]
+            dn = [a.copy() for a in args]
+            up[which][i, t] = base + np.float32(h)
+            dn[which][i, t] = base - np.float32(h)
+            fd = (loss(*up) - loss(*dn)) / (2 * h)
+            assert abs(fd - g0) < 5e-4 * max(1.0, abs(g0)), (which, i, t, fd, g0)
 
 
 def test_threads_reported():
