@@ -27,7 +27,7 @@ if ROOT not in sys.path:
 import numpy as np
 import torch
 
-from paper_2506_16640_b200.inputs import WORKLOADS, make_inputs, sample_rows, scaled
+from paper_2506_16640_b200.inputs import WORKLOADS, make_inputs, sample_rows, scaled, seeded_d_o
 
 METRIC = "entmax_attn_fwd_bwd_useful_tflops_n32k"
 UNIT = "TFLOP/s"
@@ -137,9 +137,7 @@ def make_bench_inputs(alpha: float):
     """The long-context workload plus a seeded dO (the workload itself is forward-only)."""
     w = WORKLOADS[4]
     inp = make_inputs(w)
-    gen = torch.Generator(device="cpu")
-    gen.manual_seed(20250616 + 404)
-    inp.d_o = torch.randn((w.B, w.H, w.N, w.d), generator=gen, dtype=torch.float32).to(torch.bfloat16)
+    inp.d_o = seeded_d_o(w)
     return w, inp
 
 

@@ -29,8 +29,11 @@
  *     innermost and contiguous; the other three strides come from the params struct (in elements).
  *     tau is [batch, heads, seq] float32, contiguous.  beta, gamma, delta are [heads] float32.
  *   - All tensor pointers must be 16-byte aligned and all strides multiples of 8 elements.
- *   - Functions return ENTMAX_ATTN_OK (0) or a negative entmax_attn_status; on a negative return
- *     nothing has been enqueued.  Device-side conditions are reported through `device_status`.
+ *   - Functions return ENTMAX_ATTN_OK (0) or a negative entmax_attn_status.  On a validation error
+ *     (every code except ENTMAX_ATTN_ECUDA) nothing has been enqueued; after ENTMAX_ATTN_ECUDA some of the
+ *     call's work may already be on the stream and the outputs are undefined
+ *     (entmax_attn_last_cuda_error() gives the CUDA error, for every entry point).  Device-side conditions
+ *     are reported through `device_status`.
  *   - Non-finite values in Q, K, V or dO give unspecified results (never a fault).
  *   - Sequences of different lengths in one batch: pad them on the right.  Under the causal mask a valid
  *     row never sees a padded key, so no extra mask is needed; give the padded rows dO = 0 and their
@@ -99,7 +102,7 @@ size_t entmax_attn_workspace_bytes(const entmax_attn_params* params, int is_bwd)
  *   workspace    device scratch, 256-byte aligned, >= entmax_attn_workspace_bytes(params, 0); contents
  *                on return: see entmax_attn_workspace_layout
  *   device_status  optional device int32[ENTMAX_ATTN_STATUS_WORDS]
- * Errors: negative status, nothing enqueued. */
+ * Errors: negative status (see the general conventions). */
 int entmax_attn_fwd(const entmax_attn_params* params, const void* q, const void* k, const void* v,
                     const float* beta, const float* gamma, const float* delta, void* o, float* tau,
                     void* workspace, size_t workspace_bytes, int32_t* device_status, void* cuda_stream);
@@ -200,6 +203,9 @@ int entmax_attn_bwd_ex(const entmax_attn_params* params, const void* q, const vo
  *   row_count  int32 [batch*heads*seq]: support size of the row, or -2 when the row was computed by the
  *              dense path and its list is not kept (a row goes there when one of its two candidate
  *              half-lists could not be kept at `keep_limit` entries at some point of the sweep)
+ *   dense_count int32 [batch*heads*seq][2]: for a row with row_count == -2, the number of keys with p > 0
+ *              counted by each of the two threads that formed the row's probabilities; their sum is the
+ *              support size (other rows: unspecified)
  *   entries    {float y; int32 j;} [batch*heads*seq][capacity]: the first row_count slots hold the
  *              support, y = (alpha-1) s_ij as the kernel computed it (fp32), in no particular order
  *   scale      float32 [heads*seq]: c_i
@@ -208,6 +214,7 @@ typedef struct {
   size_t row_count_offset;
   size_t entries_offset;
   size_t scale_offset;
+  size_t dense_count_offset;
   int32_t capacity;
   int32_t keep_limit; /* see row_count                                                                        */
 } entmax_attn_ws_layout;
@@ -266,7 +273,8 @@ int entmax_attn_decode_fwd(const entmax_attn_decode_params* params, const void* 
  * fp32 problems alike, so it is meant for small and medium problems, not for the long-context ones.
  *
  * Size limit: round_up(heads*seq, 32) + 64 * round_up(seq, 32) floats must fit the scratch
- * (e.g. 16 heads up to seq 26214).  Larger problems return ENTMAX_ATTN_ETOOLARGE, nothing enqueued.
+ * (e.g. 16 heads up to seq 26208).  Larger problems return ENTMAX_ATTN_ETOOLARGE, nothing enqueued; the size
+ * is checked before the pointers are.
  *
  * Set-up: the first call on each device looks up the device address of the scratch array
  * (cudaGetSymbolAddress) with that device current; make that first call outside any stream capture.

@@ -37,7 +37,8 @@ class DecodeParams(ctypes.Structure):
 
 class WsLayout(ctypes.Structure):
     _fields_ = [("row_count_offset", ctypes.c_size_t), ("entries_offset", ctypes.c_size_t),
-                ("scale_offset", ctypes.c_size_t), ("capacity", ctypes.c_int32), ("keep_limit", ctypes.c_int32)]
+                ("scale_offset", ctypes.c_size_t), ("dense_count_offset", ctypes.c_size_t),
+                ("capacity", ctypes.c_int32), ("keep_limit", ctypes.c_int32)]
 
 
 class Extras(ctypes.Structure):
@@ -424,3 +425,15 @@ def read_support(params: Params, workspace: torch.Tensor, rows):
         else:
             out.append((ent_h[r, :c, 1].to(torch.int64), ent_h[r, :c, 0].contiguous().view(torch.float32)))
     return out
+
+
+def read_dense_support_sizes(params: Params, workspace: torch.Tensor, rows):
+    """Support sizes of rows the dense path computed (row_count == -2), for global row ids `rows`: int64 tensor,
+    -1 where the row kept a list instead (use read_support there)."""
+    lay = entmax_attn_workspace_layout(params)
+    total = params.batch * params.heads * params.seq
+    cnt = workspace[lay.row_count_offset: lay.row_count_offset + 4 * total].view(torch.int32)
+    dense = workspace[lay.dense_count_offset: lay.dense_count_offset + 8 * total].view(torch.int32).view(total, 2)
+    rows_t = torch.as_tensor(rows, dtype=torch.long, device=workspace.device)
+    size = dense[rows_t].sum(dim=1).to(torch.int64)
+    return torch.where(cnt[rows_t] == -2, size, torch.full_like(size, -1)).cpu()

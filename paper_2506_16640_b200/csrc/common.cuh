@@ -52,6 +52,15 @@ struct WsLayout {
 
 WsLayout make_layout(const Problem& p, bool is_bwd);
 
+// Argument checks shared by every entry point (defined in entmax_attn_api.cu).
+// make_problem validates params and fills the internal problem description; check_scale_ptrs wants beta, gamma,
+// delta all given or all NULL; fail_cuda records the cudaError_t for entmax_attn_last_cuda_error() on the calling
+// thread and returns ENTMAX_ATTN_ECUDA.
+int make_problem(const entmax_attn_params* params, Problem* out);
+int check_scale_ptrs(const float* beta, const float* gamma, const float* delta, Problem* p);
+int fail_cuda(cudaError_t err);
+inline bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+
 // y^e and y^(e-1) of a clamped y >= 0 (0 where the entry is outside the support: ok == false), with the
 // exponent class fixed at compile time so that the per-element code stays a few instructions
 template <int EC>
@@ -100,7 +109,7 @@ cudaError_t launch_scale_table(const Problem& p, const float* beta, const float*
 
 // dense-row path (CUDA cores): all rows (row_list == nullptr) or the rows in row_list[0 .. *row_count)
 cudaError_t launch_dense_fwd(const Problem& p, const void* q, const void* k, const void* v, const float* scale,
-                             void* o, float* tau, int32_t* row_cnt, Entry* entries, const int32_t* row_list,
+                             void* o, float* tau, int32_t* row_cnt, int32_t* dense_cnt, Entry* entries, const int32_t* row_list,
                              const int32_t* row_count, float* scratch, size_t scratch_floats, int ctas,
                              cudaStream_t stream);
 cudaError_t launch_dense_bwd(const Problem& p, const void* q, const void* k, const void* v, const void* d_o,
@@ -118,10 +127,11 @@ cudaError_t launch_sweep(const Problem& p, const void* q, const void* k, const f
                          float* dump, int dump_bh, int32_t* status, cudaStream_t stream);
 
 // Dense-tile forward on the tensor cores (bf16): recomputes the Q tiles (128 rows) listed in tile_list
-// and writes O and tau of their rows marked row_cnt == -2.
+// and writes O and tau of their rows marked row_cnt == -2, and into dense_cnt [B*H*N][2] the number of keys
+// with p > 0 each of the row's two threads saw (their sum is the row's support size).
 cudaError_t launch_tile_fwd(const Problem& p, const void* q, const void* k, const void* v, const float* scale,
-                            const int32_t* tile_list, const int32_t* tile_count, const int32_t* row_cnt, void* o,
-                            float* tau, int32_t* status, cudaStream_t stream);
+                            const int32_t* tile_list, const int32_t* tile_count, const int32_t* row_cnt,
+                            int32_t* dense_cnt, void* o, float* tau, int32_t* status, cudaStream_t stream);
 
 // Dense-tile backward on the tensor cores (bf16): the rows in row_list[0 .. *row_count) are marked in
 // tile_mask, their 128-row Q tiles listed, and dQ (and dc_rows) of those rows written; their dK and dV

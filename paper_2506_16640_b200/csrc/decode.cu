@@ -357,21 +357,21 @@ extern "C" int entmax_attn_decode_fwd(const entmax_attn_decode_params* params, c
   a.n_chunks = lay.n_chunks;
   a.score_stride = lay.score_stride;
   int dev = 0, major = 0;
-  if (cudaGetDevice(&dev) != cudaSuccess || cudaDeviceGetAttribute(&major, cudaDevAttrComputeCapabilityMajor, dev) != cudaSuccess)
-    return ENTMAX_ATTN_ECUDA;
+  cudaError_t err = cudaGetDevice(&dev);
+  if (err == cudaSuccess) err = cudaDeviceGetAttribute(&major, cudaDevAttrComputeCapabilityMajor, dev);
+  if (err != cudaSuccess) return fail_cuda(err);
   if (major != 10) return ENTMAX_ATTN_EUNSUPPORTED;          // the score kernel needs tcgen05 / TMA
   cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
   uint8_t* ws = static_cast<uint8_t*>(workspace);
   float* chunk_max = reinterpret_cast<float*>(ws + lay.chunk_max);
   float* scores = reinterpret_cast<float*>(ws + lay.scores);
-  cudaError_t err;
   if (device_status) {
     err = cudaMemsetAsync(device_status, 0, sizeof(int32_t) * ENTMAX_ATTN_STATUS_WORDS, stream);
-    if (err != cudaSuccess) return ENTMAX_ATTN_ECUDA;
+    if (err != cudaSuccess) return fail_cuda(err);
   }
   const int rows = a.B * a.H * a.QL;
   err = launch_decode_scores_tc(a, q, k, scores, chunk_max, device_status, stream);
-  if (err != cudaSuccess) return ENTMAX_ATTN_ECUDA;
+  if (err != cudaSuccess) return fail_cuda(err);
   const __nv_bfloat16* vb = static_cast<const __nv_bfloat16*>(v);
   __nv_bfloat16* ob = static_cast<__nv_bfloat16*>(o);
   // long rows: more threads per row (more loads in flight); many short rows: smaller CTAs
@@ -384,5 +384,5 @@ extern "C" int entmax_attn_decode_fwd(const entmax_attn_decode_params* params, c
   }
 #undef ENTMAX_SOLVE
   err = cudaGetLastError();
-  return err == cudaSuccess ? ENTMAX_ATTN_OK : ENTMAX_ATTN_ECUDA;
+  return err == cudaSuccess ? ENTMAX_ATTN_OK : fail_cuda(err);
 }

@@ -170,7 +170,8 @@ template <typename T, int D>
 __global__ void __launch_bounds__(kThreads) dense_fwd_kernel(Problem p, const T* __restrict__ q, const T* __restrict__ k,
                                                              const T* __restrict__ v, const float* __restrict__ scale,
                                                              T* __restrict__ o, float* __restrict__ tau_out,
-                                                             int32_t* __restrict__ row_cnt, Entry* __restrict__ entries,
+                                                             int32_t* __restrict__ row_cnt, int32_t* __restrict__ dense_cnt,
+                                                             Entry* __restrict__ entries,
                                                              const int32_t* __restrict__ row_list,
                                                              const int32_t* __restrict__ row_count,
                                                              float* __restrict__ scratch, size_t scratch_floats) {
@@ -225,6 +226,8 @@ __global__ void __launch_bounds__(kThreads) dense_fwd_kernel(Problem p, const T*
     if (threadIdx.x == 0) {
       tau_out[r.grow] = tau;
       if (row_cnt) row_cnt[r.grow] = supp_count <= kListCap ? supp_count : -2;
+      // a support too long for the list: its size alone is kept (same place and form as the dense-tile kernel's)
+      if (dense_cnt && supp_count > kListCap) { dense_cnt[2 * (size_t)r.grow] = supp_count; dense_cnt[2 * (size_t)r.grow + 1] = 0; }
     }
     __syncthreads();
   }
@@ -407,12 +410,12 @@ cudaError_t launch_scale_table(const Problem& p, const float* beta, const float*
 }
 
 cudaError_t launch_dense_fwd(const Problem& p, const void* q, const void* k, const void* v, const float* scale,
-                             void* o, float* tau, int32_t* row_cnt, Entry* entries, const int32_t* row_list,
-                             const int32_t* row_count, float* scratch, size_t scratch_floats, int ctas,
-                             cudaStream_t stream) {
+                             void* o, float* tau, int32_t* row_cnt, int32_t* dense_cnt, Entry* entries,
+                             const int32_t* row_list, const int32_t* row_count, float* scratch, size_t scratch_floats,
+                             int ctas, cudaStream_t stream) {
 #define ENTMAX_LAUNCH(T, D)                                                                                        \
   dense_fwd_kernel<T, D><<<ctas, kThreads, 0, stream>>>(p, (const T*)q, (const T*)k, (const T*)v, scale, (T*)o, \
-                                                        tau, row_cnt, entries, row_list, row_count, scratch,     \
+                                                        tau, row_cnt, dense_cnt, entries, row_list, row_count, scratch, \
                                                         scratch_floats)
   if (p.dtype == ENTMAX_ATTN_DTYPE_FP32) {
     if (p.D == 64) ENTMAX_LAUNCH(float, 64); else ENTMAX_LAUNCH(float, 128);

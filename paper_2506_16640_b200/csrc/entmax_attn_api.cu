@@ -59,12 +59,27 @@ SavedLayout saved_layout(const Problem& p) {
   return l;
 }
 
+int check_workspace(const Problem& p, bool is_bwd, void* ws, size_t ws_bytes, WsLayout* lay) {
+  *lay = make_layout(p, is_bwd);
+  if (!ws || (reinterpret_cast<uintptr_t>(ws) & 255u) != 0 || ws_bytes < lay->total) return ENTMAX_ATTN_EINVAL_WORKSPACE;
+  return ENTMAX_ATTN_OK;
+}
+
+int check_device_for_bf16() {
+  int dev = 0, major = 0;
+  cudaError_t err = cudaGetDevice(&dev);
+  if (err != cudaSuccess) return fail_cuda(err);
+  err = cudaDeviceGetAttribute(&major, cudaDevAttrComputeCapabilityMajor, dev);
+  if (err != cudaSuccess) return fail_cuda(err);
+  return major == 10 ? ENTMAX_ATTN_OK : ENTMAX_ATTN_EUNSUPPORTED;
+}
+
+}  // namespace
+
 int fail_cuda(cudaError_t err) {
   g_last_cuda_error = (int)err;
   return ENTMAX_ATTN_ECUDA;
 }
-
-bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
 
 // Validates params and fills the internal problem description.  Returns a status code.
 int make_problem(const entmax_attn_params* params, Problem* out) {
@@ -107,23 +122,6 @@ int check_scale_ptrs(const float* beta, const float* gamma, const float* delta, 
   p->has_scale = given == 3;
   return ENTMAX_ATTN_OK;
 }
-
-int check_workspace(const Problem& p, bool is_bwd, void* ws, size_t ws_bytes, WsLayout* lay) {
-  *lay = make_layout(p, is_bwd);
-  if (!ws || (reinterpret_cast<uintptr_t>(ws) & 255u) != 0 || ws_bytes < lay->total) return ENTMAX_ATTN_EINVAL_WORKSPACE;
-  return ENTMAX_ATTN_OK;
-}
-
-int check_device_for_bf16() {
-  int dev = 0, major = 0;
-  cudaError_t err = cudaGetDevice(&dev);
-  if (err != cudaSuccess) return fail_cuda(err);
-  err = cudaDeviceGetAttribute(&major, cudaDevAttrComputeCapabilityMajor, dev);
-  if (err != cudaSuccess) return fail_cuda(err);
-  return major == 10 ? ENTMAX_ATTN_OK : ENTMAX_ATTN_EUNSUPPORTED;
-}
-
-}  // namespace
 
 WsLayout make_layout(const Problem& p, bool is_bwd) {
   WsLayout l;
@@ -180,6 +178,7 @@ int entmax_attn_workspace_layout(const entmax_attn_params* params, entmax_attn_w
   out->row_count_offset = l.row_cnt;
   out->entries_offset = l.entries;
   out->scale_offset = l.scale;
+  out->dense_count_offset = l.half_cnt;
   out->capacity = kListCap;
   out->keep_limit = kHalfKeep;
   return ENTMAX_ATTN_OK;
@@ -237,7 +236,7 @@ int fwd_impl(const entmax_attn_params* params, const void* q, const void* k, con
     if (err != cudaSuccess) return fail_cuda(err);
   }
   if (p.dtype == ENTMAX_ATTN_DTYPE_FP32) {
-    err = launch_dense_fwd(p, q, k, v, scale, o, tau, row_cnt, entries, nullptr, nullptr, scratch, lay.scratch_floats,
+    err = launch_dense_fwd(p, q, k, v, scale, o, tau, row_cnt, half_cnt, entries, nullptr, nullptr, scratch, lay.scratch_floats,
                            lay.scratch_ctas, stream);
     return err == cudaSuccess ? ENTMAX_ATTN_OK : fail_cuda(err);
   }
@@ -257,7 +256,7 @@ int fwd_impl(const entmax_attn_params* params, const void* q, const void* k, con
                        tile_count, device_status, stream);
   if (err != cudaSuccess) return fail_cuda(err);
   // rows whose support does not fit the lists: dense tiles on the tensor cores
-  err = launch_tile_fwd(p, q, k, v, scale, tile_list, tile_count, row_cnt, o, tau, device_status, stream);
+  err = launch_tile_fwd(p, q, k, v, scale, tile_list, tile_count, row_cnt, half_cnt, o, tau, device_status, stream);
   return err == cudaSuccess ? ENTMAX_ATTN_OK : fail_cuda(err);
 }
 

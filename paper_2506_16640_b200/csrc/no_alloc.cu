@@ -60,46 +60,18 @@ using namespace entmax;
 extern "C" int entmax_attn_fwd_static(const entmax_attn_params* params, const void* q, const void* k, const void* v,
                                       const float* beta, const float* gamma, const float* delta, void* o, float* tau,
                                       int32_t* device_status, void* cuda_stream) {
-  // ---- validation (same rules and codes as entmax_attn_fwd), before any CUDA call
-  if (!params) return ENTMAX_ATTN_EINVAL_NULL;
+  // ---- validation (the rules and codes of entmax_attn_fwd), before any CUDA call
   Problem p;
-  p.B = params->batch; p.H = params->heads; p.N = params->seq; p.D = params->head_dim;
-  if (p.B < 1 || p.H < 1 || p.N < 1) return ENTMAX_ATTN_EINVAL_SHAPE;
-  if (p.D != 64 && p.D != 128) return ENTMAX_ATTN_EINVAL_SHAPE;
-  if ((long long)p.B * p.H * p.N > 0x7fffffffLL / 2) return ENTMAX_ATTN_EINVAL_SHAPE;
-  if (params->dtype != ENTMAX_ATTN_DTYPE_BF16 && params->dtype != ENTMAX_ATTN_DTYPE_FP32) return ENTMAX_ATTN_EINVAL_DTYPE;
-  p.dtype = params->dtype;
-  p.causal = params->causal ? 1 : 0;
-  p.n_mode = params->n_mode ? 1 : 0;
-  p.alpha = params->alpha;
-  if (!(p.alpha > 1.0f) || !(p.alpha <= 2.0f)) return ENTMAX_ATTN_EINVAL_ALPHA;
-  p.sm_scale = params->sm_scale;
-  if (!(p.sm_scale >= 0.f) || !(p.sm_scale < INFINITY)) return ENTMAX_ATTN_EINVAL_ALPHA;
-  if (p.sm_scale == 0.f) p.sm_scale = 1.0f / sqrtf((float)p.D);
-  p.expo = 1.0f / (p.alpha - 1.0f);
-  p.expo_class = p.alpha == 2.0f ? kExpo1 : p.alpha == 1.5f ? kExpo2 : p.alpha == 1.25f ? kExpo4 : kExpoGeneral;
-  if (params->stride_b == 0 && params->stride_h == 0 && params->stride_n == 0) {
-    p.sn = p.D;
-    p.sh = (int64_t)p.N * p.D;
-    p.sb = (int64_t)p.H * p.N * p.D;
-  } else {
-    p.sb = params->stride_b; p.sh = params->stride_h; p.sn = params->stride_n;
-    if (p.sn < p.D || p.sh < 1 || p.sb < 1) return ENTMAX_ATTN_EINVAL_SHAPE;
-    if (p.sn % 8 || p.sh % 8 || p.sb % 8) return ENTMAX_ATTN_EINVAL_SHAPE;
-  }
-  if (!q || !k || !v || !o || !tau) return ENTMAX_ATTN_EINVAL_NULL;
-  const int given = (beta != nullptr) + (gamma != nullptr) + (delta != nullptr);
-  if (given != 0 && given != 3) return ENTMAX_ATTN_EINVAL_NULL;
-  p.has_scale = given == 3;
-  p.scale_sb = 0;
-  p.alibi = nullptr;
-  auto aligned16 = [](const void* ptr) { return (reinterpret_cast<uintptr_t>(ptr) & 15u) == 0; };
-  if (!aligned16(q) || !aligned16(k) || !aligned16(v) || !aligned16(o) || !aligned16(tau)) return ENTMAX_ATTN_EINVAL_ALIGN;
-
+  int rc = make_problem(params, &p);
+  if (rc != ENTMAX_ATTN_OK) return rc;
   // ---- the size limit: scale table + at least kMinCtas score rows must fit the fixed array
   const size_t row_floats = round_up32((size_t)p.N);
   const size_t scale_floats = round_up32((size_t)p.H * p.N);
   if (scale_floats + (size_t)kMinCtas * row_floats > kStaticFloats) return ENTMAX_ATTN_ETOOLARGE;
+  if (!q || !k || !v || !o || !tau) return ENTMAX_ATTN_EINVAL_NULL;
+  rc = check_scale_ptrs(beta, gamma, delta, &p);
+  if (rc != ENTMAX_ATTN_OK) return rc;
+  if (!aligned16(q) || !aligned16(k) || !aligned16(v) || !aligned16(o) || !aligned16(tau)) return ENTMAX_ATTN_EINVAL_ALIGN;
   const size_t rows = (size_t)p.B * p.H * p.N;
   size_t ctas = (kStaticFloats - scale_floats) / row_floats;
   if (ctas > (size_t)kMaxCtas) ctas = kMaxCtas;
@@ -107,19 +79,19 @@ extern "C" int entmax_attn_fwd_static(const entmax_attn_params* params, const vo
 
   float* scratch = nullptr;
   cudaError_t err = scratch_address(&scratch);
-  if (err != cudaSuccess) return ENTMAX_ATTN_ECUDA;
+  if (err != cudaSuccess) return fail_cuda(err);
   cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
   if (device_status) {
     err = cudaMemsetAsync(device_status, 0, sizeof(int32_t) * ENTMAX_ATTN_STATUS_WORDS, stream);
-    if (err != cudaSuccess) return ENTMAX_ATTN_ECUDA;
+    if (err != cudaSuccess) return fail_cuda(err);
   }
   // Nothing in the scratch has to start at zero: the scale table is written in full before it is read,
   // and every CTA fills its score row for the keys of a query before it reads them.
   float* scale = scratch;
   float* score_rows = scratch + scale_floats;
   err = launch_scale_table(p, beta, gamma, delta, scale, device_status, stream);
-  if (err != cudaSuccess) return ENTMAX_ATTN_ECUDA;
-  err = launch_dense_fwd(p, q, k, v, scale, o, tau, nullptr, nullptr, nullptr, nullptr, score_rows, row_floats,
+  if (err != cudaSuccess) return fail_cuda(err);
+  err = launch_dense_fwd(p, q, k, v, scale, o, tau, nullptr, nullptr, nullptr, nullptr, nullptr, score_rows, row_floats,
                          (int)ctas, stream);
-  return err == cudaSuccess ? ENTMAX_ATTN_OK : ENTMAX_ATTN_ECUDA;
+  return err == cudaSuccess ? ENTMAX_ATTN_OK : fail_cuda(err);
 }

@@ -38,7 +38,8 @@ struct BCfg {
   static constexpr int kHalves = HD / 64;
   static constexpr int kQBytes = TM * HD * 2;       // Q tile; also dO, K, V tiles
   static constexpr int kBarBytes = 256;
-  static constexpr int kSmemBytes = 4 * kQBytes + 2 * kTileBytes + 1024 + kBarBytes;
+  static constexpr int kSmemBytes = 4 * kQBytes + 3 * kTileBytes + 1024 + kBarBytes;
+  static_assert(kSmemBytes <= 232448, "shared memory of one CTA");
   static constexpr int kTmemS = 0, kTmemDP = TN, kTmemDQ = 2 * TN, kTmemT = 2 * TN + 128;
 };
 
@@ -123,8 +124,9 @@ __global__ void __launch_bounds__(kThreadsB, 1) tile_bwd_kernel(const __grid_con
   const uint32_t k_smem = do_smem + C::kQBytes;
   const uint32_t v_smem = k_smem + C::kQBytes;
   const uint32_t p_smem = v_smem + C::kQBytes;           // P tile, [128 rows][128 keys] bf16, swizzled
-  const uint32_t ds_smem = p_smem + kTileBytes;           // g dS tile, same layout
-  const uint32_t bars = ds_smem + kTileBytes;
+  const uint32_t ds_smem = p_smem + kTileBytes;           // g dS tile (bf16), same layout
+  const uint32_t dl_smem = ds_smem + kTileBytes;          // what the bf16 rounding of g dS left over, same layout
+  const uint32_t bars = dl_smem + kTileBytes;
   const uint32_t qdo_full = bars, qdo_empty = bars + 8;
   const uint32_t kv_full = bars + 16, kv_empty = bars + 24;
   const uint32_t sd_full = bars + 32, sd_empty = bars + 40;
@@ -211,7 +213,7 @@ __global__ void __launch_bounds__(kThreadsB, 1) tile_bwd_kernel(const __grid_con
       constexpr uint32_t id_mn = idesc_mn<HD>();
       const uint32_t q_lo = smem_desc_lo(q_smem), do_lo = smem_desc_lo(do_smem);
       const uint32_t k_lo = smem_desc_lo(k_smem), v_lo = smem_desc_lo(v_smem);
-      const uint32_t ds_lo = smem_desc_lo(ds_smem);
+      const uint32_t ds_lo = smem_desc_lo(ds_smem), dl_lo = smem_desc_lo(dl_smem);
       const uint32_t k_n_lo = mn_desc_lo(k_smem), q_n_lo = mn_desc_lo(q_smem), do_n_lo = mn_desc_lo(do_smem);
       const uint32_t ds_m_lo = mn_desc_lo(ds_smem), p_m_lo = mn_desc_lo(p_smem);
       uint32_t kvphase = 0, qphase = 0, sdphase = 0, pdsphase = 0, tphase = 0, dqphase = 0;
@@ -263,6 +265,15 @@ __global__ void __launch_bounds__(kThreadsB, 1) tile_bwd_kernel(const __grid_con
             const uint32_t b_off = kk * ((16 * 128) >> 4);                           // 16 keys = 16 rows of 128 B
             umma_bf16_ab(tmem_base + C::kTmemDQ, ds_lo + a_off, kDescHi, k_n_lo + b_off, kDescHi, id_kn,
                          (t > tiles || kk > 0) ? 1u : 0u);
+          }
+          // the rounding remainder of g dS as a second operand: the rows of dS sum to zero, so when a row's keys are
+          // nearly equal vectors (retrieval: several copies of one key) dQ is what is left after a cancellation, and
+          // the bf16 rounding of dS alone (2^-9 of every term) would be a large part of it
+#pragma unroll
+          for (int kk = 0; kk < TN / 16; ++kk) {
+            const uint32_t a_off = (kk >> 2) * ((TM * 128) >> 4) + (kk & 3) * 2;
+            const uint32_t b_off = kk * ((16 * 128) >> 4);
+            umma_bf16_ab(tmem_base + C::kTmemDQ, dl_lo + a_off, kDescHi, k_n_lo + b_off, kDescHi, id_kn, 1u);
           }
           alive = mbar_wait(t_empty, tphase ^ 1u, abort_flag);
           tphase ^= 1u;
@@ -362,7 +373,7 @@ __global__ void __launch_bounds__(kThreadsB, 1) tile_bwd_kernel(const __grid_con
             const uint32_t blk = (uint32_t)(c >> 1) * (TM * 128) + (uint32_t)row_local * 128u;
 #pragma unroll
             for (int u4 = 0; u4 < 4; ++u4) {
-              float pv[8], dv[8];
+              float pv[8], dv[8], dl[8];
 #pragma unroll
               for (int z = 0; z < 8; ++z) {
                 const int u = u4 * 8 + z;
@@ -373,6 +384,7 @@ __global__ void __launch_bounds__(kThreadsB, 1) tile_bwd_kernel(const __grid_con
                 const float ds = ye1 * (dp[u] - rho);
                 pv[z] = ye;
                 dv[z] = g * ds;
+                dl[z] = dv[z] - __bfloat162float(__float2bfloat16_rn(dv[z]));
                 dcs[z & 1] = fmaf(ds, sa[u], dcs[z & 1]);
               }
               const uint32_t unit = (uint32_t)((c & 1) * 4 + u4);
@@ -384,6 +396,10 @@ __global__ void __launch_bounds__(kThreadsB, 1) tile_bwd_kernel(const __grid_con
               asm volatile("st.shared::cta.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(ds_smem + off),
                            "r"(pack_bf16(dv[0], dv[1])), "r"(pack_bf16(dv[2], dv[3])), "r"(pack_bf16(dv[4], dv[5])),
                            "r"(pack_bf16(dv[6], dv[7]))
+                           : "memory");
+              asm volatile("st.shared::cta.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(dl_smem + off),
+                           "r"(pack_bf16(dl[0], dl[1])), "r"(pack_bf16(dl[2], dl[3])), "r"(pack_bf16(dl[4], dl[5])),
+                           "r"(pack_bf16(dl[6], dl[7]))
                            : "memory");
             }
           }

@@ -59,6 +59,7 @@ struct TileArgsK {
   const int32_t* tile_list;  // ids of the Q tiles to process: bh * tiles_per_head + tile
   const int32_t* tile_count;
   const int32_t* row_cnt;    // -2 marks the rows to write
+  int32_t* dense_cnt;        // [B*H*N][2]: support size each of a row's two threads counted (written rows only)
   void* o;                   // bf16 [B,H,N,D]
   float* tau;
   int64_t sb, sh, sn;
@@ -306,6 +307,7 @@ __global__ void __launch_bounds__(kThreadsT, 1) tile_fwd_kernel(const __grid_con
         // the vote slot two sweeps ahead is free again: nobody reads it before the next vote
         if (warp == 2 && lane == 0) sts_u32(done_word + 4 * ((s + 1) % 3), 1u);
         float s0 = 0.f, s1 = 0.f;
+        int n_supp = 0;   // output sweep: keys of this thread's columns with p > 0
         for (int t = 0; t < tiles && alive; ++t) {
           alive = __all_sync(0xffffffffu, mbar_wait(s_full + 8 * sbuf, sphase[sbuf], abort_flag));
           if (!alive) break;
@@ -370,6 +372,7 @@ __global__ void __launch_bounds__(kThreadsT, 1) tile_fwd_kernel(const __grid_con
                     const bool ok = valid && yr > 0.f && (!edge || col0 + u <= lim);
                     float ye1;
                     pow_pair_c<EC>(ok ? yr : 0.f, ok, a.expo, pv[z], ye1);
+                    n_supp += ok ? 1 : 0;
                   }
                   const __nv_bfloat162 hh = __floats2bfloat162_rn(pv[0], pv[1]);
                   w[e2] = *reinterpret_cast<const uint32_t*>(&hh);
@@ -422,6 +425,7 @@ __global__ void __launch_bounds__(kThreadsT, 1) tile_fwd_kernel(const __grid_con
             }
           }
           if (write && half == 0) a.tau[grow] = tau;
+          if (write) a.dense_cnt[grow * 2 + half] = n_supp;
           if (a.status && threadIdx.x == 64) {
             // diagnostics: sweeps spent (y_max sweep + Newton sweeps + output sweep) and tiles processed
             atomicAdd(a.status + ENTMAX_ATTN_STATUS_TILE_SWEEPS, s + 1);
@@ -558,8 +562,8 @@ cudaError_t make_tile_map(CUtensorMap* map, const void* base, int D, int N, int 
 }  // namespace sm100
 
 cudaError_t launch_tile_fwd(const Problem& p, const void* q, const void* k, const void* v, const float* scale,
-                            const int32_t* tile_list, const int32_t* tile_count, const int32_t* row_cnt, void* o,
-                            float* tau, int32_t* status, cudaStream_t stream) {
+                            const int32_t* tile_list, const int32_t* tile_count, const int32_t* row_cnt,
+                            int32_t* dense_cnt, void* o, float* tau, int32_t* status, cudaStream_t stream) {
   TileArgsK args;
   args.B = p.B; args.H = p.H; args.N = p.N;
   args.causal = p.causal;
@@ -573,6 +577,7 @@ cudaError_t launch_tile_fwd(const Problem& p, const void* q, const void* k, cons
   args.tile_list = tile_list;
   args.tile_count = tile_count;
   args.row_cnt = row_cnt;
+  args.dense_cnt = dense_cnt;
   args.o = o;
   args.tau = tau;
   args.sb = p.sb; args.sh = p.sh; args.sn = p.sn;

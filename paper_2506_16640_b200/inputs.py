@@ -162,6 +162,14 @@ def make_inputs(w: Workload, seed: Optional[int] = None) -> Inputs:
                   1.0 / math.sqrt(w.d))
 
 
+def seeded_d_o(w: Workload, seed_offset: int = 404) -> torch.Tensor:
+    """A seeded N(0,1) output gradient for a workload that has none of its own (the forward-only long-context
+    workload when the benchmark and its parity test run a backward pass on it), rounded once to the workload dtype."""
+    gen = torch.Generator(device="cpu")
+    gen.manual_seed(BASE_SEED + seed_offset)
+    return torch.randn((w.B, w.H, w.N, w.d), generator=gen, dtype=torch.float32).to(_torch_dtype(w.dtype))
+
+
 def sample_rows(inp: Inputs, bh: int, count: int, seed: int = 0) -> np.ndarray:
     """`count` distinct query rows of head index bh = b*H + h; where the head has planted rows, half
     of the sample is forced to be planted rows.  Always contains row 0 and row N-1."""

@@ -85,6 +85,21 @@ def test_rejections_happen_before_any_device_work(lib):
     assert lib.entmax_attn_version() >= 100
 
 
+def test_static_entry_point_size_limit_is_what_the_header_says(lib):
+    # return codes only, no device work: the size check comes before the pointer checks, so a problem that
+    # fits is rejected for its NULL tensors (-6) and one that does not fit for its size (-9).
+    # limit: round_up(heads*seq, 32) + 64*round_up(seq, 32) floats <= 8 MiB; 16 heads: seq 26208 fits, 26209 does not
+    nul = ctypes.c_void_p(0)
+    call = lambda p: lib.entmax_attn_fwd_static(ctypes.byref(p), nul, nul, nul, None, None, None, nul, nul, None, None)
+    assert call(_params(heads=16, seq=26208, dtype=0)) == -6
+    assert call(_params(heads=16, seq=26209, dtype=0)) == -9
+    assert call(_params(heads=16, seq=26214, dtype=0)) == -9
+    assert call(_params(heads=1, seq=32256, dtype=0)) == -6       # 32256 + 64*32256 = 2096640 floats
+    assert call(_params(heads=1, seq=32289, dtype=0)) == -9
+    assert call(_params(alpha=0.5)) == -2                         # the shared parameter checks still come first
+    assert b"scratch" in lib.entmax_attn_strerror(-9)
+
+
 def test_decode_entry_point_rejections(lib):
     from paper_2506_16640_b200.binding import DecodeParams
 

@@ -493,6 +493,58 @@ def test_cfg4_sampled_rows(alpha, cfg4_inputs):
     print("cfg4 alpha=%g mean support %.1f dense rows %d" % (alpha, np.mean(supp), int(got["status"][1])))
 
 
+@pytest.mark.parametrize("alpha", [1.25, 1.5, 2.0])
+def test_cfg4_backward_at_size(alpha, cfg4_inputs):
+    # the benchmark's own timed backward call: the long-context tensors plus the benchmark's seeded dO, through
+    # entmax_attn_bwd (tau only), then the two saved-state variants compared with it
+    inp = cfg4_inputs
+    w = inp.workload
+    if inp.d_o is None:
+        inp.d_o = inputs.seeded_d_o(w)
+    dev = _cfg4_dev(inp)
+    if dev.get("d_o") is None:
+        dev["d_o"] = inp.d_o.cuda()
+    got = parity.run_fwd(inp, alpha, dev=dev)
+    bwd = parity.run_bwd(inp, alpha, got["tau"], dev)
+    for bh in range(w.B * w.H):
+        rows = sample_rows(inp, bh, 256)
+        parity.check_bwd_rows(inp, alpha, bwd, bh, rows)
+    _gradient_invariants(inp, bwd)
+    if alpha == 1.5:
+        # one whole head against the oracle: dK and dV need every query row
+        parity.check_bwd_head(inp, alpha, bwd, 5)
+    # backward fed with the forward call's workspace, and with the compact copy of its supports
+    st = torch.zeros(binding.STATUS_WORDS, dtype=torch.int32, device="cuda")
+    full = binding.entmax_attn_bwd_ex(dev["q"], dev["k"], dev["v"], got["tau"], dev["d_o"], alpha, True, dev["beta"],
+                                      dev["gamma"], dev["delta"], fwd_workspace=got["workspace"], status=st)
+    saved = binding.entmax_attn_save_supports(dev["q"], alpha, True, got["workspace"])
+    st2 = torch.zeros(binding.STATUS_WORDS, dtype=torch.int32, device="cuda")
+    comp = binding.entmax_attn_bwd_ex(dev["q"], dev["k"], dev["v"], got["tau"], dev["d_o"], alpha, True, dev["beta"],
+                                      dev["gamma"], dev["delta"], saved_supports=saved, status=st2)
+    torch.cuda.synchronize()
+    assert int(st[binding.STATUS_FLAGS]) == 0 and int(st2[binding.STATUS_FLAGS]) == 0
+    for other in (full, comp):
+        # dQ is row-local: the same supports give the same sums up to their order; dK, dV are sums over rows.
+        # alpha = 2: u = 1 on the whole support, so a key within rounding of the threshold (the saved lists and
+        # the recomputed scores differ by one rounding) flips a row's gradient: such rows must be few and each
+        # must have a key inside the don't-care band of the threshold
+        for bh in (0, 7, 15):
+            a_dq, b_dq = other[0][0, bh].float().cpu().numpy(), bwd["dq"][0, bh].float().cpu().numpy()
+            bad = parity.grad_mismatch_rows(a_dq, b_dq)
+            if alpha < 2.0:
+                assert len(bad) == 0, ("dq (saved state vs tau-only)", bh, bad[:8])
+            else:
+                assert len(bad) <= 8, ("dq (saved state vs tau-only): too many rows differ", bh, len(bad))
+                for i in bad:
+                    assert parity.threshold_margin(inp, alpha, bh, int(i)) <= parity.BAND, (bh, int(i))
+            if alpha < 2.0 or len(bad) == 0:
+                for name, a_, b_ in (("dk", other[1], bwd["dk"]), ("dv", other[2], bwd["dv"])):
+                    parity.grad_close(name + " (saved state vs tau-only)", a_[0, bh].float().cpu().numpy(),
+                                      b_[0, bh].float().cpu().numpy())
+    del full, comp, saved, bwd, got
+    torch.cuda.empty_cache()
+
+
 _CFG4_DEV = {}
 
 
@@ -535,6 +587,20 @@ def test_long_sequences_with_byte_offsets_beyond_32_bits():
         parity.check_fwd_rows(inp, 1.5, got, bh, rows)
         parity.check_bwd_rows(inp, 1.5, bwd, bh, rows)
     _gradient_invariants(inp, bwd)
+    del got, bwd
+    torch.cuda.empty_cache()
+
+
+def test_cfg5_one_full_head_backward_at_size():
+    # dK and dV need every query row: one seeded head of the retrieval workload at its real length (the oracle
+    # spends about a minute on it), forward rows on a stride
+    inp = make_inputs(WORKLOADS[5])
+    w = inp.workload
+    got = parity.run_fwd(inp, 1.5)
+    bwd = parity.run_bwd(inp, 1.5, got["tau"], got["dev"])
+    bh = int(np.random.default_rng(20250616 + 5).integers(w.B * w.H))
+    parity.check_fwd_rows(inp, 1.5, got, bh, np.arange(0, w.N, 97))
+    parity.check_bwd_head(inp, 1.5, bwd, bh)
     del got, bwd
     torch.cuda.empty_cache()
 
