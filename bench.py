@@ -15,6 +15,7 @@ import argparse
 import ctypes
 import json
 import os
+import re
 import statistics
 import subprocess
 import sys
@@ -32,10 +33,30 @@ from paper_2506_16640_b200.inputs import WORKLOADS, make_inputs, sample_rows, sc
 METRIC = "entmax_attn_fwd_bwd_useful_tflops_n32k"
 UNIT = "TFLOP/s"
 NOMINAL_BF16_TFLOPS = 2250.0
+BASE_SEED_DENSITY = 20250616 + 808
 FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
-# DRAM bytes (read + write) of one forward score-sweep launch on the benchmark workload, from the ncu
-# capture summarised under profiles/ (None until a capture exists).
-SWEEP_DRAM_TRAFFIC_BYTES = 355845632   # dram__bytes_read 295181056 + dram__bytes_write 60664576
+# The ncu summary of the forward score sweep on the benchmark workload; its dram__bytes_read.sum and
+# dram__bytes_write.sum lines (first column: the forward launch) give `roofline.traffic`.
+SWEEP_PROFILE = os.path.join("profiles", "sweep_kernel_d128_cfg4_n32768.md")
+
+
+def sweep_dram_traffic():
+    """DRAM bytes (read + write) of one forward sweep launch as captured under ncu, read from the profile summary;
+    None when the summary is missing or says that the kernel has changed since the capture."""
+    path = os.path.join(ROOT, SWEEP_PROFILE)
+    try:
+        text = open(path).read()
+    except OSError:
+        return None
+    if "counters predate the current kernel" in text:
+        return None
+    total = 0.0
+    for name in ("dram__bytes_read.sum", "dram__bytes_write.sum"):
+        m = re.search(re.escape(name) + r"\s+Mbyte\s+([0-9.]+)", text)
+        if not m:
+            return None
+        total += float(m.group(1)) * 1e6
+    return int(total)
 
 
 def visible_pairs(w) -> int:
@@ -202,10 +223,12 @@ def run_ours(args):
     torch.cuda.synchronize()
     barrier(world)
     clocks = sampler.stop()
-    fwd_ms = sum(a.elapsed_time(b) for a, b in zip(e_start, e_mid)) / K
-    bwd_ms = sum(a.elapsed_time(b) for a, b in zip(e_mid, e_stop)) / K
-    step_ms = sum(a.elapsed_time(b) for a, b in zip(e_start, e_stop)) / K
-    sweep_ms = sum(a.elapsed_time(b) for a, b in zip(s_start, s_stop)) / K
+    fwd_all = [a.elapsed_time(b) for a, b in zip(e_start, e_mid)]
+    bwd_all = [a.elapsed_time(b) for a, b in zip(e_mid, e_stop)]
+    step_all = [a.elapsed_time(b) for a, b in zip(e_start, e_stop)]
+    sweep_all = [a.elapsed_time(b) for a, b in zip(s_start, s_stop)]
+    fwd_ms, bwd_ms, step_ms, sweep_ms = (sum(x) / K for x in (fwd_all, bwd_all, step_all, sweep_all))
+    spread = lambda xs: {"mean": sum(xs) / len(xs), "median": statistics.median(xs), "min": min(xs), "max": max(xs)}
     assert int(status[binding.STATUS_FLAGS].item()) == 0, "device status flags set during the timed region"
 
     # secondary: the backward pass fed with the forward call's workspace (its supports are reused, no second sweep)
@@ -242,6 +265,11 @@ def run_ours(args):
 
     # secondary: the decode shape on the same tensors: the last q_len rows of Q as the new queries, K and V as the cache
     decode = time_decode(d, w, alpha, flush) if world == 1 else None
+    # secondary: the temperature axis on this shape, the other alphas and the other workloads
+    density = other = None
+    if world == 1 and not args.no_secondary:
+        density = time_density_axis(d, w, alpha, flush, ws)
+        other = [time_workload(4, a2, flush, tensors=d, ws=ws) for a2 in (1.25, 2.0) if a2 != alpha]
 
     # end to end: pinned host buffers in, results back to pinned host buffers, copies inside the timed region
     names = ("q", "k", "v", "d_o", "beta", "gamma", "delta")
@@ -316,6 +344,10 @@ def run_ours(args):
     del ws_g
     e2e_ms = sum(a.elapsed_time(b) for a, b in zip(ee_start, ee_stop)) / E
 
+    if other is not None:
+        del ws, o, dq, dk, dv
+        torch.cuda.empty_cache()
+        other += [time_workload(idx, 1.5, flush) for idx in (2, 3, 5)]
     f_fwd, f_bwd = useful_flops(w)
     step_ms_all, flops_all = aggregate_over_ranks(step_ms, float(f_fwd + f_bwd), world, dev)
     e2e_ms_all, _ = aggregate_over_ranks(e2e_ms, 0.0, world, dev)
@@ -325,9 +357,18 @@ def run_ours(args):
     burst = float(peaks.get("bf16_tflops", FALLBACK_PEAKS["bf16_tflops"]))
     sustained = float(peaks.get("bf16_tflops_sustained", FALLBACK_PEAKS["bf16_tflops_sustained"]))
     sweep_flops = 2 * w.d * visible_pairs(w)                # algorithmic: one QK^T contraction per visible pair
+    sample_extra = 1.0 / 8.0 * (1.0 - (4096.0 / w.N) ** 2) if w.N >= 4096 else 0.0   # share of pairs scored twice
     sweep_tflops = sweep_flops / (sweep_ms * 1e-3) / 1e12
     fwd_tflops = f_fwd / (fwd_ms * 1e-3) / 1e12
     bwd_tflops = f_bwd / (bwd_ms * 1e-3) / 1e12
+    # Two ways of counting.  "Dense-equivalent" FLOPs (the metric: forward 4 d, backward 10 d per visible pair) are what
+    # a dense schedule would spend; the method skips almost all of it, so those rates are speed-ups over a dense
+    # schedule and may exceed the tensor peak.  "Method" FLOPs are what the calls really contract on the tensor cores:
+    # one Q K^T per visible pair in the forward sweep, one more in the tau-only backward (gathers over supports of a
+    # few keys are noise beside them).
+    method_fwd, method_bwd = sweep_flops, sweep_flops
+    ws_bytes = {"forward": binding.entmax_attn_workspace_bytes(params, False),
+                "backward": binding.entmax_attn_workspace_bytes(params, True)}
     line = {
         "metric": METRIC, "value": flops_all / (step_ms_all * 1e-3) / 1e12, "unit": UNIT, "n_gpus": world,
         "steps": K, "warmup": max(args.warmup, 3), "ms_per_step": step_ms_all, "higher_is_better": True,
@@ -336,26 +377,39 @@ def run_ours(args):
                    "alpha": alpha, "step": "entmax_attn_fwd + entmax_attn_bwd", "l2": "256 MiB memset between steps; "
                    "inputs (134 MB per tensor) and workspace (>1 GB) larger than L2",
                    "parallelism": "independent replicas, no collective" if world > 1 else "single GPU",
-                   "useful_flops": "fwd 4*d, bwd 10*d per visible (query,key) pair"},
-        "fwd": {"ms": fwd_ms, "tflops": fwd_tflops, "frac_of_measured_burst": fwd_tflops / burst,
-                "frac_of_measured_sustained": fwd_tflops / sustained, "frac_of_nominal": fwd_tflops / NOMINAL_BF16_TFLOPS},
-        "bwd": {"ms": bwd_ms, "tflops": bwd_tflops, "frac_of_measured_burst": bwd_tflops / burst},
-        "bwd_with_saved_forward_workspace": {"ms": bwd_saved_ms, "tflops": f_bwd / (bwd_saved_ms * 1e-3) / 1e12,
+                   "value_counts": "dense-equivalent FLOPs: fwd 4*d, bwd 10*d per visible (query,key) pair",
+                   "workspace_bytes": ws_bytes},
+        "ms_per_step_stats": spread(step_all),
+        "fwd": {"ms": fwd_ms, "ms_stats": spread(fwd_all),
+                "dense_equivalent_tflops": fwd_tflops, "dense_equivalent_speedup_vs_burst_peak": fwd_tflops / burst,
+                "method_tflops": method_fwd / (fwd_ms * 1e-3) / 1e12,
+                "method_frac_of_burst_peak": method_fwd / (fwd_ms * 1e-3) / 1e12 / burst,
+                "note": "method = the one Q K^T contraction the call performs; dense-equivalent = the metric's 4*d count "
+                        "(a speed-up over a dense schedule, not a fraction of peak)"},
+        "bwd": {"ms": bwd_ms, "ms_stats": spread(bwd_all),
+                "dense_equivalent_tflops": bwd_tflops, "dense_equivalent_speedup_vs_burst_peak": bwd_tflops / burst,
+                "method_tflops": method_bwd / (bwd_ms * 1e-3) / 1e12,
+                "method_frac_of_burst_peak": method_bwd / (bwd_ms * 1e-3) / 1e12 / burst},
+        "bwd_with_saved_forward_workspace": {"ms": bwd_saved_ms, "dense_equivalent_tflops": f_bwd / (bwd_saved_ms * 1e-3) / 1e12,
                                              "note": "not part of `value`: entmax_attn_bwd_ex given the forward call's "
                                                      "workspace reuses its support lists instead of sweeping QK^T again"},
-        "bwd_with_compact_saved_supports": {"ms": bwd_compact_ms, "tflops": f_bwd / (bwd_compact_ms * 1e-3) / 1e12,
+        "bwd_with_compact_saved_supports": {"ms": bwd_compact_ms, "dense_equivalent_tflops": f_bwd / (bwd_compact_ms * 1e-3) / 1e12,
                                             "saved_bytes": saved_bytes, "rows_recomputed": compact_recomputed,
                                             "note": "not part of `value`: entmax_attn_save_supports after the forward call "
                                                     "+ entmax_attn_bwd_ex fed with the compact copy"},
-        "tau_search_extra": {"tensor_flops": 0, "note": "single score sweep: the threshold is solved on the per-row "
-                             "candidate lists, no extra QK^T pass", "dense_fallback_rows": dense_rows},
-        # the sweep is timed inside the back-to-back step loop (power cap active, see `clocks`): the sustained
-        # cuBLAS figure is its denominator; the burst figure is given beside it
+        "tau_search_extra": {"tensor_flops": int(sweep_flops * sample_extra), "note": "single score sweep: the threshold is "
+                             "solved on the per-row candidate lists, no extra QK^T pass; the figure is the sampled pre-pass "
+                             "of the forward sweep (every 8th key scored once more, for rows that see 4096 keys or more)",
+                             "dense_fallback_rows": dense_rows},
+        # the timed loop lasts a fraction of a second at boost clocks (see `clocks`): the burst cuBLAS figure is the
+        # denominator; the sustained one is given beside it
         "roofline": {"bound": "tensor", "kernel": "sweep_kernel<128> (forward score sweep)", "achieved": sweep_tflops,
-                     "peak": sustained, "unit": "TFLOP/s", "frac": sweep_tflops / sustained,
-                     "peak_source": peak_kind + " sustained (kernel timed inside the step loop)",
-                     "frac_of_burst": sweep_tflops / burst, "burst_peak": burst, "ms_per_launch": sweep_ms,
-                     "algorithmic_flops_per_launch": sweep_flops, "traffic": SWEEP_DRAM_TRAFFIC_BYTES},
+                     "peak": burst, "unit": "TFLOP/s", "frac": sweep_tflops / burst,
+                     "peak_source": peak_kind + " burst (timed region %.2f s)" % (step_ms * K * 1e-3),
+                     "frac_of_sustained": sweep_tflops / sustained, "sustained_peak": sustained,
+                     "ms_per_launch": sweep_ms, "ms_per_launch_stats": spread(sweep_all),
+                     "algorithmic_flops_per_launch": sweep_flops, "traffic": sweep_dram_traffic(),
+                     "traffic_source": SWEEP_PROFILE},
         "e2e": {"value": flops_all / (e2e_ms_all * 1e-3) / 1e12, "unit": UNIT, "ms_per_step": e2e_ms_all,
                 "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h},
         # forward: scale table, score sweep, row solve, dense tiles; backward: scale table, score sweep, row
@@ -363,6 +417,13 @@ def run_ours(args):
         "gpu_launches": 11 * K,
         "clocks": clocks,
     }
+    if density is not None:
+        line["density_axis"] = {"note": "not part of `value`: the same shape and tensors with the temperature swept -- the "
+                                "paper's regime (delta = 1, gamma = -0.5, Sec. 4.1) and fixed scales c; "
+                                "supports grow as c falls", "runs": density}
+    if other is not None:
+        line["other_workloads"] = {"note": "not part of `value`: forward / backward of the other workloads and alphas, median "
+                                   "of 5 calls, L2 flushed before each", "runs": other}
     if decode is not None:
         hbm = float(peaks.get("hbm_gbs", FALLBACK_PEAKS["hbm_gbs"]))
         for entry in decode:
@@ -373,6 +434,107 @@ def run_ours(args):
     if world == 1 and not args.no_cpu_baseline:
         line["cpu_baseline"] = cpu_baseline(inp, w, alpha, budget_s=args.cpu_seconds)
     print(json.dumps(line), flush=True)
+
+
+def support_stats(params, ws, status):
+    """Realised sparsity of a finished forward call: support sizes from the workspace (list rows and dense-path rows)."""
+    from paper_2506_16640_b200 import binding
+    lay = binding.entmax_attn_workspace_layout(params)
+    total = params.batch * params.heads * params.seq
+    cnt = ws[lay.row_count_offset: lay.row_count_offset + 4 * total].view(torch.int32)
+    dn = ws[lay.dense_count_offset: lay.dense_count_offset + 8 * total].view(torch.int32).view(total, 2).sum(1)
+    supp = torch.where(cnt == -2, dn, cnt).float()
+    sample = supp[:: max(1, total // 200000)]
+    st = status.tolist()
+    return {"mean_support": float(supp.mean().item()), "p99_support": float(torch.quantile(sample, 0.99).item()),
+            "max_support": int(supp.max().item()), "dense_path_rows": st[1], "dense_path_row_frac": st[1] / total,
+            "dense_tiles": st[3], "sweeps_per_dense_tile": (st[2] / st[3]) if st[3] else 0.0}
+
+
+def time_fwd_bwd(t, alpha, causal, beta, gamma, delta, flush, ws=None, iters=5):
+    """Median forward / backward / forward-sweep times of one problem (L2 flushed before every call) and the
+    realised sparsity of the forward pass."""
+    from paper_2506_16640_b200 import binding
+    dev = t["q"].device
+    B, H, N, D = t["q"].shape
+    params = binding.make_params(t["q"], alpha, causal)
+    if ws is None:
+        ws = binding.alloc_workspace(params, True, dev)
+    st_f = torch.zeros(binding.STATUS_WORDS, dtype=torch.int32, device=dev)
+    st_b = torch.zeros(binding.STATUS_WORDS, dtype=torch.int32, device=dev)
+    o = torch.empty_like(t["q"])
+    tau = torch.empty((B, H, N), dtype=torch.float32, device=dev)
+    dq, dk, dv = (torch.empty_like(t["q"]) for _ in range(3))
+    ev = lambda: torch.cuda.Event(enable_timing=True)
+    s0, s1 = ev(), ev()
+    s0.record(); s1.record()
+    torch.cuda.synchronize()
+    binding.entmax_attn_profile_events(0, s0, s1)
+    tf, tb, tsw, stats = [], [], [], None
+    for it in range(iters + 2):
+        flush.zero_()
+        e0, e1, e2, e3 = ev(), ev(), ev(), ev()
+        e0.record()
+        binding.entmax_attn_fwd(t["q"], t["k"], t["v"], alpha, causal, beta, gamma, delta, o=o, tau=tau, workspace=ws,
+                                status=st_f)
+        e1.record()
+        torch.cuda.synchronize()
+        if stats is None:
+            stats = support_stats(params, ws, st_f)     # before the backward call reuses the workspace
+        flush.zero_()
+        e2.record()
+        binding.entmax_attn_bwd(t["q"], t["k"], t["v"], tau, t["d_o"], alpha, causal, beta, gamma, delta, dq=dq, dk=dk,
+                                dv=dv, workspace=ws, status=st_b)
+        e3.record()
+        torch.cuda.synchronize()
+        if it >= 2:
+            tf.append(e0.elapsed_time(e1)); tb.append(e2.elapsed_time(e3)); tsw.append(s0.elapsed_time(s1))
+    binding.entmax_attn_profile_events(0, None, None)
+    assert int(st_f[0].item()) == 0 and int(st_b[0].item()) == 0, "device status flags set"
+    pairs = (N * (N + 1) // 2 if causal else N * N) * B * H
+    fwd_ms, bwd_ms, sweep_ms = statistics.median(tf), statistics.median(tb), statistics.median(tsw)
+    out = {"fwd_ms": fwd_ms, "bwd_ms": bwd_ms, "fwd_sweep_ms": sweep_ms,
+           "fwd_method_tflops": 2 * D * pairs / (fwd_ms * 1e-3) / 1e12,
+           "fwd_sweep_method_tflops": 2 * D * pairs / (sweep_ms * 1e-3) / 1e12,
+           "fwd_dense_equivalent_tflops": 4 * D * pairs / (fwd_ms * 1e-3) / 1e12,
+           "bwd_dense_equivalent_tflops": 10 * D * pairs / (bwd_ms * 1e-3) / 1e12,
+           "bwd_dense_path_rows": int(st_b[1].item())}
+    out.update(stats)
+    return out
+
+
+def time_workload(index, alpha, flush, tensors=None, ws=None):
+    """One of the seeded workloads (its own tensors unless given), forward + backward."""
+    w = WORKLOADS[index]
+    if tensors is None:
+        inp = make_inputs(w)
+        if inp.d_o is None:
+            inp.d_o = seeded_d_o(w)
+        dev = flush.device
+        tensors = {n: getattr(inp, n).to(dev) for n in ("q", "k", "v", "d_o", "beta", "gamma", "delta")}
+    res = time_fwd_bwd(tensors, alpha, w.causal, tensors["beta"], tensors["gamma"], tensors["delta"], flush, ws=ws)
+    res.update({"workload": w.name, "alpha": alpha, "batch": w.B, "heads": w.H, "seq": w.N, "head_dim": w.d, "causal": w.causal})
+    return res
+
+
+def time_density_axis(d, w, alpha, flush, ws):
+    """The benchmark's shape with the temperature swept: the paper's regime (delta = 1, gamma = -0.5, beta in
+    {0.5, 1, 2}) and fixed scales c, on the workload's planted tensors and on plain seeded N(0,1) tensors."""
+    dev = d["q"].device
+    gen = torch.Generator(device=dev).manual_seed(BASE_SEED_DENSITY)
+    plain = {n: torch.randn(d["q"].shape, generator=gen, device=dev, dtype=torch.float32).to(torch.bfloat16)
+             for n in ("q", "k", "v")}
+    plain["d_o"] = d["d_o"]
+    runs = []
+    for label, t in (("planted", d), ("plain", plain)):
+        cases = [("paper: delta=1, gamma=-0.5, beta=%g" % b, b, -0.5, 1.0) for b in (0.5, 1.0, 2.0)]
+        cases += [("fixed c=%g" % c, 0.0, 1.0, c) for c in (1.0, 2.0, 4.0, 8.0)]
+        for name, b, g, dl in cases:
+            full = lambda x: torch.full((w.H,), x, dtype=torch.float32, device=dev)
+            res = time_fwd_bwd(t, alpha, w.causal, full(b), full(g), full(dl), flush, ws=ws, iters=3)
+            res.update({"tensors": label, "scale": name, "c_at_last_row": dl + b * float(np.log(w.N)) ** g})
+            runs.append(res)
+    return runs
 
 
 def time_decode(d, w, alpha, flush, iters=20):
@@ -457,10 +619,20 @@ def cpu_baseline(inp, w, alpha, budget_s: float = 15.0):
     heads = _oracle_heads(inp, w)
     rows_per_head = _sized_rows_per_head(inp, w, alpha, heads, budget_s)
     secs, flops, nrows = _oracle_pass(inp, w, alpha, heads, rows_per_head, seed=2)
-    return {"value": flops / secs / 1e12, "unit": UNIT, "cores": oracle.num_threads(), "kind": "oracle",
+    cores = oracle.num_threads()
+    # the same oracle on one thread, on a sample sized for a few seconds
+    one_rows = max(4, int(rows_per_head * 4.0 / max(secs, 1e-3) / max(cores, 1)))
+    oracle.set_num_threads(1)
+    try:
+        secs1, flops1, nrows1 = _oracle_pass(inp, w, alpha, heads, min(one_rows, rows_per_head), seed=3)
+    finally:
+        oracle.set_num_threads(cores)
+    return {"value": flops / secs / 1e12, "unit": UNIT, "cores": cores, "kind": "oracle",
             "sample": "%d sampled query rows (%d per head) of the same workload: oracle forward rows plus the "
                       "row-local backward (dQ) rows, %.1f s; useful FLOPs of those rows / time" % (nrows, rows_per_head, secs),
-            "rows_per_s": nrows / secs, "extrapolated_full_step_s": (w.B * w.H * w.N) * secs / nrows}
+            "rows_per_s": nrows / secs, "extrapolated_full_step_s": (w.B * w.H * w.N) * secs / nrows,
+            "one_thread": {"value": flops1 / secs1 / 1e12, "unit": UNIT, "rows_per_s": nrows1 / secs1,
+                           "sample": "%d rows, %.1f s" % (nrows1, secs1)}}
 
 
 def run_reference(args):
@@ -501,6 +673,7 @@ def main():
     ap.add_argument("--impl", choices=["ours", "reference"], default="ours")
     ap.add_argument("--alpha", type=float, default=1.5)
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-secondary", action="store_true", help="skip the temperature axis and the other workloads")
     ap.add_argument("--cpu-seconds", type=float, default=15.0)
     args = ap.parse_args()
     if args.impl == "reference":
