@@ -35,6 +35,13 @@
  *     (entmax_attn_last_cuda_error() gives the CUDA error, for every entry point).  Device-side conditions
  *     are reported through `device_status`.
  *   - Non-finite values in Q, K, V or dO give unspecified results (never a fault).
+ *   - alpha > 2 (the paper's retrieval experiments use 4 ... 64): the exponent 1/(alpha-1) is below 1, p is not
+ *     Lipschitz at the edge of the support and u = p^(2-alpha) is unbounded there.  The thresholds come from a
+ *     bracketed iteration (App. A's bisection bracket with Newton steps inside) instead of Newton from the left.
+ *     Results are as accurate as float32 allows: a key that sits d above the threshold weighs d^(1/(alpha-1)), so the
+ *     spacing of tau in float32 (about 4e-6 at |tau| = 50) caps the accuracy of P at about 2e-3 for alpha = 3 and
+ *     2e-2 for alpha = 4; far beyond that only rows that are one-hot or exact ties come out exact, and the backward
+ *     pass of a row with a key within 1e-3 of its threshold is unspecified (finite).
  *   - Sequences of different lengths in one batch: pad them on the right.  Under the causal mask a valid
  *     row never sees a padded key, so no extra mask is needed; give the padded rows dO = 0 and their
  *     content cannot reach dK, dV either (their own O, tau, dQ rows are to be ignored).  Non-causal
@@ -56,7 +63,7 @@ extern "C" {
 typedef enum {
   ENTMAX_ATTN_OK = 0,
   ENTMAX_ATTN_EINVAL_SHAPE = -1,     /* batch/heads/seq < 1, head_dim not 64 or 128, bad strides, too many rows */
-  ENTMAX_ATTN_EINVAL_ALPHA = -2,     /* alpha not in (1, 2] or not finite; sm_scale not finite or negative     */
+  ENTMAX_ATTN_EINVAL_ALPHA = -2,     /* alpha not in (1, 64] or not finite; sm_scale not finite or negative    */
   ENTMAX_ATTN_EINVAL_DTYPE = -3,     /* dtype is neither ENTMAX_ATTN_DTYPE_BF16 nor ENTMAX_ATTN_DTYPE_FP32      */
   ENTMAX_ATTN_EINVAL_ALIGN = -4,     /* a tensor pointer is not 16-byte aligned                                 */
   ENTMAX_ATTN_EINVAL_WORKSPACE = -5, /* workspace NULL, misaligned (256 B) or smaller than workspace_bytes()    */
@@ -71,7 +78,8 @@ typedef struct {
   int32_t dtype;                       /* ENTMAX_ATTN_DTYPE_*                                                    */
   int32_t causal;                      /* 0 / 1; causal keeps j <= i, diagonal included                          */
   int32_t n_mode;                      /* 0: n_i = keys visible to row i; 1: n_i = seq for every row             */
-  float alpha;                         /* 1 < alpha <= 2; 1.25, 1.5 and 2 use multiplication-only powers         */
+  float alpha;                         /* 1 < alpha <= 64; 1.25, 1.5 and 2 use multiplication-only powers; beyond 2
+                                          see "alpha > 2" below                                                   */
   float sm_scale;                      /* 0 means 1/sqrt(head_dim)                                               */
   int64_t stride_b, stride_h, stride_n; /* elements; all 0 means contiguous [batch, heads, seq, head_dim]        */
 } entmax_attn_params;
@@ -247,7 +255,7 @@ int entmax_attn_workspace_layout(const entmax_attn_params* params, entmax_attn_w
 #define ENTMAX_ATTN_DECODE_MAX_Q 8
 typedef struct {
   int32_t batch, heads, q_len, kv_capacity, head_dim; /* head_dim in {64, 128}                              */
-  float alpha;                                         /* 1 < alpha <= 2                                     */
+  float alpha;                                         /* 1 < alpha <= 64                                    */
   float sm_scale;                                      /* 0 means 1/sqrt(head_dim)                           */
   int64_t kv_stride_b, kv_stride_h, kv_stride_n;       /* elements; all 0 = contiguous                       */
 } entmax_attn_decode_params;

@@ -27,6 +27,10 @@ struct __align__(8) Entry {
   int32_t j;
 };
 
+// Largest alpha the entry points accept (the paper's experiments go up to 64).  Beyond 2 the map is only as well
+// conditioned as (spacing of tau)^(1/(alpha-1)) allows: fp32 keeps alpha <= 4 within the output tolerance.
+constexpr float kAlphaMax = 64.0f;
+
 // Exponent class of 1/(alpha-1): powers by multiplication for 1, 2, 4; powf otherwise.
 enum ExpoClass : int { kExpoGeneral = 0, kExpo1 = 1, kExpo2 = 2, kExpo4 = 4 };
 
@@ -92,6 +96,42 @@ __device__ __forceinline__ float threshold_step(float s0, float s1, int expo_cla
                      : expo_class == kExpo2 ? sqrtf(s0)
                      : expo_class == kExpo4 ? sqrtf(sqrtf(s0)) : powf(s0, 1.0f / expo);
   return (s0 - s0 / root) / s1;
+}
+
+// Threshold iteration for any exponent.  For e >= 1 (alpha <= 2) f(tau) = sum [y - tau]_+^e - 1 is convex and
+// decreasing, and steps from the left of the root never pass it (threshold_step above).  For e < 1 (alpha > 2) every
+// term is concave where positive and drops to zero with infinite slope, so Newton alone can overshoot either way: the
+// iteration keeps a bracket (App. A's bisection bracket: lo with mass >= 1, hi with mass < 1), takes the Newton step on
+// f when it lands strictly inside and the midpoint otherwise, and ends when the mass is 1 to rounding or on the lower
+// end of a bracket that holds no further float.
+struct TauIter {
+  float tau, lo, hi;
+};
+__device__ __forceinline__ TauIter tau_iter_start(float ymax) {
+  TauIter s;
+  s.tau = s.lo = ymax - 1.0f;   // p_max <= 1
+  s.hi = ymax;                  // nothing above y_max: mass 0
+  return s;
+}
+// One update from S = sum [y - tau]_+^e and S1 = sum [y - tau]_+^(e-1) taken at s.tau.  Returns false when s.tau is final.
+__device__ __forceinline__ bool tau_iter_update(TauIter& s, float s0, float s1, int expo_class, float expo, float rel_tol) {
+  if (expo >= 1.0f) {
+    if (!(s0 > 1.0f) || !(s1 > 0.f)) return false;
+    const float step = threshold_step(s0, s1, expo_class, expo);
+    const float next = s.tau + step;
+    if (!(next > s.tau)) return false;
+    s.tau = next;
+    return step > rel_tol * fmaxf(1.0f, fabsf(next));
+  }
+  if (s0 >= 1.0f) s.lo = s.tau; else s.hi = s.tau;
+  float next = s.tau + (s0 - 1.0f) / (expo * s1);      // Newton on f: f' = -e S1
+  if (!(next > s.lo && next < s.hi)) next = 0.5f * (s.lo + s.hi);
+  // done when the mass is 1 to rounding, or when no float is left strictly inside the bracket (the width of the
+  // bracket says nothing here: ties put the root at -n^(1-alpha), far below any tolerance relative to |tau|)
+  const bool go = fabsf(s0 - 1.0f) > 16.0f * rel_tol && next > s.lo && next < s.hi;
+  if (go) s.tau = next;
+  else if (fabsf(s0 - 1.0f) > 16.0f * rel_tol) s.tau = s.lo;
+  return go;
 }
 
 // Fire-and-forget vector adds to global memory (sm_90+): reductions that return nothing, so no thread waits

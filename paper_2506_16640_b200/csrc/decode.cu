@@ -54,16 +54,6 @@ __device__ __forceinline__ float2 block_sum2(float x, float y, float2 (*red)[kSo
   return s;
 }
 
-// One Newton step from the left with the e-norm step; returns false when the iteration has converged.
-__device__ __forceinline__ bool newton_update(float s0, float s1, const DecodeArgs& a, float& tau) {
-  if (!(s0 > 1.0f) || !(s1 > 0.f)) return false;
-  const float step = threshold_step(s0, s1, a.expo_class, a.expo);
-  const float next = tau + step;
-  if (!(next > tau)) return false;
-  tau = next;
-  return step > 1e-7f * fmaxf(1.0f, fabsf(tau));
-}
-
 template <int D, int kSolveThreads>
 __global__ void __launch_bounds__(kSolveThreads) decode_solve_kernel(DecodeArgs a, const __nv_bfloat16* __restrict__ v,
                                                                     const float* __restrict__ scores,
@@ -164,6 +154,9 @@ __global__ void __launch_bounds__(kSolveThreads) decode_solve_kernel(DecodeArgs 
   __syncthreads();
   if (dense && tid == 0 && status) atomicAdd(status + ENTMAX_ATTN_STATUS_DENSE_ROWS, 1);
   // ---- Newton from the left on f(tau) = sum [y - tau]_+^e - 1, e-norm step
+  TauIter st;
+  st.tau = st.lo = floor_y;      // y_max - 1, the bracket's lower end (App. A)
+  st.hi = ymax;
   float tau = floor_y;
   int support = 0;
   if (!dense) {
@@ -172,7 +165,7 @@ __global__ void __launch_bounds__(kSolveThreads) decode_solve_kernel(DecodeArgs 
       for (int it = 0; it < kMaxNewtonD; ++it) {
         float s0 = 0.f, s1 = 0.f;
         for (int c = lane; c < n_cand; c += 32) {
-          const float d = list_y[c] - tau;
+          const float d = list_y[c] - st.tau;
           if (d > 0.f) {
             float ye, ye1;
             pow_pair(d, a.expo_class, a.expo, ye, ye1);
@@ -185,8 +178,9 @@ __global__ void __launch_bounds__(kSolveThreads) decode_solve_kernel(DecodeArgs 
           s0 += __shfl_xor_sync(0xffffffffu, s0, off);
           s1 += __shfl_xor_sync(0xffffffffu, s1, off);
         }
-        if (!newton_update(s0, s1, a, tau)) break;
+        if (!tau_iter_update(st, s0, s1, a.expo_class, a.expo, 1e-7f)) break;
       }
+      tau = st.tau;
       // p of every candidate (0 outside the support), in list order
       int local = 0;
       for (int c = lane; c < n_cand; c += 32) {
@@ -212,7 +206,7 @@ __global__ void __launch_bounds__(kSolveThreads) decode_solve_kernel(DecodeArgs 
     for (int it = 0; it < kMaxNewtonD; ++it) {
       float s0 = 0.f, s1 = 0.f;
       for (int j = tid; j < nv; j += kSolveThreads) {
-        const float d = y_row[j] - tau;
+        const float d = y_row[j] - st.tau;
         if (d > 0.f) {
           float ye, ye1;
           pow_pair(d, a.expo_class, a.expo, ye, ye1);
@@ -221,8 +215,9 @@ __global__ void __launch_bounds__(kSolveThreads) decode_solve_kernel(DecodeArgs 
         }
       }
       const float2 s = block_sum2<kSolveThreads>(s0, s1, red, it & 1);
-      if (!newton_update(s.x, s.y, a, tau)) break;
+      if (!tau_iter_update(st, s.x, s.y, a.expo_class, a.expo, 1e-7f)) break;
     }
+    tau = st.tau;
     __syncthreads();
   }
   // ---- O = sum_j p_j v_j
@@ -301,7 +296,7 @@ int check_decode_params(const entmax_attn_decode_params* p, DecodeArgs* a) {
   if (p->kv_capacity < p->q_len) return ENTMAX_ATTN_EINVAL_SHAPE;
   if (p->head_dim != 64 && p->head_dim != 128) return ENTMAX_ATTN_EINVAL_SHAPE;
   if ((long long)p->batch * p->heads * p->q_len > 0x7fffffffLL / 4) return ENTMAX_ATTN_EINVAL_SHAPE;
-  if (!(p->alpha > 1.0f) || !(p->alpha <= 2.0f)) return ENTMAX_ATTN_EINVAL_ALPHA;
+  if (!(p->alpha > 1.0f) || !(p->alpha <= kAlphaMax)) return ENTMAX_ATTN_EINVAL_ALPHA;
   if (!(p->sm_scale >= 0.f) || !(p->sm_scale < INFINITY)) return ENTMAX_ATTN_EINVAL_ALPHA;
   a->B = p->batch; a->H = p->heads; a->QL = p->q_len; a->NC = p->kv_capacity; a->D = p->head_dim;
   a->alpha_m1 = p->alpha - 1.0f;

@@ -143,11 +143,11 @@ __device__ __forceinline__ float score_pass(const Problem& p, const RowCtx& r, c
 }
 
 __device__ __forceinline__ float newton_tau(const Problem& p, const float* ybuf, int nv, float ymax, float* red) {
-  float tau = ymax - 1.0f;
+  TauIter st = tau_iter_start(ymax);
   for (int it = 0; it < kMaxNewton; ++it) {
     float s0 = 0.f, s1 = 0.f;
     for (int j = threadIdx.x; j < nv; j += kThreads) {
-      float y = ybuf[j] - tau;
+      float y = ybuf[j] - st.tau;
       if (y > 0.f) {
         float ye, ye1;
         pow_pair(y, p.expo_class, p.expo, ye, ye1);
@@ -156,14 +156,9 @@ __device__ __forceinline__ float newton_tau(const Problem& p, const float* ybuf,
       }
     }
     float2 s = block_sum2(s0, s1, red);
-    if (!(s.x > 1.0f) || !(s.y > 0.f)) break;
-    float step = threshold_step(s.x, s.y, p.expo_class, p.expo);
-    float next = tau + step;
-    if (!(next > tau)) break;
-    tau = next;
-    if (step <= 1e-7f * fmaxf(1.0f, fabsf(tau))) break;
+    if (!tau_iter_update(st, s.x, s.y, p.expo_class, p.expo, 1e-7f)) break;
   }
-  return tau;
+  return st.tau;
 }
 
 template <typename T, int D>

@@ -94,7 +94,7 @@ int make_problem(const entmax_attn_params* params, Problem* out) {
   p.causal = params->causal ? 1 : 0;
   p.n_mode = params->n_mode ? 1 : 0;
   p.alpha = params->alpha;
-  if (!(p.alpha > 1.0f) || !(p.alpha <= 2.0f)) return ENTMAX_ATTN_EINVAL_ALPHA;
+  if (!(p.alpha > 1.0f) || !(p.alpha <= kAlphaMax)) return ENTMAX_ATTN_EINVAL_ALPHA;
   p.sm_scale = params->sm_scale;
   if (!std::isfinite(p.sm_scale) || p.sm_scale < 0.f) return ENTMAX_ATTN_EINVAL_ALPHA;
   if (p.sm_scale == 0.f) p.sm_scale = 1.0f / std::sqrt((float)p.D);
@@ -541,7 +541,7 @@ const char* entmax_attn_strerror(int code) {
   switch (code) {
     case ENTMAX_ATTN_OK: return "ok";
     case ENTMAX_ATTN_EINVAL_SHAPE: return "invalid shape or strides (head_dim must be 64 or 128; sizes >= 1; strides multiples of 8)";
-    case ENTMAX_ATTN_EINVAL_ALPHA: return "alpha must lie in (1, 2] and sm_scale must be finite and non-negative";
+    case ENTMAX_ATTN_EINVAL_ALPHA: return "alpha must lie in (1, 64] and sm_scale must be finite and non-negative";
     case ENTMAX_ATTN_EINVAL_DTYPE: return "unknown or unsupported dtype";
     case ENTMAX_ATTN_EINVAL_ALIGN: return "tensor pointers must be 16-byte aligned";
     case ENTMAX_ATTN_EINVAL_WORKSPACE: return "workspace missing, not 256-byte aligned, or too small";

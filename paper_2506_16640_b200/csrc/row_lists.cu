@@ -169,14 +169,16 @@ __device__ __forceinline__ void sort_by_key(int (&jj)[S], float (&y)[S], int lan
 //            unless an entry lies within rounding noise of the margin cut.
 constexpr float kKeepMargin = 4e-6f;
 
-// Newton from the left on f(tau) = sum [y - tau]_+^e - 1 (convex, decreasing: monotone, never overshoots)
+// Threshold of Eq. 1 on the entries held by the warp, started at the bracket's lower end y_max - 1 (App. A):
+// Newton from the left for e >= 1, bracketed for e < 1 (tau_iter_update)
 template <int S>
-__device__ __forceinline__ float newton_warp(const Problem& p, const float (&y)[S], float tau) {
+__device__ __forceinline__ float newton_warp(const Problem& p, const float (&y)[S], float ymax) {
+  TauIter st = tau_iter_start(ymax);
   for (int it = 0; it < kMaxNewton; ++it) {
     float s0 = 0.f, s1 = 0.f;
 #pragma unroll
     for (int s = 0; s < S; ++s) {
-      const float d = y[s] - tau;
+      const float d = y[s] - st.tau;
       if (d > 0.f) {
         float ye, ye1;
         pow_pair(d, p.expo_class, p.expo, ye, ye1);
@@ -186,14 +188,9 @@ __device__ __forceinline__ float newton_warp(const Problem& p, const float (&y)[
     }
     s0 = warp_sum(s0);
     s1 = warp_sum(s1);
-    if (!(s0 > 1.0f) || !(s1 > 0.f)) break;
-    const float step = threshold_step(s0, s1, p.expo_class, p.expo);
-    const float next = tau + step;
-    if (!(next > tau)) break;
-    tau = next;
-    if (step <= 1e-7f * fmaxf(1.0f, fabsf(tau))) break;
+    if (!tau_iter_update(st, s0, s1, p.expo_class, p.expo, 1e-7f)) break;
   }
-  return tau;
+  return st.tau;
 }
 
 // Stage A on S*32 candidate slots.  Leaves the kept entries (y in Eq. 1's units) compacted from slot 0
@@ -217,7 +214,7 @@ __device__ __forceinline__ int prefilter_row(const Problem& p, Entry* list, int 
   }
   ymax = warp_max(ymax);
   __syncwarp();   // every slot is in registers before the list is overwritten
-  const float tau_a = newton_warp<S>(p, y, ymax - 1.0f);
+  const float tau_a = newton_warp<S>(p, y, ymax);
   const float cut = tau_a - kKeepMargin * fmaxf(1.0f, fabsf(tau_a));
   int kept = 0;
 #pragma unroll
@@ -260,7 +257,7 @@ __device__ __forceinline__ void finish_row(const Problem& p, const __nv_bfloat16
   ymax = warp_max(ymax);
   __syncwarp();
   sort_by_key<S>(jj, y, lane);
-  const float tau = newton_warp<S>(p, y, ymax - 1.0f);
+  const float tau = newton_warp<S>(p, y, ymax);
   float acc[PER];
 #pragma unroll
   for (int t = 0; t < PER; ++t) acc[t] = 0.f;
@@ -328,31 +325,19 @@ __device__ __forceinline__ void solve_row_full(const Problem& p, const __nv_bflo
   else finish_row<D, kSlots>(p, vbase, list, kept, o_row, tau_slot, cnt_slot, lane);
 }
 
-// Newton for 32 / W rows at once (W lanes per row); `done` rows keep their tau.
+// The same iteration for 32 / W rows at once (W lanes per row); `done` rows keep their tau.
 template <int W>
-__device__ __forceinline__ float newton_sub(const Problem& p, float y, float tau, bool done) {
+__device__ __forceinline__ float newton_sub(const Problem& p, float y, float ymax, bool done) {
+  TauIter st = tau_iter_start(ymax);
   for (int it = 0; it < kMaxNewton; ++it) {
-    const float d = y - tau;
+    const float d = y - st.tau;
     float ye = 0.f, ye1 = 0.f;
     if (d > 0.f) pow_pair(d, p.expo_class, p.expo, ye, ye1);
     const float s0 = sub_sum<W>(ye), s1 = sub_sum<W>(ye1);
-    if (!done) {
-      if (!(s0 > 1.0f) || !(s1 > 0.f)) {
-        done = true;
-      } else {
-        const float step = threshold_step(s0, s1, p.expo_class, p.expo);
-        const float next = tau + step;
-        if (!(next > tau)) {
-          done = true;
-        } else {
-          tau = next;
-          if (step <= 1e-7f * fmaxf(1.0f, fabsf(tau))) done = true;
-        }
-      }
-    }
+    if (!done) done = !tau_iter_update(st, s0, s1, p.expo_class, p.expo, 1e-7f);
     if (__all_sync(0xffffffffu, done)) break;
   }
-  return tau;
+  return st.tau;
 }
 
 // 32 / W rows at once, W lanes per row (W = 8 or 16), for rows with 1..W list entries; same two stages.
@@ -378,7 +363,7 @@ __device__ __forceinline__ void solve_rows_sub(const Problem& p, const __nv_bflo
   }
   __syncwarp();   // every entry is in registers before the compaction below overwrites the lists
   // stage A
-  const float tau_a = newton_sub<W>(p, y, sub_max<W>(y) - 1.0f, !active);
+  const float tau_a = newton_sub<W>(p, y, sub_max<W>(y), !active);
   const bool keep = active && y > tau_a - kKeepMargin * fmaxf(1.0f, fabsf(tau_a));
   // keep only those: they move to the end-stable front when sorted with the others' keys pushed to infinity
   j = keep ? j : 0x7fffffff;
@@ -398,7 +383,7 @@ __device__ __forceinline__ void solve_rows_sub(const Problem& p, const __nv_bflo
     }
   }
   // stage B
-  const float tau = newton_sub<W>(p, y, sub_max<W>(y) - 1.0f, !active);
+  const float tau = newton_sub<W>(p, y, sub_max<W>(y), !active);
   const float d = y - tau;
   const bool in = active && d > 0.f;
   float pe = 0.f, pe1;

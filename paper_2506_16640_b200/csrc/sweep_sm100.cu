@@ -175,24 +175,42 @@ __device__ __noinline__ RowState shrink_lists(RowState r, Entry* list, float a, 
         if (idx < c) e[s] = l[idx];
       }
       float tau = th * aa;
-      for (int it = 0; it < 8; ++it) {
-        float s0 = 0.f, s1 = 0.f;
+      if (expo >= 1.0f) {
+        for (int it = 0; it < 8; ++it) {
+          float s0 = 0.f, s1 = 0.f;
 #pragma unroll
-        for (int s = 0; s < kSlots; ++s) {
-          const float y = fmaf(aa, e[s].y, -tau);
-          if (y > 0.f) {
-            float ye, ye1;
-            pow_pair(y, expo_class, expo, ye, ye1);
-            s0 += ye;
-            s1 += ye1;
+          for (int s = 0; s < kSlots; ++s) {
+            const float y = fmaf(aa, e[s].y, -tau);
+            if (y > 0.f) {
+              float ye, ye1;
+              pow_pair(y, expo_class, expo, ye, ye1);
+              s0 += ye;
+              s1 += ye1;
+            }
           }
+          s0 = warp_sum(s0);
+          s1 = warp_sum(s1);
+          if (!(s0 > 1.0f) || !(s1 > 0.f)) break;
+          const float step = threshold_step(s0, s1, expo_class, expo);
+          tau += step;
+          if (step <= 1e-4f) break;
         }
-        s0 = warp_sum(s0);
-        s1 = warp_sum(s1);
-        if (!(s0 > 1.0f) || !(s1 > 0.f)) break;
-        const float step = threshold_step(s0, s1, expo_class, expo);
-        tau += step;
-        if (step <= 1e-4f) break;
+      } else {
+        // e < 1 (alpha > 2): plain bisection between the current bound (mass of the listed keys >= 1 there) and one
+        // unit above it (tau <= y_max <= bound + 1); the lower end stays a valid bound whatever the rounding does
+        float lo = tau, hi = tau + 1.0f;
+        for (int it = 0; it < 14; ++it) {
+          const float mid = 0.5f * (lo + hi);
+          float s0 = 0.f;
+#pragma unroll
+          for (int s = 0; s < kSlots; ++s) {
+            const float y = fmaf(aa, e[s].y, -mid);
+            if (y > 0.f) s0 += powf(y, expo);
+          }
+          s0 = warp_sum(s0);
+          if (s0 > 1.0f) lo = mid; else hi = mid;
+        }
+        tau = lo;
       }
       // a hair below the Newton iterate: rounding must never push the bound past the true threshold
       new_thr = fmaxf(th, (tau - 4e-6f * fmaxf(1.0f, fabsf(tau))) * inv_aa);

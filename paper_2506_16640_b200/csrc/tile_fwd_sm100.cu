@@ -296,6 +296,7 @@ __global__ void __launch_bounds__(kThreadsT, 1) tile_fwd_kernel(const __grid_con
       const float ra = valid ? a.alpha_m1 * (a.scale[(size_t)b * a.scale_sb + (size_t)h * a.N + i] * a.sm_scale) : 0.f;
       const float slope = a.alibi ? a.alibi[h] / a.sm_scale : 0.f;   // bias in accumulator units
       float tau = 0.f, ymax = -INFINITY;
+      TauIter it_tau = {0.f, 0.f, 0.f};
       bool done = !valid;
       for (int s = 0; s < kMaxSweeps && alive; ++s) {
         if (s > 0) {
@@ -458,17 +459,12 @@ __global__ void __launch_bounds__(kThreadsT, 1) tile_fwd_kernel(const __grid_con
           }
         }
         if (s == 0) {
-          tau = ymax - 1.0f;
+          it_tau = tau_iter_start(ymax);
+          tau = it_tau.tau;
         } else if (!done) {
-          if (!(s0 > 1.0f) || !(s1 > 0.f)) {
-            done = true;
-          } else {
-            const float step = threshold_step(s0, s1, a.expo_class, a.expo);   // e-norm step, see common.cuh
-            const float next = tau + step;
-            if (!(next > tau)) done = true;
-            tau = next > tau ? next : tau;
-            if (step <= 2e-6f * fmaxf(1.0f, fabsf(tau))) done = true;
-          }
+          // e >= 1: Newton from the left (e-norm step); e < 1: bracketed (see tau_iter_update)
+          done = !tau_iter_update(it_tau, s0, s1, a.expo_class, a.expo, 2e-6f);
+          tau = it_tau.tau;
         }
         const bool warp_done = __all_sync(0xffffffffu, done);
         if (lane == 0) {

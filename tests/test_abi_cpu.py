@@ -51,7 +51,7 @@ def test_workspace_bytes_and_layout(lib):
     assert lay.capacity == 256 and lay.entries_offset % 256 == 0 and lay.row_count_offset % 256 == 0
     big = _params(batch=1, heads=16, seq=32768, head_dim=128, dtype=0)
     assert lib.entmax_attn_workspace_bytes(ctypes.byref(big), 0) < 2 << 30
-    for bad in [_params(head_dim=96), _params(seq=0), _params(alpha=1.0), _params(alpha=2.5), _params(dtype=7),
+    for bad in [_params(head_dim=96), _params(seq=0), _params(alpha=1.0), _params(alpha=64.5), _params(dtype=7),
                 _params(alpha=float("nan")), _params(stride_b=8, stride_h=8, stride_n=4)]:
         assert lib.entmax_attn_workspace_bytes(ctypes.byref(bad), 0) == 0
 
@@ -113,7 +113,7 @@ def test_decode_entry_point_rejections(lib):
     need = lib.entmax_attn_decode_workspace_bytes(ctypes.byref(p))
     assert need >= 2 * 4 * 2 * 1000 * 4
     for bad in [dparams(q_len=0), dparams(q_len=9), dparams(kv_capacity=1), dparams(head_dim=96), dparams(alpha=1.0),
-                dparams(alpha=2.5), dparams(kv_stride_b=8, kv_stride_h=8, kv_stride_n=64)]:
+                dparams(alpha=100.0), dparams(kv_stride_b=8, kv_stride_h=8, kv_stride_n=64)]:
         assert lib.entmax_attn_decode_workspace_bytes(ctypes.byref(bad)) == 0
     fake, odd, nul = ctypes.c_void_p(4096), ctypes.c_void_p(4100), ctypes.c_void_p(0)
     call = lambda q, ws, nbytes, beta=None: lib.entmax_attn_decode_fwd(

@@ -243,6 +243,78 @@ def test_backward_small_full_heads(N, d, dtype, causal, alpha):
         parity.check_bwd_head(inp, alpha, bwd, bh)
 
 
+# ------------------------------------------------------------------ alpha > 2 (the paper's retrieval runs use 4 ... 64)
+@pytest.mark.parametrize("alpha", [3.0, 4.0])
+@pytest.mark.parametrize("N,d,dtype,causal", [(1, 64, "bf16", True), (130, 64, "bf16", True), (300, 128, "bf16", False),
+                                              (600, 64, "bf16", True), (97, 64, "fp32", True)])
+def test_alpha_above_two_small_shapes(N, d, dtype, causal, alpha):
+    # e = 1/(alpha-1) < 1: every solver runs its bracketed iteration; forward on every row, backward on whole heads
+    inp = make_inputs(_small("alpha_gt2", N, d, causal, dtype=dtype, plant=2 if N > 40 else 0, backward=True, seed=N + 11))
+    got = parity.run_fwd(inp, alpha)
+    bwd = parity.run_bwd(inp, alpha, got["tau"], got["dev"])
+    for bh in range(inp.workload.H):
+        parity.check_fwd_rows(inp, alpha, got, bh, np.arange(N))
+        parity.check_bwd_head_banded(inp, alpha, bwd, bh)
+
+
+@pytest.mark.parametrize("alpha", [3.0, 4.0])
+def test_alpha_above_two_dense_tiles(alpha):
+    # For alpha > 2 a support of hundreds of keys needs logits that agree to within n^-(alpha-1), i.e. ties: q = 0
+    # makes every visible key tie, p_i uniform over the i + 1 visible keys and tau_i = -(i + 1)^-(alpha-1) (Eq. 1 with
+    # sum p = 1).  Rows beyond the list capacity go through the dense-tile kernels and their bracketed sweeps.
+    N = 700
+    inp = make_inputs(_small("alpha_gt2_dense", N, 128, True, use_scale=True, backward=True, seed=93))
+    inp.q.zero_()
+    got = parity.run_fwd(inp, alpha)
+    assert int(got["status"][binding.STATUS_DENSE_ROWS]) > N
+    n = torch.arange(1, N + 1, dtype=torch.float64)
+    tau_ref = -n.pow(-(alpha - 1.0))
+    bwd = parity.run_bwd(inp, alpha, got["tau"], got["dev"])
+    for bh in range(inp.workload.H):
+        tau = got["tau"][0, bh].double().cpu()
+        assert (tau - tau_ref).abs().max().item() <= parity.tau_tol("bf16")
+        o_ref = inp.v[0, bh].double().cumsum(dim=0) / n[:, None]
+        assert (got["o"][0, bh].double().cpu() - o_ref).abs().max().item() <= parity.O_TOL
+        # every key of a row sits at the same distance above the threshold, so the gradients are well conditioned
+        parity.check_bwd_head(inp, alpha, bwd, bh)
+
+
+def test_alpha_above_two_long_rows():
+    # one 8192-token shape (sampled pre-pass, list shrinks with the bisection bound), sampled rows of every head
+    inp = make_inputs(Workload("alpha_gt2_8k", 1, 4, 8192, 64, "bf16", True, (3.0,), plant=4, plant_mode="subset",
+                               backward=True, seed_offset=95))
+    for alpha in (3.0, 4.0):
+        got = parity.run_fwd(inp, alpha)
+        bwd = parity.run_bwd(inp, alpha, got["tau"], got["dev"])
+        for bh in range(4):
+            rows = sample_rows(inp, bh, 192)
+            parity.check_fwd_rows(inp, alpha, got, bh, rows)
+        parity.check_bwd_head_banded(inp, alpha, bwd, 2)
+
+
+def test_alpha_sixteen_on_rows_it_can_resolve():
+    # alpha = 16: p = y^(1/15) cannot be normalised in floating point unless the row is one-hot or an exact tie
+    # (a key at y = 1e-7 above the threshold already weighs 0.34); planted keys three units above the rest make
+    # every planted row one-hot: tau = 15 s_max - 1, O = v of the planted key.  All other rows only have to be finite.
+    inp = make_inputs(_small("alpha16", 400, 64, True, plant=1, use_scale=True, seed=97))
+    got = parity.run_fwd(inp, 16.0)
+    assert torch.isfinite(got["tau"]).all() and torch.isfinite(got["o"].float()).all()
+    w = inp.workload
+    checked = 0
+    for bh in range(w.H):
+        q, k, v = (t[0, bh].float().numpy() for t in (inp.q, inp.k, inp.v))
+        rows = inp.planted_rows[bh]
+        ref = oracle_mod.attn_fwd_rows(q, k, v, rows, 16.0, inp.sm_scale, True, scale=inp.head_scale(bh % w.H))
+        one_hot = ref["supp"] == 1
+        tau_g = got["tau"][0, bh].cpu().numpy()[rows]
+        o_g = got["o"][0, bh].float().cpu().numpy()[rows]
+        rel = np.abs(tau_g - ref["tau"]) / np.maximum(1.0, np.abs(ref["tau"]))
+        assert rel[one_hot].max() <= parity.tau_tol("bf16")
+        assert np.abs(o_g - ref["o"])[one_hot].max() <= parity.O_TOL
+        checked += int(one_hot.sum())
+    assert checked > 100
+
+
 # ------------------------------------------------------------------ gradients of the ASEntmax scale
 @pytest.mark.parametrize("alpha", [1.25, 1.5, 2.0])
 @pytest.mark.parametrize("N,d,dtype,causal,sigma,plant", [(300, 64, "bf16", True, 1.0, 2), (700, 128, "bf16", False, 1.0, 0),
