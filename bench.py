@@ -266,9 +266,10 @@ def run_ours(args):
     # secondary: the decode shape on the same tensors: the last q_len rows of Q as the new queries, K and V as the cache
     decode = time_decode(d, w, alpha, flush) if world == 1 else None
     # secondary: the temperature axis on this shape, the other alphas and the other workloads
-    density = other = None
+    density = other = nape = None
     if world == 1 and not args.no_secondary:
         density = time_density_axis(d, w, alpha, flush, ws)
+        nape = time_nape(d, w, alpha, flush, ws)
         other = [time_workload(4, a2, flush, tensors=d, ws=ws) for a2 in (1.25, 2.0) if a2 != alpha]
 
     # end to end: pinned host buffers in, results back to pinned host buffers, copies inside the timed region
@@ -421,6 +422,10 @@ def run_ours(args):
         line["density_axis"] = {"note": "not part of `value`: the same shape and tensors with the temperature swept -- the "
                                 "paper's regime (delta = 1, gamma = -0.5, Sec. 4.1) and fixed scales c; "
                                 "supports grow as c falls", "runs": density}
+    if nape is not None:
+        line["nape_alibi"] = {"note": "not part of `value`: ALiBi slopes as in the paper's NAPE scheme (App. B); the hard "
+                              "cutoff of entmax + ALiBi lets the sweep start each 256-row item at the first K tile that can "
+                              "still hold a candidate", "runs": nape}
     if other is not None:
         line["other_workloads"] = {"note": "not part of `value`: forward / backward of the other workloads and alphas, median "
                                    "of 5 calls, L2 flushed before each", "runs": other}
@@ -534,6 +539,51 @@ def time_density_axis(d, w, alpha, flush, ws):
             res = time_fwd_bwd(t, alpha, w.causal, full(b), full(g), full(dl), flush, ws=ws, iters=3)
             res.update({"tensors": label, "scale": name, "c_at_last_row": dl + b * float(np.log(w.N)) ** g})
             runs.append(res)
+    return runs
+
+
+def time_nape(d, w, alpha, flush, ws, iters=3):
+    """The paper's NAPE scheme on the benchmark's tensors: ALiBi slopes on half of the heads (the original
+    geometric sequence 2^(-8 j / n), j = 1..n), none on the other half; beside it all heads without and all heads
+    with a slope.  The score sweep leaves out the K tiles beyond each item's hard-cutoff window."""
+    from paper_2506_16640_b200 import binding
+    dev = d["q"].device
+    H = w.H
+    geo = lambda n: [2.0 ** (-8.0 * (j + 1) / n) for j in range(n)]
+    cases = [("no slopes (every head NoPE, same kernels)", [0.0] * H),
+             ("NAPE: slopes on the first half of the heads", geo(H // 2) + [0.0] * (H - H // 2)),
+             ("slopes on every head", geo(H))]
+    o = torch.empty_like(d["q"])
+    tau = torch.empty((w.B, w.H, w.N), dtype=torch.float32, device=dev)
+    dq, dk, dv = (torch.empty_like(d["q"]) for _ in range(3))
+    ev = lambda: torch.cuda.Event(enable_timing=True)
+    runs = []
+    for label, slopes in cases:
+        sl = torch.tensor(slopes, dtype=torch.float32, device=dev)
+        st_f = torch.zeros(binding.STATUS_WORDS, dtype=torch.int32, device=dev)
+        st_b = torch.zeros(binding.STATUS_WORDS, dtype=torch.int32, device=dev)
+        tf, tb = [], []
+        for it in range(iters + 2):
+            flush.zero_()
+            e0, e1, e2, e3 = ev(), ev(), ev(), ev()
+            e0.record()
+            binding.entmax_attn_fwd_ex(d["q"], d["k"], d["v"], alpha, w.causal, d["beta"], d["gamma"], d["delta"],
+                                       alibi_slopes=sl, o=o, tau=tau, workspace=ws, status=st_f)
+            e1.record()
+            flush.zero_()
+            e2.record()
+            binding.entmax_attn_bwd_ex(d["q"], d["k"], d["v"], tau, d["d_o"], alpha, w.causal, d["beta"], d["gamma"],
+                                       d["delta"], alibi_slopes=sl, dq=dq, dk=dk, dv=dv, workspace=ws, status=st_b)
+            e3.record()
+            torch.cuda.synchronize()
+            if it >= 2:
+                tf.append(e0.elapsed_time(e1)); tb.append(e2.elapsed_time(e3))
+        f, b = st_f.tolist(), st_b.tolist()
+        assert f[0] == 0 and b[0] == 0, "device status flags set"
+        runs.append({"heads": label, "slopes": slopes, "fwd_ms": statistics.median(tf), "bwd_ms": statistics.median(tb),
+                     "fwd_sweep_steps_skipped": f[4], "fwd_sweep_steps_scored": f[5],
+                     "fwd_skipped_frac": f[4] / max(f[4] + f[5], 1), "bwd_skipped_frac": b[4] / max(b[4] + b[5], 1),
+                     "dense_path_rows": f[1]})
     return runs
 
 

@@ -86,11 +86,14 @@ typedef struct {
 
 /* Words of the optional device status array (int32[ENTMAX_ATTN_STATUS_WORDS], device memory, written
  * by the kernels of a call; zeroed at the start of that call). */
-#define ENTMAX_ATTN_STATUS_WORDS 4
+#define ENTMAX_ATTN_STATUS_WORDS 8
 #define ENTMAX_ATTN_STATUS_FLAGS 0         /* bit field below; 0 = clean run                                   */
 #define ENTMAX_ATTN_STATUS_DENSE_ROWS 1    /* rows whose support did not fit the sparse list (dense fallback)  */
 #define ENTMAX_ATTN_STATUS_TILE_SWEEPS 2   /* forward: sweeps over K spent by the dense-tile path, summed over tiles */
 #define ENTMAX_ATTN_STATUS_TILES 3         /* 128-row Q tiles the dense-tile path of this call processed           */
+#define ENTMAX_ATTN_STATUS_SKIPPED_STEPS 4 /* ALiBi heads: (256-row item, 256-key tile) steps of the score sweep that
+                                              the hard-cutoff window left out ...                                 */
+#define ENTMAX_ATTN_STATUS_SCORED_STEPS 5  /* ... and steps it still scored (both 0 without ALiBi slopes)          */
 #define ENTMAX_ATTN_FLAG_WAIT_EXPIRED 1    /* a bounded on-chip wait ran out; outputs of that call are invalid */
 #define ENTMAX_ATTN_FLAG_BAD_SCALE 2       /* some c_i was not finite                                          */
 #define ENTMAX_ATTN_FLAG_BAD_LENGTH 4      /* entmax_attn_decode_fwd: some kv_len[b] outside [q_len, kv_capacity] */
@@ -311,6 +314,14 @@ int entmax_attn_scores_debug(const entmax_attn_params* params, const void* q, co
  * cudaEvent_t passed as void*; pass NULL for both to switch the hook off.  The events stay owned by
  * the caller.  No paper counterpart. */
 int entmax_attn_profile_events(int which, void* start_event, void* stop_event);
+
+/* Self-test of the bounded on-chip waits (no paper counterpart).  Every mbarrier wait in the tensor-core kernels gives
+ * up after a time limit and makes its kernel return with ENTMAX_ATTN_FLAG_WAIT_EXPIRED in the status flags instead of
+ * hanging the GPU.  This call runs one small CTA that waits, through that same code, on a barrier nothing arrives on,
+ * with `limit_ns` (1 .. 100,000,000) as its limit.  On return of the kernel device_status[ENTMAX_ATTN_STATUS_FLAGS]
+ * has ENTMAX_ATTN_FLAG_WAIT_EXPIRED set and device_status[1] holds the microseconds the wait lasted.
+ * device_status is required here. */
+int entmax_attn_selftest_wait_expiry(uint64_t limit_ns, int32_t* device_status, void* cuda_stream);
 
 /* Text for a status code (static storage). */
 const char* entmax_attn_strerror(int code);

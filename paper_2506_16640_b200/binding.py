@@ -16,8 +16,9 @@ _HERE = os.path.dirname(os.path.abspath(__file__))
 LIB_PATH = os.path.join(_HERE, "libentmax_attn.so")
 
 DTYPE_BF16, DTYPE_FP32 = 0, 1
-STATUS_WORDS = 4
+STATUS_WORDS = 8
 STATUS_FLAGS, STATUS_DENSE_ROWS, STATUS_TILE_SWEEPS, STATUS_TILES = 0, 1, 2, 3
+STATUS_SKIPPED_STEPS, STATUS_SCORED_STEPS = 4, 5
 FLAG_WAIT_EXPIRED, FLAG_BAD_SCALE, FLAG_BAD_LENGTH = 1, 2, 4
 
 
@@ -100,6 +101,8 @@ def load():
         lib.entmax_attn_scores_debug.argtypes = [pp, vp, vp, ctypes.c_int32, fp, vp, ctypes.c_size_t, ip, vp]
         lib.entmax_attn_profile_events.restype = ctypes.c_int
         lib.entmax_attn_profile_events.argtypes = [ctypes.c_int, vp, vp]
+        lib.entmax_attn_selftest_wait_expiry.restype = ctypes.c_int
+        lib.entmax_attn_selftest_wait_expiry.argtypes = [ctypes.c_uint64, ip, vp]
         lib.entmax_attn_strerror.restype = ctypes.c_char_p
         lib.entmax_attn_strerror.argtypes = [ctypes.c_int]
         lib.entmax_attn_last_cuda_error.restype = ctypes.c_int
@@ -437,3 +440,10 @@ def read_dense_support_sizes(params: Params, workspace: torch.Tensor, rows):
     rows_t = torch.as_tensor(rows, dtype=torch.long, device=workspace.device)
     size = dense[rows_t].sum(dim=1).to(torch.int64)
     return torch.where(cnt[rows_t] == -2, size, torch.full_like(size, -1)).cpu()
+
+
+def entmax_attn_selftest_wait_expiry(limit_ns: int, status: torch.Tensor, stream=None):
+    """Runs the bounded-wait self-test: one CTA waits `limit_ns` for a barrier nothing arrives on, then returns with
+    FLAG_WAIT_EXPIRED in status[0] and the microseconds it waited in status[1]."""
+    _check(load().entmax_attn_selftest_wait_expiry(int(limit_ns), _ptr(status), _stream_ptr(stream)),
+           "entmax_attn_selftest_wait_expiry")

@@ -49,7 +49,7 @@ struct Problem {
 };
 
 struct WsLayout {
-  size_t scale, row_cnt, half_cnt, half_thr, entries, fb_count, sweep_counter, tile_count, fb_list, tile_flag, tile_list, tile_mask, scratch, acc_dk, acc_dv, dc_rows, total;
+  size_t scale, row_cnt, half_cnt, half_thr, entries, fb_count, sweep_counter, tile_count, fb_list, tile_flag, tile_list, tile_mask, alibi_blob, alibi_kmax, scratch, acc_dk, acc_dv, dc_rows, total;
   int scratch_ctas;     // CTAs of the dense-row kernels (each owns scratch_floats floats)
   size_t scratch_floats;
 };
@@ -164,7 +164,8 @@ cudaError_t launch_scale_grad(const Problem& p, const float* beta, const float* 
 //   mode 0: threshold search (forward); mode 1: threshold given in tau_in (backward)
 cudaError_t launch_sweep(const Problem& p, const void* q, const void* k, const float* scale, const float* tau_in,
                          int mode, int32_t* half_cnt, float* half_thr, Entry* entries, int32_t* work_counter,
-                         float* dump, int dump_bh, int32_t* status, cudaStream_t stream);
+                         float* dump, int dump_bh, float* alibi_blob, float* alibi_kmax, int32_t* status,
+                         cudaStream_t stream);
 
 // Dense-tile forward on the tensor cores (bf16): recomputes the Q tiles (128 rows) listed in tile_list
 // and writes O and tau of their rows marked row_cnt == -2, and into dense_cnt [B*H*N][2] the number of keys

@@ -141,6 +141,10 @@ WsLayout make_layout(const Problem& p, bool is_bwd) {
   l.tile_flag = take(q_tiles * sizeof(int32_t));
   l.tile_list = take(q_tiles * sizeof(int32_t));
   l.tile_mask = take(q_tiles * 4 * sizeof(uint32_t));   // 128 row bits per Q tile (dense-tile backward)
+  // ALiBi window of the score sweep: slopes [H] + first K tile of every 256-row work item; key norms per 256-key tile
+  const size_t items = (size_t)p.B * p.H * ((p.N + 255) / 256);
+  l.alibi_blob = take(((size_t)p.H + items) * sizeof(float));
+  l.alibi_kmax = take(items * sizeof(float));
   // dense-row CTAs: enough to fill the machine, few enough that their score rows stay modest
   l.scratch_floats = align_up((size_t)p.N, 32) * (is_bwd ? 2 : 1);   // scores (+ dP in backward)
   size_t ctas = 148 * 4;
@@ -248,8 +252,9 @@ int fwd_impl(const entmax_attn_params* params, const void* q, const void* k, con
   err = cudaMemsetAsync(tile_flag, 0, (size_t)p.B * p.H * ((p.N + 127) / 128) * sizeof(int32_t), stream);
   if (err != cudaSuccess) return fail_cuda(err);
   if (g_prof_start[0]) cudaEventRecord(g_prof_start[0], stream);
-  err = launch_sweep(p, q, k, scale, nullptr, 0, half_cnt, half_thr, entries, sweep_counter, nullptr, -1, device_status,
-                     stream);
+  err = launch_sweep(p, q, k, scale, nullptr, 0, half_cnt, half_thr, entries, sweep_counter, nullptr, -1,
+                     reinterpret_cast<float*>(ws + lay.alibi_blob), reinterpret_cast<float*>(ws + lay.alibi_kmax),
+                     device_status, stream);
   if (err != cudaSuccess) return fail_cuda(err);
   if (g_prof_stop[0]) cudaEventRecord(g_prof_stop[0], stream);
   err = launch_row_fwd(p, v, scale, row_cnt, half_cnt, half_thr, entries, o, tau, fb_count, fb_list, tile_flag, tile_list,
@@ -400,8 +405,9 @@ int bwd_impl(const entmax_attn_params* params, const void* q, const void* k, con
       if (err != cudaSuccess) return fail_cuda(err);
     } else {
       if (g_prof_start[1]) cudaEventRecord(g_prof_start[1], stream);
-      err = launch_sweep(p, q, k, scale, tau, 1, half_cnt, half_thr, entries, sweep_counter, nullptr, -1, device_status,
-                         stream);
+      err = launch_sweep(p, q, k, scale, tau, 1, half_cnt, half_thr, entries, sweep_counter, nullptr, -1,
+                         reinterpret_cast<float*>(ws + lay.alibi_blob), reinterpret_cast<float*>(ws + lay.alibi_kmax),
+                         device_status, stream);
       if (err != cudaSuccess) return fail_cuda(err);
       if (g_prof_stop[1]) cudaEventRecord(g_prof_stop[1], stream);
       err = cudaStreamWaitEvent(stream, side->join, 0);     // the accumulators are clear from here on
@@ -498,7 +504,7 @@ int entmax_attn_scores_debug(const entmax_attn_params* params, const void* q, co
   if (err != cudaSuccess) return fail_cuda(err);
   err = launch_sweep(p, q, k, scale, nullptr, 0, reinterpret_cast<int32_t*>(ws + lay.half_cnt),
                      reinterpret_cast<float*>(ws + lay.half_thr), reinterpret_cast<Entry*>(ws + lay.entries),
-                     reinterpret_cast<int32_t*>(ws + lay.sweep_counter), s_out, bh, device_status, stream);
+                     reinterpret_cast<int32_t*>(ws + lay.sweep_counter), s_out, bh, nullptr, nullptr, device_status, stream);
   return err == cudaSuccess ? ENTMAX_ATTN_OK : fail_cuda(err);
 }
 

@@ -61,14 +61,15 @@ __device__ __forceinline__ uint64_t global_ns() {
 }
 // Bounded wait.  Returns false when the CTA is aborting (this or another wait ran out of time).
 // `abort_flag` is the shared-memory address of the CTA's abort word.
-static __device__ __noinline__ bool mbar_wait_slow(uint32_t bar, uint32_t parity, uint32_t abort_flag) {
+static __device__ __noinline__ bool mbar_wait_slow(uint32_t bar, uint32_t parity, uint32_t abort_flag,
+                                                   uint64_t limit_ns = kWaitLimitNs) {
   const uint64_t t0 = global_ns();
   uint32_t spins = 0;
   for (;;) {
     if (mbar_try_wait(bar, parity)) return true;
     if ((++spins & 63u) == 0u) {
       if (lds_u32(abort_flag)) return false;
-      if (global_ns() - t0 > kWaitLimitNs) {
+      if (global_ns() - t0 > limit_ns) {
         sts_u32(abort_flag, 1u);
         return false;
       }

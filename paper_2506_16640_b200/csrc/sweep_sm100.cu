@@ -139,6 +139,16 @@ __device__ __forceinline__ void tma_load_5d(uint32_t dst, const CUtensorMap* map
       : "memory");
 }
 
+// ALiBi window (kAlibi kernels).  The penalty m_h (i - j) grows with the distance, so keys farther back than a
+// bound cannot reach the support (the paper's hard cutoff d_max for entmax + ALiBi): alibi_window_kernel below
+// finds, per work item, the first K tile that can still hold a candidate, and all three roles start there.
+// In those kernels `dump` points to a blob in the workspace: float slopes [H], then int32 first tiles [n_items].
+template <bool kAlibi>
+__device__ __forceinline__ int first_tile(const SweepArgs& a, int k) {
+  if constexpr (kAlibi) return reinterpret_cast<const int32_t*>(a.dump)[a.H + k];
+  return 0;
+}
+
 // ------------------------------------------------------------- consumer side: one half-row per thread
 struct RowState {
   float thr;       // candidates are accumulators above this (accumulator units)
@@ -320,15 +330,20 @@ __global__ void __launch_bounds__(kThreads, 1) sweep_kernel(const __grid_constan
           const int tx = qtile_tiles(a, item, x);
           tiles = tx > tiles ? tx : tiles;
         }
-        const int ts = sample_tiles(a, item);
+        // tiles before tf (and sampled tiles before ts0) lie outside the ALiBi window: t counts from there
+        const int tf = first_tile<kAlibi>(a, k);
+        const int ts_all = sample_tiles(a, item);
+        const int ts0 = kAlibi ? min(tf / kSampleStride, ts_all) : 0;
+        const int ts = ts_all - ts0;
+        tiles -= tf;
         for (int t = 0; t < ts + tiles && alive; ++t) {
           alive = mbar_wait(k_empty + 8 * stage, kphase ^ 1u, abort_flag);
           if (!alive) break;
           mbar_expect_tx(k_full + 8 * stage, C::kKBytes);
           for (int hf = 0; hf < C::kHalves; ++hf) {
             const uint32_t dst = k_smem + stage * C::kKBytes + hf * (BN * 128);
-            if (t < ts) tma_load_5d(dst, &map_ks, k_full + 8 * stage, hf * 64, 0, t * BN, h, b);
-            else tma_load_4d(dst, &map_k, k_full + 8 * stage, hf * 64, (t - ts) * BN, h, b);
+            if (t < ts) tma_load_5d(dst, &map_ks, k_full + 8 * stage, hf * 64, 0, (ts0 + t) * BN, h, b);
+            else tma_load_4d(dst, &map_k, k_full + 8 * stage, hf * 64, (tf + t - ts) * BN, h, b);
           }
           if (++stage == C::kStages) { stage = 0; kphase ^= 1u; }
           if (t == 0) {
@@ -370,7 +385,11 @@ __global__ void __launch_bounds__(kThreads, 1) sweep_kernel(const __grid_constan
           tx[x] = qtile_tiles(a, item, x);
           tiles = tx[x] > tiles ? tx[x] : tiles;
         }
-        const int ts = sample_tiles(a, item);
+        const int tf = first_tile<kAlibi>(a, k);
+        const int ts_all = sample_tiles(a, item);
+        const int ts = ts_all - (kAlibi ? min(tf / kSampleStride, ts_all) : 0);
+        tiles -= tf;
+        for (int x = 0; x < kQTiles; ++x) tx[x] = tx[x] > 0 ? tx[x] - tf : 0;   // every valid Q tile reaches past tf
         for (int t = 0; t < ts + tiles && alive; ++t) {
           alive = mbar_wait(k_full + 8 * stage, kphase, abort_flag);
           if (!alive) break;
@@ -430,6 +449,7 @@ __global__ void __launch_bounds__(kThreads, 1) sweep_kernel(const __grid_constan
       decode_item(a, k, bh, item);
       const int tiles = qtile_tiles(a, item, x);
       if (tiles == 0) continue;
+      const int tf = first_tile<kAlibi>(a, k);
       const int h = bh % a.H;
       const int tile_row0 = item * kItemRows + x * BM;
       const int i = tile_row0 + row_local;
@@ -468,11 +488,18 @@ __global__ void __launch_bounds__(kThreads, 1) sweep_kernel(const __grid_constan
       // ---- sampled tiles first (forward mode, long rows): maxima only, nothing is pushed -- every sampled
       //      key comes by again in the real stream.  Column c of sampled tile t is key kSampleStride * (t*BN + c).
       const int ts = sample_tiles(a, item);
-      if (ts > 0) {
+      const int ts0 = kAlibi ? min(tf / kSampleStride, ts) : 0;
+      if (kAlibi && a.status && cw == 0 && lane == 0) {
+        // K-tile steps of this item left out by the window / still scored
+        const int t_item = max(tiles, qtile_tiles(a, item, kQTiles - 1));
+        atomicAdd(a.status + ENTMAX_ATTN_STATUS_SKIPPED_STEPS, tf);
+        atomicAdd(a.status + ENTMAX_ATTN_STATUS_SCORED_STEPS, t_item - tf);
+      }
+      if (ts > ts0) {
         // largest sampled group index that is a key this row may look at
         int glim = lim / kSampleStride;
         if (glim > a.N / kSampleStride - 1) glim = a.N / kSampleStride - 1;
-        for (int t = 0; t < ts && alive; ++t) {
+        for (int t = ts0; t < ts && alive; ++t) {
           alive = __all_sync(0xffffffffu, mbar_wait(my_full, fphase, abort_flag));
           if (!alive) break;
           fphase ^= 1u;
@@ -505,7 +532,7 @@ __global__ void __launch_bounds__(kThreads, 1) sweep_kernel(const __grid_constan
           }
         }
       }
-      for (int t = 0; t < tiles && alive; ++t) {
+      for (int t = tf; t < tiles && alive; ++t) {
         // the warp leaves together: tcgen05.ld needs all 32 lanes
         alive = __all_sync(0xffffffffu, mbar_wait(my_full, fphase, abort_flag));
         if (!alive) break;
@@ -653,6 +680,107 @@ __global__ void __launch_bounds__(kThreads, 1) sweep_kernel(const __grid_constan
   }
 }
 
+// ---------------------------------------------------------------------------- ALiBi window pre-kernels
+// Largest key norm of every K tile (BN keys) of every head: kmax[bh * k_tiles + t].
+template <int HD>
+__global__ void __launch_bounds__(BN) key_norm_kernel(const __nv_bfloat16* __restrict__ k, int H, int N, long long sb,
+                                                      long long sh, long long sn, int k_tiles, float* __restrict__ kmax) {
+  __shared__ float red[BN / 32];
+  const int bh = blockIdx.x / k_tiles, t = blockIdx.x - bh * k_tiles;
+  const int b = bh / H, h = bh - b * H;
+  const int j = t * BN + threadIdx.x;
+  float n2 = 0.f;
+  if (j < N) {
+    const __nv_bfloat16* row = k + (size_t)b * sb + (size_t)h * sh + (size_t)j * sn;
+#pragma unroll
+    for (int c = 0; c < HD / 8; ++c) {
+      const uint4 raw = *reinterpret_cast<const uint4*>(row + 8 * c);
+      const uint32_t w[4] = {raw.x, raw.y, raw.z, raw.w};
+#pragma unroll
+      for (int u = 0; u < 4; ++u) {
+        const float2 f = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(&w[u]));
+        n2 = fmaf(f.x, f.x, fmaf(f.y, f.y, n2));
+      }
+    }
+  }
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) n2 = fmaxf(n2, __shfl_xor_sync(0xffffffffu, n2, o));
+  if ((threadIdx.x & 31) == 0) red[threadIdx.x >> 5] = n2;
+  __syncthreads();
+  if (threadIdx.x == 0) {
+    float m = red[0];
+    for (int w = 1; w < BN / 32; ++w) m = fmaxf(m, red[w]);
+    kmax[blockIdx.x] = sqrtf(m);
+  }
+}
+
+// First K tile of every work item that can hold a candidate.  For row i a lower bound on its threshold is known
+// before any score: its own key (distance 0, no penalty) gives tau_i >= y_ii - 1 (App. A bracket), i.e. in
+// accumulator units thr_i >= <q_i,k_i> - 1/a_i; in backward mode thr_i is the given tau_i.  A key j of tile t scores at
+// most |q_i| max_t|k| - (m_h / sm_scale) (i - j_last(t)) (Cauchy-Schwarz; the slope in accumulator units), so the tile
+// is outside row i's support when that is <= thr_i: the paper's hard cutoff d_max for entmax with ALiBi, with the
+// logit range bounded by norms.  The item starts at the first tile some row of it still needs.
+// blob: float slopes [H] (copied here), then int32 first tiles [n_items].
+template <int HD>
+__global__ void __launch_bounds__(kItemRows) alibi_window_kernel(const __nv_bfloat16* __restrict__ q,
+                                                                 const __nv_bfloat16* __restrict__ k, SweepArgs a,
+                                                                 long long sb, long long sh, long long sn,
+                                                                 const float* __restrict__ slopes,
+                                                                 const float* __restrict__ kmax, int k_tiles,
+                                                                 float* __restrict__ blob) {
+  __shared__ int red[kItemRows / 32];
+  int bh, item;
+  decode_item(a, blockIdx.x, bh, item);
+  const int b = bh / a.H, h = bh - b * a.H;
+  const int i = item * kItemRows + threadIdx.x;
+  const float slope = slopes[h] / a.sm_scale;
+  int need = item;   // never past the tile that holds the item's first row (and its own key)
+  if (i < a.N && slope > 0.f) {
+    const size_t base = (size_t)b * sb + (size_t)h * sh + (size_t)i * sn;
+    float qq = 0.f, qk = 0.f;
+#pragma unroll
+    for (int c = 0; c < HD / 8; ++c) {
+      const uint4 rq = *reinterpret_cast<const uint4*>(q + base + 8 * c);
+      const uint4 rk = *reinterpret_cast<const uint4*>(k + base + 8 * c);
+      const uint32_t wq[4] = {rq.x, rq.y, rq.z, rq.w}, wk[4] = {rk.x, rk.y, rk.z, rk.w};
+#pragma unroll
+      for (int u = 0; u < 4; ++u) {
+        const float2 fq = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(&wq[u]));
+        const float2 fk = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(&wk[u]));
+        qq = fmaf(fq.x, fq.x, fmaf(fq.y, fq.y, qq));
+        qk = fmaf(fq.x, fk.x, fmaf(fq.y, fk.y, qk));
+      }
+    }
+    const size_t grow = (size_t)bh * a.N + i;
+    const float ra = a.alpha_m1 * (a.scale[(size_t)b * a.scale_sb + (size_t)h * a.N + i] * a.sm_scale);
+    float thr = INFINITY;          // no usable bound: the row needs every tile
+    if (ra > 0.f && ra < INFINITY) {
+      thr = a.mode == 0 ? qk - 1.0f / ra : a.tau_in[grow] / ra;
+      thr -= 1e-5f * fabsf(thr) + 1e-6f;     // rounding of the dot product and of the bound
+    }
+    const float qn = sqrtf(qq) * 1.0002f;    // rounding of the norms
+    need = 0;
+    if (thr < INFINITY) {
+      for (; need < item; ++need) {
+        const int j_last = need * BN + BN - 1;
+        if (j_last >= i) break;
+        if (qn * kmax[(size_t)bh * k_tiles + need] - slope * (float)(i - j_last) > thr) break;
+      }
+    }
+  } else if (i < a.N) {
+    need = 0;                      // no positional term on this head
+  }
+  for (int o = 16; o > 0; o >>= 1) need = min(need, __shfl_xor_sync(0xffffffffu, need, o));
+  if ((threadIdx.x & 31) == 0) red[threadIdx.x >> 5] = need;
+  __syncthreads();
+  if (threadIdx.x == 0) {
+    int m = red[0];
+    for (int w = 1; w < kItemRows / 32; ++w) m = min(m, red[w]);
+    reinterpret_cast<int32_t*>(blob)[a.H + blockIdx.x] = m;
+    blob[h] = slopes[h];
+  }
+}
+
 // cuTensorMapEncodeTiled through the runtime's driver entry point lookup (no link against libcuda)
 typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
                                   const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
@@ -738,7 +866,8 @@ cudaError_t launch_impl(const Problem& p, const void* q, const void* k, SweepArg
 
 cudaError_t launch_sweep(const Problem& p, const void* q, const void* k, const float* scale, const float* tau_in,
                          int mode, int32_t* half_cnt, float* half_thr, Entry* entries, int32_t* work_counter,
-                         float* dump, int dump_bh, int32_t* status, cudaStream_t stream) {
+                         float* dump, int dump_bh, float* alibi_blob, float* alibi_kmax, int32_t* status,
+                         cudaStream_t stream) {
   SweepArgs args;
   args.B = p.B; args.H = p.H; args.N = p.N;
   args.causal = p.causal;
@@ -753,12 +882,29 @@ cudaError_t launch_sweep(const Problem& p, const void* q, const void* k, const f
   args.half_cnt = half_cnt;
   args.half_thr = half_thr;
   args.entries = entries;
-  args.dump = p.alibi ? const_cast<float*>(p.alibi) : dump;
+  args.dump = p.alibi ? alibi_blob : dump;
   args.dump_bh = dump_bh;
   args.status = status;
   args.work_counter = work_counter;
   args.items_per_bh = (p.N + kItemRows - 1) / kItemRows;
   args.n_items = args.items_per_bh * p.B * p.H;
+  if (p.alibi && !dump) {
+    // the window: key norms per K tile, then the first tile of every item (and the slopes) into the blob
+    const int k_tiles = (p.N + BN - 1) / BN;
+    const __nv_bfloat16* qb = static_cast<const __nv_bfloat16*>(q);
+    const __nv_bfloat16* kb = static_cast<const __nv_bfloat16*>(k);
+    if (p.D == 64) {
+      key_norm_kernel<64><<<p.B * p.H * k_tiles, BN, 0, stream>>>(kb, p.H, p.N, p.sb, p.sh, p.sn, k_tiles, alibi_kmax);
+      alibi_window_kernel<64><<<args.n_items, kItemRows, 0, stream>>>(qb, kb, args, p.sb, p.sh, p.sn, p.alibi, alibi_kmax,
+                                                                      k_tiles, alibi_blob);
+    } else {
+      key_norm_kernel<128><<<p.B * p.H * k_tiles, BN, 0, stream>>>(kb, p.H, p.N, p.sb, p.sh, p.sn, k_tiles, alibi_kmax);
+      alibi_window_kernel<128><<<args.n_items, kItemRows, 0, stream>>>(qb, kb, args, p.sb, p.sh, p.sn, p.alibi, alibi_kmax,
+                                                                       k_tiles, alibi_blob);
+    }
+    cudaError_t err = cudaGetLastError();
+    if (err != cudaSuccess) return err;
+  }
   if (dump) return p.D == 64 ? launch_impl<64, true, false>(p, q, k, args, stream)
                              : launch_impl<128, true, false>(p, q, k, args, stream);
   if (p.alibi) return p.D == 64 ? launch_impl<64, false, true>(p, q, k, args, stream)

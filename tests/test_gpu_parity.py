@@ -468,6 +468,51 @@ def test_alibi_bf16_causal_sparse_rows(N, d, alpha):
     _check_alibi(inp, alpha, True, [0.0, 0.05], None)
 
 
+def test_alibi_window_skips_far_tiles_and_keeps_parity():
+    # NAPE-style heads at a length where the hard cutoff bites: slopes 0 (NoPE), 0.5, 0.1 and 0.02.  The sweep starts
+    # every work item at the first K tile that can still hold a candidate (norm bound on the logits); forward and
+    # backward (tau-only: its sweep has the exact threshold as its bound) must still match the oracle, which scores
+    # every visible key
+    N = 8192
+    inp = make_inputs(Workload("alibi_window", 1, 4, N, 64, "bf16", True, (1.5,), plant=3, plant_mode="subset",
+                               backward=True, seed_offset=83))
+    slopes = [0.0, 0.5, 0.1, 0.02]
+    dev = parity.to_device(inp)
+    sl = torch.tensor(slopes, dtype=torch.float32, device="cuda")
+    for alpha in (1.5, 2.0):
+        st = torch.zeros(binding.STATUS_WORDS, dtype=torch.int32, device="cuda")
+        o, tau = binding.entmax_attn_fwd_ex(dev["q"], dev["k"], dev["v"], alpha, True, dev["beta"], dev["gamma"],
+                                            dev["delta"], alibi_slopes=sl, status=st)
+        st2 = torch.zeros(binding.STATUS_WORDS, dtype=torch.int32, device="cuda")
+        dq, dk, dv, _, _ = binding.entmax_attn_bwd_ex(dev["q"], dev["k"], dev["v"], tau, dev["d_o"], alpha, True,
+                                                      dev["beta"], dev["gamma"], dev["delta"], alibi_slopes=sl, status=st2)
+        torch.cuda.synchronize()
+        assert int(st[binding.STATUS_FLAGS]) == 0 and int(st2[binding.STATUS_FLAGS]) == 0
+        for status in (st, st2):
+            skipped, scored = int(status[binding.STATUS_SKIPPED_STEPS]), int(status[binding.STATUS_SCORED_STEPS])
+            # 4 heads x 32 items; an item at row r sees (r + 256) / 256 key tiles: 4 * (1 + ... + 32) steps in all
+            assert skipped + scored == 4 * 32 * 33 // 2
+            assert skipped > 0.4 * (skipped + scored), (skipped, scored)
+        for h in range(4):
+            q, k, v, g = (t[0, h].float().numpy() for t in (inp.q, inp.k, inp.v, inp.d_o))
+            rows = sample_rows(inp, h, 160)
+            f = oracle_mod.attn_fwd_rows(q, k, v, rows, alpha, inp.sm_scale, True, scale=inp.head_scale(h), alibi=slopes[h])
+            rt = torch.from_numpy(rows)
+            tau_err = np.abs(tau[0, h].cpu()[rt].double().numpy() - f["tau"]) / np.maximum(1.0, np.abs(f["tau"]))
+            assert tau_err.max() <= parity.tau_tol("bf16"), (h, tau_err.max())
+            assert np.abs(o[0, h].float().cpu()[rt].numpy() - f["o"]).max() <= parity.O_TOL
+            if alpha < 2.0:
+                rq, _ = oracle_mod.attn_bwd_rows(q, k, v, g, rows, alpha, inp.sm_scale, True, scale=inp.head_scale(h),
+                                                 alibi=slopes[h])
+                parity.grad_close("dQ rows", dq[0, h].float().cpu()[rt].numpy(), rq)
+        # a whole head of dK, dV (every row contributes) on the steepest slope
+        if alpha < 2.0:
+            q, k, v, g = (t[0, 1].float().numpy() for t in (inp.q, inp.k, inp.v, inp.d_o))
+            rq, rk, rv = oracle_mod.attn_bwd_head(q, k, v, g, alpha, inp.sm_scale, True, scale=inp.head_scale(1), alibi=slopes[1])
+            parity.grad_close("dK", dk[0, 1].float().cpu().numpy(), rk)
+            parity.grad_close("dV", dv[0, 1].float().cpu().numpy(), rv)
+
+
 def test_alibi_bf16_causal_dense_rows():
     inp = make_inputs(_small("alibi_dense", 600, 128, True, backward=True, use_scale=False, sigma=0.05, seed=19))
     _check_alibi(inp, 1.5, True, [0.002, 0.0005], True)
