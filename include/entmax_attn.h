@@ -89,7 +89,7 @@ typedef struct {
 #define ENTMAX_ATTN_STATUS_WORDS 8
 #define ENTMAX_ATTN_STATUS_FLAGS 0         /* bit field below; 0 = clean run                                   */
 #define ENTMAX_ATTN_STATUS_DENSE_ROWS 1    /* rows whose support did not fit the sparse list (dense fallback)  */
-#define ENTMAX_ATTN_STATUS_TILE_SWEEPS 2   /* forward: sweeps over K spent by the dense-tile path, summed over tiles */
+#define ENTMAX_ATTN_STATUS_TILE_SWEEPS 2   /* forward: full-length sweeps over K spent by the dense-tile path, summed over tiles */
 #define ENTMAX_ATTN_STATUS_TILES 3         /* 128-row Q tiles the dense-tile path of this call processed           */
 #define ENTMAX_ATTN_STATUS_SKIPPED_STEPS 4 /* ALiBi heads: (256-row item, 256-key tile) steps of the score sweep that
                                               the hard-cutoff window left out ...                                 */

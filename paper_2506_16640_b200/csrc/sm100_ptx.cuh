@@ -172,6 +172,32 @@ __device__ __forceinline__ void tmem_ld_wait() { asm volatile("tcgen05.wait::ld.
 constexpr uint32_t kDescHi = (1024u >> 4) | (1u << 14) | (2u << 29);
 __device__ __forceinline__ uint32_t smem_desc_lo(uint32_t saddr) { return ((saddr & 0x3FFFFu) >> 4) | (1u << 16); }
 
+// Packed pairs of floats (sm_100: two fp32 operations per instruction on a 64-bit register pair)
+typedef unsigned long long f32x2;
+__device__ __forceinline__ f32x2 pack2(float a, float b) {
+  f32x2 r;
+  asm("mov.b64 %0, {%1, %2};" : "=l"(r) : "f"(a), "f"(b));
+  return r;
+}
+__device__ __forceinline__ void unpack2(f32x2 v, float& a, float& b) {
+  asm("mov.b64 {%0, %1}, %2;" : "=f"(a), "=f"(b) : "l"(v));
+}
+__device__ __forceinline__ f32x2 fma2(f32x2 a, f32x2 b, f32x2 c) {
+  f32x2 r;
+  asm("fma.rn.f32x2 %0, %1, %2, %3;" : "=l"(r) : "l"(a), "l"(b), "l"(c));
+  return r;
+}
+__device__ __forceinline__ f32x2 mul2(f32x2 a, f32x2 b) {
+  f32x2 r;
+  asm("mul.rn.f32x2 %0, %1, %2;" : "=l"(r) : "l"(a), "l"(b));
+  return r;
+}
+__device__ __forceinline__ f32x2 add2(f32x2 a, f32x2 b) {
+  f32x2 r;
+  asm("add.rn.f32x2 %0, %1, %2;" : "=l"(r) : "l"(a), "l"(b));
+  return r;
+}
+
 __device__ __forceinline__ float max3(float a, float b, float c) {
   float r;
   asm("max.f32 %0, %1, %2, %3;" : "=f"(r) : "f"(a), "f"(b), "f"(c));
@@ -193,6 +219,10 @@ __device__ __forceinline__ float warp_sum(float x) {
 // Defined in tile_fwd_sm100.cu.
 cudaError_t make_tile_map(CUtensorMap* map, const void* base, int D, int N, int H, int B, int64_t sn, int64_t sh,
                           int64_t sb, int box_rows = 128);
+// The same tensor as a 5-D map (D, key % stride, key / stride, H, B): a box of box_rows rows along "key / stride" at
+// phase 0 is every stride-th key.  Keys past stride * (N / stride) are not part of the view; N >= stride is required.
+cudaError_t make_sampled_tile_map(CUtensorMap* map, const void* base, int D, int N, int H, int B, int64_t sn, int64_t sh,
+                                  int64_t sb, int stride, int box_rows = 128);
 
 
 }  // namespace sm100

@@ -28,10 +28,25 @@ namespace {
 
 using namespace sm100;
 
+__device__ __forceinline__ void tma_load_5d(uint32_t dst, const CUtensorMap* map, uint32_t bar, int c0, int c1, int c2,
+                                            int c3, int c4) {
+  asm volatile(
+      "cp.async.bulk.tensor.5d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5, %6, %7}], [%2];"
+      ::"r"(dst), "l"(reinterpret_cast<uint64_t>(map)), "r"(bar), "r"(c0), "r"(c1), "r"(c2), "r"(c3), "r"(c4)
+      : "memory");
+}
+
 constexpr int TM = 128;            // query rows per item = TMEM lanes
 constexpr int TN = 128;            // keys per K/V tile
 constexpr int kThreadsT = 10 * 32;    // TMA warp, MMA warp, eight consumer warps
 constexpr int kMaxSweeps = 48;     // 1 max sweep + at most 46 Newton sweeps + the output sweep
+// Sampled start: long rows first solve Eq. 1's threshold on every kTileSampleStride-th key (sweeps an eighth as long).
+// The threshold of a subset never exceeds that of the whole row, so the full-row Newton iteration may start from it
+// (steps from the left of the root never pass it, e >= 1) instead of from y_max - 1, and needs no y_max sweep.
+constexpr int kTileSampleStride = 8;
+constexpr int kSampleMinTiles = 16;    // K tiles a Q tile must see for the sampled start to pay
+constexpr int kSampleSweepCap = 12;    // sampled sweeps at most
+enum SweepKind : int { kSampleMax = 0, kSampleNewton = 1, kFullMax = 2, kFullNewton = 3, kOutput = 4 };
 constexpr int kPBytes = TM * TN * 2;
 
 template <int HD>
@@ -88,6 +103,7 @@ template <int HD, int EC>
 __global__ void __launch_bounds__(kThreadsT, 1) tile_fwd_kernel(const __grid_constant__ CUtensorMap map_q,
                                                                const __grid_constant__ CUtensorMap map_k,
                                                                const __grid_constant__ CUtensorMap map_v,
+                                                               const __grid_constant__ CUtensorMap map_ks,
                                                                const TileArgsK a) {
   using C = TCfg<HD>;
   extern __shared__ uint8_t smem_raw[];
@@ -147,17 +163,42 @@ __global__ void __launch_bounds__(kThreadsT, 1) tile_fwd_kernel(const __grid_con
   tc_fence_after();
   const uint32_t tmem_base = lds_u32(tmem_slot);
 
-  // Sweep s of an item: 0 finds the row maxima, then Newton sweeps until the consumers report that every
-  // row has converged (or the cap is reached), then the output sweep.  All roles evaluate this the same way.
-  auto sweep_is_output = [&](int s) -> bool {
-    return s == kMaxSweeps - 1 || (s >= 2 && lds_u32(done_word + 4 * ((s - 1) % 3)) != 0u);
-  };
+  // Sweeps of an item.  Without the sampled start: sweep 0 finds the row maxima, then Newton sweeps until the
+  // consumers report that every row has converged (or the cap is reached), then the output sweep.  With it: a maxima
+  // sweep and Newton sweeps over the sampled keys first, then Newton sweeps over all keys from the sample's
+  // threshold, then the output sweep.  All roles evaluate this the same way, once per sweep, after the vote is in.
   auto item_tiles = [&](int tile) -> int {
     const int row0 = tile * TM;
     if (!a.causal) return (a.N + TN - 1) / TN;
     int last_row = row0 + TM - 1;
     if (last_row > a.N - 1) last_row = a.N - 1;
     return last_row / TN + 1;
+  };
+  // sampled K tiles of an item (0: no sampled start)
+  auto item_sample_tiles = [&](int tile) -> int {
+    if (a.expo < 1.0f || item_tiles(tile) < kSampleMinTiles) return 0;
+    int last_row = tile * TM + TM - 1;
+    if (last_row > a.N - 1) last_row = a.N - 1;
+    const int n_vis = a.causal ? last_row + 1 : a.N;
+    int groups = (n_vis + kTileSampleStride - 1) / kTileSampleStride;
+    if (groups > a.N / kTileSampleStride) groups = a.N / kTileSampleStride;
+    return (groups + TN - 1) / TN;
+  };
+  auto sweep_kind = [&](int s, int& phase, int& n_full) -> int {
+    const bool prev_done = s >= 1 && lds_u32(done_word + 4 * ((s - 1) % 3)) != 0u;
+    if (phase == 0) {
+      if (s == 0) return kSampleMax;
+      if ((prev_done && s >= 2) || s >= kSampleSweepCap) {
+        phase = 1;
+        n_full = 1;
+        return kFullNewton;
+      }
+      return kSampleNewton;
+    }
+    if (s == 0) return kFullMax;
+    if (s == kMaxSweeps - 1 || (prev_done && n_full >= 1)) return kOutput;
+    ++n_full;
+    return kFullNewton;
   };
 
   if (warp == 0) {
@@ -170,7 +211,8 @@ __global__ void __launch_bounds__(kThreadsT, 1) tile_fwd_kernel(const __grid_con
         const int id = a.tile_list[it];
         const int bh = id / a.tiles_per_head, tile = id - bh * a.tiles_per_head;
         const int b = bh / a.H, h = bh - b * a.H;
-        const int tiles = item_tiles(tile);
+        const int tiles = item_tiles(tile), stiles = item_sample_tiles(tile);
+        int phase = stiles > 0 ? 0 : 1, n_full = 0;
         alive = mbar_wait(q_empty, qphase ^ 1u, abort_flag);
         if (!alive) break;
         mbar_expect_tx(q_full, C::kQBytes);
@@ -183,13 +225,18 @@ __global__ void __launch_bounds__(kThreadsT, 1) tile_fwd_kernel(const __grid_con
             cphase ^= 1u;
             if (!alive) break;
           }
-          const bool output = sweep_is_output(s);
-          for (int t = 0; t < tiles && alive; ++t) {
+          const int kind = sweep_kind(s, phase, n_full);
+          const bool output = kind == kOutput, smp = kind <= kSampleNewton;
+          const int nt = smp ? stiles : tiles;
+          for (int t = 0; t < nt && alive; ++t) {
             alive = mbar_wait(kv_empty + 8 * stage, kvphase ^ 1u, abort_flag);
             if (!alive) break;
             mbar_expect_tx(kv_full + 8 * stage, output ? 2 * C::kKBytes : C::kKBytes);
-            for (int hf = 0; hf < C::kHalves; ++hf)
-              tma_load_4d(k_smem + stage * C::kKBytes + hf * (TN * 128), &map_k, kv_full + 8 * stage, hf * 64, t * TN, h, b);
+            for (int hf = 0; hf < C::kHalves; ++hf) {
+              const uint32_t dst = k_smem + stage * C::kKBytes + hf * (TN * 128);
+              if (smp) tma_load_5d(dst, &map_ks, kv_full + 8 * stage, hf * 64, 0, t * TN, h, b);
+              else tma_load_4d(dst, &map_k, kv_full + 8 * stage, hf * 64, t * TN, h, b);
+            }
             if (output) {
               for (int hf = 0; hf < C::kHalves; ++hf)
                 tma_load_4d(v_smem + stage * C::kKBytes + hf * (TN * 128), &map_v, kv_full + 8 * stage, hf * 64, t * TN, h,
@@ -215,7 +262,8 @@ __global__ void __launch_bounds__(kThreadsT, 1) tile_fwd_kernel(const __grid_con
       for (int it = blockIdx.x; it < n_tiles && alive; it += gridDim.x) {
         const int id = a.tile_list[it];
         const int tile = id % a.tiles_per_head;
-        const int tiles = item_tiles(tile);
+        const int tiles = item_tiles(tile), stiles = item_sample_tiles(tile);
+        int phase = stiles > 0 ? 0 : 1, n_full = 0;
         alive = mbar_wait(q_full, qphase, abort_flag);
         qphase ^= 1u;
         if (!alive) break;
@@ -225,14 +273,16 @@ __global__ void __launch_bounds__(kThreadsT, 1) tile_fwd_kernel(const __grid_con
             cphase ^= 1u;
             if (!alive) break;
           }
-          const bool output = sweep_is_output(s);
+          const int kind = sweep_kind(s, phase, n_full);
+          const bool output = kind == kOutput;
+          const int nt = kind <= kSampleNewton ? stiles : tiles;
           if (output) {
             // the previous item's O must have been read before this item's first PV overwrites it
             alive = mbar_wait(o_empty, ophase ^ 1u, abort_flag);
             ophase ^= 1u;
             if (!alive) break;
           }
-          for (int t = 0; t < tiles && alive; ++t) {
+          for (int t = 0; t < nt && alive; ++t) {
             alive = mbar_wait(kv_full + 8 * stage, kvphase, abort_flag);
             if (alive) alive = mbar_wait(s_empty + 8 * sbuf, sphase[sbuf] ^ 1u, abort_flag);
             if (!alive) break;
@@ -288,11 +338,15 @@ __global__ void __launch_bounds__(kThreadsT, 1) tile_fwd_kernel(const __grid_con
       const int id = a.tile_list[it];
       const int bh = id / a.tiles_per_head, tile = id - bh * a.tiles_per_head;
       const int b = bh / a.H, h = bh - b * a.H;
-      const int tiles = item_tiles(tile);
+      const int tiles = item_tiles(tile), stiles = item_sample_tiles(tile);
+      int phase = stiles > 0 ? 0 : 1, n_full = 0, n_smp = 0;
       const int i = tile * TM + row_local;
       const bool valid = i < a.N;
       const size_t grow = (size_t)bh * a.N + (valid ? i : 0);
       const int lim = a.causal ? i : a.N - 1;
+      // last sampled column (key kTileSampleStride * column) this row may look at
+      int glim = lim / kTileSampleStride;
+      if (glim > a.N / kTileSampleStride - 1) glim = a.N / kTileSampleStride - 1;
       const float ra = valid ? a.alpha_m1 * (a.scale[(size_t)b * a.scale_sb + (size_t)h * a.N + i] * a.sm_scale) : 0.f;
       const float slope = a.alibi ? a.alibi[h] / a.sm_scale : 0.f;   // bias in accumulator units
       float tau = 0.f, ymax = -INFINITY;
@@ -304,12 +358,19 @@ __global__ void __launch_bounds__(kThreadsT, 1) tile_fwd_kernel(const __grid_con
           cphase ^= 1u;
           if (!alive) break;
         }
-        const bool output = sweep_is_output(s);
+        const int kind = sweep_kind(s, phase, n_full);
+        const bool output = kind == kOutput, smp = kind <= kSampleNewton;
+        const bool find_max = kind == kSampleMax || kind == kFullMax;
+        const int nt = smp ? stiles : tiles;
+        const int lim_c = smp ? glim : lim;            // in the column space of this sweep
+        const float slope_c = smp ? slope * (float)kTileSampleStride : slope;
+        if (kind == kFullNewton && n_full == 1 && stiles > 0) done = !valid;   // the full-row iteration starts here
+        n_smp += smp ? 1 : 0;
         // the vote slot two sweeps ahead is free again: nobody reads it before the next vote
         if (warp == 2 && lane == 0) sts_u32(done_word + 4 * ((s + 1) % 3), 1u);
         float s0 = 0.f, s1 = 0.f;
         int n_supp = 0;   // output sweep: keys of this thread's columns with p > 0
-        for (int t = 0; t < tiles && alive; ++t) {
+        for (int t = 0; t < nt && alive; ++t) {
           alive = __all_sync(0xffffffffu, mbar_wait(s_full + 8 * sbuf, sphase[sbuf], abort_flag));
           if (!alive) break;
           sphase[sbuf] ^= 1u;
@@ -327,28 +388,65 @@ __global__ void __launch_bounds__(kThreadsT, 1) tile_fwd_kernel(const __grid_con
             tmem_ld_wait();
             const int col0 = t * TN + c * 32;
             if (slope != 0.f) {
+              // bias m_h (key - i) in accumulator units; a sampled column stands for key kTileSampleStride * column
 #pragma unroll
-              for (int u = 0; u < 32; ++u) va[u] = fmaf(slope, (float)(col0 + u - i), va[u]);
+              for (int u = 0; u < 32; ++u) va[u] = fmaf(slope_c, (float)(col0 + u), va[u]) - slope * (float)i;
             }
             // columns past the row's last visible key only occur in the tiles at the causal diagonal / the tail
-            const bool edge = col0 + 31 > lim;
-            if (s == 0) {
+            const bool edge = col0 + 31 > lim_c;
+            if (find_max) {
               // y_max over the visible keys
               float m[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
 #pragma unroll
               for (int u = 0; u < 32; ++u) {
                 const float yv = ra * va[u];
-                m[u & 3] = fmaxf(m[u & 3], (!edge || col0 + u <= lim) ? yv : -INFINITY);
+                m[u & 3] = fmaxf(m[u & 3], (!edge || col0 + u <= lim_c) ? yv : -INFINITY);
               }
               ymax = fmaxf(ymax, fmaxf(fmaxf(m[0], m[1]), fmaxf(m[2], m[3])));
             } else if (!output) {
+              if (EC != kExpoGeneral && !edge) {
+                // the bulk of a Newton sweep: two columns per instruction (packed fp32 pairs) for y = a acc - tau,
+                // its powers and the two running sums; the clamp at zero has no packed form.  Four lanes of
+                // partial sums per total (two packed accumulators), as below.
+                const f32x2 ra2 = pack2(ra, ra), nt2 = pack2(-tau, -tau);
+                f32x2 q0[2] = {0ull, 0ull}, q1[2] = {0ull, 0ull};
+#pragma unroll
+                for (int u = 0; u < 32; u += 2) {
+                  float ya, yb;
+                  unpack2(fma2(ra2, pack2(va[u], va[u + 1]), nt2), ya, yb);
+                  ya = fmaxf(ya, 0.f);
+                  yb = fmaxf(yb, 0.f);
+                  const f32x2 y2 = pack2(ya, yb);
+                  f32x2 ye2, ye12;
+                  if constexpr (EC == kExpo2) {
+                    ye12 = y2;
+                    ye2 = mul2(y2, y2);
+                  } else if constexpr (EC == kExpo4) {
+                    const f32x2 t2 = mul2(y2, y2);
+                    ye12 = mul2(t2, y2);
+                    ye2 = mul2(t2, t2);
+                  } else {
+                    ye2 = y2;
+                    ye12 = pack2(ya > 0.f ? 1.0f : 0.f, yb > 0.f ? 1.0f : 0.f);
+                  }
+                  q0[(u >> 1) & 1] = add2(q0[(u >> 1) & 1], ye2);
+                  q1[(u >> 1) & 1] = add2(q1[(u >> 1) & 1], ye12);
+                }
+                float x0, x1, x2, x3;
+                unpack2(q0[0], x0, x1);
+                unpack2(q0[1], x2, x3);
+                s0 += (x0 + x1) + (x2 + x3);
+                unpack2(q1[0], x0, x1);
+                unpack2(q1[1], x2, x3);
+                s1 += (x0 + x1) + (x2 + x3);
+              } else {
               // four independent partial sums each: one thread owns the row, so the additions would
               // otherwise form two serial chains of 128 dependent operations per tile
               float p0[4] = {0.f, 0.f, 0.f, 0.f}, p1[4] = {0.f, 0.f, 0.f, 0.f};
 #pragma unroll
               for (int u = 0; u < 32; ++u) {
                 const float yr = fmaf(ra, va[u], -tau);
-                const bool ok = yr > 0.f && (!edge || col0 + u <= lim);
+                const bool ok = yr > 0.f && (!edge || col0 + u <= lim_c);
                 float ye, ye1;
                 pow_pair_c<EC>(ok ? yr : 0.f, ok, a.expo, ye, ye1);
                 p0[u & 3] += ye;
@@ -356,6 +454,7 @@ __global__ void __launch_bounds__(kThreadsT, 1) tile_fwd_kernel(const __grid_con
               }
               s0 += (p0[0] + p0[1]) + (p0[2] + p0[3]);
               s1 += (p1[0] + p1[1]) + (p1[2] + p1[3]);
+              }
             } else {
               // P -> bf16 -> shared memory, K-major with 128-byte swizzle: row r, 16-byte unit u of the
               // 64-key block sits at r*128 + ((u ^ (r & 7)) * 16)
@@ -428,8 +527,9 @@ __global__ void __launch_bounds__(kThreadsT, 1) tile_fwd_kernel(const __grid_con
           if (write && half == 0) a.tau[grow] = tau;
           if (write) a.dense_cnt[grow * 2 + half] = n_supp;
           if (a.status && threadIdx.x == 64) {
-            // diagnostics: sweeps spent (y_max sweep + Newton sweeps + output sweep) and tiles processed
-            atomicAdd(a.status + ENTMAX_ATTN_STATUS_TILE_SWEEPS, s + 1);
+            // diagnostics: full-length sweeps spent (y_max sweep if any, Newton sweeps, output sweep; the sampled
+            // sweeps, an eighth as long, are not counted) and tiles processed
+            atomicAdd(a.status + ENTMAX_ATTN_STATUS_TILE_SWEEPS, s + 1 - n_smp);
             atomicAdd(a.status + ENTMAX_ATTN_STATUS_TILES, 1);
           }
           tc_fence_before();
@@ -443,7 +543,7 @@ __global__ void __launch_bounds__(kThreadsT, 1) tile_fwd_kernel(const __grid_con
         {
           const uint32_t mine = xchg + (uint32_t)(half * TM + row_local) * 8u;
           const uint32_t theirs = xchg + (uint32_t)((half ^ 1) * TM + row_local) * 8u;
-          sts_u32(mine, __float_as_uint(s == 0 ? ymax : s0));
+          sts_u32(mine, __float_as_uint(find_max ? ymax : s0));
           sts_u32(mine + 4, __float_as_uint(s1));
           __syncwarp();
           if (lane == 0) mbar_arrive(x_bar);
@@ -451,14 +551,14 @@ __global__ void __launch_bounds__(kThreadsT, 1) tile_fwd_kernel(const __grid_con
           xphase ^= 1u;
           if (!alive) break;
           const float o0 = __uint_as_float(lds_u32(theirs)), o1 = __uint_as_float(lds_u32(theirs + 4));
-          if (s == 0) {
+          if (find_max) {
             ymax = fmaxf(ymax, o0);
           } else {
             s0 = half == 0 ? s0 + o0 : o0 + s0;
             s1 = half == 0 ? s1 + o1 : o1 + s1;
           }
         }
-        if (s == 0) {
+        if (find_max) {
           it_tau = tau_iter_start(ymax);
           tau = it_tau.tau;
         } else if (!done) {
@@ -468,7 +568,7 @@ __global__ void __launch_bounds__(kThreadsT, 1) tile_fwd_kernel(const __grid_con
         }
         const bool warp_done = __all_sync(0xffffffffu, done);
         if (lane == 0) {
-          if (!warp_done || s == 0) atomicAnd(reinterpret_cast<unsigned*>(__cvta_shared_to_generic(done_word + 4 * (s % 3))), 0u);
+          if (!warp_done || find_max) atomicAnd(reinterpret_cast<unsigned*>(__cvta_shared_to_generic(done_word + 4 * (s % 3))), 0u);
           mbar_arrive(ctl);
         }
       }
@@ -500,6 +600,11 @@ cudaError_t launch_tile_impl(const Problem& p, const void* q, const void* k, con
   if (err != cudaSuccess) return err;
   err = make_tile_map(&map_v, v, p.D, p.N, p.H, p.B, p.sn, p.sh, p.sb);
   if (err != cudaSuccess) return err;
+  CUtensorMap map_ks = map_k;   // short sequences never take the sampled start
+  if (p.N >= kSampleMinTiles * TN) {
+    err = make_sampled_tile_map(&map_ks, k, p.D, p.N, p.H, p.B, p.sn, p.sh, p.sb, kTileSampleStride);
+    if (err != cudaSuccess) return err;
+  }
   err = cudaFuncSetAttribute(tile_fwd_kernel<HD, EC>, cudaFuncAttributeMaxDynamicSharedMemorySize, TCfg<HD>::kSmemBytes);
   if (err != cudaSuccess) return err;
   int dev = 0, sms = 0;
@@ -509,7 +614,7 @@ cudaError_t launch_tile_impl(const Problem& p, const void* q, const void* k, con
   if (err != cudaSuccess) return err;
   const long all_tiles = (long)p.B * p.H * args.tiles_per_head;
   const int grid = (int)(all_tiles < sms ? all_tiles : sms);
-  tile_fwd_kernel<HD, EC><<<grid, kThreadsT, TCfg<HD>::kSmemBytes, stream>>>(map_q, map_k, map_v, args);
+  tile_fwd_kernel<HD, EC><<<grid, kThreadsT, TCfg<HD>::kSmemBytes, stream>>>(map_q, map_k, map_v, map_ks, args);
   return cudaGetLastError();
 }
 
@@ -550,6 +655,22 @@ cudaError_t make_tile_map(CUtensorMap* map, const void* base, int D, int N, int 
   cuuint32_t box[4] = {64, (cuuint32_t)box_rows, 1, 1};
   cuuint32_t estr[4] = {1, 1, 1, 1};
   CUresult r = fn(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, const_cast<void*>(base), dims, strides, box, estr,
+                  CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                  CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  return r == CUDA_SUCCESS ? cudaSuccess : cudaErrorInvalidValue;
+}
+
+cudaError_t make_sampled_tile_map(CUtensorMap* map, const void* base, int D, int N, int H, int B, int64_t sn, int64_t sh,
+                                  int64_t sb, int stride, int box_rows) {
+  EncodeTiledFn fn;
+  cudaError_t err = encode_fn(&fn);
+  if (err != cudaSuccess) return err;
+  const cuuint64_t groups = (cuuint64_t)(N / stride);
+  cuuint64_t dims[5] = {(cuuint64_t)D, (cuuint64_t)stride, groups > 0 ? groups : 1, (cuuint64_t)H, (cuuint64_t)B};
+  cuuint64_t strides[4] = {(cuuint64_t)sn * 2, (cuuint64_t)sn * 2 * stride, (cuuint64_t)sh * 2, (cuuint64_t)sb * 2};
+  cuuint32_t box[5] = {64, 1, (cuuint32_t)box_rows, 1, 1};
+  cuuint32_t estr[5] = {1, 1, 1, 1, 1};
+  CUresult r = fn(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 5, const_cast<void*>(base), dims, strides, box, estr,
                   CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
                   CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
   return r == CUDA_SUCCESS ? cudaSuccess : cudaErrorInvalidValue;
