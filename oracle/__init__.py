@@ -58,6 +58,11 @@ def _load():
             lib.oracle_attn_bwd_rows.argtypes = [fp, fp, fp, fp] + common + [ip, ctypes.c_long, dp, dp]
             lib.oracle_attn_bwd_scale_head.restype = ctypes.c_int
             lib.oracle_attn_bwd_scale_head.argtypes = [fp, fp, fp, fp] + common + [dp, dp]
+            proj = [ctypes.c_long] * 4 + [ctypes.c_double, ctypes.c_int, ctypes.c_int]
+            lib.oracle_scale_projection.restype = ctypes.c_int
+            lib.oracle_scale_projection.argtypes = [dp, dp, dp, dp] + proj + [dp, dp, dp]
+            lib.oracle_scale_projection_bwd.restype = ctypes.c_int
+            lib.oracle_scale_projection_bwd.argtypes = [dp, dp, dp, dp] + proj + [dp, dp, dp, dp]
             lib.oracle_num_threads.restype = ctypes.c_int
             lib.oracle_set_num_threads.argtypes = [ctypes.c_int]
             _lib = lib
@@ -183,3 +188,35 @@ def attn_bwd_scale_head(q, k, v, d_o, alpha, sm_scale, causal, scale=None, n_mod
     if rc != 0:
         raise RuntimeError("oracle_attn_bwd_scale_head failed: %d" % rc)
     return dc, (float(grads[0]), float(grads[1]), float(grads[2]))
+
+
+def _f64(a):
+    return np.ascontiguousarray(np.asarray(a, dtype=np.float64))
+
+
+def scale_projection(x, w_beta, w_gamma, delta, s, causal, n_mode=0):
+    """ASEntmax's content-dependent scale (Sec. 4.1) from the layer input x [B, N, dm] and per-head weights [H, dm].
+    Returns (c, beta, gamma), each float64 [B, H, N]."""
+    x, w_beta, w_gamma, delta = _f64(x), _f64(w_beta), _f64(w_gamma), _f64(delta)
+    B, N, dm = x.shape
+    H = w_beta.shape[0]
+    c, beta, gamma = (np.empty((B, H, N), dtype=np.float64) for _ in range(3))
+    rc = _load().oracle_scale_projection(_dptr(x), _dptr(w_beta), _dptr(w_gamma), _dptr(delta), B, H, N, dm, float(s),
+                                         int(bool(causal)), int(n_mode), _dptr(c), _dptr(beta), _dptr(gamma))
+    if rc != 0:
+        raise RuntimeError("oracle_scale_projection failed: %d" % rc)
+    return c, beta, gamma
+
+
+def scale_projection_bwd(x, w_beta, w_gamma, dc, s, causal, n_mode=0):
+    """Chain rule of scale_projection. Returns (dw_beta [H, dm], dw_gamma [H, dm], ddelta [H], dx [B, N, dm])."""
+    x, w_beta, w_gamma, dc = _f64(x), _f64(w_beta), _f64(w_gamma), _f64(dc)
+    B, N, dm = x.shape
+    H = w_beta.shape[0]
+    dwb, dwg = np.empty((H, dm), dtype=np.float64), np.empty((H, dm), dtype=np.float64)
+    dd, dx = np.empty(H, dtype=np.float64), np.empty((B, N, dm), dtype=np.float64)
+    rc = _load().oracle_scale_projection_bwd(_dptr(x), _dptr(w_beta), _dptr(w_gamma), _dptr(dc), B, H, N, dm, float(s),
+                                             int(bool(causal)), int(n_mode), _dptr(dwb), _dptr(dwg), _dptr(dd), _dptr(dx))
+    if rc != 0:
+        raise RuntimeError("oracle_scale_projection_bwd failed: %d" % rc)
+    return dwb, dwg, dd, dx

@@ -18,6 +18,9 @@
  *                              dp_j/ds_k = u_j (delta_jk - u_k / sum u), u = p^(2-alpha).
  *   oracle_attn_bwd_scale_head chain rule through Eq. "asentmax": gradients of the per-row scale c_i and of
  *                              the head's beta, gamma, delta.
+ *   oracle_scale_projection(_bwd)  Sec. 4.1: the content-dependent scale, beta = softplus(X w_beta),
+ *                              gamma = s tanh(X w_gamma) per query and head, c = delta + beta (log n)^gamma, and the
+ *                              chain rule back to w_beta, w_gamma, delta and X.
  *
  * Pins (tests that do not use this file's own arithmetic): the paper's worked sparsemax example,
  * the two-level closed form of Lemma 2, brute-force enumeration of supports for n <= 8, the
@@ -456,6 +459,71 @@ int oracle_attn_bwd_scale_head(const float* q, const float* k, const float* v, c
     }
   }
   grads_out[0] = gb; grads_out[1] = gg; grads_out[2] = gd;
+  return 0;
+}
+
+/* Sec. 4.1: ASEntmax's scale from the layer input.  For token i of batch element b and head h
+ *   beta = softplus(<x_bi, w_beta_h>),  gamma = s tanh(<x_bi, w_gamma_h>),  c = delta_h + beta (log n_i)^gamma
+ * (c = delta_h when n_i = 1), n_i = i + 1 under the causal mask, N otherwise or with n_mode = 1.
+ *   x [B,N,dm], w_beta, w_gamma [H,dm], delta [H]; outputs c, beta_out, gamma_out [B,H,N] (the last two may be NULL). */
+int oracle_scale_projection(const double* x, const double* w_beta, const double* w_gamma, const double* delta,
+                            long B, long H, long N, long dm, double s, int causal, int n_mode,
+                            double* c, double* beta_out, double* gamma_out) {
+  if (B <= 0 || H <= 0 || N <= 0 || dm <= 0) return -1;
+  for (long b = 0; b < B; ++b)
+    for (long h = 0; h < H; ++h)
+      for (long i = 0; i < N; ++i) {
+        const double* xi = x + ((size_t)b * N + i) * dm;
+        double pb = 0.0, pg = 0.0;
+        for (long t = 0; t < dm; ++t) { pb += xi[t] * w_beta[h * dm + t]; pg += xi[t] * w_gamma[h * dm + t]; }
+        double beta = pb > 0.0 ? pb + log1p(exp(-pb)) : log1p(exp(pb));   /* softplus, written for both signs */
+        double gamma = s * tanh(pg);
+        long n_i = (n_mode || !causal) ? N : i + 1;
+        size_t at = ((size_t)b * H + h) * N + i;
+        c[at] = oracle_asentmax_scale(beta, gamma, delta[h], n_i);
+        if (beta_out) beta_out[at] = beta;
+        if (gamma_out) gamma_out[at] = gamma;
+      }
+  return 0;
+}
+
+/* Chain rule of the above: given dc = dL/dc [B,H,N],
+ *   dL/ddelta_h = sum dc;  with L = log n_i (rows with n_i > 1 only):
+ *   dL/dbeta = dc L^gamma,  dL/dgamma = dc beta L^gamma log L,
+ *   d beta / d pre_beta = sigmoid(pre_beta),  d gamma / d pre_gamma = s (1 - tanh^2(pre_gamma)),
+ *   dL/dw_beta_h = sum_{b,i} g_beta x_bi,  dL/dw_gamma_h likewise,  dL/dx_bi = sum_h (g_beta w_beta_h + g_gamma w_gamma_h).
+ * Outputs dw_beta, dw_gamma [H,dm], ddelta [H], dx [B,N,dm] (overwritten). */
+int oracle_scale_projection_bwd(const double* x, const double* w_beta, const double* w_gamma, const double* dc,
+                                long B, long H, long N, long dm, double s, int causal, int n_mode,
+                                double* dw_beta, double* dw_gamma, double* ddelta, double* dx) {
+  if (B <= 0 || H <= 0 || N <= 0 || dm <= 0) return -1;
+  memset(dw_beta, 0, sizeof(double) * (size_t)H * dm);
+  memset(dw_gamma, 0, sizeof(double) * (size_t)H * dm);
+  memset(ddelta, 0, sizeof(double) * (size_t)H);
+  memset(dx, 0, sizeof(double) * (size_t)B * N * dm);
+  for (long b = 0; b < B; ++b)
+    for (long h = 0; h < H; ++h)
+      for (long i = 0; i < N; ++i) {
+        const double* xi = x + ((size_t)b * N + i) * dm;
+        double* dxi = dx + ((size_t)b * N + i) * dm;
+        double pb = 0.0, pg = 0.0;
+        for (long t = 0; t < dm; ++t) { pb += xi[t] * w_beta[h * dm + t]; pg += xi[t] * w_gamma[h * dm + t]; }
+        double g = dc[((size_t)b * H + h) * N + i];
+        ddelta[h] += g;
+        long n_i = (n_mode || !causal) ? N : i + 1;
+        if (n_i <= 1) continue;
+        double beta = pb > 0.0 ? pb + log1p(exp(-pb)) : log1p(exp(pb));
+        double th = tanh(pg);
+        double gamma = s * th;
+        double L = log((double)n_i), Lg = pow(L, gamma);
+        double gb = g * Lg * (1.0 / (1.0 + exp(-pb)));
+        double gg = g * beta * Lg * log(L) * s * (1.0 - th * th);
+        for (long t = 0; t < dm; ++t) {
+          dw_beta[h * dm + t] += gb * xi[t];
+          dw_gamma[h * dm + t] += gg * xi[t];
+          dxi[t] += gb * w_beta[h * dm + t] + gg * w_gamma[h * dm + t];
+        }
+      }
   return 0;
 }
 

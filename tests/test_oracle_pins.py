@@ -573,5 +573,61 @@ def test_alibi_noncausal_backward_matches_finite_differences():
             assert abs(fd - g0) < 5e-4 * max(1.0, abs(g0)), (which, i, t, fd, g0)
 
 
+# ---------------------------------------------------------------- content-dependent scale (Sec. 4.1)
+def test_scale_projection_values_and_limits():
+    rng = np.random.default_rng(41)
+    B, H, N, dm, s = 2, 3, 9, 5, 2.0
+    x = rng.normal(size=(B, N, dm))
+    wb, wg = rng.normal(size=(H, dm)) * 0.5, rng.normal(size=(H, dm)) * 0.5
+    delta = np.array([1.0, 0.5, 1.5])
+    c, beta, gamma = oracle.scale_projection(x, wb, wg, delta, s, True)
+    # written out with numpy: softplus and tanh of the projections, then Eq. "asentmax" through its own function
+    pb = np.einsum("bnd,hd->bhn", x, wb)
+    pg = np.einsum("bnd,hd->bhn", x, wg)
+    np.testing.assert_allclose(beta, np.logaddexp(0.0, pb), rtol=1e-13)
+    np.testing.assert_allclose(gamma, s * np.tanh(pg), rtol=1e-13)
+    assert np.all(beta > 0) and np.all(np.abs(gamma) < s)          # beta > 0, gamma in (-s, s) as the paper states
+    for b, h, i in [(0, 0, 0), (1, 2, 4), (0, 1, 8)]:
+        assert abs(c[b, h, i] - oracle.asentmax_scale(beta[b, h, i], gamma[b, h, i], delta[h], i + 1)) < 1e-14
+    assert np.all(c[:, :, 0] == delta[None, :])                    # one visible key: c = delta
+    # zero weights: beta = log 2, gamma = 0, so c = delta + log 2 for every row that sees more than one key
+    c0, _, _ = oracle.scale_projection(x, np.zeros_like(wb), np.zeros_like(wg), delta, s, True)
+    np.testing.assert_allclose(c0[:, :, 1:], (delta + math.log(2.0))[None, :, None] * np.ones((B, H, N - 1)), rtol=1e-14)
+    # the non-causal problem and n_mode = 1 use the total length for every row
+    cn, bn, gn = oracle.scale_projection(x, wb, wg, delta, s, False)
+    cm, _, _ = oracle.scale_projection(x, wb, wg, delta, s, True, n_mode=1)
+    np.testing.assert_allclose(cn, cm, rtol=0, atol=0)
+    np.testing.assert_allclose(cn, delta[None, :, None] + bn * math.log(N) ** gn, rtol=1e-13)
+    # very negative / positive projections: softplus stays finite and positive
+    big = np.full((1, 3, dm), 40.0)
+    cb, bb, _ = oracle.scale_projection(big, np.ones((1, dm)), np.zeros((1, dm)), np.array([0.0]), s, False)
+    assert np.all(np.isfinite(bb)) and abs(bb[0, 0, 0] - 200.0) < 1e-9
+    _, bs, _ = oracle.scale_projection(-big, np.ones((1, dm)), np.zeros((1, dm)), np.array([0.0]), s, False)
+    assert np.all(bs > 0) and bs[0, 0, 0] < 1e-80
+
+
+def test_scale_projection_backward_matches_finite_differences():
+    rng = np.random.default_rng(43)
+    B, H, N, dm, s = 2, 2, 6, 4, 1.5
+    x = rng.normal(size=(B, N, dm))
+    wb, wg = rng.normal(size=(H, dm)) * 0.7, rng.normal(size=(H, dm)) * 0.7
+    delta = np.array([1.0, 0.6])
+    dc = rng.normal(size=(B, H, N))
+    for causal in (True, False):
+        loss = lambda x_, wb_, wg_, dl_: float(np.sum(oracle.scale_projection(x_, wb_, wg_, dl_, s, causal)[0] * dc))
+        dwb, dwg, dd, dx = oracle.scale_projection_bwd(x, wb, wg, dc, s, causal)
+        e = 1e-6
+        for arr, grad, which in ((wb, dwb, 1), (wg, dwg, 2), (delta, dd, 3), (x, dx, 0)):
+            for _ in range(6):
+                idx = tuple(int(rng.integers(n)) for n in arr.shape)
+                args = [x.copy(), wb.copy(), wg.copy(), delta.copy()]
+                up = [a.copy() for a in args]
+                dn = [a.copy() for a in args]
+                up[which][idx] += e
+                dn[which][idx] -= e
+                fd = (loss(*up) - loss(*dn)) / (2 * e)
+                assert abs(fd - grad[idx]) <= 1e-6 * max(1.0, abs(fd)), (which, idx, fd, grad[idx])
+
+
 def test_threads_reported():
     assert oracle.num_threads() >= 1
