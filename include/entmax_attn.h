@@ -162,6 +162,32 @@ int entmax_attn_bwd_rowscale(const entmax_attn_params* params, const void* q, co
                              float* d_scale_rows, void* workspace, size_t workspace_bytes, int32_t* device_status,
                              void* cuda_stream);
 
+/* The content-dependent scale itself (Sec. 4.1): for query token i of batch element b and head h
+ *   beta = softplus(<x_bi, w_beta_h>),  gamma = gamma_range * tanh(<x_bi, w_gamma_h>),
+ *   c = delta_h + beta (log n_i)^gamma        (Eq. "asentmax"; c = delta_h when n_i = 1),
+ * n_i = i + 1 when causal and n_mode = 0, seq otherwise.  The forward call writes the table that
+ * entmax_attn_fwd_rowscale / entmax_attn_bwd_rowscale take; the backward call takes the d_scale_rows those return and
+ * applies the chain rule: dL/dw_beta, dL/dw_gamma [heads, d_model], dL/ddelta [heads] and dL/dx (the part of it that
+ * flows through the scale; the caller adds it to the gradient x gets from its other uses).
+ *   x            in,  device [batch, seq, d_model] contiguous, x_dtype (ENTMAX_ATTN_DTYPE_*)
+ *   w_beta, w_gamma   in, device float32 [heads, d_model]; delta in, device float32 [heads]
+ *   c_rows       out, device float32 [batch, heads, seq]
+ *   d_scale_rows in,  device float32 [batch, heads, seq]
+ *   dw_beta, dw_gamma out, device float32 [heads, d_model] (overwritten); ddelta out, float32 [heads] or NULL;
+ *   dx           out, device [batch, seq, d_model] in x_dtype (overwritten) or NULL
+ * heads <= 64.  Errors as for the other entry points (gamma_range must be positive and finite: EINVAL_ALPHA). */
+typedef struct {
+  int32_t batch, heads, seq, d_model;
+  int32_t x_dtype;
+  int32_t causal, n_mode;
+  float gamma_range;
+} entmax_attn_proj_params;
+int entmax_attn_scale_proj_fwd(const entmax_attn_proj_params* params, const void* x, const float* w_beta,
+                               const float* w_gamma, const float* delta, float* c_rows, void* cuda_stream);
+int entmax_attn_scale_proj_bwd(const entmax_attn_proj_params* params, const void* x, const float* w_beta,
+                               const float* w_gamma, const float* d_scale_rows, float* dw_beta, float* dw_gamma,
+                               float* ddelta, void* dx, void* cuda_stream);
+
 /* Extended forward / backward: every optional input and output of the calls above in one struct, plus the
  * ALiBi positional term of the paper's NAPE scheme (App. B: half of the heads add m_h (j - i) to the
  * logits z_ij = <q_i,k_j> sm_scale, j <= i; the other half use slope 0).  The ASEntmax scale multiplies

@@ -36,6 +36,12 @@ class DecodeParams(ctypes.Structure):
                 ("kv_stride_n", ctypes.c_int64)]
 
 
+class ProjParams(ctypes.Structure):
+    _fields_ = [("batch", ctypes.c_int32), ("heads", ctypes.c_int32), ("seq", ctypes.c_int32), ("d_model", ctypes.c_int32),
+                ("x_dtype", ctypes.c_int32), ("causal", ctypes.c_int32), ("n_mode", ctypes.c_int32),
+                ("gamma_range", ctypes.c_float)]
+
+
 class WsLayout(ctypes.Structure):
     _fields_ = [("row_count_offset", ctypes.c_size_t), ("entries_offset", ctypes.c_size_t),
                 ("scale_offset", ctypes.c_size_t), ("dense_count_offset", ctypes.c_size_t),
@@ -101,6 +107,11 @@ def load():
         lib.entmax_attn_scores_debug.argtypes = [pp, vp, vp, ctypes.c_int32, fp, vp, ctypes.c_size_t, ip, vp]
         lib.entmax_attn_profile_events.restype = ctypes.c_int
         lib.entmax_attn_profile_events.argtypes = [ctypes.c_int, vp, vp]
+        jp = ctypes.POINTER(ProjParams)
+        lib.entmax_attn_scale_proj_fwd.restype = ctypes.c_int
+        lib.entmax_attn_scale_proj_fwd.argtypes = [jp, vp, fp, fp, fp, fp, vp]
+        lib.entmax_attn_scale_proj_bwd.restype = ctypes.c_int
+        lib.entmax_attn_scale_proj_bwd.argtypes = [jp, vp, fp, fp, fp, fp, fp, fp, vp, vp]
         lib.entmax_attn_selftest_wait_expiry.restype = ctypes.c_int
         lib.entmax_attn_selftest_wait_expiry.argtypes = [ctypes.c_uint64, ip, vp]
         lib.entmax_attn_strerror.restype = ctypes.c_char_p
@@ -447,3 +458,41 @@ def entmax_attn_selftest_wait_expiry(limit_ns: int, status: torch.Tensor, stream
     FLAG_WAIT_EXPIRED in status[0] and the microseconds it waited in status[1]."""
     _check(load().entmax_attn_selftest_wait_expiry(int(limit_ns), _ptr(status), _stream_ptr(stream)),
            "entmax_attn_selftest_wait_expiry")
+
+
+def _proj_params(x, heads, causal, n_mode, gamma_range):
+    if x.dim() != 3 or not x.is_contiguous():
+        raise EntmaxAttnError("x must be a contiguous [batch, seq, d_model] tensor")
+    if x.dtype == torch.bfloat16:
+        dt = DTYPE_BF16
+    elif x.dtype == torch.float32:
+        dt = DTYPE_FP32
+    else:
+        raise EntmaxAttnError("x must be bfloat16 or float32")
+    B, N, dm = x.shape
+    return ProjParams(B, int(heads), N, dm, dt, int(bool(causal)), int(n_mode), float(gamma_range))
+
+
+def entmax_attn_scale_proj_fwd(x, w_beta, w_gamma, delta, gamma_range, causal, *, n_mode=0, c_rows=None, stream=None):
+    """c_rows [B, H, N] (float32) from the layer input x [B, N, d_model] and per-head weights [H, d_model]."""
+    H = w_beta.shape[0]
+    params = _proj_params(x, H, causal, n_mode, gamma_range)
+    if c_rows is None:
+        c_rows = torch.empty((x.shape[0], H, x.shape[1]), dtype=torch.float32, device=x.device)
+    _check(load().entmax_attn_scale_proj_fwd(ctypes.byref(params), _ptr(x), _ptr(w_beta), _ptr(w_gamma), _ptr(delta),
+                                             _ptr(c_rows), _stream_ptr(stream)), "entmax_attn_scale_proj_fwd")
+    return c_rows
+
+
+def entmax_attn_scale_proj_bwd(x, w_beta, w_gamma, d_scale_rows, gamma_range, causal, *, n_mode=0, want_dx=True,
+                               stream=None):
+    """Chain rule of the projection.  Returns (dw_beta, dw_gamma, ddelta, dx or None)."""
+    H = w_beta.shape[0]
+    params = _proj_params(x, H, causal, n_mode, gamma_range)
+    dwb, dwg = torch.empty_like(w_beta), torch.empty_like(w_gamma)
+    dd = torch.empty((H,), dtype=torch.float32, device=x.device)
+    dx = torch.empty_like(x) if want_dx else None
+    _check(load().entmax_attn_scale_proj_bwd(ctypes.byref(params), _ptr(x), _ptr(w_beta), _ptr(w_gamma), _ptr(d_scale_rows),
+                                             _ptr(dwb), _ptr(dwg), _ptr(dd), _ptr(dx), _stream_ptr(stream)),
+           "entmax_attn_scale_proj_bwd")
+    return dwb, dwg, dd, dx

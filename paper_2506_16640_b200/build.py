@@ -13,7 +13,7 @@ _ROOT = os.path.dirname(_HERE)
 CSRC = os.path.join(_HERE, "csrc")
 INCLUDE = os.path.join(_ROOT, "include")
 LIB = os.path.join(_HERE, "libentmax_attn.so")
-SOURCES = ["entmax_attn_api.cu", "dense_rows.cu", "row_lists.cu", "sweep_sm100.cu", "tile_fwd_sm100.cu", "tile_bwd_sm100.cu", "decode.cu", "decode_scores_sm100.cu", "no_alloc.cu", "selftest.cu"]
+SOURCES = ["entmax_attn_api.cu", "dense_rows.cu", "row_lists.cu", "sweep_sm100.cu", "tile_fwd_sm100.cu", "tile_bwd_sm100.cu", "decode.cu", "decode_scores_sm100.cu", "no_alloc.cu", "selftest.cu", "scale_proj.cu"]
 
 
 def _nvcc() -> str:

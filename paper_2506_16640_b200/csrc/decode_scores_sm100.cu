@@ -68,7 +68,9 @@ __global__ void __launch_bounds__(kThreadsD, 2) decode_scores_tc_kernel(const __
   const uint32_t s_empty = s_full + 16;                     // [2]
   const uint32_t tmem_slot = s_empty + 16;
   const uint32_t abort_flag = tmem_slot + 4;
-  static_assert(8 * (1 + 2 * kStagesD + 4) + 8 <= C::kBarBytes, "barrier area");
+  const uint32_t drain_bar = tmem_slot + 8;       // teardown: every MMA issued so far has finished
+  const uint32_t drain_fail = drain_bar + 8;      // uint32: a teardown wait ran out as well
+  static_assert(8 * (1 + 2 * kStagesD + 4) + 8 + 16 <= C::kBarBytes, "barrier area");
 
   const int warp = threadIdx.x >> 5;
   const int lane = threadIdx.x & 31;
@@ -82,6 +84,8 @@ __global__ void __launch_bounds__(kThreadsD, 2) decode_scores_tc_kernel(const __
       mbar_init(s_full + 8 * s, 1);
       mbar_init(s_empty + 8 * s, 4);
     }
+    mbar_init(drain_bar, 1);
+    sts_u32(drain_fail, 0u);
     sts_u32(abort_flag, 0u);
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
@@ -102,13 +106,22 @@ __global__ void __launch_bounds__(kThreadsD, 2) decode_scores_tc_kernel(const __
       for (int hf = 0; hf < C::kHalves; ++hf) tma_load_4d(q_smem + hf * (kQPad * 128), &map_q, q_full, hf * 64, 0, h, b);
       int stage = 0;
       uint32_t phase = 0;
+      bool alive = true;
       for (int t = 0; t < tiles; ++t) {
-        if (!mbar_wait(kv_empty + 8 * stage, phase ^ 1u, abort_flag)) break;
+        alive = mbar_wait(kv_empty + 8 * stage, phase ^ 1u, abort_flag);
+        if (!alive) break;
         mbar_expect_tx(kv_full + 8 * stage, C::kKBytes);
         for (int hf = 0; hf < C::kHalves; ++hf)
           tma_load_4d(k_smem + stage * C::kKBytes + hf * (kTile * 128), &map_k, kv_full + 8 * stage, hf * 64,
                       key0 + t * kTile, h, b);
         if (++stage == kStagesD) { stage = 0; phase ^= 1u; }
+      }
+      if (!alive) {
+        // a wait ran out somewhere in the CTA: the copies this thread armed barriers for must land before shared
+        // memory goes away (stages before `stage`: this round of the ring; the others: the previous round)
+        bool ok = mbar_drain(q_full, 0u);
+        for (int st = 0; st < kStagesD; ++st) ok &= mbar_drain(kv_full + 8 * st, st < stage ? phase : phase ^ 1u);
+        if (!ok) sts_u32(drain_fail, 1u);
       }
     }
   } else if (warp == 1) {
@@ -136,6 +149,11 @@ __global__ void __launch_bounds__(kThreadsD, 2) decode_scores_tc_kernel(const __
         umma_commit(kv_empty + 8 * stage);
         buf ^= 1;
         if (++stage == kStagesD) { stage = 0; phase ^= 1u; }
+      }
+      if (!alive) {
+        // the tensor core must be done with shared memory and TMEM before they are released
+        umma_commit(drain_bar);
+        if (!mbar_drain(drain_bar, 0u)) sts_u32(drain_fail, 1u);
       }
     }
   } else {
@@ -213,8 +231,12 @@ __global__ void __launch_bounds__(kThreadsD, 2) decode_scores_tc_kernel(const __
   __syncthreads();
   if (lds_u32(abort_flag)) {
     if (threadIdx.x == 0 && status) atomicOr(status + ENTMAX_ATTN_STATUS_FLAGS, ENTMAX_ATTN_FLAG_WAIT_EXPIRED);
-    const uint64_t t0 = global_ns();
-    while (global_ns() - t0 < 200000ull) { }
+    // the producer and the MMA issuer have waited for their copies and MMAs in flight; only if one of those waits ran
+    // out as well is there nothing left but to give the hardware time
+    if (lds_u32(drain_fail)) {
+      const uint64_t t0 = global_ns();
+      while (global_ns() - t0 < 200000ull) { }
+    }
     __syncthreads();
   }
   if (warp == 1) {

@@ -76,6 +76,16 @@ static __device__ __noinline__ bool mbar_wait_slow(uint32_t bar, uint32_t parity
     }
   }
 }
+// Teardown after an expired wait: waits, with a bound of its own and without looking at the abort word, until phase
+// `parity` of `bar` has completed -- a copy this thread armed the barrier for has landed, or the tensor-core work it
+// committed to the barrier has finished -- so that shared memory and TMEM are not released under work in flight.
+__device__ __forceinline__ bool mbar_drain(uint32_t bar, uint32_t parity, uint64_t limit_ns = 1000000ull) {
+  const uint64_t t0 = global_ns();
+  while (!mbar_try_wait(bar, parity)) {
+    if (global_ns() - t0 > limit_ns) return false;
+  }
+  return true;
+}
 __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, uint32_t abort_flag) {
   if (mbar_try_wait(bar, parity)) return true;
   if (mbar_try_wait(bar, parity)) return true;

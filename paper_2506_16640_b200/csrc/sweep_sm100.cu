@@ -28,7 +28,8 @@
 // the warp saw a value above its threshold re-reads the groups that hold candidates (four groups per
 // round trip to TMEM); it hands the accumulator back as soon as the last values it needs are in registers.  While the consumers of one Q tile scan, the tensor core works on the other.
 // Every mbarrier wait is bounded: on expiry the CTA raises ENTMAX_ATTN_FLAG_WAIT_EXPIRED, all roles
-// leave their loops, in-flight copies are given time to land, TMEM is freed and the CTA returns.
+// leave their loops, the producer waits for the copies it armed barriers for and the MMA issuer for the tensor-core
+// work it issued (each with a bound of its own), TMEM is freed and the CTA returns.
 #include <cuda.h>
 
 #include "common.cuh"
@@ -272,7 +273,9 @@ __global__ void __launch_bounds__(kThreads, 1) sweep_kernel(const __grid_constan
   const uint32_t w_item = w_empty + 8 * kSchedSlots;       // int32 [kSchedSlots]
   const uint32_t tmem_slot = w_item + 4 * kSchedSlots;     // uint32
   const uint32_t abort_flag = tmem_slot + 4;               // uint32
-  static_assert((4 * kQTiles + 2 * C::kStages + 2 * kSchedSlots) * 8 + kSchedSlots * 4 + 8 <= C::kBarBytes,
+  const uint32_t drain_bar = tmem_slot + 8;                // teardown: "every MMA issued so far has finished"
+  const uint32_t drain_fail = drain_bar + 8;               // uint32: a teardown wait ran out as well
+  static_assert((4 * kQTiles + 2 * C::kStages + 2 * kSchedSlots) * 8 + kSchedSlots * 4 + 8 + 16 <= C::kBarBytes,
                 "barrier area");
 
   const int warp = threadIdx.x >> 5;
@@ -293,7 +296,9 @@ __global__ void __launch_bounds__(kThreads, 1) sweep_kernel(const __grid_constan
       mbar_init(w_full + 8 * t, 1);
       mbar_init(w_empty + 8 * t, 1 + kConsumerWarps);   // MMA issuer + one arrival per consumer warp
     }
+    mbar_init(drain_bar, 1);
     sts_u32(abort_flag, 0u);
+    sts_u32(drain_fail, 0u);
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
   }
@@ -362,6 +367,15 @@ __global__ void __launch_bounds__(kThreads, 1) sweep_kernel(const __grid_constan
           }
         }
       }
+      if (!alive) {
+        // a wait ran out somewhere in the CTA: every copy this thread armed a barrier for must have landed before
+        // shared memory goes away.  Stages before `stage` were armed in this round of the ring, the others in the
+        // previous one (a barrier that was never armed reports its "previous" phase as complete at once).
+        bool ok = true;
+        for (int st = 0; st < C::kStages; ++st) ok &= mbar_drain(k_full + 8 * st, st < stage ? kphase : kphase ^ 1u);
+        for (int x = 0; x < kQTiles; ++x) ok &= mbar_drain(q_full + 8 * x, ((qphase >> x) & 1u) ^ 1u);
+        if (!ok) sts_u32(drain_fail, 1u);
+      }
     }
   } else if (warp == 1) {
     // ------------------------------------------------------------------ MMA issuer
@@ -421,6 +435,11 @@ __global__ void __launch_bounds__(kThreads, 1) sweep_kernel(const __grid_constan
           umma_commit(k_empty + 8 * stage);
           if (++stage == C::kStages) { stage = 0; kphase ^= 1u; }
         }
+      }
+      if (!alive) {
+        // the tensor core must be done with shared memory and TMEM before they are released
+        umma_commit(drain_bar);
+        if (!mbar_drain(drain_bar, 0u)) sts_u32(drain_fail, 1u);
       }
     }
   } else {
@@ -669,9 +688,12 @@ __global__ void __launch_bounds__(kThreads, 1) sweep_kernel(const __grid_constan
   __syncthreads();
   if (lds_u32(abort_flag)) {
     if (threadIdx.x == 0 && a.status) atomicOr(a.status + ENTMAX_ATTN_STATUS_FLAGS, ENTMAX_ATTN_FLAG_WAIT_EXPIRED);
-    // give copies and MMAs that may still be in flight time to land before shared memory and TMEM go away
-    const uint64_t t0 = global_ns();
-    while (global_ns() - t0 < 200000ull) { }
+    // the producer and the MMA issuer have waited for their copies and MMAs in flight (above); only if one of those
+    // waits ran out as well is there nothing left but to give the hardware time
+    if (lds_u32(drain_fail)) {
+      const uint64_t t0 = global_ns();
+      while (global_ns() - t0 < 200000ull) { }
+    }
     __syncthreads();
   }
   if (warp == 1) {

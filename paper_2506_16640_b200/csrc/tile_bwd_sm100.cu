@@ -135,6 +135,8 @@ __global__ void __launch_bounds__(kThreadsB, 1) tile_bwd_kernel(const __grid_con
   const uint32_t dq_full = bars + 80, dq_empty = bars + 88;
   const uint32_t tmem_slot = bars + 96;
   const uint32_t abort_flag = bars + 100;
+  const uint32_t drain_bar = bars + 104;      // teardown: every MMA issued so far has finished
+  const uint32_t drain_fail = bars + 112;     // uint32: a teardown wait ran out as well
 
   const int warp = threadIdx.x >> 5;
   const int lane = threadIdx.x & 31;
@@ -153,6 +155,8 @@ __global__ void __launch_bounds__(kThreadsB, 1) tile_bwd_kernel(const __grid_con
     mbar_init(t_empty, 4);
     mbar_init(dq_full, 1);
     mbar_init(dq_empty, 4);
+    mbar_init(drain_bar, 1);
+    sts_u32(drain_fail, 0u);
     sts_u32(abort_flag, 0u);
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
@@ -203,6 +207,13 @@ __global__ void __launch_bounds__(kThreadsB, 1) tile_bwd_kernel(const __grid_con
             tma_load_4d(v_smem + hf * (TN * 128), &map_v, kv_full, hf * 64, kt * TN, h, b);
           }
         }
+      }
+      if (!alive) {
+        // a wait ran out somewhere in the CTA: the copies this thread armed barriers for must land before shared
+        // memory goes away (after n arms a phase word holds n mod 2 and the last armed phase has the other parity)
+        bool ok = mbar_drain(qdo_full, qphase ^ 1u);
+        ok &= mbar_drain(kv_full, kvphase ^ 1u);
+        if (!ok) sts_u32(drain_fail, 1u);
       }
     }
   } else if (warp == 1) {
@@ -300,6 +311,11 @@ __global__ void __launch_bounds__(kThreadsB, 1) tile_bwd_kernel(const __grid_con
           if (t == 2 * tiles - 1) umma_commit(dq_full);
         }
         umma_commit(qdo_empty);
+      }
+      if (!alive) {
+        // the tensor core must be done with shared memory and TMEM before they are released
+        umma_commit(drain_bar);
+        if (!mbar_drain(drain_bar, 0u)) sts_u32(drain_fail, 1u);
       }
     }
   } else {
@@ -473,8 +489,12 @@ __global__ void __launch_bounds__(kThreadsB, 1) tile_bwd_kernel(const __grid_con
   __syncthreads();
   if (lds_u32(abort_flag)) {
     if (threadIdx.x == 0 && a.status) atomicOr(a.status + ENTMAX_ATTN_STATUS_FLAGS, ENTMAX_ATTN_FLAG_WAIT_EXPIRED);
-    const uint64_t t0 = global_ns();
-    while (global_ns() - t0 < 200000ull) { }
+    // the producer and the MMA issuer have waited for their copies and MMAs in flight; only if one of those waits ran
+    // out as well is there nothing left but to give the hardware time
+    if (lds_u32(drain_fail)) {
+      const uint64_t t0 = global_ns();
+      while (global_ns() - t0 < 200000ull) { }
+    }
     __syncthreads();
   }
   if (warp == 1) {

@@ -125,8 +125,10 @@ __global__ void __launch_bounds__(kThreadsT, 1) tile_fwd_kernel(const __grid_con
   const uint32_t x_bar = done_word + 16;                              // partial sums of a sweep are in shared memory
   const uint32_t tmem_slot = x_bar + 8;
   const uint32_t abort_flag = tmem_slot + 4;
+  const uint32_t drain_bar = tmem_slot + 8;                           // teardown: every MMA issued so far has finished
+  const uint32_t drain_fail = drain_bar + 8;                          // uint32: a teardown wait ran out as well
   const uint32_t xchg = bars + C::kBarBytes;                          // float2 [2][TM]
-  static_assert(8 * (2 + 2 * C::kStages + 4 + 4 + 1) + 16 + 8 + 8 <= C::kBarBytes, "barrier area");
+  static_assert(8 * (2 + 2 * C::kStages + 4 + 4 + 1) + 16 + 8 + 8 + 16 <= C::kBarBytes, "barrier area");
 
   const int warp = threadIdx.x >> 5;
   const int lane = threadIdx.x & 31;
@@ -150,6 +152,8 @@ __global__ void __launch_bounds__(kThreadsT, 1) tile_fwd_kernel(const __grid_con
     mbar_init(ctl, 8);
     mbar_init(x_bar, 8);
     for (int t = 0; t < 3; ++t) sts_u32(done_word + 4 * t, 1u);
+    mbar_init(drain_bar, 1);
+    sts_u32(drain_fail, 0u);
     sts_u32(abort_flag, 0u);
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
@@ -247,6 +251,13 @@ __global__ void __launch_bounds__(kThreadsT, 1) tile_fwd_kernel(const __grid_con
           if (output) break;
         }
       }
+      if (!alive) {
+        // a wait ran out somewhere in the CTA: the copies this thread armed barriers for must land before shared
+        // memory goes away (stages before `stage`: this round of the ring; the others: the previous round)
+        bool ok = mbar_drain(q_full, qphase ^ 1u);
+        for (int st = 0; st < C::kStages; ++st) ok &= mbar_drain(kv_full + 8 * st, st < stage ? kvphase : kvphase ^ 1u);
+        if (!ok) sts_u32(drain_fail, 1u);
+      }
     }
   } else if (warp == 1) {
     // ------------------------------------------------------------------ MMA issuer
@@ -322,6 +333,11 @@ __global__ void __launch_bounds__(kThreadsT, 1) tile_fwd_kernel(const __grid_con
           if (output) break;
         }
         umma_commit(q_empty);
+      }
+      if (!alive) {
+        // the tensor core must be done with shared memory and TMEM before they are released
+        umma_commit(drain_bar);
+        if (!mbar_drain(drain_bar, 0u)) sts_u32(drain_fail, 1u);
       }
     }
   } else {
@@ -580,8 +596,12 @@ __global__ void __launch_bounds__(kThreadsT, 1) tile_fwd_kernel(const __grid_con
   __syncthreads();
   if (lds_u32(abort_flag)) {
     if (threadIdx.x == 0 && a.status) atomicOr(a.status + ENTMAX_ATTN_STATUS_FLAGS, ENTMAX_ATTN_FLAG_WAIT_EXPIRED);
-    const uint64_t t0 = global_ns();
-    while (global_ns() - t0 < 200000ull) { }
+    // the producer and the MMA issuer have waited for their copies and MMAs in flight; only if one of those waits ran
+    // out as well is there nothing left but to give the hardware time
+    if (lds_u32(drain_fail)) {
+      const uint64_t t0 = global_ns();
+      while (global_ns() - t0 < 200000ull) { }
+    }
     __syncthreads();
   }
   if (warp == 1) {
