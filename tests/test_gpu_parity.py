@@ -96,6 +96,27 @@ def test_dense_tiles_on_tensor_cores(N, d, causal, alpha):
     assert int(got["status"][binding.STATUS_DENSE_ROWS]) > N
 
 
+@pytest.mark.parametrize("sigma,expect", [(0.55, 200), (0.3, 1000), (0.18, 4000)])
+def test_dense_path_at_supports_of_hundreds_to_thousands(sigma, expect):
+    # long rows whose supports run to about 200, 1000 and 4000 keys (fixed temperature, logits of std sigma^2): forward
+    # (tau, O and the support size the dense-tile kernel counted) on sampled rows, backward on sampled dQ rows, at
+    # N = 8192 so that the dense-tile kernels take their sampled start
+    N = 8192
+    inp = make_inputs(Workload("dense_support_%d" % expect, 1, 2, N, 64, "bf16", True, (1.5,), qk_sigma=sigma, use_scale=False,
+                               backward=True, seed_offset=140 + expect % 97))
+    got = parity.run_fwd(inp, 1.5)
+    bwd = parity.run_bwd(inp, 1.5, got["tau"], got["dev"])
+    late = np.arange(N - 1536, N, 24)                        # rows that see the whole sequence, more or less
+    rows = np.unique(np.concatenate([sample_rows(inp, 0, 64), late]))
+    sizes = []
+    for bh in range(2):
+        st = parity.check_fwd_rows(inp, 1.5, got, bh, rows)
+        parity.check_bwd_rows(inp, 1.5, bwd, bh, rows)
+        sizes.append(st["supp_max"])
+        assert st["dense_rows"] > len(late) // 2             # these rows went through the dense-tile kernels
+    assert 0.4 * expect <= max(sizes) <= 2.5 * expect, sizes
+
+
 def test_mixed_sparse_and_dense_rows_in_one_tile():
     # planted keys make some rows one-hot while the others stay dense: both paths write into the same Q tiles
     inp = make_inputs(_small("mixed", 1000, 128, True, plant=3, use_scale=False, sigma=0.05, seed=21))
