@@ -55,47 +55,6 @@ __device__ __forceinline__ float block_max(float a, float* red) {
   return r;
 }
 
-template <int PER>
-__device__ __forceinline__ void load_slice(const float* p, float (&x)[PER]) {
-  if constexpr (PER == 2) { float2 t = *reinterpret_cast<const float2*>(p); x[0] = t.x; x[1] = t.y; }
-  else { float4 t = *reinterpret_cast<const float4*>(p); x[0] = t.x; x[1] = t.y; x[2] = t.z; x[3] = t.w; }
-}
-template <int PER>
-__device__ __forceinline__ void load_slice(const __nv_bfloat16* p, float (&x)[PER]) {
-  if constexpr (PER == 2) {
-    float2 t = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(p));
-    x[0] = t.x; x[1] = t.y;
-  } else {
-    uint2 raw = *reinterpret_cast<const uint2*>(p);
-    float2 t0 = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(&raw.x));
-    float2 t1 = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(&raw.y));
-    x[0] = t0.x; x[1] = t0.y; x[2] = t1.x; x[3] = t1.y;
-  }
-}
-template <int PER>
-__device__ __forceinline__ void store_slice(float* p, const float (&x)[PER]) {
-  if constexpr (PER == 2) *reinterpret_cast<float2*>(p) = make_float2(x[0], x[1]);
-  else *reinterpret_cast<float4*>(p) = make_float4(x[0], x[1], x[2], x[3]);
-}
-template <int PER>
-__device__ __forceinline__ void store_slice(__nv_bfloat16* p, const float (&x)[PER]) {
-  if constexpr (PER == 2) {
-    *reinterpret_cast<__nv_bfloat162*>(p) = __floats2bfloat162_rn(x[0], x[1]);
-  } else {
-    __nv_bfloat162 a = __floats2bfloat162_rn(x[0], x[1]);
-    __nv_bfloat162 b = __floats2bfloat162_rn(x[2], x[3]);
-    uint2 raw;
-    raw.x = *reinterpret_cast<uint32_t*>(&a);
-    raw.y = *reinterpret_cast<uint32_t*>(&b);
-    *reinterpret_cast<uint2*>(p) = raw;
-  }
-}
-template <int PER>
-__device__ __forceinline__ void atomic_add_slice(float* p, const float (&x)[PER]) {
-  if constexpr (PER == 2) red_add_v2(p, x[0], x[1]);
-  else red_add_v4(p, x[0], x[1], x[2], x[3]);
-}
-
 struct RowCtx {
   int grow, bh, b, h, i, nv;
   float c, a, g;

@@ -32,36 +32,11 @@ __device__ __forceinline__ float warp_max(float x) {
   return x;
 }
 
+// the row-slice helpers of common.cuh under the names this file uses
 template <int PER>
-__device__ __forceinline__ void load_bf16(const __nv_bfloat16* p, float (&x)[PER]) {
-  if constexpr (PER == 2) {
-    float2 t = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(p));
-    x[0] = t.x; x[1] = t.y;
-  } else {
-    uint2 raw = *reinterpret_cast<const uint2*>(p);
-    float2 t0 = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(&raw.x));
-    float2 t1 = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(&raw.y));
-    x[0] = t0.x; x[1] = t0.y; x[2] = t1.x; x[3] = t1.y;
-  }
-}
+__device__ __forceinline__ void load_bf16(const __nv_bfloat16* p, float (&x)[PER]) { load_slice<PER>(p, x); }
 template <int PER>
-__device__ __forceinline__ void store_bf16(__nv_bfloat16* p, const float (&x)[PER]) {
-  if constexpr (PER == 2) {
-    *reinterpret_cast<__nv_bfloat162*>(p) = __floats2bfloat162_rn(x[0], x[1]);
-  } else {
-    __nv_bfloat162 a = __floats2bfloat162_rn(x[0], x[1]);
-    __nv_bfloat162 b = __floats2bfloat162_rn(x[2], x[3]);
-    uint2 raw;
-    raw.x = *reinterpret_cast<uint32_t*>(&a);
-    raw.y = *reinterpret_cast<uint32_t*>(&b);
-    *reinterpret_cast<uint2*>(p) = raw;
-  }
-}
-template <int PER>
-__device__ __forceinline__ void atomic_add_slice(float* p, const float (&x)[PER]) {
-  if constexpr (PER == 2) red_add_v2(p, x[0], x[1]);
-  else red_add_v4(p, x[0], x[1], x[2], x[3]);
-}
+__device__ __forceinline__ void store_bf16(__nv_bfloat16* p, const float (&x)[PER]) { store_slice<PER>(p, x); }
 
 
 // reductions over aligned groups of W lanes (W = 8 or 16); the sum takes ascending strides like warp_sum
