@@ -147,8 +147,11 @@ constexpr float kKeepMargin = 4e-6f;
 // Threshold of Eq. 1 on the entries held by the warp, started at the bracket's lower end y_max - 1 (App. A):
 // Newton from the left for e >= 1, bracketed for e < 1 (tau_iter_update)
 template <int S>
-__device__ __forceinline__ float newton_warp(const Problem& p, const float (&y)[S], float ymax) {
+__device__ __forceinline__ float newton_warp(const Problem& p, const float (&y)[S], float ymax,
+                                             float known_below = -INFINITY) {
+  // known_below: a value the threshold is known not to lie below (mass >= 1 there); -inf: the bracket's own lower end
   TauIter st = tau_iter_start(ymax);
+  st.tau = st.lo = fmaxf(st.lo, known_below);
   for (int it = 0; it < kMaxNewton; ++it) {
     float s0 = 0.f, s1 = 0.f;
 #pragma unroll
@@ -171,7 +174,8 @@ __device__ __forceinline__ float newton_warp(const Problem& p, const float (&y)[
 // Stage A on S*32 candidate slots.  Leaves the kept entries (y in Eq. 1's units) compacted from slot 0
 // of the row's list and returns how many there are.
 template <int S>
-__device__ __forceinline__ int prefilter_row(const Problem& p, Entry* list, int c0, int c1, float a, int lane) {
+__device__ __forceinline__ int prefilter_row(const Problem& p, Entry* list, int c0, int c1, float a, int lane,
+                                             float bound) {
   float y[S];
   int jj[S];
   float ymax = -INFINITY;
@@ -189,7 +193,9 @@ __device__ __forceinline__ int prefilter_row(const Problem& p, Entry* list, int 
   }
   ymax = warp_max(ymax);
   __syncwarp();   // every slot is in registers before the list is overwritten
-  const float tau_a = newton_warp<S>(p, y, ymax);
+  // stage A may start from the bound the sweep ended with (a lower bound of the row's threshold, and every key above
+  // it is in the list): only its cut is used, so where it starts does not reach the result
+  const float tau_a = newton_warp<S>(p, y, ymax, bound);
   const float cut = tau_a - kKeepMargin * fmaxf(1.0f, fabsf(tau_a));
   int kept = 0;
 #pragma unroll
@@ -269,11 +275,12 @@ __device__ __forceinline__ void finish_row(const Problem& p, const __nv_bfloat16
 }
 
 // Out-of-line forms for the rare rows with more than 32 candidates (kept out of the hot loop's code)
-__device__ __noinline__ int prefilter_long(const Problem& p, Entry* list, int c0, int c1, float a, int lane) {
+__device__ __noinline__ int prefilter_long(const Problem& p, Entry* list, int c0, int c1, float a, int lane,
+                                           float bound) {
   const int n = c0 + c1;
-  if (n <= 64) return prefilter_row<2>(p, list, c0, c1, a, lane);
-  if (n <= 128) return prefilter_row<4>(p, list, c0, c1, a, lane);
-  return prefilter_row<kSlots>(p, list, c0, c1, a, lane);
+  if (n <= 64) return prefilter_row<2>(p, list, c0, c1, a, lane, bound);
+  if (n <= 128) return prefilter_row<4>(p, list, c0, c1, a, lane, bound);
+  return prefilter_row<kSlots>(p, list, c0, c1, a, lane, bound);
 }
 template <int D>
 __device__ __noinline__ void finish_long(const Problem& p, const __nv_bfloat16* __restrict__ vbase, Entry* list, int kept,
@@ -286,14 +293,14 @@ __device__ __noinline__ void finish_long(const Problem& p, const __nv_bfloat16* 
 // One row with the whole warp.
 template <int D>
 __device__ __forceinline__ void solve_row_full(const Problem& p, const __nv_bfloat16* __restrict__ vbase, Entry* list,
-                                               int c0, int c1, float a, __nv_bfloat16* o_row, float* tau_slot,
-                                               int32_t* cnt_slot, int lane) {
+                                               int c0, int c1, float a, float bound, __nv_bfloat16* o_row,
+                                               float* tau_slot, int32_t* cnt_slot, int lane) {
   const int n = c0 + c1;
   int kept;
-  if (n <= 32) kept = prefilter_row<1>(p, list, c0, c1, a, lane);
-  else if (n <= 64) kept = prefilter_row<2>(p, list, c0, c1, a, lane);
-  else if (n <= 128) kept = prefilter_row<4>(p, list, c0, c1, a, lane);
-  else kept = prefilter_row<kSlots>(p, list, c0, c1, a, lane);
+  if (n <= 32) kept = prefilter_row<1>(p, list, c0, c1, a, lane, bound);
+  else if (n <= 64) kept = prefilter_row<2>(p, list, c0, c1, a, lane, bound);
+  else if (n <= 128) kept = prefilter_row<4>(p, list, c0, c1, a, lane, bound);
+  else kept = prefilter_row<kSlots>(p, list, c0, c1, a, lane, bound);
   if (kept <= 32) finish_row<D, 1>(p, vbase, list, kept, o_row, tau_slot, cnt_slot, lane);
   else if (kept <= 64) finish_row<D, 2>(p, vbase, list, kept, o_row, tau_slot, cnt_slot, lane);
   else if (kept <= 128) finish_row<D, 4>(p, vbase, list, kept, o_row, tau_slot, cnt_slot, lane);
@@ -302,8 +309,10 @@ __device__ __forceinline__ void solve_row_full(const Problem& p, const __nv_bflo
 
 // The same iteration for 32 / W rows at once (W lanes per row); `done` rows keep their tau.
 template <int W>
-__device__ __forceinline__ float newton_sub(const Problem& p, float y, float ymax, bool done) {
+__device__ __forceinline__ float newton_sub(const Problem& p, float y, float ymax, bool done,
+                                            float known_below = -INFINITY) {
   TauIter st = tau_iter_start(ymax);
+  st.tau = st.lo = fmaxf(st.lo, known_below);
   for (int it = 0; it < kMaxNewton; ++it) {
     const float d = y - st.tau;
     float ye = 0.f, ye1 = 0.f;
@@ -320,8 +329,8 @@ template <int D, int W>
 __device__ __forceinline__ void solve_rows_sub(const Problem& p, const __nv_bfloat16* __restrict__ v,
                                                 const float* __restrict__ scale, Entry* __restrict__ entries,
                                                 __nv_bfloat16* __restrict__ o, float* __restrict__ tau_out,
-                                                int32_t* __restrict__ row_cnt, int grow, bool active, int c0, int c1,
-                                                int lane) {
+                                                int32_t* __restrict__ row_cnt, const float* __restrict__ half_thr,
+                                                int grow, bool active, int c0, int c1, int lane) {
   constexpr int PL = D / W;                        // elements of a V / O row per lane
   const int sl = lane & (W - 1);
   const int base = lane & (32 - W);
@@ -338,7 +347,14 @@ __device__ __forceinline__ void solve_rows_sub(const Problem& p, const __nv_bflo
   }
   __syncwarp();   // every entry is in registers before the compaction below overwrites the lists
   // stage A
-  const float tau_a = newton_sub<W>(p, y, sub_max<W>(y), !active);
+  // stage A starts from the bound the sweep ended with (see prefilter_row)
+  float bound = -INFINITY;
+  if (active) {
+    const float2 ht = *reinterpret_cast<const float2*>(half_thr + 2 * (size_t)grow);
+    bound = fmaxf(ht.x, ht.y);
+    bound -= kKeepMargin * fmaxf(1.0f, fabsf(bound));
+  }
+  const float tau_a = newton_sub<W>(p, y, sub_max<W>(y), !active, bound);
   const bool keep = active && y > tau_a - kKeepMargin * fmaxf(1.0f, fabsf(tau_a));
   // keep only those: they move to the end-stable front when sorted with the others' keys pushed to infinity
   j = keep ? j : 0x7fffffff;
@@ -529,6 +545,7 @@ __global__ void __launch_bounds__(kWarpsPerCta * 32) row_fwd_kernel(Problem p, c
                                                                     const float* __restrict__ scale,
                                                                     int32_t* __restrict__ row_cnt,
                                                                     const int32_t* __restrict__ half_cnt,
+                                                                    const float* __restrict__ half_thr,
                                                                     Entry* __restrict__ entries,
                                                                     __nv_bfloat16* __restrict__ o,
                                                                     float* __restrict__ tau_out, int32_t* fb_count,
@@ -587,7 +604,8 @@ __global__ void __launch_bounds__(kWarpsPerCta * 32) row_fwd_kernel(Problem p, c
           const int src = 4 * g + (lane >> 3);
           const bool active = (m8 >> src) & 1u;
           const int c0 = __shfl_sync(0xffffffffu, mc0, src), c1 = __shfl_sync(0xffffffffu, mc1, src);
-          solve_rows_sub<D, 8>(p, v, scale, entries, o, tau_out, row_cnt, active ? 16 * blk + src : 0, active, c0, c1, lane);
+          solve_rows_sub<D, 8>(p, v, scale, entries, o, tau_out, row_cnt, half_thr, active ? 16 * blk + src : 0, active, c0,
+                               c1, lane);
         } else {
           mfull |= (m8 | m16) & gm;
         }
@@ -608,6 +626,9 @@ __global__ void __launch_bounds__(kWarpsPerCta * 32) row_fwd_kernel(Problem p, c
       const int bh = grow / p.N, i = grow - bh * p.N, b = bh / p.H, h = bh - b * p.H;
       const float a = (p.alpha - 1.0f) * (scale[(size_t)b * p.scale_sb + (size_t)h * p.N + i] * p.sm_scale);
       Entry* list = entries + (size_t)grow * kListCap;
+      const float2 ht = *reinterpret_cast<const float2*>(half_thr + 2 * (size_t)grow);
+      float bound = fmaxf(ht.x, ht.y);
+      bound -= kKeepMargin * fmaxf(1.0f, fabsf(bound));
       if constexpr (kClosed) {
         // up to 32 entries: closed form with the whole warp; more: Newton prefilter first, and the closed form
         // if what it keeps fits the warp
@@ -616,7 +637,7 @@ __global__ void __launch_bounds__(kWarpsPerCta * 32) row_fwd_kernel(Problem p, c
           solve_rows_closed<D, 32, EC>(p, v, scale, entries, o, tau_out, row_cnt, grow, true, c0, c1, false, lane);
           continue;
         }
-        const int kept = prefilter_long(p, list, c0, c1, a, lane);
+        const int kept = prefilter_long(p, list, c0, c1, a, lane, bound);
         if (kept <= 32) {
           solve_rows_closed<D, 32, EC>(p, v, scale, entries, o, tau_out, row_cnt, grow, true, kept, 0, true, lane);
           continue;
@@ -627,7 +648,7 @@ __global__ void __launch_bounds__(kWarpsPerCta * 32) row_fwd_kernel(Problem p, c
       } else {
         const __nv_bfloat16* vbase = v + (size_t)b * p.sb + (size_t)h * p.sh + lane * PER;
         __nv_bfloat16* o_row = o + (size_t)b * p.sb + (size_t)h * p.sh + (size_t)i * p.sn + lane * PER;
-        solve_row_full<D>(p, vbase, list, c0, c1, a, o_row, tau_out + grow, row_cnt + grow, lane);
+        solve_row_full<D>(p, vbase, list, c0, c1, a, bound, o_row, tau_out + grow, row_cnt + grow, lane);
       }
     }
   }
@@ -985,7 +1006,8 @@ cudaError_t launch_row_fwd(const Problem& p, const void* v, const float* scale, 
   const int grid = row_grid(p);
 #define ENTMAX_ROW_FWD(D, EC)                                                                                         \
   row_fwd_kernel<D, EC><<<grid, kWarpsPerCta * 32, 0, stream>>>(p, (const __nv_bfloat16*)v, scale, row_cnt, half_cnt, \
-                                                                entries, (__nv_bfloat16*)o, tau, fb_count, fb_list,   \
+                                                                half_thr, entries, (__nv_bfloat16*)o, tau, fb_count,  \
+                                                                fb_list,                                              \
                                                                 tile_flag, tile_list, tile_count, status)
   if (p.D == 64) {
     if (p.expo_class == kExpo2) ENTMAX_ROW_FWD(64, kExpo2);
