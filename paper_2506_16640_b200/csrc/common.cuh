@@ -209,19 +209,28 @@ cudaError_t launch_sweep(const Problem& p, const void* q, const void* k, const f
                          float* dump, int dump_bh, float* alibi_blob, float* alibi_kmax, int32_t* status,
                          cudaStream_t stream);
 
-// Dense-tile forward on the tensor cores (bf16): recomputes the Q tiles (128 rows) listed in tile_list
-// and writes O and tau of their rows marked row_cnt == -2, and into dense_cnt [B*H*N][2] the number of keys
-// with p > 0 each of the row's two threads saw (their sum is the row's support size).
+// Puts tile_list[0 .. *tile_count) (the Q tiles flagged in tile_flag) into the order the dense-tile kernels hand
+// them out in: longest first on causal problems.
+cudaError_t order_tiles(const Problem& p, const int32_t* tile_flag, int32_t* tile_list, const int32_t* tile_count,
+                        cudaStream_t stream);
+
+// Dense-tile forward on the tensor cores (bf16): recomputes the Q tiles (128 rows) listed in tile_list (= flagged
+// in tile_flag; the list is reordered) and writes O and tau of their rows marked row_cnt == -2, and into dense_cnt
+// [B*H*N][2] the number of keys with p > 0 each of the row's two threads saw (their sum is the row's support
+// size).  *work_counter must be zero on entry.
 cudaError_t launch_tile_fwd(const Problem& p, const void* q, const void* k, const void* v, const float* scale,
-                            const int32_t* tile_list, const int32_t* tile_count, const int32_t* row_cnt,
-                            int32_t* dense_cnt, void* o, float* tau, int32_t* status, cudaStream_t stream);
+                            const int32_t* tile_flag, int32_t* tile_list, const int32_t* tile_count,
+                            int32_t* work_counter, const int32_t* row_cnt, int32_t* dense_cnt, void* o, float* tau,
+                            int32_t* status, cudaStream_t stream);
 
 // Dense-tile backward on the tensor cores (bf16): the rows in row_list[0 .. *row_count) are marked in
 // tile_mask, their 128-row Q tiles listed, and dQ (and dc_rows) of those rows written; their dK and dV
-// contributions are added to the fp32 accumulators.  tile_mask, tile_flag and *tile_count must be zero on entry.
+// contributions are added to the fp32 accumulators.  tile_mask, tile_flag, *tile_count and *work_counter must be
+// zero on entry.
 cudaError_t launch_tile_bwd(const Problem& p, const void* q, const void* k, const void* v, const void* d_o,
                             const float* scale, const float* tau, const int32_t* row_list, const int32_t* row_count,
-                            uint32_t* tile_mask, int32_t* tile_flag, int32_t* tile_list, int32_t* tile_count, void* dq,
+                            uint32_t* tile_mask, int32_t* tile_flag, int32_t* tile_list, int32_t* tile_count,
+                            int32_t* work_counter, void* dq,
                             float* acc_dk, float* acc_dv, float* dc_rows, int32_t* status, cudaStream_t stream);
 
 // per-row solve + gather kernels working on the lists (bf16 path); the forward one also lists the

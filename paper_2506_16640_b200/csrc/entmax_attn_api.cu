@@ -135,7 +135,7 @@ WsLayout make_layout(const Problem& p, bool is_bwd) {
   l.entries = take(rows * kListCap * sizeof(Entry));
   l.fb_count = take(256);
   l.sweep_counter = l.fb_count + 64;   // same 256-byte block: [0] dense-row count, [16] sweep work counter,
-  l.tile_count = l.fb_count + 128;     // [32] number of listed dense tiles
+  l.tile_count = l.fb_count + 128;     // [32] number of listed dense tiles, [48] the dense-tile kernels' work counter
   l.fb_list = take(rows * sizeof(int32_t));
   const size_t q_tiles = (size_t)p.B * p.H * ((p.N + 127) / 128);
   l.tile_flag = take(q_tiles * sizeof(int32_t));
@@ -261,7 +261,8 @@ int fwd_impl(const entmax_attn_params* params, const void* q, const void* k, con
                        tile_count, device_status, stream);
   if (err != cudaSuccess) return fail_cuda(err);
   // rows whose support does not fit the lists: dense tiles on the tensor cores
-  err = launch_tile_fwd(p, q, k, v, scale, tile_list, tile_count, row_cnt, half_cnt, o, tau, device_status, stream);
+  err = launch_tile_fwd(p, q, k, v, scale, tile_flag, tile_list, tile_count, tile_count + 16, row_cnt, half_cnt, o, tau,
+                        device_status, stream);
   return err == cudaSuccess ? ENTMAX_ATTN_OK : fail_cuda(err);
 }
 
@@ -417,7 +418,7 @@ int bwd_impl(const entmax_attn_params* params, const void* q, const void* k, con
       if (err != cudaSuccess) return fail_cuda(err);
     }
     // rows whose support does not fit the lists: dense tiles on the tensor cores
-    err = launch_tile_bwd(p, q, k, v, d_o, scale, tau, fb_list, fb_count, tile_mask, tile_flag, tile_list, tile_count, dq,
+    err = launch_tile_bwd(p, q, k, v, d_o, scale, tau, fb_list, fb_count, tile_mask, tile_flag, tile_list, tile_count, tile_count + 16, dq,
                           acc_dk, acc_dv, dc_rows, device_status, stream);
     if (err != cudaSuccess) return fail_cuda(err);
   }

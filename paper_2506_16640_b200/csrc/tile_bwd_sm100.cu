@@ -55,6 +55,7 @@ struct TileBwdArgs {
   long long scale_sb;
   const int32_t* tile_list;  // ids of the Q tiles to process: bh * tiles_per_head + tile
   const int32_t* tile_count;
+  int32_t* work_counter;     // next position of tile_list to hand out (zero on entry)
   const uint32_t* tile_mask; // [tiles, 4]: bit r of a tile's 128-bit mask marks row r for this kernel
   const float* tau;
   void* dq;                  // bf16 [B,H,N,D]
@@ -137,6 +138,9 @@ __global__ void __launch_bounds__(kThreadsB, 1) tile_bwd_kernel(const __grid_con
   const uint32_t abort_flag = bars + 100;
   const uint32_t drain_bar = bars + 104;      // teardown: every MMA issued so far has finished
   const uint32_t drain_fail = bars + 112;     // uint32: a teardown wait ran out as well
+  const uint32_t w_full = bars + 120;         // [2] a work item has been published
+  const uint32_t w_empty = bars + 136;        // [2] ... and read by the MMA issuer and every consumer warp
+  const uint32_t w_item = bars + 152;         // int32 [2]: tile id, -1 = no more work
 
   const int warp = threadIdx.x >> 5;
   const int lane = threadIdx.x & 31;
@@ -156,6 +160,10 @@ __global__ void __launch_bounds__(kThreadsB, 1) tile_bwd_kernel(const __grid_con
     mbar_init(dq_full, 1);
     mbar_init(dq_empty, 4);
     mbar_init(drain_bar, 1);
+    for (int t = 0; t < 2; ++t) {
+      mbar_init(w_full + 8 * t, 1);
+      mbar_init(w_empty + 8 * t, 5);   // MMA issuer + four consumer warps
+    }
     sts_u32(drain_fail, 0u);
     sts_u32(abort_flag, 0u);
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -181,10 +189,19 @@ __global__ void __launch_bounds__(kThreadsB, 1) tile_bwd_kernel(const __grid_con
   if (warp == 0) {
     // ------------------------------------------------------------------ TMA producer
     if (lane == 0) {
-      uint32_t kvphase = 0, qphase = 0;
+      uint32_t kvphase = 0, qphase = 0, wphase = 0;
+      int slot = 0;
       bool alive = true;
-      for (int it = blockIdx.x; it < n_tiles && alive; it += gridDim.x) {
-        const int id = a.tile_list[it];
+      while (alive) {
+        // items are handed out from a shared counter, in the list's order (longest first on causal problems)
+        alive = mbar_wait(w_empty + 8 * slot, wphase ^ 1u, abort_flag);
+        if (!alive) break;
+        const int it = atomicAdd(a.work_counter, 1);
+        const int id = it < n_tiles ? a.tile_list[it] : -1;
+        sts_u32(w_item + 4 * slot, (uint32_t)id);
+        mbar_arrive(w_full + 8 * slot);
+        if (++slot == 2) { slot = 0; wphase ^= 1u; }
+        if (id < 0) break;
         const int bh = id / a.tiles_per_head, tile = id - bh * a.tiles_per_head;
         const int b = bh / a.H, h = bh - b * a.H;
         const int tiles = item_tiles(tile);
@@ -227,10 +244,16 @@ __global__ void __launch_bounds__(kThreadsB, 1) tile_bwd_kernel(const __grid_con
       const uint32_t ds_lo = smem_desc_lo(ds_smem), dl_lo = smem_desc_lo(dl_smem);
       const uint32_t k_n_lo = mn_desc_lo(k_smem), q_n_lo = mn_desc_lo(q_smem), do_n_lo = mn_desc_lo(do_smem);
       const uint32_t ds_m_lo = mn_desc_lo(ds_smem), p_m_lo = mn_desc_lo(p_smem);
-      uint32_t kvphase = 0, qphase = 0, sdphase = 0, pdsphase = 0, tphase = 0, dqphase = 0;
+      uint32_t kvphase = 0, qphase = 0, sdphase = 0, pdsphase = 0, tphase = 0, dqphase = 0, wphase = 0;
+      int slot = 0;
       bool alive = true;
-      for (int it = blockIdx.x; it < n_tiles && alive; it += gridDim.x) {
-        const int id = a.tile_list[it];
+      while (alive) {
+        alive = mbar_wait(w_full + 8 * slot, wphase, abort_flag);
+        if (!alive) break;
+        const int id = (int)lds_u32(w_item + 4 * slot);
+        mbar_arrive(w_empty + 8 * slot);
+        if (++slot == 2) { slot = 0; wphase ^= 1u; }
+        if (id < 0) break;
         const int tile = id % a.tiles_per_head;
         const int tiles = item_tiles(tile);
         alive = mbar_wait(qdo_full, qphase, abort_flag);
@@ -323,10 +346,17 @@ __global__ void __launch_bounds__(kThreadsB, 1) tile_bwd_kernel(const __grid_con
     const int quad = warp & 3;
     const int row_local = quad * 32 + lane;
     const uint32_t taddr_row = tmem_base + ((uint32_t)(quad * 32) << 16);
-    uint32_t sdphase = 0, pdsphase = 0, tphase = 0, dqphase = 0;
+    uint32_t sdphase = 0, pdsphase = 0, tphase = 0, dqphase = 0, wphase = 0;
+    int slot = 0;
     bool alive = true;
-    for (int it = blockIdx.x; it < n_tiles && alive; it += gridDim.x) {
-      const int id = a.tile_list[it];
+    while (alive) {
+      alive = __all_sync(0xffffffffu, mbar_wait(w_full + 8 * slot, wphase, abort_flag));
+      if (!alive) break;
+      const int id = (int)lds_u32(w_item + 4 * slot);
+      __syncwarp();
+      if (lane == 0) mbar_arrive(w_empty + 8 * slot);
+      if (++slot == 2) { slot = 0; wphase ^= 1u; }
+      if (id < 0) break;
       const int bh = id / a.tiles_per_head, tile = id - bh * a.tiles_per_head;
       const int b = bh / a.H, h = bh - b * a.H;
       const int tiles = item_tiles(tile);
@@ -532,12 +562,14 @@ cudaError_t launch_tile_bwd_impl(const Problem& p, const void* q, const void* k,
 
 cudaError_t launch_tile_bwd(const Problem& p, const void* q, const void* k, const void* v, const void* d_o,
                             const float* scale, const float* tau, const int32_t* row_list, const int32_t* row_count,
-                            uint32_t* tile_mask, int32_t* tile_flag, int32_t* tile_list, int32_t* tile_count, void* dq,
-                            float* acc_dk, float* acc_dv, float* dc_rows, int32_t* status, cudaStream_t stream) {
+                            uint32_t* tile_mask, int32_t* tile_flag, int32_t* tile_list, int32_t* tile_count,
+                            int32_t* work_counter, void* dq, float* acc_dk, float* acc_dv, float* dc_rows, int32_t* status, cudaStream_t stream) {
   const int tiles_per_head = (p.N + TM - 1) / TM;
   mark_tiles_kernel<<<148, 256, 0, stream>>>(p.N, tiles_per_head, row_list, row_count, tile_mask, tile_flag, tile_list,
                                              tile_count);
   cudaError_t err = cudaGetLastError();
+  if (err != cudaSuccess) return err;
+  err = order_tiles(p, tile_flag, tile_list, tile_count, stream);
   if (err != cudaSuccess) return err;
   TileBwdArgs args;
   args.B = p.B; args.H = p.H; args.N = p.N;
@@ -551,6 +583,7 @@ cudaError_t launch_tile_bwd(const Problem& p, const void* q, const void* k, cons
   args.scale_sb = p.scale_sb;
   args.tile_list = tile_list;
   args.tile_count = tile_count;
+  args.work_counter = work_counter;
   args.tile_mask = tile_mask;
   args.tau = tau;
   args.dq = dq;

@@ -73,6 +73,7 @@ struct TileArgsK {
   long long scale_sb;
   const int32_t* tile_list;  // ids of the Q tiles to process: bh * tiles_per_head + tile
   const int32_t* tile_count;
+  int32_t* work_counter;     // next position of tile_list to hand out (zero on entry)
   const int32_t* row_cnt;    // -2 marks the rows to write
   int32_t* dense_cnt;        // [B*H*N][2]: support size each of a row's two threads counted (written rows only)
   void* o;                   // bf16 [B,H,N,D]
@@ -127,8 +128,11 @@ __global__ void __launch_bounds__(kThreadsT, 1) tile_fwd_kernel(const __grid_con
   const uint32_t abort_flag = tmem_slot + 4;
   const uint32_t drain_bar = tmem_slot + 8;                           // teardown: every MMA issued so far has finished
   const uint32_t drain_fail = drain_bar + 8;                          // uint32: a teardown wait ran out as well
+  const uint32_t w_full = drain_fail + 8;                             // [2] a work item has been published
+  const uint32_t w_empty = w_full + 16;                               // [2] ... and read by the MMA issuer and every consumer warp
+  const uint32_t w_item = w_empty + 16;                               // int32 [2]: tile id, -1 = no more work
   const uint32_t xchg = bars + C::kBarBytes;                          // float2 [2][TM]
-  static_assert(8 * (2 + 2 * C::kStages + 4 + 4 + 1) + 16 + 8 + 8 + 16 <= C::kBarBytes, "barrier area");
+  static_assert(8 * (2 + 2 * C::kStages + 4 + 4 + 1) + 16 + 8 + 8 + 16 + 40 <= C::kBarBytes, "barrier area");
 
   const int warp = threadIdx.x >> 5;
   const int lane = threadIdx.x & 31;
@@ -153,6 +157,10 @@ __global__ void __launch_bounds__(kThreadsT, 1) tile_fwd_kernel(const __grid_con
     mbar_init(x_bar, 8);
     for (int t = 0; t < 3; ++t) sts_u32(done_word + 4 * t, 1u);
     mbar_init(drain_bar, 1);
+    for (int t = 0; t < 2; ++t) {
+      mbar_init(w_full + 8 * t, 1);
+      mbar_init(w_empty + 8 * t, 9);   // MMA issuer + eight consumer warps
+    }
     sts_u32(drain_fail, 0u);
     sts_u32(abort_flag, 0u);
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -208,11 +216,20 @@ __global__ void __launch_bounds__(kThreadsT, 1) tile_fwd_kernel(const __grid_con
   if (warp == 0) {
     // ------------------------------------------------------------------ TMA producer
     if (lane == 0) {
-      int stage = 0;
-      uint32_t kvphase = 0, qphase = 0, cphase = 0;
+      int stage = 0, slot = 0;
+      uint32_t kvphase = 0, qphase = 0, cphase = 0, wphase = 0;
       bool alive = true;
-      for (int it = blockIdx.x; it < n_tiles && alive; it += gridDim.x) {
-        const int id = a.tile_list[it];
+      while (alive) {
+        // items are handed out from a shared counter, in the list's order (longest first on causal problems), so
+        // that the CTAs finish together whatever the Q tiles' lengths and sweep counts are
+        alive = mbar_wait(w_empty + 8 * slot, wphase ^ 1u, abort_flag);
+        if (!alive) break;
+        const int it = atomicAdd(a.work_counter, 1);
+        const int id = it < n_tiles ? a.tile_list[it] : -1;
+        sts_u32(w_item + 4 * slot, (uint32_t)id);
+        mbar_arrive(w_full + 8 * slot);
+        if (++slot == 2) { slot = 0; wphase ^= 1u; }
+        if (id < 0) break;
         const int bh = id / a.tiles_per_head, tile = id - bh * a.tiles_per_head;
         const int b = bh / a.H, h = bh - b * a.H;
         const int tiles = item_tiles(tile), stiles = item_sample_tiles(tile);
@@ -268,10 +285,16 @@ __global__ void __launch_bounds__(kThreadsT, 1) tile_fwd_kernel(const __grid_con
       const uint32_t v_lo = v_desc_lo(v_smem);
       int stage = 0;
       uint32_t kvphase = 0, qphase = 0, cphase = 0, sphase[2] = {0, 0}, pphase = 0, ophase = 0;
-      int sbuf = 0;
+      int sbuf = 0, slot = 0;
+      uint32_t wphase = 0;
       bool alive = true;
-      for (int it = blockIdx.x; it < n_tiles && alive; it += gridDim.x) {
-        const int id = a.tile_list[it];
+      while (alive) {
+        alive = mbar_wait(w_full + 8 * slot, wphase, abort_flag);
+        if (!alive) break;
+        const int id = (int)lds_u32(w_item + 4 * slot);
+        mbar_arrive(w_empty + 8 * slot);
+        if (++slot == 2) { slot = 0; wphase ^= 1u; }
+        if (id < 0) break;
         const int tile = id % a.tiles_per_head;
         const int tiles = item_tiles(tile), stiles = item_sample_tiles(tile);
         int phase = stiles > 0 ? 0 : 1, n_full = 0;
@@ -348,10 +371,17 @@ __global__ void __launch_bounds__(kThreadsT, 1) tile_fwd_kernel(const __grid_con
     const int row_local = quad * 32 + lane;
     const uint32_t taddr_row = tmem_base + ((uint32_t)(quad * 32) << 16);
     uint32_t sphase[2] = {0, 0}, pphase = 0, ophase = 0, cphase = 0, xphase = 0;
-    int sbuf = 0;
+    int sbuf = 0, slot = 0;
+    uint32_t wphase = 0;
     bool alive = true;
-    for (int it = blockIdx.x; it < n_tiles && alive; it += gridDim.x) {
-      const int id = a.tile_list[it];
+    while (alive) {
+      alive = __all_sync(0xffffffffu, mbar_wait(w_full + 8 * slot, wphase, abort_flag));
+      if (!alive) break;
+      const int id = (int)lds_u32(w_item + 4 * slot);
+      __syncwarp();
+      if (lane == 0) mbar_arrive(w_empty + 8 * slot);
+      if (++slot == 2) { slot = 0; wphase ^= 1u; }
+      if (id < 0) break;
       const int bh = id / a.tiles_per_head, tile = id - bh * a.tiles_per_head;
       const int b = bh / a.H, h = bh - b * a.H;
       const int tiles = item_tiles(tile), stiles = item_sample_tiles(tile);
@@ -610,6 +640,44 @@ __global__ void __launch_bounds__(kThreadsT, 1) tile_fwd_kernel(const __grid_con
   }
 }
 
+// Rewrites tile_list[0 .. *tile_count) in the order the dense-tile kernels hand the Q tiles out: on causal problems
+// the tiles that see the most keys first (descending tile index, the heads interleaved).  The listed tiles are the
+// ones flagged in tile_flag; the kernel compacts the flags in that order.  One CTA.
+__global__ void __launch_bounds__(1024) order_tiles_kernel(const int32_t* __restrict__ tile_flag, int tiles_per_head,
+                                                           int n_bh, int32_t* __restrict__ tile_list,
+                                                           const int32_t* __restrict__ tile_count) {
+  __shared__ int warp_sum[32];
+  __shared__ int base;
+  if (*tile_count == 0) return;
+  const int lane = threadIdx.x & 31, w = threadIdx.x >> 5;
+  const long long total = (long long)tiles_per_head * n_bh;
+  if (threadIdx.x == 0) base = 0;
+  __syncthreads();
+  for (long long c0 = 0; c0 < total; c0 += 1024) {
+    const long long pos = c0 + threadIdx.x;
+    int id = -1;
+    bool f = false;
+    if (pos < total) {
+      const int tile = tiles_per_head - 1 - (int)(pos / n_bh);
+      id = (int)(pos % n_bh) * tiles_per_head + tile;
+      f = tile_flag[id] != 0;
+    }
+    const unsigned bal = __ballot_sync(0xffffffffu, f);
+    if (lane == 0) warp_sum[w] = __popc(bal);
+    __syncthreads();
+    int off = base;
+    for (int x = 0; x < w; ++x) off += warp_sum[x];
+    if (f) tile_list[off + __popc(bal & ((1u << lane) - 1u))] = id;
+    __syncthreads();
+    if (threadIdx.x == 0) {
+      int sum = 0;
+      for (int x = 0; x < 32; ++x) sum += warp_sum[x];
+      base += sum;
+    }
+    __syncthreads();
+  }
+}
+
 template <int HD, int EC>
 cudaError_t launch_tile_impl(const Problem& p, const void* q, const void* k, const void* v, const TileArgsK& args,
                              cudaStream_t stream) {
@@ -698,9 +766,19 @@ cudaError_t make_sampled_tile_map(CUtensorMap* map, const void* base, int D, int
 
 }  // namespace sm100
 
+cudaError_t order_tiles(const Problem& p, const int32_t* tile_flag, int32_t* tile_list, const int32_t* tile_count,
+                        cudaStream_t stream) {
+  if (!p.causal) return cudaSuccess;   // every Q tile sees the same keys: any order will do
+  order_tiles_kernel<<<1, 1024, 0, stream>>>(tile_flag, (p.N + TM - 1) / TM, p.B * p.H, tile_list, tile_count);
+  return cudaGetLastError();
+}
+
 cudaError_t launch_tile_fwd(const Problem& p, const void* q, const void* k, const void* v, const float* scale,
-                            const int32_t* tile_list, const int32_t* tile_count, const int32_t* row_cnt,
-                            int32_t* dense_cnt, void* o, float* tau, int32_t* status, cudaStream_t stream) {
+                            const int32_t* tile_flag, int32_t* tile_list, const int32_t* tile_count,
+                            int32_t* work_counter, const int32_t* row_cnt, int32_t* dense_cnt, void* o, float* tau,
+                            int32_t* status, cudaStream_t stream) {
+  cudaError_t oerr = order_tiles(p, tile_flag, tile_list, tile_count, stream);
+  if (oerr != cudaSuccess) return oerr;
   TileArgsK args;
   args.B = p.B; args.H = p.H; args.N = p.N;
   args.causal = p.causal;
@@ -713,6 +791,7 @@ cudaError_t launch_tile_fwd(const Problem& p, const void* q, const void* k, cons
   args.scale_sb = p.scale_sb;
   args.tile_list = tile_list;
   args.tile_count = tile_count;
+  args.work_counter = work_counter;
   args.row_cnt = row_cnt;
   args.dense_cnt = dense_cnt;
   args.o = o;
