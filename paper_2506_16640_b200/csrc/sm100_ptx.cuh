@@ -144,6 +144,29 @@ __device__ __forceinline__ void umma_bf16_ab(uint32_t d_tmem, uint32_t a_lo, uin
       : "memory");
 }
 // mbarrier arrive once every MMA issued so far by this thread has completed
+// The same with both descriptors given as 64-bit values (kept in uniform registers by warp-uniform callers).
+__device__ __forceinline__ void umma_bf16_desc(uint32_t d_tmem, uint64_t adesc, uint64_t bdesc, uint32_t idesc,
+                                               uint32_t accumulate) {
+  asm volatile(
+      "{\n"
+      " .reg .pred p;\n"
+      " setp.ne.b32 p, %4, 0;\n"
+      " tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n"
+      "}\n" ::"r"(d_tmem), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate)
+      : "memory");
+}
+// True in exactly one lane of a converged warp.
+__device__ __forceinline__ bool elect_one() {
+  uint32_t ok;
+  asm volatile(
+      "{\n"
+      " .reg .pred p;\n"
+      " elect.sync _|p, 0xffffffff;\n"
+      " selp.u32 %0, 1, 0, p;\n"
+      "}\n"
+      : "=r"(ok));
+  return ok != 0;
+}
 __device__ __forceinline__ void umma_commit(uint32_t bar) {
   asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar)
                : "memory");
@@ -208,6 +231,13 @@ __device__ __forceinline__ f32x2 add2(f32x2 a, f32x2 b) {
   return r;
 }
 
+// 1 for m > 0, 0 for m == 0 (m >= 0), on the FMA pipe: the product with 2^100 saturated to [0, 1].  A clamped
+// difference fma(a, x, -tau) that is positive is at least 2^-47 of the larger operand, far above 2^-100.
+__device__ __forceinline__ float positive_indicator(float m) {
+  float r;
+  asm("fma.rn.sat.f32 %0, %1, 0f71800000, 0f00000000;" : "=f"(r) : "f"(m));
+  return r;
+}
 __device__ __forceinline__ float max3(float a, float b, float c) {
   float r;
   asm("max.f32 %0, %1, %2, %3;" : "=f"(r) : "f"(a), "f"(b), "f"(c));

@@ -11,9 +11,9 @@
 // A work item is one Q tile of 128 rows that holds at least one such row (a list written by the row
 // kernel); only the rows flagged there are written back.
 //
-// CTA: warp 0 TMA producer, warp 1 MMA issuer, warps 2..9 consumers: TMEM lane = query row, two threads per
-// row (warps w and w + 4 read the same lane quadrant), each scanning 64 of a K tile's 128 columns; at the end of a
-// sweep the two swap their partial sums through shared memory.  The number of Newton sweeps is decided by the
+// CTA: warp 0 TMA producer, warp 1 MMA issuer, warps 2..17 consumers: TMEM lane = query row, four threads per
+// row (warps w, w + 4, w + 8, w + 12 read the same lane quadrant), each scanning 32 of a K tile's 128 columns; at the
+// end of a sweep the four swap their partial sums through shared memory.  The number of Newton sweeps is decided by the
 // consumers; they publish "all rows converged" through shared memory and a control mbarrier that every role
 // waits on between sweeps.  Every wait is bounded (see sm100_ptx.cuh); on expiry the CTA flags the call's status
 // word and leaves.
@@ -38,7 +38,9 @@ __device__ __forceinline__ void tma_load_5d(uint32_t dst, const CUtensorMap* map
 
 constexpr int TM = 128;            // query rows per item = TMEM lanes
 constexpr int TN = 128;            // keys per K/V tile
-constexpr int kThreadsT = 10 * 32;    // TMA warp, MMA warp, eight consumer warps
+constexpr int kConsGroups = 4;                       // threads per query row
+constexpr int kConsWarps = 4 * kConsGroups;           // four TMEM lane quadrants each
+constexpr int kThreadsT = (2 + kConsWarps) * 32;      // TMA warp, MMA warp, the consumer warps
 constexpr int kMaxSweeps = 48;     // 1 max sweep + at most 46 Newton sweeps + the output sweep
 // Sampled start: long rows first solve Eq. 1's threshold on every kTileSampleStride-th key (sweeps an eighth as long).
 // The threshold of a subset never exceeds that of the whole row, so the full-row Newton iteration may start from it
@@ -54,9 +56,10 @@ struct TCfg {
   static constexpr int kHalves = HD / 64;
   static constexpr int kQBytes = TM * HD * 2;
   static constexpr int kKBytes = TN * HD * 2;      // also the size of a V tile
-  static constexpr int kBarBytes = 256;
-  static constexpr int kXchgBytes = 2 * TM * 8;    // one float2 per (half, row): partial sums between the two threads of a row
-  static constexpr int kStages = HD == 64 ? 4 : 2;   // K/V ring depth: what fits beside Q and P
+  static constexpr int kBarBytes = 384;
+  static constexpr int kXchgBytes = 2 * kConsGroups * TM * 8;   // one float2 per (exchange parity, thread of a row, row)
+  static constexpr int kStages = HD == 64 ? 4 : 2;   // K/V ring depth of the output sweep: what fits beside Q and P
+  static constexpr int kSlots = 2 * kStages;         // tile slots; the other sweeps load K only and use all of them
   static constexpr int kSmemBytes = kQBytes + kStages * 2 * kKBytes + kPBytes + 1024 + kBarBytes + kXchgBytes;
   static constexpr int kTmemO = 2 * TN;            // first TMEM column of the O accumulator
 };
@@ -110,14 +113,16 @@ __global__ void __launch_bounds__(kThreadsT, 1) tile_fwd_kernel(const __grid_con
   extern __shared__ uint8_t smem_raw[];
   const uint32_t sbase = (smem_u32(smem_raw) + 1023u) & ~1023u;
   const uint32_t q_smem = sbase;
-  const uint32_t k_smem = q_smem + C::kQBytes;                       // [C::kStages] K tiles
-  const uint32_t v_smem = k_smem + C::kStages * C::kKBytes;            // [C::kStages] V tiles
+  // tile slots: the output sweep keeps K tiles in the first half and V tiles in the second, (K, V) of a stage
+  // arriving on the stage's barrier; the other sweeps run a K ring over all slots, one barrier per slot
+  const uint32_t k_smem = q_smem + C::kQBytes;                       // [C::kSlots] tiles
+  const uint32_t v_smem = k_smem + C::kStages * C::kKBytes;            // = slot C::kStages
   const uint32_t p_smem = v_smem + C::kStages * C::kKBytes;            // P tile, A-operand layout
   const uint32_t bars = p_smem + kPBytes;
   const uint32_t q_full = bars, q_empty = bars + 8;
-  const uint32_t kv_full = bars + 16;                                 // [C::kStages]
-  const uint32_t kv_empty = kv_full + 8 * C::kStages;                   // [C::kStages]
-  const uint32_t s_full = kv_empty + 8 * C::kStages;                    // [2]
+  const uint32_t kv_full = bars + 16;                                 // [C::kSlots]
+  const uint32_t kv_empty = kv_full + 8 * C::kSlots;                    // [C::kSlots]
+  const uint32_t s_full = kv_empty + 8 * C::kSlots;                     // [2]
   const uint32_t s_empty = s_full + 16;                               // [2]
   const uint32_t p_full = s_empty + 16, p_empty = p_full + 8;
   const uint32_t o_full = p_empty + 8, o_empty = o_full + 8;
@@ -131,8 +136,8 @@ __global__ void __launch_bounds__(kThreadsT, 1) tile_fwd_kernel(const __grid_con
   const uint32_t w_full = drain_fail + 8;                             // [2] a work item has been published
   const uint32_t w_empty = w_full + 16;                               // [2] ... and read by the MMA issuer and every consumer warp
   const uint32_t w_item = w_empty + 16;                               // int32 [2]: tile id, -1 = no more work
-  const uint32_t xchg = bars + C::kBarBytes;                          // float2 [2][TM]
-  static_assert(8 * (2 + 2 * C::kStages + 4 + 4 + 1) + 16 + 8 + 8 + 16 + 40 <= C::kBarBytes, "barrier area");
+  const uint32_t xchg = bars + C::kBarBytes;                          // float2 [2][kConsGroups][TM]
+  static_assert(8 * (2 + 2 * C::kSlots + 4 + 4 + 1) + 16 + 8 + 8 + 16 + 40 <= C::kBarBytes, "barrier area");
 
   const int warp = threadIdx.x >> 5;
   const int lane = threadIdx.x & 31;
@@ -141,25 +146,25 @@ __global__ void __launch_bounds__(kThreadsT, 1) tile_fwd_kernel(const __grid_con
   if (threadIdx.x == 0) {
     mbar_init(q_full, 1);
     mbar_init(q_empty, 1);
-    for (int t = 0; t < C::kStages; ++t) {
+    for (int t = 0; t < C::kSlots; ++t) {
       mbar_init(kv_full + 8 * t, 1);
       mbar_init(kv_empty + 8 * t, 1);
     }
     for (int t = 0; t < 2; ++t) {
       mbar_init(s_full + 8 * t, 1);
-      mbar_init(s_empty + 8 * t, 8);
+      mbar_init(s_empty + 8 * t, kConsWarps);
     }
-    mbar_init(p_full, 8);
+    mbar_init(p_full, kConsWarps);
     mbar_init(p_empty, 1);
     mbar_init(o_full, 1);
-    mbar_init(o_empty, 8);
-    mbar_init(ctl, 8);
-    mbar_init(x_bar, 8);
+    mbar_init(o_empty, kConsWarps);
+    mbar_init(ctl, kConsWarps);
+    mbar_init(x_bar, kConsWarps);
     for (int t = 0; t < 3; ++t) sts_u32(done_word + 4 * t, 1u);
     mbar_init(drain_bar, 1);
     for (int t = 0; t < 2; ++t) {
       mbar_init(w_full + 8 * t, 1);
-      mbar_init(w_empty + 8 * t, 9);   // MMA issuer + eight consumer warps
+      mbar_init(w_empty + 8 * t, 1 + kConsWarps);   // MMA issuer + the consumer warps
     }
     sts_u32(drain_fail, 0u);
     sts_u32(abort_flag, 0u);
@@ -216,8 +221,8 @@ __global__ void __launch_bounds__(kThreadsT, 1) tile_fwd_kernel(const __grid_con
   if (warp == 0) {
     // ------------------------------------------------------------------ TMA producer
     if (lane == 0) {
-      int stage = 0, slot = 0;
-      uint32_t kvphase = 0, qphase = 0, cphase = 0, wphase = 0;
+      int slot = 0;
+      uint32_t kvbits = 0 /* bit x: times barrier pair x has been armed, mod 2 */, qphase = 0, cphase = 0, wphase = 0;
       bool alive = true;
       while (alive) {
         // items are handed out from a shared counter, in the list's order (longest first on causal problems), so
@@ -249,9 +254,12 @@ __global__ void __launch_bounds__(kThreadsT, 1) tile_fwd_kernel(const __grid_con
           const int kind = sweep_kind(s, phase, n_full);
           const bool output = kind == kOutput, smp = kind <= kSampleNewton;
           const int nt = smp ? stiles : tiles;
+          const int ring = output ? C::kStages : C::kSlots;   // every sweep starts at slot 0
+          int stage = 0;
           for (int t = 0; t < nt && alive; ++t) {
-            alive = mbar_wait(kv_empty + 8 * stage, kvphase ^ 1u, abort_flag);
+            alive = mbar_wait(kv_empty + 8 * stage, ((kvbits >> stage) & 1u) ^ 1u, abort_flag);
             if (!alive) break;
+            kvbits ^= 1u << stage;
             mbar_expect_tx(kv_full + 8 * stage, output ? 2 * C::kKBytes : C::kKBytes);
             for (int hf = 0; hf < C::kHalves; ++hf) {
               const uint32_t dst = k_smem + stage * C::kKBytes + hf * (TN * 128);
@@ -263,117 +271,180 @@ __global__ void __launch_bounds__(kThreadsT, 1) tile_fwd_kernel(const __grid_con
                 tma_load_4d(v_smem + stage * C::kKBytes + hf * (TN * 128), &map_v, kv_full + 8 * stage, hf * 64, t * TN, h,
                             b);
             }
-            if (++stage == C::kStages) { stage = 0; kvphase ^= 1u; }
+            if (++stage == ring) stage = 0;
           }
           if (output) break;
         }
       }
       if (!alive) {
         // a wait ran out somewhere in the CTA: the copies this thread armed barriers for must land before shared
-        // memory goes away (stages before `stage`: this round of the ring; the others: the previous round)
+        // memory goes away (the phase armed last has the parity opposite to the arm count's)
         bool ok = mbar_drain(q_full, qphase ^ 1u);
-        for (int st = 0; st < C::kStages; ++st) ok &= mbar_drain(kv_full + 8 * st, st < stage ? kvphase : kvphase ^ 1u);
+        for (int st = 0; st < C::kSlots; ++st) ok &= mbar_drain(kv_full + 8 * st, ((kvbits >> st) & 1u) ^ 1u);
         if (!ok) sts_u32(drain_fail, 1u);
       }
     }
   } else if (warp == 1) {
     // ------------------------------------------------------------------ MMA issuer
-    if (lane == 0) {
+    // The whole warp runs this role's control flow (waits are voted on, values read from shared memory are
+    // broadcast), so that descriptors, addresses and counters are warp-uniform; one elected lane issues the tensor
+    // core instructions.  A single lane inside a divergent branch would compete for issue slots with the consumer
+    // warps of its scheduler for every address calculation of every MMA.
+    {
       constexpr uint32_t id_qk = idesc_qk();
       constexpr uint32_t id_pv = idesc_pv<HD>();
-      const uint32_t q_lo = smem_desc_lo(q_smem), k_lo = smem_desc_lo(k_smem), p_lo = smem_desc_lo(p_smem);
-      const uint32_t v_lo = v_desc_lo(v_smem);
-      int stage = 0;
-      uint32_t kvphase = 0, qphase = 0, cphase = 0, sphase[2] = {0, 0}, pphase = 0, ophase = 0;
+      const uint64_t hi = (uint64_t)kDescHi << 32;
+      const uint64_t q_desc = hi | smem_desc_lo(q_smem), k_desc = hi | smem_desc_lo(k_smem);
+      const uint64_t p_desc = hi | smem_desc_lo(p_smem), v_desc = hi | v_desc_lo(v_smem);
+      uint32_t kvbits = 0 /* bit x: phase of barrier pair x to wait for */, qphase = 0, cphase = 0, sphase[2] = {0, 0},
+               pphase = 0, ophase = 0;
       int sbuf = 0, slot = 0;
       uint32_t wphase = 0;
       bool alive = true;
+      auto wait_all = [&](uint32_t bar, uint32_t parity) -> bool {
+        return __all_sync(0xffffffffu, mbar_wait(bar, parity, abort_flag));
+      };
       while (alive) {
-        alive = mbar_wait(w_full + 8 * slot, wphase, abort_flag);
+        alive = wait_all(w_full + 8 * slot, wphase);
         if (!alive) break;
-        const int id = (int)lds_u32(w_item + 4 * slot);
-        mbar_arrive(w_empty + 8 * slot);
+        const int id = __shfl_sync(0xffffffffu, (int)lds_u32(w_item + 4 * slot), 0);
+        __syncwarp();
+        if (lane == 0) mbar_arrive(w_empty + 8 * slot);
         if (++slot == 2) { slot = 0; wphase ^= 1u; }
         if (id < 0) break;
         const int tile = id % a.tiles_per_head;
         const int tiles = item_tiles(tile), stiles = item_sample_tiles(tile);
         int phase = stiles > 0 ? 0 : 1, n_full = 0;
-        alive = mbar_wait(q_full, qphase, abort_flag);
+        alive = wait_all(q_full, qphase);
         qphase ^= 1u;
         if (!alive) break;
         for (int s = 0; s < kMaxSweeps && alive; ++s) {
           if (s > 0) {
-            alive = mbar_wait(ctl, cphase, abort_flag);
+            alive = wait_all(ctl, cphase);
             cphase ^= 1u;
             if (!alive) break;
           }
-          const int kind = sweep_kind(s, phase, n_full);
+          int kind = sweep_kind(s, phase, n_full);
+          kind = __shfl_sync(0xffffffffu, kind, 0);
+          phase = __shfl_sync(0xffffffffu, phase, 0);
+          n_full = __shfl_sync(0xffffffffu, n_full, 0);
           const bool output = kind == kOutput;
           const int nt = kind <= kSampleNewton ? stiles : tiles;
           if (output) {
             // the previous item's O must have been read before this item's first PV overwrites it
-            alive = mbar_wait(o_empty, ophase ^ 1u, abort_flag);
+            alive = wait_all(o_empty, ophase ^ 1u);
             ophase ^= 1u;
             if (!alive) break;
           }
-          for (int t = 0; t < nt && alive; ++t) {
-            alive = mbar_wait(kv_full + 8 * stage, kvphase, abort_flag);
-            if (alive) alive = mbar_wait(s_empty + 8 * sbuf, sphase[sbuf] ^ 1u, abort_flag);
-            if (!alive) break;
+          const int ring = output ? C::kStages : C::kSlots;   // every sweep starts at slot 0
+          int stage = 0;
+          // S = Q K^T of the next K tile into the accumulator the consumers have handed back
+          auto issue_qk = [&]() -> bool {
+            bool ok = wait_all(kv_full + 8 * stage, (kvbits >> stage) & 1u);
+            if (ok) ok = wait_all(s_empty + 8 * sbuf, sphase[sbuf] ^ 1u);
+            if (!ok) return false;
+            kvbits ^= 1u << stage;
             sphase[sbuf] ^= 1u;
             tc_fence_after();
-            const uint32_t b_lo = k_lo + stage * (C::kKBytes >> 4);
+            const uint64_t b_desc = k_desc + (uint64_t)(stage * (C::kKBytes >> 4));
+            const uint32_t d_tmem = tmem_base + sbuf * TN;
+            if (elect_one()) {
 #pragma unroll
-            for (int kk = 0; kk < HD / 16; ++kk) {
-              const uint32_t a_off = (kk >> 2) * ((TM * 128) >> 4) + (kk & 3) * 2;
-              const uint32_t b_off = (kk >> 2) * ((TN * 128) >> 4) + (kk & 3) * 2;
-              umma_bf16(tmem_base + sbuf * TN, q_lo + a_off, b_lo + b_off, kDescHi, id_qk, kk > 0 ? 1u : 0u);
+              for (int kk = 0; kk < HD / 16; ++kk) {
+                const uint32_t a_off = (kk >> 2) * ((TM * 128) >> 4) + (kk & 3) * 2;
+                const uint32_t b_off = (kk >> 2) * ((TN * 128) >> 4) + (kk & 3) * 2;
+                umma_bf16_desc(d_tmem, q_desc + a_off, b_desc + b_off, id_qk, kk > 0 ? 1u : 0u);
+              }
+              umma_commit(s_full + 8 * sbuf);
             }
-            umma_commit(s_full + 8 * sbuf);
+            __syncwarp();
             sbuf ^= 1;
-            if (!output) {
-              umma_commit(kv_empty + 8 * stage);
-            } else {
+            return true;
+          };
+          if (!output) {
+            for (int t = 0; t < nt && alive; ++t) {
+              alive = issue_qk();
+              if (!alive) break;
+              if (elect_one()) umma_commit(kv_empty + 8 * stage);
+              __syncwarp();
+              if (++stage == ring) stage = 0;
+            }
+          } else {
+            // output sweep: the scores of tile t + 1 are issued before P of tile t is waited for, so that the
+            // consumers never wait for a contraction that could have run while they formed P
+            int vstage = stage;   // stage that holds the V tile of the next P V
+            alive = issue_qk();
+            if (alive && ++stage == ring) stage = 0;
+            for (int t = 0; t < nt && alive; ++t) {
+              if (t + 1 < nt) {
+                alive = issue_qk();
+                if (!alive) break;
+                if (++stage == ring) stage = 0;
+              }
               // O += P V for this tile once the consumers have written P
-              alive = mbar_wait(p_full, pphase, abort_flag);
+              alive = wait_all(p_full, pphase);
               pphase ^= 1u;
               if (!alive) break;
               tc_fence_after();
-              const uint32_t vb_lo = v_lo + stage * (C::kKBytes >> 4);
+              const uint64_t vb_desc = v_desc + (uint64_t)(vstage * (C::kKBytes >> 4));
+              if (elect_one()) {
 #pragma unroll
-              for (int kk = 0; kk < TN / 16; ++kk) {
-                const uint32_t a_off = (kk >> 2) * ((TM * 128) >> 4) + (kk & 3) * 2;   // 64 keys per 128-byte row
-                const uint32_t b_off = kk * ((16 * 128) >> 4);                           // 16 keys = 16 rows of 128 B
-                umma_bf16_ab(tmem_base + C::kTmemO, p_lo + a_off, kDescHi, vb_lo + b_off, kDescHi, id_pv,
-                             (t > 0 || kk > 0) ? 1u : 0u);
+                for (int kk = 0; kk < TN / 16; ++kk) {
+                  const uint32_t a_off = (kk >> 2) * ((TM * 128) >> 4) + (kk & 3) * 2;   // 64 keys per 128-byte row
+                  const uint32_t b_off = kk * ((16 * 128) >> 4);                           // 16 keys = 16 rows of 128 B
+                  umma_bf16_desc(tmem_base + C::kTmemO, p_desc + a_off, vb_desc + b_off, id_pv,
+                                 (t > 0 || kk > 0) ? 1u : 0u);
+                }
+                umma_commit(p_empty);
+                umma_commit(kv_empty + 8 * vstage);
+                if (t == nt - 1) umma_commit(o_full);
               }
-              umma_commit(p_empty);
-              umma_commit(kv_empty + 8 * stage);
-              if (t == tiles - 1) umma_commit(o_full);
+              __syncwarp();
+              if (++vstage == ring) vstage = 0;
             }
-            if (++stage == C::kStages) { stage = 0; kvphase ^= 1u; }
           }
           if (output) break;
         }
-        umma_commit(q_empty);
+        if (elect_one()) umma_commit(q_empty);
+        __syncwarp();
       }
-      if (!alive) {
+      if (!alive && lane == 0) {
         // the tensor core must be done with shared memory and TMEM before they are released
         umma_commit(drain_bar);
         if (!mbar_drain(drain_bar, 0u)) sts_u32(drain_fail, 1u);
       }
     }
   } else {
-    // ------------------------------------------------------------------ consumers: two threads per query row
-    // (warps w and w + 4 share a TMEM lane quadrant; `half` picks the 64 of a tile's 128 columns a thread scans)
+    // ------------------------------------------------------------------ consumers: four threads per query row
+    // (warps w, w + 4, w + 8, w + 12 share a TMEM lane quadrant; `quarter` picks the 32 of a tile's 128 columns a
+    // thread scans).  A thread's share of a tile is one TMEM load; the accumulator goes back to the MMA issuer as
+    // soon as the load has landed in registers.
     const int quad = warp & 3;
-    const int half = (warp - 2) >> 2;
+    const int quarter = (warp - 2) >> 2;
     const int row_local = quad * 32 + lane;
     const uint32_t taddr_row = tmem_base + ((uint32_t)(quad * 32) << 16);
-    uint32_t sphase[2] = {0, 0}, pphase = 0, ophase = 0, cphase = 0, xphase = 0;
+    uint32_t sphase[2] = {0, 0}, pphase = 0, ophase = 0, cphase = 0, xphase = 0, wphase = 0;
     int sbuf = 0, slot = 0;
-    uint32_t wphase = 0;
     bool alive = true;
+    // the four threads of a row swap partial results through shared memory: slot [exchange parity][quarter][row]; all
+    // four then add the same four numbers in the same order
+    auto swap4 = [&](float x0, float x1, float (&r0)[4], float (&r1)[4]) -> bool {
+      const uint32_t base = xchg + xphase * (uint32_t)(kConsGroups * TM * 8);
+      const uint32_t mine = base + (uint32_t)(quarter * TM + row_local) * 8u;
+      sts_u32(mine, __float_as_uint(x0));
+      sts_u32(mine + 4, __float_as_uint(x1));
+      __syncwarp();
+      if (lane == 0) mbar_arrive(x_bar);
+      const bool ok = __all_sync(0xffffffffu, mbar_wait(x_bar, xphase, abort_flag));
+      xphase ^= 1u;
+      if (!ok) return false;
+#pragma unroll
+      for (int g = 0; g < kConsGroups; ++g) {
+        r0[g] = __uint_as_float(lds_u32(base + (uint32_t)(g * TM + row_local) * 8u));
+        r1[g] = __uint_as_float(lds_u32(base + (uint32_t)(g * TM + row_local) * 8u + 4u));
+      }
+      return true;
+    };
     while (alive) {
       alive = __all_sync(0xffffffffu, mbar_wait(w_full + 8 * slot, wphase, abort_flag));
       if (!alive) break;
@@ -421,73 +492,56 @@ __global__ void __launch_bounds__(kThreadsT, 1) tile_fwd_kernel(const __grid_con
           if (!alive) break;
           sphase[sbuf] ^= 1u;
           tc_fence_after();
-          if (output) {
-            // P of the previous tile must have been consumed before its buffer is rewritten
-            alive = __all_sync(0xffffffffu, mbar_wait(p_empty, pphase ^ 1u, abort_flag));
-            pphase ^= 1u;
-            if (!alive) break;
-          }
-#pragma unroll 1
-          for (int c = 2 * half; c < 2 * half + 2; ++c) {
-            float va[32];
-            tmem_ld32(taddr_row + sbuf * TN + c * 32, va);
-            tmem_ld_wait();
-            const int col0 = t * TN + c * 32;
-            if (slope != 0.f) {
-              // bias m_h (key - i) in accumulator units; a sampled column stands for key kTileSampleStride * column
+          float va[32];
+          tmem_ld32(taddr_row + sbuf * TN + quarter * 32, va);
+          tmem_ld_wait();
+          // the scores are in registers: the accumulator can take the tile after next
+          tc_fence_before();
+          __syncwarp();
+          if (lane == 0) mbar_arrive(s_empty + 8 * sbuf);
+          sbuf ^= 1;
+          const int col0 = t * TN + quarter * 32;
+          if (slope != 0.f) {
+            // bias m_h (key - i) in accumulator units; a sampled column stands for key kTileSampleStride * column
 #pragma unroll
-              for (int u = 0; u < 32; ++u) va[u] = fmaf(slope_c, (float)(col0 + u), va[u]) - slope * (float)i;
+            for (int u = 0; u < 32; ++u) va[u] = fmaf(slope_c, (float)(col0 + u), va[u]) - slope * (float)i;
+          }
+          // columns past the row's last visible key only occur in the tiles at the causal diagonal / the tail
+          const bool edge = col0 + 31 > lim_c;
+          if (find_max) {
+            // y_max over the visible keys
+            float m[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
+#pragma unroll
+            for (int u = 0; u < 32; ++u) {
+              const float yv = ra * va[u];
+              m[u & 3] = fmaxf(m[u & 3], (!edge || col0 + u <= lim_c) ? yv : -INFINITY);
             }
-            // columns past the row's last visible key only occur in the tiles at the causal diagonal / the tail
-            const bool edge = col0 + 31 > lim_c;
-            if (find_max) {
-              // y_max over the visible keys
-              float m[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
+            ymax = fmaxf(ymax, fmaxf(fmaxf(m[0], m[1]), fmaxf(m[2], m[3])));
+          } else if (!output) {
+            if (EC != kExpoGeneral && !edge) {
+              // the bulk of a Newton sweep.  What limits it is the ALU pipe (half the FMA pipe's rate), so per
+              // element one clamp there and everything else as FMA-pipe work: y = a acc - tau, its powers fused
+              // into the running sums (four partial sums per total)
+              float p0[4] = {0.f, 0.f, 0.f, 0.f}, p1[4] = {0.f, 0.f, 0.f, 0.f};
 #pragma unroll
               for (int u = 0; u < 32; ++u) {
-                const float yv = ra * va[u];
-                m[u & 3] = fmaxf(m[u & 3], (!edge || col0 + u <= lim_c) ? yv : -INFINITY);
-              }
-              ymax = fmaxf(ymax, fmaxf(fmaxf(m[0], m[1]), fmaxf(m[2], m[3])));
-            } else if (!output) {
-              if (EC != kExpoGeneral && !edge) {
-                // the bulk of a Newton sweep: two columns per instruction (packed fp32 pairs) for y = a acc - tau,
-                // its powers and the two running sums; the clamp at zero has no packed form.  Four lanes of
-                // partial sums per total (two packed accumulators), as below.
-                const f32x2 ra2 = pack2(ra, ra), nt2 = pack2(-tau, -tau);
-                f32x2 q0[2] = {0ull, 0ull}, q1[2] = {0ull, 0ull};
-#pragma unroll
-                for (int u = 0; u < 32; u += 2) {
-                  float ya, yb;
-                  unpack2(fma2(ra2, pack2(va[u], va[u + 1]), nt2), ya, yb);
-                  ya = fmaxf(ya, 0.f);
-                  yb = fmaxf(yb, 0.f);
-                  const f32x2 y2 = pack2(ya, yb);
-                  f32x2 ye2, ye12;
-                  if constexpr (EC == kExpo2) {
-                    ye12 = y2;
-                    ye2 = mul2(y2, y2);
-                  } else if constexpr (EC == kExpo4) {
-                    const f32x2 t2 = mul2(y2, y2);
-                    ye12 = mul2(t2, y2);
-                    ye2 = mul2(t2, t2);
-                  } else {
-                    ye2 = y2;
-                    ye12 = pack2(ya > 0.f ? 1.0f : 0.f, yb > 0.f ? 1.0f : 0.f);
-                  }
-                  q0[(u >> 1) & 1] = add2(q0[(u >> 1) & 1], ye2);
-                  q1[(u >> 1) & 1] = add2(q1[(u >> 1) & 1], ye12);
+                const float m = fmaxf(fmaf(ra, va[u], -tau), 0.f);
+                if constexpr (EC == kExpo2) {
+                  p0[u & 3] = fmaf(m, m, p0[u & 3]);
+                  p1[u & 3] += m;
+                } else if constexpr (EC == kExpo4) {
+                  const float t2 = m * m;
+                  p0[u & 3] = fmaf(t2, t2, p0[u & 3]);
+                  p1[u & 3] = fmaf(t2, m, p1[u & 3]);
+                } else {
+                  p0[u & 3] += m;
+                  p1[u & 3] += positive_indicator(m);
                 }
-                float x0, x1, x2, x3;
-                unpack2(q0[0], x0, x1);
-                unpack2(q0[1], x2, x3);
-                s0 += (x0 + x1) + (x2 + x3);
-                unpack2(q1[0], x0, x1);
-                unpack2(q1[1], x2, x3);
-                s1 += (x0 + x1) + (x2 + x3);
-              } else {
-              // four independent partial sums each: one thread owns the row, so the additions would
-              // otherwise form two serial chains of 128 dependent operations per tile
+              }
+              s0 += (p0[0] + p0[1]) + (p0[2] + p0[3]);
+              s1 += (p1[0] + p1[1]) + (p1[2] + p1[3]);
+            } else {
+              // four independent partial sums each, so that the additions do not form one serial chain
               float p0[4] = {0.f, 0.f, 0.f, 0.f}, p1[4] = {0.f, 0.f, 0.f, 0.f};
 #pragma unroll
               for (int u = 0; u < 32; ++u) {
@@ -500,43 +554,62 @@ __global__ void __launch_bounds__(kThreadsT, 1) tile_fwd_kernel(const __grid_con
               }
               s0 += (p0[0] + p0[1]) + (p0[2] + p0[3]);
               s1 += (p1[0] + p1[1]) + (p1[2] + p1[3]);
-              }
-            } else {
-              // P -> bf16 -> shared memory, K-major with 128-byte swizzle: row r, 16-byte unit u of the
-              // 64-key block sits at r*128 + ((u ^ (r & 7)) * 16)
-              const uint32_t blk = p_smem + (uint32_t)(c >> 1) * (TM * 128) + (uint32_t)row_local * 128u;
+            }
+          } else {
+            // P -> bf16, formed in registers while the tensor core still reads the previous P tile
+            uint32_t w[16];
+            if (EC != kExpoGeneral && !edge) {
+              // as in the Newton sweeps: one ALU-pipe clamp per element, the rest on the FMA pipe (the count of
+              // positive entries too: an indicator formed by a saturating multiply).  Rows past the end of the
+              // sequence have a = 0, tau = 0: all zero.
+              float cnt[4] = {0.f, 0.f, 0.f, 0.f};
 #pragma unroll
-              for (int u4 = 0; u4 < 4; ++u4) {
-                uint32_t w[4];
+              for (int e2 = 0; e2 < 16; ++e2) {
+                float pv[2];
 #pragma unroll
-                for (int e2 = 0; e2 < 4; ++e2) {
-                  float pv[2];
-#pragma unroll
-                  for (int z = 0; z < 2; ++z) {
-                    const int u = u4 * 8 + e2 * 2 + z;
-                    const float yr = fmaf(ra, va[u], -tau);
-                    const bool ok = valid && yr > 0.f && (!edge || col0 + u <= lim);
-                    float ye1;
-                    pow_pair_c<EC>(ok ? yr : 0.f, ok, a.expo, pv[z], ye1);
-                    n_supp += ok ? 1 : 0;
-                  }
-                  const __nv_bfloat162 hh = __floats2bfloat162_rn(pv[0], pv[1]);
-                  w[e2] = *reinterpret_cast<const uint32_t*>(&hh);
+                for (int z = 0; z < 2; ++z) {
+                  const float m = fmaxf(fmaf(ra, va[e2 * 2 + z], -tau), 0.f);
+                  if constexpr (EC == kExpo2) pv[z] = m * m;
+                  else if constexpr (EC == kExpo4) { const float t2 = m * m; pv[z] = t2 * t2; }
+                  else pv[z] = m;
+                  cnt[(e2 * 2 + z) & 3] += positive_indicator(m);
                 }
-                const uint32_t unit = (uint32_t)((c & 1) * 4 + u4);
-                const uint32_t addr = blk + ((unit ^ (uint32_t)(row_local & 7)) << 4);
-                asm volatile("st.shared::cta.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(addr), "r"(w[0]), "r"(w[1]), "r"(w[2]),
-                             "r"(w[3])
-                             : "memory");
+                const __nv_bfloat162 hh = __floats2bfloat162_rn(pv[0], pv[1]);
+                w[e2] = *reinterpret_cast<const uint32_t*>(&hh);
+              }
+              n_supp += (int)((cnt[0] + cnt[1]) + (cnt[2] + cnt[3]));
+            } else {
+#pragma unroll
+              for (int e2 = 0; e2 < 16; ++e2) {
+                float pv[2];
+#pragma unroll
+                for (int z = 0; z < 2; ++z) {
+                  const int u = e2 * 2 + z;
+                  const float yr = fmaf(ra, va[u], -tau);
+                  const bool ok = valid && yr > 0.f && (!edge || col0 + u <= lim);
+                  float ye1;
+                  pow_pair_c<EC>(ok ? yr : 0.f, ok, a.expo, pv[z], ye1);
+                  n_supp += ok ? 1 : 0;
+                }
+                const __nv_bfloat162 hh = __floats2bfloat162_rn(pv[0], pv[1]);
+                w[e2] = *reinterpret_cast<const uint32_t*>(&hh);
               }
             }
-          }
-          // the accumulator has been read
-          tc_fence_before();
-          __syncwarp();
-          if (lane == 0) mbar_arrive(s_empty + 8 * sbuf);
-          sbuf ^= 1;
-          if (output) {
+            // P of the previous tile must have been consumed before its buffer is rewritten
+            alive = __all_sync(0xffffffffu, mbar_wait(p_empty, pphase ^ 1u, abort_flag));
+            pphase ^= 1u;
+            if (!alive) break;
+            // shared memory, K-major with 128-byte swizzle: row r, 16-byte unit u of the 64-key block sits at
+            // r*128 + ((u ^ (r & 7)) * 16)
+            const uint32_t blk = p_smem + (uint32_t)(quarter >> 1) * (TM * 128) + (uint32_t)row_local * 128u;
+#pragma unroll
+            for (int u4 = 0; u4 < 4; ++u4) {
+              const uint32_t unit = (uint32_t)((quarter & 1) * 4 + u4);
+              const uint32_t addr = blk + ((unit ^ (uint32_t)(row_local & 7)) << 4);
+              asm volatile("st.shared::cta.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(addr), "r"(w[4 * u4]),
+                           "r"(w[4 * u4 + 1]), "r"(w[4 * u4 + 2]), "r"(w[4 * u4 + 3])
+                           : "memory");
+            }
             // make the P stores visible to the tensor core (async proxy), then hand the tile over
             asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
             __syncwarp();
@@ -552,8 +625,7 @@ __global__ void __launch_bounds__(kThreadsT, 1) tile_fwd_kernel(const __grid_con
           const bool write = valid && a.row_cnt[grow] == -2;
           __nv_bfloat16* orow =
               reinterpret_cast<__nv_bfloat16*>(a.o) + (size_t)b * a.sb + (size_t)h * a.sh + (size_t)i * a.sn;
-#pragma unroll
-          for (int c = half * (HD / 64); c < (half + 1) * (HD / 64); ++c) {
+          for (int c = quarter; c < HD / 32; c += kConsGroups) {
             float va[32];
             tmem_ld32(taddr_row + C::kTmemO + c * 32, va);
             tmem_ld_wait();
@@ -570,38 +642,34 @@ __global__ void __launch_bounds__(kThreadsT, 1) tile_fwd_kernel(const __grid_con
               }
             }
           }
-          if (write && half == 0) a.tau[grow] = tau;
-          if (write) a.dense_cnt[grow * 2 + half] = n_supp;
+          tc_fence_before();
+          __syncwarp();
+          if (lane == 0) mbar_arrive(o_empty);
+          // the row's support size, as two halves (keys of the tile's first / second 64 columns)
+          float n4[4], unused[4];
+          alive = swap4((float)n_supp, 0.f, n4, unused);
+          if (!alive) break;
+          if (write && quarter == 0) a.tau[grow] = tau;
+          if (write && (quarter & 1) == 0) a.dense_cnt[grow * 2 + (quarter >> 1)] = (int)(n4[quarter] + n4[quarter + 1]);
           if (a.status && threadIdx.x == 64) {
             // diagnostics: full-length sweeps spent (y_max sweep if any, Newton sweeps, output sweep; the sampled
             // sweeps, an eighth as long, are not counted) and tiles processed
             atomicAdd(a.status + ENTMAX_ATTN_STATUS_TILE_SWEEPS, s + 1 - n_smp);
             atomicAdd(a.status + ENTMAX_ATTN_STATUS_TILES, 1);
           }
-          tc_fence_before();
-          __syncwarp();
-          if (lane == 0) mbar_arrive(o_empty);
           break;
         }
-        // ---- between sweeps: the two threads of a row swap their partial results through shared memory (both
-        //      then hold the same totals, added in the same order), Newton update, and the vote "every row of
-        //      the tile has converged"
+        // ---- between sweeps: the threads of a row swap their partial results, Newton update, and the vote "every
+        //      row of the tile has converged"
         {
-          const uint32_t mine = xchg + (uint32_t)(half * TM + row_local) * 8u;
-          const uint32_t theirs = xchg + (uint32_t)((half ^ 1) * TM + row_local) * 8u;
-          sts_u32(mine, __float_as_uint(find_max ? ymax : s0));
-          sts_u32(mine + 4, __float_as_uint(s1));
-          __syncwarp();
-          if (lane == 0) mbar_arrive(x_bar);
-          alive = __all_sync(0xffffffffu, mbar_wait(x_bar, xphase, abort_flag));
-          xphase ^= 1u;
+          float r0[4], r1[4];
+          alive = swap4(find_max ? ymax : s0, s1, r0, r1);
           if (!alive) break;
-          const float o0 = __uint_as_float(lds_u32(theirs)), o1 = __uint_as_float(lds_u32(theirs + 4));
           if (find_max) {
-            ymax = fmaxf(ymax, o0);
+            ymax = fmaxf(fmaxf(r0[0], r0[1]), fmaxf(r0[2], r0[3]));
           } else {
-            s0 = half == 0 ? s0 + o0 : o0 + s0;
-            s1 = half == 0 ? s1 + o1 : o1 + s1;
+            s0 = (r0[0] + r0[1]) + (r0[2] + r0[3]);
+            s1 = (r1[0] + r1[1]) + (r1[2] + r1[3]);
           }
         }
         if (find_max) {
