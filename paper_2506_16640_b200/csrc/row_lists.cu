@@ -87,10 +87,20 @@ __device__ __forceinline__ void atomic_add_vec(float* p, const float (&x)[N]) {
     red_add_v4(p + 4 * c, x[4 * c], x[4 * c + 1], x[4 * c + 2], x[4 * c + 3]);
 }
 
-__device__ __forceinline__ void push_dense_row(int grow, int32_t* fb_count, int32_t* fb_list, int32_t* status) {
-  const int slot = atomicAdd(fb_count, 1);
-  fb_list[slot] = grow;
-  if (status) atomicAdd(status + ENTMAX_ATTN_STATUS_DENSE_ROWS, 1);
+// The rows of a warp that go to the dense path (mask over the warp's lanes, lane l holding row `grow`): one
+// slot reservation and one status update for all of them.  A counter bumped once per row is a chain of
+// dependent L2 atomics on one address; with every row dense that chain, not the rows' work, set the kernel's time.
+__device__ __forceinline__ void push_dense_rows(unsigned mask, int grow, int32_t* fb_count, int32_t* fb_list,
+                                                int32_t* status, int lane) {
+  if (mask == 0u) return;
+  const int leader = __ffs(mask) - 1;
+  int base = 0;
+  if (lane == leader) {
+    base = atomicAdd(fb_count, __popc(mask));
+    if (status) atomicAdd(status + ENTMAX_ATTN_STATUS_DENSE_ROWS, __popc(mask));
+  }
+  base = __shfl_sync(0xffffffffu, base, leader);
+  if ((mask >> lane) & 1u) fb_list[base + __popc(mask & ((1u << lane) - 1u))] = grow;
 }
 
 // Bitonic sort of 32*S (key j, value y) pairs held as S registers per lane (element index = 32*s + lane),
@@ -528,15 +538,21 @@ __device__ __forceinline__ void solve_rows_closed(const Problem& p, const __nv_b
   }
 }
 
-// Forward: a row for the dense-tile path.  Its 128-row Q tile is listed once (tile_flag arbitrates).
-__device__ __forceinline__ void push_dense_tile(const Problem& p, int grow, int32_t* fb_count, int32_t* fb_list,
-                                                int32_t* tile_flag, int32_t* tile_list, int32_t* tile_count,
-                                                int32_t* status) {
-  push_dense_row(grow, fb_count, fb_list, status);
-  const int tiles_per_head = (p.N + 127) / 128;
-  const int bh = grow / p.N, i = grow - bh * p.N;
-  const int id = bh * tiles_per_head + i / 128;
-  if (atomicExch(tile_flag + id, 1) == 0) tile_list[atomicAdd(tile_count, 1)] = id;
+// Forward: the rows of a warp for the dense-tile path (see push_dense_rows).  Their 128-row Q tiles are listed once
+// (tile_flag arbitrates); of the lanes that name the same tile only the lowest asks.
+__device__ __forceinline__ void push_dense_tiles(const Problem& p, unsigned mask, int grow, int32_t* row_cnt,
+                                                 int32_t* fb_count, int32_t* fb_list, int32_t* tile_flag,
+                                                 int32_t* tile_list, int32_t* tile_count, int32_t* status, int lane) {
+  if (mask == 0u) return;
+  push_dense_rows(mask, grow, fb_count, fb_list, status, lane);
+  if ((mask >> lane) & 1u) {
+    row_cnt[grow] = -2;
+    const int tiles_per_head = (p.N + 127) / 128;
+    const int bh = grow / p.N, i = grow - bh * p.N;
+    const int id = bh * tiles_per_head + i / 128;
+    const unsigned same = __match_any_sync(mask, id);
+    if (lane == __ffs(same) - 1 && atomicExch(tile_flag + id, 1) == 0) tile_list[atomicAdd(tile_count, 1)] = id;
+  }
 }
 
 // EC: kExpo2 / kExpo1 select the closed-form solvers, kExpoGeneral the Newton ones (any exponent)
@@ -574,6 +590,13 @@ __global__ void __launch_bounds__(kWarpsPerCta * 32) row_fwd_kernel(Problem p, c
     unsigned m8 = __ballot_sync(0xffffffffu, lane < 16 && cls == 0);
     unsigned m16 = __ballot_sync(0xffffffffu, lane < 16 && cls == 1);
     unsigned mfull = __ballot_sync(0xffffffffu, lane < 16 && cls == 2);
+    {
+      // rows without a usable list go to the dense-tile path, all of the warp's at once
+      const unsigned mdense =
+          __ballot_sync(0xffffffffu, lane < 16 && my_row < total && (mc0 < 0 || mc1 < 0 || mc0 + mc1 == 0));
+      push_dense_tiles(p, mdense, my_row, row_cnt, fb_count, fb_list, tile_flag, tile_list, tile_count, status, lane);
+      mfull &= ~mdense;
+    }
     if constexpr (kClosed) {
       while (m8) {
         const unsigned src = __fns(m8, 0, (lane >> 3) + 1);        // the row of this group of eight lanes
@@ -616,13 +639,6 @@ __global__ void __launch_bounds__(kWarpsPerCta * 32) row_fwd_kernel(Problem p, c
       mfull &= mfull - 1;
       const int grow = 16 * blk + src;
       const int c0 = __shfl_sync(0xffffffffu, mc0, src), c1 = __shfl_sync(0xffffffffu, mc1, src);
-      if (c0 < 0 || c1 < 0 || c0 + c1 == 0) {
-        if (lane == 0) {
-          row_cnt[grow] = -2;
-          push_dense_tile(p, grow, fb_count, fb_list, tile_flag, tile_list, tile_count, status);
-        }
-        continue;
-      }
       const int bh = grow / p.N, i = grow - bh * p.N, b = bh / p.H, h = bh - b * p.H;
       const float a = (p.alpha - 1.0f) * (scale[(size_t)b * p.scale_sb + (size_t)h * p.N + i] * p.sm_scale);
       Entry* list = entries + (size_t)grow * kListCap;
@@ -936,6 +952,12 @@ __global__ void __launch_bounds__(kWarpsPerCta * 32, 4) row_bwd_kernel(
     unsigned m16 = __ballot_sync(0xffffffffu, lane < 16 && cls == 1);
     unsigned m32 = __ballot_sync(0xffffffffu, lane < 16 && cls == 2);
     unsigned mlong = __ballot_sync(0xffffffffu, lane < 16 && cls == 3);
+    {
+      // rows without a usable list go to the dense path, all of the warp's at once
+      const unsigned mdense = __ballot_sync(0xffffffffu, lane < 16 && my_row < total && (mc0 < 0 || mc1 < 0));
+      push_dense_rows(mdense, my_row, fb_count, fb_list, status, lane);
+      mlong &= ~mdense;
+    }
     while (m8) {
       const unsigned src = __fns(m8, 0, (lane >> 3) + 1);          // the row of this group of eight lanes
       const bool active = src < 32u;
@@ -966,10 +988,6 @@ __global__ void __launch_bounds__(kWarpsPerCta * 32, 4) row_bwd_kernel(
       mlong &= mlong - 1;
       const int grow = 16 * blk + src;
       const int c0 = __shfl_sync(0xffffffffu, mc0, src), c1 = __shfl_sync(0xffffffffu, mc1, src);
-      if (c0 < 0 || c1 < 0) {
-        if (lane == 0) push_dense_row(grow, fb_count, fb_list, status);
-        continue;
-      }
       bwd_row_full<D>(p, q, k, v, d_o, scale, tau_in, entries, dq, acc_dk, acc_dv, dc_rows, grow, c0, c1, saved != 0, pitch, lane);
     }
   }

@@ -314,17 +314,25 @@ __global__ void __launch_bounds__(kThreads, 1) sweep_kernel(const __grid_constan
 
   if (warp == 0) {
     // ------------------------------------------------------------- scheduler + TMA producer
-    if (lane == 0) {
+    // (the whole warp runs the control flow, one elected lane issues the copies: see the MMA issuer)
+    {
       int stage = 0, slot = 0;
       uint32_t kphase = 0, qphase = 0 /* bit x: phase of Q tile slot x */, wphase = 0;
       bool alive = true;
+      auto wait_all = [&](uint32_t bar, uint32_t parity) -> bool {
+        return __all_sync(0xffffffffu, mbar_wait(bar, parity, abort_flag));
+      };
       while (alive) {
-        alive = mbar_wait(w_empty + 8 * slot, wphase ^ 1u, abort_flag);
+        alive = wait_all(w_empty + 8 * slot, wphase ^ 1u);
         if (!alive) break;
-        int k = atomicAdd(a.work_counter, 1);
-        if (k >= a.n_items) k = -1;
-        sts_u32(w_item + 4 * slot, (uint32_t)k);
-        mbar_arrive(w_full + 8 * slot);
+        int k = 0;
+        if (lane == 0) {
+          k = atomicAdd(a.work_counter, 1);
+          if (k >= a.n_items) k = -1;
+          sts_u32(w_item + 4 * slot, (uint32_t)k);
+          mbar_arrive(w_full + 8 * slot);
+        }
+        k = __shfl_sync(0xffffffffu, k, 0);
         if (++slot == kSchedSlots) { slot = 0; wphase ^= 1u; }
         if (k < 0) break;
         int bh, item;
@@ -336,39 +344,45 @@ __global__ void __launch_bounds__(kThreads, 1) sweep_kernel(const __grid_constan
           tiles = tx > tiles ? tx : tiles;
         }
         // tiles before tf (and sampled tiles before ts0) lie outside the ALiBi window: t counts from there
-        const int tf = first_tile<kAlibi>(a, k);
+        const int tf = __shfl_sync(0xffffffffu, first_tile<kAlibi>(a, k), 0);
         const int ts_all = sample_tiles(a, item);
         const int ts0 = kAlibi ? min(tf / kSampleStride, ts_all) : 0;
         const int ts = ts_all - ts0;
         tiles -= tf;
         for (int t = 0; t < ts + tiles && alive; ++t) {
-          alive = mbar_wait(k_empty + 8 * stage, kphase ^ 1u, abort_flag);
+          alive = wait_all(k_empty + 8 * stage, kphase ^ 1u);
           if (!alive) break;
-          mbar_expect_tx(k_full + 8 * stage, C::kKBytes);
-          for (int hf = 0; hf < C::kHalves; ++hf) {
-            const uint32_t dst = k_smem + stage * C::kKBytes + hf * (BN * 128);
-            if (t < ts) tma_load_5d(dst, &map_ks, k_full + 8 * stage, hf * 64, 0, (ts0 + t) * BN, h, b);
-            else tma_load_4d(dst, &map_k, k_full + 8 * stage, hf * 64, (tf + t - ts) * BN, h, b);
+          if (elect_one()) {
+            mbar_expect_tx(k_full + 8 * stage, C::kKBytes);
+            for (int hf = 0; hf < C::kHalves; ++hf) {
+              const uint32_t dst = k_smem + stage * C::kKBytes + hf * (BN * 128);
+              if (t < ts) tma_load_5d(dst, &map_ks, k_full + 8 * stage, hf * 64, 0, (ts0 + t) * BN, h, b);
+              else tma_load_4d(dst, &map_k, k_full + 8 * stage, hf * 64, (tf + t - ts) * BN, h, b);
+            }
           }
+          __syncwarp();
           if (++stage == C::kStages) { stage = 0; kphase ^= 1u; }
           if (t == 0) {
             // Q tile slots past the end of the sequence are neither loaded nor used; each slot keeps
             // its own phase bit so that producer and MMA issuer stay in step
             for (int x = 0; x < kQTiles && alive; ++x) {
               if (qtile_tiles(a, item, x) == 0) continue;
-              alive = mbar_wait(q_empty + 8 * x, ((qphase >> x) & 1u) ^ 1u, abort_flag);
+              alive = wait_all(q_empty + 8 * x, ((qphase >> x) & 1u) ^ 1u);
               if (!alive) break;
               qphase ^= 1u << x;
-              mbar_expect_tx(q_full + 8 * x, C::kQBytes);
-              for (int hf = 0; hf < C::kHalves; ++hf)
-                tma_load_4d(q_smem + x * C::kQBytes + hf * (BM * 128), &map_q, q_full + 8 * x, hf * 64,
-                            item * kItemRows + x * BM, h, b);
+              if (elect_one()) {
+                mbar_expect_tx(q_full + 8 * x, C::kQBytes);
+                for (int hf = 0; hf < C::kHalves; ++hf)
+                  tma_load_4d(q_smem + x * C::kQBytes + hf * (BM * 128), &map_q, q_full + 8 * x, hf * 64,
+                              item * kItemRows + x * BM, h, b);
+              }
+              __syncwarp();
             }
           }
         }
       }
-      if (!alive) {
-        // a wait ran out somewhere in the CTA: every copy this thread armed a barrier for must have landed before
+      if (!alive && lane == 0) {
+        // a wait ran out somewhere in the CTA: every copy this warp armed a barrier for must have landed before
         // shared memory goes away.  Stages before `stage` were armed in this round of the ring, the others in the
         // previous one (a barrier that was never armed reports its "previous" phase as complete at once).
         bool ok = true;
@@ -379,17 +393,25 @@ __global__ void __launch_bounds__(kThreads, 1) sweep_kernel(const __grid_constan
     }
   } else if (warp == 1) {
     // ------------------------------------------------------------------ MMA issuer
-    if (lane == 0) {
+    // The whole warp runs the control flow (waits are voted on, what is read from shared memory is broadcast), so
+    // that descriptors, addresses and counters are warp-uniform; one elected lane issues the tensor-core
+    // instructions.
+    {
       constexpr uint32_t idesc = make_idesc();
-      const uint32_t q_lo = smem_desc_lo(q_smem), k_lo = smem_desc_lo(k_smem);
+      const uint64_t hi = (uint64_t)kDescHi << 32;
+      const uint64_t q_desc = hi | smem_desc_lo(q_smem), k_desc = hi | smem_desc_lo(k_smem);
       int stage = 0, slot = 0;
       uint32_t kphase = 0, qphase = 0, wphase = 0, sphase[kQTiles] = {};
       bool alive = true;
+      auto wait_all = [&](uint32_t bar, uint32_t parity) -> bool {
+        return __all_sync(0xffffffffu, mbar_wait(bar, parity, abort_flag));
+      };
       while (alive) {
-        alive = mbar_wait(w_full + 8 * slot, wphase, abort_flag);
+        alive = wait_all(w_full + 8 * slot, wphase);
         if (!alive) break;
-        const int k = (int)lds_u32(w_item + 4 * slot);
-        mbar_arrive(w_empty + 8 * slot);
+        const int k = __shfl_sync(0xffffffffu, (int)lds_u32(w_item + 4 * slot), 0);
+        __syncwarp();
+        if (lane == 0) mbar_arrive(w_empty + 8 * slot);
         if (++slot == kSchedSlots) { slot = 0; wphase ^= 1u; }
         if (k < 0) break;
         int bh, item;
@@ -399,44 +421,48 @@ __global__ void __launch_bounds__(kThreads, 1) sweep_kernel(const __grid_constan
           tx[x] = qtile_tiles(a, item, x);
           tiles = tx[x] > tiles ? tx[x] : tiles;
         }
-        const int tf = first_tile<kAlibi>(a, k);
+        const int tf = __shfl_sync(0xffffffffu, first_tile<kAlibi>(a, k), 0);
         const int ts_all = sample_tiles(a, item);
         const int ts = ts_all - (kAlibi ? min(tf / kSampleStride, ts_all) : 0);
         tiles -= tf;
         for (int x = 0; x < kQTiles; ++x) tx[x] = tx[x] > 0 ? tx[x] - tf : 0;   // every valid Q tile reaches past tf
         for (int t = 0; t < ts + tiles && alive; ++t) {
-          alive = mbar_wait(k_full + 8 * stage, kphase, abort_flag);
+          alive = wait_all(k_full + 8 * stage, kphase);
           if (!alive) break;
-          const uint32_t b_lo = k_lo + stage * (C::kKBytes >> 4);
+          const uint64_t b_desc = k_desc + (uint64_t)(stage * (C::kKBytes >> 4));
 #pragma unroll
           for (int x = 0; x < kQTiles; ++x) {
             // every valid Q tile takes all sampled tiles, then its own share of the real ones
             if (tx[x] == 0 || t >= ts + tx[x] || !alive) continue;
             if (t == 0) {
-              alive = mbar_wait(q_full + 8 * x, (qphase >> x) & 1u, abort_flag);
+              alive = wait_all(q_full + 8 * x, (qphase >> x) & 1u);
               qphase ^= 1u << x;
             }
-            if (alive) alive = mbar_wait(s_empty + 8 * x, sphase[x] ^ 1u, abort_flag);
+            if (alive) alive = wait_all(s_empty + 8 * x, sphase[x] ^ 1u);
             if (!alive) continue;
             sphase[x] ^= 1u;
             tc_fence_after();
-            const uint32_t a_lo = q_lo + x * (C::kQBytes >> 4);
+            const uint64_t a_desc = q_desc + (uint64_t)(x * (C::kQBytes >> 4));
+            if (elect_one()) {
 #pragma unroll
-            for (int kk = 0; kk < HD / 16; ++kk) {
-              // k-step kk: 64-column half kk / 4 (its own swizzled block), 32 bytes per step inside the half
-              const uint32_t a_off = (kk >> 2) * ((BM * 128) >> 4) + (kk & 3) * 2;
-              const uint32_t b_off = (kk >> 2) * ((BN * 128) >> 4) + (kk & 3) * 2;
-              umma_bf16(tmem_base + x * BN, a_lo + a_off, b_lo + b_off, kDescHi, idesc, kk > 0 ? 1u : 0u);
+              for (int kk = 0; kk < HD / 16; ++kk) {
+                // k-step kk: 64-column half kk / 4 (its own swizzled block), 32 bytes per step inside the half
+                const uint32_t a_off = (kk >> 2) * ((BM * 128) >> 4) + (kk & 3) * 2;
+                const uint32_t b_off = (kk >> 2) * ((BN * 128) >> 4) + (kk & 3) * 2;
+                umma_bf16_desc(tmem_base + x * BN, a_desc + a_off, b_desc + b_off, idesc, kk > 0 ? 1u : 0u);
+              }
+              umma_commit(s_full + 8 * x);
+              if (t == ts + tx[x] - 1) umma_commit(q_empty + 8 * x);
             }
-            umma_commit(s_full + 8 * x);
-            if (t == ts + tx[x] - 1) umma_commit(q_empty + 8 * x);
+            __syncwarp();
           }
           if (!alive) break;
-          umma_commit(k_empty + 8 * stage);
+          if (elect_one()) umma_commit(k_empty + 8 * stage);
+          __syncwarp();
           if (++stage == C::kStages) { stage = 0; kphase ^= 1u; }
         }
       }
-      if (!alive) {
+      if (!alive && lane == 0) {
         // the tensor core must be done with shared memory and TMEM before they are released
         umma_commit(drain_bar);
         if (!mbar_drain(drain_bar, 0u)) sts_u32(drain_fail, 1u);

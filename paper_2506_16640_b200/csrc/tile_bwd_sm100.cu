@@ -15,7 +15,7 @@
 // Rows of the tile that are not marked contribute zeros (their P and dS rows are written as zero) and
 // their dQ is not stored: the list kernels have already handled them.
 //
-// CTA: warp 0 TMA producer, warp 1 MMA issuer, warps 2..5 one thread per TMEM lane.  Every wait is
+// CTA: warp 0 TMA producer, warp 1 MMA issuer, warps 2..17 four threads per TMEM lane (32 columns each).  Every wait is
 // bounded (see sm100_ptx.cuh); on expiry the CTA flags the call's status word and leaves.
 #include <cuda.h>
 
@@ -30,7 +30,9 @@ using namespace sm100;
 
 constexpr int TM = 128;            // query rows per item = TMEM lanes
 constexpr int TN = 128;            // keys per K/V tile
-constexpr int kThreadsB = 6 * 32;
+constexpr int kConsGroups = 4;                       // threads per TMEM lane
+constexpr int kConsWarps = 4 * kConsGroups;           // four lane quadrants each
+constexpr int kThreadsB = (2 + kConsWarps) * 32;      // TMA warp, MMA warp, the consumer warps
 constexpr int kTileBytes = TM * TN * 2;   // P or dS tile, bf16
 
 template <int HD>
@@ -129,7 +131,7 @@ __global__ void __launch_bounds__(kThreadsB, 1) tile_bwd_kernel(const __grid_con
   const uint32_t dl_smem = ds_smem + kTileBytes;          // what the bf16 rounding of g dS left over, same layout
   const uint32_t bars = dl_smem + kTileBytes;
   const uint32_t qdo_full = bars, qdo_empty = bars + 8;
-  const uint32_t kv_full = bars + 16, kv_empty = bars + 24;
+  const uint32_t k_full = bars + 16, k_empty = bars + 24;
   const uint32_t sd_full = bars + 32, sd_empty = bars + 40;
   const uint32_t pds_full = bars + 48, pds_empty = bars + 56;
   const uint32_t t_full = bars + 64, t_empty = bars + 72;
@@ -141,6 +143,8 @@ __global__ void __launch_bounds__(kThreadsB, 1) tile_bwd_kernel(const __grid_con
   const uint32_t w_full = bars + 120;         // [2] a work item has been published
   const uint32_t w_empty = bars + 136;        // [2] ... and read by the MMA issuer and every consumer warp
   const uint32_t w_item = bars + 152;         // int32 [2]: tile id, -1 = no more work
+  const uint32_t x_bar = bars + 160;          // the threads of a row have written their partial sums
+  const uint32_t v_full = bars + 168, v_empty = bars + 176;
 
   const int warp = threadIdx.x >> 5;
   const int lane = threadIdx.x & 31;
@@ -149,20 +153,23 @@ __global__ void __launch_bounds__(kThreadsB, 1) tile_bwd_kernel(const __grid_con
   if (threadIdx.x == 0) {
     mbar_init(qdo_full, 1);
     mbar_init(qdo_empty, 1);
-    mbar_init(kv_full, 1);
-    mbar_init(kv_empty, 1);
+    mbar_init(k_full, 1);
+    mbar_init(k_empty, 1);
+    mbar_init(v_full, 1);
+    mbar_init(v_empty, 1);
     mbar_init(sd_full, 1);
-    mbar_init(sd_empty, 4);
-    mbar_init(pds_full, 4);
+    mbar_init(sd_empty, kConsWarps);
+    mbar_init(pds_full, kConsWarps);
     mbar_init(pds_empty, 1);
     mbar_init(t_full, 1);
-    mbar_init(t_empty, 4);
+    mbar_init(t_empty, kConsWarps);
     mbar_init(dq_full, 1);
-    mbar_init(dq_empty, 4);
+    mbar_init(dq_empty, kConsWarps);
+    mbar_init(x_bar, kConsWarps);
     mbar_init(drain_bar, 1);
     for (int t = 0; t < 2; ++t) {
       mbar_init(w_full + 8 * t, 1);
-      mbar_init(w_empty + 8 * t, 5);   // MMA issuer + four consumer warps
+      mbar_init(w_empty + 8 * t, 1 + kConsWarps);   // MMA issuer + the consumer warps
     }
     sts_u32(drain_fail, 0u);
     sts_u32(abort_flag, 0u);
@@ -188,167 +195,242 @@ __global__ void __launch_bounds__(kThreadsB, 1) tile_bwd_kernel(const __grid_con
 
   if (warp == 0) {
     // ------------------------------------------------------------------ TMA producer
-    if (lane == 0) {
-      uint32_t kvphase = 0, qphase = 0, wphase = 0;
+    // (the whole warp runs the control flow, one elected lane issues the copies: see the MMA issuer).  K and V
+    // tiles have barriers of their own: in pass B the V tile is free again once dP has been formed and the K tile
+    // once dQ has taken it, so the next tile's copies run under the dK / dV contractions of this one.
+    {
+      uint32_t kphase = 0, vphase = 0, qphase = 0, wphase = 0;
       int slot = 0;
       bool alive = true;
+      auto wait_all = [&](uint32_t bar, uint32_t parity) -> bool {
+        return __all_sync(0xffffffffu, mbar_wait(bar, parity, abort_flag));
+      };
       while (alive) {
         // items are handed out from a shared counter, in the list's order (longest first on causal problems)
-        alive = mbar_wait(w_empty + 8 * slot, wphase ^ 1u, abort_flag);
+        alive = wait_all(w_empty + 8 * slot, wphase ^ 1u);
         if (!alive) break;
-        const int it = atomicAdd(a.work_counter, 1);
-        const int id = it < n_tiles ? a.tile_list[it] : -1;
-        sts_u32(w_item + 4 * slot, (uint32_t)id);
-        mbar_arrive(w_full + 8 * slot);
+        int id = 0;
+        if (lane == 0) {
+          const int it = atomicAdd(a.work_counter, 1);
+          id = it < n_tiles ? a.tile_list[it] : -1;
+          sts_u32(w_item + 4 * slot, (uint32_t)id);
+          mbar_arrive(w_full + 8 * slot);
+        }
+        id = __shfl_sync(0xffffffffu, id, 0);
         if (++slot == 2) { slot = 0; wphase ^= 1u; }
         if (id < 0) break;
         const int bh = id / a.tiles_per_head, tile = id - bh * a.tiles_per_head;
         const int b = bh / a.H, h = bh - b * a.H;
         const int tiles = item_tiles(tile);
-        alive = mbar_wait(qdo_empty, qphase ^ 1u, abort_flag);
+        alive = wait_all(qdo_empty, qphase ^ 1u);
         if (!alive) break;
         qphase ^= 1u;
-        mbar_expect_tx(qdo_full, 2 * C::kQBytes);
-        for (int hf = 0; hf < C::kHalves; ++hf) {
-          tma_load_4d(q_smem + hf * (TM * 128), &map_q, qdo_full, hf * 64, tile * TM, h, b);
-          tma_load_4d(do_smem + hf * (TM * 128), &map_do, qdo_full, hf * 64, tile * TM, h, b);
-        }
-        for (int t = 0; t < 2 * tiles && alive; ++t) {
-          const int kt = t < tiles ? t : t - tiles;
-          alive = mbar_wait(kv_empty, kvphase ^ 1u, abort_flag);
-          if (!alive) break;
-          kvphase ^= 1u;
-          mbar_expect_tx(kv_full, 2 * C::kQBytes);
+        if (elect_one()) {
+          mbar_expect_tx(qdo_full, 2 * C::kQBytes);
           for (int hf = 0; hf < C::kHalves; ++hf) {
-            tma_load_4d(k_smem + hf * (TN * 128), &map_k, kv_full, hf * 64, kt * TN, h, b);
-            tma_load_4d(v_smem + hf * (TN * 128), &map_v, kv_full, hf * 64, kt * TN, h, b);
+            tma_load_4d(q_smem + hf * (TM * 128), &map_q, qdo_full, hf * 64, tile * TM, h, b);
+            tma_load_4d(do_smem + hf * (TM * 128), &map_do, qdo_full, hf * 64, tile * TM, h, b);
           }
         }
+        __syncwarp();
+        for (int t = 0; t < 2 * tiles && alive; ++t) {
+          const int kt = t < tiles ? t : t - tiles;
+          alive = wait_all(v_empty, vphase ^ 1u);
+          if (!alive) break;
+          vphase ^= 1u;
+          if (elect_one()) {
+            mbar_expect_tx(v_full, C::kQBytes);
+            for (int hf = 0; hf < C::kHalves; ++hf)
+              tma_load_4d(v_smem + hf * (TN * 128), &map_v, v_full, hf * 64, kt * TN, h, b);
+          }
+          __syncwarp();
+          alive = wait_all(k_empty, kphase ^ 1u);
+          if (!alive) break;
+          kphase ^= 1u;
+          if (elect_one()) {
+            mbar_expect_tx(k_full, C::kQBytes);
+            for (int hf = 0; hf < C::kHalves; ++hf)
+              tma_load_4d(k_smem + hf * (TN * 128), &map_k, k_full, hf * 64, kt * TN, h, b);
+          }
+          __syncwarp();
+        }
       }
-      if (!alive) {
-        // a wait ran out somewhere in the CTA: the copies this thread armed barriers for must land before shared
+      if (!alive && lane == 0) {
+        // a wait ran out somewhere in the CTA: the copies this warp armed barriers for must land before shared
         // memory goes away (after n arms a phase word holds n mod 2 and the last armed phase has the other parity)
         bool ok = mbar_drain(qdo_full, qphase ^ 1u);
-        ok &= mbar_drain(kv_full, kvphase ^ 1u);
+        ok &= mbar_drain(k_full, kphase ^ 1u);
+        ok &= mbar_drain(v_full, vphase ^ 1u);
         if (!ok) sts_u32(drain_fail, 1u);
       }
     }
   } else if (warp == 1) {
     // ------------------------------------------------------------------ MMA issuer
-    if (lane == 0) {
+    // The whole warp runs the control flow (waits are voted on, what is read from shared memory is broadcast), so
+    // that descriptors, addresses and counters are warp-uniform; one elected lane issues the tensor-core
+    // instructions.
+    {
       constexpr uint32_t id_kk = idesc_kk();
       constexpr uint32_t id_kn = idesc_kn<HD>();
       constexpr uint32_t id_mn = idesc_mn<HD>();
-      const uint32_t q_lo = smem_desc_lo(q_smem), do_lo = smem_desc_lo(do_smem);
-      const uint32_t k_lo = smem_desc_lo(k_smem), v_lo = smem_desc_lo(v_smem);
-      const uint32_t ds_lo = smem_desc_lo(ds_smem), dl_lo = smem_desc_lo(dl_smem);
-      const uint32_t k_n_lo = mn_desc_lo(k_smem), q_n_lo = mn_desc_lo(q_smem), do_n_lo = mn_desc_lo(do_smem);
-      const uint32_t ds_m_lo = mn_desc_lo(ds_smem), p_m_lo = mn_desc_lo(p_smem);
-      uint32_t kvphase = 0, qphase = 0, sdphase = 0, pdsphase = 0, tphase = 0, dqphase = 0, wphase = 0;
+      const uint64_t hi = (uint64_t)kDescHi << 32;
+      const uint64_t q_d = hi | smem_desc_lo(q_smem), do_d = hi | smem_desc_lo(do_smem);
+      const uint64_t k_d = hi | smem_desc_lo(k_smem), v_d = hi | smem_desc_lo(v_smem);
+      const uint64_t ds_d = hi | smem_desc_lo(ds_smem), dl_d = hi | smem_desc_lo(dl_smem);
+      const uint64_t k_n_d = hi | mn_desc_lo(k_smem), q_n_d = hi | mn_desc_lo(q_smem), do_n_d = hi | mn_desc_lo(do_smem);
+      const uint64_t ds_m_d = hi | mn_desc_lo(ds_smem), p_m_d = hi | mn_desc_lo(p_smem);
+      uint32_t kphase = 0, vphase = 0, qphase = 0, sdphase = 0, pdsphase = 0, tphase = 0, dqphase = 0, wphase = 0;
       int slot = 0;
       bool alive = true;
+      auto wait_all = [&](uint32_t bar, uint32_t parity) -> bool {
+        return __all_sync(0xffffffffu, mbar_wait(bar, parity, abort_flag));
+      };
       while (alive) {
-        alive = mbar_wait(w_full + 8 * slot, wphase, abort_flag);
+        alive = wait_all(w_full + 8 * slot, wphase);
         if (!alive) break;
-        const int id = (int)lds_u32(w_item + 4 * slot);
-        mbar_arrive(w_empty + 8 * slot);
+        const int id = __shfl_sync(0xffffffffu, (int)lds_u32(w_item + 4 * slot), 0);
+        __syncwarp();
+        if (lane == 0) mbar_arrive(w_empty + 8 * slot);
         if (++slot == 2) { slot = 0; wphase ^= 1u; }
         if (id < 0) break;
         const int tile = id % a.tiles_per_head;
         const int tiles = item_tiles(tile);
-        alive = mbar_wait(qdo_full, qphase, abort_flag);
+        alive = wait_all(qdo_full, qphase);
         qphase ^= 1u;
         if (!alive) break;
         for (int t = 0; t < 2 * tiles && alive; ++t) {
           const bool pass_b = t >= tiles;
           if (t == tiles) {
             // the previous item's dQ must have been read before this item's first dQ MMA overwrites it
-            alive = mbar_wait(dq_empty, dqphase ^ 1u, abort_flag);
+            alive = wait_all(dq_empty, dqphase ^ 1u);
             dqphase ^= 1u;
             if (!alive) break;
           }
-          alive = mbar_wait(kv_full, kvphase, abort_flag);
-          kvphase ^= 1u;
-          if (alive) alive = mbar_wait(sd_empty, sdphase ^ 1u, abort_flag);
+          alive = wait_all(k_full, kphase);
+          kphase ^= 1u;
+          if (alive) alive = wait_all(v_full, vphase);
+          vphase ^= 1u;
+          if (alive) alive = wait_all(sd_empty, sdphase ^ 1u);
           if (!alive) break;
           sdphase ^= 1u;
           tc_fence_after();
+          if (elect_one()) {
 #pragma unroll
-          for (int kk = 0; kk < HD / 16; ++kk) {
-            const uint32_t off = (kk >> 2) * ((TM * 128) >> 4) + (kk & 3) * 2;
-            umma_bf16(tmem_base + C::kTmemS, q_lo + off, k_lo + off, kDescHi, id_kk, kk > 0 ? 1u : 0u);
-          }
+            for (int kk = 0; kk < HD / 16; ++kk) {
+              const uint32_t off = (kk >> 2) * ((TM * 128) >> 4) + (kk & 3) * 2;
+              umma_bf16_desc(tmem_base + C::kTmemS, q_d + off, k_d + off, id_kk, kk > 0 ? 1u : 0u);
+            }
 #pragma unroll
-          for (int kk = 0; kk < HD / 16; ++kk) {
-            const uint32_t off = (kk >> 2) * ((TM * 128) >> 4) + (kk & 3) * 2;
-            umma_bf16(tmem_base + C::kTmemDP, do_lo + off, v_lo + off, kDescHi, id_kk, kk > 0 ? 1u : 0u);
+            for (int kk = 0; kk < HD / 16; ++kk) {
+              const uint32_t off = (kk >> 2) * ((TM * 128) >> 4) + (kk & 3) * 2;
+              umma_bf16_desc(tmem_base + C::kTmemDP, do_d + off, v_d + off, id_kk, kk > 0 ? 1u : 0u);
+            }
+            umma_commit(sd_full);
+            umma_commit(v_empty);              // dP has been formed: the V tile is free
+            if (!pass_b) umma_commit(k_empty);
           }
-          umma_commit(sd_full);
-          if (!pass_b) {
-            umma_commit(kv_empty);
-            continue;
-          }
+          __syncwarp();
+          if (!pass_b) continue;
           // P and g dS of this tile are in shared memory
-          alive = mbar_wait(pds_full, pdsphase, abort_flag);
+          alive = wait_all(pds_full, pdsphase);
           pdsphase ^= 1u;
           if (!alive) break;
           tc_fence_after();
+          if (elect_one()) {
 #pragma unroll
-          for (int kk = 0; kk < TN / 16; ++kk) {
-            const uint32_t a_off = (kk >> 2) * ((TM * 128) >> 4) + (kk & 3) * 2;   // 64 keys per 128-byte row
-            const uint32_t b_off = kk * ((16 * 128) >> 4);                           // 16 keys = 16 rows of 128 B
-            umma_bf16_ab(tmem_base + C::kTmemDQ, ds_lo + a_off, kDescHi, k_n_lo + b_off, kDescHi, id_kn,
-                         (t > tiles || kk > 0) ? 1u : 0u);
-          }
-          // the rounding remainder of g dS as a second operand: the rows of dS sum to zero, so when a row's keys are
-          // nearly equal vectors (retrieval: several copies of one key) dQ is what is left after a cancellation, and
-          // the bf16 rounding of dS alone (2^-9 of every term) would be a large part of it
+            for (int kk = 0; kk < TN / 16; ++kk) {
+              const uint32_t a_off = (kk >> 2) * ((TM * 128) >> 4) + (kk & 3) * 2;   // 64 keys per 128-byte row
+              const uint32_t b_off = kk * ((16 * 128) >> 4);                           // 16 keys = 16 rows of 128 B
+              umma_bf16_desc(tmem_base + C::kTmemDQ, ds_d + a_off, k_n_d + b_off, id_kn, (t > tiles || kk > 0) ? 1u : 0u);
+            }
+            // the rounding remainder of g dS as a second operand: the rows of dS sum to zero, so when a row's keys
+            // are nearly equal vectors (retrieval: several copies of one key) dQ is what is left after a
+            // cancellation, and the bf16 rounding of dS alone (2^-9 of every term) would be a large part of it
 #pragma unroll
-          for (int kk = 0; kk < TN / 16; ++kk) {
-            const uint32_t a_off = (kk >> 2) * ((TM * 128) >> 4) + (kk & 3) * 2;
-            const uint32_t b_off = kk * ((16 * 128) >> 4);
-            umma_bf16_ab(tmem_base + C::kTmemDQ, dl_lo + a_off, kDescHi, k_n_lo + b_off, kDescHi, id_kn, 1u);
+            for (int kk = 0; kk < TN / 16; ++kk) {
+              const uint32_t a_off = (kk >> 2) * ((TM * 128) >> 4) + (kk & 3) * 2;
+              const uint32_t b_off = kk * ((16 * 128) >> 4);
+              umma_bf16_desc(tmem_base + C::kTmemDQ, dl_d + a_off, k_n_d + b_off, id_kn, 1u);
+            }
+            umma_commit(k_empty);              // dQ has taken the K tile
           }
-          alive = mbar_wait(t_empty, tphase ^ 1u, abort_flag);
+          __syncwarp();
+          alive = wait_all(t_empty, tphase ^ 1u);
           tphase ^= 1u;
           if (!alive) break;
           tc_fence_after();
+          if (elect_one()) {
 #pragma unroll
-          for (int kk = 0; kk < TM / 16; ++kk) {
-            const uint32_t off = kk * ((16 * 128) >> 4);                             // 16 query rows
-            umma_bf16_ab(tmem_base + C::kTmemT, ds_m_lo + off, kDescHi, q_n_lo + off, kDescHi, id_mn, kk > 0 ? 1u : 0u);
+            for (int kk = 0; kk < TM / 16; ++kk) {
+              const uint32_t off = kk * ((16 * 128) >> 4);                             // 16 query rows
+              umma_bf16_desc(tmem_base + C::kTmemT, ds_m_d + off, q_n_d + off, id_mn, kk > 0 ? 1u : 0u);
+            }
+            umma_commit(t_full);
           }
-          umma_commit(t_full);
-          alive = mbar_wait(t_empty, tphase ^ 1u, abort_flag);
+          __syncwarp();
+          alive = wait_all(t_empty, tphase ^ 1u);
           tphase ^= 1u;
           if (!alive) break;
           tc_fence_after();
+          if (elect_one()) {
 #pragma unroll
-          for (int kk = 0; kk < TM / 16; ++kk) {
-            const uint32_t off = kk * ((16 * 128) >> 4);
-            umma_bf16_ab(tmem_base + C::kTmemT, p_m_lo + off, kDescHi, do_n_lo + off, kDescHi, id_mn, kk > 0 ? 1u : 0u);
+            for (int kk = 0; kk < TM / 16; ++kk) {
+              const uint32_t off = kk * ((16 * 128) >> 4);
+              umma_bf16_desc(tmem_base + C::kTmemT, p_m_d + off, do_n_d + off, id_mn, kk > 0 ? 1u : 0u);
+            }
+            umma_commit(t_full);
+            umma_commit(pds_empty);
+            if (t == 2 * tiles - 1) umma_commit(dq_full);
           }
-          umma_commit(t_full);
-          umma_commit(pds_empty);
-          umma_commit(kv_empty);
-          if (t == 2 * tiles - 1) umma_commit(dq_full);
+          __syncwarp();
         }
-        umma_commit(qdo_empty);
+        if (elect_one()) umma_commit(qdo_empty);
+        __syncwarp();
       }
-      if (!alive) {
+      if (!alive && lane == 0) {
         // the tensor core must be done with shared memory and TMEM before they are released
         umma_commit(drain_bar);
         if (!mbar_drain(drain_bar, 0u)) sts_u32(drain_fail, 1u);
       }
     }
   } else {
-    // ------------------------------------------------------------------ one thread per TMEM lane
+    // ------------------------------------------------------------------ consumers: four threads per TMEM lane
+    // (warps w, w + 4, w + 8, w + 12 share a lane quadrant; `quarter` picks the 32 of a tile's 128 columns -- or
+    // the 32-column chunk of a head-dim-wide accumulator -- a thread works on)
     const int quad = warp & 3;
+    const int quarter = (warp - 2) >> 2;
     const int row_local = quad * 32 + lane;
     const uint32_t taddr_row = tmem_base + ((uint32_t)(quad * 32) << 16);
-    uint32_t sdphase = 0, pdsphase = 0, tphase = 0, dqphase = 0, wphase = 0;
+    uint32_t sdphase = 0, pdsphase = 0, tphase = 0, dqphase = 0, wphase = 0, xphase = 0;
     int slot = 0;
     bool alive = true;
+    // The four threads of a row swap partial sums through shared memory.  The slots live in the remainder tile's
+    // buffer, which is idle whenever a swap happens (between the passes: not yet written; after the item's last
+    // contraction: no longer read); a second round of the barrier keeps a fast warp from rewriting the buffer while
+    // a slow one still reads it.  All four threads add the same four numbers in the same order.
+    auto swap4 = [&](float x0, float x1, float& r0, float& r1) -> bool {
+      const uint32_t mine = dl_smem + (uint32_t)(quarter * TM + row_local) * 8u;
+      sts_u32(mine, __float_as_uint(x0));
+      sts_u32(mine + 4, __float_as_uint(x1));
+      __syncwarp();
+      if (lane == 0) mbar_arrive(x_bar);
+      bool ok = __all_sync(0xffffffffu, mbar_wait(x_bar, xphase, abort_flag));
+      xphase ^= 1u;
+      if (!ok) return false;
+      float a0[kConsGroups], a1[kConsGroups];
+#pragma unroll
+      for (int gq = 0; gq < kConsGroups; ++gq) {
+        a0[gq] = __uint_as_float(lds_u32(dl_smem + (uint32_t)(gq * TM + row_local) * 8u));
+        a1[gq] = __uint_as_float(lds_u32(dl_smem + (uint32_t)(gq * TM + row_local) * 8u + 4u));
+      }
+      r0 = (a0[0] + a0[1]) + (a0[2] + a0[3]);
+      r1 = (a1[0] + a1[1]) + (a1[2] + a1[3]);
+      __syncwarp();
+      if (lane == 0) mbar_arrive(x_bar);
+      ok = __all_sync(0xffffffffu, mbar_wait(x_bar, xphase, abort_flag));
+      xphase ^= 1u;
+      return ok;
+    };
     while (alive) {
       alive = __all_sync(0xffffffffu, mbar_wait(w_full + 8 * slot, wphase, abort_flag));
       if (!alive) break;
@@ -375,7 +457,13 @@ __global__ void __launch_bounds__(kThreadsB, 1) tile_bwd_kernel(const __grid_con
       for (int t = 0; t < 2 * tiles && alive; ++t) {
         const bool pass_b = t >= tiles;
         const int kt = pass_b ? t - tiles : t;
-        if (t == tiles) rho = su > 0.f ? sud / su : 0.f;
+        if (t == tiles) {
+          // rho of the row from the four threads' shares of sum u and sum u dP
+          float su_all, sud_all;
+          alive = swap4(su, sud, su_all, sud_all);
+          if (!alive) break;
+          rho = su_all > 0.f ? sud_all / su_all : 0.f;
+        }
         alive = __all_sync(0xffffffffu, mbar_wait(sd_full, sdphase, abort_flag));
         if (!alive) break;
         sdphase ^= 1u;
@@ -386,24 +474,24 @@ __global__ void __launch_bounds__(kThreadsB, 1) tile_bwd_kernel(const __grid_con
           pdsphase ^= 1u;
           if (!alive) break;
         }
+        // this thread's 32 columns, 16 at a time
 #pragma unroll 1
-        for (int c = 0; c < TN / 32; ++c) {
-          float sa[32], dp[32];
-          tmem_ld32(taddr_row + C::kTmemS + c * 32, sa);
-          tmem_ld32(taddr_row + C::kTmemDP + c * 32, dp);
+        for (int hc = 0; hc < 2; ++hc) {
+          float sa[16], dp[16];
+          tmem_ld16(taddr_row + C::kTmemS + quarter * 32 + hc * 16, sa);
+          tmem_ld16(taddr_row + C::kTmemDP + quarter * 32 + hc * 16, dp);
           tmem_ld_wait();
-          const int col0 = kt * TN + c * 32;
+          const int col0 = kt * TN + quarter * 32 + hc * 16;
           if (slope != 0.f) {
 #pragma unroll
-            for (int u = 0; u < 32; ++u) sa[u] = fmaf(slope, (float)(col0 + u - i), sa[u]);
+            for (int u = 0; u < 16; ++u) sa[u] = fmaf(slope, (float)(col0 + u - i), sa[u]);
           }
-          const bool edge = col0 + 31 > lim;
+          const bool edge = col0 + 15 > lim;
           if (!pass_b) {
-            // four independent partial sums each: one thread owns the row, so the additions would otherwise
-            // form two serial chains of 128 dependent operations per tile
+            // four independent partial sums each, so that the additions do not form one serial chain
             float p0[4] = {0.f, 0.f, 0.f, 0.f}, p1[4] = {0.f, 0.f, 0.f, 0.f};
 #pragma unroll
-            for (int u = 0; u < 32; ++u) {
+            for (int u = 0; u < 16; ++u) {
               const float yr = fmaf(ra, sa[u], -tau);
               const bool ok = yr > 0.f && (!edge || col0 + u <= lim);
               float ye, ye1;
@@ -416,9 +504,9 @@ __global__ void __launch_bounds__(kThreadsB, 1) tile_bwd_kernel(const __grid_con
           } else {
             // P and g dS -> bf16 -> shared memory, K-major with 128-byte swizzle: row r, 16-byte unit u of
             // the 64-key block sits at r*128 + ((u ^ (r & 7)) * 16)
-            const uint32_t blk = (uint32_t)(c >> 1) * (TM * 128) + (uint32_t)row_local * 128u;
+            const uint32_t blk = (uint32_t)(quarter >> 1) * (TM * 128) + (uint32_t)row_local * 128u;
 #pragma unroll
-            for (int u4 = 0; u4 < 4; ++u4) {
+            for (int u4 = 0; u4 < 2; ++u4) {
               float pv[8], dv[8], dl[8];
 #pragma unroll
               for (int z = 0; z < 8; ++z) {
@@ -433,7 +521,7 @@ __global__ void __launch_bounds__(kThreadsB, 1) tile_bwd_kernel(const __grid_con
                 dl[z] = dv[z] - __bfloat162float(__float2bfloat16_rn(dv[z]));
                 dcs[z & 1] = fmaf(ds, sa[u], dcs[z & 1]);
               }
-              const uint32_t unit = (uint32_t)((c & 1) * 4 + u4);
+              const uint32_t unit = (uint32_t)((quarter & 1) * 4 + hc * 2 + u4);
               const uint32_t off = blk + ((unit ^ (uint32_t)(row_local & 7)) << 4);
               asm volatile("st.shared::cta.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(p_smem + off),
                            "r"(pack_bf16(pv[0], pv[1])), "r"(pack_bf16(pv[2], pv[3])), "r"(pack_bf16(pv[4], pv[5])),
@@ -459,7 +547,7 @@ __global__ void __launch_bounds__(kThreadsB, 1) tile_bwd_kernel(const __grid_con
         asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
         __syncwarp();
         if (lane == 0) mbar_arrive(pds_full);
-        // dK then dV of this K tile: TMEM lane = key
+        // dK then dV of this K tile: TMEM lane = key; a thread adds its 32-column chunks of the head dimension
         const int key = kt * TN + row_local;
 #pragma unroll 1
         for (int which = 0; which < 2 && alive; ++which) {
@@ -468,8 +556,7 @@ __global__ void __launch_bounds__(kThreadsB, 1) tile_bwd_kernel(const __grid_con
           tphase ^= 1u;
           tc_fence_after();
           float* dst = (which == 0 ? a.acc_dk : a.acc_dv) + ((size_t)bh * a.N + (key < a.N ? key : 0)) * HD;
-#pragma unroll
-          for (int c = 0; c < HD / 32; ++c) {
+          for (int c = quarter; c < HD / 32; c += kConsGroups) {
             float va[32];
             tmem_ld32(taddr_row + C::kTmemT + c * 32, va);
             tmem_ld_wait();
@@ -492,8 +579,7 @@ __global__ void __launch_bounds__(kThreadsB, 1) tile_bwd_kernel(const __grid_con
       tc_fence_after();
       __nv_bfloat16* dqrow =
           reinterpret_cast<__nv_bfloat16*>(a.dq) + (size_t)b * a.sb + (size_t)h * a.sh + (size_t)i * a.sn;
-#pragma unroll
-      for (int c = 0; c < HD / 32; ++c) {
+      for (int c = quarter; c < HD / 32; c += kConsGroups) {
         float va[32];
         tmem_ld32(taddr_row + C::kTmemDQ + c * 32, va);
         tmem_ld_wait();
@@ -505,12 +591,18 @@ __global__ void __launch_bounds__(kThreadsB, 1) tile_bwd_kernel(const __grid_con
                            pack_bf16(va[u8 * 8 + 4], va[u8 * 8 + 5]), pack_bf16(va[u8 * 8 + 6], va[u8 * 8 + 7]));
         }
       }
-      // dL/dc_i = sum_j dS_ij z_ij with z_ij = sm_scale * (accumulator + bias in accumulator units)
-      if (marked && a.dc_rows) a.dc_rows[grow] = (dcs[0] + dcs[1]) * a.sm_scale;
-      if (a.status && threadIdx.x == 64) atomicAdd(a.status + ENTMAX_ATTN_STATUS_TILES, 1);
       tc_fence_before();
       __syncwarp();
       if (lane == 0) mbar_arrive(dq_empty);
+      // dL/dc_i = sum_j dS_ij z_ij with z_ij = sm_scale * (accumulator + bias in accumulator units); every
+      // contraction of the item has finished (dq_full), so the swap buffer is free
+      if (a.dc_rows) {
+        float dc_all, unused;
+        alive = swap4(dcs[0] + dcs[1], 0.f, dc_all, unused);
+        if (!alive) break;
+        if (marked && quarter == 0) a.dc_rows[grow] = dc_all * a.sm_scale;
+      }
+      if (a.status && threadIdx.x == 64) atomicAdd(a.status + ENTMAX_ATTN_STATUS_TILES, 1);
     }
   }
 

@@ -220,64 +220,81 @@ __global__ void __launch_bounds__(kThreadsT, 1) tile_fwd_kernel(const __grid_con
 
   if (warp == 0) {
     // ------------------------------------------------------------------ TMA producer
-    if (lane == 0) {
+    // (the whole warp runs the control flow, one elected lane issues the copies: see the MMA issuer)
+    {
       int slot = 0;
       uint32_t kvbits = 0 /* bit x: times barrier pair x has been armed, mod 2 */, qphase = 0, cphase = 0, wphase = 0;
       bool alive = true;
+      auto wait_all = [&](uint32_t bar, uint32_t parity) -> bool {
+        return __all_sync(0xffffffffu, mbar_wait(bar, parity, abort_flag));
+      };
       while (alive) {
         // items are handed out from a shared counter, in the list's order (longest first on causal problems), so
         // that the CTAs finish together whatever the Q tiles' lengths and sweep counts are
-        alive = mbar_wait(w_empty + 8 * slot, wphase ^ 1u, abort_flag);
+        alive = wait_all(w_empty + 8 * slot, wphase ^ 1u);
         if (!alive) break;
-        const int it = atomicAdd(a.work_counter, 1);
-        const int id = it < n_tiles ? a.tile_list[it] : -1;
-        sts_u32(w_item + 4 * slot, (uint32_t)id);
-        mbar_arrive(w_full + 8 * slot);
+        int id = 0;
+        if (lane == 0) {
+          const int it = atomicAdd(a.work_counter, 1);
+          id = it < n_tiles ? a.tile_list[it] : -1;
+          sts_u32(w_item + 4 * slot, (uint32_t)id);
+          mbar_arrive(w_full + 8 * slot);
+        }
+        id = __shfl_sync(0xffffffffu, id, 0);
         if (++slot == 2) { slot = 0; wphase ^= 1u; }
         if (id < 0) break;
         const int bh = id / a.tiles_per_head, tile = id - bh * a.tiles_per_head;
         const int b = bh / a.H, h = bh - b * a.H;
         const int tiles = item_tiles(tile), stiles = item_sample_tiles(tile);
         int phase = stiles > 0 ? 0 : 1, n_full = 0;
-        alive = mbar_wait(q_empty, qphase ^ 1u, abort_flag);
+        alive = wait_all(q_empty, qphase ^ 1u);
         if (!alive) break;
-        mbar_expect_tx(q_full, C::kQBytes);
-        for (int hf = 0; hf < C::kHalves; ++hf)
-          tma_load_4d(q_smem + hf * (TM * 128), &map_q, q_full, hf * 64, tile * TM, h, b);
+        if (elect_one()) {
+          mbar_expect_tx(q_full, C::kQBytes);
+          for (int hf = 0; hf < C::kHalves; ++hf)
+            tma_load_4d(q_smem + hf * (TM * 128), &map_q, q_full, hf * 64, tile * TM, h, b);
+        }
+        __syncwarp();
         qphase ^= 1u;
         for (int s = 0; s < kMaxSweeps && alive; ++s) {
           if (s > 0) {
-            alive = mbar_wait(ctl, cphase, abort_flag);
+            alive = wait_all(ctl, cphase);
             cphase ^= 1u;
             if (!alive) break;
           }
-          const int kind = sweep_kind(s, phase, n_full);
+          int kind = sweep_kind(s, phase, n_full);
+          kind = __shfl_sync(0xffffffffu, kind, 0);
+          phase = __shfl_sync(0xffffffffu, phase, 0);
+          n_full = __shfl_sync(0xffffffffu, n_full, 0);
           const bool output = kind == kOutput, smp = kind <= kSampleNewton;
           const int nt = smp ? stiles : tiles;
           const int ring = output ? C::kStages : C::kSlots;   // every sweep starts at slot 0
           int stage = 0;
           for (int t = 0; t < nt && alive; ++t) {
-            alive = mbar_wait(kv_empty + 8 * stage, ((kvbits >> stage) & 1u) ^ 1u, abort_flag);
+            alive = wait_all(kv_empty + 8 * stage, ((kvbits >> stage) & 1u) ^ 1u);
             if (!alive) break;
             kvbits ^= 1u << stage;
-            mbar_expect_tx(kv_full + 8 * stage, output ? 2 * C::kKBytes : C::kKBytes);
-            for (int hf = 0; hf < C::kHalves; ++hf) {
-              const uint32_t dst = k_smem + stage * C::kKBytes + hf * (TN * 128);
-              if (smp) tma_load_5d(dst, &map_ks, kv_full + 8 * stage, hf * 64, 0, t * TN, h, b);
-              else tma_load_4d(dst, &map_k, kv_full + 8 * stage, hf * 64, t * TN, h, b);
+            if (elect_one()) {
+              mbar_expect_tx(kv_full + 8 * stage, output ? 2 * C::kKBytes : C::kKBytes);
+              for (int hf = 0; hf < C::kHalves; ++hf) {
+                const uint32_t dst = k_smem + stage * C::kKBytes + hf * (TN * 128);
+                if (smp) tma_load_5d(dst, &map_ks, kv_full + 8 * stage, hf * 64, 0, t * TN, h, b);
+                else tma_load_4d(dst, &map_k, kv_full + 8 * stage, hf * 64, t * TN, h, b);
+              }
+              if (output) {
+                for (int hf = 0; hf < C::kHalves; ++hf)
+                  tma_load_4d(v_smem + stage * C::kKBytes + hf * (TN * 128), &map_v, kv_full + 8 * stage, hf * 64, t * TN,
+                              h, b);
+              }
             }
-            if (output) {
-              for (int hf = 0; hf < C::kHalves; ++hf)
-                tma_load_4d(v_smem + stage * C::kKBytes + hf * (TN * 128), &map_v, kv_full + 8 * stage, hf * 64, t * TN, h,
-                            b);
-            }
+            __syncwarp();
             if (++stage == ring) stage = 0;
           }
           if (output) break;
         }
       }
-      if (!alive) {
-        // a wait ran out somewhere in the CTA: the copies this thread armed barriers for must land before shared
+      if (!alive && lane == 0) {
+        // a wait ran out somewhere in the CTA: the copies this warp armed barriers for must land before shared
         // memory goes away (the phase armed last has the parity opposite to the arm count's)
         bool ok = mbar_drain(q_full, qphase ^ 1u);
         for (int st = 0; st < C::kSlots; ++st) ok &= mbar_drain(kv_full + 8 * st, ((kvbits >> st) & 1u) ^ 1u);
