@@ -12,8 +12,10 @@
 // kernel); only the rows flagged there are written back.
 //
 // CTA: warp 0 TMA producer, warp 1 MMA issuer, warps 2..17 consumers: TMEM lane = query row, four threads per
-// row (warps w, w + 4, w + 8, w + 12 read the same lane quadrant), each scanning 32 of a K tile's 128 columns; at the
-// end of a sweep the four swap their partial sums through shared memory.  The number of Newton sweeps is decided by the
+// row (warps w, w + 4, w + 8, w + 12 read the same lane quadrant).  The maxima and Newton sweeps walk 256-key tiles
+// (N = 256 MMA groups into two 256-column accumulators, a thread scanning 64 columns), the output sweep 128-key
+// tiles (two 128-column S accumulators beside the O accumulator, a thread scanning 32 columns); at the end of a
+// sweep the four threads of a row swap their partial sums through shared memory.  The number of Newton sweeps is decided by the
 // consumers; they publish "all rows converged" through shared memory and a control mbarrier that every role
 // waits on between sweeps.  Every wait is bounded (see sm100_ptx.cuh); on expiry the CTA flags the call's status
 // word and leaves.
@@ -37,7 +39,8 @@ __device__ __forceinline__ void tma_load_5d(uint32_t dst, const CUtensorMap* map
 }
 
 constexpr int TM = 128;            // query rows per item = TMEM lanes
-constexpr int TN = 128;            // keys per K/V tile
+constexpr int TN = 128;            // keys per K/V tile of the output sweep
+constexpr int TW = 2 * TN;         // keys per K tile of every other sweep (two tile slots, one MMA group of N = 256)
 constexpr int kConsGroups = 4;                       // threads per query row
 constexpr int kConsWarps = 4 * kConsGroups;           // four TMEM lane quadrants each
 constexpr int kThreadsT = (2 + kConsWarps) * 32;      // TMA warp, MMA warp, the consumer warps
@@ -59,7 +62,6 @@ struct TCfg {
   static constexpr int kBarBytes = 384;
   static constexpr int kXchgBytes = 2 * kConsGroups * TM * 8;   // one float2 per (exchange parity, thread of a row, row)
   static constexpr int kStages = HD == 64 ? 4 : 2;   // K/V ring depth of the output sweep: what fits beside Q and P
-  static constexpr int kSlots = 2 * kStages;         // tile slots; the other sweeps load K only and use all of them
   static constexpr int kSmemBytes = kQBytes + kStages * 2 * kKBytes + kPBytes + 1024 + kBarBytes + kXchgBytes;
   static constexpr int kTmemO = 2 * TN;            // first TMEM column of the O accumulator
 };
@@ -86,9 +88,9 @@ struct TileArgsK {
   int tiles_per_head;
 };
 
-// S = Q K^T: A, B bf16 K-major, fp32 accumulate, M = 128, N = TN
-__host__ __device__ constexpr uint32_t idesc_qk() {
-  return (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(TN >> 3) << 17) | ((uint32_t)(TM >> 4) << 24);
+// S = Q K^T: A, B bf16 K-major, fp32 accumulate, M = 128, N = TN (output sweep) or TW (the other sweeps)
+__host__ __device__ constexpr uint32_t idesc_qk(int n) {
+  return (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(n >> 3) << 17) | ((uint32_t)(TM >> 4) << 24);
 }
 // O += P V: A = P K-major, B = V with N (head dim) contiguous ("MN-major", bit 16), M = 128, N = HD
 template <int HD>
@@ -113,16 +115,16 @@ __global__ void __launch_bounds__(kThreadsT, 1) tile_fwd_kernel(const __grid_con
   extern __shared__ uint8_t smem_raw[];
   const uint32_t sbase = (smem_u32(smem_raw) + 1023u) & ~1023u;
   const uint32_t q_smem = sbase;
-  // tile slots: the output sweep keeps K tiles in the first half and V tiles in the second, (K, V) of a stage
-  // arriving on the stage's barrier; the other sweeps run a K ring over all slots, one barrier per slot
-  const uint32_t k_smem = q_smem + C::kQBytes;                       // [C::kSlots] tiles
+  // tile slots: the output sweep keeps 128-key K tiles in the first half and V tiles in the second, (K, V) of a
+  // stage arriving on the stage's barrier; the other sweeps keep one 256-key K tile per stage in two adjacent slots
+  const uint32_t k_smem = q_smem + C::kQBytes;                       // [2 * C::kStages] tile slots
   const uint32_t v_smem = k_smem + C::kStages * C::kKBytes;            // = slot C::kStages
   const uint32_t p_smem = v_smem + C::kStages * C::kKBytes;            // P tile, A-operand layout
   const uint32_t bars = p_smem + kPBytes;
   const uint32_t q_full = bars, q_empty = bars + 8;
-  const uint32_t kv_full = bars + 16;                                 // [C::kSlots]
-  const uint32_t kv_empty = kv_full + 8 * C::kSlots;                    // [C::kSlots]
-  const uint32_t s_full = kv_empty + 8 * C::kSlots;                     // [2]
+  const uint32_t kv_full = bars + 16;                                 // [C::kStages]
+  const uint32_t kv_empty = kv_full + 8 * C::kStages;                   // [C::kStages]
+  const uint32_t s_full = kv_empty + 8 * C::kStages;                    // [2]
   const uint32_t s_empty = s_full + 16;                               // [2]
   const uint32_t p_full = s_empty + 16, p_empty = p_full + 8;
   const uint32_t o_full = p_empty + 8, o_empty = o_full + 8;
@@ -137,7 +139,7 @@ __global__ void __launch_bounds__(kThreadsT, 1) tile_fwd_kernel(const __grid_con
   const uint32_t w_empty = w_full + 16;                               // [2] ... and read by the MMA issuer and every consumer warp
   const uint32_t w_item = w_empty + 16;                               // int32 [2]: tile id, -1 = no more work
   const uint32_t xchg = bars + C::kBarBytes;                          // float2 [2][kConsGroups][TM]
-  static_assert(8 * (2 + 2 * C::kSlots + 4 + 4 + 1) + 16 + 8 + 8 + 16 + 40 <= C::kBarBytes, "barrier area");
+  static_assert(8 * (2 + 2 * C::kStages + 4 + 4 + 1) + 16 + 8 + 8 + 16 + 40 <= C::kBarBytes, "barrier area");
 
   const int warp = threadIdx.x >> 5;
   const int lane = threadIdx.x & 31;
@@ -146,7 +148,7 @@ __global__ void __launch_bounds__(kThreadsT, 1) tile_fwd_kernel(const __grid_con
   if (threadIdx.x == 0) {
     mbar_init(q_full, 1);
     mbar_init(q_empty, 1);
-    for (int t = 0; t < C::kSlots; ++t) {
+    for (int t = 0; t < C::kStages; ++t) {
       mbar_init(kv_full + 8 * t, 1);
       mbar_init(kv_empty + 8 * t, 1);
     }
@@ -267,24 +269,33 @@ __global__ void __launch_bounds__(kThreadsT, 1) tile_fwd_kernel(const __grid_con
           phase = __shfl_sync(0xffffffffu, phase, 0);
           n_full = __shfl_sync(0xffffffffu, n_full, 0);
           const bool output = kind == kOutput, smp = kind <= kSampleNewton;
-          const int nt = smp ? stiles : tiles;
-          const int ring = output ? C::kStages : C::kSlots;   // every sweep starts at slot 0
+          // the output sweep walks 128-key tiles (K and V of a stage on one barrier); every other sweep walks
+          // 256-key tiles, two tile slots to a stage, rows 128.. of a 64-column block right behind rows 0..127
+          const int nt = output ? tiles : ((smp ? stiles : tiles) + 1) / 2;
+          const int ring = C::kStages;   // every sweep starts at stage 0
           int stage = 0;
           for (int t = 0; t < nt && alive; ++t) {
             alive = wait_all(kv_empty + 8 * stage, ((kvbits >> stage) & 1u) ^ 1u);
             if (!alive) break;
             kvbits ^= 1u << stage;
             if (elect_one()) {
-              mbar_expect_tx(kv_full + 8 * stage, output ? 2 * C::kKBytes : C::kKBytes);
-              for (int hf = 0; hf < C::kHalves; ++hf) {
-                const uint32_t dst = k_smem + stage * C::kKBytes + hf * (TN * 128);
-                if (smp) tma_load_5d(dst, &map_ks, kv_full + 8 * stage, hf * 64, 0, t * TN, h, b);
-                else tma_load_4d(dst, &map_k, kv_full + 8 * stage, hf * 64, t * TN, h, b);
-              }
+              mbar_expect_tx(kv_full + 8 * stage, 2 * C::kKBytes);
               if (output) {
-                for (int hf = 0; hf < C::kHalves; ++hf)
+                for (int hf = 0; hf < C::kHalves; ++hf) {
+                  tma_load_4d(k_smem + stage * C::kKBytes + hf * (TN * 128), &map_k, kv_full + 8 * stage, hf * 64, t * TN,
+                              h, b);
                   tma_load_4d(v_smem + stage * C::kKBytes + hf * (TN * 128), &map_v, kv_full + 8 * stage, hf * 64, t * TN,
                               h, b);
+                }
+              } else {
+                for (int hf = 0; hf < C::kHalves; ++hf) {
+#pragma unroll
+                  for (int rh = 0; rh < 2; ++rh) {
+                    const uint32_t dst = k_smem + stage * 2 * C::kKBytes + hf * (TW * 128) + rh * (TN * 128);
+                    if (smp) tma_load_5d(dst, &map_ks, kv_full + 8 * stage, hf * 64, 0, t * TW + rh * TN, h, b);
+                    else tma_load_4d(dst, &map_k, kv_full + 8 * stage, hf * 64, t * TW + rh * TN, h, b);
+                  }
+                }
               }
             }
             __syncwarp();
@@ -297,7 +308,7 @@ __global__ void __launch_bounds__(kThreadsT, 1) tile_fwd_kernel(const __grid_con
         // a wait ran out somewhere in the CTA: the copies this warp armed barriers for must land before shared
         // memory goes away (the phase armed last has the parity opposite to the arm count's)
         bool ok = mbar_drain(q_full, qphase ^ 1u);
-        for (int st = 0; st < C::kSlots; ++st) ok &= mbar_drain(kv_full + 8 * st, ((kvbits >> st) & 1u) ^ 1u);
+        for (int st = 0; st < C::kStages; ++st) ok &= mbar_drain(kv_full + 8 * st, ((kvbits >> st) & 1u) ^ 1u);
         if (!ok) sts_u32(drain_fail, 1u);
       }
     }
@@ -308,7 +319,7 @@ __global__ void __launch_bounds__(kThreadsT, 1) tile_fwd_kernel(const __grid_con
     // core instructions.  A single lane inside a divergent branch would compete for issue slots with the consumer
     // warps of its scheduler for every address calculation of every MMA.
     {
-      constexpr uint32_t id_qk = idesc_qk();
+      constexpr uint32_t id_qk = idesc_qk(TN), id_qk_wide = idesc_qk(TW);
       constexpr uint32_t id_pv = idesc_pv<HD>();
       const uint64_t hi = (uint64_t)kDescHi << 32;
       const uint64_t q_desc = hi | smem_desc_lo(q_smem), k_desc = hi | smem_desc_lo(k_smem);
@@ -335,6 +346,11 @@ __global__ void __launch_bounds__(kThreadsT, 1) tile_fwd_kernel(const __grid_con
         alive = wait_all(q_full, qphase);
         qphase ^= 1u;
         if (!alive) break;
+        // the previous item's O must have been read before this item's MMAs start: its columns are the second wide
+        // accumulator of the sweeps that come first, and the O accumulator of the output sweep
+        alive = wait_all(o_empty, ophase ^ 1u);
+        ophase ^= 1u;
+        if (!alive) break;
         for (int s = 0; s < kMaxSweeps && alive; ++s) {
           if (s > 0) {
             alive = wait_all(ctl, cphase);
@@ -346,16 +362,11 @@ __global__ void __launch_bounds__(kThreadsT, 1) tile_fwd_kernel(const __grid_con
           phase = __shfl_sync(0xffffffffu, phase, 0);
           n_full = __shfl_sync(0xffffffffu, n_full, 0);
           const bool output = kind == kOutput;
-          const int nt = kind <= kSampleNewton ? stiles : tiles;
-          if (output) {
-            // the previous item's O must have been read before this item's first PV overwrites it
-            alive = wait_all(o_empty, ophase ^ 1u);
-            ophase ^= 1u;
-            if (!alive) break;
-          }
-          const int ring = output ? C::kStages : C::kSlots;   // every sweep starts at slot 0
+          const int nt = output ? tiles : ((kind <= kSampleNewton ? stiles : tiles) + 1) / 2;
+          const int ring = C::kStages;   // every sweep starts at stage 0
           int stage = 0;
-          // S = Q K^T of the next K tile into the accumulator the consumers have handed back
+          // S = Q K^T of the next K tile into the accumulator the consumers have handed back: 128 keys and columns
+          // in the output sweep, 256 in the others (which do not use the O accumulator's columns for O)
           auto issue_qk = [&]() -> bool {
             bool ok = wait_all(kv_full + 8 * stage, (kvbits >> stage) & 1u);
             if (ok) ok = wait_all(s_empty + 8 * sbuf, sphase[sbuf] ^ 1u);
@@ -363,16 +374,30 @@ __global__ void __launch_bounds__(kThreadsT, 1) tile_fwd_kernel(const __grid_con
             kvbits ^= 1u << stage;
             sphase[sbuf] ^= 1u;
             tc_fence_after();
-            const uint64_t b_desc = k_desc + (uint64_t)(stage * (C::kKBytes >> 4));
-            const uint32_t d_tmem = tmem_base + sbuf * TN;
-            if (elect_one()) {
+            if (output) {
+              const uint64_t b_desc = k_desc + (uint64_t)(stage * (C::kKBytes >> 4));
+              const uint32_t d_tmem = tmem_base + sbuf * TN;
+              if (elect_one()) {
 #pragma unroll
-              for (int kk = 0; kk < HD / 16; ++kk) {
-                const uint32_t a_off = (kk >> 2) * ((TM * 128) >> 4) + (kk & 3) * 2;
-                const uint32_t b_off = (kk >> 2) * ((TN * 128) >> 4) + (kk & 3) * 2;
-                umma_bf16_desc(d_tmem, q_desc + a_off, b_desc + b_off, id_qk, kk > 0 ? 1u : 0u);
+                for (int kk = 0; kk < HD / 16; ++kk) {
+                  const uint32_t a_off = (kk >> 2) * ((TM * 128) >> 4) + (kk & 3) * 2;
+                  const uint32_t b_off = (kk >> 2) * ((TN * 128) >> 4) + (kk & 3) * 2;
+                  umma_bf16_desc(d_tmem, q_desc + a_off, b_desc + b_off, id_qk, kk > 0 ? 1u : 0u);
+                }
+                umma_commit(s_full + 8 * sbuf);
               }
-              umma_commit(s_full + 8 * sbuf);
+            } else {
+              const uint64_t b_desc = k_desc + (uint64_t)(stage * (2 * C::kKBytes >> 4));
+              const uint32_t d_tmem = tmem_base + sbuf * TW;
+              if (elect_one()) {
+#pragma unroll
+                for (int kk = 0; kk < HD / 16; ++kk) {
+                  const uint32_t a_off = (kk >> 2) * ((TM * 128) >> 4) + (kk & 3) * 2;
+                  const uint32_t b_off = (kk >> 2) * ((TW * 128) >> 4) + (kk & 3) * 2;
+                  umma_bf16_desc(d_tmem, q_desc + a_off, b_desc + b_off, id_qk_wide, kk > 0 ? 1u : 0u);
+                }
+                umma_commit(s_full + 8 * sbuf);
+              }
             }
             __syncwarp();
             sbuf ^= 1;
@@ -495,7 +520,9 @@ __global__ void __launch_bounds__(kThreadsT, 1) tile_fwd_kernel(const __grid_con
         const int kind = sweep_kind(s, phase, n_full);
         const bool output = kind == kOutput, smp = kind <= kSampleNewton;
         const bool find_max = kind == kSampleMax || kind == kFullMax;
-        const int nt = smp ? stiles : tiles;
+        // the output sweep walks 128-key tiles (a thread scans 32 columns); every other sweep walks 256-key tiles
+        // (two accumulators of 256 columns; a thread scans 64 columns as two chunks)
+        const int nt = output ? tiles : ((smp ? stiles : tiles) + 1) / 2;
         const int lim_c = smp ? glim : lim;            // in the column space of this sweep
         const float slope_c = smp ? slope * (float)kTileSampleStride : slope;
         if (kind == kFullNewton && n_full == 1 && stiles > 0) done = !valid;   // the full-row iteration starts here
@@ -504,20 +531,8 @@ __global__ void __launch_bounds__(kThreadsT, 1) tile_fwd_kernel(const __grid_con
         if (warp == 2 && lane == 0) sts_u32(done_word + 4 * ((s + 1) % 3), 1u);
         float s0 = 0.f, s1 = 0.f;
         int n_supp = 0;   // output sweep: keys of this thread's columns with p > 0
-        for (int t = 0; t < nt && alive; ++t) {
-          alive = __all_sync(0xffffffffu, mbar_wait(s_full + 8 * sbuf, sphase[sbuf], abort_flag));
-          if (!alive) break;
-          sphase[sbuf] ^= 1u;
-          tc_fence_after();
-          float va[32];
-          tmem_ld32(taddr_row + sbuf * TN + quarter * 32, va);
-          tmem_ld_wait();
-          // the scores are in registers: the accumulator can take the tile after next
-          tc_fence_before();
-          __syncwarp();
-          if (lane == 0) mbar_arrive(s_empty + 8 * sbuf);
-          sbuf ^= 1;
-          const int col0 = t * TN + quarter * 32;
+        // one 32-column chunk of a maxima or Newton sweep
+        auto scan_chunk = [&](float (&va)[32], const int col0) {
           if (slope != 0.f) {
             // bias m_h (key - i) in accumulator units; a sampled column stands for key kTileSampleStride * column
 #pragma unroll
@@ -534,7 +549,7 @@ __global__ void __launch_bounds__(kThreadsT, 1) tile_fwd_kernel(const __grid_con
               m[u & 3] = fmaxf(m[u & 3], (!edge || col0 + u <= lim_c) ? yv : -INFINITY);
             }
             ymax = fmaxf(ymax, fmaxf(fmaxf(m[0], m[1]), fmaxf(m[2], m[3])));
-          } else if (!output) {
+          } else {
             if (EC != kExpoGeneral && !edge) {
               // the bulk of a Newton sweep.  What limits it is the ALU pipe (half the FMA pipe's rate), so per
               // element one clamp there and everything else as FMA-pipe work: y = a acc - tau, its powers fused
@@ -572,7 +587,44 @@ __global__ void __launch_bounds__(kThreadsT, 1) tile_fwd_kernel(const __grid_con
               s0 += (p0[0] + p0[1]) + (p0[2] + p0[3]);
               s1 += (p1[0] + p1[1]) + (p1[2] + p1[3]);
             }
-          } else {
+          }
+        };
+        for (int t = 0; t < nt && alive; ++t) {
+          alive = __all_sync(0xffffffffu, mbar_wait(s_full + 8 * sbuf, sphase[sbuf], abort_flag));
+          if (!alive) break;
+          sphase[sbuf] ^= 1u;
+          tc_fence_after();
+          if (!output) {
+            float va0[32], va1[32];
+            tmem_ld32(taddr_row + sbuf * TW + quarter * 64, va0);
+            tmem_ld32(taddr_row + sbuf * TW + quarter * 64 + 32, va1);
+            tmem_ld_wait();
+            // the scores are in registers: the accumulator can take the tile after next
+            tc_fence_before();
+            __syncwarp();
+            if (lane == 0) mbar_arrive(s_empty + 8 * sbuf);
+            sbuf ^= 1;
+            scan_chunk(va0, t * TW + quarter * 64);
+            scan_chunk(va1, t * TW + quarter * 64 + 32);
+            continue;
+          }
+          float va[32];
+          tmem_ld32(taddr_row + sbuf * TN + quarter * 32, va);
+          tmem_ld_wait();
+          // the scores are in registers: the accumulator can take the tile after next
+          tc_fence_before();
+          __syncwarp();
+          if (lane == 0) mbar_arrive(s_empty + 8 * sbuf);
+          sbuf ^= 1;
+          const int col0 = t * TN + quarter * 32;
+          if (slope != 0.f) {
+            // bias m_h (key - i) in accumulator units
+#pragma unroll
+            for (int u = 0; u < 32; ++u) va[u] = fmaf(slope, (float)(col0 + u), va[u]) - slope * (float)i;
+          }
+          // columns past the row's last visible key only occur in the tiles at the causal diagonal / the tail
+          const bool edge = col0 + 31 > lim;
+          {
             // P -> bf16, formed in registers while the tensor core still reads the previous P tile
             uint32_t w[16];
             if (EC != kExpoGeneral && !edge) {
