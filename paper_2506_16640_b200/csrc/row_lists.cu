@@ -538,6 +538,23 @@ __device__ __forceinline__ void solve_rows_closed(const Problem& p, const __nv_b
   }
 }
 
+// Rows with more than 32 list entries take the whole warp for a long time each (two-stage solves, gathers over
+// dozens of keys) and come in runs -- the start of every causal head, where all visible keys are candidates.  A
+// warp that met sixteen of them in its block would work through them one after the other while the rest of the grid
+// has finished, so they are only listed here (from the far end of the dense-row list, which has a slot for every
+// row) and a second launch gives each of them a warp of its own.  kLongCounter: their count, in the counter block
+// that starts at fb_count.
+constexpr int kLongCounter = 56;
+__device__ __forceinline__ void push_long_rows(unsigned mask, int grow, int total, int32_t* fb_count, int32_t* fb_list,
+                                               int lane) {
+  if (mask == 0u) return;
+  const int leader = __ffs(mask) - 1;
+  int base = 0;
+  if (lane == leader) base = atomicAdd(fb_count + kLongCounter, __popc(mask));
+  base = __shfl_sync(0xffffffffu, base, leader);
+  if ((mask >> lane) & 1u) fb_list[total - 1 - (base + __popc(mask & ((1u << lane) - 1u)))] = grow;
+}
+
 // Forward: the rows of a warp for the dense-tile path (see push_dense_rows).  Their 128-row Q tiles are listed once
 // (tile_flag arbitrates); of the lanes that name the same tile only the lowest asks.
 __device__ __forceinline__ void push_dense_tiles(const Problem& p, unsigned mask, int grow, int32_t* row_cnt,
@@ -555,6 +572,67 @@ __device__ __forceinline__ void push_dense_tiles(const Problem& p, unsigned mask
   }
 }
 
+// One row with the whole warp: lists of more than 16 entries (closed forms) or any list the sub-warp Newton
+// solver did not take.
+template <int D, int EC>
+__device__ __forceinline__ void row_fwd_whole_warp(const Problem& p, const __nv_bfloat16* __restrict__ v,
+                                                   const float* __restrict__ scale, int32_t* __restrict__ row_cnt,
+                                                   const float* __restrict__ half_thr, Entry* __restrict__ entries,
+                                                   __nv_bfloat16* __restrict__ o, float* __restrict__ tau_out, int grow,
+                                                   int c0, int c1, int lane) {
+  constexpr int PER = D / 32;
+  constexpr bool kClosed = EC == kExpo2 || EC == kExpo1;
+  const int bh = grow / p.N, i = grow - bh * p.N, b = bh / p.H, h = bh - b * p.H;
+  const float a = (p.alpha - 1.0f) * (scale[(size_t)b * p.scale_sb + (size_t)h * p.N + i] * p.sm_scale);
+  Entry* list = entries + (size_t)grow * kListCap;
+  const float2 ht = *reinterpret_cast<const float2*>(half_thr + 2 * (size_t)grow);
+  float bound = fmaxf(ht.x, ht.y);
+  bound -= kKeepMargin * fmaxf(1.0f, fabsf(bound));
+  if constexpr (kClosed) {
+    // up to 32 entries: closed form with the whole warp; more: Newton prefilter first, and the closed form
+    // if what it keeps fits the warp
+    const int n = c0 + c1;
+    if (n <= 32) {
+      solve_rows_closed<D, 32, EC>(p, v, scale, entries, o, tau_out, row_cnt, grow, true, c0, c1, false, lane);
+      return;
+    }
+    const int kept = prefilter_long(p, list, c0, c1, a, lane, bound);
+    if (kept <= 32) {
+      solve_rows_closed<D, 32, EC>(p, v, scale, entries, o, tau_out, row_cnt, grow, true, kept, 0, true, lane);
+      return;
+    }
+    const __nv_bfloat16* vbase = v + (size_t)b * p.sb + (size_t)h * p.sh + lane * PER;
+    __nv_bfloat16* o_row = o + (size_t)b * p.sb + (size_t)h * p.sh + (size_t)i * p.sn + lane * PER;
+    finish_long<D>(p, vbase, list, kept, o_row, tau_out + grow, row_cnt + grow, lane);
+  } else {
+    const __nv_bfloat16* vbase = v + (size_t)b * p.sb + (size_t)h * p.sh + lane * PER;
+    __nv_bfloat16* o_row = o + (size_t)b * p.sb + (size_t)h * p.sh + (size_t)i * p.sn + lane * PER;
+    solve_row_full<D>(p, vbase, list, c0, c1, a, bound, o_row, tau_out + grow, row_cnt + grow, lane);
+  }
+}
+
+// The rows row_fwd_kernel listed as long (push_long_rows): one warp per row.
+template <int D, int EC>
+__global__ void __launch_bounds__(kWarpsPerCta * 32) row_fwd_long_kernel(Problem p, const __nv_bfloat16* __restrict__ v,
+                                                                         const float* __restrict__ scale,
+                                                                         int32_t* __restrict__ row_cnt,
+                                                                         const int32_t* __restrict__ half_cnt,
+                                                                         const float* __restrict__ half_thr,
+                                                                         Entry* __restrict__ entries,
+                                                                         __nv_bfloat16* __restrict__ o,
+                                                                         float* __restrict__ tau_out,
+                                                                         const int32_t* __restrict__ fb_count,
+                                                                         const int32_t* __restrict__ fb_list) {
+  const int lane = threadIdx.x & 31;
+  const int total = p.B * p.H * p.N;
+  const int n_long = fb_count[kLongCounter];
+  for (int t = blockIdx.x * kWarpsPerCta + (threadIdx.x >> 5); t < n_long; t += gridDim.x * kWarpsPerCta) {
+    const int grow = fb_list[total - 1 - t];
+    const int2 c = *reinterpret_cast<const int2*>(half_cnt + 2 * (size_t)grow);
+    row_fwd_whole_warp<D, EC>(p, v, scale, row_cnt, half_thr, entries, o, tau_out, grow, c.x, c.y, lane);
+  }
+}
+
 // EC: kExpo2 / kExpo1 select the closed-form solvers, kExpoGeneral the Newton ones (any exponent)
 template <int D, int EC>
 __global__ void __launch_bounds__(kWarpsPerCta * 32) row_fwd_kernel(Problem p, const __nv_bfloat16* __restrict__ v,
@@ -568,7 +646,6 @@ __global__ void __launch_bounds__(kWarpsPerCta * 32) row_fwd_kernel(Problem p, c
                                                                     int32_t* fb_list, int32_t* tile_flag,
                                                                     int32_t* tile_list, int32_t* tile_count,
                                                                     int32_t* status) {
-  constexpr int PER = D / 32;
   const int lane = threadIdx.x & 31;
   const int total = p.B * p.H * p.N;
   const int blocks = (total + 15) / 16;
@@ -596,6 +673,10 @@ __global__ void __launch_bounds__(kWarpsPerCta * 32) row_fwd_kernel(Problem p, c
           __ballot_sync(0xffffffffu, lane < 16 && my_row < total && (mc0 < 0 || mc1 < 0 || mc0 + mc1 == 0));
       push_dense_tiles(p, mdense, my_row, row_cnt, fb_count, fb_list, tile_flag, tile_list, tile_count, status, lane);
       mfull &= ~mdense;
+      // ... and the ones with long lists to a launch of their own
+      const unsigned mlong = __ballot_sync(0xffffffffu, lane < 16 && ((mfull >> lane) & 1u) && mc0 + mc1 > 32);
+      push_long_rows(mlong, my_row, total, fb_count, fb_list, lane);
+      mfull &= ~mlong;
     }
     if constexpr (kClosed) {
       while (m8) {
@@ -639,33 +720,7 @@ __global__ void __launch_bounds__(kWarpsPerCta * 32) row_fwd_kernel(Problem p, c
       mfull &= mfull - 1;
       const int grow = 16 * blk + src;
       const int c0 = __shfl_sync(0xffffffffu, mc0, src), c1 = __shfl_sync(0xffffffffu, mc1, src);
-      const int bh = grow / p.N, i = grow - bh * p.N, b = bh / p.H, h = bh - b * p.H;
-      const float a = (p.alpha - 1.0f) * (scale[(size_t)b * p.scale_sb + (size_t)h * p.N + i] * p.sm_scale);
-      Entry* list = entries + (size_t)grow * kListCap;
-      const float2 ht = *reinterpret_cast<const float2*>(half_thr + 2 * (size_t)grow);
-      float bound = fmaxf(ht.x, ht.y);
-      bound -= kKeepMargin * fmaxf(1.0f, fabsf(bound));
-      if constexpr (kClosed) {
-        // up to 32 entries: closed form with the whole warp; more: Newton prefilter first, and the closed form
-        // if what it keeps fits the warp
-        const int n = c0 + c1;
-        if (n <= 32) {
-          solve_rows_closed<D, 32, EC>(p, v, scale, entries, o, tau_out, row_cnt, grow, true, c0, c1, false, lane);
-          continue;
-        }
-        const int kept = prefilter_long(p, list, c0, c1, a, lane, bound);
-        if (kept <= 32) {
-          solve_rows_closed<D, 32, EC>(p, v, scale, entries, o, tau_out, row_cnt, grow, true, kept, 0, true, lane);
-          continue;
-        }
-        const __nv_bfloat16* vbase = v + (size_t)b * p.sb + (size_t)h * p.sh + lane * PER;
-        __nv_bfloat16* o_row = o + (size_t)b * p.sb + (size_t)h * p.sh + (size_t)i * p.sn + lane * PER;
-        finish_long<D>(p, vbase, list, kept, o_row, tau_out + grow, row_cnt + grow, lane);
-      } else {
-        const __nv_bfloat16* vbase = v + (size_t)b * p.sb + (size_t)h * p.sh + lane * PER;
-        __nv_bfloat16* o_row = o + (size_t)b * p.sb + (size_t)h * p.sh + (size_t)i * p.sn + lane * PER;
-        solve_row_full<D>(p, vbase, list, c0, c1, a, bound, o_row, tau_out + grow, row_cnt + grow, lane);
-      }
+      row_fwd_whole_warp<D, EC>(p, v, scale, row_cnt, half_thr, entries, o, tau_out, grow, c0, c1, lane);
     }
   }
 }
@@ -957,6 +1012,9 @@ __global__ void __launch_bounds__(kWarpsPerCta * 32, 4) row_bwd_kernel(
       const unsigned mdense = __ballot_sync(0xffffffffu, lane < 16 && my_row < total && (mc0 < 0 || mc1 < 0));
       push_dense_rows(mdense, my_row, fb_count, fb_list, status, lane);
       mlong &= ~mdense;
+      // ... and the ones with long lists to a launch of their own (see push_long_rows)
+      push_long_rows(mlong, my_row, total, fb_count, fb_list, lane);
+      mlong = 0u;
     }
     while (m8) {
       const unsigned src = __fns(m8, 0, (lane >> 3) + 1);          // the row of this group of eight lanes
@@ -983,13 +1041,33 @@ __global__ void __launch_bounds__(kWarpsPerCta * 32, 4) row_bwd_kernel(
       bwd_rows_sub<D, 32>(p, q, k, v, d_o, scale, tau_in, entries, dq, acc_dk, acc_dv, dc_rows, 16 * blk + src, true, c0, c1,
                           saved != 0, pitch, lane);
     }
-    while (mlong) {
-      const int src = __ffs(mlong) - 1;
-      mlong &= mlong - 1;
-      const int grow = 16 * blk + src;
-      const int c0 = __shfl_sync(0xffffffffu, mc0, src), c1 = __shfl_sync(0xffffffffu, mc1, src);
-      bwd_row_full<D>(p, q, k, v, d_o, scale, tau_in, entries, dq, acc_dk, acc_dv, dc_rows, grow, c0, c1, saved != 0, pitch, lane);
+  }
+}
+
+// The rows row_bwd_kernel listed as long (push_long_rows): one warp per row.
+template <int D>
+__global__ void __launch_bounds__(kWarpsPerCta * 32, 4) row_bwd_long_kernel(
+    Problem p, const __nv_bfloat16* __restrict__ q, const __nv_bfloat16* __restrict__ k,
+    const __nv_bfloat16* __restrict__ v, const __nv_bfloat16* __restrict__ d_o, const float* __restrict__ scale,
+    const float* __restrict__ tau_in, const int32_t* __restrict__ half_cnt, const Entry* __restrict__ entries,
+    __nv_bfloat16* __restrict__ dq, float* __restrict__ acc_dk, float* __restrict__ acc_dv,
+    float* __restrict__ dc_rows, const int32_t* __restrict__ fb_count, const int32_t* __restrict__ fb_list, int saved,
+    int pitch) {
+  const int lane = threadIdx.x & 31;
+  const int total = p.B * p.H * p.N;
+  const int n_long = fb_count[kLongCounter];
+  for (int t = blockIdx.x * kWarpsPerCta + (threadIdx.x >> 5); t < n_long; t += gridDim.x * kWarpsPerCta) {
+    const int grow = fb_list[total - 1 - t];
+    int c0, c1 = 0;
+    if (saved) {
+      c0 = half_cnt[grow];
+    } else {
+      const int2 c = *reinterpret_cast<const int2*>(half_cnt + 2 * (size_t)grow);
+      c0 = c.x;
+      c1 = c.y;
     }
+    bwd_row_full<D>(p, q, k, v, d_o, scale, tau_in, entries, dq, acc_dk, acc_dv, dc_rows, grow, c0, c1, saved != 0, pitch,
+                    lane);
   }
 }
 
@@ -1037,6 +1115,24 @@ cudaError_t launch_row_fwd(const Problem& p, const void* v, const float* scale, 
     else ENTMAX_ROW_FWD(128, kExpoGeneral);
   }
 #undef ENTMAX_ROW_FWD
+  cudaError_t err = cudaGetLastError();
+  if (err != cudaSuccess) return err;
+  // the rows it listed as long, one warp each (normally none or a few: the launch then ends at once)
+  const int lgrid = grid < 148 * 4 ? grid : 148 * 4;
+#define ENTMAX_ROW_FWD_LONG(D, EC)                                                                                     \
+  row_fwd_long_kernel<D, EC><<<lgrid, kWarpsPerCta * 32, 0, stream>>>(p, (const __nv_bfloat16*)v, scale, row_cnt,       \
+                                                                      half_cnt, half_thr, entries, (__nv_bfloat16*)o,  \
+                                                                      tau, fb_count, fb_list)
+  if (p.D == 64) {
+    if (p.expo_class == kExpo2) ENTMAX_ROW_FWD_LONG(64, kExpo2);
+    else if (p.expo_class == kExpo1) ENTMAX_ROW_FWD_LONG(64, kExpo1);
+    else ENTMAX_ROW_FWD_LONG(64, kExpoGeneral);
+  } else {
+    if (p.expo_class == kExpo2) ENTMAX_ROW_FWD_LONG(128, kExpo2);
+    else if (p.expo_class == kExpo1) ENTMAX_ROW_FWD_LONG(128, kExpo1);
+    else ENTMAX_ROW_FWD_LONG(128, kExpoGeneral);
+  }
+#undef ENTMAX_ROW_FWD_LONG
   return cudaGetLastError();
 }
 
@@ -1062,6 +1158,18 @@ cudaError_t launch_row_bwd(const Problem& p, const void* q, const void* k, const
     row_bwd_kernel<128><<<grid, kWarpsPerCta * 32, 0, stream>>>(
         p, (const __nv_bfloat16*)q, (const __nv_bfloat16*)k, (const __nv_bfloat16*)v, (const __nv_bfloat16*)d_o, scale,
         tau, half_cnt, entries, (__nv_bfloat16*)dq, acc_dk, acc_dv, dc_rows, fb_count, fb_list, status, saved, pitch);
+  cudaError_t err = cudaGetLastError();
+  if (err != cudaSuccess) return err;
+  // the rows it listed as long, one warp each (normally none or a few: the launch then ends at once)
+  const int lgrid = grid < 148 * 4 ? grid : 148 * 4;
+  if (p.D == 64)
+    row_bwd_long_kernel<64><<<lgrid, kWarpsPerCta * 32, 0, stream>>>(
+        p, (const __nv_bfloat16*)q, (const __nv_bfloat16*)k, (const __nv_bfloat16*)v, (const __nv_bfloat16*)d_o, scale,
+        tau, half_cnt, entries, (__nv_bfloat16*)dq, acc_dk, acc_dv, dc_rows, fb_count, fb_list, saved, pitch);
+  else
+    row_bwd_long_kernel<128><<<lgrid, kWarpsPerCta * 32, 0, stream>>>(
+        p, (const __nv_bfloat16*)q, (const __nv_bfloat16*)k, (const __nv_bfloat16*)v, (const __nv_bfloat16*)d_o, scale,
+        tau, half_cnt, entries, (__nv_bfloat16*)dq, acc_dk, acc_dv, dc_rows, fb_count, fb_list, saved, pitch);
   return cudaGetLastError();
 }
 
