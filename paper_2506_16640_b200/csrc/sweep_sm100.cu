@@ -185,8 +185,29 @@ __device__ __noinline__ RowState shrink_lists(RowState r, Entry* list, float a, 
         e[s].j = 0;
         if (idx < c) e[s] = l[idx];
       }
+      // A sure case first.  With y_max the largest of the c listed keys, sum_j (y_max - tau)^e >= sum_j [y_j - tau]_+^e
+      // = 1 at the list's own threshold tau*, so tau* <= y_max - c^(-1/e): every listed key above that is in the
+      // list's support.  If those alone are more than a half-list may keep, the row goes to the dense path without a
+      // solve (rows of flat logits, which would otherwise each pay a full Newton solve just to be handed over).
+      bool sure_dense = false;
+      {
+        float ym = -INFINITY;
+#pragma unroll
+        for (int s = 0; s < kSlots; ++s) ym = fmaxf(ym, e[s].y);
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) ym = fmaxf(ym, __shfl_xor_sync(0xffffffffu, ym, o));
+        const float width = expo_class == kExpo2 ? rsqrtf((float)c) : expo_class == kExpo1 ? 1.0f / (float)c
+                                                                                           : powf((float)c, -1.0f / expo);
+        const float cut = ym - width * inv_aa;
+        int sure = 0;
+#pragma unroll
+        for (int s = 0; s < kSlots; ++s) sure += __popc(__ballot_sync(0xffffffffu, e[s].y > cut));
+        sure_dense = sure > kHalfKeep;
+      }
       float tau = th * aa;
-      if (expo >= 1.0f) {
+      if (sure_dense) {
+        // nothing to solve
+      } else if (expo >= 1.0f) {
         for (int it = 0; it < 8; ++it) {
           float s0 = 0.f, s1 = 0.f;
 #pragma unroll
@@ -227,14 +248,16 @@ __device__ __noinline__ RowState shrink_lists(RowState r, Entry* list, float a, 
       new_thr = fmaxf(th, (tau - 4e-6f * fmaxf(1.0f, fabsf(tau))) * inv_aa);
       __syncwarp();
       kept = 0;
+      if (!sure_dense) {
 #pragma unroll
-      for (int s = 0; s < kSlots; ++s) {
-        const bool keep = e[s].y > new_thr;
-        const unsigned m = __ballot_sync(0xffffffffu, keep);
-        if (keep) l[kept + __popc(m & ((1u << lane) - 1u))] = e[s];
-        kept += __popc(m);
+        for (int s = 0; s < kSlots; ++s) {
+          const bool keep = e[s].y > new_thr;
+          const unsigned m = __ballot_sync(0xffffffffu, keep);
+          if (keep) l[kept + __popc(m & ((1u << lane) - 1u))] = e[s];
+          kept += __popc(m);
+        }
       }
-      if (kept > kHalfKeep) {
+      if (kept > kHalfKeep || sure_dense) {
         kept = -1;
         new_thr = INFINITY;
       }
