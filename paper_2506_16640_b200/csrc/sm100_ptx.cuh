@@ -240,6 +240,9 @@ __device__ __forceinline__ float warp_sum(float x) {
 // Defined in tile_fwd_sm100.cu.
 cudaError_t make_tile_map(CUtensorMap* map, const void* base, int D, int N, int H, int B, int64_t sn, int64_t sh,
                           int64_t sb, int box_rows = 128);
+// A contiguous fp32 [BH, N, D] accumulator as a 3-D map (D, N, BH); box = 32 columns (one 128-byte swizzle row) by 128
+// rows, 128-byte swizzle: the target of bulk reductions from a staging tile in shared memory.
+cudaError_t make_acc_map(CUtensorMap* map, const float* base, int D, int N, int BH);
 // The same tensor as a 5-D map (D, key % stride, key / stride, H, B): a box of box_rows rows along "key / stride" at
 // phase 0 is every stride-th key.  Keys past stride * (N / stride) are not part of the view; N >= stride is required.
 cudaError_t make_sampled_tile_map(CUtensorMap* map, const void* base, int D, int N, int H, int B, int64_t sn, int64_t sh,

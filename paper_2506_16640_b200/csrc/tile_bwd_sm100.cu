@@ -10,8 +10,8 @@
 //   pass B   S and dP again; the row threads write P and g dS (bf16) to shared memory; then
 //            dQ += (g dS) K     (A = g dS K-major, B = K tile with the head dim contiguous)   kept in TMEM,
 //            dK_t = (g dS)^T Q  (A = the same shared tile read M-major, B = Q tile, head dim contiguous)
-//            dV_t = P^T dO      (likewise), both through one TMEM buffer, added to the fp32 dK / dV
-//            accumulators in global memory (vector reductions) by the thread that owns the key.
+//            dV_t = P^T dO      (likewise), both through one TMEM buffer and a staging tile in shared memory, added
+//            to the fp32 dK / dV accumulators in global memory by bulk tensor reductions.
 // Rows of the tile that are not marked contribute zeros (their P and dS rows are written as zero) and
 // their dQ is not stored: the list kernels have already handled them.
 //
@@ -118,6 +118,8 @@ __global__ void __launch_bounds__(kThreadsB, 1) tile_bwd_kernel(const __grid_con
                                                                const __grid_constant__ CUtensorMap map_k,
                                                                const __grid_constant__ CUtensorMap map_v,
                                                                const __grid_constant__ CUtensorMap map_do,
+                                                               const __grid_constant__ CUtensorMap map_dk,
+                                                               const __grid_constant__ CUtensorMap map_dv,
                                                                const TileBwdArgs a) {
   using C = BCfg<HD>;
   extern __shared__ uint8_t smem_raw[];
@@ -547,28 +549,59 @@ __global__ void __launch_bounds__(kThreadsB, 1) tile_bwd_kernel(const __grid_con
         asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
         __syncwarp();
         if (lane == 0) mbar_arrive(pds_full);
-        // dK then dV of this K tile: TMEM lane = key; a thread adds its 32-column chunks of the head dimension
-        const int key = kt * TN + row_local;
+        // dK then dV of this K tile: TMEM lane = key.  The tile is added to the fp32 accumulators in global memory by
+        // bulk reductions from shared memory (the copy engine's, not 128 x 32 vector reductions per thread group, which
+        // held the threads -- and through them the accumulator -- for thousands of cycles per tile): a thread copies its
+        // 32-column chunk of the head dimension into a staging tile, [chunk][128 keys][128 bytes] with the 128-byte
+        // swizzle of a tensor-map box, in the g dS and remainder buffers (free: the contractions that read them
+        // precede the one whose result is being read); one thread then issues a reduction per chunk.  Keys past the
+        // end of the sequence are outside the map and not written.
+        const int key0 = kt * TN;
 #pragma unroll 1
         for (int which = 0; which < 2 && alive; ++which) {
           alive = __all_sync(0xffffffffu, mbar_wait(t_full, tphase, abort_flag));
           if (!alive) break;
           tphase ^= 1u;
           tc_fence_after();
-          float* dst = (which == 0 ? a.acc_dk : a.acc_dv) + ((size_t)bh * a.N + (key < a.N ? key : 0)) * HD;
-          for (int c = quarter; c < HD / 32; c += kConsGroups) {
+          if (quarter < HD / 32) {
             float va[32];
-            tmem_ld32(taddr_row + C::kTmemT + c * 32, va);
+            tmem_ld32(taddr_row + C::kTmemT + quarter * 32, va);
             tmem_ld_wait();
-            if (key < a.N) {
+            const uint32_t dst = ds_smem + (uint32_t)quarter * (TM * 128) + (uint32_t)row_local * 128u;
 #pragma unroll
-              for (int m = 0; m < 8; ++m)
-                red_add_v4(dst + c * 32 + 4 * m, va[4 * m], va[4 * m + 1], va[4 * m + 2], va[4 * m + 3]);
-            }
+            for (int u = 0; u < 8; ++u)
+              asm volatile("st.shared::cta.v4.f32 [%0], {%1, %2, %3, %4};" ::"r"(dst + (((uint32_t)u ^ (uint32_t)(row_local & 7)) << 4)),
+                           "f"(va[4 * u]), "f"(va[4 * u + 1]), "f"(va[4 * u + 2]), "f"(va[4 * u + 3])
+                           : "memory");
           }
+          // the result is out of TMEM: the next contraction may overwrite it
           tc_fence_before();
+          asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
           __syncwarp();
-          if (lane == 0) mbar_arrive(t_empty);
+          if (lane == 0) {
+            mbar_arrive(t_empty);
+            mbar_arrive(x_bar);
+          }
+          alive = __all_sync(0xffffffffu, mbar_wait(x_bar, xphase, abort_flag));
+          xphase ^= 1u;
+          if (!alive) break;
+          if (threadIdx.x == 64) {
+            const CUtensorMap* map = which == 0 ? &map_dk : &map_dv;
+#pragma unroll
+            for (int c = 0; c < HD / 32; ++c)
+              asm volatile(
+                  "cp.reduce.async.bulk.tensor.3d.global.shared::cta.add.tile.bulk_group [%0, {%2, %3, %4}], [%1];" ::"l"(
+                      reinterpret_cast<uint64_t>(map)),
+                  "r"(ds_smem + (uint32_t)c * (TM * 128)), "r"(c * 32), "r"(key0), "r"(bh)
+                  : "memory");
+            asm volatile("cp.async.bulk.commit_group;" ::: "memory");
+            // the staging tile may be rewritten once the reductions have read it
+            asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory");
+          }
+          __syncwarp();
+          if (lane == 0) mbar_arrive(x_bar);
+          alive = __all_sync(0xffffffffu, mbar_wait(x_bar, xphase, abort_flag));
+          xphase ^= 1u;
         }
       }
       if (!alive) break;
@@ -604,6 +637,8 @@ __global__ void __launch_bounds__(kThreadsB, 1) tile_bwd_kernel(const __grid_con
       }
       if (a.status && threadIdx.x == 64) atomicAdd(a.status + ENTMAX_ATTN_STATUS_TILES, 1);
     }
+    // every bulk reduction this thread issued has been performed before the CTA leaves
+    if (threadIdx.x == 64) asm volatile("cp.async.bulk.wait_group 0;" ::: "memory");
   }
 
   // ---------------------------------------------------------------------- teardown
@@ -637,6 +672,11 @@ cudaError_t launch_tile_bwd_impl(const Problem& p, const void* q, const void* k,
   if (err != cudaSuccess) return err;
   err = make_tile_map(&map_do, d_o, p.D, p.N, p.H, p.B, p.sn, p.sh, p.sb);
   if (err != cudaSuccess) return err;
+  CUtensorMap map_dk, map_dv;
+  err = make_acc_map(&map_dk, args.acc_dk, p.D, p.N, p.B * p.H);
+  if (err != cudaSuccess) return err;
+  err = make_acc_map(&map_dv, args.acc_dv, p.D, p.N, p.B * p.H);
+  if (err != cudaSuccess) return err;
   err = cudaFuncSetAttribute(tile_bwd_kernel<HD, EC>, cudaFuncAttributeMaxDynamicSharedMemorySize, BCfg<HD>::kSmemBytes);
   if (err != cudaSuccess) return err;
   int dev = 0, sms = 0;
@@ -646,7 +686,8 @@ cudaError_t launch_tile_bwd_impl(const Problem& p, const void* q, const void* k,
   if (err != cudaSuccess) return err;
   const long all_tiles = (long)p.B * p.H * args.tiles_per_head;
   const int grid = (int)(all_tiles < sms ? all_tiles : sms);
-  tile_bwd_kernel<HD, EC><<<grid, kThreadsB, BCfg<HD>::kSmemBytes, stream>>>(map_q, map_k, map_v, map_do, args);
+  tile_bwd_kernel<HD, EC><<<grid, kThreadsB, BCfg<HD>::kSmemBytes, stream>>>(map_q, map_k, map_v, map_do, map_dk, map_dv,
+                                                                             args);
   return cudaGetLastError();
 }
 
