@@ -225,12 +225,12 @@ cudaError_t launch_tile_fwd(const Problem& p, const void* q, const void* k, cons
 
 // Dense-tile backward on the tensor cores (bf16): the rows in row_list[0 .. *row_count) are marked in
 // tile_mask, their 128-row Q tiles listed, and dQ (and dc_rows) of those rows written; their dK and dV
-// contributions are added to the fp32 accumulators.  tile_mask, tile_flag, *tile_count and *work_counter must be
-// zero on entry.
+// contributions are added to the fp32 accumulators.  tile_mask, tile_flag, *tile_count, *work_counter and
+// work_counter[12] must be zero on entry; rho: [B*H*N] floats of scratch.
 cudaError_t launch_tile_bwd(const Problem& p, const void* q, const void* k, const void* v, const void* d_o,
                             const float* scale, const float* tau, const int32_t* row_list, const int32_t* row_count,
                             uint32_t* tile_mask, int32_t* tile_flag, int32_t* tile_list, int32_t* tile_count,
-                            int32_t* work_counter, void* dq,
+                            int32_t* work_counter, float* rho, void* dq,
                             float* acc_dk, float* acc_dv, float* dc_rows, int32_t* status, cudaStream_t stream);
 
 // per-row solve + gather kernels working on the lists (bf16 path); the forward one also lists the

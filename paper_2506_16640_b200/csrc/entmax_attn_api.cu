@@ -418,7 +418,8 @@ int bwd_impl(const entmax_attn_params* params, const void* q, const void* k, con
       if (err != cudaSuccess) return fail_cuda(err);
     }
     // rows whose support does not fit the lists: dense tiles on the tensor cores
-    err = launch_tile_bwd(p, q, k, v, d_o, scale, tau, fb_list, fb_count, tile_mask, tile_flag, tile_list, tile_count, tile_count + 16, dq,
+    err = launch_tile_bwd(p, q, k, v, d_o, scale, tau, fb_list, fb_count, tile_mask, tile_flag, tile_list, tile_count, tile_count + 16,
+                          reinterpret_cast<float*>(ws + lay.half_thr) /* idle after the sweep: rho of the dense rows */, dq,
                           acc_dk, acc_dv, dc_rows, device_status, stream);
     if (err != cudaSuccess) return fail_cuda(err);
   }

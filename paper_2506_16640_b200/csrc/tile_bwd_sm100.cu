@@ -4,16 +4,20 @@
 //   dP_ij = dO_i . v_j,   rho_i = sum_j u_ij dP_ij / sum_j u_ij,   dS_ij = u_ij (dP_ij - rho_i),
 //   dQ_i = g_i sum_j dS_ij k_j,   dK_j = sum_i g_i dS_ij q_i,   dV_j = sum_i p_ij dO_i,
 //   dL/dc_i = sum_j dS_ij z_ij                      (g_i = c_i * sm_scale, c_i the ASEntmax scale)
-// A work item is one Q tile of 128 rows that holds at least one such row.  Two passes over its visible
-// K/V tiles, five tcgen05 contractions:
-//   pass A   S = Q K^T and dP = dO V^T into TMEM; the row threads accumulate sum u and sum u dP;
-//   pass B   S and dP again; the row threads write P and g dS (bf16) to shared memory; then
-//            dQ += (g dS) K     (A = g dS K-major, B = K tile with the head dim contiguous)   kept in TMEM,
-//            dK_t = (g dS)^T Q  (A = the same shared tile read M-major, B = Q tile, head dim contiguous)
-//            dV_t = P^T dO      (likewise), both through one TMEM buffer and a staging tile in shared memory, added
-//            to the fp32 dK / dV accumulators in global memory by bulk tensor reductions.
-// Rows of the tile that are not marked contribute zeros (their P and dS rows are written as zero) and
-// their dQ is not stored: the list kernels have already handled them.
+// Two kernels.  tile_bwd_kernel, query-major: a work item is one Q tile of 128 rows that holds at least one such
+// row; two passes over its visible K/V tiles:
+//   pass A   S = Q K^T and dP = dO V^T into TMEM; the row threads accumulate sum u and sum u dP: rho_i (kept for the
+//            second kernel);
+//   pass B   S and dP again; the row threads write g dS (bf16, and what the rounding left over) to shared memory;
+//            dQ += (g dS) K     (A = g dS K-major, B = K tile with the head dim contiguous)   kept in TMEM.
+// tile_bwd_kv_kernel, key-major: a work item is one K/V tile; over the marked Q tiles that see it, S and dP once
+// more, P and g dS to shared memory, and
+//            dK_t += (g dS)^T Q (A = the shared tile read M-major, B = Q tile, head dim contiguous)
+//            dV_t += P^T dO     (likewise), accumulated in TMEM over those Q tiles and added to the fp32 dK / dV
+//            accumulators in global memory once per K/V tile, by bulk tensor reductions from a staging tile.
+// (One kernel that also formed dK_t and dV_t per (Q tile, K tile) pair was bound by those reductions in L2: 128 KB of
+// them per pair.)  Rows of a Q tile that are not marked contribute zeros (their P and dS rows are written as zero)
+// and their dQ is not stored: the list kernels have already handled them.
 //
 // CTA: warp 0 TMA producer, warp 1 MMA issuer, warps 2..17 four threads per TMEM lane (32 columns each).  Every wait is
 // bounded (see sm100_ptx.cuh); on expiry the CTA flags the call's status word and leaves.
@@ -42,7 +46,7 @@ struct BCfg {
   static constexpr int kBarBytes = 256;
   static constexpr int kSmemBytes = 4 * kQBytes + 3 * kTileBytes + 1024 + kBarBytes;
   static_assert(kSmemBytes <= 232448, "shared memory of one CTA");
-  static constexpr int kTmemS = 0, kTmemDP = TN, kTmemDQ = 2 * TN, kTmemT = 2 * TN + 128;
+  static constexpr int kTmemS = 0, kTmemDP = TN, kTmemDQ = 2 * TN;
 };
 
 struct TileBwdArgs {
@@ -64,6 +68,9 @@ struct TileBwdArgs {
   float* acc_dk;             // fp32 [B,H,N,D] contiguous
   float* acc_dv;
   float* dc_rows;            // [B,H,N] or nullptr
+  float* rho;                // [B,H,N]: rho_i of the marked rows, from the query-major to the key-major kernel
+  const int32_t* tile_flag;  // [tiles]: nonzero for the Q tiles in tile_list
+  int32_t* kv_counter;       // next item of the key-major kernel (zero on entry)
   int64_t sb, sh, sn;
   int32_t* status;
   int tiles_per_head;
@@ -118,8 +125,6 @@ __global__ void __launch_bounds__(kThreadsB, 1) tile_bwd_kernel(const __grid_con
                                                                const __grid_constant__ CUtensorMap map_k,
                                                                const __grid_constant__ CUtensorMap map_v,
                                                                const __grid_constant__ CUtensorMap map_do,
-                                                               const __grid_constant__ CUtensorMap map_dk,
-                                                               const __grid_constant__ CUtensorMap map_dv,
                                                                const TileBwdArgs a) {
   using C = BCfg<HD>;
   extern __shared__ uint8_t smem_raw[];
@@ -128,7 +133,7 @@ __global__ void __launch_bounds__(kThreadsB, 1) tile_bwd_kernel(const __grid_con
   const uint32_t do_smem = q_smem + C::kQBytes;
   const uint32_t k_smem = do_smem + C::kQBytes;
   const uint32_t v_smem = k_smem + C::kQBytes;
-  const uint32_t p_smem = v_smem + C::kQBytes;           // P tile, [128 rows][128 keys] bf16, swizzled
+  const uint32_t p_smem = v_smem + C::kQBytes;           // (the key-major kernel's P tile; not used here)
   const uint32_t ds_smem = p_smem + kTileBytes;           // g dS tile (bf16), same layout
   const uint32_t dl_smem = ds_smem + kTileBytes;          // what the bf16 rounding of g dS left over, same layout
   const uint32_t bars = dl_smem + kTileBytes;
@@ -136,7 +141,6 @@ __global__ void __launch_bounds__(kThreadsB, 1) tile_bwd_kernel(const __grid_con
   const uint32_t k_full = bars + 16, k_empty = bars + 24;
   const uint32_t sd_full = bars + 32, sd_empty = bars + 40;
   const uint32_t pds_full = bars + 48, pds_empty = bars + 56;
-  const uint32_t t_full = bars + 64, t_empty = bars + 72;
   const uint32_t dq_full = bars + 80, dq_empty = bars + 88;
   const uint32_t tmem_slot = bars + 96;
   const uint32_t abort_flag = bars + 100;
@@ -163,8 +167,6 @@ __global__ void __launch_bounds__(kThreadsB, 1) tile_bwd_kernel(const __grid_con
     mbar_init(sd_empty, kConsWarps);
     mbar_init(pds_full, kConsWarps);
     mbar_init(pds_empty, 1);
-    mbar_init(t_full, 1);
-    mbar_init(t_empty, kConsWarps);
     mbar_init(dq_full, 1);
     mbar_init(dq_empty, kConsWarps);
     mbar_init(x_bar, kConsWarps);
@@ -274,14 +276,12 @@ __global__ void __launch_bounds__(kThreadsB, 1) tile_bwd_kernel(const __grid_con
     {
       constexpr uint32_t id_kk = idesc_kk();
       constexpr uint32_t id_kn = idesc_kn<HD>();
-      constexpr uint32_t id_mn = idesc_mn<HD>();
       const uint64_t hi = (uint64_t)kDescHi << 32;
       const uint64_t q_d = hi | smem_desc_lo(q_smem), do_d = hi | smem_desc_lo(do_smem);
       const uint64_t k_d = hi | smem_desc_lo(k_smem), v_d = hi | smem_desc_lo(v_smem);
       const uint64_t ds_d = hi | smem_desc_lo(ds_smem), dl_d = hi | smem_desc_lo(dl_smem);
-      const uint64_t k_n_d = hi | mn_desc_lo(k_smem), q_n_d = hi | mn_desc_lo(q_smem), do_n_d = hi | mn_desc_lo(do_smem);
-      const uint64_t ds_m_d = hi | mn_desc_lo(ds_smem), p_m_d = hi | mn_desc_lo(p_smem);
-      uint32_t kphase = 0, vphase = 0, qphase = 0, sdphase = 0, pdsphase = 0, tphase = 0, dqphase = 0, wphase = 0;
+      const uint64_t k_n_d = hi | mn_desc_lo(k_smem);
+      uint32_t kphase = 0, vphase = 0, qphase = 0, sdphase = 0, pdsphase = 0, dqphase = 0, wphase = 0;
       int slot = 0;
       bool alive = true;
       auto wait_all = [&](uint32_t bar, uint32_t parity) -> bool {
@@ -355,32 +355,6 @@ __global__ void __launch_bounds__(kThreadsB, 1) tile_bwd_kernel(const __grid_con
               umma_bf16_desc(tmem_base + C::kTmemDQ, dl_d + a_off, k_n_d + b_off, id_kn, 1u);
             }
             umma_commit(k_empty);              // dQ has taken the K tile
-          }
-          __syncwarp();
-          alive = wait_all(t_empty, tphase ^ 1u);
-          tphase ^= 1u;
-          if (!alive) break;
-          tc_fence_after();
-          if (elect_one()) {
-#pragma unroll
-            for (int kk = 0; kk < TM / 16; ++kk) {
-              const uint32_t off = kk * ((16 * 128) >> 4);                             // 16 query rows
-              umma_bf16_desc(tmem_base + C::kTmemT, ds_m_d + off, q_n_d + off, id_mn, kk > 0 ? 1u : 0u);
-            }
-            umma_commit(t_full);
-          }
-          __syncwarp();
-          alive = wait_all(t_empty, tphase ^ 1u);
-          tphase ^= 1u;
-          if (!alive) break;
-          tc_fence_after();
-          if (elect_one()) {
-#pragma unroll
-            for (int kk = 0; kk < TM / 16; ++kk) {
-              const uint32_t off = kk * ((16 * 128) >> 4);
-              umma_bf16_desc(tmem_base + C::kTmemT, p_m_d + off, do_n_d + off, id_mn, kk > 0 ? 1u : 0u);
-            }
-            umma_commit(t_full);
             umma_commit(pds_empty);
             if (t == 2 * tiles - 1) umma_commit(dq_full);
           }
@@ -403,7 +377,7 @@ __global__ void __launch_bounds__(kThreadsB, 1) tile_bwd_kernel(const __grid_con
     const int quarter = (warp - 2) >> 2;
     const int row_local = quad * 32 + lane;
     const uint32_t taddr_row = tmem_base + ((uint32_t)(quad * 32) << 16);
-    uint32_t sdphase = 0, pdsphase = 0, tphase = 0, dqphase = 0, wphase = 0, xphase = 0;
+    uint32_t sdphase = 0, pdsphase = 0, dqphase = 0, wphase = 0, xphase = 0;
     int slot = 0;
     bool alive = true;
     // The four threads of a row swap partial sums through shared memory.  The slots live in the remainder tile's
@@ -465,6 +439,7 @@ __global__ void __launch_bounds__(kThreadsB, 1) tile_bwd_kernel(const __grid_con
           alive = swap4(su, sud, su_all, sud_all);
           if (!alive) break;
           rho = su_all > 0.f ? sud_all / su_all : 0.f;
+          if (marked && quarter == 0) a.rho[grow] = rho;   // for the key-major kernel
         }
         alive = __all_sync(0xffffffffu, mbar_wait(sd_full, sdphase, abort_flag));
         if (!alive) break;
@@ -509,7 +484,7 @@ __global__ void __launch_bounds__(kThreadsB, 1) tile_bwd_kernel(const __grid_con
             const uint32_t blk = (uint32_t)(quarter >> 1) * (TM * 128) + (uint32_t)row_local * 128u;
 #pragma unroll
             for (int u4 = 0; u4 < 2; ++u4) {
-              float pv[8], dv[8], dl[8];
+              float dv[8], dl[8];
 #pragma unroll
               for (int z = 0; z < 8; ++z) {
                 const int u = u4 * 8 + z;
@@ -518,17 +493,12 @@ __global__ void __launch_bounds__(kThreadsB, 1) tile_bwd_kernel(const __grid_con
                 float ye, ye1;
                 pow_pair_c<EC>(ok ? yr : 0.f, ok, a.expo, ye, ye1);
                 const float ds = ye1 * (dp[u] - rho);
-                pv[z] = ye;
                 dv[z] = g * ds;
                 dl[z] = dv[z] - __bfloat162float(__float2bfloat16_rn(dv[z]));
                 dcs[z & 1] = fmaf(ds, sa[u], dcs[z & 1]);
               }
               const uint32_t unit = (uint32_t)((quarter & 1) * 4 + hc * 2 + u4);
               const uint32_t off = blk + ((unit ^ (uint32_t)(row_local & 7)) << 4);
-              asm volatile("st.shared::cta.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(p_smem + off),
-                           "r"(pack_bf16(pv[0], pv[1])), "r"(pack_bf16(pv[2], pv[3])), "r"(pack_bf16(pv[4], pv[5])),
-                           "r"(pack_bf16(pv[6], pv[7]))
-                           : "memory");
               asm volatile("st.shared::cta.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(ds_smem + off),
                            "r"(pack_bf16(dv[0], dv[1])), "r"(pack_bf16(dv[2], dv[3])), "r"(pack_bf16(dv[4], dv[5])),
                            "r"(pack_bf16(dv[6], dv[7]))
@@ -549,60 +519,6 @@ __global__ void __launch_bounds__(kThreadsB, 1) tile_bwd_kernel(const __grid_con
         asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
         __syncwarp();
         if (lane == 0) mbar_arrive(pds_full);
-        // dK then dV of this K tile: TMEM lane = key.  The tile is added to the fp32 accumulators in global memory by
-        // bulk reductions from shared memory (the copy engine's, not 128 x 32 vector reductions per thread group, which
-        // held the threads -- and through them the accumulator -- for thousands of cycles per tile): a thread copies its
-        // 32-column chunk of the head dimension into a staging tile, [chunk][128 keys][128 bytes] with the 128-byte
-        // swizzle of a tensor-map box, in the g dS and remainder buffers (free: the contractions that read them
-        // precede the one whose result is being read); one thread then issues a reduction per chunk.  Keys past the
-        // end of the sequence are outside the map and not written.
-        const int key0 = kt * TN;
-#pragma unroll 1
-        for (int which = 0; which < 2 && alive; ++which) {
-          alive = __all_sync(0xffffffffu, mbar_wait(t_full, tphase, abort_flag));
-          if (!alive) break;
-          tphase ^= 1u;
-          tc_fence_after();
-          if (quarter < HD / 32) {
-            float va[32];
-            tmem_ld32(taddr_row + C::kTmemT + quarter * 32, va);
-            tmem_ld_wait();
-            const uint32_t dst = ds_smem + (uint32_t)quarter * (TM * 128) + (uint32_t)row_local * 128u;
-#pragma unroll
-            for (int u = 0; u < 8; ++u)
-              asm volatile("st.shared::cta.v4.f32 [%0], {%1, %2, %3, %4};" ::"r"(dst + (((uint32_t)u ^ (uint32_t)(row_local & 7)) << 4)),
-                           "f"(va[4 * u]), "f"(va[4 * u + 1]), "f"(va[4 * u + 2]), "f"(va[4 * u + 3])
-                           : "memory");
-          }
-          // the result is out of TMEM: the next contraction may overwrite it
-          tc_fence_before();
-          asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
-          __syncwarp();
-          if (lane == 0) {
-            mbar_arrive(t_empty);
-            mbar_arrive(x_bar);
-          }
-          alive = __all_sync(0xffffffffu, mbar_wait(x_bar, xphase, abort_flag));
-          xphase ^= 1u;
-          if (!alive) break;
-          if (threadIdx.x == 64) {
-            const CUtensorMap* map = which == 0 ? &map_dk : &map_dv;
-#pragma unroll
-            for (int c = 0; c < HD / 32; ++c)
-              asm volatile(
-                  "cp.reduce.async.bulk.tensor.3d.global.shared::cta.add.tile.bulk_group [%0, {%2, %3, %4}], [%1];" ::"l"(
-                      reinterpret_cast<uint64_t>(map)),
-                  "r"(ds_smem + (uint32_t)c * (TM * 128)), "r"(c * 32), "r"(key0), "r"(bh)
-                  : "memory");
-            asm volatile("cp.async.bulk.commit_group;" ::: "memory");
-            // the staging tile may be rewritten once the reductions have read it
-            asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory");
-          }
-          __syncwarp();
-          if (lane == 0) mbar_arrive(x_bar);
-          alive = __all_sync(0xffffffffu, mbar_wait(x_bar, xphase, abort_flag));
-          xphase ^= 1u;
-        }
       }
       if (!alive) break;
       // ---- dQ of the item
@@ -637,8 +553,6 @@ __global__ void __launch_bounds__(kThreadsB, 1) tile_bwd_kernel(const __grid_con
       }
       if (a.status && threadIdx.x == 64) atomicAdd(a.status + ENTMAX_ATTN_STATUS_TILES, 1);
     }
-    // every bulk reduction this thread issued has been performed before the CTA leaves
-    if (threadIdx.x == 64) asm volatile("cp.async.bulk.wait_group 0;" ::: "memory");
   }
 
   // ---------------------------------------------------------------------- teardown
@@ -648,6 +562,393 @@ __global__ void __launch_bounds__(kThreadsB, 1) tile_bwd_kernel(const __grid_con
     if (threadIdx.x == 0 && a.status) atomicOr(a.status + ENTMAX_ATTN_STATUS_FLAGS, ENTMAX_ATTN_FLAG_WAIT_EXPIRED);
     // the producer and the MMA issuer have waited for their copies and MMAs in flight; only if one of those waits ran
     // out as well is there nothing left but to give the hardware time
+    if (lds_u32(drain_fail)) {
+      const uint64_t t0 = global_ns();
+      while (global_ns() - t0 < 200000ull) { }
+    }
+    __syncthreads();
+  }
+  if (warp == 1) {
+    tc_fence_after();
+    tmem_dealloc(tmem_base, 512);
+  }
+}
+
+// Key-major pass of the dense-tile backward: dK and dV of the marked Q tiles.  A work item is one K/V tile (128 keys
+// of one head); it walks the head's marked Q tiles that see it, recomputes S = Q K^T and dP = dO V^T, forms P and
+// g dS with the thresholds and the rho the query-major pass left in global memory, and accumulates
+//   dK_t += (g dS)^T Q   and   dV_t += P^T dO
+// in TMEM over all those Q tiles, so that each K/V tile is added to the fp32 accumulators once (by bulk tensor
+// reductions from a staging tile) instead of once per (Q tile, K tile) pair -- the reductions in L2 were what bounded
+// the single-kernel form.  Same roles and conventions as tile_bwd_kernel.
+template <int HD, int EC>
+__global__ void __launch_bounds__(kThreadsB, 1) tile_bwd_kv_kernel(const __grid_constant__ CUtensorMap map_q,
+                                                                  const __grid_constant__ CUtensorMap map_k,
+                                                                  const __grid_constant__ CUtensorMap map_v,
+                                                                  const __grid_constant__ CUtensorMap map_do,
+                                                                  const __grid_constant__ CUtensorMap map_dk,
+                                                                  const __grid_constant__ CUtensorMap map_dv,
+                                                                  const TileBwdArgs a) {
+  using C = BCfg<HD>;
+  extern __shared__ uint8_t smem_raw[];
+  const uint32_t sbase = (smem_u32(smem_raw) + 1023u) & ~1023u;
+  const uint32_t q_smem = sbase;
+  const uint32_t do_smem = q_smem + C::kQBytes;
+  const uint32_t k_smem = do_smem + C::kQBytes;
+  const uint32_t v_smem = k_smem + C::kQBytes;
+  const uint32_t p_smem = v_smem + C::kQBytes;           // P tile, [128 rows][128 keys] bf16, swizzled
+  const uint32_t ds_smem = p_smem + kTileBytes;           // g dS tile (bf16), same layout; with P the staging tile
+  const uint32_t bars = ds_smem + 2 * kTileBytes;         // (the query-major kernel's layout: the third tile is unused)
+  const uint32_t qdo_full = bars, qdo_empty = bars + 8;
+  const uint32_t kv_full = bars + 16, kv_empty = bars + 24;
+  const uint32_t sd_full = bars + 32, sd_empty = bars + 40;
+  const uint32_t pds_full = bars + 48, pds_empty = bars + 56;
+  const uint32_t acc_full = bars + 64, acc_empty = bars + 72;
+  const uint32_t tmem_slot = bars + 96;
+  const uint32_t abort_flag = bars + 100;
+  const uint32_t drain_bar = bars + 104;
+  const uint32_t drain_fail = bars + 112;
+  const uint32_t w_full = bars + 120;         // [2]
+  const uint32_t w_empty = bars + 136;        // [2]
+  const uint32_t w_item = bars + 152;         // int32 [2]: item, -1 = no more work
+  const uint32_t x_bar = bars + 160;
+  constexpr int kTmemDK = 2 * TN, kTmemDV = 2 * TN + 128;
+
+  const int warp = threadIdx.x >> 5;
+  const int lane = threadIdx.x & 31;
+  const int n_bh = a.B * a.H;
+  const int n_items = (*a.tile_count > 0) ? n_bh * a.tiles_per_head : 0;   // nothing marked: nothing to do
+
+  if (threadIdx.x == 0) {
+    mbar_init(qdo_full, 1);
+    mbar_init(qdo_empty, 1);
+    mbar_init(kv_full, 1);
+    mbar_init(kv_empty, 1);
+    mbar_init(sd_full, 1);
+    mbar_init(sd_empty, kConsWarps);
+    mbar_init(pds_full, kConsWarps);
+    mbar_init(pds_empty, 1);
+    mbar_init(acc_full, 1);
+    mbar_init(acc_empty, kConsWarps);
+    mbar_init(x_bar, kConsWarps);
+    mbar_init(drain_bar, 1);
+    for (int t = 0; t < 2; ++t) {
+      mbar_init(w_full + 8 * t, 1);
+      mbar_init(w_empty + 8 * t, 1 + kConsWarps);
+    }
+    sts_u32(drain_fail, 0u);
+    sts_u32(abort_flag, 0u);
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+  }
+  if (warp == 1) {
+    tmem_alloc(tmem_slot, 512);
+    tmem_relinquish();
+  }
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem_base = lds_u32(tmem_slot);
+
+  // Items are numbered kt * n_bh + bh: on causal problems the K tiles most Q tiles see come first.  The Q tiles of an
+  // item: the head's marked ones, from the tile that holds the K tile's own rows on (causal) or all of them.
+  auto first_q = [&](int kt) -> int { return a.causal ? kt : 0; };
+  auto next_marked = [&](int bh, int qt) -> int {      // first marked Q tile >= qt of head bh, or tiles_per_head
+    while (qt < a.tiles_per_head && a.tile_flag[bh * a.tiles_per_head + qt] == 0) ++qt;
+    return qt;
+  };
+
+  if (warp == 0) {
+    // ------------------------------------------------------------------ TMA producer
+    uint32_t kvphase = 0, qphase = 0, wphase = 0;
+    int slot = 0;
+    bool alive = true;
+    auto wait_all = [&](uint32_t bar, uint32_t parity) -> bool {
+      return __all_sync(0xffffffffu, mbar_wait(bar, parity, abort_flag));
+    };
+    while (alive) {
+      alive = wait_all(w_empty + 8 * slot, wphase ^ 1u);
+      if (!alive) break;
+      int it = 0;
+      if (lane == 0) {
+        it = atomicAdd(a.kv_counter, 1);
+        if (it >= n_items) it = -1;
+        sts_u32(w_item + 4 * slot, (uint32_t)it);
+        mbar_arrive(w_full + 8 * slot);
+      }
+      it = __shfl_sync(0xffffffffu, it, 0);
+      if (++slot == 2) { slot = 0; wphase ^= 1u; }
+      if (it < 0) break;
+      const int kt = it / n_bh, bh = it - kt * n_bh;
+      const int b = bh / a.H, h = bh - b * a.H;
+      int qt = __shfl_sync(0xffffffffu, next_marked(bh, first_q(kt)), 0);
+      if (qt >= a.tiles_per_head) continue;            // no marked Q tile sees these keys
+      alive = wait_all(kv_empty, kvphase ^ 1u);
+      if (!alive) break;
+      kvphase ^= 1u;
+      if (elect_one()) {
+        mbar_expect_tx(kv_full, 2 * C::kQBytes);
+        for (int hf = 0; hf < C::kHalves; ++hf) {
+          tma_load_4d(k_smem + hf * (TN * 128), &map_k, kv_full, hf * 64, kt * TN, h, b);
+          tma_load_4d(v_smem + hf * (TN * 128), &map_v, kv_full, hf * 64, kt * TN, h, b);
+        }
+      }
+      __syncwarp();
+      while (qt < a.tiles_per_head && alive) {
+        alive = wait_all(qdo_empty, qphase ^ 1u);
+        if (!alive) break;
+        qphase ^= 1u;
+        if (elect_one()) {
+          mbar_expect_tx(qdo_full, 2 * C::kQBytes);
+          for (int hf = 0; hf < C::kHalves; ++hf) {
+            tma_load_4d(q_smem + hf * (TM * 128), &map_q, qdo_full, hf * 64, qt * TM, h, b);
+            tma_load_4d(do_smem + hf * (TM * 128), &map_do, qdo_full, hf * 64, qt * TM, h, b);
+          }
+        }
+        __syncwarp();
+        qt = __shfl_sync(0xffffffffu, next_marked(bh, qt + 1), 0);
+      }
+    }
+    if (!alive && lane == 0) {
+      bool ok = mbar_drain(qdo_full, qphase ^ 1u);
+      ok &= mbar_drain(kv_full, kvphase ^ 1u);
+      if (!ok) sts_u32(drain_fail, 1u);
+    }
+  } else if (warp == 1) {
+    // ------------------------------------------------------------------ MMA issuer
+    constexpr uint32_t id_kk = idesc_kk();
+    constexpr uint32_t id_mn = idesc_mn<HD>();
+    const uint64_t hi = (uint64_t)kDescHi << 32;
+    const uint64_t q_d = hi | smem_desc_lo(q_smem), do_d = hi | smem_desc_lo(do_smem);
+    const uint64_t k_d = hi | smem_desc_lo(k_smem), v_d = hi | smem_desc_lo(v_smem);
+    const uint64_t q_n_d = hi | mn_desc_lo(q_smem), do_n_d = hi | mn_desc_lo(do_smem);
+    const uint64_t ds_m_d = hi | mn_desc_lo(ds_smem), p_m_d = hi | mn_desc_lo(p_smem);
+    uint32_t kvphase = 0, qphase = 0, sdphase = 0, pdsphase = 0, accphase = 0, wphase = 0;
+    int slot = 0;
+    bool alive = true;
+    auto wait_all = [&](uint32_t bar, uint32_t parity) -> bool {
+      return __all_sync(0xffffffffu, mbar_wait(bar, parity, abort_flag));
+    };
+    while (alive) {
+      alive = wait_all(w_full + 8 * slot, wphase);
+      if (!alive) break;
+      const int it = __shfl_sync(0xffffffffu, (int)lds_u32(w_item + 4 * slot), 0);
+      __syncwarp();
+      if (lane == 0) mbar_arrive(w_empty + 8 * slot);
+      if (++slot == 2) { slot = 0; wphase ^= 1u; }
+      if (it < 0) break;
+      const int kt = it / n_bh, bh = it - kt * n_bh;
+      int qt = __shfl_sync(0xffffffffu, next_marked(bh, first_q(kt)), 0);
+      if (qt >= a.tiles_per_head) continue;
+      alive = wait_all(kv_full, kvphase);
+      kvphase ^= 1u;
+      // the previous item's dK and dV must have been read before this item's first contraction overwrites them
+      if (alive) alive = wait_all(acc_empty, accphase ^ 1u);
+      accphase ^= 1u;
+      if (!alive) break;
+      bool first = true;
+      while (qt < a.tiles_per_head && alive) {
+        alive = wait_all(qdo_full, qphase);
+        qphase ^= 1u;
+        if (alive) alive = wait_all(sd_empty, sdphase ^ 1u);
+        if (!alive) break;
+        sdphase ^= 1u;
+        tc_fence_after();
+        if (elect_one()) {
+#pragma unroll
+          for (int kk = 0; kk < HD / 16; ++kk) {
+            const uint32_t off = (kk >> 2) * ((TM * 128) >> 4) + (kk & 3) * 2;
+            umma_bf16_desc(tmem_base + C::kTmemS, q_d + off, k_d + off, id_kk, kk > 0 ? 1u : 0u);
+          }
+#pragma unroll
+          for (int kk = 0; kk < HD / 16; ++kk) {
+            const uint32_t off = (kk >> 2) * ((TM * 128) >> 4) + (kk & 3) * 2;
+            umma_bf16_desc(tmem_base + C::kTmemDP, do_d + off, v_d + off, id_kk, kk > 0 ? 1u : 0u);
+          }
+          umma_commit(sd_full);
+        }
+        __syncwarp();
+        // P and g dS of this pair are in shared memory
+        alive = wait_all(pds_full, pdsphase);
+        pdsphase ^= 1u;
+        if (!alive) break;
+        tc_fence_after();
+        if (elect_one()) {
+#pragma unroll
+          for (int kk = 0; kk < TM / 16; ++kk) {
+            const uint32_t off = kk * ((16 * 128) >> 4);                             // 16 query rows
+            umma_bf16_desc(tmem_base + kTmemDK, ds_m_d + off, q_n_d + off, id_mn, (!first || kk > 0) ? 1u : 0u);
+          }
+#pragma unroll
+          for (int kk = 0; kk < TM / 16; ++kk) {
+            const uint32_t off = kk * ((16 * 128) >> 4);
+            umma_bf16_desc(tmem_base + kTmemDV, p_m_d + off, do_n_d + off, id_mn, (!first || kk > 0) ? 1u : 0u);
+          }
+          umma_commit(pds_empty);
+          umma_commit(qdo_empty);
+        }
+        __syncwarp();
+        first = false;
+        qt = __shfl_sync(0xffffffffu, next_marked(bh, qt + 1), 0);
+      }
+      if (!alive) break;
+      if (elect_one()) {
+        umma_commit(acc_full);
+        umma_commit(kv_empty);
+      }
+      __syncwarp();
+    }
+    if (!alive && lane == 0) {
+      umma_commit(drain_bar);
+      if (!mbar_drain(drain_bar, 0u)) sts_u32(drain_fail, 1u);
+    }
+  } else {
+    // ------------------------------------------------------------------ consumers: four threads per TMEM lane
+    const int quad = warp & 3;
+    const int quarter = (warp - 2) >> 2;
+    const int row_local = quad * 32 + lane;
+    const uint32_t taddr_row = tmem_base + ((uint32_t)(quad * 32) << 16);
+    uint32_t sdphase = 0, pdsphase = 0, accphase = 0, wphase = 0, xphase = 0;
+    int slot = 0;
+    bool alive = true;
+    while (alive) {
+      alive = __all_sync(0xffffffffu, mbar_wait(w_full + 8 * slot, wphase, abort_flag));
+      if (!alive) break;
+      const int it = (int)lds_u32(w_item + 4 * slot);
+      __syncwarp();
+      if (lane == 0) mbar_arrive(w_empty + 8 * slot);
+      if (++slot == 2) { slot = 0; wphase ^= 1u; }
+      if (it < 0) break;
+      const int kt = it / n_bh, bh = it - kt * n_bh;
+      const int b = bh / a.H, h = bh - b * a.H;
+      int qt = __shfl_sync(0xffffffffu, next_marked(bh, first_q(kt)), 0);
+      if (qt >= a.tiles_per_head) continue;
+      const float slope = a.alibi ? a.alibi[h] / a.sm_scale : 0.f;   // bias in accumulator units
+      while (qt < a.tiles_per_head && alive) {
+        // this thread's query row of the Q tile: TMEM lane = query row, as in the query-major pass
+        const int i = qt * TM + row_local;
+        const bool valid = i < a.N;
+        const int id = bh * a.tiles_per_head + qt;
+        const bool marked = valid && ((a.tile_mask[4 * (size_t)id + (row_local >> 5)] >> (row_local & 31)) & 1u);
+        const size_t grow = (size_t)bh * a.N + (valid ? i : 0);
+        const int lim = a.causal ? i : a.N - 1;
+        const float c_i = valid ? a.scale[(size_t)b * a.scale_sb + (size_t)h * a.N + i] : 0.f;
+        const float ra = a.alpha_m1 * (c_i * a.sm_scale);
+        const float g = c_i * a.sm_scale;
+        const float tau = marked ? a.tau[grow] : 0.f;
+        const float rho = marked ? a.rho[grow] : 0.f;
+        alive = __all_sync(0xffffffffu, mbar_wait(sd_full, sdphase, abort_flag));
+        if (!alive) break;
+        sdphase ^= 1u;
+        tc_fence_after();
+        // P and dS of the previous pair must have been consumed before their buffers are rewritten
+        alive = __all_sync(0xffffffffu, mbar_wait(pds_empty, pdsphase ^ 1u, abort_flag));
+        pdsphase ^= 1u;
+        if (!alive) break;
+#pragma unroll 1
+        for (int hc = 0; hc < 2; ++hc) {
+          float sa[16], dp[16];
+          tmem_ld16(taddr_row + C::kTmemS + quarter * 32 + hc * 16, sa);
+          tmem_ld16(taddr_row + C::kTmemDP + quarter * 32 + hc * 16, dp);
+          tmem_ld_wait();
+          const int col0 = kt * TN + quarter * 32 + hc * 16;
+          if (slope != 0.f) {
+#pragma unroll
+            for (int u = 0; u < 16; ++u) sa[u] = fmaf(slope, (float)(col0 + u - i), sa[u]);
+          }
+          const bool edge = col0 + 15 > lim;
+          const uint32_t blk = (uint32_t)(quarter >> 1) * (TM * 128) + (uint32_t)row_local * 128u;
+#pragma unroll
+          for (int u4 = 0; u4 < 2; ++u4) {
+            float pv[8], dv[8];
+#pragma unroll
+            for (int z = 0; z < 8; ++z) {
+              const int u = u4 * 8 + z;
+              const float yr = fmaf(ra, sa[u], -tau);
+              const bool ok = marked && yr > 0.f && (!edge || col0 + u <= lim);
+              float ye, ye1;
+              pow_pair_c<EC>(ok ? yr : 0.f, ok, a.expo, ye, ye1);
+              pv[z] = ye;
+              dv[z] = g * (ye1 * (dp[u] - rho));
+            }
+            const uint32_t unit = (uint32_t)((quarter & 1) * 4 + hc * 2 + u4);
+            const uint32_t off = blk + ((unit ^ (uint32_t)(row_local & 7)) << 4);
+            asm volatile("st.shared::cta.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(p_smem + off),
+                         "r"(pack_bf16(pv[0], pv[1])), "r"(pack_bf16(pv[2], pv[3])), "r"(pack_bf16(pv[4], pv[5])),
+                         "r"(pack_bf16(pv[6], pv[7]))
+                         : "memory");
+            asm volatile("st.shared::cta.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(ds_smem + off),
+                         "r"(pack_bf16(dv[0], dv[1])), "r"(pack_bf16(dv[2], dv[3])), "r"(pack_bf16(dv[4], dv[5])),
+                         "r"(pack_bf16(dv[6], dv[7]))
+                         : "memory");
+          }
+        }
+        tc_fence_before();
+        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+        __syncwarp();
+        if (lane == 0) {
+          mbar_arrive(sd_empty);
+          mbar_arrive(pds_full);
+        }
+        qt = __shfl_sync(0xffffffffu, next_marked(bh, qt + 1), 0);
+      }
+      if (!alive) break;
+      // ---- dK and dV of the K tile: TMEM lane = key; through a staging tile (the P and g dS buffers, free once the
+      //      item's last contraction has finished) and bulk tensor reductions into the fp32 accumulators
+      alive = __all_sync(0xffffffffu, mbar_wait(acc_full, accphase, abort_flag));
+      accphase ^= 1u;
+      if (!alive) break;
+      tc_fence_after();
+      const int key0 = kt * TN;
+#pragma unroll 1
+      for (int which = 0; which < 2 && alive; ++which) {
+        if (quarter < HD / 32) {
+          float va[32];
+          tmem_ld32(taddr_row + (which == 0 ? kTmemDK : kTmemDV) + quarter * 32, va);
+          tmem_ld_wait();
+          const uint32_t dst = p_smem + (uint32_t)quarter * (TM * 128) + (uint32_t)row_local * 128u;
+#pragma unroll
+          for (int u = 0; u < 8; ++u)
+            asm volatile("st.shared::cta.v4.f32 [%0], {%1, %2, %3, %4};" ::"r"(dst + (((uint32_t)u ^ (uint32_t)(row_local & 7)) << 4)),
+                         "f"(va[4 * u]), "f"(va[4 * u + 1]), "f"(va[4 * u + 2]), "f"(va[4 * u + 3])
+                         : "memory");
+        }
+        tc_fence_before();
+        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+        __syncwarp();
+        if (lane == 0) {
+          if (which == 1) mbar_arrive(acc_empty);      // both accumulators are out of TMEM
+          mbar_arrive(x_bar);
+        }
+        alive = __all_sync(0xffffffffu, mbar_wait(x_bar, xphase, abort_flag));
+        xphase ^= 1u;
+        if (!alive) break;
+        if (threadIdx.x == 64) {
+          const CUtensorMap* map = which == 0 ? &map_dk : &map_dv;
+#pragma unroll
+          for (int c = 0; c < HD / 32; ++c)
+            asm volatile(
+                "cp.reduce.async.bulk.tensor.3d.global.shared::cta.add.tile.bulk_group [%0, {%2, %3, %4}], [%1];" ::"l"(
+                    reinterpret_cast<uint64_t>(map)),
+                "r"(p_smem + (uint32_t)c * (TM * 128)), "r"(c * 32), "r"(key0), "r"(bh)
+                : "memory");
+          asm volatile("cp.async.bulk.commit_group;" ::: "memory");
+          asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory");
+        }
+        __syncwarp();
+        if (lane == 0) mbar_arrive(x_bar);
+        alive = __all_sync(0xffffffffu, mbar_wait(x_bar, xphase, abort_flag));
+        xphase ^= 1u;
+      }
+    }
+    if (threadIdx.x == 64) asm volatile("cp.async.bulk.wait_group 0;" ::: "memory");
+  }
+
+  // ---------------------------------------------------------------------- teardown
+  tc_fence_before();
+  __syncthreads();
+  if (lds_u32(abort_flag)) {
+    if (threadIdx.x == 0 && a.status) atomicOr(a.status + ENTMAX_ATTN_STATUS_FLAGS, ENTMAX_ATTN_FLAG_WAIT_EXPIRED);
     if (lds_u32(drain_fail)) {
       const uint64_t t0 = global_ns();
       while (global_ns() - t0 < 200000ull) { }
@@ -686,8 +987,15 @@ cudaError_t launch_tile_bwd_impl(const Problem& p, const void* q, const void* k,
   if (err != cudaSuccess) return err;
   const long all_tiles = (long)p.B * p.H * args.tiles_per_head;
   const int grid = (int)(all_tiles < sms ? all_tiles : sms);
-  tile_bwd_kernel<HD, EC><<<grid, kThreadsB, BCfg<HD>::kSmemBytes, stream>>>(map_q, map_k, map_v, map_do, map_dk, map_dv,
-                                                                             args);
+  tile_bwd_kernel<HD, EC><<<grid, kThreadsB, BCfg<HD>::kSmemBytes, stream>>>(map_q, map_k, map_v, map_do, args);
+  err = cudaGetLastError();
+  if (err != cudaSuccess) return err;
+  // dK and dV of the same Q tiles, key-major (needs the rho the kernel above leaves behind)
+  err = cudaFuncSetAttribute(tile_bwd_kv_kernel<HD, EC>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                             BCfg<HD>::kSmemBytes);
+  if (err != cudaSuccess) return err;
+  tile_bwd_kv_kernel<HD, EC><<<grid, kThreadsB, BCfg<HD>::kSmemBytes, stream>>>(map_q, map_k, map_v, map_do, map_dk,
+                                                                                map_dv, args);
   return cudaGetLastError();
 }
 
@@ -696,7 +1004,8 @@ cudaError_t launch_tile_bwd_impl(const Problem& p, const void* q, const void* k,
 cudaError_t launch_tile_bwd(const Problem& p, const void* q, const void* k, const void* v, const void* d_o,
                             const float* scale, const float* tau, const int32_t* row_list, const int32_t* row_count,
                             uint32_t* tile_mask, int32_t* tile_flag, int32_t* tile_list, int32_t* tile_count,
-                            int32_t* work_counter, void* dq, float* acc_dk, float* acc_dv, float* dc_rows, int32_t* status, cudaStream_t stream) {
+                            int32_t* work_counter, float* rho, void* dq, float* acc_dk, float* acc_dv, float* dc_rows,
+                            int32_t* status, cudaStream_t stream) {
   const int tiles_per_head = (p.N + TM - 1) / TM;
   mark_tiles_kernel<<<148, 256, 0, stream>>>(p.N, tiles_per_head, row_list, row_count, tile_mask, tile_flag, tile_list,
                                              tile_count);
@@ -717,6 +1026,9 @@ cudaError_t launch_tile_bwd(const Problem& p, const void* q, const void* k, cons
   args.tile_list = tile_list;
   args.tile_count = tile_count;
   args.work_counter = work_counter;
+  args.kv_counter = work_counter + 12;   // (the counter block's last word)
+  args.tile_flag = tile_flag;
+  args.rho = rho;
   args.tile_mask = tile_mask;
   args.tau = tau;
   args.dq = dq;
