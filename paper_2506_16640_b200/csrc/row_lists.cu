@@ -538,13 +538,14 @@ __device__ __forceinline__ void solve_rows_closed(const Problem& p, const __nv_b
   }
 }
 
-// Rows with more than 32 list entries take the whole warp for a long time each (two-stage solves, gathers over
+// Rows with more than kLongRow list entries take the whole warp for a long time each (two-stage solves, gathers over
 // dozens of keys) and come in runs -- the start of every causal head, where all visible keys are candidates.  A
 // warp that met sixteen of them in its block would work through them one after the other while the rest of the grid
 // has finished, so they are only listed here (from the far end of the dense-row list, which has a slot for every
 // row) and a second launch gives each of them a warp of its own.  kLongCounter: their count, in the counter block
 // that starts at fb_count.
 constexpr int kLongCounter = 56;
+constexpr int kLongRow = 16;   // list entries from which a row counts as long
 __device__ __forceinline__ void push_long_rows(unsigned mask, int grow, int total, int32_t* fb_count, int32_t* fb_list,
                                                int lane) {
   if (mask == 0u) return;
@@ -674,7 +675,7 @@ __global__ void __launch_bounds__(kWarpsPerCta * 32) row_fwd_kernel(Problem p, c
       push_dense_tiles(p, mdense, my_row, row_cnt, fb_count, fb_list, tile_flag, tile_list, tile_count, status, lane);
       mfull &= ~mdense;
       // ... and the ones with long lists to a launch of their own
-      const unsigned mlong = __ballot_sync(0xffffffffu, lane < 16 && ((mfull >> lane) & 1u) && mc0 + mc1 > 32);
+      const unsigned mlong = __ballot_sync(0xffffffffu, lane < 16 && ((mfull >> lane) & 1u) && mc0 + mc1 > (kClosed ? kLongRow : 32));
       push_long_rows(mlong, my_row, total, fb_count, fb_list, lane);
       mfull &= ~mlong;
     }
@@ -1013,8 +1014,7 @@ __global__ void __launch_bounds__(kWarpsPerCta * 32, 4) row_bwd_kernel(
       push_dense_rows(mdense, my_row, fb_count, fb_list, status, lane);
       mlong &= ~mdense;
       // ... and the ones with long lists to a launch of their own (see push_long_rows)
-      push_long_rows(mlong, my_row, total, fb_count, fb_list, lane);
-      mlong = 0u;
+      push_long_rows(mlong | m32, my_row, total, fb_count, fb_list, lane);
     }
     while (m8) {
       const unsigned src = __fns(m8, 0, (lane >> 3) + 1);          // the row of this group of eight lanes
@@ -1033,13 +1033,6 @@ __global__ void __launch_bounds__(kWarpsPerCta * 32, 4) row_bwd_kernel(
                           active ? 16 * blk + (int)src : 0, active, c0, c1, saved != 0, pitch, lane);
       m16 &= m16 - 1;
       m16 &= m16 - 1;
-    }
-    while (m32) {
-      const int src = __ffs(m32) - 1;
-      m32 &= m32 - 1;
-      const int c0 = __shfl_sync(0xffffffffu, mc0, src), c1 = __shfl_sync(0xffffffffu, mc1, src);
-      bwd_rows_sub<D, 32>(p, q, k, v, d_o, scale, tau_in, entries, dq, acc_dk, acc_dv, dc_rows, 16 * blk + src, true, c0, c1,
-                          saved != 0, pitch, lane);
     }
   }
 }
@@ -1066,8 +1059,12 @@ __global__ void __launch_bounds__(kWarpsPerCta * 32, 4) row_bwd_long_kernel(
       c0 = c.x;
       c1 = c.y;
     }
-    bwd_row_full<D>(p, q, k, v, d_o, scale, tau_in, entries, dq, acc_dk, acc_dv, dc_rows, grow, c0, c1, saved != 0, pitch,
-                    lane);
+    if (c0 + c1 <= 32)
+      bwd_rows_sub<D, 32>(p, q, k, v, d_o, scale, tau_in, entries, dq, acc_dk, acc_dv, dc_rows, grow, true, c0, c1,
+                          saved != 0, pitch, lane);
+    else
+      bwd_row_full<D>(p, q, k, v, d_o, scale, tau_in, entries, dq, acc_dk, acc_dv, dc_rows, grow, c0, c1, saved != 0,
+                      pitch, lane);
   }
 }
 

@@ -99,6 +99,14 @@ __device__ __forceinline__ uint32_t mn_desc_lo(uint32_t saddr) {
   return ((saddr & 0x3FFFFu) >> 4) | ((uint32_t)((128 * 128) >> 4) << 16);
 }
 
+// m^(e-1) of a clamped m >= 0 for the compile-time exponent classes (0 for m = 0, also for e = 1), FMA-pipe work only
+template <int EC>
+__device__ __forceinline__ float clamped_pow_m1(float m) {
+  if constexpr (EC == kExpo2) return m;
+  else if constexpr (EC == kExpo4) return (m * m) * m;
+  else return positive_indicator(m);
+}
+
 __device__ __forceinline__ uint32_t pack_bf16(float a, float b) {
   const __nv_bfloat162 hh = __floats2bfloat162_rn(a, b);
   return *reinterpret_cast<const uint32_t*>(&hh);
@@ -138,7 +146,7 @@ __global__ void __launch_bounds__(kThreadsB, 1) tile_bwd_kernel(const __grid_con
   const uint32_t dl_smem = ds_smem + kTileBytes;          // what the bf16 rounding of g dS left over, same layout
   const uint32_t bars = dl_smem + kTileBytes;
   const uint32_t qdo_full = bars, qdo_empty = bars + 8;
-  const uint32_t k_full = bars + 16, k_empty = bars + 24;
+  const uint32_t k_full0 = bars + 16, k_empty0 = bars + 24;
   const uint32_t sd_full = bars + 32, sd_empty = bars + 40;
   const uint32_t pds_full = bars + 48, pds_empty = bars + 56;
   const uint32_t dq_full = bars + 80, dq_empty = bars + 88;
@@ -150,7 +158,17 @@ __global__ void __launch_bounds__(kThreadsB, 1) tile_bwd_kernel(const __grid_con
   const uint32_t w_empty = bars + 136;        // [2] ... and read by the MMA issuer and every consumer warp
   const uint32_t w_item = bars + 152;         // int32 [2]: tile id, -1 = no more work
   const uint32_t x_bar = bars + 160;          // the threads of a row have written their partial sums
-  const uint32_t v_full = bars + 168, v_empty = bars + 176;
+  const uint32_t v_full0 = bars + 168, v_empty0 = bars + 176;
+  // Pass A has a second K / V stage: the P tile's buffer (the key-major kernel's; idle here) and the g dS buffer, which
+  // is idle until pass B and free again when the item's last contraction has finished -- which the producer waits for
+  // before it loads anything of the next item.
+  const uint32_t k_full1 = bars + 184, k_empty1 = bars + 192, v_full1 = bars + 200, v_empty1 = bars + 208;
+  auto k_full = [&](int st) { return st ? k_full1 : k_full0; };
+  auto k_empty = [&](int st) { return st ? k_empty1 : k_empty0; };
+  auto v_full = [&](int st) { return st ? v_full1 : v_full0; };
+  auto v_empty = [&](int st) { return st ? v_empty1 : v_empty0; };
+  auto k_stage = [&](int st) { return st ? p_smem : k_smem; };
+  auto v_stage = [&](int st) { return st ? ds_smem : v_smem; };
 
   const int warp = threadIdx.x >> 5;
   const int lane = threadIdx.x & 31;
@@ -159,10 +177,12 @@ __global__ void __launch_bounds__(kThreadsB, 1) tile_bwd_kernel(const __grid_con
   if (threadIdx.x == 0) {
     mbar_init(qdo_full, 1);
     mbar_init(qdo_empty, 1);
-    mbar_init(k_full, 1);
-    mbar_init(k_empty, 1);
-    mbar_init(v_full, 1);
-    mbar_init(v_empty, 1);
+    for (int st = 0; st < 2; ++st) {
+      mbar_init(k_full(st), 1);
+      mbar_init(k_empty(st), 1);
+      mbar_init(v_full(st), 1);
+      mbar_init(v_empty(st), 1);
+    }
     mbar_init(sd_full, 1);
     mbar_init(sd_empty, kConsWarps);
     mbar_init(pds_full, kConsWarps);
@@ -203,7 +223,7 @@ __global__ void __launch_bounds__(kThreadsB, 1) tile_bwd_kernel(const __grid_con
     // tiles have barriers of their own: in pass B the V tile is free again once dP has been formed and the K tile
     // once dQ has taken it, so the next tile's copies run under the dK / dV contractions of this one.
     {
-      uint32_t kphase = 0, vphase = 0, qphase = 0, wphase = 0;
+      uint32_t kbits = 0, vbits = 0 /* bit st: times the stage's barrier has been armed, mod 2 */, qphase = 0, wphase = 0;
       int slot = 0;
       bool alive = true;
       auto wait_all = [&](uint32_t bar, uint32_t parity) -> bool {
@@ -239,22 +259,23 @@ __global__ void __launch_bounds__(kThreadsB, 1) tile_bwd_kernel(const __grid_con
         __syncwarp();
         for (int t = 0; t < 2 * tiles && alive; ++t) {
           const int kt = t < tiles ? t : t - tiles;
-          alive = wait_all(v_empty, vphase ^ 1u);
+          const int st = t < tiles ? (t & 1) : 0;   // pass A alternates between the two stages, pass B has one
+          alive = wait_all(v_empty(st), ((vbits >> st) & 1u) ^ 1u);
           if (!alive) break;
-          vphase ^= 1u;
+          vbits ^= 1u << st;
           if (elect_one()) {
-            mbar_expect_tx(v_full, C::kQBytes);
+            mbar_expect_tx(v_full(st), C::kQBytes);
             for (int hf = 0; hf < C::kHalves; ++hf)
-              tma_load_4d(v_smem + hf * (TN * 128), &map_v, v_full, hf * 64, kt * TN, h, b);
+              tma_load_4d(v_stage(st) + hf * (TN * 128), &map_v, v_full(st), hf * 64, kt * TN, h, b);
           }
           __syncwarp();
-          alive = wait_all(k_empty, kphase ^ 1u);
+          alive = wait_all(k_empty(st), ((kbits >> st) & 1u) ^ 1u);
           if (!alive) break;
-          kphase ^= 1u;
+          kbits ^= 1u << st;
           if (elect_one()) {
-            mbar_expect_tx(k_full, C::kQBytes);
+            mbar_expect_tx(k_full(st), C::kQBytes);
             for (int hf = 0; hf < C::kHalves; ++hf)
-              tma_load_4d(k_smem + hf * (TN * 128), &map_k, k_full, hf * 64, kt * TN, h, b);
+              tma_load_4d(k_stage(st) + hf * (TN * 128), &map_k, k_full(st), hf * 64, kt * TN, h, b);
           }
           __syncwarp();
         }
@@ -263,8 +284,10 @@ __global__ void __launch_bounds__(kThreadsB, 1) tile_bwd_kernel(const __grid_con
         // a wait ran out somewhere in the CTA: the copies this warp armed barriers for must land before shared
         // memory goes away (after n arms a phase word holds n mod 2 and the last armed phase has the other parity)
         bool ok = mbar_drain(qdo_full, qphase ^ 1u);
-        ok &= mbar_drain(k_full, kphase ^ 1u);
-        ok &= mbar_drain(v_full, vphase ^ 1u);
+        for (int st = 0; st < 2; ++st) {
+          ok &= mbar_drain(k_full(st), ((kbits >> st) & 1u) ^ 1u);
+          ok &= mbar_drain(v_full(st), ((vbits >> st) & 1u) ^ 1u);
+        }
         if (!ok) sts_u32(drain_fail, 1u);
       }
     }
@@ -281,7 +304,9 @@ __global__ void __launch_bounds__(kThreadsB, 1) tile_bwd_kernel(const __grid_con
       const uint64_t k_d = hi | smem_desc_lo(k_smem), v_d = hi | smem_desc_lo(v_smem);
       const uint64_t ds_d = hi | smem_desc_lo(ds_smem), dl_d = hi | smem_desc_lo(dl_smem);
       const uint64_t k_n_d = hi | mn_desc_lo(k_smem);
-      uint32_t kphase = 0, vphase = 0, qphase = 0, sdphase = 0, pdsphase = 0, dqphase = 0, wphase = 0;
+      uint32_t kbits = 0, vbits = 0 /* bit st: phase of the stage's barrier to wait for */, qphase = 0, sdphase = 0,
+               pdsphase = 0, dqphase = 0, wphase = 0;
+      const uint64_t k1_d = hi | smem_desc_lo(p_smem), v1_d = hi | smem_desc_lo(ds_smem);   // stage 1 of pass A
       int slot = 0;
       bool alive = true;
       auto wait_all = [&](uint32_t bar, uint32_t parity) -> bool {
@@ -308,10 +333,12 @@ __global__ void __launch_bounds__(kThreadsB, 1) tile_bwd_kernel(const __grid_con
             dqphase ^= 1u;
             if (!alive) break;
           }
-          alive = wait_all(k_full, kphase);
-          kphase ^= 1u;
-          if (alive) alive = wait_all(v_full, vphase);
-          vphase ^= 1u;
+          const int st = pass_b ? 0 : (t & 1);
+          alive = wait_all(k_full(st), (kbits >> st) & 1u);
+          kbits ^= 1u << st;
+          if (alive) alive = wait_all(v_full(st), (vbits >> st) & 1u);
+          vbits ^= 1u << st;
+          const uint64_t ks_d = st ? k1_d : k_d, vs_d = st ? v1_d : v_d;
           if (alive) alive = wait_all(sd_empty, sdphase ^ 1u);
           if (!alive) break;
           sdphase ^= 1u;
@@ -320,16 +347,16 @@ __global__ void __launch_bounds__(kThreadsB, 1) tile_bwd_kernel(const __grid_con
 #pragma unroll
             for (int kk = 0; kk < HD / 16; ++kk) {
               const uint32_t off = (kk >> 2) * ((TM * 128) >> 4) + (kk & 3) * 2;
-              umma_bf16_desc(tmem_base + C::kTmemS, q_d + off, k_d + off, id_kk, kk > 0 ? 1u : 0u);
+              umma_bf16_desc(tmem_base + C::kTmemS, q_d + off, ks_d + off, id_kk, kk > 0 ? 1u : 0u);
             }
 #pragma unroll
             for (int kk = 0; kk < HD / 16; ++kk) {
               const uint32_t off = (kk >> 2) * ((TM * 128) >> 4) + (kk & 3) * 2;
-              umma_bf16_desc(tmem_base + C::kTmemDP, do_d + off, v_d + off, id_kk, kk > 0 ? 1u : 0u);
+              umma_bf16_desc(tmem_base + C::kTmemDP, do_d + off, vs_d + off, id_kk, kk > 0 ? 1u : 0u);
             }
             umma_commit(sd_full);
-            umma_commit(v_empty);              // dP has been formed: the V tile is free
-            if (!pass_b) umma_commit(k_empty);
+            umma_commit(v_empty(st));          // dP has been formed: the V tile is free
+            if (!pass_b) umma_commit(k_empty(st));
           }
           __syncwarp();
           if (!pass_b) continue;
@@ -354,7 +381,7 @@ __global__ void __launch_bounds__(kThreadsB, 1) tile_bwd_kernel(const __grid_con
               const uint32_t b_off = kk * ((16 * 128) >> 4);
               umma_bf16_desc(tmem_base + C::kTmemDQ, dl_d + a_off, k_n_d + b_off, id_kn, 1u);
             }
-            umma_commit(k_empty);              // dQ has taken the K tile
+            umma_commit(k_empty(0));           // dQ has taken the K tile
             umma_commit(pds_empty);
             if (t == 2 * tiles - 1) umma_commit(dq_full);
           }
@@ -428,6 +455,7 @@ __global__ void __launch_bounds__(kThreadsB, 1) tile_bwd_kernel(const __grid_con
       const float g = c_i * a.sm_scale;
       const float slope = a.alibi ? a.alibi[h] / a.sm_scale : 0.f;   // bias in accumulator units
       const float tau = marked ? a.tau[grow] : 0.f;
+      const float ra_m = marked ? ra : 0.f;
       float su = 0.f, sud = 0.f, rho = 0.f;
       float dcs[2] = {0.f, 0.f};   // sum_j dS_ij * (accumulator + bias), two partial sums
       for (int t = 0; t < 2 * tiles && alive; ++t) {
@@ -467,14 +495,25 @@ __global__ void __launch_bounds__(kThreadsB, 1) tile_bwd_kernel(const __grid_con
           if (!pass_b) {
             // four independent partial sums each, so that the additions do not form one serial chain
             float p0[4] = {0.f, 0.f, 0.f, 0.f}, p1[4] = {0.f, 0.f, 0.f, 0.f};
+            if (EC != kExpoGeneral && !edge) {
+              // away from the mask: one ALU-pipe clamp per element, the rest FMA-pipe work
 #pragma unroll
-            for (int u = 0; u < 16; ++u) {
-              const float yr = fmaf(ra, sa[u], -tau);
-              const bool ok = yr > 0.f && (!edge || col0 + u <= lim);
-              float ye, ye1;
-              pow_pair_c<EC>(ok ? yr : 0.f, ok, a.expo, ye, ye1);
-              p0[u & 3] += ye1;
-              p1[u & 3] = fmaf(ye1, dp[u], p1[u & 3]);
+              for (int u = 0; u < 16; ++u) {
+                const float m = fmaxf(fmaf(ra, sa[u], -tau), 0.f);
+                const float ye1 = clamped_pow_m1<EC>(m);
+                p0[u & 3] += ye1;
+                p1[u & 3] = fmaf(ye1, dp[u], p1[u & 3]);
+              }
+            } else {
+#pragma unroll
+              for (int u = 0; u < 16; ++u) {
+                const float yr = fmaf(ra, sa[u], -tau);
+                const bool ok = yr > 0.f && (!edge || col0 + u <= lim);
+                float ye, ye1;
+                pow_pair_c<EC>(ok ? yr : 0.f, ok, a.expo, ye, ye1);
+                p0[u & 3] += ye1;
+                p1[u & 3] = fmaf(ye1, dp[u], p1[u & 3]);
+              }
             }
             su += (p0[0] + p0[1]) + (p0[2] + p0[3]);
             sud += (p1[0] + p1[1]) + (p1[2] + p1[3]);
@@ -485,17 +524,35 @@ __global__ void __launch_bounds__(kThreadsB, 1) tile_bwd_kernel(const __grid_con
 #pragma unroll
             for (int u4 = 0; u4 < 2; ++u4) {
               float dv[8], dl[8];
+              if (EC != kExpoGeneral && !edge) {
+                // away from the mask (an unmarked row has a = 0, tau = 0 here: every entry clamps to zero)
 #pragma unroll
-              for (int z = 0; z < 8; ++z) {
-                const int u = u4 * 8 + z;
-                const float yr = fmaf(ra, sa[u], -tau);
-                const bool ok = marked && yr > 0.f && (!edge || col0 + u <= lim);
-                float ye, ye1;
-                pow_pair_c<EC>(ok ? yr : 0.f, ok, a.expo, ye, ye1);
-                const float ds = ye1 * (dp[u] - rho);
-                dv[z] = g * ds;
-                dl[z] = dv[z] - __bfloat162float(__float2bfloat16_rn(dv[z]));
-                dcs[z & 1] = fmaf(ds, sa[u], dcs[z & 1]);
+                for (int z = 0; z < 8; ++z) {
+                  const int u = u4 * 8 + z;
+                  const float m = fmaxf(fmaf(ra_m, sa[u], -tau), 0.f);
+                  const float ds = clamped_pow_m1<EC>(m) * (dp[u] - rho);
+                  dv[z] = g * ds;
+                  dcs[z & 1] = fmaf(ds, sa[u], dcs[z & 1]);
+                }
+              } else {
+#pragma unroll
+                for (int z = 0; z < 8; ++z) {
+                  const int u = u4 * 8 + z;
+                  const float yr = fmaf(ra, sa[u], -tau);
+                  const bool ok = marked && yr > 0.f && (!edge || col0 + u <= lim);
+                  float ye, ye1;
+                  pow_pair_c<EC>(ok ? yr : 0.f, ok, a.expo, ye, ye1);
+                  const float ds = ye1 * (dp[u] - rho);
+                  dv[z] = g * ds;
+                  dcs[z & 1] = fmaf(ds, sa[u], dcs[z & 1]);
+                }
+              }
+              // what the bf16 rounding of g dS leaves over, two entries at a time
+#pragma unroll
+              for (int z = 0; z < 8; z += 2) {
+                const float2 r2 = __bfloat1622float2(__floats2bfloat162_rn(dv[z], dv[z + 1]));
+                dl[z] = dv[z] - r2.x;
+                dl[z + 1] = dv[z + 1] - r2.y;
               }
               const uint32_t unit = (uint32_t)((quarter & 1) * 4 + hc * 2 + u4);
               const uint32_t off = blk + ((unit ^ (uint32_t)(row_local & 7)) << 4);
@@ -837,6 +894,7 @@ __global__ void __launch_bounds__(kThreadsB, 1) tile_bwd_kv_kernel(const __grid_
         const float g = c_i * a.sm_scale;
         const float tau = marked ? a.tau[grow] : 0.f;
         const float rho = marked ? a.rho[grow] : 0.f;
+        const float ra_m = marked ? ra : 0.f;
         alive = __all_sync(0xffffffffu, mbar_wait(sd_full, sdphase, abort_flag));
         if (!alive) break;
         sdphase ^= 1u;
@@ -861,15 +919,27 @@ __global__ void __launch_bounds__(kThreadsB, 1) tile_bwd_kv_kernel(const __grid_
 #pragma unroll
           for (int u4 = 0; u4 < 2; ++u4) {
             float pv[8], dv[8];
+            if (EC != kExpoGeneral && !edge) {
+              // away from the mask (an unmarked row has a = 0, tau = 0 here: every entry clamps to zero)
 #pragma unroll
-            for (int z = 0; z < 8; ++z) {
-              const int u = u4 * 8 + z;
-              const float yr = fmaf(ra, sa[u], -tau);
-              const bool ok = marked && yr > 0.f && (!edge || col0 + u <= lim);
-              float ye, ye1;
-              pow_pair_c<EC>(ok ? yr : 0.f, ok, a.expo, ye, ye1);
-              pv[z] = ye;
-              dv[z] = g * (ye1 * (dp[u] - rho));
+              for (int z = 0; z < 8; ++z) {
+                const int u = u4 * 8 + z;
+                const float m = fmaxf(fmaf(ra_m, sa[u], -tau), 0.f);
+                const float ye1 = clamped_pow_m1<EC>(m);
+                pv[z] = ye1 * m;
+                dv[z] = g * (ye1 * (dp[u] - rho));
+              }
+            } else {
+#pragma unroll
+              for (int z = 0; z < 8; ++z) {
+                const int u = u4 * 8 + z;
+                const float yr = fmaf(ra, sa[u], -tau);
+                const bool ok = marked && yr > 0.f && (!edge || col0 + u <= lim);
+                float ye, ye1;
+                pow_pair_c<EC>(ok ? yr : 0.f, ok, a.expo, ye, ye1);
+                pv[z] = ye;
+                dv[z] = g * (ye1 * (dp[u] - rho));
+              }
             }
             const uint32_t unit = (uint32_t)((quarter & 1) * 4 + hc * 2 + u4);
             const uint32_t off = blk + ((unit ^ (uint32_t)(row_local & 7)) << 4);
