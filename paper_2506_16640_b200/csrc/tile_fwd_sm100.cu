@@ -45,9 +45,11 @@ constexpr int kConsGroups = 4;                       // threads per query row
 constexpr int kConsWarps = 4 * kConsGroups;           // four TMEM lane quadrants each
 constexpr int kThreadsT = (2 + kConsWarps) * 32;      // TMA warp, MMA warp, the consumer warps
 constexpr int kMaxSweeps = 48;     // 1 max sweep + at most 46 Newton sweeps + the output sweep
-// Sampled start: long rows first solve Eq. 1's threshold on every kTileSampleStride-th key (sweeps an eighth as long).
-// The threshold of a subset never exceeds that of the whole row, so the full-row Newton iteration may start from it
-// (steps from the left of the root never pass it, e >= 1) instead of from y_max - 1, and needs no y_max sweep.
+// Sampled start: long rows first solve Eq. 1's threshold on every kTileSampleStride-th key (sweeps an eighth as long),
+// each sampled key counted kTileSampleStride times, so that the sample's threshold estimates the row's; the full-row
+// Newton iteration starts from it instead of from y_max - 1 and needs no y_max sweep.  An estimate past the root costs
+// nothing more than one from before it: F = S^(1/e) - 1 is convex and decreasing, so the first Newton step from
+// there lands at or before the root and the iteration goes on from the left (steps from the left never pass it).
 constexpr int kTileSampleStride = 8;
 constexpr int kSampleMinTiles = 16;    // K tiles a Q tile must see for the sampled start to pay
 constexpr int kSampleSweepCap = 12;    // sampled sweeps at most
@@ -745,9 +747,24 @@ __global__ void __launch_bounds__(kThreadsT, 1) tile_fwd_kernel(const __grid_con
           it_tau = tau_iter_start(ymax);
           tau = it_tau.tau;
         } else if (!done) {
-          // e >= 1: Newton from the left (e-norm step); e < 1: bracketed (see tau_iter_update)
-          done = !tau_iter_update(it_tau, s0, s1, a.expo_class, a.expo, 2e-6f);
-          tau = it_tau.tau;
+          if (smp) {
+            // a sampled key stands for kTileSampleStride keys of the row: the sample is solved for that much mass, so
+            // that its threshold estimates the row's instead of only bounding it from below
+            s0 *= (float)kTileSampleStride;
+            s1 *= (float)kTileSampleStride;
+          }
+          if (kind == kFullNewton && n_full == 1 && stiles > 0 && s0 < 0.999f && s1 > 0.f) {
+            // the estimate was past the row's threshold: F = S^(1/e) - 1 is convex and decreasing, so one Newton step
+            // from there lands at or before the root, and the iteration goes on from the left as usual
+            it_tau.tau += threshold_step(s0, s1, a.expo_class, a.expo);
+            tau = it_tau.tau;
+          } else {
+            // e >= 1: Newton from the left (e-norm step); e < 1: bracketed (see tau_iter_update)
+            // (a looser stop -- a step of 1e-4 |tau| -- saves a sweep and keeps O and tau within tolerance, but the
+            // backward pass, whose dQ is what survives the cancellation sum_j dS_ij = 0, needs the threshold to fp32)
+            done = !tau_iter_update(it_tau, s0, s1, a.expo_class, a.expo, 2e-6f);
+            tau = it_tau.tau;
+          }
         }
         const bool warp_done = __all_sync(0xffffffffu, done);
         if (lane == 0) {
