@@ -53,6 +53,10 @@ constexpr int kMaxSweeps = 48;     // 1 max sweep + at most 46 Newton sweeps + t
 constexpr int kTileSampleStride = 8;
 constexpr int kSampleMinTiles = 16;    // K tiles a Q tile must see for the sampled start to pay
 constexpr int kSampleSweepCap = 12;    // sampled sweeps at most
+// Mass sum_j p_ij at the threshold a sweep used, minus 1.  Within kNearMass before a Newton step: the step squares the
+// error, so the next sweep can be an output sweep.  Within kOutputMass in an output sweep: its O is the result (P is
+// rounded to bf16, 2^-9 relative, anyway), and the step its sums give makes the stored threshold exact to fp32.
+constexpr float kNearMass = 5e-2f, kOutputMass = 1e-3f;
 enum SweepKind : int { kSampleMax = 0, kSampleNewton = 1, kFullMax = 2, kFullNewton = 3, kOutput = 4 };
 constexpr int kPBytes = TM * TN * 2;
 
@@ -164,7 +168,7 @@ __global__ void __launch_bounds__(kThreadsT, 1) tile_fwd_kernel(const __grid_con
     mbar_init(o_empty, kConsWarps);
     mbar_init(ctl, kConsWarps);
     mbar_init(x_bar, kConsWarps);
-    for (int t = 0; t < 3; ++t) sts_u32(done_word + 4 * t, 1u);
+    for (int t = 0; t < 3; ++t) sts_u32(done_word + 4 * t, 3u);
     mbar_init(drain_bar, 1);
     for (int t = 0; t < 2; ++t) {
       mbar_init(w_full + 8 * t, 1);
@@ -205,8 +209,14 @@ __global__ void __launch_bounds__(kThreadsT, 1) tile_fwd_kernel(const __grid_con
     if (groups > a.N / kTileSampleStride) groups = a.N / kTileSampleStride;
     return (groups + TN - 1) / TN;
   };
+  // The consumers' vote on sweep s - 1: bit 0 = every row of the tile has its final threshold, bit 1 = every row's mass
+  // was within kNearMass of 1 before its last step.  An output sweep is started as soon as every row is near: it also
+  // takes the Newton sums, and if they show every row's mass within kOutputMass of 1, its O is the result (the stored
+  // threshold takes the last step too); otherwise the iteration goes on and another output sweep follows.
+  auto prev_vote = [&](int s) -> uint32_t { return s >= 1 ? lds_u32(done_word + 4 * ((s - 1) % 3)) : 0u; };
   auto sweep_kind = [&](int s, int& phase, int& n_full) -> int {
-    const bool prev_done = s >= 1 && lds_u32(done_word + 4 * ((s - 1) % 3)) != 0u;
+    const uint32_t vote = prev_vote(s);
+    const bool prev_done = (vote & 1u) != 0u;
     if (phase == 0) {
       if (s == 0) return kSampleMax;
       if ((prev_done && s >= 2) || s >= kSampleSweepCap) {
@@ -217,7 +227,7 @@ __global__ void __launch_bounds__(kThreadsT, 1) tile_fwd_kernel(const __grid_con
       return kSampleNewton;
     }
     if (s == 0) return kFullMax;
-    if (s == kMaxSweeps - 1 || (prev_done && n_full >= 1)) return kOutput;
+    if (s >= kMaxSweeps - 1 || (vote != 0u && n_full >= 1)) return kOutput;
     ++n_full;
     return kFullNewton;
   };
@@ -260,17 +270,21 @@ __global__ void __launch_bounds__(kThreadsT, 1) tile_fwd_kernel(const __grid_con
         }
         __syncwarp();
         qphase ^= 1u;
-        for (int s = 0; s < kMaxSweeps && alive; ++s) {
+        bool was_output = false;
+        for (int s = 0; alive; ++s) {
           if (s > 0) {
             alive = wait_all(ctl, cphase);
             cphase ^= 1u;
             if (!alive) break;
+            // an output sweep whose threshold the vote confirms ends the item
+            if (was_output && __shfl_sync(0xffffffffu, (int)(prev_vote(s) & 1u), 0)) break;
           }
           int kind = sweep_kind(s, phase, n_full);
           kind = __shfl_sync(0xffffffffu, kind, 0);
           phase = __shfl_sync(0xffffffffu, phase, 0);
           n_full = __shfl_sync(0xffffffffu, n_full, 0);
           const bool output = kind == kOutput, smp = kind <= kSampleNewton;
+          was_output = output;
           // the output sweep walks 128-key tiles (K and V of a stage on one barrier); every other sweep walks
           // 256-key tiles, two tile slots to a stage, rows 128.. of a 64-column block right behind rows 0..127
           const int nt = output ? tiles : ((smp ? stiles : tiles) + 1) / 2;
@@ -303,7 +317,6 @@ __global__ void __launch_bounds__(kThreadsT, 1) tile_fwd_kernel(const __grid_con
             __syncwarp();
             if (++stage == ring) stage = 0;
           }
-          if (output) break;
         }
       }
       if (!alive && lane == 0) {
@@ -353,17 +366,20 @@ __global__ void __launch_bounds__(kThreadsT, 1) tile_fwd_kernel(const __grid_con
         alive = wait_all(o_empty, ophase ^ 1u);
         ophase ^= 1u;
         if (!alive) break;
-        for (int s = 0; s < kMaxSweeps && alive; ++s) {
+        bool was_output = false;
+        for (int s = 0; alive; ++s) {
           if (s > 0) {
             alive = wait_all(ctl, cphase);
             cphase ^= 1u;
             if (!alive) break;
+            if (was_output && __shfl_sync(0xffffffffu, (int)(prev_vote(s) & 1u), 0)) break;
           }
           int kind = sweep_kind(s, phase, n_full);
           kind = __shfl_sync(0xffffffffu, kind, 0);
           phase = __shfl_sync(0xffffffffu, phase, 0);
           n_full = __shfl_sync(0xffffffffu, n_full, 0);
           const bool output = kind == kOutput;
+          was_output = output;
           const int nt = output ? tiles : ((kind <= kSampleNewton ? stiles : tiles) + 1) / 2;
           const int ring = C::kStages;   // every sweep starts at stage 0
           int stage = 0;
@@ -447,7 +463,6 @@ __global__ void __launch_bounds__(kThreadsT, 1) tile_fwd_kernel(const __grid_con
               if (++vstage == ring) vstage = 0;
             }
           }
-          if (output) break;
         }
         if (elect_one()) umma_commit(q_empty);
         __syncwarp();
@@ -512,15 +527,57 @@ __global__ void __launch_bounds__(kThreadsT, 1) tile_fwd_kernel(const __grid_con
       const float slope = a.alibi ? a.alibi[h] / a.sm_scale : 0.f;   // bias in accumulator units
       float tau = 0.f, ymax = -INFINITY;
       TauIter it_tau = {0.f, 0.f, 0.f};
-      bool done = !valid;
-      for (int s = 0; s < kMaxSweeps && alive; ++s) {
+      bool done = !valid, was_output = false;
+      int n_supp_out = 0;
+      for (int s = 0; alive; ++s) {
         if (s > 0) {
           alive = __all_sync(0xffffffffu, mbar_wait(ctl, cphase, abort_flag));
           cphase ^= 1u;
           if (!alive) break;
+          if (was_output && (prev_vote(s) & 1u)) {
+            // ---- the vote confirms the thresholds the last output sweep used: its O is the result
+            tc_fence_after();
+            const bool write = valid && a.row_cnt[grow] == -2;
+            __nv_bfloat16* orow =
+                reinterpret_cast<__nv_bfloat16*>(a.o) + (size_t)b * a.sb + (size_t)h * a.sh + (size_t)i * a.sn;
+            for (int c = quarter; c < HD / 32; c += kConsGroups) {
+              float va[32];
+              tmem_ld32(taddr_row + C::kTmemO + c * 32, va);
+              tmem_ld_wait();
+              if (write) {
+#pragma unroll
+                for (int u8 = 0; u8 < 4; ++u8) {
+                  uint32_t w[4];
+#pragma unroll
+                  for (int e2 = 0; e2 < 4; ++e2) {
+                    const __nv_bfloat162 hh = __floats2bfloat162_rn(va[u8 * 8 + e2 * 2], va[u8 * 8 + e2 * 2 + 1]);
+                    w[e2] = *reinterpret_cast<const uint32_t*>(&hh);
+                  }
+                  *reinterpret_cast<uint4*>(orow + c * 32 + u8 * 8) = make_uint4(w[0], w[1], w[2], w[3]);
+                }
+              }
+            }
+            tc_fence_before();
+            __syncwarp();
+            if (lane == 0) mbar_arrive(o_empty);
+            // the row's support size, as two halves (keys of the tile's first / second 64 columns)
+            float n4[4], unused[4];
+            alive = swap4((float)n_supp_out, 0.f, n4, unused);
+            if (!alive) break;
+            if (write && quarter == 0) a.tau[grow] = tau;
+            if (write && (quarter & 1) == 0) a.dense_cnt[grow * 2 + (quarter >> 1)] = (int)(n4[quarter] + n4[quarter + 1]);
+            if (a.status && threadIdx.x == 64) {
+              // diagnostics: full-length sweeps spent (y_max sweep if any, Newton sweeps, output sweep; the sampled
+              // sweeps, an eighth as long, are not counted) and tiles processed
+              atomicAdd(a.status + ENTMAX_ATTN_STATUS_TILE_SWEEPS, s - n_smp);
+              atomicAdd(a.status + ENTMAX_ATTN_STATUS_TILES, 1);
+            }
+            break;
+          }
         }
         const int kind = sweep_kind(s, phase, n_full);
         const bool output = kind == kOutput, smp = kind <= kSampleNewton;
+        was_output = output;
         const bool find_max = kind == kSampleMax || kind == kFullMax;
         // the output sweep walks 128-key tiles (a thread scans 32 columns); every other sweep walks 256-key tiles
         // (two accumulators of 256 columns; a thread scans 64 columns as two chunks)
@@ -529,8 +586,6 @@ __global__ void __launch_bounds__(kThreadsT, 1) tile_fwd_kernel(const __grid_con
         const float slope_c = smp ? slope * (float)kTileSampleStride : slope;
         if (kind == kFullNewton && n_full == 1 && stiles > 0) done = !valid;   // the full-row iteration starts here
         n_smp += smp ? 1 : 0;
-        // the vote slot two sweeps ahead is free again: nobody reads it before the next vote
-        if (warp == 2 && lane == 0) sts_u32(done_word + 4 * ((s + 1) % 3), 1u);
         float s0 = 0.f, s1 = 0.f;
         int n_supp = 0;   // output sweep: keys of this thread's columns with p > 0
         // one 32-column chunk of a maxima or Newton sweep
@@ -633,22 +688,29 @@ __global__ void __launch_bounds__(kThreadsT, 1) tile_fwd_kernel(const __grid_con
               // as in the Newton sweeps: one ALU-pipe clamp per element, the rest on the FMA pipe (the count of
               // positive entries too: an indicator formed by a saturating multiply).  Rows past the end of the
               // sequence have a = 0, tau = 0: all zero.
-              float cnt[4] = {0.f, 0.f, 0.f, 0.f};
+              float cnt[4] = {0.f, 0.f, 0.f, 0.f}, q0[4] = {0.f, 0.f, 0.f, 0.f}, q1[4] = {0.f, 0.f, 0.f, 0.f};
 #pragma unroll
               for (int e2 = 0; e2 < 16; ++e2) {
                 float pv[2];
 #pragma unroll
                 for (int z = 0; z < 2; ++z) {
                   const float m = fmaxf(fmaf(ra, va[e2 * 2 + z], -tau), 0.f);
-                  if constexpr (EC == kExpo2) pv[z] = m * m;
-                  else if constexpr (EC == kExpo4) { const float t2 = m * m; pv[z] = t2 * t2; }
-                  else pv[z] = m;
-                  cnt[(e2 * 2 + z) & 3] += positive_indicator(m);
+                  const float ind = positive_indicator(m);
+                  float ye1;
+                  if constexpr (EC == kExpo2) { ye1 = m; pv[z] = m * m; }
+                  else if constexpr (EC == kExpo4) { const float t2 = m * m; ye1 = t2 * m; pv[z] = t2 * t2; }
+                  else { ye1 = ind; pv[z] = m; }
+                  cnt[(e2 * 2 + z) & 3] += ind;
+                  // the Newton sums at this threshold too: they decide whether this sweep's O is the result
+                  q0[(e2 * 2 + z) & 3] += pv[z];
+                  q1[(e2 * 2 + z) & 3] += ye1;
                 }
                 const __nv_bfloat162 hh = __floats2bfloat162_rn(pv[0], pv[1]);
                 w[e2] = *reinterpret_cast<const uint32_t*>(&hh);
               }
               n_supp += (int)((cnt[0] + cnt[1]) + (cnt[2] + cnt[3]));
+              s0 += (q0[0] + q0[1]) + (q0[2] + q0[3]);
+              s1 += (q1[0] + q1[1]) + (q1[2] + q1[3]);
             } else {
 #pragma unroll
               for (int e2 = 0; e2 < 16; ++e2) {
@@ -661,6 +723,8 @@ __global__ void __launch_bounds__(kThreadsT, 1) tile_fwd_kernel(const __grid_con
                   float ye1;
                   pow_pair_c<EC>(ok ? yr : 0.f, ok, a.expo, pv[z], ye1);
                   n_supp += ok ? 1 : 0;
+                  s0 += pv[z];
+                  s1 += ye1;
                 }
                 const __nv_bfloat162 hh = __floats2bfloat162_rn(pv[0], pv[1]);
                 w[e2] = *reinterpret_cast<const uint32_t*>(&hh);
@@ -688,47 +752,15 @@ __global__ void __launch_bounds__(kThreadsT, 1) tile_fwd_kernel(const __grid_con
           }
         }
         if (!alive) break;
+        // the next sweep's vote slot: its last readers (the roles deciding the kind of sweep s - 1, or the end of the
+        // previous item) are past it once this sweep's tiles have come through
+        if (warp == 2 && lane == 0) sts_u32(done_word + 4 * ((s + 1) % 3), 3u);
         if (output) {
+          // all of this sweep's P V contractions have finished (its O stays in TMEM until the vote is in)
           alive = __all_sync(0xffffffffu, mbar_wait(o_full, ophase, abort_flag));
           ophase ^= 1u;
           if (!alive) break;
-          tc_fence_after();
-          const bool write = valid && a.row_cnt[grow] == -2;
-          __nv_bfloat16* orow =
-              reinterpret_cast<__nv_bfloat16*>(a.o) + (size_t)b * a.sb + (size_t)h * a.sh + (size_t)i * a.sn;
-          for (int c = quarter; c < HD / 32; c += kConsGroups) {
-            float va[32];
-            tmem_ld32(taddr_row + C::kTmemO + c * 32, va);
-            tmem_ld_wait();
-            if (write) {
-#pragma unroll
-              for (int u8 = 0; u8 < 4; ++u8) {
-                uint32_t w[4];
-#pragma unroll
-                for (int e2 = 0; e2 < 4; ++e2) {
-                  const __nv_bfloat162 hh = __floats2bfloat162_rn(va[u8 * 8 + e2 * 2], va[u8 * 8 + e2 * 2 + 1]);
-                  w[e2] = *reinterpret_cast<const uint32_t*>(&hh);
-                }
-                *reinterpret_cast<uint4*>(orow + c * 32 + u8 * 8) = make_uint4(w[0], w[1], w[2], w[3]);
-              }
-            }
-          }
-          tc_fence_before();
-          __syncwarp();
-          if (lane == 0) mbar_arrive(o_empty);
-          // the row's support size, as two halves (keys of the tile's first / second 64 columns)
-          float n4[4], unused[4];
-          alive = swap4((float)n_supp, 0.f, n4, unused);
-          if (!alive) break;
-          if (write && quarter == 0) a.tau[grow] = tau;
-          if (write && (quarter & 1) == 0) a.dense_cnt[grow * 2 + (quarter >> 1)] = (int)(n4[quarter] + n4[quarter + 1]);
-          if (a.status && threadIdx.x == 64) {
-            // diagnostics: full-length sweeps spent (y_max sweep if any, Newton sweeps, output sweep; the sampled
-            // sweeps, an eighth as long, are not counted) and tiles processed
-            atomicAdd(a.status + ENTMAX_ATTN_STATUS_TILE_SWEEPS, s + 1 - n_smp);
-            atomicAdd(a.status + ENTMAX_ATTN_STATUS_TILES, 1);
-          }
-          break;
+          n_supp_out = n_supp;
         }
         // ---- between sweeps: the threads of a row swap their partial results, Newton update, and the vote "every
         //      row of the tile has converged"
@@ -743,6 +775,7 @@ __global__ void __launch_bounds__(kThreadsT, 1) tile_fwd_kernel(const __grid_con
             s1 = (r1[0] + r1[1]) + (r1[2] + r1[3]);
           }
         }
+        const float mass_err = find_max ? 1.0f : fabsf((smp ? (float)kTileSampleStride * s0 : s0) - 1.0f);
         if (find_max) {
           it_tau = tau_iter_start(ymax);
           tau = it_tau.tau;
@@ -765,10 +798,14 @@ __global__ void __launch_bounds__(kThreadsT, 1) tile_fwd_kernel(const __grid_con
             done = !tau_iter_update(it_tau, s0, s1, a.expo_class, a.expo, 2e-6f);
             tau = it_tau.tau;
           }
+          if (output && mass_err <= kOutputMass) done = true;
         }
-        const bool warp_done = __all_sync(0xffffffffu, done);
+        if (output && s >= kMaxSweeps - 1) done = true;   // the cap: this sweep's O is the result
+        const bool near = done || mass_err <= kNearMass;
+        const bool warp_done = __all_sync(0xffffffffu, done), warp_near = __all_sync(0xffffffffu, near);
         if (lane == 0) {
-          if (!warp_done || find_max) atomicAnd(reinterpret_cast<unsigned*>(__cvta_shared_to_generic(done_word + 4 * (s % 3))), 0u);
+          const unsigned keep = find_max ? 0u : (warp_done ? 1u : 0u) | (warp_near ? 2u : 0u);
+          if (keep != 3u) atomicAnd(reinterpret_cast<unsigned*>(__cvta_shared_to_generic(done_word + 4 * (s % 3))), keep);
           mbar_arrive(ctl);
         }
       }
