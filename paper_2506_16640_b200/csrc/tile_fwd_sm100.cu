@@ -53,6 +53,7 @@ constexpr int kMaxSweeps = 48;     // 1 max sweep + at most 46 Newton sweeps + t
 constexpr int kTileSampleStride = 8;
 constexpr int kSampleMinTiles = 16;    // K tiles a Q tile must see for the sampled start to pay
 constexpr int kSampleSweepCap = 12;    // sampled sweeps at most
+constexpr float kSampleTol = 1e-2f;    // the sampled iteration stops at a step of this size, relative to |tau|
 // Mass sum_j p_ij at the threshold a sweep used, minus 1.  Within kNearMass before a Newton step: the step squares the
 // error, so the next sweep can be an output sweep.  Within kOutputMass in an output sweep: its O is the result (P is
 // rounded to bf16, 2^-9 relative, anyway), and the step its sums give makes the stored threshold exact to fp32.
@@ -795,7 +796,9 @@ __global__ void __launch_bounds__(kThreadsT, 1) tile_fwd_kernel(const __grid_con
             // e >= 1: Newton from the left (e-norm step); e < 1: bracketed (see tau_iter_update)
             // (a looser stop -- a step of 1e-4 |tau| -- saves a sweep and keeps O and tau within tolerance, but the
             // backward pass, whose dQ is what survives the cancellation sum_j dS_ij = 0, needs the threshold to fp32)
-            done = !tau_iter_update(it_tau, s0, s1, a.expo_class, a.expo, 2e-6f);
+            // (the sample's threshold is an estimate of the row's, a few per cent off in mass: no point in solving the
+            // sample any finer than that)
+            done = !tau_iter_update(it_tau, s0, s1, a.expo_class, a.expo, smp ? kSampleTol : 2e-6f);
             tau = it_tau.tau;
           }
           if (output && mass_err <= kOutputMass) done = true;
