@@ -145,8 +145,10 @@ __global__ void __launch_bounds__(kThreadsT, 1) tile_fwd_kernel(const __grid_con
   const uint32_t w_full = drain_fail + 8;                             // [2] a work item has been published
   const uint32_t w_empty = w_full + 16;                               // [2] ... and read by the MMA issuer and every consumer warp
   const uint32_t w_item = w_empty + 16;                               // int32 [2]: tile id, -1 = no more work
+  const uint32_t v_full = w_item + 8;                                 // [C::kStages] output sweep: V tiles on barriers
+  const uint32_t v_empty = v_full + 8 * C::kStages;                     // [C::kStages]   of their own (see the producer)
   const uint32_t xchg = bars + C::kBarBytes;                          // float2 [2][kConsGroups][TM]
-  static_assert(8 * (2 + 2 * C::kStages + 4 + 4 + 1) + 16 + 8 + 8 + 16 + 40 <= C::kBarBytes, "barrier area");
+  static_assert(8 * (2 + 4 * C::kStages + 4 + 4 + 1) + 16 + 8 + 8 + 16 + 40 <= C::kBarBytes, "barrier area");
 
   const int warp = threadIdx.x >> 5;
   const int lane = threadIdx.x & 31;
@@ -158,6 +160,8 @@ __global__ void __launch_bounds__(kThreadsT, 1) tile_fwd_kernel(const __grid_con
     for (int t = 0; t < C::kStages; ++t) {
       mbar_init(kv_full + 8 * t, 1);
       mbar_init(kv_empty + 8 * t, 1);
+      mbar_init(v_full + 8 * t, 1);
+      mbar_init(v_empty + 8 * t, 1);
     }
     for (int t = 0; t < 2; ++t) {
       mbar_init(s_full + 8 * t, 1);
@@ -238,7 +242,8 @@ __global__ void __launch_bounds__(kThreadsT, 1) tile_fwd_kernel(const __grid_con
     // (the whole warp runs the control flow, one elected lane issues the copies: see the MMA issuer)
     {
       int slot = 0;
-      uint32_t kvbits = 0 /* bit x: times barrier pair x has been armed, mod 2 */, qphase = 0, cphase = 0, wphase = 0;
+      uint32_t kvbits = 0 /* bit x: times barrier pair x has been armed, mod 2 */, vbits = 0, qphase = 0, cphase = 0,
+               wphase = 0;
       bool alive = true;
       auto wait_all = [&](uint32_t bar, uint32_t parity) -> bool {
         return __all_sync(0xffffffffu, mbar_wait(bar, parity, abort_flag));
@@ -286,32 +291,48 @@ __global__ void __launch_bounds__(kThreadsT, 1) tile_fwd_kernel(const __grid_con
           n_full = __shfl_sync(0xffffffffu, n_full, 0);
           const bool output = kind == kOutput, smp = kind <= kSampleNewton;
           was_output = output;
-          // the output sweep walks 128-key tiles (K and V of a stage on one barrier); every other sweep walks
-          // 256-key tiles, two tile slots to a stage, rows 128.. of a 64-column block right behind rows 0..127
+          // the output sweep walks 128-key tiles; every other sweep walks 256-key tiles, two tile slots to a stage,
+          // rows 128.. of a 64-column block right behind rows 0..127
           const int nt = output ? tiles : ((smp ? stiles : tiles) + 1) / 2;
           const int ring = C::kStages;   // every sweep starts at stage 0
           int stage = 0;
+          if (output) {
+            // K and V tiles on barriers of their own, K one tile ahead of V: a K slot is free as soon as the scores
+            // of the tile before last have been formed, a V slot only after that tile's P V -- on one barrier the
+            // next K tile was asked for a whole contraction late and the issuer waited out the copy on every tile
+            int ks = 0, vs = 0;
+            auto load_kv = [&](const CUtensorMap* map, uint32_t full, uint32_t empty, uint32_t smem, uint32_t& bits,
+                               int& st, int t) -> bool {
+              if (!wait_all(empty + 8 * st, ((bits >> st) & 1u) ^ 1u)) return false;
+              bits ^= 1u << st;
+              if (elect_one()) {
+                mbar_expect_tx(full + 8 * st, C::kKBytes);
+                for (int hf = 0; hf < C::kHalves; ++hf)
+                  tma_load_4d(smem + st * C::kKBytes + hf * (TN * 128), map, full + 8 * st, hf * 64, t * TN, h, b);
+              }
+              __syncwarp();
+              if (++st == ring) st = 0;
+              return true;
+            };
+            alive = load_kv(&map_k, kv_full, kv_empty, k_smem, kvbits, ks, 0);
+            for (int t = 0; t < nt && alive; ++t) {
+              if (t + 1 < nt) alive = load_kv(&map_k, kv_full, kv_empty, k_smem, kvbits, ks, t + 1);
+              if (alive) alive = load_kv(&map_v, v_full, v_empty, v_smem, vbits, vs, t);
+            }
+            continue;
+          }
           for (int t = 0; t < nt && alive; ++t) {
             alive = wait_all(kv_empty + 8 * stage, ((kvbits >> stage) & 1u) ^ 1u);
             if (!alive) break;
             kvbits ^= 1u << stage;
             if (elect_one()) {
               mbar_expect_tx(kv_full + 8 * stage, 2 * C::kKBytes);
-              if (output) {
-                for (int hf = 0; hf < C::kHalves; ++hf) {
-                  tma_load_4d(k_smem + stage * C::kKBytes + hf * (TN * 128), &map_k, kv_full + 8 * stage, hf * 64, t * TN,
-                              h, b);
-                  tma_load_4d(v_smem + stage * C::kKBytes + hf * (TN * 128), &map_v, kv_full + 8 * stage, hf * 64, t * TN,
-                              h, b);
-                }
-              } else {
-                for (int hf = 0; hf < C::kHalves; ++hf) {
+              for (int hf = 0; hf < C::kHalves; ++hf) {
 #pragma unroll
-                  for (int rh = 0; rh < 2; ++rh) {
-                    const uint32_t dst = k_smem + stage * 2 * C::kKBytes + hf * (TW * 128) + rh * (TN * 128);
-                    if (smp) tma_load_5d(dst, &map_ks, kv_full + 8 * stage, hf * 64, 0, t * TW + rh * TN, h, b);
-                    else tma_load_4d(dst, &map_k, kv_full + 8 * stage, hf * 64, t * TW + rh * TN, h, b);
-                  }
+                for (int rh = 0; rh < 2; ++rh) {
+                  const uint32_t dst = k_smem + stage * 2 * C::kKBytes + hf * (TW * 128) + rh * (TN * 128);
+                  if (smp) tma_load_5d(dst, &map_ks, kv_full + 8 * stage, hf * 64, 0, t * TW + rh * TN, h, b);
+                  else tma_load_4d(dst, &map_k, kv_full + 8 * stage, hf * 64, t * TW + rh * TN, h, b);
                 }
               }
             }
@@ -325,6 +346,7 @@ __global__ void __launch_bounds__(kThreadsT, 1) tile_fwd_kernel(const __grid_con
         // memory goes away (the phase armed last has the parity opposite to the arm count's)
         bool ok = mbar_drain(q_full, qphase ^ 1u);
         for (int st = 0; st < C::kStages; ++st) ok &= mbar_drain(kv_full + 8 * st, ((kvbits >> st) & 1u) ^ 1u);
+        for (int st = 0; st < C::kStages; ++st) ok &= mbar_drain(v_full + 8 * st, ((vbits >> st) & 1u) ^ 1u);
         if (!ok) sts_u32(drain_fail, 1u);
       }
     }
@@ -340,8 +362,8 @@ __global__ void __launch_bounds__(kThreadsT, 1) tile_fwd_kernel(const __grid_con
       const uint64_t hi = (uint64_t)kDescHi << 32;
       const uint64_t q_desc = hi | smem_desc_lo(q_smem), k_desc = hi | smem_desc_lo(k_smem);
       const uint64_t p_desc = hi | smem_desc_lo(p_smem), v_desc = hi | v_desc_lo(v_smem);
-      uint32_t kvbits = 0 /* bit x: phase of barrier pair x to wait for */, qphase = 0, cphase = 0, sphase[2] = {0, 0},
-               pphase = 0, ophase = 0;
+      uint32_t kvbits = 0 /* bit x: phase of barrier pair x to wait for */, vbits = 0, qphase = 0, cphase = 0,
+               sphase[2] = {0, 0}, pphase = 0, ophase = 0;
       int sbuf = 0, slot = 0;
       uint32_t wphase = 0;
       bool alive = true;
@@ -404,6 +426,7 @@ __global__ void __launch_bounds__(kThreadsT, 1) tile_fwd_kernel(const __grid_con
                   umma_bf16_desc(d_tmem, q_desc + a_off, b_desc + b_off, id_qk, kk > 0 ? 1u : 0u);
                 }
                 umma_commit(s_full + 8 * sbuf);
+                umma_commit(kv_empty + 8 * stage);   // the K slot is free once these scores are formed
               }
             } else {
               const uint64_t b_desc = k_desc + (uint64_t)(stage * (2 * C::kKBytes >> 4));
@@ -445,7 +468,9 @@ __global__ void __launch_bounds__(kThreadsT, 1) tile_fwd_kernel(const __grid_con
               // O += P V for this tile once the consumers have written P
               alive = wait_all(p_full, pphase);
               pphase ^= 1u;
+              if (alive) alive = wait_all(v_full + 8 * vstage, (vbits >> vstage) & 1u);
               if (!alive) break;
+              vbits ^= 1u << vstage;
               tc_fence_after();
               const uint64_t vb_desc = v_desc + (uint64_t)(vstage * (C::kKBytes >> 4));
               if (elect_one()) {
@@ -457,7 +482,7 @@ __global__ void __launch_bounds__(kThreadsT, 1) tile_fwd_kernel(const __grid_con
                                  (t > 0 || kk > 0) ? 1u : 0u);
                 }
                 umma_commit(p_empty);
-                umma_commit(kv_empty + 8 * vstage);
+                umma_commit(v_empty + 8 * vstage);
                 if (t == nt - 1) umma_commit(o_full);
               }
               __syncwarp();
