@@ -43,7 +43,8 @@ constexpr int TN = 128;            // keys per K/V tile of the output sweep
 constexpr int TW = 2 * TN;         // keys per K tile of every other sweep (two tile slots, one MMA group of N = 256)
 constexpr int kConsGroups = 4;                       // threads per query row
 constexpr int kConsWarps = 4 * kConsGroups;           // four TMEM lane quadrants each
-constexpr int kThreadsT = (2 + kConsWarps) * 32;      // TMA warp, MMA warp, the consumer warps
+constexpr int kThreadsT = (3 + kConsWarps) * 32;      // TMA warp, score MMA warp, the consumer warps, P V MMA warp
+constexpr int kPvWarp = 2 + kConsWarps;
 constexpr int kMaxSweeps = 48;     // 1 max sweep + at most 46 Newton sweeps + the output sweep
 // Sampled start: long rows first solve Eq. 1's threshold on every kTileSampleStride-th key (sweeps an eighth as long),
 // each sampled key counted kTileSampleStride times, so that the sample's threshold estimates the row's; the full-row
@@ -147,8 +148,9 @@ __global__ void __launch_bounds__(kThreadsT, 1) tile_fwd_kernel(const __grid_con
   const uint32_t w_item = w_empty + 16;                               // int32 [2]: tile id, -1 = no more work
   const uint32_t v_full = w_item + 8;                                 // [C::kStages] output sweep: V tiles on barriers
   const uint32_t v_empty = v_full + 8 * C::kStages;                     // [C::kStages]   of their own (see the producer)
+  const uint32_t drain_bar_pv = v_empty + 8 * C::kStages;               // teardown, the P V issuer's contractions
   const uint32_t xchg = bars + C::kBarBytes;                          // float2 [2][kConsGroups][TM]
-  static_assert(8 * (2 + 4 * C::kStages + 4 + 4 + 1) + 16 + 8 + 8 + 16 + 40 <= C::kBarBytes, "barrier area");
+  static_assert(8 * (2 + 4 * C::kStages + 4 + 4 + 1) + 16 + 8 + 8 + 16 + 40 + 8 <= C::kBarBytes, "barrier area");
 
   const int warp = threadIdx.x >> 5;
   const int lane = threadIdx.x & 31;
@@ -171,13 +173,14 @@ __global__ void __launch_bounds__(kThreadsT, 1) tile_fwd_kernel(const __grid_con
     mbar_init(p_empty, 1);
     mbar_init(o_full, 1);
     mbar_init(o_empty, kConsWarps);
-    mbar_init(ctl, kConsWarps);
+    mbar_init(ctl, kConsWarps + 1);                     // the consumer warps' votes and the P V issuer keeping in step
     mbar_init(x_bar, kConsWarps);
     for (int t = 0; t < 3; ++t) sts_u32(done_word + 4 * t, 3u);
     mbar_init(drain_bar, 1);
+    mbar_init(drain_bar_pv, 1);
     for (int t = 0; t < 2; ++t) {
       mbar_init(w_full + 8 * t, 1);
-      mbar_init(w_empty + 8 * t, 1 + kConsWarps);   // MMA issuer + the consumer warps
+      mbar_init(w_empty + 8 * t, 2 + kConsWarps);   // the two MMA issuers + the consumer warps
     }
     sts_u32(drain_fail, 0u);
     sts_u32(abort_flag, 0u);
@@ -351,19 +354,17 @@ __global__ void __launch_bounds__(kThreadsT, 1) tile_fwd_kernel(const __grid_con
       }
     }
   } else if (warp == 1) {
-    // ------------------------------------------------------------------ MMA issuer
+    // ------------------------------------------------------------------ MMA issuer (scores)
     // The whole warp runs this role's control flow (waits are voted on, values read from shared memory are
     // broadcast), so that descriptors, addresses and counters are warp-uniform; one elected lane issues the tensor
     // core instructions.  A single lane inside a divergent branch would compete for issue slots with the consumer
     // warps of its scheduler for every address calculation of every MMA.
     {
       constexpr uint32_t id_qk = idesc_qk(TN), id_qk_wide = idesc_qk(TW);
-      constexpr uint32_t id_pv = idesc_pv<HD>();
       const uint64_t hi = (uint64_t)kDescHi << 32;
       const uint64_t q_desc = hi | smem_desc_lo(q_smem), k_desc = hi | smem_desc_lo(k_smem);
-      const uint64_t p_desc = hi | smem_desc_lo(p_smem), v_desc = hi | v_desc_lo(v_smem);
-      uint32_t kvbits = 0 /* bit x: phase of barrier pair x to wait for */, vbits = 0, qphase = 0, cphase = 0,
-               sphase[2] = {0, 0}, pphase = 0, ophase = 0;
+      uint32_t kvbits = 0 /* bit x: phase of barrier pair x to wait for */, qphase = 0, cphase = 0, sphase[2] = {0, 0},
+               ophase = 0;
       int sbuf = 0, slot = 0;
       uint32_t wphase = 0;
       bool alive = true;
@@ -454,18 +455,68 @@ __global__ void __launch_bounds__(kThreadsT, 1) tile_fwd_kernel(const __grid_con
               if (++stage == ring) stage = 0;
             }
           } else {
-            // output sweep: the scores of tile t + 1 are issued before P of tile t is waited for, so that the
-            // consumers never wait for a contraction that could have run while they formed P
-            int vstage = stage;   // stage that holds the V tile of the next P V
-            alive = issue_qk();
-            if (alive && ++stage == ring) stage = 0;
+            // output sweep: the scores run ahead of the consumers as far as the two accumulators allow; O += P V is
+            // issued by a warp of its own, so that neither stream of contractions waits for the other's barriers and
+            // each issuer's instruction count per tile is halved (the issuers compete for issue slots with the
+            // consumer warps of their schedulers: a tile's sixteen MMAs from one warp took ~2200 cycles)
             for (int t = 0; t < nt && alive; ++t) {
-              if (t + 1 < nt) {
-                alive = issue_qk();
-                if (!alive) break;
-                if (++stage == ring) stage = 0;
-              }
-              // O += P V for this tile once the consumers have written P
+              alive = issue_qk();
+              if (!alive) break;
+              if (++stage == ring) stage = 0;
+            }
+          }
+        }
+        if (elect_one()) umma_commit(q_empty);
+        __syncwarp();
+      }
+      if (!alive && lane == 0) {
+        // the tensor core must be done with shared memory and TMEM before they are released
+        umma_commit(drain_bar);
+        if (!mbar_drain(drain_bar, 0u)) sts_u32(drain_fail, 1u);
+      }
+    }
+  } else if (warp == kPvWarp) {
+    // ------------------------------------------------------------------ P V issuer (output sweeps only)
+    // Follows the sweeps of every item like the other roles (warp-wide control flow, one elected lane issuing) and
+    // arrives on the control barrier once per sweep, so that it can never fall a whole sweep behind the consumers.
+    {
+      constexpr uint32_t id_pv = idesc_pv<HD>();
+      const uint64_t hi = (uint64_t)kDescHi << 32;
+      const uint64_t p_desc = hi | smem_desc_lo(p_smem), v_desc = hi | v_desc_lo(v_smem);
+      uint32_t vbits = 0 /* bit x: phase of V barrier pair x to wait for */, cphase = 0, pphase = 0, wphase = 0;
+      int slot = 0;
+      bool alive = true;
+      auto wait_all = [&](uint32_t bar, uint32_t parity) -> bool {
+        return __all_sync(0xffffffffu, mbar_wait(bar, parity, abort_flag));
+      };
+      while (alive) {
+        alive = wait_all(w_full + 8 * slot, wphase);
+        if (!alive) break;
+        const int id = __shfl_sync(0xffffffffu, (int)lds_u32(w_item + 4 * slot), 0);
+        __syncwarp();
+        if (lane == 0) mbar_arrive(w_empty + 8 * slot);
+        if (++slot == 2) { slot = 0; wphase ^= 1u; }
+        if (id < 0) break;
+        const int tile = id % a.tiles_per_head;
+        const int tiles = item_tiles(tile), stiles = item_sample_tiles(tile);
+        int phase = stiles > 0 ? 0 : 1, n_full = 0;
+        bool was_output = false;
+        for (int s = 0; alive; ++s) {
+          if (s > 0) {
+            alive = wait_all(ctl, cphase);
+            cphase ^= 1u;
+            if (!alive) break;
+            if (was_output && __shfl_sync(0xffffffffu, (int)(prev_vote(s) & 1u), 0)) break;
+          }
+          int kind = sweep_kind(s, phase, n_full);
+          kind = __shfl_sync(0xffffffffu, kind, 0);
+          phase = __shfl_sync(0xffffffffu, phase, 0);
+          n_full = __shfl_sync(0xffffffffu, n_full, 0);
+          was_output = kind == kOutput;
+          if (was_output) {
+            int vstage = 0;   // every sweep starts at stage 0
+            for (int t = 0; t < tiles && alive; ++t) {
+              // O += P V for this tile once the consumers have written P and the V tile has landed
               alive = wait_all(p_full, pphase);
               pphase ^= 1u;
               if (alive) alive = wait_all(v_full + 8 * vstage, (vbits >> vstage) & 1u);
@@ -483,20 +534,21 @@ __global__ void __launch_bounds__(kThreadsT, 1) tile_fwd_kernel(const __grid_con
                 }
                 umma_commit(p_empty);
                 umma_commit(v_empty + 8 * vstage);
-                if (t == nt - 1) umma_commit(o_full);
+                if (t == tiles - 1) umma_commit(o_full);
               }
               __syncwarp();
-              if (++vstage == ring) vstage = 0;
+              if (++vstage == C::kStages) vstage = 0;
             }
+            if (!alive) break;
           }
+          __syncwarp();
+          if (lane == 0) mbar_arrive(ctl);
         }
-        if (elect_one()) umma_commit(q_empty);
-        __syncwarp();
       }
       if (!alive && lane == 0) {
-        // the tensor core must be done with shared memory and TMEM before they are released
-        umma_commit(drain_bar);
-        if (!mbar_drain(drain_bar, 0u)) sts_u32(drain_fail, 1u);
+        // this warp's contractions must be done with shared memory and TMEM before they are released
+        umma_commit(drain_bar_pv);
+        if (!mbar_drain(drain_bar_pv, 0u)) sts_u32(drain_fail, 1u);
       }
     }
   } else {
