@@ -141,7 +141,7 @@ __global__ void __launch_bounds__(kThreadsB, 1) tile_bwd_kernel(const __grid_con
   const uint32_t do_smem = q_smem + C::kQBytes;
   const uint32_t k_smem = do_smem + C::kQBytes;
   const uint32_t v_smem = k_smem + C::kQBytes;
-  const uint32_t p_smem = v_smem + C::kQBytes;           // (the key-major kernel's P tile; not used here)
+  const uint32_t p_smem = v_smem + C::kQBytes;           // (the key-major kernel's P tile; here: second K stage)
   const uint32_t ds_smem = p_smem + kTileBytes;           // g dS tile (bf16), same layout
   const uint32_t dl_smem = ds_smem + kTileBytes;          // what the bf16 rounding of g dS left over, same layout
   const uint32_t bars = dl_smem + kTileBytes;
@@ -259,7 +259,10 @@ __global__ void __launch_bounds__(kThreadsB, 1) tile_bwd_kernel(const __grid_con
         __syncwarp();
         for (int t = 0; t < 2 * tiles && alive; ++t) {
           const int kt = t < tiles ? t : t - tiles;
-          const int st = t < tiles ? (t & 1) : 0;   // pass A alternates between the two stages, pass B has one
+          // K alternates between its two stages in both passes (the second one is a tile this kernel has no other use
+          // for); V does so in pass A only: its second stage is the dS tile of pass B, where a V tile is free again as
+          // soon as dP has been formed
+          const int st = t < tiles ? (t & 1) : 0, kst = t & 1;
           alive = wait_all(v_empty(st), ((vbits >> st) & 1u) ^ 1u);
           if (!alive) break;
           vbits ^= 1u << st;
@@ -269,13 +272,13 @@ __global__ void __launch_bounds__(kThreadsB, 1) tile_bwd_kernel(const __grid_con
               tma_load_4d(v_stage(st) + hf * (TN * 128), &map_v, v_full(st), hf * 64, kt * TN, h, b);
           }
           __syncwarp();
-          alive = wait_all(k_empty(st), ((kbits >> st) & 1u) ^ 1u);
+          alive = wait_all(k_empty(kst), ((kbits >> kst) & 1u) ^ 1u);
           if (!alive) break;
-          kbits ^= 1u << st;
+          kbits ^= 1u << kst;
           if (elect_one()) {
-            mbar_expect_tx(k_full(st), C::kQBytes);
+            mbar_expect_tx(k_full(kst), C::kQBytes);
             for (int hf = 0; hf < C::kHalves; ++hf)
-              tma_load_4d(k_stage(st) + hf * (TN * 128), &map_k, k_full(st), hf * 64, kt * TN, h, b);
+              tma_load_4d(k_stage(kst) + hf * (TN * 128), &map_k, k_full(kst), hf * 64, kt * TN, h, b);
           }
           __syncwarp();
         }
@@ -303,7 +306,7 @@ __global__ void __launch_bounds__(kThreadsB, 1) tile_bwd_kernel(const __grid_con
       const uint64_t q_d = hi | smem_desc_lo(q_smem), do_d = hi | smem_desc_lo(do_smem);
       const uint64_t k_d = hi | smem_desc_lo(k_smem), v_d = hi | smem_desc_lo(v_smem);
       const uint64_t ds_d = hi | smem_desc_lo(ds_smem), dl_d = hi | smem_desc_lo(dl_smem);
-      const uint64_t k_n_d = hi | mn_desc_lo(k_smem);
+      const uint64_t k_n_d = hi | mn_desc_lo(k_smem), k1_n_d = hi | mn_desc_lo(p_smem);
       uint32_t kbits = 0, vbits = 0 /* bit st: phase of the stage's barrier to wait for */, qphase = 0, sdphase = 0,
                pdsphase = 0, dqphase = 0, wphase = 0;
       const uint64_t k1_d = hi | smem_desc_lo(p_smem), v1_d = hi | smem_desc_lo(ds_smem);   // stage 1 of pass A
@@ -325,22 +328,17 @@ __global__ void __launch_bounds__(kThreadsB, 1) tile_bwd_kernel(const __grid_con
         alive = wait_all(qdo_full, qphase);
         qphase ^= 1u;
         if (!alive) break;
-        for (int t = 0; t < 2 * tiles && alive; ++t) {
+        // S = Q K^T and dP = dO V^T of tile t (pass A: t < tiles, pass B: the same tiles again)
+        auto issue_sd = [&](int t) -> bool {
           const bool pass_b = t >= tiles;
-          if (t == tiles) {
-            // the previous item's dQ must have been read before this item's first dQ MMA overwrites it
-            alive = wait_all(dq_empty, dqphase ^ 1u);
-            dqphase ^= 1u;
-            if (!alive) break;
-          }
-          const int st = pass_b ? 0 : (t & 1);
-          alive = wait_all(k_full(st), (kbits >> st) & 1u);
-          kbits ^= 1u << st;
-          if (alive) alive = wait_all(v_full(st), (vbits >> st) & 1u);
+          const int st = pass_b ? 0 : (t & 1), kst = t & 1;
+          bool ok = wait_all(k_full(kst), (kbits >> kst) & 1u);
+          kbits ^= 1u << kst;
+          if (ok) ok = wait_all(v_full(st), (vbits >> st) & 1u);
           vbits ^= 1u << st;
-          const uint64_t ks_d = st ? k1_d : k_d, vs_d = st ? v1_d : v_d;
-          if (alive) alive = wait_all(sd_empty, sdphase ^ 1u);
-          if (!alive) break;
+          const uint64_t ks_d = kst ? k1_d : k_d, vs_d = st ? v1_d : v_d;
+          if (ok) ok = wait_all(sd_empty, sdphase ^ 1u);
+          if (!ok) return false;
           sdphase ^= 1u;
           tc_fence_after();
           if (elect_one()) {
@@ -356,11 +354,28 @@ __global__ void __launch_bounds__(kThreadsB, 1) tile_bwd_kernel(const __grid_con
             }
             umma_commit(sd_full);
             umma_commit(v_empty(st));          // dP has been formed: the V tile is free
-            if (!pass_b) umma_commit(k_empty(st));
+            if (!pass_b) umma_commit(k_empty(kst));
           }
           __syncwarp();
-          if (!pass_b) continue;
-          // P and g dS of this tile are in shared memory
+          return true;
+        };
+        for (int t = 0; t < tiles && alive; ++t) alive = issue_sd(t);
+        if (alive) {
+          // the previous item's dQ must have been read before this item's first dQ MMA overwrites it
+          alive = wait_all(dq_empty, dqphase ^ 1u);
+          dqphase ^= 1u;
+        }
+        if (alive) alive = issue_sd(tiles);
+        for (int t = tiles; t < 2 * tiles && alive; ++t) {
+          // the next tile's S and dP are issued before this tile's dS is waited for (its K tile sits in the other
+          // stage), so that they run while the consumers form dS
+          if (t + 1 < 2 * tiles) {
+            alive = issue_sd(t + 1);
+            if (!alive) break;
+          }
+          const int kst = t & 1;
+          const uint64_t kn_d = kst ? k1_n_d : k_n_d;
+          // g dS of this tile and its rounding remainder are in shared memory
           alive = wait_all(pds_full, pdsphase);
           pdsphase ^= 1u;
           if (!alive) break;
@@ -370,7 +385,7 @@ __global__ void __launch_bounds__(kThreadsB, 1) tile_bwd_kernel(const __grid_con
             for (int kk = 0; kk < TN / 16; ++kk) {
               const uint32_t a_off = (kk >> 2) * ((TM * 128) >> 4) + (kk & 3) * 2;   // 64 keys per 128-byte row
               const uint32_t b_off = kk * ((16 * 128) >> 4);                           // 16 keys = 16 rows of 128 B
-              umma_bf16_desc(tmem_base + C::kTmemDQ, ds_d + a_off, k_n_d + b_off, id_kn, (t > tiles || kk > 0) ? 1u : 0u);
+              umma_bf16_desc(tmem_base + C::kTmemDQ, ds_d + a_off, kn_d + b_off, id_kn, (t > tiles || kk > 0) ? 1u : 0u);
             }
             // the rounding remainder of g dS as a second operand: the rows of dS sum to zero, so when a row's keys
             // are nearly equal vectors (retrieval: several copies of one key) dQ is what is left after a
@@ -379,9 +394,9 @@ __global__ void __launch_bounds__(kThreadsB, 1) tile_bwd_kernel(const __grid_con
             for (int kk = 0; kk < TN / 16; ++kk) {
               const uint32_t a_off = (kk >> 2) * ((TM * 128) >> 4) + (kk & 3) * 2;
               const uint32_t b_off = kk * ((16 * 128) >> 4);
-              umma_bf16_desc(tmem_base + C::kTmemDQ, dl_d + a_off, k_n_d + b_off, id_kn, 1u);
+              umma_bf16_desc(tmem_base + C::kTmemDQ, dl_d + a_off, kn_d + b_off, id_kn, 1u);
             }
-            umma_commit(k_empty(0));           // dQ has taken the K tile
+            umma_commit(k_empty(kst));         // dQ has taken the K tile
             umma_commit(pds_empty);
             if (t == 2 * tiles - 1) umma_commit(dq_full);
           }
@@ -473,12 +488,6 @@ __global__ void __launch_bounds__(kThreadsB, 1) tile_bwd_kernel(const __grid_con
         if (!alive) break;
         sdphase ^= 1u;
         tc_fence_after();
-        if (pass_b) {
-          // P and dS of the previous tile must have been consumed before their buffers are rewritten
-          alive = __all_sync(0xffffffffu, mbar_wait(pds_empty, pdsphase ^ 1u, abort_flag));
-          pdsphase ^= 1u;
-          if (!alive) break;
-        }
         // this thread's 32 columns, 16 at a time
 #pragma unroll 1
         for (int hc = 0; hc < 2; ++hc) {
@@ -554,6 +563,14 @@ __global__ void __launch_bounds__(kThreadsB, 1) tile_bwd_kernel(const __grid_con
                 dl[z] = dv[z] - r2.x;
                 dl[z + 1] = dv[z + 1] - r2.y;
               }
+              if (hc == 0 && u4 == 0) {
+                // g dS of the previous tile and its remainder must have been consumed before their buffers are
+                // rewritten (waited for here, not before the loads: that tile's dQ contraction runs under this
+                // tile's first element code)
+                alive = __all_sync(0xffffffffu, mbar_wait(pds_empty, pdsphase ^ 1u, abort_flag));
+                pdsphase ^= 1u;
+              }
+              if (!alive) continue;
               const uint32_t unit = (uint32_t)((quarter & 1) * 4 + hc * 2 + u4);
               const uint32_t off = blk + ((unit ^ (uint32_t)(row_local & 7)) << 4);
               asm volatile("st.shared::cta.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(ds_smem + off),
@@ -567,6 +584,7 @@ __global__ void __launch_bounds__(kThreadsB, 1) tile_bwd_kernel(const __grid_con
             }
           }
         }
+        if (!alive) break;
         // S and dP have been read
         tc_fence_before();
         __syncwarp();
